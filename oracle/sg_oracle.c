@@ -1,0 +1,355 @@
+/*
+ * sg_oracle.c -- CPU oracle for the fused dense contraction
+ *
+ *     D = act(alpha * A.B + beta * C + bias)
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.  It exists so that the CUDA
+ * library can be compared element by element with a plain, slow, obviously
+ * correct definition.  Only the tests, the smoke check and the benchmark's
+ * cpu-baseline / reference arm may load it.  It shares no code, header, table or
+ * helper with the CUDA path and is never tuned for speed.
+ *
+ * Everything is evaluated in fp64.  bf16 inputs are widened exactly; a product
+ * of two bf16 values (8-bit significands) is exact in fp64, so the only error
+ * is the summation's (<= K * 2^-53 relative to sum |a||b|).
+ *
+ * What each function follows in the paper (arXiv 2603.29010):
+ *   gemm / batched / grouped  -- the DSL operations gemm(), batched_gemm(),
+ *       grouped_gemm(expert_count=E) with .with_dtype(input, acc, output),
+ *       .with_layout(A, B, C) and .with_scaling(alpha, beta)  (Appendix A.1,
+ *       grammar: OPERATIONS and CONFIGURATION); "each output element is a dot
+ *       product" (Appendix A.2, section 1 of the SOL report).
+ *   conv2d_fprop -- conv2d_fprop(kernel_h, kernel_w) on TensorNHWC input /
+ *       filter / output (Appendix A.1; Table 1a "Conv2d ... NHWC").
+ *   epilogue -- the `>>` chain bias(), relu(), gelu(), silu() compiled into one
+ *       fused epilogue (Section 3, "Epilogue fusion"; Table 1c).
+ *   sol -- the four-step Speed-of-Light analysis of Section 4.1 and its worked
+ *       report in Appendix A.2.
+ *
+ * Readings taken where the paper is silent (listed in full in the design notes):
+ *   bias is added after alpha/beta scaling and is not scaled by alpha; it holds
+ *   one value per output column (GEMM) / output channel (conv); gelu is the tanh
+ *   form; conv is cross-correlation with zero padding; the conv FLOP count
+ *   includes the taps that fall in the padding halo; the result is NOT rounded
+ *   to the output type here (the comparison tolerance absorbs that rounding).
+ *
+ * Build: gcc -O2 -fopenmp -shared -fPIC sg_oracle.c -o libsg_oracle.so -lm
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORC_ROW_MAJOR = 0, ORC_COL_MAJOR = 1 };
+enum { ORC_BF16 = 0, ORC_F32 = 1 };
+enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4 };
+
+/* Number of host threads the parallel loops use. */
+int orc_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* bf16 -> fp64, exact: a bf16 is the upper half of an IEEE binary32. */
+static double bf16_to_f64(uint16_t bits) {
+    uint32_t u = (uint32_t)bits << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+static double load_as_f64(const void* p, int dtype, int64_t idx) {
+    if (dtype == ORC_BF16) return bf16_to_f64(((const uint16_t*)p)[idx]);
+    return (double)((const float*)p)[idx];
+}
+
+/*
+ * Activations of the fused epilogue (Table 1c built-ins relu, gelu, silu).
+ * BIAS and NONE are the identity: the bias itself is added by the caller.
+ */
+double orc_act(int epi, double x) {
+    switch (epi) {
+        case ORC_EPI_RELU:
+            return x > 0.0 ? x : 0.0;
+        case ORC_EPI_GELU: {
+            const double c = 0.79788456080286535588; /* sqrt(2/pi) */
+            return 0.5 * x * (1.0 + tanh(c * (x + 0.044715 * x * x * x)));
+        }
+        case ORC_EPI_SILU:
+            return x / (1.0 + exp(-x));
+        default:
+            return x;
+    }
+}
+
+/* -------------------------------------------------------------------------------------------
+ * GEMM.   a(i,k) = A[i*lda + k] (row-major) or A[k*lda + i] (column-major)
+ *         b(k,j) = B[k*ldb + j] (row-major) or B[j*ldb + k] (column-major)
+ *         C and the result are row-major.
+ * ----------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t M, N, K;
+    int layout_a, layout_b;
+    const uint16_t* A; int64_t lda;
+    const uint16_t* B; int64_t ldb;
+    const void* C; int c_dtype; int64_t ldc;     /* read only when beta != 0 */
+    const uint16_t* bias;                        /* [N] or NULL */
+    double alpha, beta;
+    int epi;
+} gemm_problem;
+
+/* One output element and, optionally, the magnitude sum used to scale fp32 tolerances. */
+static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* absacc) {
+    double sum = 0.0, asum = 0.0;
+    for (int64_t k = 0; k < g->K; ++k) {
+        double a = bf16_to_f64(g->layout_a == ORC_ROW_MAJOR ? g->A[i * g->lda + k] : g->A[k * g->lda + i]);
+        double b = bf16_to_f64(g->layout_b == ORC_ROW_MAJOR ? g->B[k * g->ldb + j] : g->B[j * g->ldb + k]);
+        sum += a * b;
+        asum += fabs(a * b);
+    }
+    double v = g->alpha * sum;
+    double av = fabs(g->alpha) * asum;
+    if (g->beta != 0.0) {                       /* beta == 0: C is never read */
+        double c = load_as_f64(g->C, g->c_dtype, i * g->ldc + j);
+        v += g->beta * c;
+        av += fabs(g->beta * c);
+    }
+    if (g->bias) {
+        double bj = bf16_to_f64(g->bias[j]);
+        v += bj;
+        av += fabs(bj);
+    }
+    if (absacc) *absacc = av;
+    return orc_act(g->epi, v);
+}
+
+/*
+ * Rows [row_begin, row_end) of the result.  ref (and absacc, if not NULL) hold
+ * (row_end-row_begin) x N values, row stride ldr, row 0 = row_begin.
+ */
+int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
+             const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+             const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
+             double alpha, double beta, int epi,
+             int64_t row_begin, int64_t row_end, double* ref, double* absacc, int64_t ldr) {
+    if (M < 0 || N < 0 || K < 0 || row_begin < 0 || row_end > M || row_begin > row_end) return 1;
+    if (beta != 0.0 && !C) return 2;
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi};
+#pragma omp parallel for schedule(static)
+    for (int64_t i = row_begin; i < row_end; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            double av;
+            double v = gemm_element(&g, i, j, &av);
+            ref[(i - row_begin) * ldr + j] = v;
+            if (absacc) absacc[(i - row_begin) * ldr + j] = av;
+        }
+    }
+    return 0;
+}
+
+/* The listed elements (pi[t], pj[t]) only: used to spot-check full-size problems. */
+int orc_gemm_points(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
+                    const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
+                    const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
+                    double alpha, double beta, int epi,
+                    int64_t npts, const int64_t* pi, const int64_t* pj, double* ref, double* absacc) {
+    if (beta != 0.0 && !C) return 2;
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi};
+    for (int64_t t = 0; t < npts; ++t)
+        if (pi[t] < 0 || pi[t] >= M || pj[t] < 0 || pj[t] >= N) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < npts; ++t) {
+        double av;
+        ref[t] = gemm_element(&g, pi[t], pj[t], &av);
+        if (absacc) absacc[t] = av;
+    }
+    return 0;
+}
+
+/* -------------------------------------------------------------------------------------------
+ * conv2d forward (cross-correlation), X in NHWC, filter in KRSC, output in NPQK:
+ *   P = floor((H + 2 pad_h - dil_h (R-1) - 1) / stride_h) + 1, Q likewise,
+ *   y[n,p,q,k] = act( alpha * sum_{r,s,c} X[n, p stride_h - pad_h + r dil_h,
+ *                                            q stride_w - pad_w + s dil_w, c] * Wf[k,r,s,c]
+ *                     + beta * Cin[n,p,q,k] + bias[k] ),  taps outside the image contribute 0.
+ * ----------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t N, H, W, C, K, R, S;
+    int64_t pad_h, pad_w, stride_h, stride_w, dil_h, dil_w;
+    int64_t P, Q;
+    const uint16_t* X; const uint16_t* Wf;
+    const void* Cin; int c_dtype;
+    const uint16_t* bias;
+    double alpha, beta;
+    int epi;
+} conv_problem;
+
+int64_t orc_conv_out_extent(int64_t in, int64_t pad, int64_t dil, int64_t filt, int64_t stride) {
+    int64_t span = in + 2 * pad - dil * (filt - 1) - 1;
+    if (span < 0) return 0;
+    return span / stride + 1;
+}
+
+static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t q, int64_t k, double* absacc) {
+    double sum = 0.0, asum = 0.0;
+    for (int64_t r = 0; r < cv->R; ++r) {
+        int64_t h = p * cv->stride_h - cv->pad_h + r * cv->dil_h;
+        if (h < 0 || h >= cv->H) continue;
+        for (int64_t s = 0; s < cv->S; ++s) {
+            int64_t w = q * cv->stride_w - cv->pad_w + s * cv->dil_w;
+            if (w < 0 || w >= cv->W) continue;
+            const uint16_t* xp = cv->X + ((n * cv->H + h) * cv->W + w) * cv->C;
+            const uint16_t* wp = cv->Wf + ((k * cv->R + r) * cv->S + s) * cv->C;
+            for (int64_t c = 0; c < cv->C; ++c) {
+                double t = bf16_to_f64(xp[c]) * bf16_to_f64(wp[c]);
+                sum += t;
+                asum += fabs(t);
+            }
+        }
+    }
+    double v = cv->alpha * sum;
+    double av = fabs(cv->alpha) * asum;
+    if (cv->beta != 0.0) {
+        double c = load_as_f64(cv->Cin, cv->c_dtype, ((n * cv->P + p) * cv->Q + q) * cv->K + k);
+        v += cv->beta * c;
+        av += fabs(cv->beta * c);
+    }
+    if (cv->bias) {
+        double bk = bf16_to_f64(cv->bias[k]);
+        v += bk;
+        av += fabs(bk);
+    }
+    if (absacc) *absacc = av;
+    return orc_act(cv->epi, v);
+}
+
+static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, const uint16_t* Wf,
+                      const void* Cin, int c_dtype, const uint16_t* bias, double alpha, double beta, int epi) {
+    cv->N = d[0]; cv->H = d[1]; cv->W = d[2]; cv->C = d[3]; cv->K = d[4]; cv->R = d[5]; cv->S = d[6];
+    cv->pad_h = d[7]; cv->pad_w = d[8]; cv->stride_h = d[9]; cv->stride_w = d[10];
+    cv->dil_h = d[11]; cv->dil_w = d[12];
+    if (cv->N < 0 || cv->H < 0 || cv->W < 0 || cv->C < 0 || cv->K < 0 || cv->R < 1 || cv->S < 1) return 1;
+    if (cv->stride_h < 1 || cv->stride_w < 1 || cv->dil_h < 1 || cv->dil_w < 1 || cv->pad_h < 0 || cv->pad_w < 0) return 1;
+    if (beta != 0.0 && !Cin) return 2;
+    cv->P = orc_conv_out_extent(cv->H, cv->pad_h, cv->dil_h, cv->R, cv->stride_h);
+    cv->Q = orc_conv_out_extent(cv->W, cv->pad_w, cv->dil_w, cv->S, cv->stride_w);
+    cv->X = X; cv->Wf = Wf; cv->Cin = Cin; cv->c_dtype = c_dtype; cv->bias = bias;
+    cv->alpha = alpha; cv->beta = beta; cv->epi = epi;
+    return 0;
+}
+
+/*
+ * dims = {N,H,W,C,K,R,S,pad_h,pad_w,stride_h,stride_w,dil_h,dil_w}.
+ * Output pixels [pix_begin, pix_end) in flattened (n,p,q) order; ref holds
+ * (pix_end-pix_begin) x K values.
+ */
+int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
+                     const void* Cin, int c_dtype, const uint16_t* bias,
+                     double alpha, double beta, int epi,
+                     int64_t pix_begin, int64_t pix_end, double* ref, double* absacc) {
+    conv_problem cv;
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi);
+    if (rc) return rc;
+    if (pix_begin < 0 || pix_end > cv.N * cv.P * cv.Q || pix_begin > pix_end) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t pix = pix_begin; pix < pix_end; ++pix) {
+        int64_t n = pix / (cv.P * cv.Q);
+        int64_t p = (pix / cv.Q) % cv.P;
+        int64_t q = pix % cv.Q;
+        for (int64_t k = 0; k < cv.K; ++k) {
+            double av;
+            double v = conv_element(&cv, n, p, q, k, &av);
+            ref[(pix - pix_begin) * cv.K + k] = v;
+            if (absacc) absacc[(pix - pix_begin) * cv.K + k] = av;
+        }
+    }
+    return 0;
+}
+
+/* The listed (flattened pixel, output channel) pairs only. */
+int orc_conv2d_points(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
+                      const void* Cin, int c_dtype, const uint16_t* bias,
+                      double alpha, double beta, int epi,
+                      int64_t npts, const int64_t* ppix, const int64_t* pk, double* ref, double* absacc) {
+    conv_problem cv;
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi);
+    if (rc) return rc;
+    for (int64_t t = 0; t < npts; ++t)
+        if (ppix[t] < 0 || ppix[t] >= cv.N * cv.P * cv.Q || pk[t] < 0 || pk[t] >= cv.K) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < npts; ++t) {
+        int64_t pix = ppix[t];
+        double av;
+        ref[t] = conv_element(&cv, pix / (cv.P * cv.Q), (pix / cv.Q) % cv.P, pix % cv.Q, pk[t], &av);
+        if (absacc) absacc[t] = av;
+    }
+    return 0;
+}
+
+/* -------------------------------------------------------------------------------------------
+ * Speed-of-Light bound (Section 4.1; worked example in Appendix A.2).
+ *   step 1  FLOPs (2 per multiply-accumulate) and best-case DRAM bytes: every
+ *           unique input element read once, every output written once.
+ *   step 2  peaks from the specification, scaled linearly by current/max clock.
+ *   step 3  T_compute = FLOPs/peak, T_mem = bytes/bandwidth, t_SOL = max of them.
+ *   step 4  arithmetic intensity against the ridge point peak/bandwidth.
+ * ----------------------------------------------------------------------------------------- */
+int64_t orc_gemm_flops(int64_t M, int64_t N, int64_t K) { return 2 * M * N * K; }
+
+/* has_c: C is read (beta != 0); has_bias: a bias vector of N input-type elements is read. */
+int64_t orc_gemm_bytes(int64_t M, int64_t N, int64_t K, int64_t eb_in, int64_t eb_out, int has_c, int has_bias) {
+    int64_t bytes = (M * K + K * N) * eb_in + M * N * eb_out;
+    if (has_c) bytes += M * N * eb_out;
+    if (has_bias) bytes += N * eb_in;
+    return bytes;
+}
+
+int64_t orc_conv_flops(const int64_t* dims) {
+    int64_t P = orc_conv_out_extent(dims[1], dims[7], dims[11], dims[5], dims[9]);
+    int64_t Q = orc_conv_out_extent(dims[2], dims[8], dims[12], dims[6], dims[10]);
+    return 2 * (dims[0] * P * Q) * dims[4] * (dims[3] * dims[5] * dims[6]);
+}
+
+int64_t orc_conv_bytes(const int64_t* dims, int64_t eb_in, int64_t eb_out, int has_c, int has_bias) {
+    int64_t P = orc_conv_out_extent(dims[1], dims[7], dims[11], dims[5], dims[9]);
+    int64_t Q = orc_conv_out_extent(dims[2], dims[8], dims[12], dims[6], dims[10]);
+    int64_t x = dims[0] * dims[1] * dims[2] * dims[3];
+    int64_t w = dims[4] * dims[5] * dims[6] * dims[3];
+    int64_t y = dims[0] * P * Q * dims[4];
+    int64_t bytes = (x + w) * eb_in + y * eb_out;
+    if (has_c) bytes += y * eb_out;
+    if (has_bias) bytes += dims[4] * eb_in;
+    return bytes;
+}
+
+/*
+ * hw = {peak_flops, peak_bytes_per_s, sm_clock, sm_clock_max, mem_clock, mem_clock_max}
+ *      (a zero clock or zero max clock means "do not scale": ratio 1).
+ * out = {ai, t_compute_s, t_mem_s, t_sol_s, ridge, eff_peak_flops, eff_bytes_per_s, compute_bound}
+ */
+int orc_sol_bound(int64_t flops, int64_t bytes, const double* hw, double* out) {
+    if (flops < 0 || bytes < 0 || hw[0] <= 0.0 || hw[1] <= 0.0) return 1;
+    double sm_ratio = (hw[2] > 0.0 && hw[3] > 0.0) ? hw[2] / hw[3] : 1.0;
+    double mem_ratio = (hw[4] > 0.0 && hw[5] > 0.0) ? hw[4] / hw[5] : 1.0;
+    double eff_peak = hw[0] * sm_ratio;
+    double eff_bw = hw[1] * mem_ratio;
+    double t_c = (double)flops / eff_peak;
+    double t_m = (double)bytes / eff_bw;
+    double ai = bytes > 0 ? (double)flops / (double)bytes : INFINITY;
+    double ridge = eff_peak / eff_bw;
+    out[0] = ai;
+    out[1] = t_c;
+    out[2] = t_m;
+    out[3] = t_c > t_m ? t_c : t_m;
+    out[4] = ridge;
+    out[5] = eff_peak;
+    out[6] = eff_bw;
+    out[7] = ai > ridge ? 1.0 : 0.0;
+    return 0;
+}

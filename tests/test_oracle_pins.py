@@ -1,0 +1,352 @@
+"""Pins for the CPU oracle: closed forms, hand-computed cases, invariants and library special cases.
+
+None of these compares the oracle with itself through a retyped formula: each
+expected value is either written by hand, a mathematical identity, or comes
+from an unrelated library routine (torch fp64 matmul / conv2d / activations).
+A plausible mistake in the oracle (dropped term, wrong sign or index,
+transposed operand, wrong bias direction, wrong padding) fails at least one.
+"""
+import math
+
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2603_29010_b200 import inputs
+from tests import parity
+
+
+def bf(x):
+    return torch.tensor(x, dtype=torch.float64).to(torch.bfloat16)
+
+
+def randi(shape, seed, tid, lo=-3, hi=3):
+    return inputs.small_integers(shape, seed, tid, lo, hi)
+
+
+# ---------------------------------------------------------------- GEMM: hand-written cases
+
+def test_gemm_tiny_hand_computed_tn():
+    # A (row-major) = [[1,2,3],[4,5,6]]; B as a matrix (K x N) = [[1,0],[2,1],[0,3]],
+    # stored column-major, i.e. as its transpose [N,K] = [[1,2,0],[0,1,3]].
+    A = bf([[1, 2, 3], [4, 5, 6]])
+    Bt = bf([[1, 2, 0], [0, 1, 3]])
+    ref, absacc = orc.gemm(A, Bt, layout_a="row", layout_b="col")
+    assert ref.tolist() == [[5.0, 11.0], [14.0, 23.0]]
+    assert absacc.tolist() == [[5.0, 11.0], [14.0, 23.0]]
+
+
+def test_gemm_tiny_hand_computed_all_layouts():
+    Am = [[1, -2, 3], [4, 5, -6]]              # M=2, K=3
+    Bm = [[1, 0], [2, 1], [0, 3]]              # K=3, N=2
+    want = [[-3.0, 7.0], [14.0, -13.0]]
+    A_row, A_col = bf(Am), bf(Am).t().contiguous()
+    B_row, B_col = bf(Bm), bf(Bm).t().contiguous()
+    for la, A in (("row", A_row), ("col", A_col)):
+        for lb, B in (("row", B_row), ("col", B_col)):
+            ref, _ = orc.gemm(A, B, layout_a=la, layout_b=lb)
+            assert ref.tolist() == want, (la, lb)
+
+
+def test_gemm_scaling_bias_order_hand_computed():
+    # acc = [[5, 11]], alpha=2, beta=-1, C=[[1, 3]], bias=[10, -40]:
+    # 2*5 - 1 + 10 = 19 ; 2*11 - 3 - 40 = -21 ; bias is NOT multiplied by alpha.
+    A = bf([[1, 2, 3]])
+    Bt = bf([[1, 2, 0], [0, 1, 3]])
+    C = bf([[1, 3]])
+    bias = bf([10, -40])
+    ref, absacc = orc.gemm(A, Bt, C=C, bias=bias, alpha=2.0, beta=-1.0, epi="bias")
+    assert ref.tolist() == [[19.0, -21.0]]
+    assert absacc.tolist() == [[10.0 + 1.0 + 10.0, 22.0 + 3.0 + 40.0]]
+    ref, _ = orc.gemm(A, Bt, C=C, bias=bias, alpha=2.0, beta=-1.0, epi="relu")
+    assert ref.tolist() == [[19.0, 0.0]]
+
+
+def test_gemm_identity_and_one_hot():
+    K = N = 7
+    Bt = randi([N, K], 1, 2)                                   # column-major storage of b(k,j) = Bt[j,k]
+    eye = torch.eye(K, dtype=torch.bfloat16)
+    ref, _ = orc.gemm(eye, Bt)                                 # I . B = B  -> D[i,j] = b(i,j) = Bt[j,i]
+    assert torch.equal(ref, Bt.t().double())
+    A = randi([5, K], 1, 1)
+    onehot = torch.zeros(N, K, dtype=torch.bfloat16)
+    onehot[3, 2] = 1                                           # b(2,3) = 1: column 3 of D picks column 2 of A
+    ref, _ = orc.gemm(A, onehot)
+    want = torch.zeros(5, N, dtype=torch.float64)
+    want[:, 3] = A[:, 2].double()
+    assert torch.equal(ref, want)
+
+
+@pytest.mark.parametrize("K", [256, 512, 2304, 4096])
+def test_gemm_all_ones_gives_k(K):
+    A = torch.ones(3, K, dtype=torch.bfloat16)
+    Bt = torch.ones(4, K, dtype=torch.bfloat16)
+    ref, absacc = orc.gemm(A, Bt)
+    assert torch.equal(ref, torch.full((3, 4), float(K), dtype=torch.float64))
+    assert torch.equal(absacc, ref)
+
+
+def test_gemm_ones_a_gives_column_sums():
+    K, N = 33, 9
+    Bt = randi([N, K], 2, 2)
+    ref, _ = orc.gemm(torch.ones(2, K, dtype=torch.bfloat16), Bt)
+    assert torch.equal(ref[0], Bt.double().sum(dim=1))
+    assert torch.equal(ref[1], ref[0])
+
+
+# ---------------------------------------------------------------- GEMM: library and invariants
+
+@pytest.mark.parametrize("la,lb", [("row", "col"), ("row", "row"), ("col", "col"), ("col", "row")])
+def test_gemm_matches_torch_fp64_matmul(la, lb):
+    M, N, K = 37, 29, 83
+    Am = inputs.uniform([M, K], 3, 1)
+    Bm = inputs.uniform([K, N], 3, 2)
+    A = Am if la == "row" else Am.t().contiguous()
+    B = Bm if lb == "row" else Bm.t().contiguous()
+    ref, absacc = orc.gemm(A, B, layout_a=la, layout_b=lb)
+    want = Am.double() @ Bm.double()
+    assert torch.allclose(ref, want, rtol=0, atol=1e-12)
+    assert torch.allclose(absacc, Am.double().abs() @ Bm.double().abs(), rtol=0, atol=1e-12)
+
+
+def test_gemm_transpose_identity_through_layout_flags():
+    # (A.B)^T = B^T.A^T : swap operands and flip both layout flags (operand-swap identity).
+    M, N, K = 11, 13, 17
+    A = randi([M, K], 4, 1)            # row-major A
+    Bt = randi([N, K], 4, 2)           # column-major B
+    d, _ = orc.gemm(A, Bt, layout_a="row", layout_b="col")
+    # B^T is N x K: its row-major storage is exactly Bt.  A^T is K x M: its column-major storage is A.
+    dt, _ = orc.gemm(Bt, A, layout_a="row", layout_b="col")
+    assert torch.equal(dt, d.t())
+
+
+def test_gemm_leading_dimensions():
+    M, N, K = 6, 5, 12
+    bigA = randi([M, K + 8], 5, 1)
+    bigB = randi([N, K + 16], 5, 2)
+    ref, _ = orc.gemm(bigA[:, :K], bigB[:, :K])
+    want, _ = orc.gemm(bigA[:, :K].contiguous(), bigB[:, :K].contiguous())
+    assert torch.equal(ref, want)
+    assert torch.equal(ref, bigA[:, :K].double() @ bigB[:, :K].double().t())
+
+
+def test_gemm_alpha_linearity_beta_and_nan_c():
+    M, N, K = 8, 8, 16
+    A, Bt = randi([M, K], 6, 1), randi([N, K], 6, 2)
+    C = randi([M, N], 6, 3)
+    base, _ = orc.gemm(A, Bt)
+    twice, _ = orc.gemm(A, Bt, alpha=2.0)
+    assert torch.equal(twice, 2 * base)
+    plus_c, _ = orc.gemm(A, Bt, C=C, beta=1.0)
+    assert torch.equal(plus_c, base + C.double())
+    c32 = C.float()
+    plus_c32, _ = orc.gemm(A, Bt, C=c32, beta=0.5)
+    assert torch.equal(plus_c32, base + 0.5 * C.double())
+    nan_c = torch.full((M, N), float("nan"), dtype=torch.bfloat16)
+    ignored, _ = orc.gemm(A, Bt, C=nan_c, beta=0.0)
+    assert torch.equal(ignored, base)
+
+
+def test_gemm_bias_is_per_column():
+    M, N, K = 4, 6, 8
+    zeros = torch.zeros(M, K, dtype=torch.bfloat16)
+    bias = bf([1, 2, 3, 4, 5, 6])
+    ref, _ = orc.gemm(zeros, randi([N, K], 7, 2), bias=bias, epi="bias")
+    assert torch.equal(ref, bias.double().expand(M, N))
+
+
+def test_gemm_k_zero_is_the_empty_sum():
+    A = torch.zeros(3, 0, dtype=torch.bfloat16)
+    Bt = torch.zeros(2, 0, dtype=torch.bfloat16)
+    ref, _ = orc.gemm(A, Bt, bias=bf([1.5, -2]), epi="relu")
+    assert ref.tolist() == [[1.5, 0.0]] * 3
+
+
+def test_gemm_rows_and_points_agree_with_full():
+    M, N, K = 19, 7, 31
+    A, Bt = inputs.uniform([M, K], 8, 1), inputs.uniform([N, K], 8, 2)
+    bias = inputs.normal([N], 8, 4)
+    full, facc = orc.gemm(A, Bt, bias=bias, epi="silu")
+    part, pacc = orc.gemm(A, Bt, bias=bias, epi="silu", rows=(5, 11))
+    assert torch.equal(part, full[5:11]) and torch.equal(pacc, facc[5:11])
+    pi, pj = [0, 18, 7, 7], [6, 0, 3, 4]
+    pts, ptacc = orc.gemm_points(A, Bt, pi, pj, bias=bias, epi="silu")
+    assert torch.equal(pts, full[pi, pj]) and torch.equal(ptacc, facc[pi, pj])
+
+
+def test_batched_and_grouped_reduce_to_gemm():
+    A = randi([3, 5, 8], 9, 1)
+    B = randi([3, 4, 8], 9, 2)
+    ref, _ = orc.batched_gemm(A, B)
+    for b in range(3):
+        assert torch.equal(ref[b], A[b].double() @ B[b].double().t())
+    one, _ = orc.batched_gemm(A[:1], B[:1])
+    assert torch.equal(one[0], orc.gemm(A[0], B[0])[0])
+    refs, _ = orc.grouped_gemm([A[0], A[1][:2], A[2][:0]], [B[0], B[1], B[2]])
+    assert torch.equal(refs[0], ref[0]) and torch.equal(refs[1], ref[1][:2]) and refs[2].shape == (0, 4)
+    # permuting groups permutes outputs
+    perm, _ = orc.grouped_gemm([A[1][:2], A[0]], [B[1], B[0]])
+    assert torch.equal(perm[0], refs[1]) and torch.equal(perm[1], refs[0])
+
+
+# ---------------------------------------------------------------- activations
+
+def test_activation_closed_forms():
+    assert orc.act("relu", -3.0) == 0.0 and orc.act("relu", 0.0) == 0.0 and orc.act("relu", 2.5) == 2.5
+    assert orc.act("none", -3.0) == -3.0 and orc.act("bias", -3.0) == -3.0
+    assert orc.act("gelu", 0.0) == 0.0 and orc.act("silu", 0.0) == 0.0
+    assert orc.act("silu", 1.0) == pytest.approx(1.0 / (1.0 + math.exp(-1.0)), rel=1e-15)
+    assert orc.act("silu", 1.0) == pytest.approx(0.7310585786300049, rel=1e-14)
+    assert orc.act("gelu", 1.0) == pytest.approx(0.5 * (1.0 + math.tanh(math.sqrt(2 / math.pi) * 1.044715)), rel=1e-15)
+    assert orc.act("gelu", 1.0) == pytest.approx(0.8411919906082768, rel=1e-13)
+    # the tanh form, not the erf form (they differ by ~1.5e-4 at x = 1)
+    erf_form = 0.5 * (1.0 + math.erf(1.0 / math.sqrt(2.0)))
+    assert abs(orc.act("gelu", 1.0) - erf_form) > 1e-4
+
+
+@pytest.mark.parametrize("x", [0.1, 0.5, 1.0, 2.0, 3.7, 9.0])
+def test_activation_odd_part_identities_and_limits(x):
+    # gelu(x) - gelu(-x) = x and silu(x) - silu(-x) = x hold exactly in real arithmetic.
+    assert orc.act("gelu", x) - orc.act("gelu", -x) == pytest.approx(x, rel=1e-14)
+    assert orc.act("silu", x) - orc.act("silu", -x) == pytest.approx(x, rel=1e-14)
+    assert orc.act("gelu", 40.0) == 40.0 and abs(orc.act("gelu", -40.0)) == 0.0
+    assert orc.act("silu", 50.0) == pytest.approx(50.0, rel=1e-15) and abs(orc.act("silu", -50.0)) < 1e-19
+
+
+def test_activations_match_torch_library_fp64():
+    xs = torch.linspace(-6, 6, 97, dtype=torch.float64)
+    for name, fn in (("gelu", lambda t: torch.nn.functional.gelu(t, approximate="tanh")),
+                     ("silu", torch.nn.functional.silu), ("relu", torch.relu)):
+        got = torch.tensor([orc.act(name, float(x)) for x in xs], dtype=torch.float64)
+        assert torch.allclose(got, fn(xs), rtol=1e-13, atol=1e-15), name
+
+
+# ---------------------------------------------------------------- convolution
+
+def test_conv_tiny_hand_computed():
+    # 1 image, 3x3, 1 channel, values 1..9; 2x2 filter [[1,2],[3,4]], no padding, stride 1.
+    X = bf([[1, 2, 3], [4, 5, 6], [7, 8, 9]]).view(1, 3, 3, 1)
+    Wf = bf([[1, 2], [3, 4]]).view(1, 2, 2, 1)
+    ref, _ = orc.conv2d_fprop(X, Wf)
+    # y[0,0] = 1*1 + 2*2 + 4*3 + 5*4 = 37 (cross-correlation: no filter flip)
+    assert ref.view(2, 2).tolist() == [[37.0, 47.0], [67.0, 77.0]]
+    # stride 2 with padding 1: windows anchored at (-1,-1), (-1,1), (1,-1), (1,1)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1), stride=(2, 2))
+    assert ref.view(2, 2).tolist() == [[4.0, 3 * 2 + 4 * 3.0], [2 * 4 + 4 * 7.0, 5 + 6 * 2 + 8 * 3 + 9 * 4.0]]
+    # dilation 2: taps at rows {0,2} x cols {0,2}
+    ref, _ = orc.conv2d_fprop(X, Wf, dil=(2, 2))
+    assert ref.view(1).tolist() == [1 * 1 + 3 * 2 + 7 * 3 + 9 * 4.0]
+
+
+def test_conv_hand_computed_rectangular_two_channels():
+    # H=2, W=3, C=2; K=2 filters of size R=1, S=2.  Written out by hand.
+    X = bf([[[1, 10], [2, 20], [3, 30]], [[4, 40], [5, 50], [6, 60]]]).view(1, 2, 3, 2)
+    Wf = bf([[[1, 0], [0, 1]], [[-1, 1], [2, 0]]]).view(2, 1, 2, 2)     # [K][R=1][S][C]
+    ref, _ = orc.conv2d_fprop(X, Wf)
+    # k=0: x[.,q,0] + x[.,q+1,1];   k=1: -x[.,q,0] + x[.,q,1] + 2 x[.,q+1,0]
+    want = [[[1 + 20.0, -1 + 10 + 4.0], [2 + 30.0, -2 + 20 + 6.0]],
+            [[4 + 50.0, -4 + 40 + 10.0], [5 + 60.0, -5 + 50 + 12.0]]]
+    assert ref.view(2, 2, 2).tolist() == want
+
+
+def test_conv_delta_filter_reproduces_input():
+    N, H, W, C = 2, 5, 6, 4
+    X = randi([N, H, W, C], 10, 6)
+    Wf = torch.zeros(C, 3, 3, C, dtype=torch.bfloat16)
+    for k in range(C):
+        Wf[k, 1, 1, k] = 1
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    assert torch.equal(ref, X.double())
+
+
+def test_conv_all_ones_counts_valid_taps():
+    C = 3
+    X = torch.ones(1, 5, 7, C, dtype=torch.bfloat16)
+    Wf = torch.ones(2, 3, 3, C, dtype=torch.bfloat16)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    y = ref[0, :, :, 0]
+    assert y[2, 3] == 9 * C and y[0, 3] == 6 * C and y[2, 0] == 6 * C and y[0, 0] == 4 * C and y[4, 6] == 4 * C
+    assert torch.equal(ref[..., 0], ref[..., 1])
+
+
+def test_conv_1x1_is_a_gemm():
+    N, H, W, C, K = 2, 3, 4, 8, 5
+    X = randi([N, H, W, C], 11, 6)
+    Wf = randi([K, 1, 1, C], 11, 7)
+    bias = bf([1, -2, 3, -4, 5])
+    conv, cacc = orc.conv2d_fprop(X, Wf, bias=bias, epi="relu")
+    gemm, gacc = orc.gemm(X.view(-1, C), Wf.view(K, C), bias=bias, epi="relu")
+    assert torch.equal(conv.view(-1, K), gemm) and torch.equal(cacc.view(-1, K), gacc)
+
+
+@pytest.mark.parametrize("pad,stride,dil,R,S", [((1, 1), (1, 1), (1, 1), 3, 3), ((0, 2), (2, 1), (1, 1), 2, 3),
+                                              ((2, 2), (1, 2), (2, 2), 3, 3), ((0, 0), (3, 3), (1, 1), 1, 1)])
+def test_conv_matches_torch_fp64_conv2d(pad, stride, dil, R, S):
+    N, H, W, C, K = 2, 9, 8, 5, 4
+    X = inputs.uniform([N, H, W, C], 12, 6)
+    Wf = inputs.uniform([K, R, S, C], 12, 7)
+    ref, absacc = orc.conv2d_fprop(X, Wf, pad=pad, stride=stride, dil=dil)
+    want = torch.nn.functional.conv2d(X.double().permute(0, 3, 1, 2), Wf.double().permute(0, 3, 1, 2),
+                                      stride=stride, padding=pad, dilation=dil).permute(0, 2, 3, 1)
+    assert ref.shape == want.shape
+    assert torch.allclose(ref, want, rtol=0, atol=1e-12)
+    wabs = torch.nn.functional.conv2d(X.double().abs().permute(0, 3, 1, 2), Wf.double().abs().permute(0, 3, 1, 2),
+                                      stride=stride, padding=pad, dilation=dil).permute(0, 2, 3, 1)
+    assert torch.allclose(absacc, wabs, rtol=0, atol=1e-12)
+
+
+def test_conv_shift_equivariance_in_the_interior():
+    X = randi([1, 8, 8, 2], 13, 6)
+    Wf = randi([3, 3, 3, 2], 13, 7)
+    shifted = torch.zeros_like(X)
+    shifted[:, :, 1:, :] = X[:, :, :-1, :]
+    y, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    ys, _ = orc.conv2d_fprop(shifted, Wf, pad=(1, 1))
+    assert torch.equal(ys[:, :, 2:-1, :], y[:, :, 1:-2, :])
+
+
+def test_conv_beta_bias_and_ranges():
+    N, H, W, C, K = 1, 4, 4, 2, 3
+    X, Wf = randi([N, H, W, C], 14, 6), randi([K, 3, 3, C], 14, 7)
+    Cin = randi([N, H, W, K], 14, 3)
+    bias = bf([0.5, -1, 2])
+    base, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    full, facc = orc.conv2d_fprop(X, Wf, pad=(1, 1), Cin=Cin, bias=bias, alpha=3.0, beta=2.0, epi="bias")
+    assert torch.equal(full, 3 * base + 2 * Cin.double() + bias.double())
+    part, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1), Cin=Cin, bias=bias, alpha=3.0, beta=2.0, epi="bias", pixels=(3, 9))
+    assert torch.equal(part, full.view(-1, K)[3:9])
+    pts, pacc = orc.conv2d_points(X, Wf, [0, 15, 6], [2, 0, 1], pad=(1, 1), Cin=Cin, bias=bias, alpha=3.0, beta=2.0,
+                                  epi="bias")
+    assert torch.equal(pts, full.view(-1, K)[[0, 15, 6], [2, 0, 1]])
+    assert torch.equal(pacc, facc.view(-1, K)[[0, 15, 6], [2, 0, 1]])
+
+
+def test_conv_output_extent():
+    assert orc.conv_out_extent(56, 1, 1, 3, 1) == 56
+    assert orc.conv_out_extent(7, 0, 1, 3, 2) == 3
+    assert orc.conv_out_extent(7, 1, 2, 3, 2) == 3     # (7 + 2 - 4 - 1) / 2 + 1
+    assert orc.conv_out_extent(2, 0, 1, 3, 1) == 0
+
+
+# ---------------------------------------------------------------- tolerance is not vacuous
+
+def test_tolerance_accepts_bf16_rounding_and_rejects_skipped_work():
+    M, N, K = 64, 96, 512
+    A, Bt, bias = inputs.make_gemm(M, N, K, "normal", K ** -0.25, bias=True, seed=15)   # outputs ~ N(0,1)
+    ref, absacc = orc.gemm(A, Bt, bias=bias, epi="relu")
+    parity.assert_matches(ref.to(torch.bfloat16), ref, absacc, "exact result rounded to bf16")
+    parity.assert_matches(ref.to(torch.float32), ref, absacc, "exact result rounded to fp32")
+    # the "skipped computation step" defects: a dropped 64-wide K block, no bias, no activation
+    dropped, _ = orc.gemm(A[:, :K - 64], Bt[:, :K - 64], bias=bias, epi="relu")
+    no_bias, _ = orc.gemm(A, Bt, epi="relu")
+    no_act, _ = orc.gemm(A, Bt, bias=bias, epi="bias")
+    for name, wrong in (("dropped K block", dropped), ("no bias", no_bias), ("no activation", no_act)):
+        for dt in (torch.bfloat16, torch.float32):
+            assert parity.mismatches(wrong.to(dt), ref, absacc).any(), (name, dt)
+    # erf-GELU instead of tanh-GELU is caught on the fp32 path when nothing cancels (K = 1: absacc = |x|)
+    x = torch.linspace(-4, 4, 64, dtype=torch.float64).to(torch.bfloat16).view(-1, 1)
+    want, wacc = orc.gemm(x, torch.ones(1, 1, dtype=torch.bfloat16), epi="gelu")
+    assert torch.equal(wacc, x.double().abs())
+    erf = torch.nn.functional.gelu(x.double())
+    assert not parity.mismatches(want.float(), want, wacc).any()
+    assert parity.mismatches(erf.float(), want, wacc).any()
