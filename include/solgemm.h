@@ -1,0 +1,205 @@
+/*
+ * solgemm.h -- C ABI of libsolgemm: fused dense tensor-core contractions for NVIDIA B200 (sm_100a)
+ *
+ *     D = act(alpha * A.B + beta * C + bias)
+ *
+ * for one GEMM, a strided batch of GEMMs, a ragged group of GEMMs and a 2-D forward
+ * convolution evaluated as an implicit GEMM, plus the Speed-of-Light bound
+ * t_SOL = max(FLOPs / peak, bytes / bandwidth) used to judge their headroom.
+ *
+ * These are the operations the muCUTLASS DSL of arXiv 2603.29010 names gemm(),
+ * batched_gemm(), grouped_gemm(expert_count=E) and conv2d_fprop(kernel_h, kernel_w),
+ * with its .with_dtype / .with_layout / .with_scaling clauses and its `>>` epilogue chain
+ * (Section 3, Table 1, Appendix A.1), and the SOL analysis of Section 4.1 / Appendix A.2.
+ *
+ * General rules (they hold for every entry point unless it says otherwise)
+ *  - Pointers named *_host are host memory; every other data pointer is DEVICE memory on the
+ *    current CUDA device.  The caller owns all buffers; the library allocates no device memory.
+ *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *    enqueue work on that stream and return; they never synchronise.
+ *  - Inputs A, B, bias (and conv X, Wf) are bf16.  The output D is bf16 or fp32 (`out_dtype`);
+ *    C, when read, has the output's dtype and shape.  Accumulation and the epilogue run in fp32;
+ *    the result is rounded to nearest-even.
+ *  - Epilogue: v = alpha*acc (+ beta*C if beta != 0) (+ bias[j] if bias != NULL); D = act(v).
+ *    bias holds one value per output column j (GEMM) or output channel (conv); it is NOT scaled
+ *    by alpha.  SG_EPI_BIAS is the identity activation and requires bias != NULL; every other
+ *    activation accepts an optional bias.  SG_EPI_GELU is the tanh form
+ *    0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))).  beta == 0 means C is never read.
+ *  - Alignment (the TMA rule of the paper's Appendix A.1, constraint 3): every base pointer must
+ *    be 16-byte aligned and every leading dimension / batch stride a multiple of 16 bytes
+ *    (8 bf16 or 4 fp32 elements), else SG_ERR_ALIGNMENT.
+ *  - Errors that can be detected from the arguments return before anything is launched and
+ *    leave D untouched.  Exceptions never cross this boundary.  sg_last_error() gives a
+ *    thread-local, human readable reason for the last non-OK status.
+ *  - A device-side wait that runs out (it should never) makes the kernel stop early and record a
+ *    code; sg_poll_status() reports it after the caller has synchronised the stream.
+ */
+#ifndef SOLGEMM_H_
+#define SOLGEMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SG_OK = 0,
+    SG_ERR_INVALID_ARG = 1,   /* negative size, ld smaller than the extent, unknown enum value */
+    SG_ERR_NULL_POINTER = 2,  /* a required pointer is NULL */
+    SG_ERR_ALIGNMENT = 3,     /* base pointer or stride breaks the 16-byte rule */
+    SG_ERR_UNSUPPORTED = 4,   /* valid request this build does not implement */
+    SG_ERR_ARCH = 5,          /* current device is not compute capability 10.0 */
+    SG_ERR_WORKSPACE = 6,     /* workspace NULL, misaligned or too small */
+    SG_ERR_CUDA = 7,          /* a CUDA runtime/driver call failed */
+    SG_ERR_TIMEOUT = 8        /* a bounded device-side wait expired (see sg_poll_status) */
+} sg_status_t;
+
+typedef enum { SG_BF16 = 0, SG_F32 = 1 } sg_dtype_t;
+typedef enum { SG_ROW_MAJOR = 0, SG_COL_MAJOR = 1 } sg_layout_t;
+typedef enum { SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4 } sg_epilogue_t;
+
+/*
+ * One GEMM problem (DSL: gemm().with_dtype(...).with_layout(A,B,C).with_scaling(alpha,beta) >> ...).
+ *   a(i,k) = A[i*lda + k] (row-major) or A[k*lda + i] (column-major)
+ *   b(k,j) = B[k*ldb + j] (row-major) or B[j*ldb + k] (column-major)
+ *   C and D are row-major with leading dimensions ldc, ldd.  All ld* are in ELEMENTS.
+ * Enum-valued fields are int32_t so that the layout is the same from C, C++ and ctypes.
+ */
+typedef struct sg_gemm_desc {
+    int64_t M, N, K;
+    int32_t layout_a, layout_b;   /* sg_layout_t */
+    int64_t lda, ldb, ldc, ldd;
+    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype must be SG_BF16 */
+    float alpha, beta;
+    int32_t epi;                  /* sg_epilogue_t */
+    int32_t reserved;             /* must be 0 */
+} sg_gemm_desc_t;
+
+/*
+ * sg_gemm: D[M,N] = act(alpha * A.B + beta * C + bias).      (paper: gemm(), Table 1a, Appendix A.1)
+ *   A, B   device, bf16, laid out as layout_a / layout_b and lda / ldb say.
+ *   C      device, out_dtype, [M,N] row-major; may be NULL when beta == 0.
+ *   bias   device, bf16, [N]; may be NULL unless epi == SG_EPI_BIAS.
+ *   D      device, out_dtype, [M,N] row-major; written in full (all M x N elements).
+ * M == 0 or N == 0: SG_OK, nothing is launched.  K == 0: D = act(beta*C + bias).
+ */
+sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C,
+                    const void* bias, void* D, void* cuda_stream);
+
+/*
+ * sg_batched_gemm: the same product for b = 0 .. batch-1, operand X of problem b starting at
+ * X + b*strideX elements.                                      (paper: batched_gemm(), Appendix A.1)
+ *   strideBias == 0 shares one bias vector between all problems.
+ * batch == 0: SG_OK, nothing is launched.
+ */
+sg_status_t sg_batched_gemm(const sg_gemm_desc_t* desc, int64_t batch,
+                            int64_t strideA, int64_t strideB, int64_t strideC, int64_t strideD,
+                            int64_t strideBias,
+                            const void* A, const void* B, const void* C, const void* bias, void* D,
+                            void* cuda_stream);
+
+/*
+ * sg_grouped_gemm: `groups` independent products D_g[M_g,N] = act(alpha*A_g.B_g + beta*C_g + bias_g)
+ * in one launch; N, K, layouts, leading dimensions, dtypes, alpha, beta and epi come from `common`
+ * (its M is ignored), M_g from M_host.              (paper: grouped_gemm(expert_count=E), Table 1a)
+ *   M_host           host, [groups], M_g >= 0 (a group with M_g == 0 is skipped).
+ *   *_ptrs_host      host arrays of `groups` DEVICE pointers.  C_ptrs_host may be NULL when
+ *                    beta == 0; bias_ptrs_host may be NULL (no bias) unless epi == SG_EPI_BIAS.
+ *   workspace_dev    device scratch of at least sg_grouped_gemm_workspace_size(groups) bytes,
+ *                    128-byte aligned; the call writes per-group tensor maps and the tile table
+ *                    into it with a stream-ordered copy.  It must stay untouched until the work
+ *                    enqueued by this call has finished.  The host arrays may be freed on return.
+ */
+sg_status_t sg_grouped_gemm_workspace_size(int32_t groups, size_t* bytes);
+sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const int64_t* M_host,
+                            const void* const* A_ptrs_host, const void* const* B_ptrs_host,
+                            const void* const* C_ptrs_host, const void* const* bias_ptrs_host,
+                            void* const* D_ptrs_host,
+                            void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * One forward convolution (cross-correlation, groups = 1), tensors in the paper's TensorNHWC
+ * layout (Table 1a "Conv2d ... NHWC"; Appendix A.1 conv2d_fprop(kernel_h=R, kernel_w=S)):
+ *   X [N,H,W,C], Wf [K,R,S,C], Y and Cin [N,P,Q,K], bias [K], all contiguous;
+ *   P = floor((H + 2 pad_h - dil_h (R-1) - 1) / stride_h) + 1, Q likewise;
+ *   Y[n,p,q,k] = act( alpha * sum_{r,s,c} X[n, p stride_h - pad_h + r dil_h, q stride_w - pad_w + s dil_w, c]
+ *                                         * Wf[k,r,s,c]  + beta * Cin[n,p,q,k] + bias[k] ),
+ *   taps outside the image contribute zero.  The im2col matrix is never materialised.
+ * Requires C % 8 == 0 and K % 8 == 0 (16-byte rule) and pads / filter extents within the TMA
+ * im2col limits (pad <= 127, (R-1) dil_h <= 255, (S-1) dil_w <= 255), else SG_ERR_ALIGNMENT /
+ * SG_ERR_UNSUPPORTED.
+ */
+typedef struct sg_conv2d_desc {
+    int64_t N, H, W, C, K, R, S;
+    int32_t pad_h, pad_w, stride_h, stride_w, dil_h, dil_w;
+    int32_t in_dtype, out_dtype;  /* sg_dtype_t */
+    float alpha, beta;
+    int32_t epi;                  /* sg_epilogue_t */
+    int32_t reserved;             /* must be 0 */
+} sg_conv2d_desc_t;
+
+sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const void* Wf,
+                            const void* Cin, const void* bias, void* Y, void* cuda_stream);
+
+/*
+ * Speed-of-Light bound (paper: Section 4.1 steps 1-4; worked example in Appendix A.2).
+ * Host-only, pure function of its arguments.
+ *   flops = 2 per multiply-accumulate of the contraction (halo taps of a padded conv included;
+ *           epilogue arithmetic excluded);
+ *   bytes = every unique input element read once + every output element written once
+ *           (C only if beta != 0, bias only if has_bias);
+ *   peaks scaled linearly by current/max clock (a zero clock means ratio 1);
+ *   t_compute = flops / eff_peak, t_mem = bytes / eff_bandwidth, t_sol = max of the two;
+ *   ai = flops / bytes, ridge = eff_peak / eff_bandwidth, compute_bound = ai > ridge.
+ *   op                SG_OP_GEMM / SG_OP_BATCHED / SG_OP_GROUPED: desc is sg_gemm_desc_t;
+ *                     SG_OP_CONV2D: desc is sg_conv2d_desc_t.
+ *   batch_or_groups   batch count (BATCHED), group count (GROUPED), ignored otherwise.
+ *   M_host            [groups] for GROUPED (desc->M ignored), else may be NULL.
+ *   has_bias          0 none; 1 one bias vector per problem; for BATCHED, 2 = one shared vector.
+ */
+typedef struct sg_hw {
+    double peak_flops, peak_bytes_per_s;                 /* at maximum clocks */
+    double sm_clock_mhz, sm_clock_max_mhz, mem_clock_mhz, mem_clock_max_mhz;
+} sg_hw_t;
+
+typedef struct sg_sol {
+    int64_t flops, bytes;
+    double ai, t_compute_s, t_mem_s, t_sol_s, ridge, eff_peak_flops, eff_bytes_per_s;
+    int32_t compute_bound;
+    int32_t reserved;
+} sg_sol_t;
+
+typedef enum { SG_OP_GEMM = 0, SG_OP_BATCHED = 1, SG_OP_GROUPED = 2, SG_OP_CONV2D = 3 } sg_op_t;
+
+sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, const int64_t* M_host,
+                         int32_t elem_bytes_in, int32_t elem_bytes_out, int32_t has_bias,
+                         const sg_hw_t* hw, sg_sol_t* out);
+
+/* Status helpers.  sg_status_string / sg_last_error return pointers to static / thread-local text. */
+const char* sg_status_string(sg_status_t status);
+const char* sg_last_error(void);
+
+/*
+ * sg_poll_status: reads (and clears) the device-side status word of the current device.  Call it
+ * after synchronising the stream(s) the work was enqueued on; `cuda_stream` is used for the read.
+ * SG_OK, or SG_ERR_TIMEOUT with the role / tile / barrier that gave up in sg_last_error().  While
+ * the word is set, later kernels of this library return at once without computing.
+ */
+sg_status_t sg_poll_status(void* cuda_stream);
+
+/*
+ * Tuning knobs for experiments (not needed for correct use): a non-negative value overrides the
+ * shape heuristic for later calls from any thread; -1 restores the heuristic.
+ *   tile_n    64, 128 or 256            cta_pair   0 = one CTA per tile, 1 = two-CTA tiles
+ */
+sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair);
+
+/* Number of kernel launches this library has enqueued from this process (monotonic). */
+int64_t sg_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOLGEMM_H_ */

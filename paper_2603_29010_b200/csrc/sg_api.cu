@@ -1,0 +1,720 @@
+// Host side of libsolgemm: argument validation, tensor-map construction, tile-shape choice,
+// launches, the Speed-of-Light calculator and the status helpers declared in include/solgemm.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "solgemm.h"
+#include "sg_kernel.cuh"
+
+namespace {
+
+using namespace sg;
+
+// ------------------------------------------------------------------------------------------ errors
+thread_local char t_err[512] = "";
+
+sg_status_t fail(sg_status_t st, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_err, sizeof t_err, fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+#define SG_CUDA(call)                                                                              \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess) return fail(SG_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));  \
+    } while (0)
+
+// ------------------------------------------------------------------------------------------ per-device state
+__device__ uint32_t g_status_words[8];
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t,
+                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceState {
+    bool ready = false;
+    sg_status_t init_status = SG_OK;
+    char init_error[256] = "";
+    int sm_count = 0;
+    int max_pairs = 0;               // CTA pairs that can be resident at once
+    uint32_t* status_dev = nullptr;  // device address of g_status_words on this device
+};
+
+constexpr int kMaxDevices = 64;
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_tune_tile_n{-1}, g_tune_pair{-1};
+
+using KernelFn = void (*)(const Params);
+
+struct KernelEntry {
+    KernelFn fn;
+    int smem;
+};
+
+template <int BN, bool kPair, bool kF32>
+KernelEntry entry() {
+    return KernelEntry{contract_kernel<BN, kPair, kF32>, Config<BN, kPair>::SMEM_BYTES};
+}
+
+// index: [bn_idx (64,128,256)][pair][f32]
+KernelEntry kernel_for(int bn, bool pair, bool f32) {
+    switch (bn) {
+        case 64:
+            return pair ? (f32 ? entry<64, true, true>() : entry<64, true, false>())
+                        : (f32 ? entry<64, false, true>() : entry<64, false, false>());
+        case 128:
+            return pair ? (f32 ? entry<128, true, true>() : entry<128, true, false>())
+                        : (f32 ? entry<128, false, true>() : entry<128, false, false>());
+        default:
+            return pair ? (f32 ? entry<256, true, true>() : entry<256, true, false>())
+                        : (f32 ? entry<256, false, true>() : entry<256, false, false>());
+    }
+}
+
+sg_status_t device_state(DeviceState** out) {
+    int dev = 0;
+    SG_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(SG_ERR_CUDA, "device index %d out of range", dev);
+    DeviceState& d = g_dev[dev];
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (!d.ready) {
+        d.ready = true;
+        d.init_status = SG_OK;
+        auto bad = [&](sg_status_t st, const char* what, const char* detail) {
+            d.init_status = st;
+            snprintf(d.init_error, sizeof d.init_error, "%s: %s", what, detail);
+        };
+        cudaDeviceProp prop;
+        cudaError_t e = cudaGetDeviceProperties(&prop, dev);
+        if (e != cudaSuccess) {
+            bad(SG_ERR_CUDA, "cudaGetDeviceProperties", cudaGetErrorString(e));
+        } else if (prop.major != 10 || prop.minor != 0) {
+            char buf[64];
+            snprintf(buf, sizeof buf, "compute capability %d.%d", prop.major, prop.minor);
+            bad(SG_ERR_ARCH, "this library runs on compute capability 10.0 (B200) only, found", buf);
+        } else {
+            d.sm_count = prop.multiProcessorCount;
+            if (!g_encode_tiled) {
+                cudaDriverEntryPointQueryResult q;
+                void* fn = nullptr;
+                e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &q);
+                if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn)
+                    bad(SG_ERR_CUDA, "driver entry point", "cuTensorMapEncodeTiled not found");
+                g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+                fn = nullptr;
+                e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeIm2col", &fn, 12000, cudaEnableDefault, &q);
+                if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn)
+                    bad(SG_ERR_CUDA, "driver entry point", "cuTensorMapEncodeIm2col not found");
+                g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
+            }
+            if (d.init_status == SG_OK) {
+                e = cudaGetSymbolAddress(reinterpret_cast<void**>(&d.status_dev), g_status_words);
+                if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaGetSymbolAddress", cudaGetErrorString(e));
+            }
+            const int bns[3] = {64, 128, 256};
+            for (int i = 0; i < 3 && d.init_status == SG_OK; ++i)
+                for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
+                    for (int f32 = 0; f32 < 2 && d.init_status == SG_OK; ++f32) {
+                        KernelEntry k = kernel_for(bns[i], pair != 0, f32 != 0);
+                        e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
+                        if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
+                    }
+            if (d.init_status == SG_OK) {
+                // how many 2-CTA clusters fit at once (some GPCs may not pair up all of their SMs)
+                KernelEntry k = kernel_for(256, true, false);
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(2 * d.sm_count);
+                cfg.blockDim = dim3(192);
+                cfg.dynamicSmemBytes = k.smem;
+                cudaLaunchAttribute attr;
+                attr.id = cudaLaunchAttributeClusterDimension;
+                attr.val.clusterDim.x = 2;
+                attr.val.clusterDim.y = 1;
+                attr.val.clusterDim.z = 1;
+                cfg.attrs = &attr;
+                cfg.numAttrs = 1;
+                int clusters = 0;
+                e = cudaOccupancyMaxActiveClusters(&clusters, k.fn, &cfg);
+                if (e != cudaSuccess || clusters <= 0) {
+                    cudaGetLastError();
+                    clusters = d.sm_count / 2;
+                }
+                d.max_pairs = clusters < d.sm_count / 2 ? clusters : d.sm_count / 2;
+            }
+        }
+    }
+    if (d.init_status != SG_OK) return fail(d.init_status, "%s", d.init_error);
+    *out = &d;
+    return SG_OK;
+}
+
+// ------------------------------------------------------------------------------------------ tensor maps
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// 3-D tiled map over a row-major [batch][rows][inner] tensor with 128-byte swizzled boxes.
+sg_status_t make_tiled_map(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base, uint64_t inner,
+                           uint64_t rows, uint64_t batch, uint64_t row_stride_elems, uint64_t batch_stride_elems,
+                           uint32_t box_inner, uint32_t box_rows, const char* what) {
+    cuuint64_t dims[3] = {inner, rows, batch};
+    cuuint64_t strides[2] = {row_stride_elems * esize, batch_stride_elems * esize};
+    if (batch <= 1) strides[1] = strides[0] * (rows > 0 ? rows : 1);
+    cuuint32_t box[3] = {box_inner, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode_tiled(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(%s) failed with CUresult %d (dims %llu x %llu x %llu, strides %llu, %llu)",
+                    what, static_cast<int>(r), (unsigned long long)inner, (unsigned long long)rows,
+                    (unsigned long long)batch, (unsigned long long)strides[0], (unsigned long long)strides[1]);
+    return SG_OK;
+}
+
+// ------------------------------------------------------------------------------------------ validation
+struct Checked {
+    bool f32_out;
+    int esize_out;
+};
+
+sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, int32_t reserved,
+                         Checked* c) {
+    if (in_dtype != SG_BF16) return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: only SG_BF16 inputs are implemented", in_dtype);
+    if (out_dtype != SG_BF16 && out_dtype != SG_F32) return fail(SG_ERR_INVALID_ARG, "out_dtype %d is not a sg_dtype_t", out_dtype);
+    if (epi < SG_EPI_NONE || epi > SG_EPI_SILU) return fail(SG_ERR_INVALID_ARG, "epi %d is not a sg_epilogue_t", epi);
+    if (!std::isfinite(alpha) || !std::isfinite(beta)) return fail(SG_ERR_INVALID_ARG, "alpha and beta must be finite");
+    if (reserved != 0) return fail(SG_ERR_INVALID_ARG, "reserved field must be 0");
+    c->f32_out = (out_dtype == SG_F32);
+    c->esize_out = c->f32_out ? 4 : 2;
+    return SG_OK;
+}
+
+sg_status_t check_gemm_desc(const sg_gemm_desc_t* d, bool grouped, Checked* c) {
+    if (!d) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
+    sg_status_t st = check_common(d->in_dtype, d->out_dtype, d->epi, d->alpha, d->beta, d->reserved, c);
+    if (st != SG_OK) return st;
+    if ((!grouped && d->M < 0) || d->N < 0 || d->K < 0) return fail(SG_ERR_INVALID_ARG, "M, N, K must be >= 0");
+    if ((!grouped && d->M > INT32_MAX) || d->N > INT32_MAX || d->K > INT32_MAX)
+        return fail(SG_ERR_UNSUPPORTED, "extents above 2^31-1 are not supported");
+    if (d->layout_a != SG_ROW_MAJOR && d->layout_a != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_a %d is not a sg_layout_t", d->layout_a);
+    if (d->layout_b != SG_ROW_MAJOR && d->layout_b != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_b %d is not a sg_layout_t", d->layout_b);
+    if (d->layout_a != SG_ROW_MAJOR || d->layout_b != SG_COL_MAJOR)
+        return fail(SG_ERR_UNSUPPORTED, "only the K-contiguous operand pair (A row-major, B column-major) is implemented");
+    const int64_t M = grouped ? 1 : d->M;
+    if (d->lda < (d->K > 1 ? d->K : 1) && M > 0) return fail(SG_ERR_INVALID_ARG, "lda %lld < K %lld", (long long)d->lda, (long long)d->K);
+    if (d->ldb < (d->K > 1 ? d->K : 1) && d->N > 0) return fail(SG_ERR_INVALID_ARG, "ldb %lld < K %lld", (long long)d->ldb, (long long)d->K);
+    if (d->ldd < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldd %lld < N %lld", (long long)d->ldd, (long long)d->N);
+    if (d->beta != 0.0f && d->ldc < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldc %lld < N %lld", (long long)d->ldc, (long long)d->N);
+    if ((d->lda * 2) % 16 || (d->ldb * 2) % 16) return fail(SG_ERR_ALIGNMENT, "lda and ldb must be multiples of 8 elements (16 bytes)");
+    if ((d->ldd * c->esize_out) % 16) return fail(SG_ERR_ALIGNMENT, "ldd must be a multiple of 16 bytes");
+    if (d->beta != 0.0f && (d->ldc * c->esize_out) % 16) return fail(SG_ERR_ALIGNMENT, "ldc must be a multiple of 16 bytes");
+    return SG_OK;
+}
+
+sg_status_t check_ptrs(const void* A, const void* B, const void* C, const void* bias, const void* D, int64_t K, float beta,
+                       int32_t epi, const char* who) {
+    if (!D) return fail(SG_ERR_NULL_POINTER, "%s: D is NULL", who);
+    if (K > 0 && (!A || !B)) return fail(SG_ERR_NULL_POINTER, "%s: A or B is NULL", who);
+    if (beta != 0.0f && !C) return fail(SG_ERR_NULL_POINTER, "%s: beta != 0 needs C", who);
+    if (epi == SG_EPI_BIAS && !bias) return fail(SG_ERR_NULL_POINTER, "%s: SG_EPI_BIAS needs bias", who);
+    if (!aligned16(D) || (K > 0 && (!aligned16(A) || !aligned16(B))) || (beta != 0.0f && !aligned16(C)))
+        return fail(SG_ERR_ALIGNMENT, "%s: base pointers must be 16-byte aligned", who);
+    if (bias && (reinterpret_cast<uintptr_t>(bias) & 1u)) return fail(SG_ERR_ALIGNMENT, "%s: bias must be 2-byte aligned", who);
+    return SG_OK;
+}
+
+// ------------------------------------------------------------------------------------------ tile shape
+struct Shape {
+    int bn;
+    bool pair;
+};
+
+// Rough cost model: waves of tiles over the SMs times the tile's area, with a penalty for narrow
+// tiles (their MMAs are bound by shared-memory reads, not by the tensor pipe).
+Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N) {
+    const int force_bn = g_tune_tile_n.load();
+    const int force_pair = g_tune_pair.load();
+    const int bns[3] = {256, 128, 64};
+    const double narrow_penalty[3] = {1.0, 1.08, 1.5};
+    Shape best{256, false};
+    double best_cost = 1e300;
+    for (int pi = 0; pi < 2; ++pi) {
+        if (force_pair >= 0 && pi != force_pair) continue;
+        if (force_pair < 0 && pi == 1) continue;            // pairs only on request until tuned per shape
+        for (int bi = 0; bi < 3; ++bi) {
+            const int bn = bns[bi];
+            if (force_bn > 0 && bn != force_bn) continue;
+            if (pi == 1 && bn / 2 < 32) continue;
+            const int tile_m = pi ? 256 : 128;
+            int64_t tiles = 0;
+            for (int64_t r : rows_per_problem) tiles += ((r + tile_m - 1) / tile_m) * ((N + bn - 1) / bn);
+            tiles *= batch_mult;
+            const int64_t slots = pi ? d.max_pairs : d.sm_count;
+            const int64_t waves = (tiles + slots - 1) / slots;
+            const double cost = static_cast<double>(waves) * bn * narrow_penalty[bi] + 24.0;   // + fixed epilogue tail
+            if (cost < best_cost) {
+                best_cost = cost;
+                best = Shape{bn, pi != 0};
+            }
+        }
+    }
+    return best;
+}
+
+sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params& p, cudaStream_t stream) {
+    KernelEntry k = kernel_for(s.bn, s.pair, f32);
+    const int ctas_per_tile = s.pair ? 2 : 1;
+    const int slots = s.pair ? d.max_pairs : d.sm_count;
+    const int tiles = p.num_tiles < slots ? p.num_tiles : slots;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles * ctas_per_tile);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = k.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = ctas_per_tile;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    SG_CUDA(cudaLaunchKernelEx(&cfg, k.fn, p));
+    g_launches.fetch_add(1);
+    return SG_OK;
+}
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait inside one launch
+
+void base_params(Params* p, const DeviceState& d, float alpha, float beta, int32_t epi) {
+    memset(p, 0, sizeof *p);
+    p->alpha = alpha;
+    p->beta = beta;
+    p->epi = epi;
+    p->status = d.status_dev;
+    p->timeout_ns = kWaitLimitNs;
+}
+
+sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int64_t sB, int64_t sC, int64_t sD,
+                      int64_t sBias, const void* A, const void* B, const void* C, const void* bias, void* D,
+                      void* stream, const char* who) {
+    Checked c;
+    sg_status_t st = check_gemm_desc(desc, false, &c);
+    if (st != SG_OK) return st;
+    if (batch < 0) return fail(SG_ERR_INVALID_ARG, "%s: batch must be >= 0", who);
+    if (batch > 65535 * 16) return fail(SG_ERR_UNSUPPORTED, "%s: batch too large", who);
+    if (desc->M == 0 || desc->N == 0 || batch == 0) return SG_OK;
+    st = check_ptrs(A, B, C, bias, D, desc->K, desc->beta, desc->epi, who);
+    if (st != SG_OK) return st;
+    if (batch > 1) {
+        if (sA < 0 || sB < 0 || sC < 0 || sD < 0 || sBias < 0) return fail(SG_ERR_INVALID_ARG, "%s: negative batch stride", who);
+        if ((sA * 2) % 16 || (sB * 2) % 16 || (sD * c.esize_out) % 16 || (desc->beta != 0.0f && (sC * c.esize_out) % 16))
+            return fail(SG_ERR_ALIGNMENT, "%s: batch strides must be multiples of 16 bytes", who);
+        if (sD < (desc->M - 1) * desc->ldd + desc->N) return fail(SG_ERR_INVALID_ARG, "%s: strideD smaller than one output", who);
+    }
+    DeviceState* d = nullptr;
+    st = device_state(&d);
+    if (st != SG_OK) return st;
+
+    Params p;
+    base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
+    const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N);
+    const int tile_m = s.pair ? 256 : 128;
+    p.mode = MODE_DENSE;
+    p.M = static_cast<int32_t>(desc->M);
+    p.N = static_cast<int32_t>(desc->N);
+    p.K = static_cast<int32_t>(desc->K);
+    p.batch = static_cast<int32_t>(batch);
+    p.tiles_m = static_cast<int32_t>((desc->M + tile_m - 1) / tile_m);
+    p.tiles_n = static_cast<int32_t>((desc->N + s.bn - 1) / s.bn);
+    const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n * batch;
+    if (tiles > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
+    p.num_tiles = static_cast<int32_t>(tiles);
+    p.num_kb = static_cast<int32_t>((desc->K + 63) / 64);
+    p.bias = bias;
+    p.C = desc->beta != 0.0f ? C : nullptr;
+    p.ldc = desc->ldc;
+    p.strideC = sC;
+    p.strideBias = sBias;
+    if (desc->K > 0) {
+        st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
+        if (st != SG_OK) return st;
+        st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+                            s.pair ? s.bn / 2 : s.bn, "B");
+        if (st != SG_OK) return st;
+    }
+    st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, D,
+                        desc->N, desc->M, batch, desc->ldd, sD, c.f32_out ? 32 : 64, 32, "D");
+    if (st != SG_OK) return st;
+    if (desc->K == 0) { p.tmA = p.tmD; p.tmB = p.tmD; }   // never used for loads; keeps the prefetch harmless
+    return launch(*d, s, c.f32_out, p, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------------------------------------------------ grouped
+struct GroupedLayout {
+    size_t off_maps, off_tile_start, off_M, off_bias, off_C, total;
+};
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+GroupedLayout grouped_layout(int32_t groups) {
+    GroupedLayout L;
+    size_t o = 0;
+    L.off_maps = o;        o = round_up(o + static_cast<size_t>(groups) * 3 * sizeof(CUtensorMap), 128);
+    L.off_tile_start = o;  o = round_up(o + (static_cast<size_t>(groups) + 1) * 4, 128);
+    L.off_M = o;           o = round_up(o + static_cast<size_t>(groups) * 4, 128);
+    L.off_bias = o;        o = round_up(o + static_cast<size_t>(groups) * 8, 128);
+    L.off_C = o;           o = round_up(o + static_cast<size_t>(groups) * 8, 128);
+    L.total = o;
+    return L;
+}
+
+// Copies a block of host bytes that travels in the kernel's parameter space into device memory,
+// so that the table reaches the workspace in stream order without a staging allocation.
+constexpr int kBlobBytes = 3840;
+struct Blob {
+    uint8_t bytes[kBlobBytes];
+};
+__global__ void scatter_blob_kernel(const __grid_constant__ Blob blob, uint8_t* dst, int n) {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(blob.bytes);
+    uint32_t* out = reinterpret_cast<uint32_t*>(dst);
+    for (int i = threadIdx.x; i < n / 4; i += blockDim.x) out[i] = src[i];
+}
+
+sg_status_t upload(const std::vector<uint8_t>& host, void* dev, cudaStream_t stream) {
+    for (size_t off = 0; off < host.size(); off += kBlobBytes) {
+        Blob b;
+        const size_t n = host.size() - off < static_cast<size_t>(kBlobBytes) ? host.size() - off : kBlobBytes;
+        memcpy(b.bytes, host.data() + off, n);
+        scatter_blob_kernel<<<1, 256, 0, stream>>>(b, static_cast<uint8_t*>(dev) + off, static_cast<int>(round_up(n, 4)));
+        SG_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    return SG_OK;
+}
+
+}  // namespace
+
+// ============================================================================================ C ABI
+extern "C" {
+
+const char* sg_status_string(sg_status_t s) {
+    switch (s) {
+        case SG_OK: return "SG_OK";
+        case SG_ERR_INVALID_ARG: return "SG_ERR_INVALID_ARG";
+        case SG_ERR_NULL_POINTER: return "SG_ERR_NULL_POINTER";
+        case SG_ERR_ALIGNMENT: return "SG_ERR_ALIGNMENT";
+        case SG_ERR_UNSUPPORTED: return "SG_ERR_UNSUPPORTED";
+        case SG_ERR_ARCH: return "SG_ERR_ARCH";
+        case SG_ERR_WORKSPACE: return "SG_ERR_WORKSPACE";
+        case SG_ERR_CUDA: return "SG_ERR_CUDA";
+        case SG_ERR_TIMEOUT: return "SG_ERR_TIMEOUT";
+    }
+    return "SG_ERR_UNKNOWN";
+}
+
+const char* sg_last_error(void) { return t_err; }
+
+int64_t sg_launch_count(void) { return g_launches.load(); }
+
+sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair) {
+    if (tile_n != -1 && tile_n != 64 && tile_n != 128 && tile_n != 256) return fail(SG_ERR_INVALID_ARG, "tile_n must be -1, 64, 128 or 256");
+    if (cta_pair < -1 || cta_pair > 1) return fail(SG_ERR_INVALID_ARG, "cta_pair must be -1, 0 or 1");
+    g_tune_tile_n.store(tile_n);
+    g_tune_pair.store(cta_pair);
+    return SG_OK;
+}
+
+sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C, const void* bias, void* D,
+                    void* cuda_stream) {
+    return run_dense(desc, 1, 0, 0, 0, 0, 0, A, B, C, bias, D, cuda_stream, "sg_gemm");
+}
+
+sg_status_t sg_batched_gemm(const sg_gemm_desc_t* desc, int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
+                            int64_t strideD, int64_t strideBias, const void* A, const void* B, const void* C,
+                            const void* bias, void* D, void* cuda_stream) {
+    return run_dense(desc, batch, strideA, strideB, strideC, strideD, strideBias, A, B, C, bias, D, cuda_stream,
+                     "sg_batched_gemm");
+}
+
+sg_status_t sg_grouped_gemm_workspace_size(int32_t groups, size_t* bytes) {
+    if (!bytes) return fail(SG_ERR_NULL_POINTER, "bytes is NULL");
+    if (groups < 0) return fail(SG_ERR_INVALID_ARG, "groups must be >= 0");
+    *bytes = grouped_layout(groups > 0 ? groups : 1).total;
+    return SG_OK;
+}
+
+sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const int64_t* M_host,
+                            const void* const* A_ptrs_host, const void* const* B_ptrs_host,
+                            const void* const* C_ptrs_host, const void* const* bias_ptrs_host, void* const* D_ptrs_host,
+                            void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+    Checked c;
+    sg_status_t st = check_gemm_desc(common, true, &c);
+    if (st != SG_OK) return st;
+    if (groups < 0) return fail(SG_ERR_INVALID_ARG, "groups must be >= 0");
+    if (groups == 0 || common->N == 0) return SG_OK;
+    if (!M_host || !A_ptrs_host || !B_ptrs_host || !D_ptrs_host) return fail(SG_ERR_NULL_POINTER, "sg_grouped_gemm: a host array is NULL");
+    if (common->beta != 0.0f && !C_ptrs_host) return fail(SG_ERR_NULL_POINTER, "sg_grouped_gemm: beta != 0 needs C_ptrs_host");
+    if (common->epi == SG_EPI_BIAS && !bias_ptrs_host) return fail(SG_ERR_NULL_POINTER, "sg_grouped_gemm: SG_EPI_BIAS needs bias_ptrs_host");
+    int64_t total_rows = 0;
+    std::vector<int64_t> rows(groups);
+    for (int g = 0; g < groups; ++g) {
+        if (M_host[g] < 0 || M_host[g] > INT32_MAX) return fail(SG_ERR_INVALID_ARG, "sg_grouped_gemm: M[%d] = %lld", g, (long long)M_host[g]);
+        rows[g] = M_host[g];
+        total_rows += M_host[g];
+        if (M_host[g] == 0) continue;
+        st = check_ptrs(A_ptrs_host[g], B_ptrs_host[g], C_ptrs_host ? C_ptrs_host[g] : nullptr,
+                        bias_ptrs_host ? bias_ptrs_host[g] : nullptr, D_ptrs_host[g], common->K, common->beta, common->epi,
+                        "sg_grouped_gemm");
+        if (st != SG_OK) return st;
+        if (bias_ptrs_host && !bias_ptrs_host[g]) return fail(SG_ERR_NULL_POINTER, "sg_grouped_gemm: bias pointer of group %d is NULL", g);
+    }
+    if (total_rows == 0) return SG_OK;
+    const GroupedLayout L = grouped_layout(groups);
+    if (!workspace_dev) return fail(SG_ERR_WORKSPACE, "sg_grouped_gemm: workspace is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 127u) return fail(SG_ERR_WORKSPACE, "sg_grouped_gemm: workspace must be 128-byte aligned");
+    if (workspace_bytes < L.total) return fail(SG_ERR_WORKSPACE, "sg_grouped_gemm: workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
+
+    DeviceState* d = nullptr;
+    st = device_state(&d);
+    if (st != SG_OK) return st;
+    const Shape s = choose_shape(*d, rows, 1, common->N);
+    const int tile_m = s.pair ? 256 : 128;
+    const int tiles_n = static_cast<int>((common->N + s.bn - 1) / s.bn);
+
+    std::vector<uint8_t> host(L.total, 0);
+    CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(host.data() + L.off_maps);
+    int32_t* tile_start = reinterpret_cast<int32_t*>(host.data() + L.off_tile_start);
+    int32_t* gM = reinterpret_cast<int32_t*>(host.data() + L.off_M);
+    const void** gbias = reinterpret_cast<const void**>(host.data() + L.off_bias);
+    const void** gC = reinterpret_cast<const void**>(host.data() + L.off_C);
+    int64_t tiles = 0;
+    for (int g = 0; g < groups; ++g) {
+        tile_start[g] = static_cast<int32_t>(tiles);
+        gM[g] = static_cast<int32_t>(rows[g]);
+        gbias[g] = bias_ptrs_host ? bias_ptrs_host[g] : nullptr;
+        gC[g] = (common->beta != 0.0f && C_ptrs_host) ? C_ptrs_host[g] : nullptr;
+        if (rows[g] == 0) continue;
+        tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
+        if (tiles > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
+        if (common->K > 0) {
+            st = make_tiled_map(&maps[3 * g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A_ptrs_host[g], common->K, rows[g], 1,
+                                common->lda, 0, 64, 128, "A_g");
+            if (st != SG_OK) return st;
+            st = make_tiled_map(&maps[3 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                                common->ldb, 0, 64, s.pair ? s.bn / 2 : s.bn, "B_g");
+            if (st != SG_OK) return st;
+        }
+        st = make_tiled_map(&maps[3 * g + 2], c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                            c.esize_out, D_ptrs_host[g], common->N, rows[g], 1, common->ldd, 0, c.f32_out ? 32 : 64, 32, "D_g");
+        if (st != SG_OK) return st;
+    }
+    tile_start[groups] = static_cast<int32_t>(tiles);
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = upload(host, workspace_dev, stream);
+    if (st != SG_OK) return st;
+
+    Params p;
+    base_params(&p, *d, common->alpha, common->beta, common->epi);
+    uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
+    p.mode = MODE_GROUPED;
+    p.gmaps = reinterpret_cast<const CUtensorMap*>(ws + L.off_maps);
+    p.g_tile_start = reinterpret_cast<const int32_t*>(ws + L.off_tile_start);
+    p.g_M = reinterpret_cast<const int32_t*>(ws + L.off_M);
+    p.g_bias = bias_ptrs_host ? reinterpret_cast<const void* const*>(ws + L.off_bias) : nullptr;
+    p.g_C = common->beta != 0.0f ? reinterpret_cast<const void* const*>(ws + L.off_C) : nullptr;
+    p.ldc = common->ldc;
+    p.N = static_cast<int32_t>(common->N);
+    p.K = static_cast<int32_t>(common->K);
+    p.batch = groups;
+    p.tiles_n = tiles_n;
+    p.num_tiles = static_cast<int32_t>(tiles);
+    p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
+    return launch(*d, s, c.f32_out, p, stream);
+}
+
+sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const void* Wf, const void* Cin, const void* bias,
+                            void* Y, void* cuda_stream) {
+    if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
+    Checked c;
+    sg_status_t st = check_common(desc->in_dtype, desc->out_dtype, desc->epi, desc->alpha, desc->beta, desc->reserved, &c);
+    if (st != SG_OK) return st;
+    if (desc->N < 0 || desc->H < 0 || desc->W < 0 || desc->C < 0 || desc->K < 0 || desc->R < 1 || desc->S < 1)
+        return fail(SG_ERR_INVALID_ARG, "sg_conv2d_fprop: extents must be >= 0 and the filter at least 1x1");
+    if (desc->stride_h < 1 || desc->stride_w < 1 || desc->dil_h < 1 || desc->dil_w < 1 || desc->pad_h < 0 || desc->pad_w < 0)
+        return fail(SG_ERR_INVALID_ARG, "sg_conv2d_fprop: strides and dilations must be >= 1, pads >= 0");
+    const int64_t span_h = desc->H + 2 * desc->pad_h - desc->dil_h * (desc->R - 1) - 1;
+    const int64_t span_w = desc->W + 2 * desc->pad_w - desc->dil_w * (desc->S - 1) - 1;
+    const int64_t P = span_h < 0 ? 0 : span_h / desc->stride_h + 1;
+    const int64_t Q = span_w < 0 ? 0 : span_w / desc->stride_w + 1;
+    const int64_t Mg = desc->N * P * Q;
+    if (Mg == 0 || desc->K == 0) return SG_OK;
+    if (Mg > INT32_MAX || desc->C * desc->R * desc->S > INT32_MAX || desc->K > INT32_MAX || desc->H > 65535 || desc->W > 65535)
+        return fail(SG_ERR_UNSUPPORTED, "sg_conv2d_fprop: extents too large");
+    if (desc->C % 8 || desc->K % 8) return fail(SG_ERR_ALIGNMENT, "sg_conv2d_fprop: C and K must be multiples of 8 (16-byte rule)");
+    if (desc->pad_h > 127 || desc->pad_w > 127 || (desc->R - 1) * desc->dil_h > 255 || (desc->S - 1) * desc->dil_w > 255 ||
+        desc->pad_h - (desc->R - 1) * desc->dil_h < -128 || desc->pad_w - (desc->S - 1) * desc->dil_w < -128 ||
+        desc->stride_h > 8 || desc->stride_w > 8)
+        return fail(SG_ERR_UNSUPPORTED, "sg_conv2d_fprop: pad / filter extent / stride outside the im2col TMA limits");
+    const int64_t Kg = desc->C * desc->R * desc->S;
+    st = check_ptrs(X, Wf, Cin, bias, Y, Kg, desc->beta, desc->epi, "sg_conv2d_fprop");
+    if (st != SG_OK) return st;
+    if (desc->C == 0) return fail(SG_ERR_UNSUPPORTED, "sg_conv2d_fprop: C == 0");
+
+    DeviceState* d = nullptr;
+    st = device_state(&d);
+    if (st != SG_OK) return st;
+    Params p;
+    base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
+    const Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K);
+    const int tile_m = s.pair ? 256 : 128;
+    p.mode = MODE_CONV;
+    p.M = static_cast<int32_t>(Mg);
+    p.N = static_cast<int32_t>(desc->K);
+    p.K = static_cast<int32_t>(Kg);
+    p.batch = 1;
+    p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
+    p.tiles_n = static_cast<int32_t>((desc->K + s.bn - 1) / s.bn);
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.cblocks = static_cast<int32_t>((desc->C + 63) / 64);
+    p.num_kb = static_cast<int32_t>(desc->R * desc->S) * p.cblocks;
+    p.bias = bias;
+    p.C = desc->beta != 0.0f ? Cin : nullptr;
+    p.ldc = desc->K;
+    p.P = static_cast<int32_t>(P);
+    p.Q = static_cast<int32_t>(Q);
+    p.stride_h = desc->stride_h; p.stride_w = desc->stride_w;
+    p.pad_h = desc->pad_h; p.pad_w = desc->pad_w;
+    p.dil_h = desc->dil_h; p.dil_w = desc->dil_w;
+    p.S = static_cast<int32_t>(desc->S);
+
+    // A: im2col view of X [N,H,W,C]: 128 output pixels x 64 channels per load; the bounding box of
+    // base pixels starts at -pad and ends where the last filter tap still touches the padded image.
+    {
+        cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->W),
+                              static_cast<cuuint64_t>(desc->H), static_cast<cuuint64_t>(desc->N)};
+        cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->C) * 2, static_cast<cuuint64_t>(desc->W * desc->C) * 2,
+                                 static_cast<cuuint64_t>(desc->H * desc->W * desc->C) * 2};
+        int lower[2] = {-desc->pad_w, -desc->pad_h};
+        int upper[2] = {static_cast<int>(desc->pad_w - (desc->S - 1) * desc->dil_w),
+                        static_cast<int>(desc->pad_h - (desc->R - 1) * desc->dil_h)};
+        cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(desc->stride_w), static_cast<cuuint32_t>(desc->stride_h), 1};
+        CUresult r = g_encode_im2col(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(X), dims, strides, lower, upper,
+                                     64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(X) failed with CUresult %d", static_cast<int>(r));
+    }
+    // B: filter [K][R*S][C] -> rows = output channels, one tap and 64 input channels per load
+    {
+        cuuint64_t dims[3] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->R * desc->S),
+                              static_cast<cuuint64_t>(desc->K)};
+        cuuint64_t strides[2] = {static_cast<cuuint64_t>(desc->C) * 2, static_cast<cuuint64_t>(Kg) * 2};
+        cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(s.pair ? s.bn / 2 : s.bn)};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = g_encode_tiled(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(Wf), dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
+    }
+    st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, Y,
+                        desc->K, Mg, 1, desc->K, 0, c.f32_out ? 32 : 64, 32, "Y");
+    if (st != SG_OK) return st;
+    return launch(*d, s, c.f32_out, p, static_cast<cudaStream_t>(cuda_stream));
+}
+
+sg_status_t sg_poll_status(void* cuda_stream) {
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    uint32_t words[8] = {0};
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    SG_CUDA(cudaMemcpyAsync(words, d->status_dev, sizeof words, cudaMemcpyDeviceToHost, stream));
+    SG_CUDA(cudaStreamSynchronize(stream));
+    if (words[0] == 0) return SG_OK;
+    SG_CUDA(cudaMemsetAsync(d->status_dev, 0, sizeof words, stream));
+    SG_CUDA(cudaStreamSynchronize(stream));
+    static const char* roles[] = {"?", "producer", "mma", "epilogue", "setup"};
+    const uint32_t role = words[0] >> 24;
+    return fail(SG_ERR_TIMEOUT, "device-side wait expired: role %s, barrier %u, tile %u, parity %u, block %u",
+                roles[role < 5 ? role : 0], words[0] & 0xFFFFFF, words[1], words[2], words[3]);
+}
+
+sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, const int64_t* M_host, int32_t eb_in,
+                         int32_t eb_out, int32_t has_bias, const sg_hw_t* hw, sg_sol_t* out) {
+    if (!desc || !hw || !out) return fail(SG_ERR_NULL_POINTER, "sg_sol_bound: desc, hw and out are required");
+    if (eb_in <= 0 || eb_out <= 0 || has_bias < 0 || has_bias > 2) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: bad element size or has_bias");
+    if (!(hw->peak_flops > 0.0) || !(hw->peak_bytes_per_s > 0.0)) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: peaks must be positive");
+    int64_t macs = 0, elems_in = 0, elems_out = 0;   // inputs counted in input-type elements, C and D in output-type elements
+    if (op == SG_OP_GEMM || op == SG_OP_BATCHED || op == SG_OP_GROUPED) {
+        const sg_gemm_desc_t* g = static_cast<const sg_gemm_desc_t*>(desc);
+        if (g->N < 0 || g->K < 0) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: negative extent");
+        const bool reads_c = g->beta != 0.0f;
+        if (op == SG_OP_GROUPED) {
+            if (!M_host || batch_or_groups < 0) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: grouped needs M_host and groups >= 0");
+            for (int64_t i = 0; i < batch_or_groups; ++i) {
+                const int64_t m = M_host[i];
+                if (m < 0) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: negative M");
+                macs += m * g->N * g->K;
+                elems_in += m * g->K + g->K * g->N + (has_bias ? g->N : 0);
+                elems_out += m * g->N * (reads_c ? 2 : 1);
+            }
+        } else {
+            const int64_t b = (op == SG_OP_BATCHED) ? batch_or_groups : 1;
+            if (g->M < 0 || b < 0) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: negative extent");
+            macs = b * g->M * g->N * g->K;
+            elems_in = b * (g->M * g->K + g->K * g->N);
+            if (has_bias == 1) elems_in += b * g->N;
+            if (has_bias == 2) elems_in += g->N;
+            elems_out = b * g->M * g->N * (reads_c ? 2 : 1);
+        }
+    } else if (op == SG_OP_CONV2D) {
+        const sg_conv2d_desc_t* cv = static_cast<const sg_conv2d_desc_t*>(desc);
+        if (cv->N < 0 || cv->H < 0 || cv->W < 0 || cv->C < 0 || cv->K < 0 || cv->R < 1 || cv->S < 1 || cv->stride_h < 1 ||
+            cv->stride_w < 1 || cv->dil_h < 1 || cv->dil_w < 1 || cv->pad_h < 0 || cv->pad_w < 0)
+            return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: bad convolution descriptor");
+        const int64_t sh = cv->H + 2 * cv->pad_h - cv->dil_h * (cv->R - 1) - 1;
+        const int64_t sw = cv->W + 2 * cv->pad_w - cv->dil_w * (cv->S - 1) - 1;
+        const int64_t P = sh < 0 ? 0 : sh / cv->stride_h + 1;
+        const int64_t Q = sw < 0 ? 0 : sw / cv->stride_w + 1;
+        macs = cv->N * P * Q * cv->K * cv->C * cv->R * cv->S;
+        elems_in = cv->N * cv->H * cv->W * cv->C + cv->K * cv->R * cv->S * cv->C + (has_bias ? cv->K : 0);
+        elems_out = cv->N * P * Q * cv->K * (cv->beta != 0.0f ? 2 : 1);
+    } else {
+        return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: op %d is not a sg_op_t", op);
+    }
+    out->flops = 2 * macs;
+    out->bytes = elems_in * eb_in + elems_out * eb_out;
+    const double sm_ratio = (hw->sm_clock_mhz > 0.0 && hw->sm_clock_max_mhz > 0.0) ? hw->sm_clock_mhz / hw->sm_clock_max_mhz : 1.0;
+    const double mem_ratio = (hw->mem_clock_mhz > 0.0 && hw->mem_clock_max_mhz > 0.0) ? hw->mem_clock_mhz / hw->mem_clock_max_mhz : 1.0;
+    out->eff_peak_flops = hw->peak_flops * sm_ratio;
+    out->eff_bytes_per_s = hw->peak_bytes_per_s * mem_ratio;
+    out->t_compute_s = static_cast<double>(out->flops) / out->eff_peak_flops;
+    out->t_mem_s = static_cast<double>(out->bytes) / out->eff_bytes_per_s;
+    out->t_sol_s = out->t_compute_s > out->t_mem_s ? out->t_compute_s : out->t_mem_s;
+    out->ai = out->bytes > 0 ? static_cast<double>(out->flops) / static_cast<double>(out->bytes) : INFINITY;
+    out->ridge = out->eff_peak_flops / out->eff_bytes_per_s;
+    out->compute_bound = out->ai > out->ridge ? 1 : 0;
+    out->reserved = 0;
+    return SG_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,501 @@
+// The persistent, warp-specialised tcgen05 contraction kernel shared by sg_gemm, sg_batched_gemm,
+// sg_grouped_gemm and sg_conv2d_fprop.
+//
+// One CTA (or a pair of CTAs on neighbouring SMs) owns one output tile at a time and walks a static
+// round-robin list of tiles.  Inside the CTA the work is split by warp:
+//
+//   warp 0      producer   one lane issues TMA loads of the A and B k-blocks into a ring of
+//                          shared-memory stages (128-byte swizzled rows of 64 bf16)
+//   warp 1      MMA        allocates TMEM; one lane issues tcgen05.mma (bf16 x bf16 -> fp32 in
+//                          TMEM) for every k-block and commits to mbarriers
+//   warps 2-5   epilogue   tcgen05.ld TMEM -> registers, v = alpha*acc + beta*C + bias, activation,
+//                          cast, swizzled st.shared, one TMA store per 32-row x 128-byte chunk
+//
+// Two accumulator buffers live in TMEM, so the epilogue of tile i overlaps the main loop of tile
+// i+1.  Every mbarrier wait is bounded: when one expires the kernel records where, raises a flag all
+// roles poll, lets outstanding copies land, frees TMEM and returns.
+#pragma once
+#include <cuda_bf16.h>
+#include "sg_ptx.cuh"
+
+namespace sg {
+
+enum : int32_t { MODE_DENSE = 0, MODE_GROUPED = 1, MODE_CONV = 2 };
+enum : int32_t { EPI_NONE = 0, EPI_BIAS = 1, EPI_RELU = 2, EPI_GELU = 3, EPI_SILU = 4 };
+
+// status word 0: 0 = fine, else (role << 24 | detail); words 1..3 hold tile / barrier / block of the first failure
+enum : uint32_t { ROLE_PRODUCER = 1, ROLE_MMA = 2, ROLE_EPILOGUE = 3, ROLE_SETUP = 4 };
+
+struct alignas(64) Params {
+    CUtensorMap tmA, tmB, tmD;          // dense / batched / conv operands (3-D; conv A is a 4-D im2col map)
+    const CUtensorMap* gmaps;           // grouped: A_g, B_g, D_g maps at [3g], [3g+1], [3g+2]
+    const int32_t* g_tile_start;        // grouped: first tile of group g, [groups + 1]
+    const int32_t* g_M;                 // grouped: rows of group g
+    const void* const* g_bias;          // grouped: per-group bias pointers (or null)
+    const void* const* g_C;             // grouped: per-group C pointers (or null)
+    const void* bias;                   // bf16 [N] (+ b * strideBias)
+    const void* C;                      // out dtype, row-major (+ b * strideC)
+    int64_t ldc, strideC, strideBias;   // elements
+    int32_t M, N, K, batch;             // batch = number of problems (dense) or groups (grouped)
+    int32_t tiles_m, tiles_n, num_tiles, num_kb;
+    float alpha, beta;
+    int32_t epi, mode;
+    int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
+    uint32_t* status;                   // device status words (8 x u32)
+    uint64_t timeout_ns;                // bound of every device-side wait
+};
+
+struct Tile {
+    int m0, n0, b, rows;   // first row / column, problem index, number of valid rows of the problem
+};
+
+template <int TILE_M>
+__device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint) {
+    Tile ti;
+    if (p.mode == MODE_GROUPED) {
+        int g = g_hint;
+        while (t >= p.g_tile_start[g + 1]) ++g;      // tiles are visited in increasing order
+        g_hint = g;
+        const int rows = p.g_M[g];
+        const int tm = (rows + TILE_M - 1) / TILE_M;
+        const int r = t - p.g_tile_start[g];
+        ti.b = g;
+        ti.rows = rows;
+        ti.n0 = r / tm;
+        ti.m0 = (r - ti.n0 * tm) * TILE_M;
+    } else {
+        const int per = p.tiles_m * p.tiles_n;
+        ti.b = t / per;
+        const int r = t - ti.b * per;
+        ti.n0 = r / p.tiles_m;
+        ti.m0 = (r - ti.n0 * p.tiles_m) * TILE_M;
+        ti.rows = p.M;
+    }
+    return ti;   // n0 still counts tiles: the caller scales it by the tile width
+}
+
+// Bounded mbarrier wait.  Returns false when the wait expired or another role already gave up.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Params& p, uint32_t role, uint32_t tile,
+                                       uint32_t which) {
+    volatile uint32_t* st = p.status;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 63u) == 0) {
+            if (st[0] != 0) return false;
+            if (global_timer_ns() - t0 > p.timeout_ns) {
+                if (atomicCAS(p.status, 0u, (role << 24) | (which & 0xFFFFFF)) == 0u) {
+                    st[1] = tile;
+                    st[2] = parity;
+                    st[3] = blockIdx.x;
+                }
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Params& p, uint32_t role, uint32_t tile,
+                                         uint32_t which) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, p, role, tile, which);
+}
+
+__device__ __forceinline__ float apply_act(float v, int epi) {
+    switch (epi) {
+        case EPI_RELU:
+            return fmaxf(v, 0.0f);
+        case EPI_GELU: {
+            // 0.5 v (1 + tanh(u)) == v * sigmoid(2u),  u = sqrt(2/pi) (v + 0.044715 v^3)
+            const float u2 = 1.5957691216057308f * (v + 0.044715f * v * v * v);
+            return __fdividef(v, 1.0f + __expf(-u2));
+        }
+        case EPI_SILU:
+            return __fdividef(v, 1.0f + __expf(-v));
+        default:
+            return v;
+    }
+}
+
+template <int BN, bool kPair>
+struct Config {
+    static constexpr int kCtas = kPair ? 2 : 1;
+    static constexpr int BM = 128;                 // rows per CTA (= TMEM lanes)
+    static constexpr int TILE_M = BM * kCtas;      // rows per tile
+    static constexpr int BK = 64;                  // 64 bf16 = one 128-byte swizzled row
+    static constexpr int B_ROWS = BN / kCtas;      // rows of the B tile this CTA loads
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = B_ROWS * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES_RAW = (192 * 1024) / STAGE_BYTES;
+    static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;   // BN in {64,128,256} -> power of two
+    static constexpr int STAGING_BYTES = 4 * 2 * 4096;             // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
+    static constexpr int OFF_STAGING = STAGES * STAGE_BYTES;
+    static constexpr int OFF_BIAS = OFF_STAGING + STAGING_BYTES;
+    static constexpr int OFF_BAR = OFF_BIAS + 4 * BN * 2;                 // 4 epilogue warps x BN bf16 bias values
+    static constexpr int NUM_BARS = 2 * STAGES + 5;                // full, empty, tmem_full[2], tmem_empty[2], drain
+    static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
+    static constexpr int THREADS = 192;
+};
+
+template <int BN, bool kPair, bool kOutF32>
+__global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant__ Params p) {
+    using Cfg = Config<BN, kPair>;
+    constexpr int kCtas = Cfg::kCtas;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr int CH = kOutF32 ? 32 : 64;          // output columns per 128-byte staging row
+    constexpr int NCHUNK = BN / CH;
+    constexpr uint32_t IDESC = umma_idesc_bf16_f32(Cfg::TILE_M, BN);
+
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
+    const bool leader = (cta_rank == 0);
+
+    const uint32_t bar_base = smem_base + Cfg::OFF_BAR;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 4);
+    const uint32_t tmem_slot = bar_base + 8u * Cfg::NUM_BARS;
+    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem + Cfg::OFF_BAR + 8 * Cfg::NUM_BARS);
+
+    // A sticky failure from an earlier launch, or a misaligned dynamic shared-memory base: do nothing.
+    bool dead = (*reinterpret_cast<volatile uint32_t*>(p.status) != 0u);
+    if ((smem_base & 1023u) != 0u) {
+        if (threadIdx.x == 0) atomicCAS(p.status, 0u, (ROLE_SETUP << 24) | 1u);
+        dead = true;
+    }
+    // Both CTAs of a pair take the same decision: the word can only have been set by an earlier
+    // launch (a wait of this launch cannot expire this early), and the base is the same in every CTA.
+    if (dead) return;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 4 * kCtas);
+        }
+        mbar_init(drain_bar, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc<kPair>(tmem_slot, Cfg::TMEM_COLS);
+        tmem_relinquish<kPair>();
+    }
+    if (warp == 0 && lane == 0 && p.mode != MODE_GROUPED) {
+        prefetch_tensormap(&p.tmA);
+        prefetch_tensormap(&p.tmB);
+        prefetch_tensormap(&p.tmD);
+    }
+    tc_fence_before_sync();
+    if constexpr (kPair) {
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    const int num_kb = p.num_kb;
+    const int first_tile = blockIdx.x / kCtas;
+    const int tile_step = gridDim.x / kCtas;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int g_hint = 0, g_fenced = -1;
+            for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
+                Tile ti = decode_tile<Cfg::TILE_M>(p, t, g_hint);
+                const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
+                const int nb0 = ti.n0 * BN + static_cast<int>(cta_rank) * Cfg::B_ROWS;
+                const CUtensorMap* mapA = &p.tmA;
+                const CUtensorMap* mapB = &p.tmB;
+                int bz = ti.b;
+                if (p.mode == MODE_GROUPED) {
+                    mapA = p.gmaps + 3 * ti.b;
+                    mapB = mapA + 1;
+                    bz = 0;
+                    if (g_fenced != ti.b) {
+                        fence_tensormap_acquire(mapA);
+                        fence_tensormap_acquire(mapB);
+                        g_fenced = ti.b;
+                    }
+                }
+                int cw = 0, ch = 0, cn = 0;
+                if (p.mode == MODE_CONV) {
+                    const int pq = p.P * p.Q;
+                    cn = m0 / pq;
+                    const int rem = m0 - cn * pq;
+                    const int op = rem / p.Q;
+                    const int oq = rem - op * p.Q;
+                    cw = oq * p.stride_w - p.pad_w;
+                    ch = op * p.stride_h - p.pad_h;
+                }
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!wait_bar(empty_bar(stage), phase ^ 1u, p, ROLE_PRODUCER, t, stage)) { ok = false; break; }
+                    const uint32_t a_dst = smem_base + stage * Cfg::STAGE_BYTES;
+                    const uint32_t b_dst = a_dst + Cfg::A_BYTES;
+                    uint32_t fb = full_bar(stage);
+                    if constexpr (kPair) fb = map_to_cta(fb, 0);
+                    if (leader) mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES * kCtas);
+                    if (p.mode == MODE_CONV) {
+                        const int tap = kb / p.cblocks;
+                        const int c0 = (kb - tap * p.cblocks) * Cfg::BK;
+                        const int r = tap / p.S;
+                        const int s = tap - r * p.S;
+                        tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(s * p.dil_w),
+                                                  static_cast<uint16_t>(r * p.dil_h));
+                        tma_load_3d<kPair>(b_dst, mapB, fb, c0, tap, nb0);
+                    } else {
+                        tma_load_3d<kPair>(a_dst, mapA, fb, kb * Cfg::BK, m0, bz);
+                        tma_load_3d<kPair>(b_dst, mapB, fb, kb * Cfg::BK, nb0, bz);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (leader && elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int iter = 0;
+            for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step, ++iter) {
+                const int acc = iter & 1;
+                const uint32_t acc_phase = (iter >> 1) & 1u;
+                if (!wait_bar(tempty_bar(acc), acc_phase ^ 1u, p, ROLE_MMA, t, 100 + acc)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!wait_bar(full_bar(stage), phase, p, ROLE_MMA, t, stage)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_src = smem_base + stage * Cfg::STAGE_BYTES;
+                    const uint64_t a_desc = smem_desc_k_major_sw128(a_src);
+                    const uint64_t b_desc = smem_desc_k_major_sw128(a_src + Cfg::A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < Cfg::BK / 16; ++kk) {
+                        // 16 bf16 along K = 32 bytes = 2 units of the descriptor's address field
+                        umma_bf16<kPair>(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, IDESC, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit<kPair>(empty_bar(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit<kPair>(tfull_bar(acc));
+            }
+            if (!ok) {
+                // let every MMA already issued finish before TMEM is freed
+                umma_commit<kPair>(drain_bar);
+                const uint64_t t0 = global_timer_ns();
+                while (!mbar_try_wait(drain_bar, 0) && global_timer_ns() - t0 < 100000000ull) {}
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue warps 2..5
+        const int q = warp & 3;               // TMEM lane quarter this warp may read
+        const int ew = warp - 2;              // staging slot
+        uint16_t* bias_w = reinterpret_cast<uint16_t*>(smem + Cfg::OFF_BIAS) + ew * BN;   // this warp's bf16 copy
+        const bool has_bias = (p.mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
+        const bool has_c = (p.beta != 0.0f);
+        const float alpha = p.alpha, beta = p.beta;
+        const int epi = p.epi;
+        int iter = 0, g_hint = 0, g_fenced = -1;
+        uint32_t chunk_ctr = 0;
+        uint32_t tempty_remote[2];
+#pragma unroll
+        for (int a = 0; a < 2; ++a) tempty_remote[a] = kPair ? map_to_cta(tempty_bar(a), 0) : tempty_bar(a);
+
+        for (int t = first_tile; t < p.num_tiles && ok; t += tile_step, ++iter) {
+            const int acc = iter & 1;
+            const uint32_t acc_phase = (iter >> 1) & 1u;
+            Tile ti = decode_tile<Cfg::TILE_M>(p, t, g_hint);
+            const int n0 = ti.n0 * BN;
+            const int row0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32;
+            const CUtensorMap* mapD = &p.tmD;
+            const __nv_bfloat16* bias_g = reinterpret_cast<const __nv_bfloat16*>(p.bias);
+            const uint8_t* c_g = reinterpret_cast<const uint8_t*>(p.C);
+            int bz = ti.b;
+            if (p.mode == MODE_GROUPED) {
+                mapD = p.gmaps + 3 * ti.b + 2;
+                bz = 0;
+                if (has_bias) bias_g = reinterpret_cast<const __nv_bfloat16*>(p.g_bias[ti.b]);
+                if (has_c) c_g = reinterpret_cast<const uint8_t*>(p.g_C[ti.b]);
+                if (g_fenced != ti.b) {
+                    fence_tensormap_acquire(mapD);
+                    g_fenced = ti.b;
+                }
+            } else {
+                if (has_bias) bias_g += static_cast<int64_t>(ti.b) * p.strideBias;
+                if (has_c) c_g += static_cast<int64_t>(ti.b) * p.strideC * (kOutF32 ? 4 : 2);
+            }
+            if (has_bias) {
+                // every warp keeps its own copy of the tile's bias values, so no barrier between warps is needed
+                __syncwarp();
+                const uint16_t* bsrc = reinterpret_cast<const uint16_t*>(bias_g);
+                for (int i = lane; i < BN; i += 32) {
+                    const int n = n0 + i;
+                    bias_w[i] = (n < p.N) ? bsrc[n] : static_cast<uint16_t>(0);
+                }
+                __syncwarp();
+            }
+            if (num_kb > 0) {
+                if (!wait_bar(tfull_bar(acc), acc_phase, p, ROLE_EPILOGUE, t, 200 + acc)) { ok = false; break; }
+                tc_fence_after_sync();
+            }
+            const int ncols = min(BN, p.N - n0);
+            const int nchunks = (ncols + CH - 1) / CH;
+            const bool rows_live = row0 < ti.rows;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
+            const int row = row0 + lane;
+
+#pragma unroll 1
+            for (int c = 0; c < nchunks; ++c) {
+                float v[CH];
+                if (num_kb > 0) {
+                    uint32_t r0[32];
+                    tmem_ld_32x32(t_row + c * CH, r0);
+                    if constexpr (!kOutF32) {
+                        uint32_t r1[32];
+                        tmem_ld_32x32(t_row + c * CH + 32, r1);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            v[i] = __uint_as_float(r0[i]);
+                            v[32 + i] = __uint_as_float(r1[i]);
+                        }
+                    } else {
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+                    }
+                    if (c == nchunks - 1) {
+                        // this accumulator buffer is drained: hand it back to the MMA warp
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
+                            else mbar_arrive(tempty_remote[acc]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) v[i] = 0.0f;
+                }
+                if (!rows_live) continue;       // nothing of this warp's 32 rows exists (ragged last tile)
+
+#pragma unroll
+                for (int i = 0; i < CH; ++i) v[i] *= alpha;
+                if (has_c && row < ti.rows) {
+                    const int col0 = n0 + c * CH;
+                    if constexpr (kOutF32) {
+                        const float* cp = reinterpret_cast<const float*>(c_g) + static_cast<int64_t>(row) * p.ldc + col0;
+                        if (col0 + CH <= p.N) {
+#pragma unroll
+                            for (int i = 0; i < CH; i += 4) {
+                                const float4 cv = *reinterpret_cast<const float4*>(cp + i);
+                                v[i] += beta * cv.x; v[i + 1] += beta * cv.y; v[i + 2] += beta * cv.z; v[i + 3] += beta * cv.w;
+                            }
+                        } else {
+                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += beta * cp[i];
+                        }
+                    } else {
+                        const __nv_bfloat16* cp = reinterpret_cast<const __nv_bfloat16*>(c_g) + static_cast<int64_t>(row) * p.ldc + col0;
+                        if (col0 + CH <= p.N) {
+#pragma unroll
+                            for (int i = 0; i < CH; i += 8) {
+                                const uint4 cv = *reinterpret_cast<const uint4*>(cp + i);
+                                const uint32_t w[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    v[i + 2 * j] += beta * __uint_as_float(w[j] << 16);
+                                    v[i + 2 * j + 1] += beta * __uint_as_float(w[j] & 0xFFFF0000u);
+                                }
+                            }
+                        } else {
+                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += beta * __bfloat162float(cp[i]);
+                        }
+                    }
+                }
+                if (has_bias) {
+#pragma unroll
+                    for (int i = 0; i < CH; i += 4) {
+                        const uint2 b2 = *reinterpret_cast<const uint2*>(bias_w + c * CH + i);   // 4 bf16, broadcast read
+                        v[i] += __uint_as_float(b2.x << 16); v[i + 1] += __uint_as_float(b2.x & 0xFFFF0000u);
+                        v[i + 2] += __uint_as_float(b2.y << 16); v[i + 3] += __uint_as_float(b2.y & 0xFFFF0000u);
+                    }
+                }
+                if (epi >= EPI_RELU) {
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) v[i] = apply_act(v[i], epi);
+                }
+
+                // stage the 32 x 128-byte block (row = lane) in the swizzled layout the store map expects
+                const uint32_t sb = chunk_ctr & 1u;
+                ++chunk_ctr;
+                if (lane == 0) tma_store_wait_read<1>();     // the store that last read this buffer is done
+                __syncwarp();
+                const uint32_t stg = smem_base + Cfg::OFF_STAGING + (ew * 2 + sb) * 4096u;
+                const uint32_t row_addr = stg + lane * 128u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t w0, w1, w2, w3;
+                    if constexpr (kOutF32) {
+                        w0 = __float_as_uint(v[4 * j]); w1 = __float_as_uint(v[4 * j + 1]);
+                        w2 = __float_as_uint(v[4 * j + 2]); w3 = __float_as_uint(v[4 * j + 3]);
+                    } else {
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * j], v[8 * j + 1]);
+                        __nv_bfloat162 h1 = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+                        __nv_bfloat162 h3 = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+                        w0 = *reinterpret_cast<uint32_t*>(&h0); w1 = *reinterpret_cast<uint32_t*>(&h1);
+                        w2 = *reinterpret_cast<uint32_t*>(&h2); w3 = *reinterpret_cast<uint32_t*>(&h3);
+                    }
+                    const uint32_t addr = row_addr + ((static_cast<uint32_t>(j) ^ (lane & 7u)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_3d(mapD, stg, n0 + c * CH, row0, bz);
+                    tma_store_commit();
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*reinterpret_cast<volatile uint32_t*>(p.status) != 0u) {
+        // a wait expired somewhere: give copies still in flight time to land before the CTA retires
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before_sync();
+    if constexpr (kPair) {
+        cluster_arrive();
+        cluster_wait();
+    } else {
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc<kPair>(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace sg

@@ -1,0 +1,282 @@
+"""Thin ctypes binding of libsolgemm (``include/solgemm.h``): argument marshalling only.
+
+Every function takes CUDA torch tensors (torch supplies device memory and the
+stream, nothing else), fills the C descriptor, and calls the entry point of the
+same name.  There is no CPU path and no fallback: importing this module raises
+if ``libsolgemm.so`` has not been built, and every call raises ``SolgemmError``
+on a non-OK status.
+
+Operand conventions (the library's): ``A`` is passed as stored, ``[M, K]`` for
+row-major / ``[K, M]`` for column-major; ``B`` is ``[K, N]`` row-major /
+``[N, K]`` column-major; inner stride 1, outer stride = leading dimension.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+from .build import LIB_PATH
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_29010_b200.build` "
+                      "(there is no CPU fallback)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+SG_OK = 0
+STATUS_NAMES = ["SG_OK", "SG_ERR_INVALID_ARG", "SG_ERR_NULL_POINTER", "SG_ERR_ALIGNMENT", "SG_ERR_UNSUPPORTED",
+                "SG_ERR_ARCH", "SG_ERR_WORKSPACE", "SG_ERR_CUDA", "SG_ERR_TIMEOUT"]
+LAYOUTS = {"row": 0, "col": 1}
+EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4}
+DTYPES = {torch.bfloat16: 0, torch.float32: 1}
+OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
+EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm", "sg_conv2d_fprop",
+            "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count"]
+
+
+class SolgemmError(RuntimeError):
+    def __init__(self, status: int, detail: str):
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{name}: {detail}")
+        self.status = status
+        self.status_name = name
+
+
+class GemmDesc(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("layout_a", ctypes.c_int32), ("layout_b", ctypes.c_int32),
+                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64), ("ldd", ctypes.c_int64),
+                ("in_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+                ("alpha", ctypes.c_float), ("beta", ctypes.c_float),
+                ("epi", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class Conv2dDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("N", "H", "W", "C", "K", "R", "S")] + \
+               [(n, ctypes.c_int32) for n in ("pad_h", "pad_w", "stride_h", "stride_w", "dil_h", "dil_w",
+                                              "in_dtype", "out_dtype")] + \
+               [("alpha", ctypes.c_float), ("beta", ctypes.c_float), ("epi", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+class Hw(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in ("peak_flops", "peak_bytes_per_s", "sm_clock_mhz", "sm_clock_max_mhz",
+                                               "mem_clock_mhz", "mem_clock_max_mhz")]
+
+
+class Sol(ctypes.Structure):
+    _fields_ = [("flops", ctypes.c_int64), ("bytes", ctypes.c_int64)] + \
+               [(n, ctypes.c_double) for n in ("ai", "t_compute_s", "t_mem_s", "t_sol_s", "ridge", "eff_peak_flops",
+                                               "eff_bytes_per_s")] + \
+               [("compute_bound", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+_vp, _i64, _i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+_lib.sg_gemm.restype = ctypes.c_int
+_lib.sg_gemm.argtypes = [ctypes.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_batched_gemm.restype = ctypes.c_int
+_lib.sg_batched_gemm.argtypes = [ctypes.POINTER(GemmDesc), _i64, _i64, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_grouped_gemm_workspace_size.restype = ctypes.c_int
+_lib.sg_grouped_gemm_workspace_size.argtypes = [_i32, ctypes.POINTER(ctypes.c_size_t)]
+_lib.sg_grouped_gemm.restype = ctypes.c_int
+_lib.sg_grouped_gemm.argtypes = [ctypes.POINTER(GemmDesc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]
+_lib.sg_conv2d_fprop.restype = ctypes.c_int
+_lib.sg_conv2d_fprop.argtypes = [ctypes.POINTER(Conv2dDesc), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_sol_bound.restype = ctypes.c_int
+_lib.sg_sol_bound.argtypes = [_i32, _vp, _i64, _vp, _i32, _i32, _i32, ctypes.POINTER(Hw), ctypes.POINTER(Sol)]
+_lib.sg_status_string.restype = ctypes.c_char_p
+_lib.sg_status_string.argtypes = [ctypes.c_int]
+_lib.sg_last_error.restype = ctypes.c_char_p
+_lib.sg_poll_status.restype = ctypes.c_int
+_lib.sg_poll_status.argtypes = [_vp]
+_lib.sg_set_tuning.restype = ctypes.c_int
+_lib.sg_set_tuning.argtypes = [_i32, _i32]
+_lib.sg_launch_count.restype = _i64
+
+
+def raw_lib() -> ctypes.CDLL:
+    """The loaded shared library, for callers that want to drive the C ABI directly."""
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != SG_OK:
+        raise SolgemmError(status, _lib.sg_last_error().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ld(t: torch.Tensor) -> int:
+    """Leading dimension of a 2-D operand as stored (outer stride; the row length if there is one row)."""
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError("operands must be 2-D with inner stride 1")
+    return t.stride(0) if t.shape[0] > 1 else max(t.shape[1], 1)
+
+
+def _gemm_desc(M, N, K, lda, ldb, ldc, ldd, layout_a, layout_b, out_dtype, alpha, beta, epi) -> GemmDesc:
+    return GemmDesc(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], lda, ldb, ldc, ldd, 0, DTYPES[out_dtype],
+                    float(alpha), float(beta), EPILOGUES[epi], 0)
+
+
+def _mnk(A, B, layout_a, layout_b):
+    M, K = (A.shape[-2], A.shape[-1]) if layout_a == "row" else (A.shape[-1], A.shape[-2])
+    Kb, N = (B.shape[-2], B.shape[-1]) if layout_b == "row" else (B.shape[-1], B.shape[-2])
+    if K != Kb:
+        raise ValueError("A and B disagree on K")
+    return M, N, K
+
+
+def gemm(A: torch.Tensor, B: torch.Tensor, *, C: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+         out: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.bfloat16, alpha: float = 1.0,
+         beta: float = 0.0, epi: str = "none", layout_a: str = "row", layout_b: str = "col", stream=None) -> torch.Tensor:
+    """D = act(alpha A.B + beta C + bias) through ``sg_gemm``.  Returns D (``out`` if given)."""
+    M, N, K = _mnk(A, B, layout_a, layout_b)
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    desc = _gemm_desc(M, N, K, _ld(A), _ld(B), _ld(C) if C is not None else max(N, 1), _ld(out), layout_a, layout_b,
+                      out.dtype, alpha, beta, epi)
+    _check(_lib.sg_gemm(ctypes.byref(desc), _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
+    return out
+
+
+def batched_gemm(A: torch.Tensor, B: torch.Tensor, *, C=None, bias=None, out=None, out_dtype=torch.bfloat16,
+                 alpha=1.0, beta=0.0, epi="none", layout_a="row", layout_b="col", stream=None) -> torch.Tensor:
+    """The same product for every leading index through ``sg_batched_gemm``; ``bias`` is [N] or [batch, N]."""
+    batch = A.shape[0]
+    M, N, K = _mnk(A, B, layout_a, layout_b)
+    if out is None:
+        out = torch.empty((batch, M, N), dtype=out_dtype, device=A.device)
+    for t in (A, B, out) + ((C,) if C is not None else ()):
+        if t.dim() != 3 or (t.shape[2] > 1 and t.stride(2) != 1):
+            raise ValueError("batched operands must be 3-D with inner stride 1")
+    sbias = 0 if bias is None or bias.dim() == 1 else bias.stride(0)
+    desc = _gemm_desc(M, N, K, A.stride(1), B.stride(1), C.stride(1) if C is not None else max(N, 1), out.stride(1),
+                      layout_a, layout_b, out.dtype, alpha, beta, epi)
+    _check(_lib.sg_batched_gemm(ctypes.byref(desc), batch, A.stride(0), B.stride(0),
+                                C.stride(0) if C is not None else 0, out.stride(0), sbias,
+                                _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
+    return out
+
+
+def grouped_workspace_size(groups: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(_lib.sg_grouped_gemm_workspace_size(groups, ctypes.byref(n)))
+    return int(n.value)
+
+
+def _ptr_array(tensors: Optional[Sequence[Optional[torch.Tensor]]]):
+    if tensors is None:
+        return None
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = None if t is None else t.data_ptr()
+    return arr
+
+
+def grouped_gemm(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=None, biases=None,
+                 outs: Optional[Sequence[torch.Tensor]] = None, out_dtype=torch.bfloat16, alpha=1.0, beta=0.0,
+                 epi="none", layout_a="row", layout_b="col", workspace: Optional[torch.Tensor] = None,
+                 stream=None) -> List[torch.Tensor]:
+    """One launch of ``sg_grouped_gemm`` over groups with their own M_g; N, K and leading dimensions are common."""
+    groups = len(As)
+    if groups == 0:
+        return []
+    _, N, K = _mnk(As[0], Bs[0], layout_a, layout_b)
+    Ms = [(_mnk(a, b, layout_a, layout_b))[0] for a, b in zip(As, Bs)]
+    if outs is None:
+        outs = [torch.empty((m, N), dtype=out_dtype, device=As[0].device) for m in Ms]
+    ld = lambda ts, default: next((_ld(t) for t in ts if t.shape[0] > 1), default)
+    desc = _gemm_desc(0, N, K, ld(As, max(K, 1)), ld(Bs, max(K, 1)), ld(Cs, max(N, 1)) if Cs is not None else max(N, 1),
+                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi)
+    if workspace is None:
+        workspace = torch.empty(grouped_workspace_size(groups), dtype=torch.uint8, device=As[0].device)
+    m_arr = (ctypes.c_int64 * groups)(*Ms)
+    _check(_lib.sg_grouped_gemm(ctypes.byref(desc), groups, m_arr, _ptr_array(As), _ptr_array(Bs), _ptr_array(Cs),
+                                _ptr_array(biases), _ptr_array(outs), _ptr(workspace), workspace.numel(),
+                                _stream(stream)))
+    return list(outs)
+
+
+def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1), dil=(1, 1), Cin=None, bias=None,
+                 out=None, out_dtype=torch.bfloat16, alpha=1.0, beta=0.0, epi="none", stream=None) -> torch.Tensor:
+    """NHWC x KRSC -> NPQK forward convolution through ``sg_conv2d_fprop`` (implicit GEMM, nothing materialised)."""
+    if X.dim() != 4 or Wf.dim() != 4 or not X.is_contiguous() or not Wf.is_contiguous():
+        raise ValueError("X (NHWC) and Wf (KRSC) must be contiguous 4-D tensors")
+    N, H, W, C = X.shape
+    K, R, S, Cw = Wf.shape
+    if C != Cw:
+        raise ValueError("X and Wf disagree on C")
+    ext = lambda size, p, d, f, s: max((size + 2 * p - d * (f - 1) - 1) // s + 1, 0) if size + 2 * p - d * (f - 1) - 1 >= 0 else 0
+    P, Q = ext(H, pad[0], dil[0], R, stride[0]), ext(W, pad[1], dil[1], S, stride[1])
+    if out is None:
+        out = torch.empty((N, P, Q, K), dtype=out_dtype, device=X.device)
+    desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], 0, DTYPES[out.dtype],
+                      float(alpha), float(beta), EPILOGUES[epi], 0)
+    _check(_lib.sg_conv2d_fprop(ctypes.byref(desc), _ptr(X), _ptr(Wf), _ptr(Cin), _ptr(bias), _ptr(out), _stream(stream)))
+    return out
+
+
+def gemm_host(A_host: torch.Tensor, B_host: torch.Tensor, out_host: torch.Tensor, *, bias_host=None, epi="none",
+              alpha=1.0, device="cuda", scratch: Optional[dict] = None, stream=None) -> torch.Tensor:
+    """End-to-end GEMM for callers whose data lives in (pinned) host memory.
+
+    Copies A, B (and bias) to the device, runs ``sg_gemm`` and copies D back into ``out_host``,
+    all on one stream.  ``scratch`` may hold preallocated device buffers ("A", "B", "bias", "D").
+    """
+    scratch = {} if scratch is None else scratch
+    dev = {}
+    for name, t in (("A", A_host), ("B", B_host), ("bias", bias_host)):
+        if t is None:
+            dev[name] = None
+            continue
+        if name not in scratch:
+            scratch[name] = torch.empty(t.shape, dtype=t.dtype, device=device)
+        scratch[name].copy_(t, non_blocking=True)
+        dev[name] = scratch[name]
+    if "D" not in scratch:
+        scratch["D"] = torch.empty(out_host.shape, dtype=out_host.dtype, device=device)
+    gemm(dev["A"], dev["B"], bias=dev["bias"], out=scratch["D"], alpha=alpha, epi=epi, stream=stream)
+    out_host.copy_(scratch["D"], non_blocking=True)
+    return out_host
+
+
+def sol_bound(op: str, *, M=0, N=0, K=0, batch_or_groups=1, Ms: Optional[Sequence[int]] = None, conv: Optional[dict] = None,
+              beta=0.0, elem_bytes_in=2, elem_bytes_out=2, has_bias=0, peak_flops: float, peak_bytes_per_s: float,
+              sm_clock_mhz=0.0, sm_clock_max_mhz=0.0, mem_clock_mhz=0.0, mem_clock_max_mhz=0.0) -> dict:
+    """``sg_sol_bound``: FLOPs, best-case bytes and t_SOL = max(FLOPs/peak, bytes/bandwidth) (host only)."""
+    if op == "conv2d":
+        c = conv
+        desc = Conv2dDesc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], *c.get("pad", (0, 0)),
+                          *c.get("stride", (1, 1)), *c.get("dil", (1, 1)), 0, 0, 1.0, float(beta), 0, 0)
+    else:
+        desc = GemmDesc(M, N, K, 0, 1, max(K, 1), max(K, 1), max(N, 1), max(N, 1), 0, 0, 1.0, float(beta), 0, 0)
+    m_arr = (ctypes.c_int64 * len(Ms))(*Ms) if Ms is not None else None
+    hw = Hw(peak_flops, peak_bytes_per_s, sm_clock_mhz, sm_clock_max_mhz, mem_clock_mhz, mem_clock_max_mhz)
+    out = Sol()
+    _check(_lib.sg_sol_bound(OPS[op], ctypes.byref(desc), batch_or_groups, m_arr, elem_bytes_in, elem_bytes_out,
+                             int(has_bias), ctypes.byref(hw), ctypes.byref(out)))
+    res = {n: getattr(out, n) for n, _ in Sol._fields_ if n != "reserved"}
+    res["compute_bound"] = bool(res["compute_bound"])
+    return res
+
+
+def poll_status(stream=None) -> None:
+    """Raise ``SolgemmError`` if a kernel recorded an expired device-side wait (after the caller has synchronised)."""
+    _check(_lib.sg_poll_status(_stream(stream)))
+
+
+def set_tuning(tile_n: int = -1, cta_pair: int = -1) -> None:
+    _check(_lib.sg_set_tuning(tile_n, cta_pair))
+
+
+def launch_count() -> int:
+    return int(_lib.sg_launch_count())

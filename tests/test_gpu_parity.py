@@ -1,0 +1,282 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+
+Integer-valued problems must match bit for bit (every partial sum is exact in
+fp32 and the result is exact in the output type, so accumulation order cannot
+matter); real-valued problems must match within the stated tolerance on every
+element (small shapes) or on tile-edge rows plus seeded samples (full-size shapes).
+"""
+import math
+
+import pytest
+import torch
+
+from paper_2603_29010_b200 import inputs
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+from oracle import oracle as orc                      # noqa: E402
+from paper_2603_29010_b200 import solgemm as sg       # noqa: E402
+
+DEV = "cuda"
+
+
+@pytest.fixture(autouse=True)
+def _clean_status():
+    sg.set_tuning(-1, -1)
+    yield
+    torch.cuda.synchronize()
+    sg.poll_status()          # raises if any kernel recorded an expired wait
+    sg.set_tuning(-1, -1)
+
+
+def guarded(shape, dtype, pad_rows=8):
+    """An output buffer with NaN guard bands before and after; returns (view, whole)."""
+    rows, cols = shape[-2], shape[-1]
+    lead = int(math.prod(shape[:-2])) if len(shape) > 2 else 1
+    whole = torch.full((lead * rows + 2 * pad_rows, cols), float("nan"), dtype=dtype, device=DEV)
+    view = whole[pad_rows:pad_rows + lead * rows].view(*shape)
+    return view, whole
+
+
+def guards_intact(whole, pad_rows=8):
+    return bool(torch.isnan(whole[:pad_rows]).all() and torch.isnan(whole[-pad_rows:]).all())
+
+
+SHAPES_EXACT = [(128, 64, 64), (256, 256, 256), (300, 200, 136), (129, 72, 8), (1000, 520, 328), (17, 8, 200),
+                (640, 768, 1024)]
+TILINGS = [(64, 0), (128, 0), (256, 0), (64, 1), (128, 1), (256, 1)]
+
+
+@pytest.mark.parametrize("tile_n,pair", TILINGS)
+@pytest.mark.parametrize("M,N,K", SHAPES_EXACT)
+def test_gemm_integer_inputs_bit_exact(M, N, K, tile_n, pair):
+    sg.set_tuning(tile_n, pair)
+    A = inputs.small_integers([M, K], 101, 1)
+    B = inputs.small_integers([N, K], 101, 2)
+    ref, _ = orc.gemm(A, B)
+    assert float(ref.abs().max()) <= 256
+    D, whole = guarded((M, N), torch.bfloat16)
+    sg.gemm(A.to(DEV), B.to(DEV), out=D)
+    parity.assert_bit_exact(D, ref, f"gemm {M}x{N}x{K} tile_n={tile_n} pair={pair}")
+    assert guards_intact(whole)
+
+
+@pytest.mark.parametrize("pair", [0, 1])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("epi", ["none", "bias", "relu", "gelu", "silu"])
+def test_gemm_epilogues_alpha_beta_bias(epi, out_dtype, pair):
+    sg.set_tuning(128, pair)
+    M, N, K = 200, 328, 264
+    A, B, bias = inputs.make_gemm(M, N, K, "normal", K ** -0.25, bias=True, seed=202)
+    C = inputs.normal([M, N], 202, 3).to(out_dtype)
+    ref, absacc = orc.gemm(A, B, C=C, bias=bias, alpha=0.75, beta=-0.5, epi=epi)
+    D = sg.gemm(A.to(DEV), B.to(DEV), C=C.to(DEV), bias=bias.to(DEV), out_dtype=out_dtype, alpha=0.75, beta=-0.5, epi=epi)
+    parity.assert_matches(D, ref, absacc, f"gemm epi={epi} {out_dtype}")
+    if epi != "bias":
+        ref2, acc2 = orc.gemm(A, B, epi=epi)
+        D2 = sg.gemm(A.to(DEV), B.to(DEV), out_dtype=out_dtype, epi=epi)
+        parity.assert_matches(D2, ref2, acc2, f"gemm epi={epi} no bias {out_dtype}")
+
+
+def test_gemm_activation_form_is_pinned_on_the_fp32_path():
+    # K = 1: D = act(x), tolerance 1e-4 |x| -- tight enough to tell tanh-GELU from erf-GELU
+    x = torch.linspace(-6, 6, 256, dtype=torch.float64).to(torch.bfloat16).view(-1, 1)
+    a = torch.zeros(256, 8, dtype=torch.bfloat16)
+    a[:, :1] = x
+    b = torch.zeros(8, 8, dtype=torch.bfloat16)
+    b[:, 0] = 1
+    for epi in ("gelu", "silu", "relu"):
+        ref, absacc = orc.gemm(a, b, epi=epi)
+        D = sg.gemm(a.to(DEV), b.to(DEV), out_dtype=torch.float32, epi=epi)
+        parity.assert_matches(D, ref, absacc, epi)
+
+
+def test_gemm_leading_dimensions_and_k_tail():
+    M, N, K = 150, 90, 100                      # K not a multiple of 64, N not a multiple of 8
+    bigA = inputs.small_integers([M, K + 28], 303, 1)
+    bigB = inputs.small_integers([N, K + 4], 303, 2)
+    ref, _ = orc.gemm(bigA[:, :K], bigB[:, :K])
+    dA, dB = bigA.to(DEV), bigB.to(DEV)
+    bigD = torch.full((M, 104), float("nan"), dtype=torch.bfloat16, device=DEV)
+    sg.gemm(dA[:, :K], dB[:, :K], out=bigD[:, :N])
+    parity.assert_bit_exact(bigD[:, :N], ref, "padded leading dimensions")
+    assert bool(torch.isnan(bigD[:, N:]).all())
+
+
+def test_gemm_k_zero_and_empty():
+    bias = inputs.normal([16], 404, 4)
+    A = torch.zeros(40, 0, dtype=torch.bfloat16)
+    B = torch.zeros(16, 0, dtype=torch.bfloat16)
+    C = inputs.normal([40, 16], 404, 3)
+    ref, absacc = orc.gemm(A, B, C=C, bias=bias, beta=2.0, epi="relu")
+    dA = torch.zeros(40, 8, dtype=torch.bfloat16, device=DEV)[:, :0]
+    dB = torch.zeros(16, 8, dtype=torch.bfloat16, device=DEV)[:, :0]
+    D = sg.gemm(dA, dB, C=C.to(DEV), bias=bias.to(DEV), beta=2.0, epi="relu")
+    parity.assert_matches(D, ref, absacc, "K == 0")
+    launches = sg.launch_count()
+    untouched = torch.full((0, 16), 1.0, dtype=torch.bfloat16, device=DEV)
+    sg.gemm(torch.zeros(0, 8, dtype=torch.bfloat16, device=DEV), torch.zeros(16, 8, dtype=torch.bfloat16, device=DEV),
+            out=untouched)
+    assert sg.launch_count() == launches        # M == 0: nothing launched
+
+
+def test_gemm_beta_zero_never_reads_c():
+    M, N, K = 64, 64, 64
+    A, B = inputs.small_integers([M, K], 505, 1), inputs.small_integers([N, K], 505, 2)
+    ref, _ = orc.gemm(A, B)
+    nan_c = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=DEV)
+    D = sg.gemm(A.to(DEV), B.to(DEV), C=nan_c, beta=0.0)
+    parity.assert_bit_exact(D, ref, "beta == 0 with NaN C")
+
+
+def test_same_pointers_new_contents_and_side_stream():
+    # nothing may be cached by pointer; work must run on the caller's stream, in order
+    M, N, K = 256, 128, 192
+    dA = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+    dB = torch.empty(N, K, dtype=torch.bfloat16, device=DEV)
+    dD = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    side = torch.cuda.Stream()
+    for seed in (1, 2, 3):
+        A, B = inputs.small_integers([M, K], seed, 1), inputs.small_integers([N, K], seed, 2)
+        ref, _ = orc.gemm(A, B)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            dA.copy_(A, non_blocking=True)
+            dB.copy_(B, non_blocking=True)
+            sg.gemm(dA, dB, out=dD)
+            doubled = dD.float() * 2          # dependent op queued behind the kernel on the same stream
+        side.synchronize()
+        parity.assert_bit_exact(dD, ref, f"seed {seed}")
+        assert torch.equal(doubled.cpu().double(), 2 * ref)
+
+
+# ---------------------------------------------------------------------------------------- batched
+
+@pytest.mark.parametrize("tile_n,pair", [(64, 0), (256, 0), (128, 1)])
+def test_batched_gemm_bit_exact_with_strides(tile_n, pair):
+    sg.set_tuning(tile_n, pair)
+    batch, M, N, K = 5, 136, 200, 72
+    Apad = inputs.small_integers([batch, M + 8, K + 8], 606, 1)               # padded batch stride and ld
+    A = Apad[:, :M, :K]
+    B = inputs.small_integers([batch, N, K], 606, 2)
+    ref, _ = orc.batched_gemm(A, B)
+    D, whole = guarded((batch, M, N), torch.bfloat16)
+    sg.batched_gemm(Apad.to(DEV)[:, :M, :K], B.to(DEV), out=D)
+    parity.assert_bit_exact(D, ref, "batched")
+    assert guards_intact(whole)
+    one = sg.batched_gemm(A[:1].to(DEV), B[:1].to(DEV))
+    assert torch.equal(one[0].cpu(), sg.gemm(A[0].to(DEV), B[0].to(DEV)).cpu())
+
+
+def test_batched_gemm_bias_per_batch_and_shared_fp32():
+    batch, M, N, K = 3, 64, 72, 128
+    A = inputs.uniform([batch, M, K], 707, 1)
+    B = inputs.uniform([batch, N, K], 707, 2)
+    bias2 = inputs.normal([batch, N], 707, 4)
+    C = inputs.normal([batch, M, N], 707, 3).float()
+    for bias in (bias2, bias2[0].contiguous()):
+        ref, absacc = orc.batched_gemm(A, B, C=C, bias=bias, beta=1.0, epi="gelu")
+        D = sg.batched_gemm(A.to(DEV), B.to(DEV), C=C.to(DEV), bias=bias.to(DEV), beta=1.0, epi="gelu",
+                            out_dtype=torch.float32)
+        parity.assert_matches(D, ref, absacc, f"batched bias dim {bias.dim()}")
+
+
+# ---------------------------------------------------------------------------------------- grouped
+
+@pytest.mark.parametrize("tile_n,pair", [(128, 0), (256, 0), (256, 1)])
+def test_grouped_gemm_ragged_bit_exact(tile_n, pair):
+    sg.set_tuning(tile_n, pair)
+    Ms = [130, 0, 1, 257, 128, 511]
+    N, K = 264, 136
+    As = [inputs.small_integers([m, K], 808 + g, 1) for g, m in enumerate(Ms)]
+    Bs = [inputs.small_integers([N, K], 808 + g, 2) for g in range(len(Ms))]
+    refs, _ = orc.grouped_gemm(As, Bs)
+    views, wholes = zip(*[guarded((max(m, 1), N), torch.bfloat16) for m in Ms])
+    outs = [v[:m] for v, m in zip(views, Ms)]
+    sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs], outs=outs)
+    for g, m in enumerate(Ms):
+        parity.assert_bit_exact(outs[g], refs[g], f"group {g}")
+        assert bool(torch.isnan(wholes[g][:8]).all() and torch.isnan(wholes[g][8 + m:]).all()), f"guards of group {g}"
+    # a permutation of the groups permutes the outputs; equal groups reduce to the batched call
+    perm = [3, 0, 5]
+    outs_p = sg.grouped_gemm([As[i].to(DEV) for i in perm], [Bs[i].to(DEV) for i in perm])
+    for j, i in enumerate(perm):
+        assert torch.equal(outs_p[j].cpu(), outs[i].cpu())
+
+
+def test_grouped_gemm_epilogue_bias_and_c():
+    Ms = [96, 200, 40]
+    N, K = 136, 264
+    As, Bs = inputs.make_grouped(Ms, N, K, "normal", K ** -0.25, seed=909)
+    biases = [inputs.normal([N], 909 + g, 4) for g in range(len(Ms))]
+    Cs = [inputs.normal([m, N], 909 + g, 3) for g, m in enumerate(Ms)]
+    refs, accs = orc.grouped_gemm(As, Bs, Cs=Cs, biases=biases, alpha=1.5, beta=0.25, epi="silu")
+    outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs], Cs=[c.to(DEV) for c in Cs],
+                           biases=[b.to(DEV) for b in biases], alpha=1.5, beta=0.25, epi="silu")
+    for g in range(len(Ms)):
+        parity.assert_matches(outs[g], refs[g], accs[g], f"group {g}")
+
+
+def test_grouped_equal_sizes_match_batched():
+    groups, M, N, K = 4, 128, 128, 64
+    A = inputs.small_integers([groups, M, K], 111, 1).to(DEV)
+    B = inputs.small_integers([groups, N, K], 111, 2).to(DEV)
+    outs = sg.grouped_gemm(list(A), list(B))
+    bat = sg.batched_gemm(A, B)
+    for g in range(groups):
+        assert torch.equal(outs[g], bat[g])
+
+
+# ---------------------------------------------------------------------------------------- convolution
+
+CONV_CASES = [
+    # N, H, W, C, K, R, S, pad, stride, dil
+    (2, 9, 11, 64, 64, 3, 3, (1, 1), (1, 1), (1, 1)),
+    (3, 14, 14, 24, 40, 3, 3, (1, 1), (1, 1), (1, 1)),       # C, K not multiples of 64
+    (2, 12, 10, 72, 136, 1, 1, (0, 0), (1, 1), (1, 1)),
+    (2, 15, 13, 32, 72, 3, 2, (1, 0), (2, 2), (1, 1)),
+    (1, 17, 19, 16, 64, 3, 3, (2, 2), (1, 2), (2, 2)),
+    (2, 8, 8, 128, 264, 5, 5, (2, 2), (1, 1), (1, 1)),
+]
+
+
+@pytest.mark.parametrize("pair", [0, 1])
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_conv_integer_inputs_bit_exact(case, pair):
+    sg.set_tuning(-1, pair)
+    N, H, W, C, K, R, S, pad, stride, dil = case
+    X = inputs.small_integers([N, H, W, C], 121, 6, -1, 1)
+    Wf = inputs.small_integers([K, R, S, C], 121, 7, -1, 1)
+    keep = inputs.small_integers([K, R, S, C], 122, 7, 0, 3) == 0       # thin the filter so sums stay small
+    Wf = Wf * keep.to(torch.bfloat16)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=pad, stride=stride, dil=dil)
+    assert float(ref.abs().max()) <= 256
+    Y, whole = guarded((ref.shape[0] * ref.shape[1] * ref.shape[2], K), torch.bfloat16)
+    sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=pad, stride=stride, dil=dil, out=Y.view(ref.shape))
+    parity.assert_bit_exact(Y, ref.view(-1, K), f"conv {case}")
+    assert guards_intact(whole)
+
+
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_conv_epilogue_bias_relu_and_residual(out_dtype):
+    N, H, W, C, K = 2, 10, 12, 72, 80
+    X, Wf, bias = inputs.make_conv(N, H, W, C, K, 3, 3, "normal", (C * 9) ** -0.25, bias=True, seed=131)
+    Cin = inputs.normal([N, H, W, K], 131, 3).to(out_dtype)
+    ref, absacc = orc.conv2d_fprop(X, Wf, pad=(1, 1), Cin=Cin, bias=bias, alpha=0.5, beta=1.0, epi="relu")
+    Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1), Cin=Cin.to(DEV), bias=bias.to(DEV), alpha=0.5, beta=1.0,
+                        epi="relu", out_dtype=out_dtype)
+    parity.assert_matches(Y, ref, absacc, f"conv epilogue {out_dtype}")
+
+
+def test_conv_delta_filter_reproduces_input_on_gpu():
+    N, H, W, C = 2, 7, 9, 64
+    X = inputs.uniform([N, H, W, C], 141, 6)
+    Wf = torch.zeros(C, 3, 3, C, dtype=torch.bfloat16)
+    for k in range(C):
+        Wf[k, 1, 1, k] = 1
+    Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1))
+    assert torch.equal(Y.cpu(), X)
