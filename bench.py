@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of libsolgemm's hot path on synthetic data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--all-configs]
+
+One "step" is one pass of the whole hot path -- operand load, tcgen05 contraction, fused epilogue,
+store -- over one batch: a single ``sg_gemm`` launch of the GEMM 4096^3 + bias + ReLU problem
+(bf16 in, fp32 accumulate, bf16 out).  Rank 0 prints ONE JSON line:
+
+* ``value``      TFLOP/s of the whole job (all ranks), operands resident in HBM, CUDA-event timed,
+                 max over ranks; every step uses the next of several distinct buffer sets whose total
+                 size exceeds the 126 MB L2, so no step finds its operands left in L2 by the step before.
+* ``e2e``        the same metric through the public API with pinned HOST buffers: H2D of A, B, bias,
+                 the kernel, and D2H of D inside the timed region.
+* ``roofline``   the kernel's achieved TFLOP/s against the measured dense-bf16 peak of this machine.
+* ``cpu_baseline``  the fp64 CPU oracle, as it stands, timed on a bounded sample of the same problem.
+* ``clocks``     SM clock and throttle reasons sampled during the timed region.
+
+``--impl reference`` times the CPU oracle alone (it is this project's reference implementation).
+With N > 1 (under torchrun) every rank runs the same problem on its own GPU: independent shards,
+no collective on the data path ("weak" scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "TFLOP/s and % of SOL (max of FLOP/peak, bytes/HBM) per config at 1 B200"
+WORKLOAD = "c2_gemm_4096_bias_relu"
+L2_BYTES = 126 * 1024 * 1024
+SPEC_PEAK_FLOPS = 2250e12      # NVIDIA B200 dense bf16 (datasheet)
+SPEC_PEAK_BW = 8000e9          # NVIDIA B200 HBM3e (datasheet)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the
+# ncu capture summarised under profiles/; None until a capture exists.
+NCU_DRAM_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons in a background thread (NVML; read-only)."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+        self._period = period_s
+
+    def sample_once(self):
+        if self._h is None:
+            return
+        try:
+            self.samples.append(int(self._nv.nvmlDeviceGetClockInfo(self._h, self._nv.NVML_CLOCK_SM)))
+            mask = int(self._nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) \
+                if hasattr(self._nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                else int(self._nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            for bit, name in self.REASONS.items():
+                if mask & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample_once()
+            self._stop.wait(self._period)
+
+    def start(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "samples": len(s),
+                "reasons": sorted(self.reasons)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
+
+def oracle_rows_for(seconds: float, hA, hB, hb, epi: str, M: int):
+    """Pick a row count whose oracle run lasts about `seconds`, from a short pilot. Returns (rows, rows_per_s)."""
+    from oracle import oracle as orc
+    pilot = 8
+    t0 = time.perf_counter()
+    orc.gemm(hA, hB, bias=hb, epi=epi, rows=(0, pilot))
+    rate = pilot / max(time.perf_counter() - t0, 1e-6)
+    rows = int(max(1, min(M, rate * seconds)))
+    return rows, rate
+
+
+def run_reference(args, rank: int, world: int) -> None:
+    if rank != 0:
+        return
+    import torch
+    from oracle import oracle as orc
+    from paper_2603_29010_b200 import inputs
+    c = inputs.CONFIGS[WORKLOAD]
+    M, N, K = c["M"], c["N"], c["K"]
+    hA, hB, hb = inputs.make_gemm(M, N, K, c["dist"], c["scale"], bias=True)
+    total = max(args.steps + args.warmup, 1)
+    per_step_s = min(15.0, 150.0 / total)
+    rows, _ = oracle_rows_for(per_step_s, hA, hB, hb, c["epi"], M)
+    for _ in range(args.warmup):
+        orc.gemm(hA, hB, bias=hb, epi=c["epi"], rows=(0, rows))
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        r0 = (s * rows) % max(M - rows + 1, 1)
+        orc.gemm(hA, hB, bias=hb, epi=c["epi"], rows=(r0, r0 + rows))
+    dt = time.perf_counter() - t0
+    flops = 2.0 * rows * N * K * args.steps
+    value = flops / dt / 1e12
+    cores = orc.num_threads()
+    sample = f"{rows} of {M} output rows per step ({rows * N} of {M * N} elements), all N and K"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "M": M, "N": N, "K": K, "layout": "A row-major, B column-major",
+                       "epilogue": "bias+relu", "accumulate": "fp64", "out": "fp64 (unrounded)",
+                       "note": "CPU oracle (plain fp64 loops, OpenMP over rows), timed as it stands on a bounded sample"},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ our arm
+
+def time_steps(fn, steps: int, torch) -> float:
+    """Seconds for `steps` calls of fn(i) on the current stream, CUDA-event timed."""
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(steps):
+        fn(i)
+    stop.record()
+    stop.synchronize()
+    return start.elapsed_time(stop) * 1e-3
+
+
+def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int) -> dict:
+    """Kernel-only timings of the other four configurations (reported inside the one JSON line)."""
+    out = {}
+    hw = dict(peak_flops=peaks["bf16_tflops"] * 1e12, peak_bytes_per_s=peaks["hbm_gbs"] * 1e9)
+    spec = dict(peak_flops=SPEC_PEAK_FLOPS, peak_bytes_per_s=SPEC_PEAK_BW)
+
+    def record(name, fn_factory, sets, sol_kw, nsteps):
+        # One CUDA graph holding one launch per buffer set, replayed back to back: the short kernels of the
+        # small configurations are then timed without host launch gaps between them.
+        fns = [fn_factory(i) for i in range(sets)]
+        for i in range(min(3, sets)):
+            fns[i]()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for f in fns:
+                f()
+        reps = max(3, -(-nsteps // sets))
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        dt = time_steps(lambda i: graph.replay(), reps, torch) / (reps * sets)
+        sol_m = sg.sol_bound(**sol_kw, **hw)
+        sol_s = sg.sol_bound(**sol_kw, **spec)
+        out[name] = {"us": dt * 1e6, "tflops": sol_m["flops"] / dt / 1e12, "gbs": sol_m["bytes"] / dt / 1e9,
+                     "flops": sol_m["flops"], "bytes": sol_m["bytes"],
+                     "t_sol_measured_us": sol_m["t_sol_s"] * 1e6, "frac_of_sol_measured": sol_m["t_sol_s"] / dt,
+                     "t_sol_spec_us": sol_s["t_sol_s"] * 1e6, "frac_of_sol_spec": sol_s["t_sol_s"] / dt,
+                     "bound": "tensor" if sol_m["compute_bound"] else "hbm", "buffer_sets": sets,
+                     "launches_timed": reps * sets, "timing": "CUDA graph of one launch per buffer set, replayed"}
+
+    C = inputs.CONFIGS
+    c = C["c1_gemm_256"]
+    sets = 64
+    data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev) for i in range(4)]
+    outs = [torch.empty(c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+    record("c1_gemm_256", lambda i: (lambda: sg.gemm(data[i % 4][0], data[i % 4][1], out=outs[i])), sets,
+           dict(op="gemm", M=c["M"], N=c["N"], K=c["K"]), max(steps, 200))
+
+    c = C["c3_batched_128x256x256x512_gelu"]
+    sets = 8      # 8 x 84 MB > L2
+    data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev, batch=c["batch"])
+            for i in range(sets)]
+    outs = [torch.empty(c["batch"], c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+    record("c3_batched_128x256x256x512_gelu",
+           lambda i: (lambda: sg.batched_gemm(data[i][0], data[i][1], out=outs[i], epi=c["epi"])), sets,
+           dict(op="batched", M=c["M"], N=c["N"], K=c["K"], batch_or_groups=c["batch"]), max(steps, 200))
+
+    c4 = C["c4_conv_32x56x56x256_k256_3x3_bias_relu"]
+    sets = 4
+    data4 = [inputs.make_conv(c4["N"], c4["H"], c4["W"], c4["C"], c4["K"], c4["R"], c4["S"], c4["dist"], c4["scale"],
+                              bias=True, seed=i, device=dev) for i in range(sets)]
+    outs4 = [torch.empty(c4["N"], 56, 56, c4["K"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+    record("c4_conv_32x56x56x256_k256_3x3_bias_relu",
+           lambda i: (lambda: sg.conv2d_fprop(data4[i][0], data4[i][1], pad=c4["pad"], bias=data4[i][2], out=outs4[i],
+                                              epi=c4["epi"])), sets,
+           dict(op="conv2d", conv={k: c4[k] for k in ("N", "H", "W", "C", "K", "R", "S", "pad")}, has_bias=1),
+           max(steps // 2, 50))
+
+    c5 = C["c5_grouped_16xMx4096x4096_silu"]
+    Ms = inputs.grouped_sizes(c5["groups"], c5["M_lo"], c5["M_hi"])
+    As, Bs = inputs.make_grouped(Ms, c5["N"], c5["K"], c5["dist"], c5["scale"], device=dev)     # 1.1 GB > L2
+    outs5 = [torch.empty(m, c5["N"], dtype=torch.bfloat16, device=dev) for m in Ms]
+    ws = torch.empty(sg.grouped_workspace_size(len(Ms)), dtype=torch.uint8, device=dev)
+    record("c5_grouped_16xMx4096x4096_silu",
+           lambda i: (lambda: sg.grouped_gemm(As, Bs, outs=outs5, epi=c5["epi"], workspace=ws)), 1,
+           dict(op="grouped", N=c5["N"], K=c5["K"], batch_or_groups=len(Ms), Ms=Ms), max(steps // 10, 20))
+    out["c5_grouped_16xMx4096x4096_silu"]["M_i"] = Ms
+    return out
+
+
+def run_ours(args, rank: int, world: int, local_rank: int) -> None:
+    import torch
+    import torch.distributed as dist
+    from paper_2603_29010_b200 import inputs
+    from paper_2603_29010_b200 import solgemm as sg      # raises if the CUDA library is missing
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    c = inputs.CONFIGS[WORKLOAD]
+    M, N, K = c["M"], c["N"], c["K"]
+    peaks, peaks_kind = measured_peaks()
+    footprint = 2 * (M * K + N * K + M * N) + 2 * N
+    sets = -(-4 * L2_BYTES // footprint) + 1                       # distinct buffer sets cycled through: > 4x L2 in total
+    data = [inputs.make_gemm(M, N, K, c["dist"], c["scale"], bias=True, seed=inputs.BASE_SEED + 17 * rank + i, device=dev)
+            for i in range(sets)]
+    outs = [torch.empty(M, N, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+
+    def step(i):
+        A, B, bias = data[i % sets]
+        sg.gemm(A, B, bias=bias, out=outs[i % sets], epi=c["epi"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    launches0 = sg.launch_count()
+    dt = time_steps(step, args.steps, torch)
+    sampler.sample_once()
+    launches = sg.launch_count() - launches0
+    barrier()
+    clocks = sampler.stop()
+    sg.poll_status()
+    if world > 1:
+        t = torch.tensor([dt], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+
+    # ---- end to end: pinned host buffers, copies inside the timed region
+    hA, hB, hb = (t.cpu().pin_memory() for t in data[0])
+    hD = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
+    scratch = {}
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        sg.gemm_host(hA, hB, hD, bias_host=hb, epi=c["epi"], device=dev, scratch=scratch)
+    barrier()
+    dt_e2e = time_steps(lambda i: sg.gemm_host(hA, hB, hD, bias_host=hb, epi=c["epi"], device=dev, scratch=scratch),
+                        e2e_steps, torch)
+    barrier()
+    if world > 1:
+        t = torch.tensor([dt_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt_e2e = float(t.item())
+    h2d = 2 * (M * K + N * K) + 2 * N
+    d2h = 2 * M * N
+
+    flops = 2.0 * M * N * K
+    per_launch = dt / args.steps
+    achieved = flops / per_launch / 1e12
+    sustained = dt >= 1.0
+    peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    sol_spec = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=SPEC_PEAK_FLOPS, peak_bytes_per_s=SPEC_PEAK_BW)
+    sol_meas = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=peaks["bf16_tflops"] * 1e12,
+                            peak_bytes_per_s=peaks["hbm_gbs"] * 1e9)
+    sol_clock = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=SPEC_PEAK_FLOPS, peak_bytes_per_s=SPEC_PEAK_BW,
+                             sm_clock_mhz=float(clocks["sm_mhz"] or 0), sm_clock_max_mhz=float(clocks["sm_max_mhz"] or 0))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = {
+        "metric": METRIC, "value": world * achieved, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": per_launch * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": M, "N": N, "K": K, "layout": "A row-major, B column-major",
+                   "epilogue": "bias+relu", "accumulate": "fp32", "out": "bf16",
+                   "l2": f"inputs larger than L2: {sets} distinct buffer sets ({sets * footprint / 1e6:.0f} MB) used in turn",
+                   "per_gpu": "every rank runs the whole problem on its own GPU (no collective)"},
+        "clocks": clocks,
+        "e2e": {"value": world * flops / (dt_e2e / e2e_steps) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": dt_e2e / e2e_steps * 1e3},
+        "gpu_launches": launches,
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": NCU_DRAM_BYTES_PER_LAUNCH, "algorithmic_flops_per_launch": int(flops),
+                     "algorithmic_bytes_per_launch": int(sol_spec["bytes"]),
+                     "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16 of {peaks_kind} peaks",
+                     "kernel": "sg::contract_kernel"},
+        "sol": {"flops": sol_spec["flops"], "bytes": sol_spec["bytes"], "ai": sol_spec["ai"],
+                "t_sol_us_spec": sol_spec["t_sol_s"] * 1e6, "frac_of_sol_spec": sol_spec["t_sol_s"] / per_launch,
+                "t_sol_us_measured_peaks": sol_meas["t_sol_s"] * 1e6, "frac_of_sol_measured_peaks": sol_meas["t_sol_s"] / per_launch,
+                "t_sol_us_clock_scaled": sol_clock["t_sol_s"] * 1e6, "frac_of_sol_clock_scaled": sol_clock["t_sol_s"] / per_launch,
+                "suspicious_faster_than_0.9_sol": bool(per_launch < 0.9 * sol_spec["t_sol_s"])},
+    }
+
+    if world == 1:
+        from oracle import oracle as orc
+        hA2, hB2, hb2 = (t.cpu() for t in data[0])
+        rows, _ = oracle_rows_for(12.0, hA2, hB2, hb2, c["epi"], M)
+        t0 = time.perf_counter()
+        ref, absacc = orc.gemm(hA2, hB2, bias=hb2, epi=c["epi"], rows=(0, rows))
+        cpu_dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": 2.0 * rows * N * K / cpu_dt / 1e12, "unit": "TFLOP/s", "cores": orc.num_threads(),
+                                "kind": "oracle", "seconds": cpu_dt,
+                                "sample": f"rows 0..{rows} of {M} ({rows * N} of {M * N} output elements), all N and K"}
+        # the same rows double as a parity spot check of the timed configuration
+        step(0)
+        torch.cuda.synchronize()
+        got = outs[0][:rows].cpu().double()
+        line["parity_sample_ok"] = bool(((got - ref).abs() <= 1e-2 + 1e-2 * ref.abs()).all())
+        if args.all_configs:
+            line["per_config"] = bench_extra_configs(sg, inputs, torch, dev, peaks, args.steps)
+            if args.torch_ref:
+                A, B, bias = data[0]
+                f = lambda i: torch.relu(torch.addmm(bias, data[i % sets][0], data[i % sets][1].t()))
+                for i in range(3):
+                    f(i)
+                torch.cuda.synchronize()
+                tt = time_steps(f, args.steps, torch) / args.steps
+                line["torch_reference"] = {"what": "torch.relu(torch.addmm(bias, A, B.T)) (library kernels, not this code)",
+                                           "tflops": flops / tt / 1e12, "us": tt * 1e6}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (N=1 only)")
+    ap.add_argument("--torch-ref", action="store_true", help="with --all-configs: also time torch's library kernels")
+    args = ap.parse_args()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus > 1 and world == 1:
+        # not under torchrun: start one process per GPU on this node
+        port = os.environ.get("MASTER_PORT", "29511")
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", port, os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    if args.impl == "reference":
+        if args.steps < 1:
+            args.steps = 1
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

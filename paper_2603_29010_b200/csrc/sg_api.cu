@@ -354,6 +354,9 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.ldc = desc->ldc;
     p.strideC = sC;
     p.strideBias = sBias;
+    p.D = D;
+    p.ldd = desc->ldd;
+    p.strideD = sD;
     if (desc->K > 0) {
         st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
         if (st != SG_OK) return st;
@@ -370,7 +373,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
 
 // ------------------------------------------------------------------------------------------ grouped
 struct GroupedLayout {
-    size_t off_maps, off_tile_start, off_M, off_bias, off_C, total;
+    size_t off_maps, off_tile_start, off_M, off_bias, off_C, off_D, total;
 };
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -383,6 +386,7 @@ GroupedLayout grouped_layout(int32_t groups) {
     L.off_M = o;           o = round_up(o + static_cast<size_t>(groups) * 4, 128);
     L.off_bias = o;        o = round_up(o + static_cast<size_t>(groups) * 8, 128);
     L.off_C = o;           o = round_up(o + static_cast<size_t>(groups) * 8, 128);
+    L.off_D = o;           o = round_up(o + static_cast<size_t>(groups) * 8, 128);
     L.total = o;
     return L;
 }
@@ -506,12 +510,14 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     int32_t* gM = reinterpret_cast<int32_t*>(host.data() + L.off_M);
     const void** gbias = reinterpret_cast<const void**>(host.data() + L.off_bias);
     const void** gC = reinterpret_cast<const void**>(host.data() + L.off_C);
+    void** gD = reinterpret_cast<void**>(host.data() + L.off_D);
     int64_t tiles = 0;
     for (int g = 0; g < groups; ++g) {
         tile_start[g] = static_cast<int32_t>(tiles);
         gM[g] = static_cast<int32_t>(rows[g]);
         gbias[g] = bias_ptrs_host ? bias_ptrs_host[g] : nullptr;
         gC[g] = (common->beta != 0.0f && C_ptrs_host) ? C_ptrs_host[g] : nullptr;
+        gD[g] = D_ptrs_host[g];
         if (rows[g] == 0) continue;
         tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
         if (tiles > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
@@ -542,7 +548,9 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     p.g_M = reinterpret_cast<const int32_t*>(ws + L.off_M);
     p.g_bias = bias_ptrs_host ? reinterpret_cast<const void* const*>(ws + L.off_bias) : nullptr;
     p.g_C = common->beta != 0.0f ? reinterpret_cast<const void* const*>(ws + L.off_C) : nullptr;
+    p.g_D = reinterpret_cast<void* const*>(ws + L.off_D);
     p.ldc = common->ldc;
+    p.ldd = common->ldd;
     p.N = static_cast<int32_t>(common->N);
     p.K = static_cast<int32_t>(common->K);
     p.batch = groups;
@@ -600,6 +608,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     p.bias = bias;
     p.C = desc->beta != 0.0f ? Cin : nullptr;
     p.ldc = desc->K;
+    p.D = Y;
+    p.ldd = desc->K;
     p.P = static_cast<int32_t>(P);
     p.Q = static_cast<int32_t>(Q);
     p.stride_h = desc->stride_h; p.stride_w = desc->stride_w;

@@ -33,6 +33,9 @@ struct alignas(64) Params {
     const int32_t* g_M;                 // grouped: rows of group g
     const void* const* g_bias;          // grouped: per-group bias pointers (or null)
     const void* const* g_C;             // grouped: per-group C pointers (or null)
+    void* const* g_D;                   // grouped: per-group D pointers
+    void* D;                            // out dtype, row-major (+ b * strideD); used for ragged column tails only
+    int64_t ldd, strideD;               // elements
     const void* bias;                   // bf16 [N] (+ b * strideBias)
     const void* C;                      // out dtype, row-major (+ b * strideC)
     int64_t ldc, strideC, strideBias;   // elements
@@ -328,12 +331,14 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
             const CUtensorMap* mapD = &p.tmD;
             const __nv_bfloat16* bias_g = reinterpret_cast<const __nv_bfloat16*>(p.bias);
             const uint8_t* c_g = reinterpret_cast<const uint8_t*>(p.C);
+            uint8_t* d_g = reinterpret_cast<uint8_t*>(p.D);
             int bz = ti.b;
             if (p.mode == MODE_GROUPED) {
                 mapD = p.gmaps + 3 * ti.b + 2;
                 bz = 0;
                 if (has_bias) bias_g = reinterpret_cast<const __nv_bfloat16*>(p.g_bias[ti.b]);
                 if (has_c) c_g = reinterpret_cast<const uint8_t*>(p.g_C[ti.b]);
+                d_g = reinterpret_cast<uint8_t*>(p.g_D[ti.b]);
                 if (g_fenced != ti.b) {
                     fence_tensormap_acquire(mapD);
                     g_fenced = ti.b;
@@ -341,6 +346,7 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
             } else {
                 if (has_bias) bias_g += static_cast<int64_t>(ti.b) * p.strideBias;
                 if (has_c) c_g += static_cast<int64_t>(ti.b) * p.strideC * (kOutF32 ? 4 : 2);
+                d_g += static_cast<int64_t>(ti.b) * p.strideD * (kOutF32 ? 4 : 2);
             }
             if (has_bias) {
                 // every warp keeps its own copy of the tile's bias values, so no barrier between warps is needed
@@ -441,6 +447,24 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                 if (epi >= EPI_RELU) {
 #pragma unroll
                     for (int i = 0; i < CH; ++i) v[i] = apply_act(v[i], epi);
+                }
+
+                // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
+                // the last, partial chunk is therefore written with plain stores so nothing beyond column N changes.
+                constexpr int kElemsPer16B = kOutF32 ? 4 : 8;
+                if (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0) {
+                    if (row < ti.rows) {
+                        const int col0 = n0 + c * CH;
+                        if constexpr (kOutF32) {
+                            float* dp = reinterpret_cast<float*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
+                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) dp[i] = v[i];
+                        } else {
+                            __nv_bfloat16* dp = reinterpret_cast<__nv_bfloat16*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
+                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) dp[i] = __float2bfloat16_rn(v[i]);
+                        }
+                    }
+                    __syncwarp();
+                    continue;
                 }
 
                 // stage the 32 x 128-byte block (row = lane) in the swizzled layout the store map expects
