@@ -285,7 +285,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
     launches0 = sg.launch_count()
+    torch.cuda.profiler.start()            # lets `ncu --profile-from-start off` see the timed region only
     dt = time_steps(step, args.steps, torch)
+    torch.cuda.profiler.stop()
     sampler.sample_once()
     launches = sg.launch_count() - launches0
     barrier()
@@ -297,17 +299,19 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         dt = float(t.item())
 
     # ---- end to end: pinned host buffers, copies inside the timed region
-    hA, hB, hb = (t.cpu().pin_memory() for t in data[0])
-    hD = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
-    scratch = {}
     e2e_steps = max(3, min(args.steps, 20))
-    for _ in range(3):
-        sg.gemm_host(hA, hB, hD, bias_host=hb, epi=c["epi"], device=dev, scratch=scratch)
-    barrier()
-    dt_e2e = time_steps(lambda i: sg.gemm_host(hA, hB, hD, bias_host=hb, epi=c["epi"], device=dev, scratch=scratch),
-                        e2e_steps, torch)
-    barrier()
-    if world > 1:
+    dt_e2e = float("nan")
+    if not args.kernel_only:
+        hA, hB, hb = (t.cpu().pin_memory() for t in data[0])
+        hD = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
+        scratch = {}
+        for _ in range(3):
+            sg.gemm_host(hA, hB, hD, bias_host=hb, epi=c["epi"], device=dev, scratch=scratch)
+        barrier()
+        dt_e2e = time_steps(lambda i: sg.gemm_host(hA, hB, hD, bias_host=hb, epi=c["epi"], device=dev, scratch=scratch),
+                            e2e_steps, torch)
+        barrier()
+    if world > 1 and not args.kernel_only:
         t = torch.tensor([dt_e2e], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dt_e2e = float(t.item())
@@ -317,7 +321,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     flops = 2.0 * M * N * K
     per_launch = dt / args.steps
     achieved = flops / per_launch / 1e12
-    sustained = dt >= 1.0
+    # Denominator: the burst cuBLAS figure for short timed regions; the sustained one when the region ran long
+    # enough (>= 0.1 s of back-to-back launches) to be held at the board's power cap, as the clock record shows.
+    sustained = dt >= 0.1 and "sw_power_cap" in clocks["reasons"]
     peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     sol_spec = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=SPEC_PEAK_FLOPS, peak_bytes_per_s=SPEC_PEAK_BW)
     sol_meas = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=peaks["bf16_tflops"] * 1e12,
@@ -346,6 +352,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                      "traffic": NCU_DRAM_BYTES_PER_LAUNCH, "algorithmic_flops_per_launch": int(flops),
                      "algorithmic_bytes_per_launch": int(sol_spec["bytes"]),
                      "peak_source": f"{'sustained' if sustained else 'burst'} cuBLAS bf16 of {peaks_kind} peaks",
+                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                     "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                     "tiling": sg.last_launch_plan(),
                      "kernel": "sg::contract_kernel"},
         "sol": {"flops": sol_spec["flops"], "bytes": sol_spec["bytes"], "ai": sol_spec["ai"],
                 "t_sol_us_spec": sol_spec["t_sol_s"] * 1e6, "frac_of_sol_spec": sol_spec["t_sol_s"] / per_launch,
@@ -354,7 +363,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                 "suspicious_faster_than_0.9_sol": bool(per_launch < 0.9 * sol_spec["t_sol_s"])},
     }
 
-    if world == 1:
+    if args.kernel_only:
+        line["e2e"] = None
+    if world == 1 and not args.kernel_only:
         from oracle import oracle as orc
         hA2, hB2, hb2 = (t.cpu() for t in data[0])
         rows, _ = oracle_rows_for(12.0, hA2, hB2, hb2, c["epi"], M)
@@ -393,6 +404,8 @@ def main() -> None:
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (N=1 only)")
     ap.add_argument("--torch-ref", action="store_true", help="with --all-configs: also time torch's library kernels")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernel)")
     args = ap.parse_args()
 
     world = int(os.environ.get("WORLD_SIZE", "1"))

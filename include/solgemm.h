@@ -199,6 +199,14 @@ sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair);
 /* Number of kernel launches this library has enqueued from this process (monotonic). */
 int64_t sg_launch_count(void);
 
+/*
+ * How the calling thread's most recent contraction launch was tiled, for tests and benchmark records:
+ *   plan6[0] tile width in columns, [1] 1 for two-CTA tiles, [2] tail split (the tiles of the last,
+ *   partial wave are cut into this many column slices; 1 = none), [3] length of the tile list,
+ *   [4] list position of the first slice, [5] grid size in CTAs.
+ */
+sg_status_t sg_last_launch_plan(int32_t* plan6);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,15 +25,19 @@ def is_stale() -> bool:
     return any(os.path.getmtime(os.path.join(_CSRC, d)) > built for d in _DEPS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the CUDA sources into ``libsolgemm.so`` next to this file and return its path."""
-    if not force and not is_stale():
+def build(force: bool = False, verbose: bool = False, extra_flags=(), out_path: str = LIB_PATH) -> str:
+    """Compile the CUDA sources into ``libsolgemm.so`` next to this file and return its path.
+
+    ``extra_flags`` / ``out_path`` build an experimental variant (e.g. ``-DSG_MAX_STAGES=4``) beside the
+    product library; ``SOLGEMM_LIB`` makes the binding load it.
+    """
+    if out_path == LIB_PATH and not extra_flags and not force and not is_stale():
         return LIB_PATH
-    tmp = LIB_PATH + ".tmp%d" % os.getpid()
+    tmp = out_path + ".tmp%d" % os.getpid()
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v",
            "-I", os.path.join(_ROOT, "include"), "-I", _CSRC]
-    cmd += [os.path.join(_CSRC, s) for s in _SOURCES] + ["-o", tmp]
+    cmd += list(extra_flags) + [os.path.join(_CSRC, s) for s in _SOURCES] + ["-o", tmp]
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or proc.returncode != 0:
         sys.stderr.write(proc.stdout + proc.stderr)
@@ -41,8 +45,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed building libsolgemm.so")
     with open(os.path.join(_PKG, "ptxas.log"), "w") as f:
         f.write(proc.stderr)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out_path)
+    return out_path
 
 
 if __name__ == "__main__":

@@ -37,7 +37,7 @@ sg_status_t fail(sg_status_t st, const char* fmt, ...) {
     } while (0)
 
 // ------------------------------------------------------------------------------------------ per-device state
-__device__ uint32_t g_status_words[8];
+__device__ uint32_t g_status_words[8 + 32];   // 8 status words, then scratch for experimental time stamps
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -63,31 +63,41 @@ EncodeTiledFn g_encode_tiled = nullptr;
 EncodeIm2colFn g_encode_im2col = nullptr;
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_tune_tile_n{-1}, g_tune_pair{-1};
+thread_local int32_t t_last_plan[6] = {0, 0, 0, 0, 0, 0};   // tile_n, cta_pair, tail split, tile-list length, first split position, grid
 
 using KernelFn = void (*)(const Params);
 
 struct KernelEntry {
     KernelFn fn;
     int smem;
+    int threads;
 };
 
-template <int BN, bool kPair, bool kF32>
+template <int BN, bool kPair, bool kF32, int kEpiWarps>
 KernelEntry entry() {
-    return KernelEntry{contract_kernel<BN, kPair, kF32>, Config<BN, kPair>::SMEM_BYTES};
+    using Cfg = Config<BN, kPair, kEpiWarps>;
+    return KernelEntry{contract_kernel<BN, kPair, kF32, kEpiWarps>, Cfg::SMEM_BYTES, Cfg::THREADS};
 }
 
-// index: [bn_idx (64,128,256)][pair][f32]
-KernelEntry kernel_for(int bn, bool pair, bool f32) {
+template <int BN, int kEpiWarps>
+KernelEntry entry_for(bool pair, bool f32) {
+    return pair ? (f32 ? entry<BN, true, true, kEpiWarps>() : entry<BN, true, false, kEpiWarps>())
+                : (f32 ? entry<BN, false, true, kEpiWarps>() : entry<BN, false, false, kEpiWarps>());
+}
+
+// tile width (64, 128, 256) x CTA pairing x output type x number of epilogue warps (4 or 8)
+KernelEntry kernel_for(int bn, bool pair, bool f32, int epi_warps) {
+    if (epi_warps == 8) {
+        switch (bn) {
+            case 64: return entry_for<64, 8>(pair, f32);
+            case 128: return entry_for<128, 8>(pair, f32);
+            default: return entry_for<256, 8>(pair, f32);
+        }
+    }
     switch (bn) {
-        case 64:
-            return pair ? (f32 ? entry<64, true, true>() : entry<64, true, false>())
-                        : (f32 ? entry<64, false, true>() : entry<64, false, false>());
-        case 128:
-            return pair ? (f32 ? entry<128, true, true>() : entry<128, true, false>())
-                        : (f32 ? entry<128, false, true>() : entry<128, false, false>());
-        default:
-            return pair ? (f32 ? entry<256, true, true>() : entry<256, true, false>())
-                        : (f32 ? entry<256, false, true>() : entry<256, false, false>());
+        case 64: return entry_for<64, 4>(pair, f32);
+        case 128: return entry_for<128, 4>(pair, f32);
+        default: return entry_for<256, 4>(pair, f32);
     }
 }
 
@@ -134,17 +144,18 @@ sg_status_t device_state(DeviceState** out) {
             const int bns[3] = {64, 128, 256};
             for (int i = 0; i < 3 && d.init_status == SG_OK; ++i)
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
-                    for (int f32 = 0; f32 < 2 && d.init_status == SG_OK; ++f32) {
-                        KernelEntry k = kernel_for(bns[i], pair != 0, f32 != 0);
-                        e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
-                        if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
-                    }
+                    for (int f32 = 0; f32 < 2 && d.init_status == SG_OK; ++f32)
+                        for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4) {
+                            KernelEntry k = kernel_for(bns[i], pair != 0, f32 != 0, ew);
+                            e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
+                            if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
+                        }
             if (d.init_status == SG_OK) {
                 // how many 2-CTA clusters fit at once (some GPCs may not pair up all of their SMs)
-                KernelEntry k = kernel_for(256, true, false);
+                KernelEntry k = kernel_for(256, true, false, 8);
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(2 * d.sm_count);
-                cfg.blockDim = dim3(192);
+                cfg.blockDim = dim3(k.threads);
                 cfg.dynamicSmemBytes = k.smem;
                 cudaLaunchAttribute attr;
                 attr.id = cudaLaunchAttributeClusterDimension;
@@ -246,48 +257,93 @@ sg_status_t check_ptrs(const void* A, const void* B, const void* C, const void* 
 struct Shape {
     int bn;
     bool pair;
+    int epi_warps;
 };
 
-// Rough cost model: waves of tiles over the SMs times the tile's area, with a penalty for narrow
-// tiles (their MMAs are bound by shared-memory reads, not by the tensor pipe).
-Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N) {
+// Tile-shape choice.  Cost = waves of tiles over the SMs x tile width x a measured per-area factor
+// (wide two-CTA tiles move the fewest operand bytes per FLOP; narrow tiles are bound by shared-memory
+// and L2 reads, not by the tensor pipe).  Two-CTA tiles pay a fixed cluster set-up cost, so they are
+// used only when the K loop is long and there is at least one full wave of them.
+Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N,
+                   int64_t K) {
     const int force_bn = g_tune_tile_n.load();
     const int force_pair = g_tune_pair.load();
     const int bns[3] = {256, 128, 64};
-    const double narrow_penalty[3] = {1.0, 1.08, 1.5};
-    Shape best{256, false};
+    const double factor[2][3] = {{1.18, 1.30, 1.89}, {1.00, 1.26, 2.57}};   // [pair][bn index], relative time per output area
+    auto tiles_for = [&](int tile_m, int bn) {
+        int64_t tiles = 0;
+        for (int64_t r : rows_per_problem) tiles += ((r + tile_m - 1) / tile_m) * ((N + bn - 1) / bn);
+        return tiles * batch_mult;
+    };
+    const bool pair_worthwhile = K >= 1024 && d.max_pairs > 0 && tiles_for(256, 256) >= d.max_pairs;
+    // Eight epilogue warps drain an accumulator twice as fast; that pays when the K loop is too short to hide
+    // the epilogue (short K, heavy activations) and costs a little when it is long.
+    static const int forced_ew = getenv("SG_EPI_WARPS") ? atoi(getenv("SG_EPI_WARPS")) : 0;   // experiments: 4 or 8
+    const int epi_warps = (forced_ew == 4 || forced_ew == 8) ? forced_ew : (K <= 1024 ? 8 : 4);
+    Shape best{256, false, epi_warps};
     double best_cost = 1e300;
     for (int pi = 0; pi < 2; ++pi) {
-        if (force_pair >= 0 && pi != force_pair) continue;
-        if (force_pair < 0 && pi == 1) continue;            // pairs only on request until tuned per shape
+        if (force_pair >= 0 ? pi != force_pair : (pi == 1) != pair_worthwhile) continue;
         for (int bi = 0; bi < 3; ++bi) {
             const int bn = bns[bi];
             if (force_bn > 0 && bn != force_bn) continue;
-            if (pi == 1 && bn / 2 < 32) continue;
-            const int tile_m = pi ? 256 : 128;
-            int64_t tiles = 0;
-            for (int64_t r : rows_per_problem) tiles += ((r + tile_m - 1) / tile_m) * ((N + bn - 1) / bn);
-            tiles *= batch_mult;
+            const int64_t tiles = tiles_for(pi ? 256 : 128, bn);
             const int64_t slots = pi ? d.max_pairs : d.sm_count;
             const int64_t waves = (tiles + slots - 1) / slots;
-            const double cost = static_cast<double>(waves) * bn * narrow_penalty[bi] + 24.0;   // + fixed epilogue tail
+            // the K-independent part of a tile (pipeline fill, epilogue drain) weighs more when K is short
+            const double cost = static_cast<double>(waves) * bn * (factor[pi][bi] + 96.0 / static_cast<double>(K > 64 ? K : 64));
             if (cost < best_cost) {
                 best_cost = cost;
-                best = Shape{bn, pi != 0};
+                best = Shape{bn, pi != 0, epi_warps};
             }
         }
     }
     return best;
 }
 
+// Wave quantisation: when the tiles do not fill a whole number of waves, the tiles of the last wave are
+// cut into `split` column slices so that the idle SMs of that wave take a share.  Narrow slices cost more
+// per output area (same factors as in choose_shape), so a split is used only when it shortens the tail.
+// Sets p->split_begin, p->split and p->num_tiles (the length of the tile list) from the full-width count.
+void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params* p) {
+    const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
+    const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
+    int best_split = 1;
+    const int64_t rem = full_tiles % slots;
+    static const int forced = getenv("SG_TAIL_SPLIT") ? atoi(getenv("SG_TAIL_SPLIT")) : 0;   // experiments: 1, 2 or 4
+    if (rem != 0) {
+        double best = 1.0;      // cost of the unsplit tail wave, in units of one full-width tile
+        for (int k = 1; k <= 2; ++k) {
+            const int split = 1 << k;
+            if (s.bn / split < 64) break;
+            const int64_t waves = (rem * split + slots - 1) / slots;
+            const double cost = static_cast<double>(waves) / split * factor[s.pair ? 1 : 0][k];
+            if (cost < best - 0.05) {
+                best = cost;
+                best_split = split;
+            }
+        }
+        if (forced == 1 || forced == 2 || forced == 4) best_split = (s.bn / forced >= 64) ? forced : 1;
+    }
+    // raster bands: keep a band's A panels (band_m x TILE_M rows x K) within about 32 MB of L2
+    const int64_t panel_bytes = static_cast<int64_t>(s.pair ? 256 : 128) * (p->K > 0 ? p->K : 1) * 2;
+    int64_t band = (32ll << 20) / panel_bytes;
+    static const int forced_band = getenv("SG_BAND_M") ? atoi(getenv("SG_BAND_M")) : 0;   // experiments
+    if (forced_band > 0) band = forced_band;
+    p->band_m = static_cast<int32_t>(band < 1 ? 1 : (band > 4096 ? 4096 : band));
+    p->split = best_split;
+    p->split_begin = static_cast<int32_t>(best_split > 1 ? full_tiles - rem : full_tiles);
+    p->num_tiles = static_cast<int32_t>(best_split > 1 ? full_tiles - rem + rem * best_split : full_tiles);
+}
+
 sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params& p, cudaStream_t stream) {
-    KernelEntry k = kernel_for(s.bn, s.pair, f32);
+    KernelEntry k = kernel_for(s.bn, s.pair, f32, s.epi_warps);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;
     const int tiles = p.num_tiles < slots ? p.num_tiles : slots;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles * ctas_per_tile);
-    cfg.blockDim = dim3(192);
+    cfg.blockDim = dim3(k.threads);
     cfg.dynamicSmemBytes = k.smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr;
@@ -299,6 +355,12 @@ sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params&
     cfg.numAttrs = 1;
     SG_CUDA(cudaLaunchKernelEx(&cfg, k.fn, p));
     g_launches.fetch_add(1);
+    t_last_plan[0] = s.bn;
+    t_last_plan[1] = s.pair ? 1 : 0;
+    t_last_plan[2] = p.split;
+    t_last_plan[3] = p.num_tiles;
+    t_last_plan[4] = p.split_begin;
+    t_last_plan[5] = tiles * ctas_per_tile;
     return SG_OK;
 }
 
@@ -336,7 +398,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
 
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
-    const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N);
+    const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_DENSE;
     p.M = static_cast<int32_t>(desc->M);
@@ -346,8 +408,8 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.tiles_m = static_cast<int32_t>((desc->M + tile_m - 1) / tile_m);
     p.tiles_n = static_cast<int32_t>((desc->N + s.bn - 1) / s.bn);
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n * batch;
-    if (tiles > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
-    p.num_tiles = static_cast<int32_t>(tiles);
+    if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
+    plan_tail(*d, s, tiles, &p);
     p.num_kb = static_cast<int32_t>((desc->K + 63) / 64);
     p.bias = bias;
     p.C = desc->beta != 0.0f ? C : nullptr;
@@ -363,11 +425,14 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
         st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
                             s.pair ? s.bn / 2 : s.bn, "B");
         if (st != SG_OK) return st;
+        st = make_tiled_map(&p.tmB2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+                            (s.pair ? s.bn / 2 : s.bn) / p.split, "B (narrow)");
+        if (st != SG_OK) return st;
     }
     st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, D,
                         desc->N, desc->M, batch, desc->ldd, sD, c.f32_out ? 32 : 64, 32, "D");
     if (st != SG_OK) return st;
-    if (desc->K == 0) { p.tmA = p.tmD; p.tmB = p.tmD; }   // never used for loads; keeps the prefetch harmless
+    if (desc->K == 0) { p.tmA = p.tmD; p.tmB = p.tmD; p.tmB2 = p.tmD; }   // never used for loads; keeps the prefetch harmless
     return launch(*d, s, c.f32_out, p, static_cast<cudaStream_t>(stream));
 }
 
@@ -381,7 +446,7 @@ size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 GroupedLayout grouped_layout(int32_t groups) {
     GroupedLayout L;
     size_t o = 0;
-    L.off_maps = o;        o = round_up(o + static_cast<size_t>(groups) * 3 * sizeof(CUtensorMap), 128);
+    L.off_maps = o;        o = round_up(o + static_cast<size_t>(groups) * 4 * sizeof(CUtensorMap), 128);
     L.off_tile_start = o;  o = round_up(o + (static_cast<size_t>(groups) + 1) * 4, 128);
     L.off_M = o;           o = round_up(o + static_cast<size_t>(groups) * 4, 128);
     L.off_bias = o;        o = round_up(o + static_cast<size_t>(groups) * 8, 128);
@@ -438,6 +503,23 @@ const char* sg_status_string(sg_status_t s) {
 const char* sg_last_error(void) { return t_err; }
 
 int64_t sg_launch_count(void) { return g_launches.load(); }
+
+#ifdef SG_DEBUG_STAMPS
+sg_status_t sg_debug_stamps(uint64_t* out16) {
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    SG_CUDA(cudaDeviceSynchronize());
+    SG_CUDA(cudaMemcpy(out16, d->status_dev + 8, 16 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    return SG_OK;
+}
+#endif
+
+sg_status_t sg_last_launch_plan(int32_t* plan6) {
+    if (!plan6) return fail(SG_ERR_NULL_POINTER, "plan6 is NULL");
+    for (int i = 0; i < 6; ++i) plan6[i] = t_last_plan[i];
+    return SG_OK;
+}
 
 sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair) {
     if (tile_n != -1 && tile_n != 64 && tile_n != 128 && tile_n != 256) return fail(SG_ERR_INVALID_ARG, "tile_n must be -1, 64, 128 or 256");
@@ -500,9 +582,17 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     DeviceState* d = nullptr;
     st = device_state(&d);
     if (st != SG_OK) return st;
-    const Shape s = choose_shape(*d, rows, 1, common->N);
+    const Shape s = choose_shape(*d, rows, 1, common->N, common->K);
     const int tile_m = s.pair ? 256 : 128;
     const int tiles_n = static_cast<int>((common->N + s.bn - 1) / s.bn);
+
+    Params p;
+    base_params(&p, *d, common->alpha, common->beta, common->epi);
+    int64_t tiles = 0;
+    for (int g = 0; g < groups; ++g) tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
+    if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
+    p.K = static_cast<int32_t>(common->K);
+    plan_tail(*d, s, tiles, &p);
 
     std::vector<uint8_t> host(L.total, 0);
     CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(host.data() + L.off_maps);
@@ -511,7 +601,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     const void** gbias = reinterpret_cast<const void**>(host.data() + L.off_bias);
     const void** gC = reinterpret_cast<const void**>(host.data() + L.off_C);
     void** gD = reinterpret_cast<void**>(host.data() + L.off_D);
-    int64_t tiles = 0;
+    tiles = 0;
     for (int g = 0; g < groups; ++g) {
         tile_start[g] = static_cast<int32_t>(tiles);
         gM[g] = static_cast<int32_t>(rows[g]);
@@ -520,16 +610,19 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
         gD[g] = D_ptrs_host[g];
         if (rows[g] == 0) continue;
         tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
-        if (tiles > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
+        const uint32_t b_box = static_cast<uint32_t>(s.pair ? s.bn / 2 : s.bn);
         if (common->K > 0) {
-            st = make_tiled_map(&maps[3 * g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A_ptrs_host[g], common->K, rows[g], 1,
+            st = make_tiled_map(&maps[4 * g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A_ptrs_host[g], common->K, rows[g], 1,
                                 common->lda, 0, 64, 128, "A_g");
             if (st != SG_OK) return st;
-            st = make_tiled_map(&maps[3 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
-                                common->ldb, 0, 64, s.pair ? s.bn / 2 : s.bn, "B_g");
+            st = make_tiled_map(&maps[4 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                                common->ldb, 0, 64, b_box, "B_g");
+            if (st != SG_OK) return st;
+            st = make_tiled_map(&maps[4 * g + 3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                                common->ldb, 0, 64, b_box / p.split, "B_g (narrow)");
             if (st != SG_OK) return st;
         }
-        st = make_tiled_map(&maps[3 * g + 2], c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+        st = make_tiled_map(&maps[4 * g + 2], c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
                             c.esize_out, D_ptrs_host[g], common->N, rows[g], 1, common->ldd, 0, c.f32_out ? 32 : 64, 32, "D_g");
         if (st != SG_OK) return st;
     }
@@ -539,8 +632,6 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     st = upload(host, workspace_dev, stream);
     if (st != SG_OK) return st;
 
-    Params p;
-    base_params(&p, *d, common->alpha, common->beta, common->epi);
     uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
     p.mode = MODE_GROUPED;
     p.gmaps = reinterpret_cast<const CUtensorMap*>(ws + L.off_maps);
@@ -555,7 +646,6 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     p.K = static_cast<int32_t>(common->K);
     p.batch = groups;
     p.tiles_n = tiles_n;
-    p.num_tiles = static_cast<int32_t>(tiles);
     p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
     return launch(*d, s, c.f32_out, p, stream);
 }
@@ -593,7 +683,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     if (st != SG_OK) return st;
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
-    const Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K);
+    const Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_CONV;
     p.M = static_cast<int32_t>(Mg);
@@ -602,7 +692,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     p.batch = 1;
     p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
     p.tiles_n = static_cast<int32_t>((desc->K + s.bn - 1) / s.bn);
-    p.num_tiles = p.tiles_m * p.tiles_n;
+    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p);
     p.cblocks = static_cast<int32_t>((desc->C + 63) / 64);
     p.num_kb = static_cast<int32_t>(desc->R * desc->S) * p.cblocks;
     p.bias = bias;
@@ -644,6 +734,11 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
+        box[2] /= static_cast<cuuint32_t>(p.split);
+        r = g_encode_tiled(&p.tmB2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(Wf), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf, narrow) failed with CUresult %d", static_cast<int>(r));
     }
     st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, Y,
                         desc->K, Mg, 1, desc->K, 0, c.f32_out ? 32 : 64, 32, "Y");

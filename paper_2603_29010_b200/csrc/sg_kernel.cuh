@@ -28,7 +28,8 @@ enum : uint32_t { ROLE_PRODUCER = 1, ROLE_MMA = 2, ROLE_EPILOGUE = 3, ROLE_SETUP
 
 struct alignas(64) Params {
     CUtensorMap tmA, tmB, tmD;          // dense / batched / conv operands (3-D; conv A is a 4-D im2col map)
-    const CUtensorMap* gmaps;           // grouped: A_g, B_g, D_g maps at [3g], [3g+1], [3g+2]
+    CUtensorMap tmB2;                   // B with the narrower box of split tail tiles
+    const CUtensorMap* gmaps;           // grouped: A_g, B_g, D_g, B2_g maps at [4g] .. [4g+3]
     const int32_t* g_tile_start;        // grouped: first tile of group g, [groups + 1]
     const int32_t* g_M;                 // grouped: rows of group g
     const void* const* g_bias;          // grouped: per-group bias pointers (or null)
@@ -41,6 +42,8 @@ struct alignas(64) Params {
     int64_t ldc, strideC, strideBias;   // elements
     int32_t M, N, K, batch;             // batch = number of problems (dense) or groups (grouped)
     int32_t tiles_m, tiles_n, num_tiles, num_kb;
+    int32_t split_begin, split;         // tiles at list positions >= split_begin are 1/split-wide column slices
+    int32_t band_m;                     // raster: tiles are walked in bands of this many tile rows, column by column
     float alpha, beta;
     int32_t epi, mode;
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
@@ -48,33 +51,67 @@ struct alignas(64) Params {
     uint64_t timeout_ns;                // bound of every device-side wait
 };
 
+// Experiments only (-DSG_DEBUG_STAMPS): CTA `SG_DEBUG_STAMPS - 1` records globaltimer values at a few points of
+// its life into the words after the status words.
+#ifdef SG_DEBUG_STAMPS
+#define SG_STAMP(slot)                                                                           \
+    do {                                                                                         \
+        if (blockIdx.x == (SG_DEBUG_STAMPS - 1)) {                                               \
+            reinterpret_cast<volatile uint64_t*>(p.status + 8)[slot] = global_timer_ns();        \
+        }                                                                                        \
+    } while (0)
+#else
+#define SG_STAMP(slot) do {} while (0)
+#endif
+
 struct Tile {
-    int m0, n0, b, rows;   // first row / column, problem index, number of valid rows of the problem
+    int m0, n0, b, rows, width;   // first row / column, problem index, valid rows of the problem, tile width in columns
 };
 
-template <int TILE_M>
+// Tile r of one problem -> (tile row, tile column).  Tiles are walked in horizontal bands of band_m tile
+// rows; inside a band the walk goes down a column of the band, then to the next column.  The tiles running
+// at the same time then share few A and B panels, and a band's A rows stay in L2 while its columns stream by.
+__device__ __forceinline__ void raster(const Params& p, int r, int tiles_m, int& tm, int& tn) {
+    const int band_tiles = p.band_m * p.tiles_n;
+    const int band = r / band_tiles;
+    const int in_band = r - band * band_tiles;
+    const int band_rows = min(p.band_m, tiles_m - band * p.band_m);
+    tn = in_band / band_rows;
+    tm = band * p.band_m + (in_band - tn * band_rows);
+}
+
+// Position t of the tile list -> tile.  The list holds the full-width tiles of all complete waves first;
+// the tiles of the last, partial wave follow as `split` column slices each, so that more SMs share them.
+template <int TILE_M, int BN>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint) {
     Tile ti;
+    int sub = 0;
+    ti.width = BN;
+    if (t >= p.split_begin) {
+        const int u = t - p.split_begin;
+        const int parent = u / p.split;
+        sub = u - parent * p.split;
+        t = p.split_begin + parent;
+        ti.width = BN / p.split;
+    }
+    int tm, tn;
     if (p.mode == MODE_GROUPED) {
         int g = g_hint;
         while (t >= p.g_tile_start[g + 1]) ++g;      // tiles are visited in increasing order
         g_hint = g;
         const int rows = p.g_M[g];
-        const int tm = (rows + TILE_M - 1) / TILE_M;
-        const int r = t - p.g_tile_start[g];
         ti.b = g;
         ti.rows = rows;
-        ti.n0 = r / tm;
-        ti.m0 = (r - ti.n0 * tm) * TILE_M;
+        raster(p, t - p.g_tile_start[g], (rows + TILE_M - 1) / TILE_M, tm, tn);
     } else {
         const int per = p.tiles_m * p.tiles_n;
         ti.b = t / per;
-        const int r = t - ti.b * per;
-        ti.n0 = r / p.tiles_m;
-        ti.m0 = (r - ti.n0 * p.tiles_m) * TILE_M;
         ti.rows = p.M;
+        raster(p, t - ti.b * per, p.tiles_m, tm, tn);
     }
-    return ti;   // n0 still counts tiles: the caller scales it by the tile width
+    ti.m0 = tm * TILE_M;
+    ti.n0 = tn * BN + sub * ti.width;
+    return ti;
 }
 
 // Bounded mbarrier wait.  Returns false when the wait expired or another role already gave up.
@@ -104,12 +141,15 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Pa
     return wait_slow(bar, parity, p, role, tile, which);
 }
 
+// Activation of the fused epilogue, evaluated with one exp and one division (two special-function
+// operations per element; measured faster here than the single tanh.approx form), accurate to a few fp32 ulps:
+//   gelu(v) = 0.5 v (1 + tanh(u)) = v * sigmoid(2u),  u = sqrt(2/pi) (v + 0.044715 v^3)
+//   silu(v) = v * sigmoid(v)
 __device__ __forceinline__ float apply_act(float v, int epi) {
     switch (epi) {
         case EPI_RELU:
             return fmaxf(v, 0.0f);
         case EPI_GELU: {
-            // 0.5 v (1 + tanh(u)) == v * sigmoid(2u),  u = sqrt(2/pi) (v + 0.044715 v^3)
             const float u2 = 1.5957691216057308f * (v + 0.044715f * v * v * v);
             return __fdividef(v, 1.0f + __expf(-u2));
         }
@@ -120,7 +160,7 @@ __device__ __forceinline__ float apply_act(float v, int epi) {
     }
 }
 
-template <int BN, bool kPair>
+template <int BN, bool kPair, int kEpiWarps = 4>
 struct Config {
     static constexpr int kCtas = kPair ? 2 : 1;
     static constexpr int BM = 128;                 // rows per CTA (= TMEM lanes)
@@ -131,25 +171,32 @@ struct Config {
     static constexpr int B_BYTES = B_ROWS * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES_RAW = (192 * 1024) / STAGE_BYTES;
+#ifdef SG_MAX_STAGES
+    static constexpr int STAGES = STAGES_RAW > SG_MAX_STAGES ? SG_MAX_STAGES : STAGES_RAW;   // experiments only
+#else
     static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+#endif
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;   // BN in {64,128,256} -> power of two
-    static constexpr int STAGING_BYTES = 4 * 2 * 4096;             // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
+    static constexpr int EPI_WARPS = kEpiWarps;                    // 4: one per TMEM lane quarter; 8: two, alternating chunks
+    static constexpr int CHUNK_STEP = EPI_WARPS / 4;
+    static constexpr int STAGING_BUFS = 8 / EPI_WARPS;             // 32-row x 128-byte staging blocks per warp
+    static constexpr int STAGING_BYTES = 8 * 4096;
     static constexpr int OFF_STAGING = STAGES * STAGE_BYTES;
     static constexpr int OFF_BIAS = OFF_STAGING + STAGING_BYTES;
-    static constexpr int OFF_BAR = OFF_BIAS + 4 * BN * 2;                 // 4 epilogue warps x BN bf16 bias values
+    static constexpr int BIAS_SLOTS = BN / CHUNK_STEP < 64 ? 64 : BN / CHUNK_STEP;   // per warp: bf16 bias of its chunks
+    static constexpr int OFF_BAR = OFF_BIAS + EPI_WARPS * BIAS_SLOTS * 2;
     static constexpr int NUM_BARS = 2 * STAGES + 5;                // full, empty, tmem_full[2], tmem_empty[2], drain
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
-    static constexpr int THREADS = 192;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    static_assert(SMEM_BYTES <= 227 * 1024, "configuration exceeds the shared memory of one CTA");
 };
 
-template <int BN, bool kPair, bool kOutF32>
-__global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant__ Params p) {
-    using Cfg = Config<BN, kPair>;
+template <int BN, bool kPair, bool kOutF32, int kEpiWarps>
+__global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) contract_kernel(const __grid_constant__ Params p) {
+    using Cfg = Config<BN, kPair, kEpiWarps>;
     constexpr int kCtas = Cfg::kCtas;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int CH = kOutF32 ? 32 : 64;          // output columns per 128-byte staging row
-    constexpr int NCHUNK = BN / CH;
-    constexpr uint32_t IDESC = umma_idesc_bf16_f32(Cfg::TILE_M, BN);
 
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t smem_base = smem_u32(smem);
@@ -167,16 +214,23 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
     const uint32_t tmem_slot = bar_base + 8u * Cfg::NUM_BARS;
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem + Cfg::OFF_BAR + 8 * Cfg::NUM_BARS);
 
-    // A sticky failure from an earlier launch, or a misaligned dynamic shared-memory base: do nothing.
-    bool dead = (*reinterpret_cast<volatile uint32_t*>(p.status) != 0u);
+    if (threadIdx.x == 0) SG_STAMP(0);
+#ifdef SG_DEBUG_STAMPS
+    if (threadIdx.x == 32 && blockIdx.x == (SG_DEBUG_STAMPS - 1)) {
+        reinterpret_cast<volatile uint64_t*>(p.status + 8)[11] = clock64();
+        reinterpret_cast<volatile uint64_t*>(p.status + 8)[13] = global_timer_ns();
+    }
+#endif
+    // A sticky failure recorded by an earlier launch, or a misaligned dynamic shared-memory base, makes this
+    // launch a no-op.  The status word is fetched by one thread while the others set up, and the block-wide
+    // OR below doubles as the set-up barrier.  (Both CTAs of a pair decide alike: the word can only have been
+    // set by an earlier launch, and the base is the same in every CTA.)
+    uint32_t bad = 0;
+    if (threadIdx.x == 64) bad = *reinterpret_cast<volatile uint32_t*>(p.status);
     if ((smem_base & 1023u) != 0u) {
         if (threadIdx.x == 0) atomicCAS(p.status, 0u, (ROLE_SETUP << 24) | 1u);
-        dead = true;
+        bad = 1;
     }
-    // Both CTAs of a pair take the same decision: the word can only have been set by an earlier
-    // launch (a wait of this launch cannot expire this early), and the base is the same in every CTA.
-    if (dead) return;
-
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
@@ -184,7 +238,7 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 4 * kCtas);
+            mbar_init(tempty_bar(a), Cfg::EPI_WARPS * kCtas);
         }
         mbar_init(drain_bar, 1);
         fence_barrier_init();
@@ -199,19 +253,19 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
         prefetch_tensormap(&p.tmD);
     }
     tc_fence_before_sync();
+    const bool dead = __syncthreads_or(bad != 0u) != 0;
     if constexpr (kPair) {
         cluster_arrive();
         cluster_wait();
-    } else {
-        __syncthreads();
     }
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    if (threadIdx.x == 0) SG_STAMP(1);
 
     const int num_kb = p.num_kb;
     const int first_tile = blockIdx.x / kCtas;
     const int tile_step = gridDim.x / kCtas;
-    bool ok = true;
+    bool ok = !dead;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -220,19 +274,24 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
             uint32_t phase = 0;
             int g_hint = 0, g_fenced = -1;
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                Tile ti = decode_tile<Cfg::TILE_M>(p, t, g_hint);
+                Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
+                if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
-                const int nb0 = ti.n0 * BN + static_cast<int>(cta_rank) * Cfg::B_ROWS;
+                const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
+                const int nb0 = ti.n0 + static_cast<int>(cta_rank) * b_rows;
+                const uint32_t stage_tx = static_cast<uint32_t>(Cfg::A_BYTES + b_rows * Cfg::BK * 2) * kCtas;
+                const bool narrow = ti.width != BN;
                 const CUtensorMap* mapA = &p.tmA;
-                const CUtensorMap* mapB = &p.tmB;
+                const CUtensorMap* mapB = narrow ? &p.tmB2 : &p.tmB;
                 int bz = ti.b;
                 if (p.mode == MODE_GROUPED) {
-                    mapA = p.gmaps + 3 * ti.b;
-                    mapB = mapA + 1;
+                    mapA = p.gmaps + 4 * ti.b;
+                    mapB = mapA + (narrow ? 3 : 1);
                     bz = 0;
                     if (g_fenced != ti.b) {
                         fence_tensormap_acquire(mapA);
-                        fence_tensormap_acquire(mapB);
+                        fence_tensormap_acquire(mapA + 1);
+                        fence_tensormap_acquire(mapA + 3);
                         g_fenced = ti.b;
                     }
                 }
@@ -252,7 +311,7 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                     const uint32_t b_dst = a_dst + Cfg::A_BYTES;
                     uint32_t fb = full_bar(stage);
                     if constexpr (kPair) fb = map_to_cta(fb, 0);
-                    if (leader) mbar_arrive_expect_tx(full_bar(stage), Cfg::STAGE_BYTES * kCtas);
+                    if (leader) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
                     if (p.mode == MODE_CONV) {
                         const int tap = kb / p.cblocks;
                         const int c0 = (kb - tap * p.cblocks) * Cfg::BK;
@@ -266,8 +325,10 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                         tma_load_3d<kPair>(b_dst, mapB, fb, kb * Cfg::BK, nb0, bz);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    if (t == first_tile && kb == 0) SG_STAMP(2);
                 }
             }
+            SG_STAMP(3);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -276,14 +337,20 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
             int stage = 0;
             uint32_t phase = 0;
             int iter = 0;
-            for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step, ++iter) {
+            int g_hint = 0;
+            for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
+                const Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
+                if (ti.n0 >= p.N) continue;
+                const uint32_t idesc = umma_idesc_bf16_f32(Cfg::TILE_M, ti.width);
                 const int acc = iter & 1;
                 const uint32_t acc_phase = (iter >> 1) & 1u;
+                ++iter;
                 if (!wait_bar(tempty_bar(acc), acc_phase ^ 1u, p, ROLE_MMA, t, 100 + acc)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_bar(full_bar(stage), phase, p, ROLE_MMA, t, stage)) { ok = false; break; }
+                    if (t == first_tile && kb == 0) SG_STAMP(4);
                     tc_fence_after_sync();
                     const uint32_t a_src = smem_base + stage * Cfg::STAGE_BYTES;
                     const uint64_t a_desc = smem_desc_k_major_sw128(a_src);
@@ -291,14 +358,16 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
 #pragma unroll
                     for (int kk = 0; kk < Cfg::BK / 16; ++kk) {
                         // 16 bf16 along K = 32 bytes = 2 units of the descriptor's address field
-                        umma_bf16<kPair>(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, IDESC, (kb | kk) != 0 ? 1u : 0u);
+                        umma_bf16<kPair>(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
                     }
                     umma_commit<kPair>(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
                 umma_commit<kPair>(tfull_bar(acc));
+                if (t == first_tile) SG_STAMP(5);
             }
+            SG_STAMP(6);
             if (!ok) {
                 // let every MMA already issued finish before TMEM is freed
                 umma_commit<kPair>(drain_bar);
@@ -308,25 +377,32 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue warps 2..5
+        // ------------------------------------------------------------------ epilogue warps 2..9
+        // Two warps serve each TMEM lane quarter; the warp with half == 0 takes the even 128-byte column
+        // chunks of a tile, its partner the odd ones.
         const int q = warp & 3;               // TMEM lane quarter this warp may read
         const int ew = warp - 2;              // staging slot
-        uint16_t* bias_w = reinterpret_cast<uint16_t*>(smem + Cfg::OFF_BIAS) + ew * BN;   // this warp's bf16 copy
+        const int half = ew >> 2;             // which chunks of a tile this warp takes (always 0 with four warps)
+        constexpr int kStep = Cfg::CHUNK_STEP;
+        uint32_t chunk_ctr = 0;
+        uint16_t* bias_w = reinterpret_cast<uint16_t*>(smem + Cfg::OFF_BIAS) + ew * Cfg::BIAS_SLOTS;   // bf16 bias of its chunks
+        constexpr int kMyBiasSlots = ((BN / CH + kStep - 1) / kStep) * CH;     // columns of the chunks one warp handles
         const bool has_bias = (p.mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
         const bool has_c = (p.beta != 0.0f);
         const float alpha = p.alpha, beta = p.beta;
         const int epi = p.epi;
         int iter = 0, g_hint = 0, g_fenced = -1;
-        uint32_t chunk_ctr = 0;
         uint32_t tempty_remote[2];
 #pragma unroll
         for (int a = 0; a < 2; ++a) tempty_remote[a] = kPair ? map_to_cta(tempty_bar(a), 0) : tempty_bar(a);
 
-        for (int t = first_tile; t < p.num_tiles && ok; t += tile_step, ++iter) {
+        for (int t = first_tile; t < p.num_tiles && ok; t += tile_step) {
+            Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
+            if (ti.n0 >= p.N) continue;
             const int acc = iter & 1;
             const uint32_t acc_phase = (iter >> 1) & 1u;
-            Tile ti = decode_tile<Cfg::TILE_M>(p, t, g_hint);
-            const int n0 = ti.n0 * BN;
+            ++iter;
+            const int n0 = ti.n0;
             const int row0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32;
             const CUtensorMap* mapD = &p.tmD;
             const __nv_bfloat16* bias_g = reinterpret_cast<const __nv_bfloat16*>(p.bias);
@@ -334,7 +410,7 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
             uint8_t* d_g = reinterpret_cast<uint8_t*>(p.D);
             int bz = ti.b;
             if (p.mode == MODE_GROUPED) {
-                mapD = p.gmaps + 3 * ti.b + 2;
+                mapD = p.gmaps + 4 * ti.b + 2;
                 bz = 0;
                 if (has_bias) bias_g = reinterpret_cast<const __nv_bfloat16*>(p.g_bias[ti.b]);
                 if (has_c) c_g = reinterpret_cast<const uint8_t*>(p.g_C[ti.b]);
@@ -352,24 +428,38 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                 // every warp keeps its own copy of the tile's bias values, so no barrier between warps is needed
                 __syncwarp();
                 const uint16_t* bsrc = reinterpret_cast<const uint16_t*>(bias_g);
-                for (int i = lane; i < BN; i += 32) {
-                    const int n = n0 + i;
+                for (int i = lane; i < kMyBiasSlots; i += 32) {
+                    const int n = n0 + ((i / CH) * kStep + half) * CH + (i % CH);     // column of local slot i
                     bias_w[i] = (n < p.N) ? bsrc[n] : static_cast<uint16_t>(0);
                 }
                 __syncwarp();
             }
             if (num_kb > 0) {
-                if (!wait_bar(tfull_bar(acc), acc_phase, p, ROLE_EPILOGUE, t, 200 + acc)) { ok = false; break; }
+                // one lane polls; the other 31 wait at the warp barrier without issuing instructions
+                uint32_t done = 1;
+                if (lane == 0) done = wait_bar(tfull_bar(acc), acc_phase, p, ROLE_EPILOGUE, t, 200 + acc) ? 1u : 0u;
+                done = __shfl_sync(0xFFFFFFFFu, done, 0);
+                if (!done) { ok = false; break; }
                 tc_fence_after_sync();
+                if (warp == 2 && lane == 0 && t == first_tile) SG_STAMP(7);
             }
-            const int ncols = min(BN, p.N - n0);
+            const int ncols = min(ti.width, p.N - n0);
             const int nchunks = (ncols + CH - 1) / CH;
             const bool rows_live = row0 < ti.rows;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
             const int row = row0 + lane;
 
+            if (num_kb > 0 && half >= nchunks) {
+                // no chunk of this tile is this warp's: it still has to hand the accumulator back
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
+                    else mbar_arrive(tempty_remote[acc]);
+                }
+            }
 #pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
+            for (int c = half; c < nchunks; c += kStep) {
                 float v[CH];
                 if (num_kb > 0) {
                     uint32_t r0[32];
@@ -388,8 +478,8 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
                     }
-                    if (c == nchunks - 1) {
-                        // this accumulator buffer is drained: hand it back to the MMA warp
+                    if (c + kStep >= nchunks) {
+                        // this warp has read its last columns of the accumulator: hand its share back to the MMA warp
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) {
@@ -439,7 +529,7 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                 if (has_bias) {
 #pragma unroll
                     for (int i = 0; i < CH; i += 4) {
-                        const uint2 b2 = *reinterpret_cast<const uint2*>(bias_w + c * CH + i);   // 4 bf16, broadcast read
+                        const uint2 b2 = *reinterpret_cast<const uint2*>(bias_w + (c / kStep) * CH + i);   // 4 bf16, broadcast read
                         v[i] += __uint_as_float(b2.x << 16); v[i + 1] += __uint_as_float(b2.x & 0xFFFF0000u);
                         v[i + 2] += __uint_as_float(b2.y << 16); v[i + 3] += __uint_as_float(b2.y & 0xFFFF0000u);
                     }
@@ -467,12 +557,15 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                     continue;
                 }
 
+#if defined(SG_DEBUG_SKIP) && (SG_DEBUG_SKIP & 4)
+                if (v[0] != 12345.678f) continue;
+#endif
                 // stage the 32 x 128-byte block (row = lane) in the swizzled layout the store map expects
-                const uint32_t sb = chunk_ctr & 1u;
+                const uint32_t sb = chunk_ctr % Cfg::STAGING_BUFS;
                 ++chunk_ctr;
-                if (lane == 0) tma_store_wait_read<1>();     // the store that last read this buffer is done
+                if (lane == 0) tma_store_wait_read<Cfg::STAGING_BUFS - 1>();   // the store that last read this block is done
                 __syncwarp();
-                const uint32_t stg = smem_base + Cfg::OFF_STAGING + (ew * 2 + sb) * 4096u;
+                const uint32_t stg = smem_base + Cfg::OFF_STAGING + (ew * Cfg::STAGING_BUFS + sb) * 4096u;
                 const uint32_t row_addr = stg + lane * 128u;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -493,33 +586,42 @@ __global__ void __launch_bounds__(192, 1) contract_kernel(const __grid_constant_
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
+#if !(defined(SG_DEBUG_SKIP) && (SG_DEBUG_SKIP & 1))
                 if (lane == 0) {
                     tma_store_3d(mapD, stg, n0 + c * CH, row0, bz);
                     tma_store_commit();
                 }
+#endif
             }
         }
+        if (warp == 2 && lane == 0) SG_STAMP(8);
         if (lane == 0) tma_store_wait_all();
+        if (warp == 2 && lane == 0) SG_STAMP(9);
         __syncwarp();
     }
 
     // ---------------------------------------------------------------------- teardown
-    if (*reinterpret_cast<volatile uint32_t*>(p.status) != 0u) {
+    tc_fence_before_sync();
+    if (__syncthreads_or(!ok && !dead)) {
         // a wait expired somewhere: give copies still in flight time to land before the CTA retires
         const uint64_t t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
     }
-    tc_fence_before_sync();
     if constexpr (kPair) {
         cluster_arrive();
         cluster_wait();
-    } else {
-        __syncthreads();
     }
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc<kPair>(tmem_base, Cfg::TMEM_COLS);
     }
+    if (threadIdx.x == 32) SG_STAMP(10);
+#ifdef SG_DEBUG_STAMPS
+    if (threadIdx.x == 32 && blockIdx.x == (SG_DEBUG_STAMPS - 1)) {
+        reinterpret_cast<volatile uint64_t*>(p.status + 8)[12] = clock64();
+        reinterpret_cast<volatile uint64_t*>(p.status + 8)[14] = global_timer_ns();
+    }
+#endif
 }
 
 }  // namespace sg

@@ -20,10 +20,11 @@ import torch
 
 from .build import LIB_PATH
 
-if not os.path.exists(LIB_PATH):
-    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_29010_b200.build` "
+_LIB_FILE = os.environ.get("SOLGEMM_LIB", LIB_PATH)     # an experimental build may be selected explicitly
+if not os.path.exists(_LIB_FILE):
+    raise ImportError(f"{_LIB_FILE} is missing: build it with `python -m paper_2603_29010_b200.build` "
                       "(there is no CPU fallback)")
-_lib = ctypes.CDLL(LIB_PATH)
+_lib = ctypes.CDLL(_LIB_FILE)
 
 SG_OK = 0
 STATUS_NAMES = ["SG_OK", "SG_ERR_INVALID_ARG", "SG_ERR_NULL_POINTER", "SG_ERR_ALIGNMENT", "SG_ERR_UNSUPPORTED",
@@ -33,7 +34,8 @@ EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4}
 DTYPES = {torch.bfloat16: 0, torch.float32: 1}
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm", "sg_conv2d_fprop",
-            "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count"]
+            "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
+            "sg_last_launch_plan"]
 
 
 class SolgemmError(RuntimeError):
@@ -94,6 +96,8 @@ _lib.sg_poll_status.argtypes = [_vp]
 _lib.sg_set_tuning.restype = ctypes.c_int
 _lib.sg_set_tuning.argtypes = [_i32, _i32]
 _lib.sg_launch_count.restype = _i64
+_lib.sg_last_launch_plan.restype = ctypes.c_int
+_lib.sg_last_launch_plan.argtypes = [ctypes.POINTER(ctypes.c_int32)]
 
 
 def raw_lib() -> ctypes.CDLL:
@@ -280,3 +284,10 @@ def set_tuning(tile_n: int = -1, cta_pair: int = -1) -> None:
 
 def launch_count() -> int:
     return int(_lib.sg_launch_count())
+
+
+def last_launch_plan() -> dict:
+    """Tiling of this thread's most recent contraction launch (``sg_last_launch_plan``)."""
+    a = (ctypes.c_int32 * 6)()
+    _check(_lib.sg_last_launch_plan(a))
+    return dict(zip(("tile_n", "cta_pair", "tail_split", "tiles", "split_begin", "grid"), (int(x) for x in a)))

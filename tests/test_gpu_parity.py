@@ -37,13 +37,20 @@ def guarded(shape, dtype, pad_rows=8):
     """An output buffer with NaN guard bands before and after; returns (view, whole)."""
     rows, cols = shape[-2], shape[-1]
     lead = int(math.prod(shape[:-2])) if len(shape) > 2 else 1
-    whole = torch.full((lead * rows + 2 * pad_rows, cols), float("nan"), dtype=dtype, device=DEV)
-    view = whole[pad_rows:pad_rows + lead * rows].view(*shape)
-    return view, whole
+    if cols % 8 == 0:
+        whole = torch.full((lead * rows + 2 * pad_rows, cols), float("nan"), dtype=dtype, device=DEV)
+        view = whole[pad_rows:pad_rows + lead * rows].view(*shape)
+        return view, whole
+    assert len(shape) == 2                    # ragged width: pad the leading dimension to the 16-byte rule
+    whole = torch.full((rows + 2 * pad_rows, (cols + 15) // 8 * 8), float("nan"), dtype=dtype, device=DEV)
+    return whole[pad_rows:pad_rows + rows, :cols], whole
 
 
-def guards_intact(whole, pad_rows=8):
-    return bool(torch.isnan(whole[:pad_rows]).all() and torch.isnan(whole[-pad_rows:]).all())
+def guards_intact(whole, pad_rows=8, cols=None):
+    ok = bool(torch.isnan(whole[:pad_rows]).all() and torch.isnan(whole[-pad_rows:]).all())
+    if cols is not None and cols < whole.shape[1]:
+        ok = ok and bool(torch.isnan(whole[:, cols:]).all())
+    return ok
 
 
 SHAPES_EXACT = [(128, 64, 64), (256, 256, 256), (300, 200, 136), (129, 72, 8), (1000, 520, 328), (17, 8, 200),
@@ -93,6 +100,44 @@ def test_gemm_activation_form_is_pinned_on_the_fp32_path():
         ref, absacc = orc.gemm(a, b, epi=epi)
         D = sg.gemm(a.to(DEV), b.to(DEV), out_dtype=torch.float32, epi=epi)
         parity.assert_matches(D, ref, absacc, epi)
+
+
+@pytest.mark.parametrize("tile_n,pair,M,N,K", [(256, 0, 128 * 149, 200, 72), (256, 0, 128 * 149, 190, 72),
+                                              (256, 1, 256 * 75, 190, 136), (128, 0, 128 * 149, 136, 72),
+                                              (128, 1, 256 * 77, 100, 64)])
+def test_gemm_tail_wave_split_into_column_slices(tile_n, pair, M, N, K):
+    # one tile more than a whole number of waves: the planner cuts the last wave's tiles into narrower slices
+    sg.set_tuning(tile_n, pair)
+    A = inputs.small_integers([M, K], 313, 1)
+    B = inputs.small_integers([N, K], 313, 2)
+    ref, _ = orc.gemm(A, B)
+    D, whole = guarded((M, N), torch.bfloat16)
+    sg.gemm(A.to(DEV), B.to(DEV), out=D)
+    plan = sg.last_launch_plan()
+    assert plan["tail_split"] > 1 and plan["tiles"] > plan["split_begin"], plan
+    parity.assert_bit_exact(D, ref, f"tail split {plan}")
+    assert guards_intact(whole, cols=N)
+
+
+@pytest.mark.parametrize("out_dtype,N", [(torch.bfloat16, 90), (torch.float32, 90), (torch.float32, 67), (torch.bfloat16, 9)])
+def test_ragged_columns_never_touch_memory_past_n(out_dtype, N):
+    M, K = 150, 72
+    A, B = inputs.small_integers([M, K], 323, 1), inputs.small_integers([N, K], 323, 2)
+    ref, _ = orc.gemm(A, B)
+    ld = (N + 15) // 8 * 8
+    big = torch.full((M, ld), float("nan"), dtype=out_dtype, device=DEV)
+    sg.gemm(A.to(DEV), B.to(DEV), out=big[:, :N])
+    parity.assert_bit_exact(big[:, :N], ref, "ragged N")
+    assert bool(torch.isnan(big[:, N:]).all())
+    # the same through the batched and grouped entry points
+    bigb = torch.full((2, M, ld), float("nan"), dtype=out_dtype, device=DEV)
+    sg.batched_gemm(torch.stack([A, A]).to(DEV), torch.stack([B, B]).to(DEV), out=bigb[:, :, :N])
+    assert bool(torch.isnan(bigb[:, :, N:]).all())
+    parity.assert_bit_exact(bigb[1, :, :N], ref, "ragged N batched")
+    bigg = torch.full((M, ld), float("nan"), dtype=out_dtype, device=DEV)
+    sg.grouped_gemm([A.to(DEV)], [B.to(DEV)], outs=[bigg[:, :N]])
+    assert bool(torch.isnan(bigg[:, N:]).all())
+    parity.assert_bit_exact(bigg[:, :N], ref, "ragged N grouped")
 
 
 def test_gemm_leading_dimensions_and_k_tail():
@@ -206,6 +251,25 @@ def test_grouped_gemm_ragged_bit_exact(tile_n, pair):
     outs_p = sg.grouped_gemm([As[i].to(DEV) for i in perm], [Bs[i].to(DEV) for i in perm])
     for j, i in enumerate(perm):
         assert torch.equal(outs_p[j].cpu(), outs[i].cpu())
+
+
+def test_grouped_and_conv_tail_split():
+    sg.set_tuning(256, 0)
+    Ms = [128 * 100, 128 * 49, 77]                     # 150 tiles of 128 x 256: two more than a wave of 148
+    N, K = 200, 72
+    As = [inputs.small_integers([m, K], 818 + g, 1) for g, m in enumerate(Ms)]
+    Bs = [inputs.small_integers([N, K], 818 + g, 2) for g in range(len(Ms))]
+    refs, _ = orc.grouped_gemm(As, Bs)
+    outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs])
+    assert sg.last_launch_plan()["tail_split"] > 1
+    for g in range(len(Ms)):
+        parity.assert_bit_exact(outs[g], refs[g], f"group {g} with split tail")
+    X = inputs.small_integers([2, 100, 96, 16], 828, 6, -1, 1)
+    Wf = inputs.small_integers([256, 3, 3, 16], 828, 7, -1, 1)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1))
+    assert sg.last_launch_plan()["tail_split"] > 1
+    parity.assert_bit_exact(Y, ref, "conv with split tail")
 
 
 def test_grouped_gemm_epilogue_bias_and_c():

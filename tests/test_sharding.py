@@ -1,0 +1,73 @@
+"""Multi-GPU host logic on CPU: partitions are disjoint, cover everything, and are balanced.
+The two-rank test runs real processes over the gloo backend and cross-checks the ranks' shards."""
+import os
+import socket
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2603_29010_b200 import inputs, sharding
+
+
+@pytest.mark.parametrize("total,world,multiple", [(4096, 8, 128), (100352, 8, 128), (1000, 3, 128), (5, 8, 1), (0, 2, 128),
+                                                  (129, 2, 128)])
+def test_split_range_covers_disjointly(total, world, multiple):
+    cuts = [sharding.split_range(total, world, r, multiple) for r in range(world)]
+    assert cuts[0][0] == 0 and cuts[-1][1] == total
+    for (b0, e0), (b1, e1) in zip(cuts, cuts[1:]):
+        assert e0 == b1 and b0 <= e0
+    for b, e in cuts[:-1]:
+        assert b % multiple == 0 and (e % multiple == 0 or e == total)
+    sizes = [-(-(e - b) // multiple) for b, e in cuts]
+    assert max(sizes) - min(sizes) <= 1
+
+
+def test_group_assignment_is_balanced_and_complete():
+    Ms = inputs.grouped_sizes(16, 128, 4096)
+    for world in (1, 2, 4, 8):
+        owned = sharding.assign_groups(Ms, world)
+        assert sorted(g for lst in owned for g in lst) == list(range(16))
+        loads = [sum(Ms[g] for g in lst) for lst in owned]
+        assert max(loads) - min(loads) <= max(Ms)
+    assert sharding.assign_groups([], 2) == [[], []]
+    with pytest.raises(ValueError):
+        sharding.split_range(10, 0, 0)
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, M, batch, Ms):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        rows = sharding.gemm_rows(M, world, rank)
+        bat = sharding.batch_entries(batch, world, rank)
+        groups = sharding.assign_groups(Ms, world)[rank]
+        # mark what this rank owns; the sum over ranks must be exactly one everywhere
+        own_rows = torch.zeros(M, dtype=torch.int64)
+        own_rows[rows[0]:rows[1]] = 1
+        own_batch = torch.zeros(batch, dtype=torch.int64)
+        own_batch[bat[0]:bat[1]] = 1
+        own_groups = torch.zeros(len(Ms), dtype=torch.int64)
+        own_groups[groups] = 1
+        for t in (own_rows, own_batch, own_groups):
+            dist.all_reduce(t)
+            assert bool((t == 1).all())
+        # weak-scaling bookkeeping of the benchmark: the job's time is the slowest rank's
+        t = torch.tensor([1.0 + rank], dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        assert float(t) == float(world)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_partition_every_operation_over_gloo():
+    world = 2
+    Ms = inputs.grouped_sizes(16, 128, 4096)
+    mp.spawn(_worker, args=(world, _free_port(), 4096, 128, Ms), nprocs=world, join=True)
