@@ -120,6 +120,29 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
                             void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * sg_grouped_gemm_static: sg_grouped_gemm for callers that cannot provide a workspace because they cannot
+ * allocate device memory at all -- for example code that runs after its process has handed the whole GPU to
+ * a memory pool it may not draw from, or a latency-critical path where cudaMalloc (which may synchronise the
+ * device) is forbidden.  (The paper has no counterpart: its generated wrappers allocate their workspace.)
+ *   The per-group tensor maps and the tile table go into a fixed scratch array that is part of the library
+ *   image (about 36 KB of device memory on every GPU that loads the library, held until the process exits),
+ *   so the call takes no workspace arguments and performs no device allocation of any kind.  Inputs and
+ *   outputs are still the caller's buffers; all other arguments and the result are those of sg_grouped_gemm.
+ *   groups > SG_STATIC_MAX_GROUPS           -> SG_ERR_WORKSPACE, nothing is launched.
+ *   The first call on a device looks up the array's device address (once per device, with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls on a device share the one array and it keeps the previous call's tables until they are
+ *   overwritten: every call rewrites all entries it uses before its kernel reads them, but two calls whose
+ *   work overlaps on the GPU (different streams, or the same stream from two threads) race on it.  Serialise
+ *   such calls or use sg_grouped_gemm with separate workspaces.
+ */
+#define SG_STATIC_MAX_GROUPS 64
+sg_status_t sg_grouped_gemm_static(const sg_gemm_desc_t* common, int32_t groups, const int64_t* M_host,
+                                   const void* const* A_ptrs_host, const void* const* B_ptrs_host,
+                                   const void* const* C_ptrs_host, const void* const* bias_ptrs_host,
+                                   void* const* D_ptrs_host, void* cuda_stream);
+
+/*
  * One forward convolution (cross-correlation, groups = 1), tensors in the paper's TensorNHWC
  * layout (Table 1a "Conv2d ... NHWC"; Appendix A.1 conv2d_fprop(kernel_h=R, kernel_w=S)):
  *   X [N,H,W,C], Wf [K,R,S,C], Y and Cin [N,P,Q,K], bias [K], all contiguous;

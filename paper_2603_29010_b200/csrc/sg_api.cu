@@ -650,6 +650,44 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     return launch(*d, s, c.f32_out, p, stream);
 }
 
+// ---- grouped GEMM without any device allocation by anyone -----------------------------------------------
+// Scratch for the tensor maps and tile table of up to SG_STATIC_MAX_GROUPS groups.  In host code this name is
+// only a handle for the runtime: the address a kernel can use comes from cudaGetSymbolAddress, per device.
+constexpr size_t kStaticWsBytes = 36 * 1024;
+static __device__ __align__(256) unsigned char g_static_grouped_ws[kStaticWsBytes];
+static void* g_static_ws_ptr[kMaxDevices] = {nullptr};
+
+sg_status_t sg_grouped_gemm_static(const sg_gemm_desc_t* common, int32_t groups, const int64_t* M_host,
+                                   const void* const* A_ptrs_host, const void* const* B_ptrs_host,
+                                   const void* const* C_ptrs_host, const void* const* bias_ptrs_host,
+                                   void* const* D_ptrs_host, void* cuda_stream) {
+    if (groups > SG_STATIC_MAX_GROUPS)
+        return fail(SG_ERR_WORKSPACE, "sg_grouped_gemm_static: %d groups exceed the built-in scratch for %d groups; "
+                    "use sg_grouped_gemm with a caller-provided workspace", groups, SG_STATIC_MAX_GROUPS);
+    if (groups > 0 && grouped_layout(groups).total > kStaticWsBytes)
+        return fail(SG_ERR_WORKSPACE, "sg_grouped_gemm_static: internal scratch too small for %d groups", groups);
+    int dev = 0;
+    SG_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(SG_ERR_CUDA, "device index %d out of range", dev);
+    void* ws = nullptr;
+    {
+        // first call on this device: resolve the device address of the scratch array (the current device is `dev`)
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!g_static_ws_ptr[dev]) {
+            void* ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_grouped_ws);
+            if (e != cudaSuccess || !ptr)
+                return fail(SG_ERR_CUDA, "cudaGetSymbolAddress(static scratch): %s", cudaGetErrorString(e));
+            g_static_ws_ptr[dev] = ptr;
+        }
+        ws = g_static_ws_ptr[dev];
+    }
+    // Every table entry the kernel reads is rewritten by this call's stream-ordered upload, so nothing left by
+    // an earlier call can be seen; the existing entry point does the rest and allocates no device memory.
+    return sg_grouped_gemm(common, groups, M_host, A_ptrs_host, B_ptrs_host, C_ptrs_host, bias_ptrs_host, D_ptrs_host, ws,
+                           kStaticWsBytes, cuda_stream);
+}
+
 sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const void* Wf, const void* Cin, const void* bias,
                             void* Y, void* cuda_stream) {
     if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");

@@ -33,7 +33,8 @@ LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4}
 DTYPES = {torch.bfloat16: 0, torch.float32: 1}
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
-EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm", "sg_conv2d_fprop",
+EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
+            "sg_grouped_gemm_static", "sg_conv2d_fprop",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan"]
 
@@ -84,6 +85,8 @@ _lib.sg_grouped_gemm_workspace_size.restype = ctypes.c_int
 _lib.sg_grouped_gemm_workspace_size.argtypes = [_i32, ctypes.POINTER(ctypes.c_size_t)]
 _lib.sg_grouped_gemm.restype = ctypes.c_int
 _lib.sg_grouped_gemm.argtypes = [ctypes.POINTER(GemmDesc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]
+_lib.sg_grouped_gemm_static.restype = ctypes.c_int
+_lib.sg_grouped_gemm_static.argtypes = [ctypes.POINTER(GemmDesc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_conv2d_fprop.restype = ctypes.c_int
 _lib.sg_conv2d_fprop.argtypes = [ctypes.POINTER(Conv2dDesc), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sol_bound.restype = ctypes.c_int
@@ -207,6 +210,32 @@ def grouped_gemm(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=N
     _check(_lib.sg_grouped_gemm(ctypes.byref(desc), groups, m_arr, _ptr_array(As), _ptr_array(Bs), _ptr_array(Cs),
                                 _ptr_array(biases), _ptr_array(outs), _ptr(workspace), workspace.numel(),
                                 _stream(stream)))
+    return list(outs)
+
+
+STATIC_MAX_GROUPS = 64
+
+
+def grouped_gemm_static(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=None, biases=None,
+                        outs: Sequence[torch.Tensor], alpha=1.0, beta=0.0, epi="none", layout_a="row", layout_b="col",
+                        stream=None) -> List[torch.Tensor]:
+    """``sg_grouped_gemm_static``: the grouped product for callers that may not allocate device memory.
+
+    Unlike :func:`grouped_gemm` this wrapper allocates nothing either: ``outs`` must be given, and the
+    library keeps its tables in a scratch array built into its image (at most ``STATIC_MAX_GROUPS``
+    groups).  Calls on one device share that array, so calls that overlap on the GPU must be serialised.
+    """
+    groups = len(As)
+    if groups == 0:
+        return []
+    _, N, K = _mnk(As[0], Bs[0], layout_a, layout_b)
+    Ms = [(_mnk(a, b, layout_a, layout_b))[0] for a, b in zip(As, Bs)]
+    ld = lambda ts, default: next((_ld(t) for t in ts if t.shape[0] > 1), default)
+    desc = _gemm_desc(0, N, K, ld(As, max(K, 1)), ld(Bs, max(K, 1)), ld(Cs, max(N, 1)) if Cs is not None else max(N, 1),
+                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi)
+    m_arr = (ctypes.c_int64 * groups)(*Ms)
+    _check(_lib.sg_grouped_gemm_static(ctypes.byref(desc), groups, m_arr, _ptr_array(As), _ptr_array(Bs),
+                                       _ptr_array(Cs), _ptr_array(biases), _ptr_array(outs), _stream(stream)))
     return list(outs)
 
 
