@@ -219,13 +219,35 @@ sg_status_t sg_poll_status(void* cuda_stream);
  */
 sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair);
 
+/*
+ * sg_set_tail_mode: how the tiles of the last, partial wave are shared between SMs (tuning / tests):
+ *   -1 let the planner decide (default), 0 leave them whole, 1 cut them into column slices,
+ *    2 cut their K loop into ranges exchanged through the scratch (needs sg_set_scratch; else as 1).
+ */
+sg_status_t sg_set_tail_mode(int32_t mode);
+
+/*
+ * sg_set_scratch: lends the library a device buffer (current device) that later contraction calls may use to
+ * balance their last, partial wave of tiles: several SM groups then share one output tile's K loop and exchange
+ * fp32 partial sums through the buffer ("stream-K" for the tail; paper: scheduler tile=stream_k, Appendix A.1).
+ * Optional: without a scratch the tail tiles are cut into column slices instead, and results are the same up to
+ * fp32 summation order.  (As measured so far the exchange costs about as much as it saves, so the planner
+ * prefers column slices; sg_set_tail_mode(2) forces the K ranges.)  256-byte aligned; SG_SCRATCH_BYTES_RECOMMENDED covers every shape; the first 8 KB are
+ * cleared synchronously by this call.  The caller keeps ownership and must keep the buffer alive and untouched
+ * until it calls sg_set_scratch(NULL, 0).  All calls on the device share it: work that overlaps on the GPU
+ * (several streams) must not use it concurrently -- unregister it, or serialise such calls.
+ */
+#define SG_SCRATCH_BYTES_RECOMMENDED (32u << 20)
+sg_status_t sg_set_scratch(void* scratch_dev, size_t bytes);
+
 /* Number of kernel launches this library has enqueued from this process (monotonic). */
 int64_t sg_launch_count(void);
 
 /*
  * How the calling thread's most recent contraction launch was tiled, for tests and benchmark records:
  *   plan6[0] tile width in columns, [1] 1 for two-CTA tiles, [2] tail split (the tiles of the last,
- *   partial wave are cut into this many column slices; 1 = none), [3] length of the tile list,
+ *   partial wave are cut into this many column slices; 1 = none; a negative value -k means they are
+ *   cut into k ranges of the K loop through the scratch instead), [3] length of the tile list,
  *   [4] list position of the first slice, [5] grid size in CTAs.
  */
 sg_status_t sg_last_launch_plan(int32_t* plan6);

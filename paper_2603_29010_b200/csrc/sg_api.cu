@@ -54,7 +54,12 @@ struct DeviceState {
     int sm_count = 0;
     int max_pairs = 0;               // CTA pairs that can be resident at once
     uint32_t* status_dev = nullptr;  // device address of g_status_words on this device
+    void* scratch = nullptr;         // caller-registered scratch for K-split tail tiles (sg_set_scratch)
+    size_t scratch_bytes = 0;
 };
+
+constexpr size_t kScratchFlagBytes = 8192;     // 1024 arrival counters + 1024 consumed counters
+constexpr int kScratchMaxBuffers = 1024;
 
 constexpr int kMaxDevices = 64;
 DeviceState g_dev[kMaxDevices];
@@ -62,7 +67,7 @@ std::mutex g_mutex;
 EncodeTiledFn g_encode_tiled = nullptr;
 EncodeIm2colFn g_encode_im2col = nullptr;
 std::atomic<int64_t> g_launches{0};
-std::atomic<int> g_tune_tile_n{-1}, g_tune_pair{-1};
+std::atomic<int> g_tune_tile_n{-1}, g_tune_pair{-1}, g_tune_tail{-1};
 thread_local int32_t t_last_plan[6] = {0, 0, 0, 0, 0, 0};   // tile_n, cta_pair, tail split, tile-list length, first split position, grid
 
 using KernelFn = void (*)(const Params);
@@ -308,10 +313,13 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
 void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params* p) {
     const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
-    int best_split = 1;
+    int best_split = 1, best_ksplit = 1;
     const int64_t rem = full_tiles % slots;
     static const int forced = getenv("SG_TAIL_SPLIT") ? atoi(getenv("SG_TAIL_SPLIT")) : 0;   // experiments: 1, 2 or 4
-    if (rem != 0) {
+    static const int env_k = getenv("SG_TAIL_KSPLIT") ? atoi(getenv("SG_TAIL_KSPLIT")) : -1;   // experiments: 0 = off
+    const int tail_mode = g_tune_tail.load();      // -1 auto, 0 none, 1 column slices, 2 K ranges
+    const int forced_k = tail_mode == 2 ? 4 : (tail_mode == 0 || tail_mode == 1 ? 0 : env_k);
+    if (rem != 0 && tail_mode != 0) {
         double best = 1.0;      // cost of the unsplit tail wave, in units of one full-width tile
         for (int k = 1; k <= 2; ++k) {
             const int split = 1 << k;
@@ -323,7 +331,28 @@ void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params*
                 best_split = split;
             }
         }
-        if (forced == 1 || forced == 2 || forced == 4) best_split = (s.bn / forced >= 64) ? forced : 1;
+        if (forced == 1 || forced == 2 || forced == 4) {
+            best_split = (s.bn / forced >= 64) ? forced : 1;
+            best = 0.9;
+        }
+        // K-split through the registered scratch: ksplit SM groups share one tail tile's K loop; the owner adds the
+        // helpers' fp32 partial tiles in its epilogue.  Costs the partials' round trip through L2 (~0.1 tile).
+        if (d.scratch && forced_k != 0 && p->num_kb >= 2 && rem * 2 <= slots) {
+            int64_t ks = slots / rem;
+            if (ks > 4) ks = 4;
+            if (ks > p->num_kb) ks = p->num_kb;
+            if (forced_k >= 2 && forced_k <= ks) ks = forced_k;
+            const size_t buf_bytes = static_cast<size_t>(s.pair ? 2 : 1) * 128 * s.bn * sizeof(float);
+            size_t max_buffers = d.scratch_bytes > kScratchFlagBytes ? (d.scratch_bytes - kScratchFlagBytes) / buf_bytes : 0;
+            if (max_buffers > static_cast<size_t>(kScratchMaxBuffers)) max_buffers = kScratchMaxBuffers;
+            // measured: helpers' dump, the owner's wait and its reads of the partials cost about 0.45 of a tile
+            const double cost = 1.0 / static_cast<double>(ks) + 0.45;
+            if (ks >= 2 && static_cast<size_t>(rem * (ks - 1)) <= max_buffers && rem <= kScratchMaxBuffers &&
+                (cost < best - 0.05 || forced_k >= 2)) {
+                best_ksplit = static_cast<int>(ks);
+                best_split = 1;
+            }
+        }
     }
     // raster bands: keep a band's A panels (band_m x TILE_M rows x K) within about 32 MB of L2
     const int64_t panel_bytes = static_cast<int64_t>(s.pair ? 256 : 128) * (p->K > 0 ? p->K : 1) * 2;
@@ -331,9 +360,17 @@ void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params*
     static const int forced_band = getenv("SG_BAND_M") ? atoi(getenv("SG_BAND_M")) : 0;   // experiments
     if (forced_band > 0) band = forced_band;
     p->band_m = static_cast<int32_t>(band < 1 ? 1 : (band > 4096 ? 4096 : band));
+    const int parts = best_ksplit > 1 ? best_ksplit : best_split;
     p->split = best_split;
-    p->split_begin = static_cast<int32_t>(best_split > 1 ? full_tiles - rem : full_tiles);
-    p->num_tiles = static_cast<int32_t>(best_split > 1 ? full_tiles - rem + rem * best_split : full_tiles);
+    p->ksplit = best_ksplit;
+    p->split_begin = static_cast<int32_t>(parts > 1 ? full_tiles - rem : full_tiles);
+    p->num_tiles = static_cast<int32_t>(parts > 1 ? full_tiles - rem + rem * parts : full_tiles);
+    if (best_ksplit > 1) {
+        p->sk_flags = static_cast<uint32_t*>(d.scratch);
+        p->sk_consumed_off = kScratchMaxBuffers;
+        p->sk_partials = reinterpret_cast<float*>(static_cast<uint8_t*>(d.scratch) + kScratchFlagBytes);
+        p->sk_arrivals = s.epi_warps * (s.pair ? 2 : 1);
+    }
 }
 
 sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params& p, cudaStream_t stream) {
@@ -357,7 +394,7 @@ sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params&
     g_launches.fetch_add(1);
     t_last_plan[0] = s.bn;
     t_last_plan[1] = s.pair ? 1 : 0;
-    t_last_plan[2] = p.split;
+    t_last_plan[2] = p.ksplit > 1 ? -p.ksplit : p.split;
     t_last_plan[3] = p.num_tiles;
     t_last_plan[4] = p.split_begin;
     t_last_plan[5] = tiles * ctas_per_tile;
@@ -409,8 +446,8 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.tiles_n = static_cast<int32_t>((desc->N + s.bn - 1) / s.bn);
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n * batch;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
-    plan_tail(*d, s, tiles, &p);
     p.num_kb = static_cast<int32_t>((desc->K + 63) / 64);
+    plan_tail(*d, s, tiles, &p);
     p.bias = bias;
     p.C = desc->beta != 0.0f ? C : nullptr;
     p.ldc = desc->ldc;
@@ -515,6 +552,23 @@ sg_status_t sg_debug_stamps(uint64_t* out16) {
 }
 #endif
 
+sg_status_t sg_set_scratch(void* scratch_dev, size_t bytes) {
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    if (!scratch_dev || bytes == 0) {
+        d->scratch = nullptr;
+        d->scratch_bytes = 0;
+        return SG_OK;
+    }
+    if (reinterpret_cast<uintptr_t>(scratch_dev) & 255u) return fail(SG_ERR_WORKSPACE, "sg_set_scratch: scratch must be 256-byte aligned");
+    if (bytes < kScratchFlagBytes + (1u << 20)) return fail(SG_ERR_WORKSPACE, "sg_set_scratch: at least %zu bytes are needed", kScratchFlagBytes + (1u << 20));
+    SG_CUDA(cudaMemset(scratch_dev, 0, kScratchFlagBytes));      // counters start at zero (synchronous)
+    d->scratch = scratch_dev;
+    d->scratch_bytes = bytes;
+    return SG_OK;
+}
+
 sg_status_t sg_last_launch_plan(int32_t* plan6) {
     if (!plan6) return fail(SG_ERR_NULL_POINTER, "plan6 is NULL");
     for (int i = 0; i < 6; ++i) plan6[i] = t_last_plan[i];
@@ -526,6 +580,12 @@ sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair) {
     if (cta_pair < -1 || cta_pair > 1) return fail(SG_ERR_INVALID_ARG, "cta_pair must be -1, 0 or 1");
     g_tune_tile_n.store(tile_n);
     g_tune_pair.store(cta_pair);
+    return SG_OK;
+}
+
+sg_status_t sg_set_tail_mode(int32_t mode) {
+    if (mode < -1 || mode > 2) return fail(SG_ERR_INVALID_ARG, "tail mode must be -1 (auto), 0, 1 or 2");
+    g_tune_tail.store(mode);
     return SG_OK;
 }
 
@@ -592,6 +652,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     for (int g = 0; g < groups; ++g) tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
     p.K = static_cast<int32_t>(common->K);
+    p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
     plan_tail(*d, s, tiles, &p);
 
     std::vector<uint8_t> host(L.total, 0);
@@ -730,9 +791,9 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     p.batch = 1;
     p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
     p.tiles_n = static_cast<int32_t>((desc->K + s.bn - 1) / s.bn);
-    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p);
     p.cblocks = static_cast<int32_t>((desc->C + 63) / 64);
     p.num_kb = static_cast<int32_t>(desc->R * desc->S) * p.cblocks;
+    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p);
     p.bias = bias;
     p.C = desc->beta != 0.0f ? Cin : nullptr;
     p.ldc = desc->K;
@@ -794,6 +855,7 @@ sg_status_t sg_poll_status(void* cuda_stream) {
     SG_CUDA(cudaStreamSynchronize(stream));
     if (words[0] == 0) return SG_OK;
     SG_CUDA(cudaMemsetAsync(d->status_dev, 0, sizeof words, stream));
+    if (d->scratch) SG_CUDA(cudaMemsetAsync(d->scratch, 0, kScratchFlagBytes, stream));   // an aborted K-split may leave counters set
     SG_CUDA(cudaStreamSynchronize(stream));
     static const char* roles[] = {"?", "producer", "mma", "epilogue", "setup"};
     const uint32_t role = words[0] >> 24;

@@ -44,6 +44,11 @@ struct alignas(64) Params {
     int32_t tiles_m, tiles_n, num_tiles, num_kb;
     int32_t split_begin, split;         // tiles at list positions >= split_begin are 1/split-wide column slices
     int32_t band_m;                     // raster: tiles are walked in bands of this many tile rows, column by column
+    int32_t ksplit;                     // > 1: tail tiles are cut into this many K ranges instead (split is then 1)
+    int32_t sk_arrivals;                // warp arrivals that complete one helper's partial tile (epilogue warps x CTAs)
+    float* sk_partials;                 // K-split scratch: [tail tile][helper][CTA of the tile][128 rows][BN] fp32
+    uint32_t* sk_flags;                 // K-split scratch: [buffer] arrival counters, then [tail tile] consumed counters
+    int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
     float alpha, beta;
     int32_t epi, mode;
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
@@ -66,6 +71,8 @@ struct alignas(64) Params {
 
 struct Tile {
     int m0, n0, b, rows, width;   // first row / column, problem index, valid rows of the problem, tile width in columns
+    int kb0, kb1;                 // k-blocks [kb0, kb1) this work item contracts (the whole K unless the tile is K-split)
+    int part, nparts, tail;       // K-split: part 0 owns (finishes) the tile, parts 1.. help; index of the tail tile
 };
 
 // Tile r of one problem -> (tile row, tile column).  Tiles are walked in horizontal bands of band_m tile
@@ -87,12 +94,28 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
     Tile ti;
     int sub = 0;
     ti.width = BN;
+    ti.kb0 = 0;
+    ti.kb1 = p.num_kb;
+    ti.part = 0;
+    ti.nparts = 1;
+    ti.tail = 0;
     if (t >= p.split_begin) {
         const int u = t - p.split_begin;
-        const int parent = u / p.split;
-        sub = u - parent * p.split;
-        t = p.split_begin + parent;
-        ti.width = BN / p.split;
+        if (p.ksplit > 1) {
+            // the tile's K range is shared by ksplit work items: part 0 owns the tile, the others help
+            ti.nparts = p.ksplit;
+            ti.tail = u / p.ksplit;
+            ti.part = u - ti.tail * p.ksplit;
+            t = p.split_begin + ti.tail;
+            const int base = p.num_kb / p.ksplit, extra = p.num_kb - base * p.ksplit;
+            ti.kb0 = ti.part * base + min(ti.part, extra);
+            ti.kb1 = ti.kb0 + base + (ti.part < extra ? 1 : 0);
+        } else {
+            const int parent = u / p.split;
+            sub = u - parent * p.split;
+            t = p.split_begin + parent;
+            ti.width = BN / p.split;
+        }
     }
     int tm, tn;
     if (p.mode == MODE_GROUPED) {
@@ -158,6 +181,30 @@ __device__ __forceinline__ float apply_act(float v, int epi) {
         default:
             return v;
     }
+}
+
+// Bounded wait until a global arrival counter (written by another CTA of this launch with a release pattern)
+// reaches `target`.  Returns false when the wait expired or another role already gave up.
+__device__ __noinline__ bool wait_counter(const uint32_t* counter, uint32_t target, const Params& p, uint32_t tile) {
+    const volatile uint32_t* c = counter;
+    volatile uint32_t* st = p.status;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t it = 0;
+    while (*c < target) {
+        __nanosleep(64);
+        if ((++it & 63u) == 0) {
+            if (st[0] != 0) return false;
+            if (global_timer_ns() - t0 > p.timeout_ns) {
+                if (atomicCAS(p.status, 0u, (ROLE_EPILOGUE << 24) | 300u) == 0u) {
+                    st[1] = tile;
+                    st[2] = *c;
+                    st[3] = blockIdx.x;
+                }
+                return false;
+            }
+        }
+    }
+    return true;
 }
 
 template <int BN, bool kPair, int kEpiWarps = 4>
@@ -305,7 +352,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     cw = oq * p.stride_w - p.pad_w;
                     ch = op * p.stride_h - p.pad_h;
                 }
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = ti.kb0; kb < ti.kb1; ++kb) {
                     if (!wait_bar(empty_bar(stage), phase ^ 1u, p, ROLE_PRODUCER, t, stage)) { ok = false; break; }
                     const uint32_t a_dst = smem_base + stage * Cfg::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + Cfg::A_BYTES;
@@ -325,7 +372,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         tma_load_3d<kPair>(b_dst, mapB, fb, kb * Cfg::BK, nb0, bz);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                    if (t == first_tile && kb == 0) SG_STAMP(2);
+                    if (t == first_tile && kb == ti.kb0) SG_STAMP(2);
                 }
             }
             SG_STAMP(3);
@@ -348,9 +395,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (!wait_bar(tempty_bar(acc), acc_phase ^ 1u, p, ROLE_MMA, t, 100 + acc)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = ti.kb0; kb < ti.kb1; ++kb) {
                     if (!wait_bar(full_bar(stage), phase, p, ROLE_MMA, t, stage)) { ok = false; break; }
-                    if (t == first_tile && kb == 0) SG_STAMP(4);
+                    if (t == first_tile && kb == ti.kb0) SG_STAMP(4);
                     tc_fence_after_sync();
                     const uint32_t a_src = smem_base + stage * Cfg::STAGE_BYTES;
                     const uint64_t a_desc = smem_desc_k_major_sw128(a_src);
@@ -358,7 +405,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int kk = 0; kk < Cfg::BK / 16; ++kk) {
                         // 16 bf16 along K = 32 bytes = 2 units of the descriptor's address field
-                        umma_bf16<kPair>(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+                        umma_bf16<kPair>(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (kb != ti.kb0 || kk != 0) ? 1u : 0u);
                     }
                     umma_commit<kPair>(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -449,6 +496,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
             const int row = row0 + lane;
 
+            bool sk_waited = false;
             if (num_kb > 0 && half >= nchunks) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
                 tc_fence_before_sync();
@@ -492,6 +540,45 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     for (int i = 0; i < CH; ++i) v[i] = 0.0f;
                 }
                 if (!rows_live) continue;       // nothing of this warp's 32 rows exists (ragged last tile)
+
+                if (ti.nparts > 1) {
+                    // K-split tail tile.  Helpers park their raw fp32 partial sums in the scratch; the owner adds
+                    // them to its own (always in the order own + helper 1 + helper 2 ..., so results are reproducible).
+                    // Scratch layout of one CTA's partial tile: [group of 4 columns][row] float4, so that the 32
+                    // lanes (= rows) of a warp touch 512 contiguous bytes per access.
+                    const size_t tile_elems = static_cast<size_t>(Cfg::BM) * BN;
+                    const size_t my_off = static_cast<size_t>(cta_rank) * tile_elems +
+                                          (static_cast<size_t>(c * (CH / 4)) * Cfg::BM + static_cast<size_t>(q * 32 + lane)) * 4;
+                    if (ti.part > 0) {
+                        float* pb = p.sk_partials +
+                                    static_cast<size_t>(ti.tail * (p.ksplit - 1) + ti.part - 1) * kCtas * tile_elems + my_off;
+#pragma unroll
+                        for (int i = 0; i < CH; i += 4)
+                            __stcg(reinterpret_cast<float4*>(pb + static_cast<size_t>(i) * Cfg::BM),
+                                   make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+                        continue;
+                    }
+                    if (!sk_waited) {
+                        uint32_t okw = 1;
+                        if (lane == 0) {
+                            for (int h = 0; h < ti.nparts - 1 && okw; ++h)
+                                okw = wait_counter(p.sk_flags + ti.tail * (p.ksplit - 1) + h, static_cast<uint32_t>(p.sk_arrivals), p, t) ? 1u : 0u;
+                        }
+                        okw = __shfl_sync(0xFFFFFFFFu, okw, 0);
+                        if (!okw) { ok = false; break; }
+                        __threadfence();
+                        sk_waited = true;
+                    }
+                    for (int h = 0; h < ti.nparts - 1; ++h) {
+                        const float* pb = p.sk_partials +
+                                          static_cast<size_t>(ti.tail * (p.ksplit - 1) + h) * kCtas * tile_elems + my_off;
+#pragma unroll
+                        for (int i = 0; i < CH; i += 4) {
+                            const float4 x = __ldcg(reinterpret_cast<const float4*>(pb + static_cast<size_t>(i) * Cfg::BM));
+                            v[i] += x.x; v[i + 1] += x.y; v[i + 2] += x.z; v[i + 3] += x.w;
+                        }
+                    }
+                }
 
 #pragma unroll
                 for (int i = 0; i < CH; ++i) v[i] *= alpha;
@@ -592,6 +679,26 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     tma_store_commit();
                 }
 #endif
+            }
+            if (!ok) break;
+            if (ti.nparts > 1) {
+                // K-split bookkeeping, once per warp and tile whether or not the warp had columns or live rows
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) {
+                    uint32_t* flags = p.sk_flags + ti.tail * (p.ksplit - 1);
+                    if (ti.part > 0) {
+                        atomicAdd(flags + ti.part - 1, 1u);                      // this warp's share of the partial is visible
+                    } else {
+                        uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
+                        if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals) - 1u) {
+                            // last warp of the owner: every partial has been read; leave the counters at zero for the next launch
+                            for (int h = 0; h < ti.nparts - 1; ++h) flags[h] = 0u;
+                            *consumed = 0u;
+                            __threadfence();
+                        }
+                    }
+                }
             }
         }
         if (warp == 2 && lane == 0) SG_STAMP(8);

@@ -36,7 +36,7 @@ OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
-            "sg_last_launch_plan"]
+            "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode"]
 
 
 class SolgemmError(RuntimeError):
@@ -99,8 +99,45 @@ _lib.sg_poll_status.argtypes = [_vp]
 _lib.sg_set_tuning.restype = ctypes.c_int
 _lib.sg_set_tuning.argtypes = [_i32, _i32]
 _lib.sg_launch_count.restype = _i64
+_lib.sg_set_tail_mode.restype = ctypes.c_int
+_lib.sg_set_tail_mode.argtypes = [_i32]
+_lib.sg_set_scratch.restype = ctypes.c_int
+_lib.sg_set_scratch.argtypes = [_vp, ctypes.c_size_t]
 _lib.sg_last_launch_plan.restype = ctypes.c_int
 _lib.sg_last_launch_plan.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+
+
+SCRATCH_BYTES = 32 << 20
+_scratch = {}      # device index -> the torch buffer lent to the library (kept alive here)
+_scratch_enabled = os.environ.get("SOLGEMM_NO_SCRATCH", "0") != "1"
+
+
+def enable_scratch(on: bool = True) -> None:
+    """Turn the automatic lending of a scratch buffer on or off (off also takes back the current device's)."""
+    global _scratch_enabled
+    _scratch_enabled = bool(on)
+    if not on and torch.cuda.is_available() and torch.cuda.current_device() in _scratch:
+        torch.cuda.synchronize()
+        set_scratch(None)
+
+
+def set_scratch(buf: Optional[torch.Tensor]) -> None:
+    """``sg_set_scratch``: lend (or, with None, take back) the tail-balancing scratch of the current device."""
+    dev = torch.cuda.current_device()
+    if buf is None:
+        _check(_lib.sg_set_scratch(None, 0))
+        _scratch.pop(dev, None)
+    else:
+        _check(_lib.sg_set_scratch(_ptr(buf), buf.numel() * buf.element_size()))
+        _scratch[dev] = buf
+
+
+def ensure_scratch() -> None:
+    """Lend the library a scratch buffer on the current device once (torch owns the memory).
+    ``SOLGEMM_NO_SCRATCH=1`` keeps the library on its scratch-free tail strategy."""
+    dev = torch.cuda.current_device()
+    if dev not in _scratch and _scratch_enabled:
+        set_scratch(torch.empty(SCRATCH_BYTES, dtype=torch.uint8, device=f"cuda:{dev}"))
 
 
 def raw_lib() -> ctypes.CDLL:
@@ -147,6 +184,7 @@ def gemm(A: torch.Tensor, B: torch.Tensor, *, C: Optional[torch.Tensor] = None, 
          beta: float = 0.0, epi: str = "none", layout_a: str = "row", layout_b: str = "col", stream=None) -> torch.Tensor:
     """D = act(alpha A.B + beta C + bias) through ``sg_gemm``.  Returns D (``out`` if given)."""
     M, N, K = _mnk(A, B, layout_a, layout_b)
+    ensure_scratch()
     if out is None:
         out = torch.empty((M, N), dtype=out_dtype, device=A.device)
     desc = _gemm_desc(M, N, K, _ld(A), _ld(B), _ld(C) if C is not None else max(N, 1), _ld(out), layout_a, layout_b,
@@ -160,6 +198,7 @@ def batched_gemm(A: torch.Tensor, B: torch.Tensor, *, C=None, bias=None, out=Non
     """The same product for every leading index through ``sg_batched_gemm``; ``bias`` is [N] or [batch, N]."""
     batch = A.shape[0]
     M, N, K = _mnk(A, B, layout_a, layout_b)
+    ensure_scratch()
     if out is None:
         out = torch.empty((batch, M, N), dtype=out_dtype, device=A.device)
     for t in (A, B, out) + ((C,) if C is not None else ()):
@@ -197,6 +236,7 @@ def grouped_gemm(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=N
     groups = len(As)
     if groups == 0:
         return []
+    ensure_scratch()
     _, N, K = _mnk(As[0], Bs[0], layout_a, layout_b)
     Ms = [(_mnk(a, b, layout_a, layout_b))[0] for a, b in zip(As, Bs)]
     if outs is None:
@@ -250,6 +290,7 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
         raise ValueError("X and Wf disagree on C")
     ext = lambda size, p, d, f, s: max((size + 2 * p - d * (f - 1) - 1) // s + 1, 0) if size + 2 * p - d * (f - 1) - 1 >= 0 else 0
     P, Q = ext(H, pad[0], dil[0], R, stride[0]), ext(W, pad[1], dil[1], S, stride[1])
+    ensure_scratch()
     if out is None:
         out = torch.empty((N, P, Q, K), dtype=out_dtype, device=X.device)
     desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], 0, DTYPES[out.dtype],
@@ -309,6 +350,11 @@ def poll_status(stream=None) -> None:
 
 def set_tuning(tile_n: int = -1, cta_pair: int = -1) -> None:
     _check(_lib.sg_set_tuning(tile_n, cta_pair))
+
+
+def set_tail_mode(mode: int = -1) -> None:
+    """-1 planner's choice, 0 whole tail tiles, 1 column slices, 2 K ranges through the scratch."""
+    _check(_lib.sg_set_tail_mode(mode))
 
 
 def launch_count() -> int:

@@ -27,10 +27,14 @@ DEV = "cuda"
 @pytest.fixture(autouse=True)
 def _clean_status():
     sg.set_tuning(-1, -1)
+    sg.set_tail_mode(-1)
+    sg.enable_scratch(True)
     yield
     torch.cuda.synchronize()
     sg.poll_status()          # raises if any kernel recorded an expired wait
     sg.set_tuning(-1, -1)
+    sg.set_tail_mode(-1)
+    sg.enable_scratch(True)
 
 
 def guarded(shape, dtype, pad_rows=8):
@@ -102,21 +106,50 @@ def test_gemm_activation_form_is_pinned_on_the_fp32_path():
         parity.assert_matches(D, ref, absacc, epi)
 
 
+@pytest.mark.parametrize("scratch", [0, 2])
 @pytest.mark.parametrize("tile_n,pair,M,N,K", [(256, 0, 128 * 149, 200, 72), (256, 0, 128 * 149, 190, 72),
                                               (256, 1, 256 * 75, 190, 136), (128, 0, 128 * 149, 136, 72),
-                                              (128, 1, 256 * 77, 100, 64)])
-def test_gemm_tail_wave_split_into_column_slices(tile_n, pair, M, N, K):
-    # one tile more than a whole number of waves: the planner cuts the last wave's tiles into narrower slices
+                                              (128, 1, 256 * 77, 100, 64), (256, 1, 256 * 75, 192, 1024),
+                                              (256, 1, 256 * 98, 256, 192), (256, 0, 128 * 170, 264, 328)])
+def test_gemm_tail_wave_is_shared_between_sms(tile_n, pair, M, N, K, scratch):
+    # A few tiles more than a whole number of waves.  Without a scratch buffer the planner cuts the last wave's
+    # tiles into narrower column slices; with one it cuts their K loop into ranges whose fp32 partial sums the
+    # owner of the tile adds up.  Integer inputs: either way the result must be exact.
+    sg.enable_scratch(scratch == 2)
+    sg.set_tail_mode(1 if scratch == 0 else 2)
     sg.set_tuning(tile_n, pair)
     A = inputs.small_integers([M, K], 313, 1)
     B = inputs.small_integers([N, K], 313, 2)
     ref, _ = orc.gemm(A, B)
+    assert float(ref.abs().max()) <= 256
     D, whole = guarded((M, N), torch.bfloat16)
-    sg.gemm(A.to(DEV), B.to(DEV), out=D)
-    plan = sg.last_launch_plan()
-    assert plan["tail_split"] > 1 and plan["tiles"] > plan["split_begin"], plan
-    parity.assert_bit_exact(D, ref, f"tail split {plan}")
-    assert guards_intact(whole, cols=N)
+    dA, dB = A.to(DEV), B.to(DEV)
+    for _ in range(2):                    # twice: the K-split counters must be back at zero after a launch
+        D.fill_(float("nan"))
+        sg.gemm(dA, dB, out=D)
+        plan = sg.last_launch_plan()
+        assert plan["tiles"] > plan["split_begin"], plan
+        if not scratch or K <= 64:
+            assert plan["tail_split"] > 1, plan            # column slices (a single k-block cannot be cut)
+        else:
+            assert plan["tail_split"] < -1, plan           # K ranges
+        parity.assert_bit_exact(D, ref, f"tail split {plan}")
+        assert guards_intact(whole, cols=N)
+
+
+def test_k_split_tail_with_full_epilogue_matches_oracle():
+    sg.set_tuning(256, 1)
+    sg.set_tail_mode(2)
+    M, N, K = 256 * 76, 320, 520                          # 152 tiles on 74 pairs: 4 tail tiles; K tail of 8
+    A, B, bias = inputs.make_gemm(M, N, K, "normal", K ** -0.25, bias=True, seed=333)
+    C = inputs.normal([M, N], 333, 3)
+    ref, absacc = orc.gemm(A, B, C=C, bias=bias, alpha=1.25, beta=0.5, epi="gelu")
+    for out_dtype in (torch.bfloat16, torch.float32):
+        D = sg.gemm(A.to(DEV), B.to(DEV), C=C.to(out_dtype).to(DEV), bias=bias.to(DEV), alpha=1.25, beta=0.5, epi="gelu",
+                    out_dtype=out_dtype)
+        assert sg.last_launch_plan()["tail_split"] < -1
+        refd, accd = (ref, absacc) if out_dtype == torch.bfloat16 else orc.gemm(A, B, C=C.float(), bias=bias, alpha=1.25, beta=0.5, epi="gelu")
+        parity.assert_matches(D, refd, accd, f"K-split tail {out_dtype}")
 
 
 @pytest.mark.parametrize("out_dtype,N", [(torch.bfloat16, 90), (torch.float32, 90), (torch.float32, 67), (torch.bfloat16, 9)])
@@ -253,7 +286,10 @@ def test_grouped_gemm_ragged_bit_exact(tile_n, pair):
         assert torch.equal(outs_p[j].cpu(), outs[i].cpu())
 
 
-def test_grouped_and_conv_tail_split():
+@pytest.mark.parametrize("scratch", [False, True])
+def test_grouped_and_conv_tail_split(scratch):
+    sg.enable_scratch(scratch)
+    sg.set_tail_mode(2 if scratch else 1)
     sg.set_tuning(256, 0)
     Ms = [128 * 100, 128 * 49, 77]                     # 150 tiles of 128 x 256: two more than a wave of 148
     N, K = 200, 72
@@ -261,14 +297,14 @@ def test_grouped_and_conv_tail_split():
     Bs = [inputs.small_integers([N, K], 818 + g, 2) for g in range(len(Ms))]
     refs, _ = orc.grouped_gemm(As, Bs)
     outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs])
-    assert sg.last_launch_plan()["tail_split"] > 1
+    assert sg.last_launch_plan()["tail_split"] not in (0, 1, -1)
     for g in range(len(Ms)):
         parity.assert_bit_exact(outs[g], refs[g], f"group {g} with split tail")
     X = inputs.small_integers([2, 100, 96, 16], 828, 6, -1, 1)
     Wf = inputs.small_integers([256, 3, 3, 16], 828, 7, -1, 1)
     ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
     Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1))
-    assert sg.last_launch_plan()["tail_split"] > 1
+    assert sg.last_launch_plan()["tail_split"] not in (0, 1, -1)
     parity.assert_bit_exact(Y, ref, "conv with split tail")
 
 
