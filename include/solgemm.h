@@ -65,6 +65,8 @@ typedef enum { SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 
  *   a(i,k) = A[i*lda + k] (row-major) or A[k*lda + i] (column-major)
  *   b(k,j) = B[k*ldb + j] (row-major) or B[j*ldb + k] (column-major)
  *   C and D are row-major with leading dimensions ldc, ldd.  All ld* are in ELEMENTS.
+ *   All four A/B layout pairs are implemented; the K-contiguous pair (A row-major, B column-major) is the
+ *   tuned one.  (sg_grouped_gemm accepts a row-major A only: SG_ERR_UNSUPPORTED otherwise.)
  * Enum-valued fields are int32_t so that the layout is the same from C, C++ and ctypes.
  */
 typedef struct sg_gemm_desc {
@@ -218,6 +220,15 @@ sg_status_t sg_poll_status(void* cuda_stream);
  *   tile_n    64, 128 or 256            cta_pair   0 = one CTA per tile, 1 = two-CTA tiles
  */
 sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair);
+
+/*
+ * sg_last_kernel_clock: the SM clock (MHz) at which the most recent contraction kernel on the current device
+ * actually ran, measured inside the kernel (cycle counter over nanosecond timer of its first CTA).  Under a
+ * board power cap this is what the paper's clock-aware Speed-of-Light rule should scale the peak by (Section 4.1,
+ * "hardware limits ... scaled by the current clock"); management libraries may report the requested clock instead.
+ * Synchronises `cuda_stream`.  0 if no kernel has run yet.
+ */
+sg_status_t sg_last_kernel_clock(double* sm_mhz, void* cuda_stream);
 
 /*
  * sg_set_tail_mode: how the tiles of the last, partial wave are shared between SMs (tuning / tests):

@@ -233,11 +233,16 @@ sg_status_t check_gemm_desc(const sg_gemm_desc_t* d, bool grouped, Checked* c) {
         return fail(SG_ERR_UNSUPPORTED, "extents above 2^31-1 are not supported");
     if (d->layout_a != SG_ROW_MAJOR && d->layout_a != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_a %d is not a sg_layout_t", d->layout_a);
     if (d->layout_b != SG_ROW_MAJOR && d->layout_b != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_b %d is not a sg_layout_t", d->layout_b);
-    if (d->layout_a != SG_ROW_MAJOR || d->layout_b != SG_COL_MAJOR)
-        return fail(SG_ERR_UNSUPPORTED, "only the K-contiguous operand pair (A row-major, B column-major) is implemented");
+    if (grouped && d->layout_a == SG_COL_MAJOR)
+        return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: a column-major A (one leading dimension for groups of different M) is not implemented");
     const int64_t M = grouped ? 1 : d->M;
-    if (d->lda < (d->K > 1 ? d->K : 1) && M > 0) return fail(SG_ERR_INVALID_ARG, "lda %lld < K %lld", (long long)d->lda, (long long)d->K);
-    if (d->ldb < (d->K > 1 ? d->K : 1) && d->N > 0) return fail(SG_ERR_INVALID_ARG, "ldb %lld < K %lld", (long long)d->ldb, (long long)d->K);
+    // leading dimension >= the contiguous extent: K for a K-contiguous operand, M (resp. N) otherwise
+    const int64_t a_inner = d->layout_a == SG_ROW_MAJOR ? d->K : M;
+    const int64_t b_inner = d->layout_b == SG_COL_MAJOR ? d->K : d->N;
+    if (d->lda < (a_inner > 1 ? a_inner : 1) && M > 0 && d->K > 0)
+        return fail(SG_ERR_INVALID_ARG, "lda %lld is smaller than A's contiguous extent %lld", (long long)d->lda, (long long)a_inner);
+    if (d->ldb < (b_inner > 1 ? b_inner : 1) && d->N > 0 && d->K > 0)
+        return fail(SG_ERR_INVALID_ARG, "ldb %lld is smaller than B's contiguous extent %lld", (long long)d->ldb, (long long)b_inner);
     if (d->ldd < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldd %lld < N %lld", (long long)d->ldd, (long long)d->N);
     if (d->beta != 0.0f && d->ldc < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldc %lld < N %lld", (long long)d->ldc, (long long)d->N);
     if ((d->lda * 2) % 16 || (d->ldb * 2) % 16) return fail(SG_ERR_ALIGNMENT, "lda and ldb must be multiples of 8 elements (16 bytes)");
@@ -270,7 +275,7 @@ struct Shape {
 // and L2 reads, not by the tensor pipe).  Two-CTA tiles pay a fixed cluster set-up cost, so they are
 // used only when the K loop is long and there is at least one full wave of them.
 Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N,
-                   int64_t K) {
+                   int64_t K, int min_b_rows = 1) {
     const int force_bn = g_tune_tile_n.load();
     const int force_pair = g_tune_pair.load();
     const int bns[3] = {256, 128, 64};
@@ -292,6 +297,7 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
         for (int bi = 0; bi < 3; ++bi) {
             const int bn = bns[bi];
             if (force_bn > 0 && bn != force_bn) continue;
+            if (bn / (pi ? 2 : 1) < min_b_rows) continue;       // an N-contiguous B is loaded in blocks of 64 rows
             const int64_t tiles = tiles_for(pi ? 256 : 128, bn);
             const int64_t slots = pi ? d.max_pairs : d.sm_count;
             const int64_t waves = (tiles + slots - 1) / slots;
@@ -310,7 +316,7 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
 // cut into `split` column slices so that the idle SMs of that wave take a share.  Narrow slices cost more
 // per output area (same factors as in choose_shape), so a split is used only when it shortens the tail.
 // Sets p->split_begin, p->split and p->num_tiles (the length of the tile list) from the full-width count.
-void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params* p) {
+void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1) {
     const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
     int best_split = 1, best_ksplit = 1;
@@ -323,7 +329,7 @@ void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params*
         double best = 1.0;      // cost of the unsplit tail wave, in units of one full-width tile
         for (int k = 1; k <= 2; ++k) {
             const int split = 1 << k;
-            if (s.bn / split < 64) break;
+            if (s.bn / split < 64 || s.bn / split / (s.pair ? 2 : 1) < min_b_rows) break;
             const int64_t waves = (rem * split + slots - 1) / slots;
             const double cost = static_cast<double>(waves) / split * factor[s.pair ? 1 : 0][k];
             if (cost < best - 0.05) {
@@ -332,7 +338,7 @@ void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params*
             }
         }
         if (forced == 1 || forced == 2 || forced == 4) {
-            best_split = (s.bn / forced >= 64) ? forced : 1;
+            best_split = (s.bn / forced >= 64 && s.bn / forced / (s.pair ? 2 : 1) >= min_b_rows) ? forced : 1;
             best = 0.9;
         }
         // K-split through the registered scratch: ksplit SM groups share one tail tile's K loop; the owner adds the
@@ -347,8 +353,10 @@ void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params*
             if (max_buffers > static_cast<size_t>(kScratchMaxBuffers)) max_buffers = kScratchMaxBuffers;
             // measured: helpers' dump, the owner's wait and its reads of the partials cost about 0.45 of a tile
             const double cost = 1.0 / static_cast<double>(ks) + 0.45;
+            // The exchange costs a fixed ~10 us whatever the tile's K, so it can only pay for very long K loops.
+            const bool long_k = p->num_kb / ks >= 64;
             if (ks >= 2 && static_cast<size_t>(rem * (ks - 1)) <= max_buffers && rem <= kScratchMaxBuffers &&
-                (cost < best - 0.05 || forced_k >= 2)) {
+                ((cost < best - 0.05 && long_k) || forced_k >= 2)) {
                 best_ksplit = static_cast<int>(ks);
                 best_split = 1;
             }
@@ -383,13 +391,18 @@ sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params&
     cfg.blockDim = dim3(k.threads);
     cfg.dynamicSmemBytes = k.smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = ctas_per_tile;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ctas_per_tile;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    // programmatic dependent launch: this kernel's set-up may overlap the previous kernel's tail (the kernel
+    // itself waits for that kernel before it touches global memory)
+    static const bool pdl = !(getenv("SG_NO_PDL") && atoi(getenv("SG_NO_PDL")) != 0);
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 2 : 1;
     SG_CUDA(cudaLaunchKernelEx(&cfg, k.fn, p));
     g_launches.fetch_add(1);
     t_last_plan[0] = s.bn;
@@ -435,9 +448,12 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
 
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
-    const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K);
+    const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
+    const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_DENSE;
+    p.a_mn_major = desc->layout_a == SG_COL_MAJOR ? 1 : 0;
+    p.b_mn_major = desc->layout_b == SG_ROW_MAJOR ? 1 : 0;
     p.M = static_cast<int32_t>(desc->M);
     p.N = static_cast<int32_t>(desc->N);
     p.K = static_cast<int32_t>(desc->K);
@@ -447,7 +463,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n * batch;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
     p.num_kb = static_cast<int32_t>((desc->K + 63) / 64);
-    plan_tail(*d, s, tiles, &p);
+    plan_tail(*d, s, tiles, &p, min_b_rows);
     p.bias = bias;
     p.C = desc->beta != 0.0f ? C : nullptr;
     p.ldc = desc->ldc;
@@ -457,13 +473,23 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.ldd = desc->ldd;
     p.strideD = sD;
     if (desc->K > 0) {
-        st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
+        // K-contiguous operand: boxes of 64 k x tile rows.  M/N-contiguous operand (column-major A, row-major B):
+        // the map is over [k][rows] and every load is a box of 64 rows x 64 k.
+        if (p.a_mn_major)
+            st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->M, desc->K, batch, desc->lda, sA, 64, 64, "A");
+        else
+            st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
         if (st != SG_OK) return st;
-        st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
-                            s.pair ? s.bn / 2 : s.bn, "B");
-        if (st != SG_OK) return st;
-        st = make_tiled_map(&p.tmB2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
-                            (s.pair ? s.bn / 2 : s.bn) / p.split, "B (narrow)");
+        if (p.b_mn_major) {
+            st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->N, desc->K, batch, desc->ldb, sB, 64, 64, "B");
+            p.tmB2 = p.tmB;
+        } else {
+            st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+                                s.pair ? s.bn / 2 : s.bn, "B");
+            if (st != SG_OK) return st;
+            st = make_tiled_map(&p.tmB2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+                                (s.pair ? s.bn / 2 : s.bn) / p.split, "B (narrow)");
+        }
         if (st != SG_OK) return st;
     }
     st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, D,
@@ -583,6 +609,19 @@ sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair) {
     return SG_OK;
 }
 
+sg_status_t sg_last_kernel_clock(double* sm_mhz, void* cuda_stream) {
+    if (!sm_mhz) return fail(SG_ERR_NULL_POINTER, "sm_mhz is NULL");
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    uint64_t w[2] = {0, 0};
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    SG_CUDA(cudaMemcpyAsync(w, d->status_dev + 4, sizeof w, cudaMemcpyDeviceToHost, stream));
+    SG_CUDA(cudaStreamSynchronize(stream));
+    *sm_mhz = w[1] > 0 ? static_cast<double>(w[0]) / static_cast<double>(w[1]) * 1e3 : 0.0;
+    return SG_OK;
+}
+
 sg_status_t sg_set_tail_mode(int32_t mode) {
     if (mode < -1 || mode > 2) return fail(SG_ERR_INVALID_ARG, "tail mode must be -1 (auto), 0, 1 or 2");
     g_tune_tail.store(mode);
@@ -642,7 +681,8 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     DeviceState* d = nullptr;
     st = device_state(&d);
     if (st != SG_OK) return st;
-    const Shape s = choose_shape(*d, rows, 1, common->N, common->K);
+    const int min_b_rows = common->layout_b == SG_ROW_MAJOR ? 64 : 1;
+    const Shape s = choose_shape(*d, rows, 1, common->N, common->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
     const int tiles_n = static_cast<int>((common->N + s.bn - 1) / s.bn);
 
@@ -653,7 +693,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
     p.K = static_cast<int32_t>(common->K);
     p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
-    plan_tail(*d, s, tiles, &p);
+    plan_tail(*d, s, tiles, &p, min_b_rows);
 
     std::vector<uint8_t> host(L.total, 0);
     CUtensorMap* maps = reinterpret_cast<CUtensorMap*>(host.data() + L.off_maps);
@@ -676,11 +716,17 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
             st = make_tiled_map(&maps[4 * g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A_ptrs_host[g], common->K, rows[g], 1,
                                 common->lda, 0, 64, 128, "A_g");
             if (st != SG_OK) return st;
-            st = make_tiled_map(&maps[4 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
-                                common->ldb, 0, 64, b_box, "B_g");
-            if (st != SG_OK) return st;
-            st = make_tiled_map(&maps[4 * g + 3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
-                                common->ldb, 0, 64, b_box / p.split, "B_g (narrow)");
+            if (common->layout_b == SG_ROW_MAJOR) {
+                st = make_tiled_map(&maps[4 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->N, common->K, 1,
+                                    common->ldb, 0, 64, 64, "B_g");
+                maps[4 * g + 3] = maps[4 * g + 1];
+            } else {
+                st = make_tiled_map(&maps[4 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                                    common->ldb, 0, 64, b_box, "B_g");
+                if (st != SG_OK) return st;
+                st = make_tiled_map(&maps[4 * g + 3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                                    common->ldb, 0, 64, b_box / p.split, "B_g (narrow)");
+            }
             if (st != SG_OK) return st;
         }
         st = make_tiled_map(&maps[4 * g + 2], c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
@@ -695,6 +741,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
 
     uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
     p.mode = MODE_GROUPED;
+    p.b_mn_major = common->layout_b == SG_ROW_MAJOR ? 1 : 0;
     p.gmaps = reinterpret_cast<const CUtensorMap*>(ws + L.off_maps);
     p.g_tile_start = reinterpret_cast<const int32_t*>(ws + L.off_tile_start);
     p.g_M = reinterpret_cast<const int32_t*>(ws + L.off_M);

@@ -51,6 +51,7 @@ struct alignas(64) Params {
     int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
     float alpha, beta;
     int32_t epi, mode;
+    int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
     uint32_t* status;                   // device status words (8 x u32)
     uint64_t timeout_ns;                // bound of every device-side wait
@@ -262,6 +263,13 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem + Cfg::OFF_BAR + 8 * Cfg::NUM_BARS);
 
     if (threadIdx.x == 0) SG_STAMP(0);
+    // CTA 0 measures the SM clock this launch actually ran at (cycle counter against the nanosecond timer);
+    // the host reads it through sg_last_kernel_clock for clock-scaled Speed-of-Light figures.
+    uint64_t clk0 = 0, ns0 = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 96) {
+        clk0 = clock64();
+        ns0 = global_timer_ns();
+    }
 #ifdef SG_DEBUG_STAMPS
     if (threadIdx.x == 32 && blockIdx.x == (SG_DEBUG_STAMPS - 1)) {
         reinterpret_cast<volatile uint64_t*>(p.status + 8)[11] = clock64();
@@ -308,6 +316,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot_ptr;
     if (threadIdx.x == 0) SG_STAMP(1);
+    // Everything above touched only this CTA's shared memory, TMEM and the kernel parameters, so under
+    // programmatic dependent launch it may overlap the tail of the previous kernel in the stream.  From here
+    // on global memory is read and written: wait for the previous kernel, then let the next one start setting up.
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     const int num_kb = p.num_kb;
     const int first_tile = blockIdx.x / kCtas;
@@ -368,8 +381,20 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                                                   static_cast<uint16_t>(r * p.dil_h));
                         tma_load_3d<kPair>(b_dst, mapB, fb, c0, tap, nb0);
                     } else {
-                        tma_load_3d<kPair>(a_dst, mapA, fb, kb * Cfg::BK, m0, bz);
-                        tma_load_3d<kPair>(b_dst, mapB, fb, kb * Cfg::BK, nb0, bz);
+                        if (p.a_mn_major) {
+                            // column-major A: boxes of 64 rows of the tile (contiguous) x 64 k, one per 64 tile rows
+#pragma unroll
+                            for (int j = 0; j < Cfg::BM / 64; ++j)
+                                tma_load_3d<kPair>(a_dst + j * 8192, mapA, fb, m0 + j * 64, kb * Cfg::BK, bz);
+                        } else {
+                            tma_load_3d<kPair>(a_dst, mapA, fb, kb * Cfg::BK, m0, bz);
+                        }
+                        if (p.b_mn_major) {
+                            for (int j = 0; j < b_rows / 64; ++j)
+                                tma_load_3d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, kb * Cfg::BK, bz);
+                        } else {
+                            tma_load_3d<kPair>(b_dst, mapB, fb, kb * Cfg::BK, nb0, bz);
+                        }
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     if (t == first_tile && kb == ti.kb0) SG_STAMP(2);
@@ -388,7 +413,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
                 const Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
-                const uint32_t idesc = umma_idesc_bf16_f32(Cfg::TILE_M, ti.width);
+                const uint32_t idesc = umma_idesc_bf16_f32(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0);
+                const uint32_t a_step = p.a_mn_major ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
+                const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
                 const int acc = iter & 1;
                 const uint32_t acc_phase = (iter >> 1) & 1u;
                 ++iter;
@@ -400,12 +427,14 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     if (t == first_tile && kb == ti.kb0) SG_STAMP(4);
                     tc_fence_after_sync();
                     const uint32_t a_src = smem_base + stage * Cfg::STAGE_BYTES;
-                    const uint64_t a_desc = smem_desc_k_major_sw128(a_src);
-                    const uint64_t b_desc = smem_desc_k_major_sw128(a_src + Cfg::A_BYTES);
+                    const uint64_t a_desc = p.a_mn_major ? smem_desc_mn_major_sw128(a_src) : smem_desc_k_major_sw128(a_src);
+                    const uint64_t b_desc = p.b_mn_major ? smem_desc_mn_major_sw128(a_src + Cfg::A_BYTES)
+                                                         : smem_desc_k_major_sw128(a_src + Cfg::A_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < Cfg::BK / 16; ++kk) {
-                        // 16 bf16 along K = 32 bytes = 2 units of the descriptor's address field
-                        umma_bf16<kPair>(d_tmem, a_desc + 2u * kk, b_desc + 2u * kk, idesc, (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                        // one K=16 step: 32 bytes along a K-major row, or two 1 KB k-groups of an MN-major tile
+                        umma_bf16<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
+                                         (kb != ti.kb0 || kk != 0) ? 1u : 0u);
                     }
                     umma_commit<kPair>(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -721,6 +750,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc<kPair>(tmem_base, Cfg::TMEM_COLS);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 96) {
+        volatile uint64_t* w = reinterpret_cast<volatile uint64_t*>(p.status + 4);
+        w[0] = static_cast<uint64_t>(clock64()) - clk0;
+        w[1] = global_timer_ns() - ns0;
     }
     if (threadIdx.x == 32) SG_STAMP(10);
 #ifdef SG_DEBUG_STAMPS

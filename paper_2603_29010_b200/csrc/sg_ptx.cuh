@@ -50,6 +50,12 @@ __device__ __forceinline__ void cluster_wait() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// wait: blocks until the kernels this launch depends on have completed and their memory is visible.
+// launch_dependents: lets the next kernel of the stream (if it opted in) start its own prologue early.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -253,12 +259,27 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr) 
     return d;
 }
 
+// The same for an MN-major operand (the M or N index is contiguous in memory, e.g. a column-major A):
+// TMA boxes of 64 elements along M/N (128 bytes) x 64 k-rows with the 128-byte swizzle, one box per 64 rows
+// of the tile, boxes 8 KB apart.  In descriptor terms: 8 k-rows x 128 B form a 1 KB atom; the stride between
+// groups of 8 k-rows is the stride byte offset (1024 B), the stride between 64-element blocks along M/N is
+// the leading byte offset (8192 B).  One K=16 step is two k-groups: advance the start address by 2048 B.
+__device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
+    d |= static_cast<uint64_t>(8192 >> 4) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+
 // Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, both K-major, no
 // negation, dense.  bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format,
 // 15 / 16 A / B major (0 = K), 17-22 N >> 3, 24-28 M >> 4.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
-           (static_cast<uint32_t>(m >> 4) << 24);
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n, bool a_mn_major = false, bool b_mn_major = false) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
+           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 
 }  // namespace sg

@@ -36,7 +36,8 @@ OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
-            "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode"]
+            "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
+            "sg_last_kernel_clock"]
 
 
 class SolgemmError(RuntimeError):
@@ -99,6 +100,8 @@ _lib.sg_poll_status.argtypes = [_vp]
 _lib.sg_set_tuning.restype = ctypes.c_int
 _lib.sg_set_tuning.argtypes = [_i32, _i32]
 _lib.sg_launch_count.restype = _i64
+_lib.sg_last_kernel_clock.restype = ctypes.c_int
+_lib.sg_last_kernel_clock.argtypes = [ctypes.POINTER(ctypes.c_double), _vp]
 _lib.sg_set_tail_mode.restype = ctypes.c_int
 _lib.sg_set_tail_mode.argtypes = [_i32]
 _lib.sg_set_scratch.restype = ctypes.c_int
@@ -350,6 +353,13 @@ def poll_status(stream=None) -> None:
 
 def set_tuning(tile_n: int = -1, cta_pair: int = -1) -> None:
     _check(_lib.sg_set_tuning(tile_n, cta_pair))
+
+
+def last_kernel_clock_mhz(stream=None) -> float:
+    """SM clock the most recent contraction kernel really ran at (measured in the kernel); synchronises the stream."""
+    mhz = ctypes.c_double(0.0)
+    _check(_lib.sg_last_kernel_clock(ctypes.byref(mhz), _stream(stream)))
+    return float(mhz.value)
 
 
 def set_tail_mode(mode: int = -1) -> None:

@@ -76,6 +76,53 @@ def test_gemm_integer_inputs_bit_exact(M, N, K, tile_n, pair):
     assert guards_intact(whole)
 
 
+LAYOUT_TILINGS = [(64, 0), (128, 0), (256, 0), (128, 1), (256, 1), (-1, -1)]
+
+
+@pytest.mark.parametrize("tile_n,pair", LAYOUT_TILINGS)
+@pytest.mark.parametrize("la,lb", [("row", "row"), ("col", "col"), ("col", "row")])
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (300, 200, 136), (129, 72, 8), (1000, 520, 328), (128 * 149, 136, 72)])
+def test_gemm_other_operand_layouts_bit_exact(M, N, K, la, lb, tile_n, pair):
+    # column-major A and/or row-major B: the M- or N-contiguous operand goes through the MN-major descriptor
+    sg.set_tuning(tile_n, pair)
+    Am = inputs.small_integers([M, K + 8], 111, 1)[:, :K]
+    Bm = inputs.small_integers([K, N + 8], 111, 2)[:, :N]
+    ref = Am.double() @ Bm.double()
+    assert float(ref.abs().max()) <= 256
+    def stored(mat, transposed):
+        """The matrix as stored (transposed for a column-major A / B), leading dimension padded to 8 elements."""
+        m = mat.t() if transposed else mat
+        buf = torch.zeros(m.shape[0], (m.shape[1] + 7) // 8 * 8 + 8, dtype=torch.bfloat16)
+        buf[:, :m.shape[1]] = m
+        return buf, m.shape[1]
+    Abuf, a_cols = stored(Am, la == "col")                               # stored [M,K] or [K,M]
+    Bbuf, b_cols = stored(Bm, lb == "col")                               # stored [K,N] or [N,K]
+    oref, _ = orc.gemm(Abuf[:, :a_cols], Bbuf[:, :b_cols], layout_a=la, layout_b=lb)
+    assert torch.equal(oref, ref)
+    D, whole = guarded((M, N), torch.bfloat16)
+    sg.gemm(Abuf.to(DEV)[:, :a_cols], Bbuf.to(DEV)[:, :b_cols], out=D, layout_a=la, layout_b=lb)
+    parity.assert_bit_exact(D, ref, f"layouts {la}/{lb} {M}x{N}x{K} tiling {sg.last_launch_plan()}")
+    assert guards_intact(whole, cols=N)
+
+
+def test_other_layouts_with_padded_leading_dimensions_batched_and_grouped():
+    batch, M, N, K = 3, 200, 136, 72
+    Ast = inputs.small_integers([batch, K, M + 24], 121, 1)             # column-major A: [K, M] with lda = M + 24
+    Bst = inputs.small_integers([batch, K, N + 8], 121, 2)              # row-major B:    [K, N] with ldb = N + 8
+    A, B = Ast[:, :, :M], Bst[:, :, :N]
+    ref, absacc = orc.batched_gemm(A, B, layout_a="col", layout_b="row", epi="relu")
+    D = sg.batched_gemm(Ast.to(DEV)[:, :, :M], Bst.to(DEV)[:, :, :N], layout_a="col", layout_b="row", epi="relu")
+    parity.assert_bit_exact(D, ref, "batched col/row")
+    # grouped: row-major A (ragged M), row-major B
+    Ms = [130, 257, 64]
+    As = [inputs.small_integers([m, K], 131 + g, 1) for g, m in enumerate(Ms)]
+    Bs = [inputs.small_integers([K, N], 131 + g, 2) for g in range(len(Ms))]
+    refs, _ = orc.grouped_gemm(As, Bs, layout_a="row", layout_b="row")
+    outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs], layout_a="row", layout_b="row")
+    for g in range(len(Ms)):
+        parity.assert_bit_exact(outs[g], refs[g], f"grouped row/row group {g}")
+
+
 @pytest.mark.parametrize("pair", [0, 1])
 @pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("epi", ["none", "bias", "relu", "gelu", "silu"])
