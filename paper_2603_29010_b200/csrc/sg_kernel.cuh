@@ -165,20 +165,43 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Pa
     return wait_slow(bar, parity, p, role, tile, which);
 }
 
-// Activation of the fused epilogue, evaluated with one exp and one division (two special-function
-// operations per element; measured faster here than the single tanh.approx form), accurate to a few fp32 ulps:
+__device__ __forceinline__ float tanh_approx(float x) {
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Activation of the fused epilogue.
 //   gelu(v) = 0.5 v (1 + tanh(u)) = v * sigmoid(2u),  u = sqrt(2/pi) (v + 0.044715 v^3)
-//   silu(v) = v * sigmoid(v)
+//   silu(v) = v * sigmoid(v) = 0.5 v (1 + tanh(v / 2))
+// kFast (bf16 output): the hardware tanh approximation (relative error about 2^-11, an eighth of a bf16
+// rounding step), one special-function operation per element -- twice the throughput of the exact form in
+// isolation.  Otherwise (fp32 output): one exp and one division, accurate to a few fp32 ulps.
+#ifndef SG_FAST_ACT
+#define SG_FAST_ACT 1
+#endif
+template <bool kFast>
 __device__ __forceinline__ float apply_act(float v, int epi) {
     switch (epi) {
         case EPI_RELU:
             return fmaxf(v, 0.0f);
         case EPI_GELU: {
-            const float u2 = 1.5957691216057308f * (v + 0.044715f * v * v * v);
-            return __fdividef(v, 1.0f + __expf(-u2));
+            const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
+            if constexpr (kFast && SG_FAST_ACT) {
+                const float h = 0.5f * v;
+                return fmaf(h, tanh_approx(u), h);
+            } else {
+                return __fdividef(v, 1.0f + __expf(-2.0f * u));
+            }
         }
-        case EPI_SILU:
-            return __fdividef(v, 1.0f + __expf(-v));
+        case EPI_SILU: {
+            if constexpr (kFast && SG_FAST_ACT) {
+                const float h = 0.5f * v;
+                return fmaf(h, tanh_approx(h), h);
+            } else {
+                return __fdividef(v, 1.0f + __expf(-v));
+            }
+        }
         default:
             return v;
     }
@@ -652,7 +675,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 if (epi >= EPI_RELU) {
 #pragma unroll
-                    for (int i = 0; i < CH; ++i) v[i] = apply_act(v[i], epi);
+                    for (int i = 0; i < CH; ++i) v[i] = apply_act<!kOutF32>(v[i], epi);
                 }
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
