@@ -25,6 +25,8 @@
  *    by alpha.  SG_EPI_BIAS is the identity activation and requires bias != NULL; every other
  *    activation accepts an optional bias.  SG_EPI_GELU is the tanh form
  *    0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))).  beta == 0 means C is never read.
+ *    With bf16 output the transcendental activations use hardware approximations (error well below one
+ *    bf16 rounding step); with fp32 output they are evaluated to a few fp32 ulps.
  *  - Alignment (the TMA rule of the paper's Appendix A.1, constraint 3): every base pointer must
  *    be 16-byte aligned and every leading dimension / batch stride a multiple of 16 bytes
  *    (8 bf16 or 4 fp32 elements), else SG_ERR_ALIGNMENT.
@@ -58,7 +60,17 @@ typedef enum {
 
 typedef enum { SG_BF16 = 0, SG_F32 = 1 } sg_dtype_t;
 typedef enum { SG_ROW_MAJOR = 0, SG_COL_MAJOR = 1 } sg_layout_t;
-typedef enum { SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4 } sg_epilogue_t;
+typedef enum {
+    SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4,
+    /* further built-ins of the paper's Table 1c; epi_arg0 / epi_arg1 carry their parameters */
+    SG_EPI_SIGMOID = 5,     /* 1 / (1 + e^-x) */
+    SG_EPI_TANH = 6,
+    SG_EPI_MISH = 7,        /* x tanh(ln(1 + e^x)) */
+    SG_EPI_HARDSWISH = 8,   /* x min(max(x + 3, 0), 6) / 6 */
+    SG_EPI_LEAKY_RELU = 9,  /* x > 0 ? x : epi_arg0 * x */
+    SG_EPI_ELU = 10,        /* x > 0 ? x : epi_arg0 * (e^x - 1) */
+    SG_EPI_CLIP = 11        /* min(max(x, epi_arg0), epi_arg1), epi_arg0 <= epi_arg1 (the DSL's clip / clamp) */
+} sg_epilogue_t;
 
 /*
  * One GEMM problem (DSL: gemm().with_dtype(...).with_layout(A,B,C).with_scaling(alpha,beta) >> ...).
@@ -76,6 +88,7 @@ typedef struct sg_gemm_desc {
     int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype must be SG_BF16 */
     float alpha, beta;
     int32_t epi;                  /* sg_epilogue_t */
+    float epi_arg0, epi_arg1;     /* activation parameters (leaky_relu / elu slope, clip bounds); else ignored */
     int32_t reserved;             /* must be 0 */
 } sg_gemm_desc_t;
 
@@ -162,6 +175,7 @@ typedef struct sg_conv2d_desc {
     int32_t in_dtype, out_dtype;  /* sg_dtype_t */
     float alpha, beta;
     int32_t epi;                  /* sg_epilogue_t */
+    float epi_arg0, epi_arg1;     /* activation parameters, as in sg_gemm_desc_t */
     int32_t reserved;             /* must be 0 */
 } sg_conv2d_desc_t;
 

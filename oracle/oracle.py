@@ -30,7 +30,8 @@ _SRC = os.path.join(_HERE, "sg_oracle.c")
 _LIB = os.path.join(_HERE, "libsg_oracle.so")
 
 LAYOUTS = {"row": 0, "col": 1}
-EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4}
+EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
+             "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
 _DTYPES = {torch.bfloat16: 0, torch.float32: 1}
 
 
@@ -54,18 +55,20 @@ def lib() -> ctypes.CDLL:
         L.orc_num_threads.restype = ci
         L.orc_act.restype = dbl
         L.orc_act.argtypes = [ci, dbl]
+        L.orc_act2.restype = dbl
+        L.orc_act2.argtypes = [ci, dbl, dbl, dbl]
         L.orc_gemm.restype = ci
-        L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci,
+        L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl,
                                i64, i64, vp, vp, i64]
         L.orc_gemm_points.restype = ci
-        L.orc_gemm_points.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci,
+        L.orc_gemm_points.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl,
                                       i64, vp, vp, vp, vp]
         L.orc_conv_out_extent.restype = i64
         L.orc_conv_out_extent.argtypes = [i64] * 5
         L.orc_conv2d_fprop.restype = ci
-        L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, i64, i64, vp, vp]
+        L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, i64, i64, vp, vp]
         L.orc_conv2d_points.restype = ci
-        L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, i64, vp, vp, vp, vp]
+        L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, i64, vp, vp, vp, vp]
         L.orc_gemm_flops.restype = i64
         L.orc_gemm_flops.argtypes = [i64, i64, i64]
         L.orc_gemm_bytes.restype = i64
@@ -84,8 +87,8 @@ def num_threads() -> int:
     return int(lib().orc_num_threads())
 
 
-def act(epi: str, x: float) -> float:
-    return float(lib().orc_act(EPILOGUES[epi], float(x)))
+def act(epi: str, x: float, args=(0.0, 0.0)) -> float:
+    return float(lib().orc_act2(EPILOGUES[epi], float(x), float(args[0]), float(args[1])))
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -129,7 +132,7 @@ def _check_bias(bias, n):
 
 def gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a: str = "row", layout_b: str = "col",
          C: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
-         alpha: float = 1.0, beta: float = 0.0, epi: str = "none",
+         alpha: float = 1.0, beta: float = 0.0, epi: str = "none", epi_args=(0.0, 0.0),
          rows: Optional[Tuple[int, int]] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """act(alpha A.B + beta C + bias) for rows ``rows=(begin, end)`` (default: all)."""
     M, N, K, lda, ldb = _gemm_shapes(A, B, layout_a, layout_b)
@@ -140,14 +143,14 @@ def gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a: str = "row", layout_b: s
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
                         _ptr(C), c_dtype, ldc, _ptr(bias), float(alpha), float(beta), EPILOGUES[epi],
-                        r0, r1, _ptr(ref), _ptr(absacc), max(N, 1))
+                        float(epi_args[0]), float(epi_args[1]), r0, r1, _ptr(ref), _ptr(absacc), max(N, 1))
     if rc:
         raise ValueError(f"orc_gemm rejected its arguments (code {rc})")
     return ref, absacc
 
 
 def gemm_points(A, B, pi: Sequence[int], pj: Sequence[int], *, layout_a="row", layout_b="col", C=None, bias=None,
-                alpha=1.0, beta=0.0, epi="none") -> Tuple[torch.Tensor, torch.Tensor]:
+                alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)) -> Tuple[torch.Tensor, torch.Tensor]:
     """The elements (pi[t], pj[t]) of the result only."""
     M, N, K, lda, ldb = _gemm_shapes(A, B, layout_a, layout_b)
     _check_bias(bias, N)
@@ -158,32 +161,34 @@ def gemm_points(A, B, pi: Sequence[int], pj: Sequence[int], *, layout_a="row", l
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm_points(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
                                _ptr(C), c_dtype, ldc, _ptr(bias), float(alpha), float(beta), EPILOGUES[epi],
-                               pi.numel(), _ptr(pi), _ptr(pj), _ptr(ref), _ptr(absacc))
+                               float(epi_args[0]), float(epi_args[1]), pi.numel(), _ptr(pi), _ptr(pj), _ptr(ref),
+                               _ptr(absacc))
     if rc:
         raise ValueError(f"orc_gemm_points rejected its arguments (code {rc})")
     return ref, absacc
 
 
 def batched_gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a="row", layout_b="col", C=None, bias=None,
-                 alpha=1.0, beta=0.0, epi="none"):
+                 alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)):
     """The same product for every leading index b; ``bias`` is ``[N]`` (shared) or ``[batch, N]``."""
     refs, accs = [], []
     for b in range(A.shape[0]):
         bb = None if bias is None else (bias if bias.dim() == 1 else bias[b])
         r, a = gemm(A[b], B[b], layout_a=layout_a, layout_b=layout_b, C=None if C is None else C[b],
-                    bias=bb, alpha=alpha, beta=beta, epi=epi)
+                    bias=bb, alpha=alpha, beta=beta, epi=epi, epi_args=epi_args)
         refs.append(r)
         accs.append(a)
     return torch.stack(refs), torch.stack(accs)
 
 
-def grouped_gemm(As, Bs, *, layout_a="row", layout_b="col", Cs=None, biases=None, alpha=1.0, beta=0.0, epi="none"):
+def grouped_gemm(As, Bs, *, layout_a="row", layout_b="col", Cs=None, biases=None, alpha=1.0, beta=0.0, epi="none",
+                 epi_args=(0.0, 0.0)):
     """One independent product per group g with its own (M_g, A_g, B_g, C_g, bias_g)."""
     out = []
     for g in range(len(As)):
         out.append(gemm(As[g], Bs[g], layout_a=layout_a, layout_b=layout_b,
                         C=None if Cs is None else Cs[g], bias=None if biases is None else biases[g],
-                        alpha=alpha, beta=beta, epi=epi))
+                        alpha=alpha, beta=beta, epi=epi, epi_args=epi_args))
     return [o[0] for o in out], [o[1] for o in out]
 
 
@@ -216,7 +221,7 @@ def _conv_c(Cin, N, P, Q, K):
 
 
 def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1), dil=(1, 1),
-                 Cin=None, bias=None, alpha=1.0, beta=0.0, epi="none",
+                 Cin=None, bias=None, alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0),
                  pixels: Optional[Tuple[int, int]] = None):
     """Direct convolution; returns ``[N,P,Q,K]`` tensors, or ``[pixels, K]`` for a flattened pixel range."""
     d, N, P, Q, K = _conv_dims(X, Wf, pad, stride, dil)
@@ -226,7 +231,8 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
     ref = torch.empty((p1 - p0, K), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_fprop(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
-                                float(alpha), float(beta), EPILOGUES[epi], p0, p1, _ptr(ref), _ptr(absacc))
+                                float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
+                                p0, p1, _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_fprop rejected its arguments (code {rc})")
     if pixels is None:
@@ -235,7 +241,7 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
 
 
 def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), stride=(1, 1), dil=(1, 1),
-                  Cin=None, bias=None, alpha=1.0, beta=0.0, epi="none"):
+                  Cin=None, bias=None, alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)):
     """The outputs (flattened pixel ppix[t], channel pk[t]) only."""
     d, N, P, Q, K = _conv_dims(X, Wf, pad, stride, dil)
     _check_bias(bias, K)
@@ -245,8 +251,8 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
     ref = torch.empty(ppix.numel(), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_points(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
-                                 float(alpha), float(beta), EPILOGUES[epi], ppix.numel(), _ptr(ppix), _ptr(pk),
-                                 _ptr(ref), _ptr(absacc))
+                                 float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
+                                 ppix.numel(), _ptr(ppix), _ptr(pk), _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_points rejected its arguments (code {rc})")
     return ref, absacc

@@ -21,8 +21,9 @@
  *       product" (Appendix A.2, section 1 of the SOL report).
  *   conv2d_fprop -- conv2d_fprop(kernel_h, kernel_w) on TensorNHWC input /
  *       filter / output (Appendix A.1; Table 1a "Conv2d ... NHWC").
- *   epilogue -- the `>>` chain bias(), relu(), gelu(), silu() compiled into one
- *       fused epilogue (Section 3, "Epilogue fusion"; Table 1c).
+ *   epilogue -- the `>>` chain bias() followed by one of relu(), gelu(), silu(), sigmoid(), tanh(),
+ *       mish(), hardswish(), leaky_relu(alpha), elu(alpha), clip(min, max), compiled into one
+ *       fused epilogue (Section 3, "Epilogue fusion"; Table 1c; Appendix A.1 EPILOGUE).
  *   sol -- the four-step Speed-of-Light analysis of Section 4.1 and its worked
  *       report in Appendix A.2.
  *
@@ -45,7 +46,9 @@
 
 enum { ORC_ROW_MAJOR = 0, ORC_COL_MAJOR = 1 };
 enum { ORC_BF16 = 0, ORC_F32 = 1 };
-enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4 };
+enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4,
+       ORC_EPI_SIGMOID = 5, ORC_EPI_TANH = 6, ORC_EPI_MISH = 7, ORC_EPI_HARDSWISH = 8, ORC_EPI_LEAKY_RELU = 9,
+       ORC_EPI_ELU = 10, ORC_EPI_CLIP = 11 };
 
 /* Number of host threads the parallel loops use. */
 int orc_num_threads(void) {
@@ -70,10 +73,12 @@ static double load_as_f64(const void* p, int dtype, int64_t idx) {
 }
 
 /*
- * Activations of the fused epilogue (Table 1c built-ins relu, gelu, silu).
+ * Activations of the fused epilogue (Table 1c built-ins): relu, gelu (tanh form), silu, sigmoid, tanh,
+ * mish(x) = x tanh(ln(1 + e^x)), hardswish(x) = x min(max(x + 3, 0), 6) / 6, leaky_relu(x; a0) = x or a0 x,
+ * elu(x; a0) = x or a0 (e^x - 1), clip(x; a0, a1) = min(max(x, a0), a1).
  * BIAS and NONE are the identity: the bias itself is added by the caller.
  */
-double orc_act(int epi, double x) {
+double orc_act2(int epi, double x, double a0, double a1) {
     switch (epi) {
         case ORC_EPI_RELU:
             return x > 0.0 ? x : 0.0;
@@ -83,10 +88,29 @@ double orc_act(int epi, double x) {
         }
         case ORC_EPI_SILU:
             return x / (1.0 + exp(-x));
+        case ORC_EPI_SIGMOID:
+            return 1.0 / (1.0 + exp(-x));
+        case ORC_EPI_TANH:
+            return tanh(x);
+        case ORC_EPI_MISH:
+            return x * tanh(x > 30.0 ? x : log1p(exp(x)));
+        case ORC_EPI_HARDSWISH: {
+            double r = x + 3.0;
+            r = r < 0.0 ? 0.0 : (r > 6.0 ? 6.0 : r);
+            return x * r / 6.0;
+        }
+        case ORC_EPI_LEAKY_RELU:
+            return x > 0.0 ? x : a0 * x;
+        case ORC_EPI_ELU:
+            return x > 0.0 ? x : a0 * expm1(x);
+        case ORC_EPI_CLIP:
+            return x < a0 ? a0 : (x > a1 ? a1 : x);
         default:
             return x;
     }
 }
+
+double orc_act(int epi, double x) { return orc_act2(epi, x, 0.0, 0.0); }
 
 /* -------------------------------------------------------------------------------------------
  * GEMM.   a(i,k) = A[i*lda + k] (row-major) or A[k*lda + i] (column-major)
@@ -102,6 +126,7 @@ typedef struct {
     const uint16_t* bias;                        /* [N] or NULL */
     double alpha, beta;
     int epi;
+    double a0, a1;                               /* activation parameters */
 } gemm_problem;
 
 /* One output element and, optionally, the magnitude sum used to scale fp32 tolerances. */
@@ -126,7 +151,7 @@ static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* 
         av += fabs(bj);
     }
     if (absacc) *absacc = av;
-    return orc_act(g->epi, v);
+    return orc_act2(g->epi, v, g->a0, g->a1);
 }
 
 /*
@@ -136,11 +161,11 @@ static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* 
 int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
              const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
              const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
-             double alpha, double beta, int epi,
+             double alpha, double beta, int epi, double a0, double a1,
              int64_t row_begin, int64_t row_end, double* ref, double* absacc, int64_t ldr) {
     if (M < 0 || N < 0 || K < 0 || row_begin < 0 || row_end > M || row_begin > row_end) return 1;
     if (beta != 0.0 && !C) return 2;
-    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi};
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1};
 #pragma omp parallel for schedule(static)
     for (int64_t i = row_begin; i < row_end; ++i) {
         for (int64_t j = 0; j < N; ++j) {
@@ -157,10 +182,10 @@ int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
 int orc_gemm_points(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
                     const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
                     const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
-                    double alpha, double beta, int epi,
+                    double alpha, double beta, int epi, double a0, double a1,
                     int64_t npts, const int64_t* pi, const int64_t* pj, double* ref, double* absacc) {
     if (beta != 0.0 && !C) return 2;
-    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi};
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1};
     for (int64_t t = 0; t < npts; ++t)
         if (pi[t] < 0 || pi[t] >= M || pj[t] < 0 || pj[t] >= N) return 1;
 #pragma omp parallel for schedule(static)
@@ -188,6 +213,7 @@ typedef struct {
     const uint16_t* bias;
     double alpha, beta;
     int epi;
+    double a0, a1;
 } conv_problem;
 
 int64_t orc_conv_out_extent(int64_t in, int64_t pad, int64_t dil, int64_t filt, int64_t stride) {
@@ -226,11 +252,12 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
         av += fabs(bk);
     }
     if (absacc) *absacc = av;
-    return orc_act(cv->epi, v);
+    return orc_act2(cv->epi, v, cv->a0, cv->a1);
 }
 
 static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, const uint16_t* Wf,
-                      const void* Cin, int c_dtype, const uint16_t* bias, double alpha, double beta, int epi) {
+                      const void* Cin, int c_dtype, const uint16_t* bias, double alpha, double beta, int epi,
+                      double a0, double a1) {
     cv->N = d[0]; cv->H = d[1]; cv->W = d[2]; cv->C = d[3]; cv->K = d[4]; cv->R = d[5]; cv->S = d[6];
     cv->pad_h = d[7]; cv->pad_w = d[8]; cv->stride_h = d[9]; cv->stride_w = d[10];
     cv->dil_h = d[11]; cv->dil_w = d[12];
@@ -240,7 +267,7 @@ static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, con
     cv->P = orc_conv_out_extent(cv->H, cv->pad_h, cv->dil_h, cv->R, cv->stride_h);
     cv->Q = orc_conv_out_extent(cv->W, cv->pad_w, cv->dil_w, cv->S, cv->stride_w);
     cv->X = X; cv->Wf = Wf; cv->Cin = Cin; cv->c_dtype = c_dtype; cv->bias = bias;
-    cv->alpha = alpha; cv->beta = beta; cv->epi = epi;
+    cv->alpha = alpha; cv->beta = beta; cv->epi = epi; cv->a0 = a0; cv->a1 = a1;
     return 0;
 }
 
@@ -251,10 +278,10 @@ static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, con
  */
 int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
                      const void* Cin, int c_dtype, const uint16_t* bias,
-                     double alpha, double beta, int epi,
+                     double alpha, double beta, int epi, double a0, double a1,
                      int64_t pix_begin, int64_t pix_end, double* ref, double* absacc) {
     conv_problem cv;
-    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi);
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1);
     if (rc) return rc;
     if (pix_begin < 0 || pix_end > cv.N * cv.P * cv.Q || pix_begin > pix_end) return 1;
 #pragma omp parallel for schedule(static)
@@ -275,10 +302,10 @@ int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
 /* The listed (flattened pixel, output channel) pairs only. */
 int orc_conv2d_points(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
                       const void* Cin, int c_dtype, const uint16_t* bias,
-                      double alpha, double beta, int epi,
+                      double alpha, double beta, int epi, double a0, double a1,
                       int64_t npts, const int64_t* ppix, const int64_t* pk, double* ref, double* absacc) {
     conv_problem cv;
-    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi);
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1);
     if (rc) return rc;
     for (int64_t t = 0; t < npts; ++t)
         if (ppix[t] < 0 || ppix[t] >= cv.N * cv.P * cv.Q || pk[t] < 0 || pk[t] >= cv.K) return 1;

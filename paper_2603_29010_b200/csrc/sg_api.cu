@@ -212,12 +212,14 @@ struct Checked {
     int esize_out;
 };
 
-sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, int32_t reserved,
-                         Checked* c) {
+sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, float a0, float a1,
+                         int32_t reserved, Checked* c) {
     if (in_dtype != SG_BF16) return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: only SG_BF16 inputs are implemented", in_dtype);
     if (out_dtype != SG_BF16 && out_dtype != SG_F32) return fail(SG_ERR_INVALID_ARG, "out_dtype %d is not a sg_dtype_t", out_dtype);
-    if (epi < SG_EPI_NONE || epi > SG_EPI_SILU) return fail(SG_ERR_INVALID_ARG, "epi %d is not a sg_epilogue_t", epi);
+    if (epi < SG_EPI_NONE || epi > SG_EPI_CLIP) return fail(SG_ERR_INVALID_ARG, "epi %d is not a sg_epilogue_t", epi);
     if (!std::isfinite(alpha) || !std::isfinite(beta)) return fail(SG_ERR_INVALID_ARG, "alpha and beta must be finite");
+    if ((epi == SG_EPI_LEAKY_RELU || epi == SG_EPI_ELU) && !std::isfinite(a0)) return fail(SG_ERR_INVALID_ARG, "epi_arg0 (slope) must be finite");
+    if (epi == SG_EPI_CLIP && !(a0 <= a1)) return fail(SG_ERR_INVALID_ARG, "clip needs epi_arg0 <= epi_arg1");
     if (reserved != 0) return fail(SG_ERR_INVALID_ARG, "reserved field must be 0");
     c->f32_out = (out_dtype == SG_F32);
     c->esize_out = c->f32_out ? 4 : 2;
@@ -226,7 +228,7 @@ sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float
 
 sg_status_t check_gemm_desc(const sg_gemm_desc_t* d, bool grouped, Checked* c) {
     if (!d) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
-    sg_status_t st = check_common(d->in_dtype, d->out_dtype, d->epi, d->alpha, d->beta, d->reserved, c);
+    sg_status_t st = check_common(d->in_dtype, d->out_dtype, d->epi, d->alpha, d->beta, d->epi_arg0, d->epi_arg1, d->reserved, c);
     if (st != SG_OK) return st;
     if ((!grouped && d->M < 0) || d->N < 0 || d->K < 0) return fail(SG_ERR_INVALID_ARG, "M, N, K must be >= 0");
     if ((!grouped && d->M > INT32_MAX) || d->N > INT32_MAX || d->K > INT32_MAX)
@@ -416,11 +418,13 @@ sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params&
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait inside one launch
 
-void base_params(Params* p, const DeviceState& d, float alpha, float beta, int32_t epi) {
+void base_params(Params* p, const DeviceState& d, float alpha, float beta, int32_t epi, float a0, float a1) {
     memset(p, 0, sizeof *p);
     p->alpha = alpha;
     p->beta = beta;
     p->epi = epi;
+    p->epi_arg0 = a0;
+    p->epi_arg1 = a1;
     p->status = d.status_dev;
     p->timeout_ns = kWaitLimitNs;
 }
@@ -447,7 +451,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (st != SG_OK) return st;
 
     Params p;
-    base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
+    base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
     const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
     const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
@@ -687,7 +691,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     const int tiles_n = static_cast<int>((common->N + s.bn - 1) / s.bn);
 
     Params p;
-    base_params(&p, *d, common->alpha, common->beta, common->epi);
+    base_params(&p, *d, common->alpha, common->beta, common->epi, common->epi_arg0, common->epi_arg1);
     int64_t tiles = 0;
     for (int g = 0; g < groups; ++g) tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
@@ -800,7 +804,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
                             void* Y, void* cuda_stream) {
     if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
     Checked c;
-    sg_status_t st = check_common(desc->in_dtype, desc->out_dtype, desc->epi, desc->alpha, desc->beta, desc->reserved, &c);
+    sg_status_t st = check_common(desc->in_dtype, desc->out_dtype, desc->epi, desc->alpha, desc->beta, desc->epi_arg0, desc->epi_arg1,
+                                  desc->reserved, &c);
     if (st != SG_OK) return st;
     if (desc->N < 0 || desc->H < 0 || desc->W < 0 || desc->C < 0 || desc->K < 0 || desc->R < 1 || desc->S < 1)
         return fail(SG_ERR_INVALID_ARG, "sg_conv2d_fprop: extents must be >= 0 and the filter at least 1x1");
@@ -828,7 +833,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     st = device_state(&d);
     if (st != SG_OK) return st;
     Params p;
-    base_params(&p, *d, desc->alpha, desc->beta, desc->epi);
+    base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
     const Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_CONV;

@@ -21,7 +21,8 @@
 namespace sg {
 
 enum : int32_t { MODE_DENSE = 0, MODE_GROUPED = 1, MODE_CONV = 2 };
-enum : int32_t { EPI_NONE = 0, EPI_BIAS = 1, EPI_RELU = 2, EPI_GELU = 3, EPI_SILU = 4 };
+enum : int32_t { EPI_NONE = 0, EPI_BIAS = 1, EPI_RELU = 2, EPI_GELU = 3, EPI_SILU = 4, EPI_SIGMOID = 5, EPI_TANH = 6,
+                 EPI_MISH = 7, EPI_HARDSWISH = 8, EPI_LEAKY_RELU = 9, EPI_ELU = 10, EPI_CLIP = 11 };
 
 // status word 0: 0 = fine, else (role << 24 | detail); words 1..3 hold tile / barrier / block of the first failure
 enum : uint32_t { ROLE_PRODUCER = 1, ROLE_MMA = 2, ROLE_EPILOGUE = 3, ROLE_SETUP = 4 };
@@ -50,6 +51,7 @@ struct alignas(64) Params {
     uint32_t* sk_flags;                 // K-split scratch: [buffer] arrival counters, then [tail tile] consumed counters
     int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
     float alpha, beta;
+    float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
     int32_t epi, mode;
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
@@ -181,13 +183,14 @@ __device__ __forceinline__ float tanh_approx(float x) {
 #define SG_FAST_ACT 1
 #endif
 template <bool kFast>
-__device__ __forceinline__ float apply_act(float v, int epi) {
+__device__ __forceinline__ float apply_act(float v, int epi, float a0, float a1) {
+    constexpr bool fast = kFast && SG_FAST_ACT;
     switch (epi) {
         case EPI_RELU:
             return fmaxf(v, 0.0f);
         case EPI_GELU: {
             const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
-            if constexpr (kFast && SG_FAST_ACT) {
+            if constexpr (fast) {
                 const float h = 0.5f * v;
                 return fmaf(h, tanh_approx(u), h);
             } else {
@@ -195,13 +198,33 @@ __device__ __forceinline__ float apply_act(float v, int epi) {
             }
         }
         case EPI_SILU: {
-            if constexpr (kFast && SG_FAST_ACT) {
+            if constexpr (fast) {
                 const float h = 0.5f * v;
                 return fmaf(h, tanh_approx(h), h);
             } else {
                 return __fdividef(v, 1.0f + __expf(-v));
             }
         }
+        case EPI_SIGMOID:
+            if constexpr (fast) return fmaf(0.5f, tanh_approx(0.5f * v), 0.5f);
+            else return __fdividef(1.0f, 1.0f + __expf(-v));
+        case EPI_TANH:
+            if constexpr (fast) return tanh_approx(v);
+            else return tanhf(v);
+        case EPI_MISH: {
+            // x tanh(softplus(x)); softplus(x) = x beyond 20 (e^-20 is below fp32 resolution next to x)
+            if constexpr (fast) return v * tanh_approx(v > 20.0f ? v : __logf(1.0f + __expf(v)));
+            else return v * tanhf(v > 20.0f ? v : log1pf(expf(v)));
+        }
+        case EPI_HARDSWISH:
+            return v * fminf(fmaxf(v + 3.0f, 0.0f), 6.0f) * (1.0f / 6.0f);
+        case EPI_LEAKY_RELU:
+            return v > 0.0f ? v : a0 * v;
+        case EPI_ELU:
+            if constexpr (fast) return v > 0.0f ? v : a0 * (__expf(v) - 1.0f);
+            else return v > 0.0f ? v : a0 * expm1f(v);
+        case EPI_CLIP:
+            return fminf(fmaxf(v, a0), a1);
         default:
             return v;
     }
@@ -675,7 +698,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 if (epi >= EPI_RELU) {
 #pragma unroll
-                    for (int i = 0; i < CH; ++i) v[i] = apply_act<!kOutF32>(v[i], epi);
+                    for (int i = 0; i < CH; ++i) v[i] = apply_act<!kOutF32>(v[i], epi, p.epi_arg0, p.epi_arg1);
                 }
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes

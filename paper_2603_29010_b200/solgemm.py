@@ -30,7 +30,8 @@ SG_OK = 0
 STATUS_NAMES = ["SG_OK", "SG_ERR_INVALID_ARG", "SG_ERR_NULL_POINTER", "SG_ERR_ALIGNMENT", "SG_ERR_UNSUPPORTED",
                 "SG_ERR_ARCH", "SG_ERR_WORKSPACE", "SG_ERR_CUDA", "SG_ERR_TIMEOUT"]
 LAYOUTS = {"row": 0, "col": 1}
-EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4}
+EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
+             "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
 DTYPES = {torch.bfloat16: 0, torch.float32: 1}
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
@@ -54,7 +55,8 @@ class GemmDesc(ctypes.Structure):
                 ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64), ("ldd", ctypes.c_int64),
                 ("in_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
                 ("alpha", ctypes.c_float), ("beta", ctypes.c_float),
-                ("epi", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("epi", ctypes.c_int32), ("epi_arg0", ctypes.c_float), ("epi_arg1", ctypes.c_float),
+                ("reserved", ctypes.c_int32)]
 
 
 class Conv2dDesc(ctypes.Structure):
@@ -62,7 +64,7 @@ class Conv2dDesc(ctypes.Structure):
                [(n, ctypes.c_int32) for n in ("pad_h", "pad_w", "stride_h", "stride_w", "dil_h", "dil_w",
                                               "in_dtype", "out_dtype")] + \
                [("alpha", ctypes.c_float), ("beta", ctypes.c_float), ("epi", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("epi_arg0", ctypes.c_float), ("epi_arg1", ctypes.c_float), ("reserved", ctypes.c_int32)]
 
 
 class Hw(ctypes.Structure):
@@ -169,9 +171,10 @@ def _ld(t: torch.Tensor) -> int:
     return t.stride(0) if t.shape[0] > 1 else max(t.shape[1], 1)
 
 
-def _gemm_desc(M, N, K, lda, ldb, ldc, ldd, layout_a, layout_b, out_dtype, alpha, beta, epi) -> GemmDesc:
+def _gemm_desc(M, N, K, lda, ldb, ldc, ldd, layout_a, layout_b, out_dtype, alpha, beta, epi,
+               epi_args=(0.0, 0.0)) -> GemmDesc:
     return GemmDesc(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], lda, ldb, ldc, ldd, 0, DTYPES[out_dtype],
-                    float(alpha), float(beta), EPILOGUES[epi], 0)
+                    float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), 0)
 
 
 def _mnk(A, B, layout_a, layout_b):
@@ -184,20 +187,22 @@ def _mnk(A, B, layout_a, layout_b):
 
 def gemm(A: torch.Tensor, B: torch.Tensor, *, C: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
          out: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.bfloat16, alpha: float = 1.0,
-         beta: float = 0.0, epi: str = "none", layout_a: str = "row", layout_b: str = "col", stream=None) -> torch.Tensor:
+         beta: float = 0.0, epi: str = "none", epi_args=(0.0, 0.0), layout_a: str = "row", layout_b: str = "col",
+         stream=None) -> torch.Tensor:
     """D = act(alpha A.B + beta C + bias) through ``sg_gemm``.  Returns D (``out`` if given)."""
     M, N, K = _mnk(A, B, layout_a, layout_b)
     ensure_scratch()
     if out is None:
         out = torch.empty((M, N), dtype=out_dtype, device=A.device)
     desc = _gemm_desc(M, N, K, _ld(A), _ld(B), _ld(C) if C is not None else max(N, 1), _ld(out), layout_a, layout_b,
-                      out.dtype, alpha, beta, epi)
+                      out.dtype, alpha, beta, epi, epi_args)
     _check(_lib.sg_gemm(ctypes.byref(desc), _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
     return out
 
 
 def batched_gemm(A: torch.Tensor, B: torch.Tensor, *, C=None, bias=None, out=None, out_dtype=torch.bfloat16,
-                 alpha=1.0, beta=0.0, epi="none", layout_a="row", layout_b="col", stream=None) -> torch.Tensor:
+                 alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0), layout_a="row", layout_b="col",
+                 stream=None) -> torch.Tensor:
     """The same product for every leading index through ``sg_batched_gemm``; ``bias`` is [N] or [batch, N]."""
     batch = A.shape[0]
     M, N, K = _mnk(A, B, layout_a, layout_b)
@@ -209,7 +214,7 @@ def batched_gemm(A: torch.Tensor, B: torch.Tensor, *, C=None, bias=None, out=Non
             raise ValueError("batched operands must be 3-D with inner stride 1")
     sbias = 0 if bias is None or bias.dim() == 1 else bias.stride(0)
     desc = _gemm_desc(M, N, K, A.stride(1), B.stride(1), C.stride(1) if C is not None else max(N, 1), out.stride(1),
-                      layout_a, layout_b, out.dtype, alpha, beta, epi)
+                      layout_a, layout_b, out.dtype, alpha, beta, epi, epi_args)
     _check(_lib.sg_batched_gemm(ctypes.byref(desc), batch, A.stride(0), B.stride(0),
                                 C.stride(0) if C is not None else 0, out.stride(0), sbias,
                                 _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
@@ -233,8 +238,8 @@ def _ptr_array(tensors: Optional[Sequence[Optional[torch.Tensor]]]):
 
 def grouped_gemm(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=None, biases=None,
                  outs: Optional[Sequence[torch.Tensor]] = None, out_dtype=torch.bfloat16, alpha=1.0, beta=0.0,
-                 epi="none", layout_a="row", layout_b="col", workspace: Optional[torch.Tensor] = None,
-                 stream=None) -> List[torch.Tensor]:
+                 epi="none", epi_args=(0.0, 0.0), layout_a="row", layout_b="col",
+                 workspace: Optional[torch.Tensor] = None, stream=None) -> List[torch.Tensor]:
     """One launch of ``sg_grouped_gemm`` over groups with their own M_g; N, K and leading dimensions are common."""
     groups = len(As)
     if groups == 0:
@@ -246,7 +251,7 @@ def grouped_gemm(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=N
         outs = [torch.empty((m, N), dtype=out_dtype, device=As[0].device) for m in Ms]
     ld = lambda ts, default: next((_ld(t) for t in ts if t.shape[0] > 1), default)
     desc = _gemm_desc(0, N, K, ld(As, max(K, 1)), ld(Bs, max(K, 1)), ld(Cs, max(N, 1)) if Cs is not None else max(N, 1),
-                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi)
+                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi, epi_args)
     if workspace is None:
         workspace = torch.empty(grouped_workspace_size(groups), dtype=torch.uint8, device=As[0].device)
     m_arr = (ctypes.c_int64 * groups)(*Ms)
@@ -260,8 +265,8 @@ STATIC_MAX_GROUPS = 64
 
 
 def grouped_gemm_static(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=None, biases=None,
-                        outs: Sequence[torch.Tensor], alpha=1.0, beta=0.0, epi="none", layout_a="row", layout_b="col",
-                        stream=None) -> List[torch.Tensor]:
+                        outs: Sequence[torch.Tensor], alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0),
+                        layout_a="row", layout_b="col", stream=None) -> List[torch.Tensor]:
     """``sg_grouped_gemm_static``: the grouped product for callers that may not allocate device memory.
 
     Unlike :func:`grouped_gemm` this wrapper allocates nothing either: ``outs`` must be given, and the
@@ -275,7 +280,7 @@ def grouped_gemm_static(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], 
     Ms = [(_mnk(a, b, layout_a, layout_b))[0] for a, b in zip(As, Bs)]
     ld = lambda ts, default: next((_ld(t) for t in ts if t.shape[0] > 1), default)
     desc = _gemm_desc(0, N, K, ld(As, max(K, 1)), ld(Bs, max(K, 1)), ld(Cs, max(N, 1)) if Cs is not None else max(N, 1),
-                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi)
+                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi, epi_args)
     m_arr = (ctypes.c_int64 * groups)(*Ms)
     _check(_lib.sg_grouped_gemm_static(ctypes.byref(desc), groups, m_arr, _ptr_array(As), _ptr_array(Bs),
                                        _ptr_array(Cs), _ptr_array(biases), _ptr_array(outs), _stream(stream)))
@@ -283,7 +288,8 @@ def grouped_gemm_static(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], 
 
 
 def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1), dil=(1, 1), Cin=None, bias=None,
-                 out=None, out_dtype=torch.bfloat16, alpha=1.0, beta=0.0, epi="none", stream=None) -> torch.Tensor:
+                 out=None, out_dtype=torch.bfloat16, alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0),
+                 stream=None) -> torch.Tensor:
     """NHWC x KRSC -> NPQK forward convolution through ``sg_conv2d_fprop`` (implicit GEMM, nothing materialised)."""
     if X.dim() != 4 or Wf.dim() != 4 or not X.is_contiguous() or not Wf.is_contiguous():
         raise ValueError("X (NHWC) and Wf (KRSC) must be contiguous 4-D tensors")
@@ -297,7 +303,7 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
     if out is None:
         out = torch.empty((N, P, Q, K), dtype=out_dtype, device=X.device)
     desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], 0, DTYPES[out.dtype],
-                      float(alpha), float(beta), EPILOGUES[epi], 0)
+                      float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), 0)
     _check(_lib.sg_conv2d_fprop(ctypes.byref(desc), _ptr(X), _ptr(Wf), _ptr(Cin), _ptr(bias), _ptr(out), _stream(stream)))
     return out
 
@@ -333,9 +339,9 @@ def sol_bound(op: str, *, M=0, N=0, K=0, batch_or_groups=1, Ms: Optional[Sequenc
     if op == "conv2d":
         c = conv
         desc = Conv2dDesc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], *c.get("pad", (0, 0)),
-                          *c.get("stride", (1, 1)), *c.get("dil", (1, 1)), 0, 0, 1.0, float(beta), 0, 0)
+                          *c.get("stride", (1, 1)), *c.get("dil", (1, 1)), 0, 0, 1.0, float(beta), 0, 0.0, 0.0, 0)
     else:
-        desc = GemmDesc(M, N, K, 0, 1, max(K, 1), max(K, 1), max(N, 1), max(N, 1), 0, 0, 1.0, float(beta), 0, 0)
+        desc = GemmDesc(M, N, K, 0, 1, max(K, 1), max(K, 1), max(N, 1), max(N, 1), 0, 0, 1.0, float(beta), 0, 0.0, 0.0, 0)
     m_arr = (ctypes.c_int64 * len(Ms))(*Ms) if Ms is not None else None
     hw = Hw(peak_flops, peak_bytes_per_s, sm_clock_mhz, sm_clock_max_mhz, mem_clock_mhz, mem_clock_max_mhz)
     out = Sol()

@@ -140,6 +140,48 @@ def test_gemm_epilogues_alpha_beta_bias(epi, out_dtype, pair):
         parity.assert_matches(D2, ref2, acc2, f"gemm epi={epi} no bias {out_dtype}")
 
 
+FURTHER_ACTS = [("sigmoid", (0.0, 0.0)), ("tanh", (0.0, 0.0)), ("mish", (0.0, 0.0)), ("hardswish", (0.0, 0.0)),
+                ("leaky_relu", (0.125, 0.0)), ("elu", (1.5, 0.0)), ("clip", (-0.5, 2.0))]
+
+
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("epi,args", FURTHER_ACTS)
+def test_further_builtin_activations(epi, args, out_dtype):
+    M, N, K = 200, 136, 264
+    A, B, bias = inputs.make_gemm(M, N, K, "normal", K ** -0.25, bias=True, seed=515)
+    ref, absacc = orc.gemm(A, B, bias=bias, alpha=1.5, epi=epi, epi_args=args)
+    D = sg.gemm(A.to(DEV), B.to(DEV), bias=bias.to(DEV), alpha=1.5, epi=epi, epi_args=args, out_dtype=out_dtype)
+    parity.assert_matches(D, ref, absacc, f"{epi} {out_dtype}")
+    # K = 1 on the fp32 path: D = act(x) judged at 1e-4 |x|, over a range that reaches every branch
+    x = torch.linspace(-9, 9, 512, dtype=torch.float64).to(torch.bfloat16).view(-1, 1)
+    a = torch.zeros(512, 8, dtype=torch.bfloat16)
+    a[:, :1] = x
+    b = torch.zeros(8, 8, dtype=torch.bfloat16)
+    b[:, 0] = 1
+    ref1, acc1 = orc.gemm(a, b, epi=epi, epi_args=args)
+    D1 = sg.gemm(a.to(DEV), b.to(DEV), out_dtype=torch.float32, epi=epi, epi_args=args)
+    parity.assert_matches(D1, ref1, acc1, f"{epi} pointwise fp32")
+    Dbf = sg.gemm(a.to(DEV), b.to(DEV), epi=epi, epi_args=args)
+    parity.assert_matches(Dbf, ref1, acc1, f"{epi} pointwise bf16")
+
+
+def test_further_activations_through_conv_batched_and_grouped():
+    X, Wf, cb = inputs.make_conv(2, 9, 10, 40, 72, 3, 3, "normal", (40 * 9) ** -0.25, bias=True, seed=525)
+    ref, absacc = orc.conv2d_fprop(X, Wf, pad=(1, 1), bias=cb, epi="clip", epi_args=(0.0, 6.0))
+    Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1), bias=cb.to(DEV), epi="clip", epi_args=(0.0, 6.0))
+    parity.assert_matches(Y, ref, absacc, "conv + bias + clip(0, 6)")
+    A = inputs.uniform([3, 72, 136], 535, 1)
+    B = inputs.uniform([3, 64, 136], 535, 2)
+    ref, absacc = orc.batched_gemm(A, B, epi="leaky_relu", epi_args=(0.01, 0.0))
+    D = sg.batched_gemm(A.to(DEV), B.to(DEV), epi="leaky_relu", epi_args=(0.01, 0.0), out_dtype=torch.float32)
+    parity.assert_matches(D, ref, absacc, "batched leaky_relu")
+    As, Bs = inputs.make_grouped([40, 130], 72, 136, "normal", 136 ** -0.25, seed=545)
+    refs, accs = orc.grouped_gemm(As, Bs, epi="mish")
+    outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs], epi="mish")
+    for g in range(2):
+        parity.assert_matches(outs[g], refs[g], accs[g], f"grouped mish {g}")
+
+
 def test_gemm_activation_form_is_pinned_on_the_fp32_path():
     # K = 1: D = act(x), tolerance 1e-4 |x| -- tight enough to tell tanh-GELU from erf-GELU
     x = torch.linspace(-6, 6, 256, dtype=torch.float64).to(torch.bfloat16).view(-1, 1)

@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(sg):
 
 
 def test_struct_layouts_match_the_header(sg):
-    assert ctypes.sizeof(sg.GemmDesc) == 88 and ctypes.sizeof(sg.Conv2dDesc) == 104
+    assert ctypes.sizeof(sg.GemmDesc) == 96 and ctypes.sizeof(sg.Conv2dDesc) == 112
     assert ctypes.sizeof(sg.Hw) == 48 and ctypes.sizeof(sg.Sol) == 80
 
 
@@ -43,7 +43,7 @@ def test_status_strings(sg):
 
 def _desc(sg, **kw):
     base = dict(M=128, N=128, K=128, layout_a=0, layout_b=1, lda=128, ldb=128, ldc=128, ldd=128, in_dtype=0,
-                out_dtype=0, alpha=1.0, beta=0.0, epi=0, reserved=0)
+                out_dtype=0, alpha=1.0, beta=0.0, epi=0, epi_arg0=0.0, epi_arg1=0.0, reserved=0)
     base.update(kw)
     return sg.GemmDesc(*[base[n] for n, _ in sg.GemmDesc._fields_])
 
@@ -55,7 +55,9 @@ def _call_gemm(sg, desc, A=0x1000, B=0x2000, C=None, bias=None, D=0x3000):
 @pytest.mark.parametrize("kw,ptrs,want", [
     (dict(M=-1), {}, "SG_ERR_INVALID_ARG"),
     (dict(lda=64), {}, "SG_ERR_INVALID_ARG"),
-    (dict(epi=9), {}, "SG_ERR_INVALID_ARG"),
+    (dict(epi=12), {}, "SG_ERR_INVALID_ARG"),
+    (dict(epi=11, epi_arg0=1.0, epi_arg1=0.0), {}, "SG_ERR_INVALID_ARG"),      # clip with min > max
+    (dict(epi=9, epi_arg0=float("nan")), {}, "SG_ERR_INVALID_ARG"),
     (dict(out_dtype=5), {}, "SG_ERR_INVALID_ARG"),
     (dict(reserved=1), {}, "SG_ERR_INVALID_ARG"),
     (dict(lda=132), {}, "SG_ERR_ALIGNMENT"),             # 264 bytes: not a multiple of 16
@@ -110,7 +112,7 @@ def test_grouped_and_conv_validation(sg):
 
     def conv(**kw):
         base = dict(N=1, H=8, W=8, C=64, K=64, R=3, S=3, pad_h=1, pad_w=1, stride_h=1, stride_w=1, dil_h=1, dil_w=1,
-                    in_dtype=0, out_dtype=0, alpha=1.0, beta=0.0, epi=0, reserved=0)
+                    in_dtype=0, out_dtype=0, alpha=1.0, beta=0.0, epi=0, epi_arg0=0.0, epi_arg1=0.0, reserved=0)
         base.update(kw)
         return sg.Conv2dDesc(*[base[k] for k, _ in sg.Conv2dDesc._fields_])
 

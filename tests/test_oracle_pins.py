@@ -221,6 +221,35 @@ def test_activations_match_torch_library_fp64():
         assert torch.allclose(got, fn(xs), rtol=1e-13, atol=1e-15), name
 
 
+def test_further_activations_closed_forms_and_library():
+    F = torch.nn.functional
+    xs = torch.linspace(-7, 7, 113, dtype=torch.float64)
+    table = [("sigmoid", (0, 0), torch.sigmoid), ("tanh", (0, 0), torch.tanh), ("mish", (0, 0), F.mish),
+             ("hardswish", (0, 0), F.hardswish), ("leaky_relu", (0.125, 0), lambda t: F.leaky_relu(t, 0.125)),
+             ("elu", (1.5, 0), lambda t: F.elu(t, 1.5)), ("clip", (-0.5, 2.0), lambda t: torch.clamp(t, -0.5, 2.0))]
+    for name, args, fn in table:
+        got = torch.tensor([orc.act(name, float(x), args) for x in xs], dtype=torch.float64)
+        assert torch.allclose(got, fn(xs), rtol=1e-13, atol=1e-15), name
+    # hand values and identities
+    assert orc.act("sigmoid", 0.0) == 0.5 and orc.act("tanh", 0.0) == 0.0 and orc.act("mish", 0.0) == 0.0
+    assert orc.act("sigmoid", 2.0) + orc.act("sigmoid", -2.0) == pytest.approx(1.0, rel=1e-15)
+    assert orc.act("hardswish", -3.0) == 0.0 and orc.act("hardswish", 3.0) == 3.0 and orc.act("hardswish", 1.0) == pytest.approx(4.0 / 6.0)
+    assert orc.act("leaky_relu", -4.0, (0.25, 0)) == -1.0 and orc.act("leaky_relu", 4.0, (0.25, 0)) == 4.0
+    assert orc.act("elu", -1.0, (2.0, 0)) == pytest.approx(2.0 * (math.exp(-1.0) - 1.0), rel=1e-15) and orc.act("elu", 3.0, (2.0, 0)) == 3.0
+    assert orc.act("clip", 7.0, (0.0, 6.0)) == 6.0 and orc.act("clip", -1.0, (0.0, 6.0)) == 0.0 and orc.act("clip", 2.5, (0.0, 6.0)) == 2.5
+    assert orc.act("mish", 1.0) == pytest.approx(math.tanh(math.log(1.0 + math.e)), rel=1e-15)
+    assert orc.act("mish", 40.0) == 40.0 and abs(orc.act("mish", -40.0)) < 1e-15
+    # the parameters reach the GEMM and convolution entry points
+    A, Bt = bf([[1, -2]]), bf([[1, 1], [2, -1]])
+    ref, _ = orc.gemm(A, Bt, epi="leaky_relu", epi_args=(0.5, 0))
+    assert ref.tolist() == [[-0.5, 4.0]]
+    ref, _ = orc.gemm(A, Bt, epi="clip", epi_args=(-0.25, 3.0))
+    assert ref.tolist() == [[-0.25, 3.0]]
+    X, Wf = bf([[1, -2]]).view(1, 1, 1, 2), bf([[1, 1], [2, -1]]).view(2, 1, 1, 2)
+    ref, _ = orc.conv2d_fprop(X, Wf, epi="elu", epi_args=(1.0, 0))
+    assert ref.view(-1).tolist() == [pytest.approx(math.expm1(-1.0)), 4.0]
+
+
 # ---------------------------------------------------------------- convolution
 
 def test_conv_tiny_hand_computed():

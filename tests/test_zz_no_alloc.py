@@ -57,7 +57,7 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
 def test_static_scratch_rejects_too_many_groups():
     lib = sg.raw_lib()
     n = sg.STATIC_MAX_GROUPS + 1
-    desc = sg.GemmDesc(0, 64, 64, 0, 1, 64, 64, 64, 64, 0, 0, 1.0, 0.0, 0, 0)
+    desc = sg.GemmDesc(0, 64, 64, 0, 1, 64, 64, 64, 64, 0, 0, 1.0, 0.0, 0, 0.0, 0.0, 0)
     Ms = (ctypes.c_int64 * n)(*([64] * n))
     ptrs = (ctypes.c_void_p * n)(*([0x1000] * n))
     launches = sg.launch_count()
