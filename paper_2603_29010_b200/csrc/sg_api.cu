@@ -318,7 +318,7 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
 // cut into `split` column slices so that the idle SMs of that wave take a share.  Narrow slices cost more
 // per output area (same factors as in choose_shape), so a split is used only when it shortens the tail.
 // Sets p->split_begin, p->split and p->num_tiles (the length of the tile list) from the full-width count.
-void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1) {
+void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1) {
     const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
     int best_split = 1, best_ksplit = 1;
@@ -343,22 +343,34 @@ void plan_tail(const DeviceState& d, const Shape& s, int64_t full_tiles, Params*
             best_split = (s.bn / forced >= 64 && s.bn / forced / (s.pair ? 2 : 1) >= min_b_rows) ? forced : 1;
             best = 0.9;
         }
-        // K-split through the registered scratch: ksplit SM groups share one tail tile's K loop; the owner adds the
-        // helpers' fp32 partial tiles in its epilogue.  Costs the partials' round trip through L2 (~0.1 tile).
+        // K ranges through the registered scratch: ksplit SM groups share one tail tile's K loop and the owner adds
+        // the helpers' fp32 partial tiles in its epilogue (this is also what serves skinny problems with a long K:
+        // when there is less than one wave of tiles, every tile is a "tail" tile).  Measured cost of the exchange:
+        // about 8 us for the dump, wait and first partial plus 1 us per further partial, whatever the tile's K; a
+        // k-block of a tile takes about 0.25 us.  A split is planned when it saves a fifth of the tail's time.
         if (d.scratch && forced_k != 0 && p->num_kb >= 2 && rem * 2 <= slots) {
-            int64_t ks = slots / rem;
-            if (ks > 4) ks = 4;
-            if (ks > p->num_kb) ks = p->num_kb;
-            if (forced_k >= 2 && forced_k <= ks) ks = forced_k;
+            int64_t ks_max = slots / rem;
+            if (ks_max > 16) ks_max = 16;
+            if (ks_max > p->num_kb) ks_max = p->num_kb;
             const size_t buf_bytes = static_cast<size_t>(s.pair ? 2 : 1) * 128 * s.bn * sizeof(float);
             size_t max_buffers = d.scratch_bytes > kScratchFlagBytes ? (d.scratch_bytes - kScratchFlagBytes) / buf_bytes : 0;
             if (max_buffers > static_cast<size_t>(kScratchMaxBuffers)) max_buffers = kScratchMaxBuffers;
-            // measured: helpers' dump, the owner's wait and its reads of the partials cost about 0.45 of a tile
-            const double cost = 1.0 / static_cast<double>(ks) + 0.45;
-            // The exchange costs a fixed ~10 us whatever the tile's K, so it can only pay for very long K loops.
-            const bool long_k = p->num_kb / ks >= 64;
-            if (ks >= 2 && static_cast<size_t>(rem * (ks - 1)) <= max_buffers && rem <= kScratchMaxBuffers &&
-                ((cost < best - 0.05 && long_k) || forced_k >= 2)) {
+            while (ks_max >= 2 && static_cast<size_t>(rem * (ks_max - 1)) > max_buffers) --ks_max;
+            int64_t ks = 0;
+            if (forced_k >= 2) {
+                ks = forced_k < ks_max ? forced_k : ks_max;
+            } else if (rem <= kScratchMaxBuffers) {
+                const double t_tile = 0.25 * p->num_kb * best;      // us: the tail as planned so far (whole or sliced)
+                double best_time = t_tile * 0.8;
+                for (int64_t k = 2; k <= ks_max; ++k) {
+                    const double t = 0.25 * p->num_kb / static_cast<double>(k) + 8.0 + 1.0 * static_cast<double>(k - 1);
+                    if (t < best_time) {
+                        best_time = t;
+                        ks = k;
+                    }
+                }
+            }
+            if (ks >= 2 && rem <= kScratchMaxBuffers) {
                 best_ksplit = static_cast<int>(ks);
                 best_split = 1;
             }
@@ -453,7 +465,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
     const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
-    const Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
+    Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_DENSE;
     p.a_mn_major = desc->layout_a == SG_COL_MAJOR ? 1 : 0;
@@ -686,7 +698,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     st = device_state(&d);
     if (st != SG_OK) return st;
     const int min_b_rows = common->layout_b == SG_ROW_MAJOR ? 64 : 1;
-    const Shape s = choose_shape(*d, rows, 1, common->N, common->K, min_b_rows);
+    Shape s = choose_shape(*d, rows, 1, common->N, common->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
     const int tiles_n = static_cast<int>((common->N + s.bn - 1) / s.bn);
 
@@ -834,7 +846,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     if (st != SG_OK) return st;
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
-    const Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
+    Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_CONV;
     p.M = static_cast<int32_t>(Mg);
