@@ -183,6 +183,27 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
                             const void* Cin, const void* bias, void* Y, void* cuda_stream);
 
 /*
+ * sg_transpose: out[b][c][r] = convert(in[b][r][c]) for b < batch, r < rows, c < cols -- the layout-transpose
+ * stage with fused dtype conversion that the DSL's pipeline(transpose(...), kernel, transpose(...)) places
+ * around a kernel (Section 3 "Multi-stage pipelines"; Appendix A.1 transpose_op: NCL <-> NLC, and
+ * NCHW <-> NHWC "implemented by flattening HW": batch = N, rows = C, cols = H*W or the reverse).
+ *   in   device, in_dtype (bf16 or fp32), [batch][rows][cols], row stride ld_in, batch stride stride_in (elements)
+ *   out  device, out_dtype (bf16 or fp32), [batch][cols][rows], row stride ld_out, batch stride stride_out
+ *   fp32 -> bf16 rounds to nearest even; bf16 -> fp32 is exact.  in and out must not overlap.
+ * Base pointers 16-byte aligned, ld and strides multiples of 16 bytes, ld_in >= cols, ld_out >= rows.
+ * An empty extent returns SG_OK without a launch.  A memory-bound kernel: its Speed-of-Light time is
+ * batch*rows*cols*(input + output element bytes) / bandwidth (sg_sol_bound, SG_OP_TRANSPOSE).
+ */
+typedef struct sg_transpose_desc {
+    int64_t batch, rows, cols;
+    int64_t ld_in, ld_out, stride_in, stride_out;
+    int32_t in_dtype, out_dtype;  /* sg_dtype_t */
+    int32_t reserved, reserved2;  /* must be 0 */
+} sg_transpose_desc_t;
+
+sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* out, void* cuda_stream);
+
+/*
  * Speed-of-Light bound (paper: Section 4.1 steps 1-4; worked example in Appendix A.2).
  * Host-only, pure function of its arguments.
  *   flops = 2 per multiply-accumulate of the contraction (halo taps of a padded conv included;
@@ -193,7 +214,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
  *   t_compute = flops / eff_peak, t_mem = bytes / eff_bandwidth, t_sol = max of the two;
  *   ai = flops / bytes, ridge = eff_peak / eff_bandwidth, compute_bound = ai > ridge.
  *   op                SG_OP_GEMM / SG_OP_BATCHED / SG_OP_GROUPED: desc is sg_gemm_desc_t;
- *                     SG_OP_CONV2D: desc is sg_conv2d_desc_t.
+ *                     SG_OP_CONV2D: desc is sg_conv2d_desc_t; SG_OP_TRANSPOSE: desc is sg_transpose_desc_t
+ *                     (flops = 0; element sizes come from its dtypes, elem_bytes_* are ignored).
  *   batch_or_groups   batch count (BATCHED), group count (GROUPED), ignored otherwise.
  *   M_host            [groups] for GROUPED (desc->M ignored), else may be NULL.
  *   has_bias          0 none; 1 one bias vector per problem; for BATCHED, 2 = one shared vector.
@@ -210,7 +232,7 @@ typedef struct sg_sol {
     int32_t reserved;
 } sg_sol_t;
 
-typedef enum { SG_OP_GEMM = 0, SG_OP_BATCHED = 1, SG_OP_GROUPED = 2, SG_OP_CONV2D = 3 } sg_op_t;
+typedef enum { SG_OP_GEMM = 0, SG_OP_BATCHED = 1, SG_OP_GROUPED = 2, SG_OP_CONV2D = 3, SG_OP_TRANSPOSE = 4 } sg_op_t;
 
 sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, const int64_t* M_host,
                          int32_t elem_bytes_in, int32_t elem_bytes_out, int32_t has_bias,

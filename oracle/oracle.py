@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, i64, i64, vp, vp]
         L.orc_conv2d_points.restype = ci
         L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, i64, vp, vp, vp, vp]
+        L.orc_transpose.restype = ci
+        L.orc_transpose.argtypes = [i64, i64, i64, vp, ci, i64, i64, ci, vp]
+        L.orc_transpose_bytes.restype = i64
+        L.orc_transpose_bytes.argtypes = [i64] * 5
         L.orc_gemm_flops.restype = i64
         L.orc_gemm_flops.argtypes = [i64, i64, i64]
         L.orc_gemm_bytes.restype = i64
@@ -256,6 +260,23 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
     if rc:
         raise ValueError(f"orc_conv2d_points rejected its arguments (code {rc})")
     return ref, absacc
+
+
+def transpose(x: torch.Tensor, out_dtype: torch.dtype) -> torch.Tensor:
+    """out[b, c, r] = convert(x[b, r, c]) as fp64 values of the converted result; x is [batch, rows, cols]."""
+    if x.device.type != "cpu" or x.dim() != 3 or x.dtype not in _DTYPES or (x.shape[2] > 1 and x.stride(2) != 1):
+        raise ValueError("x: want a CPU [batch, rows, cols] bf16 or fp32 tensor with inner stride 1")
+    batch, rows, cols = x.shape
+    out = torch.empty((batch, cols, rows), dtype=torch.float64)
+    rc = lib().orc_transpose(batch, rows, cols, _ptr(x), _DTYPES[x.dtype], x.stride(1) if rows > 1 else max(cols, 1),
+                             x.stride(0), _DTYPES[out_dtype], _ptr(out))
+    if rc:
+        raise ValueError(f"orc_transpose rejected its arguments (code {rc})")
+    return out
+
+
+def transpose_bytes(batch: int, rows: int, cols: int, eb_in: int, eb_out: int) -> int:
+    return int(lib().orc_transpose_bytes(batch, rows, cols, eb_in, eb_out))
 
 
 # ---- Speed-of-Light bound -------------------------------------------------------------------

@@ -320,6 +320,43 @@ int orc_conv2d_points(const int64_t* dims, const uint16_t* X, const uint16_t* Wf
 }
 
 /* -------------------------------------------------------------------------------------------
+ * Layout transpose with dtype conversion (the DSL's transpose(ref, L1, L2[, dt1, dt2]) stage, Appendix A.1):
+ *   out[b][c][r] = convert(in[b][r][c]).  bf16 -> fp32 is exact; fp32 -> bf16 rounds to nearest, ties to even
+ *   (the 16 discarded bits decide; a NaN stays a NaN).  The result is returned as fp64 holding the converted value.
+ * ----------------------------------------------------------------------------------------- */
+static double round_f32_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu) != 0) {
+        u |= 0x00400000u;                       /* quiet NaN, keep it a NaN after truncation */
+    } else {
+        uint32_t lower = u & 0xFFFFu, odd = (u >> 16) & 1u;
+        if (lower > 0x8000u || (lower == 0x8000u && odd)) u += 0x10000u;   /* may carry into the exponent: correct */
+    }
+    u &= 0xFFFF0000u;
+    float r;
+    memcpy(&r, &u, sizeof r);
+    return (double)r;
+}
+
+int orc_transpose(int64_t batch, int64_t rows, int64_t cols, const void* in, int in_dtype, int64_t ld_in,
+                  int64_t stride_in, int out_dtype, double* out) {
+    if (batch < 0 || rows < 0 || cols < 0) return 1;
+    for (int64_t b = 0; b < batch; ++b)
+        for (int64_t r = 0; r < rows; ++r)
+            for (int64_t c = 0; c < cols; ++c) {
+                double v = load_as_f64(in, in_dtype, b * stride_in + r * ld_in + c);
+                if (out_dtype == ORC_BF16 && in_dtype == ORC_F32) v = round_f32_to_bf16((float)v);
+                out[(b * cols + c) * rows + r] = v;
+            }
+    return 0;
+}
+
+int64_t orc_transpose_bytes(int64_t batch, int64_t rows, int64_t cols, int64_t eb_in, int64_t eb_out) {
+    return batch * rows * cols * (eb_in + eb_out);
+}
+
+/* -------------------------------------------------------------------------------------------
  * Speed-of-Light bound (Section 4.1; worked example in Appendix A.2).
  *   step 1  FLOPs (2 per multiply-accumulate) and best-case DRAM bytes: every
  *           unique input element read once, every output written once.

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libsolgemm.so")
 _SOURCES = ["sg_api.cu"]
-_DEPS = ["sg_api.cu", "sg_kernel.cuh", "sg_ptx.cuh", os.path.join(_ROOT, "include", "solgemm.h")]
+_DEPS = ["sg_api.cu", "sg_kernel.cuh", "sg_ptx.cuh", "sg_transpose.cuh", os.path.join(_ROOT, "include", "solgemm.h")]
 
 
 def _nvcc() -> str:

@@ -14,6 +14,7 @@
 
 #include "solgemm.h"
 #include "sg_kernel.cuh"
+#include "sg_transpose.cuh"
 
 namespace {
 
@@ -909,6 +910,47 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     return launch(*d, s, c.f32_out, p, static_cast<cudaStream_t>(cuda_stream));
 }
 
+sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* out, void* cuda_stream) {
+    if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
+    if (desc->reserved != 0 || desc->reserved2 != 0) return fail(SG_ERR_INVALID_ARG, "reserved fields must be 0");
+    if ((desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F32) || (desc->out_dtype != SG_BF16 && desc->out_dtype != SG_F32))
+        return fail(SG_ERR_INVALID_ARG, "sg_transpose: dtypes must be SG_BF16 or SG_F32");
+    if (desc->batch < 0 || desc->rows < 0 || desc->cols < 0) return fail(SG_ERR_INVALID_ARG, "sg_transpose: extents must be >= 0");
+    if (desc->batch == 0 || desc->rows == 0 || desc->cols == 0) return SG_OK;
+    const int es_in = desc->in_dtype == SG_F32 ? 4 : 2, es_out = desc->out_dtype == SG_F32 ? 4 : 2;
+    if (desc->ld_in < desc->cols || desc->ld_out < desc->rows) return fail(SG_ERR_INVALID_ARG, "sg_transpose: ld_in >= cols and ld_out >= rows are required");
+    if (desc->batch > 1 && (desc->stride_in < (desc->rows - 1) * desc->ld_in + desc->cols ||
+                            desc->stride_out < (desc->cols - 1) * desc->ld_out + desc->rows))
+        return fail(SG_ERR_INVALID_ARG, "sg_transpose: batch strides smaller than one matrix");
+    if (!in || !out) return fail(SG_ERR_NULL_POINTER, "sg_transpose: in or out is NULL");
+    if (!aligned16(in) || !aligned16(out)) return fail(SG_ERR_ALIGNMENT, "sg_transpose: base pointers must be 16-byte aligned");
+    if ((desc->ld_in * es_in) % 16 || (desc->ld_out * es_out) % 16 ||
+        (desc->batch > 1 && ((desc->stride_in * es_in) % 16 || (desc->stride_out * es_out) % 16)))
+        return fail(SG_ERR_ALIGNMENT, "sg_transpose: leading dimensions and batch strides must be multiples of 16 bytes");
+    const int64_t tiles_r = (desc->rows + 63) / 64, tiles_c = (desc->cols + 63) / 64;
+    if (tiles_r * tiles_c * desc->batch > INT32_MAX || tiles_r > INT32_MAX || tiles_c > INT32_MAX)
+        return fail(SG_ERR_UNSUPPORTED, "sg_transpose: too many tiles");
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    TransposeParams tp;
+    tp.in = in;
+    tp.out = out;
+    tp.rows = desc->rows; tp.cols = desc->cols;
+    tp.ld_in = desc->ld_in; tp.ld_out = desc->ld_out;
+    tp.stride_in = desc->stride_in; tp.stride_out = desc->stride_out;
+    tp.tiles_r = static_cast<int32_t>(tiles_r); tp.tiles_c = static_cast<int32_t>(tiles_c);
+    const dim3 grid(static_cast<unsigned>(tiles_r * tiles_c * desc->batch));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32) transpose_kernel<float, float><<<grid, 256, 0, stream>>>(tp);
+    else if (desc->in_dtype == SG_F32) transpose_kernel<float, __nv_bfloat16><<<grid, 256, 0, stream>>>(tp);
+    else if (desc->out_dtype == SG_F32) transpose_kernel<__nv_bfloat16, float><<<grid, 256, 0, stream>>>(tp);
+    else transpose_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(tp);
+    SG_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return SG_OK;
+}
+
 sg_status_t sg_poll_status(void* cuda_stream) {
     DeviceState* d = nullptr;
     sg_status_t st = device_state(&d);
@@ -967,6 +1009,12 @@ sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, 
         macs = cv->N * P * Q * cv->K * cv->C * cv->R * cv->S;
         elems_in = cv->N * cv->H * cv->W * cv->C + cv->K * cv->R * cv->S * cv->C + (has_bias ? cv->K : 0);
         elems_out = cv->N * P * Q * cv->K * (cv->beta != 0.0f ? 2 : 1);
+    } else if (op == SG_OP_TRANSPOSE) {
+        const sg_transpose_desc_t* t = static_cast<const sg_transpose_desc_t*>(desc);
+        if (t->batch < 0 || t->rows < 0 || t->cols < 0) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: negative extent");
+        elems_in = elems_out = t->batch * t->rows * t->cols;
+        eb_in = t->in_dtype == SG_F32 ? 4 : 2;
+        eb_out = t->out_dtype == SG_F32 ? 4 : 2;
     } else {
         return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: op %d is not a sg_op_t", op);
     }

@@ -33,12 +33,12 @@ LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
 DTYPES = {torch.bfloat16: 0, torch.float32: 1}
-OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3}
+OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
-            "sg_last_kernel_clock"]
+            "sg_last_kernel_clock", "sg_transpose"]
 
 
 class SolgemmError(RuntimeError):
@@ -67,6 +67,11 @@ class Conv2dDesc(ctypes.Structure):
                 ("epi_arg0", ctypes.c_float), ("epi_arg1", ctypes.c_float), ("reserved", ctypes.c_int32)]
 
 
+class TransposeDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("batch", "rows", "cols", "ld_in", "ld_out", "stride_in", "stride_out")] + \
+               [(n, ctypes.c_int32) for n in ("in_dtype", "out_dtype", "reserved", "reserved2")]
+
+
 class Hw(ctypes.Structure):
     _fields_ = [(n, ctypes.c_double) for n in ("peak_flops", "peak_bytes_per_s", "sm_clock_mhz", "sm_clock_max_mhz",
                                                "mem_clock_mhz", "mem_clock_max_mhz")]
@@ -92,6 +97,8 @@ _lib.sg_grouped_gemm_static.restype = ctypes.c_int
 _lib.sg_grouped_gemm_static.argtypes = [ctypes.POINTER(GemmDesc), _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_conv2d_fprop.restype = ctypes.c_int
 _lib.sg_conv2d_fprop.argtypes = [ctypes.POINTER(Conv2dDesc), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_transpose.restype = ctypes.c_int
+_lib.sg_transpose.argtypes = [ctypes.POINTER(TransposeDesc), _vp, _vp, _vp]
 _lib.sg_sol_bound.restype = ctypes.c_int
 _lib.sg_sol_bound.argtypes = [_i32, _vp, _i64, _vp, _i32, _i32, _i32, ctypes.POINTER(Hw), ctypes.POINTER(Sol)]
 _lib.sg_status_string.restype = ctypes.c_char_p
@@ -308,6 +315,48 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
     return out
 
 
+def transpose(x: torch.Tensor, *, out: Optional[torch.Tensor] = None, out_dtype: Optional[torch.dtype] = None,
+              stream=None) -> torch.Tensor:
+    """``sg_transpose``: ``out[b, c, r] = convert(x[b, r, c])`` for a 3-D (or 2-D) tensor with inner stride 1."""
+    squeeze = x.dim() == 2
+    x3 = x.unsqueeze(0) if squeeze else x
+    if x3.dim() != 3 or (x3.shape[2] > 1 and x3.stride(2) != 1):
+        raise ValueError("transpose wants a [batch, rows, cols] tensor with inner stride 1")
+    batch, rows, cols = x3.shape
+    if out is None:
+        out = torch.empty((batch, cols, rows), dtype=out_dtype or x.dtype, device=x.device)
+        out3 = out
+        if squeeze:
+            out = out[0]
+    else:
+        out3 = out.unsqueeze(0) if squeeze else out
+    desc = TransposeDesc(batch, rows, cols, x3.stride(1) if rows > 1 else max(cols, 1),
+                         out3.stride(1) if cols > 1 else max(rows, 1), x3.stride(0), out3.stride(0),
+                         DTYPES[x.dtype], DTYPES[out3.dtype], 0, 0)
+    _check(_lib.sg_transpose(ctypes.byref(desc), _ptr(x3), _ptr(out3), _stream(stream)))
+    return out
+
+
+def nchw_to_nhwc(x: torch.Tensor, out_dtype: Optional[torch.dtype] = None) -> torch.Tensor:
+    """[N, C, H, W] -> [N, H, W, C] (with optional dtype conversion) through ``sg_transpose``."""
+    n, c, h, w = x.shape
+    return transpose(x.reshape(n, c, h * w), out_dtype=out_dtype).view(n, h, w, c)
+
+
+def nhwc_to_nchw(x: torch.Tensor, out_dtype: Optional[torch.dtype] = None) -> torch.Tensor:
+    """[N, H, W, C] -> [N, C, H, W] (with optional dtype conversion) through ``sg_transpose``."""
+    n, h, w, c = x.shape
+    return transpose(x.reshape(n, h * w, c), out_dtype=out_dtype).view(n, c, h, w)
+
+
+def conv1d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=0, stride=1, dil=1, **kw) -> torch.Tensor:
+    """1-D convolution lowered to ``sg_conv2d_fprop`` with H = 1 (the paper's Table 1a note): X [N, L, C], Wf [K, S, C]."""
+    n, l, c = X.shape
+    k, s, _ = Wf.shape
+    y = conv2d_fprop(X.view(n, 1, l, c), Wf.view(k, 1, s, c), pad=(0, pad), stride=(1, stride), dil=(1, dil), **kw)
+    return y.view(n, y.shape[2], k)
+
+
 def gemm_host(A_host: torch.Tensor, B_host: torch.Tensor, out_host: torch.Tensor, *, bias_host=None, epi="none",
               alpha=1.0, device="cuda", scratch: Optional[dict] = None, stream=None) -> torch.Tensor:
     """End-to-end GEMM for callers whose data lives in (pinned) host memory.
@@ -333,10 +382,14 @@ def gemm_host(A_host: torch.Tensor, B_host: torch.Tensor, out_host: torch.Tensor
 
 
 def sol_bound(op: str, *, M=0, N=0, K=0, batch_or_groups=1, Ms: Optional[Sequence[int]] = None, conv: Optional[dict] = None,
+              transpose_shape: Optional[tuple] = None, transpose_dtypes=(torch.bfloat16, torch.bfloat16),
               beta=0.0, elem_bytes_in=2, elem_bytes_out=2, has_bias=0, peak_flops: float, peak_bytes_per_s: float,
               sm_clock_mhz=0.0, sm_clock_max_mhz=0.0, mem_clock_mhz=0.0, mem_clock_max_mhz=0.0) -> dict:
     """``sg_sol_bound``: FLOPs, best-case bytes and t_SOL = max(FLOPs/peak, bytes/bandwidth) (host only)."""
-    if op == "conv2d":
+    if op == "transpose":
+        b, r, c_ = transpose_shape
+        desc = TransposeDesc(b, r, c_, c_, r, r * c_, r * c_, DTYPES[transpose_dtypes[0]], DTYPES[transpose_dtypes[1]], 0, 0)
+    elif op == "conv2d":
         c = conv
         desc = Conv2dDesc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], *c.get("pad", (0, 0)),
                           *c.get("stride", (1, 1)), *c.get("dil", (1, 1)), 0, 0, 1.0, float(beta), 0, 0.0, 0.0, 0)

@@ -469,3 +469,42 @@ def test_conv_delta_filter_reproduces_input_on_gpu():
         Wf[k, 1, 1, k] = 1
     Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1))
     assert torch.equal(Y.cpu(), X)
+
+
+# ---------------------------------------------------------------------------------------- transpose stage
+
+@pytest.mark.parametrize("in_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(1, 64, 64), (3, 100, 72), (2, 37, 200), (4, 256, 196), (1, 1, 8), (2, 129, 4)])
+def test_transpose_with_dtype_conversion_bit_exact(shape, in_dtype, out_dtype):
+    batch, rows, cols = shape
+    ld = (cols + 7) // 8 * 8 + 8
+    big = (inputs.normal([batch, rows, ld], 616, 1).float() * 1.37).to(in_dtype)          # padded leading dimension
+    x = big[:, :, :cols]
+    want = orc.transpose(x, out_dtype)
+    ld_out = (rows + 7) // 8 * 8 + 8
+    out_big = torch.full((batch, cols, ld_out), float("nan"), dtype=out_dtype, device=DEV)
+    sg.transpose(big.to(DEV)[:, :, :cols], out=out_big[:, :, :rows])
+    parity.assert_bit_exact(out_big[:, :, :rows], want, f"transpose {shape} {in_dtype}->{out_dtype}")
+    assert bool(torch.isnan(out_big[:, :, rows:]).all())
+    if rows % 8 == 0 and cols % 8 == 0:       # the densely packed form needs 16-byte leading dimensions itself
+        assert torch.equal(sg.transpose(x.to(DEV), out_dtype=out_dtype).cpu(), x.permute(0, 2, 1).to(out_dtype))
+
+
+def test_layout_pipeline_nchw_conv_nchw_and_conv1d():
+    # pipeline(transpose(input, NCHW, NHWC, fp32, bf16), conv2d_fprop, transpose(output, NHWC, NCHW, bf16, fp32))
+    N, C, H, W, K = 2, 64, 10, 12, 72
+    x_nchw = inputs.small_integers([N, C, H, W], 626, 6, -1, 1).float()
+    Wf = inputs.small_integers([K, 3, 3, C], 626, 7, -1, 1) * (inputs.small_integers([K, 3, 3, C], 627, 7, 0, 3) == 0).to(torch.bfloat16)
+    x_nhwc = sg.nchw_to_nhwc(x_nchw.to(DEV), out_dtype=torch.bfloat16)
+    assert torch.equal(x_nhwc.cpu(), x_nchw.permute(0, 2, 3, 1).to(torch.bfloat16))
+    y = sg.conv2d_fprop(x_nhwc, Wf.to(DEV), pad=(1, 1), epi="relu")
+    y_nchw = sg.nhwc_to_nchw(y, out_dtype=torch.float32)
+    ref, _ = orc.conv2d_fprop(x_nchw.permute(0, 2, 3, 1).contiguous().to(torch.bfloat16), Wf, pad=(1, 1), epi="relu")
+    parity.assert_bit_exact(y_nchw.permute(0, 2, 3, 1), ref, "NCHW -> conv -> NCHW")
+    # conv1d lowered to conv2d with H = 1
+    X1 = inputs.small_integers([3, 50, 32], 636, 6, -1, 1)
+    W1 = inputs.small_integers([40, 5, 32], 636, 7, -1, 1) * (inputs.small_integers([40, 5, 32], 637, 7, 0, 2) == 0).to(torch.bfloat16)
+    ref1, _ = orc.conv2d_fprop(X1.view(3, 1, 50, 32), W1.view(40, 1, 5, 32), pad=(0, 2), stride=(1, 2))
+    y1 = sg.conv1d_fprop(X1.to(DEV), W1.to(DEV), pad=2, stride=2)
+    parity.assert_bit_exact(y1, ref1.view(3, -1, 40), "conv1d")

@@ -379,3 +379,31 @@ def test_tolerance_accepts_bf16_rounding_and_rejects_skipped_work():
     erf = torch.nn.functional.gelu(x.double())
     assert not parity.mismatches(want.float(), want, wacc).any()
     assert parity.mismatches(erf.float(), want, wacc).any()
+
+
+# ---------------------------------------------------------------- transpose with dtype conversion
+
+def test_transpose_hand_cases_and_rounding_ties():
+    x = torch.tensor([[[1.0, 2.0, 3.0], [4.0, 5.0, 6.0]]], dtype=torch.float32)          # [1, 2, 3]
+    assert orc.transpose(x, torch.float32).tolist() == [[[1.0, 4.0], [2.0, 5.0], [3.0, 6.0]]]
+    # fp32 -> bf16: 8 significant bits; ties go to the even neighbour
+    ties = torch.tensor([[[1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -(1.0 + 2.0 ** -8),
+                           3.4028234663852886e38, 3.3895313892515355e38]]], dtype=torch.float32)
+    got = orc.transpose(ties, torch.bfloat16).view(-1).tolist()
+    assert got[:4] == [1.0, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7, -1.0]
+    assert got[4] == float("inf") and got[5] == 3.3895313892515355e38       # fp32 max rounds up to infinity; bf16 max stays
+    nan = orc.transpose(torch.tensor([[[float("nan")]]], dtype=torch.float32), torch.bfloat16)
+    assert math.isnan(float(nan))
+
+
+def test_transpose_matches_torch_permute_and_cast():
+    x32 = inputs.normal([3, 37, 29], 21, 1).float() * 1.2345 + torch.rand(3, 37, 29, generator=torch.Generator().manual_seed(1)) * 1e-3
+    xbf = inputs.uniform([3, 37, 29], 21, 2)
+    for x in (x32, xbf):
+        for od in (torch.float32, torch.bfloat16):
+            want = x.permute(0, 2, 1).contiguous().to(od).double()
+            assert torch.equal(orc.transpose(x, od), want), (x.dtype, od)
+    padded = x32.new_zeros(3, 37, 40)
+    padded[:, :, :29] = x32
+    assert torch.equal(orc.transpose(padded[:, :, :29], torch.bfloat16), x32.permute(0, 2, 1).to(torch.bfloat16).double())
+    assert orc.transpose_bytes(32, 256, 3136, 4, 2) == 32 * 256 * 3136 * 6
