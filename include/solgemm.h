@@ -17,9 +17,10 @@
  *    current CUDA device.  The caller owns all buffers; the library allocates no device memory.
  *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
  *    enqueue work on that stream and return; they never synchronise.
- *  - Inputs A, B, bias (and conv X, Wf) are bf16.  The output D is bf16 or fp32 (`out_dtype`);
- *    C, when read, has the output's dtype and shape.  Accumulation and the epilogue run in fp32;
- *    the result is rounded to nearest-even.
+ *  - Inputs A, B, bias (and conv X, Wf) are bf16 or fp16 (`in_dtype`, the same for all of them).  The
+ *    output D is bf16, fp16 or fp32 (`out_dtype`); C, when read, has the output's dtype and shape.
+ *    Accumulation and the epilogue run in fp32; the result is rounded to nearest-even.
+ *    (The DSL's .with_dtype(input, acc, output); its running example is input=fp16, acc=fp32, output=fp16.)
  *  - Epilogue: v = alpha*acc (+ beta*C if beta != 0) (+ bias[j] if bias != NULL); D = act(v).
  *    bias holds one value per output column j (GEMM) or output channel (conv); it is NOT scaled
  *    by alpha.  SG_EPI_BIAS is the identity activation and requires bias != NULL; every other
@@ -58,7 +59,7 @@ typedef enum {
     SG_ERR_TIMEOUT = 8        /* a bounded device-side wait expired (see sg_poll_status) */
 } sg_status_t;
 
-typedef enum { SG_BF16 = 0, SG_F32 = 1 } sg_dtype_t;
+typedef enum { SG_BF16 = 0, SG_F32 = 1, SG_F16 = 2 } sg_dtype_t;
 typedef enum { SG_ROW_MAJOR = 0, SG_COL_MAJOR = 1 } sg_layout_t;
 typedef enum {
     SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4,
@@ -85,7 +86,7 @@ typedef struct sg_gemm_desc {
     int64_t M, N, K;
     int32_t layout_a, layout_b;   /* sg_layout_t */
     int64_t lda, ldb, ldc, ldd;
-    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype must be SG_BF16 */
+    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype SG_BF16 or SG_F16 */
     float alpha, beta;
     int32_t epi;                  /* sg_epilogue_t */
     float epi_arg0, epi_arg1;     /* activation parameters (leaky_relu / elu slope, clip bounds); else ignored */
@@ -94,9 +95,9 @@ typedef struct sg_gemm_desc {
 
 /*
  * sg_gemm: D[M,N] = act(alpha * A.B + beta * C + bias).      (paper: gemm(), Table 1a, Appendix A.1)
- *   A, B   device, bf16, laid out as layout_a / layout_b and lda / ldb say.
+ *   A, B   device, in_dtype, laid out as layout_a / layout_b and lda / ldb say.
  *   C      device, out_dtype, [M,N] row-major; may be NULL when beta == 0.
- *   bias   device, bf16, [N]; may be NULL unless epi == SG_EPI_BIAS.
+ *   bias   device, in_dtype, [N]; may be NULL unless epi == SG_EPI_BIAS.
  *   D      device, out_dtype, [M,N] row-major; written in full (all M x N elements).
  * M == 0 or N == 0: SG_OK, nothing is launched.  K == 0: D = act(beta*C + bias).
  */
@@ -187,7 +188,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
  * stage with fused dtype conversion that the DSL's pipeline(transpose(...), kernel, transpose(...)) places
  * around a kernel (Section 3 "Multi-stage pipelines"; Appendix A.1 transpose_op: NCL <-> NLC, and
  * NCHW <-> NHWC "implemented by flattening HW": batch = N, rows = C, cols = H*W or the reverse).
- *   in   device, in_dtype (bf16 or fp32), [batch][rows][cols], row stride ld_in, batch stride stride_in (elements)
+ *   in   device, in_dtype (bf16 or fp32; fp16 is not implemented here), [batch][rows][cols], row stride ld_in, batch stride stride_in (elements)
  *   out  device, out_dtype (bf16 or fp32), [batch][cols][rows], row stride ld_out, batch stride stride_out
  *   fp32 -> bf16 rounds to nearest even; bf16 -> fp32 is exact.  in and out must not overlap.
  * Base pointers 16-byte aligned, ld and strides multiples of 16 bytes, ld_in >= cols, ld_out >= rows.

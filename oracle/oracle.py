@@ -32,7 +32,8 @@ _LIB = os.path.join(_HERE, "libsg_oracle.so")
 LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
-_DTYPES = {torch.bfloat16: 0, torch.float32: 1}
+_DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2}
+_IN_DTYPES = (torch.bfloat16, torch.float16)
 
 
 def build(force: bool = False) -> str:
@@ -58,17 +59,17 @@ def lib() -> ctypes.CDLL:
         L.orc_act2.restype = dbl
         L.orc_act2.argtypes = [ci, dbl, dbl, dbl]
         L.orc_gemm.restype = ci
-        L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl,
+        L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl, ci,
                                i64, i64, vp, vp, i64]
         L.orc_gemm_points.restype = ci
-        L.orc_gemm_points.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl,
+        L.orc_gemm_points.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl, ci,
                                       i64, vp, vp, vp, vp]
         L.orc_conv_out_extent.restype = i64
         L.orc_conv_out_extent.argtypes = [i64] * 5
         L.orc_conv2d_fprop.restype = ci
-        L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, i64, i64, vp, vp]
+        L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, ci, i64, i64, vp, vp]
         L.orc_conv2d_points.restype = ci
-        L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, i64, vp, vp, vp, vp]
+        L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, ci, i64, vp, vp, vp, vp]
         L.orc_transpose.restype = ci
         L.orc_transpose.argtypes = [i64, i64, i64, vp, ci, i64, i64, ci, vp]
         L.orc_transpose_bytes.restype = i64
@@ -99,9 +100,9 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
-def _check2d(t: torch.Tensor, name: str, dtype=torch.bfloat16):
-    if t.device.type != "cpu" or t.dim() != 2 or t.dtype != dtype:
-        raise ValueError(f"{name}: want a 2-D CPU {dtype} tensor")
+def _check2d(t: torch.Tensor, name: str):
+    if t.device.type != "cpu" or t.dim() != 2 or t.dtype not in _IN_DTYPES:
+        raise ValueError(f"{name}: want a 2-D CPU bf16 or fp16 tensor")
     if t.shape[1] > 1 and t.stride(1) != 1:
         raise ValueError(f"{name}: inner stride must be 1")
 
@@ -109,6 +110,8 @@ def _check2d(t: torch.Tensor, name: str, dtype=torch.bfloat16):
 def _gemm_shapes(A, B, layout_a, layout_b):
     _check2d(A, "A")
     _check2d(B, "B")
+    if A.dtype != B.dtype:
+        raise ValueError("A and B must have the same dtype")
     M, K = (A.shape if layout_a == "row" else (A.shape[1], A.shape[0]))
     Kb, N = (B.shape if layout_b == "row" else (B.shape[1], B.shape[0]))
     if K != Kb:
@@ -122,16 +125,16 @@ def _c_args(C, M, N):
     if C is None:
         return None, 0, max(N, 1)
     if C.device.type != "cpu" or C.dim() != 2 or tuple(C.shape) != (M, N) or C.dtype not in _DTYPES:
-        raise ValueError("C: want a CPU [M, N] bf16 or fp32 tensor")
+        raise ValueError("C: want a CPU [M, N] bf16, fp16 or fp32 tensor")
     if N > 1 and C.stride(1) != 1:
         raise ValueError("C: inner stride must be 1")
     return C, _DTYPES[C.dtype], (C.stride(0) if M > 1 else max(N, 1))
 
 
-def _check_bias(bias, n):
-    if bias is not None and (bias.device.type != "cpu" or bias.dtype != torch.bfloat16 or bias.numel() != n
+def _check_bias(bias, n, dtype=torch.bfloat16):
+    if bias is not None and (bias.device.type != "cpu" or bias.dtype != dtype or bias.numel() != n
                              or not bias.is_contiguous()):
-        raise ValueError("bias: want a contiguous CPU bf16 vector with one value per output column")
+        raise ValueError("bias: want a contiguous CPU vector of the inputs' dtype with one value per output column")
 
 
 def gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a: str = "row", layout_b: str = "col",
@@ -140,14 +143,15 @@ def gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a: str = "row", layout_b: s
          rows: Optional[Tuple[int, int]] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """act(alpha A.B + beta C + bias) for rows ``rows=(begin, end)`` (default: all)."""
     M, N, K, lda, ldb = _gemm_shapes(A, B, layout_a, layout_b)
-    _check_bias(bias, N)
+    _check_bias(bias, N, A.dtype)
     C, c_dtype, ldc = _c_args(C, M, N)
     r0, r1 = rows if rows is not None else (0, M)
     ref = torch.empty((r1 - r0, N), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
                         _ptr(C), c_dtype, ldc, _ptr(bias), float(alpha), float(beta), EPILOGUES[epi],
-                        float(epi_args[0]), float(epi_args[1]), r0, r1, _ptr(ref), _ptr(absacc), max(N, 1))
+                        float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], r0, r1, _ptr(ref), _ptr(absacc),
+                        max(N, 1))
     if rc:
         raise ValueError(f"orc_gemm rejected its arguments (code {rc})")
     return ref, absacc
@@ -157,7 +161,7 @@ def gemm_points(A, B, pi: Sequence[int], pj: Sequence[int], *, layout_a="row", l
                 alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)) -> Tuple[torch.Tensor, torch.Tensor]:
     """The elements (pi[t], pj[t]) of the result only."""
     M, N, K, lda, ldb = _gemm_shapes(A, B, layout_a, layout_b)
-    _check_bias(bias, N)
+    _check_bias(bias, N, A.dtype)
     C, c_dtype, ldc = _c_args(C, M, N)
     pi = torch.as_tensor(pi, dtype=torch.int64).contiguous()
     pj = torch.as_tensor(pj, dtype=torch.int64).contiguous()
@@ -165,8 +169,8 @@ def gemm_points(A, B, pi: Sequence[int], pj: Sequence[int], *, layout_a="row", l
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm_points(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
                                _ptr(C), c_dtype, ldc, _ptr(bias), float(alpha), float(beta), EPILOGUES[epi],
-                               float(epi_args[0]), float(epi_args[1]), pi.numel(), _ptr(pi), _ptr(pj), _ptr(ref),
-                               _ptr(absacc))
+                               float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], pi.numel(), _ptr(pi), _ptr(pj),
+                               _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_gemm_points rejected its arguments (code {rc})")
     return ref, absacc
@@ -201,10 +205,10 @@ def conv_out_extent(size: int, pad: int, dil: int, filt: int, stride: int) -> in
 
 
 def _conv_dims(X, Wf, pad, stride, dil):
-    if X.device.type != "cpu" or X.dim() != 4 or X.dtype != torch.bfloat16 or not X.is_contiguous():
-        raise ValueError("X: want a contiguous CPU bf16 NHWC tensor")
-    if Wf.device.type != "cpu" or Wf.dim() != 4 or Wf.dtype != torch.bfloat16 or not Wf.is_contiguous():
-        raise ValueError("Wf: want a contiguous CPU bf16 KRSC tensor")
+    if X.device.type != "cpu" or X.dim() != 4 or X.dtype not in _IN_DTYPES or not X.is_contiguous():
+        raise ValueError("X: want a contiguous CPU bf16 or fp16 NHWC tensor")
+    if Wf.device.type != "cpu" or Wf.dim() != 4 or Wf.dtype != X.dtype or not Wf.is_contiguous():
+        raise ValueError("Wf: want a contiguous CPU KRSC tensor of X's dtype")
     N, H, W, C = X.shape
     K, R, S, Cw = Wf.shape
     if C != Cw:
@@ -229,14 +233,14 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
                  pixels: Optional[Tuple[int, int]] = None):
     """Direct convolution; returns ``[N,P,Q,K]`` tensors, or ``[pixels, K]`` for a flattened pixel range."""
     d, N, P, Q, K = _conv_dims(X, Wf, pad, stride, dil)
-    _check_bias(bias, K)
+    _check_bias(bias, K, X.dtype)
     Cin, c_dtype = _conv_c(Cin, N, P, Q, K)
     p0, p1 = pixels if pixels is not None else (0, N * P * Q)
     ref = torch.empty((p1 - p0, K), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_fprop(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
                                 float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
-                                p0, p1, _ptr(ref), _ptr(absacc))
+                                _DTYPES[X.dtype], p0, p1, _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_fprop rejected its arguments (code {rc})")
     if pixels is None:
@@ -248,7 +252,7 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
                   Cin=None, bias=None, alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)):
     """The outputs (flattened pixel ppix[t], channel pk[t]) only."""
     d, N, P, Q, K = _conv_dims(X, Wf, pad, stride, dil)
-    _check_bias(bias, K)
+    _check_bias(bias, K, X.dtype)
     Cin, c_dtype = _conv_c(Cin, N, P, Q, K)
     ppix = torch.as_tensor(ppix, dtype=torch.int64).contiguous()
     pk = torch.as_tensor(pk, dtype=torch.int64).contiguous()
@@ -256,7 +260,7 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_points(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
                                  float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
-                                 ppix.numel(), _ptr(ppix), _ptr(pk), _ptr(ref), _ptr(absacc))
+                                 _DTYPES[X.dtype], ppix.numel(), _ptr(ppix), _ptr(pk), _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_points rejected its arguments (code {rc})")
     return ref, absacc

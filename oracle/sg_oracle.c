@@ -9,8 +9,8 @@
  * cpu-baseline / reference arm may load it.  It shares no code, header, table or
  * helper with the CUDA path and is never tuned for speed.
  *
- * Everything is evaluated in fp64.  bf16 inputs are widened exactly; a product
- * of two bf16 values (8-bit significands) is exact in fp64, so the only error
+ * Everything is evaluated in fp64.  bf16 / fp16 inputs are widened exactly; a product
+ * of two such values (8- or 11-bit significands) is exact in fp64, so the only error
  * is the summation's (<= K * 2^-53 relative to sum |a||b|).
  *
  * What each function follows in the paper (arXiv 2603.29010):
@@ -45,7 +45,7 @@
 #endif
 
 enum { ORC_ROW_MAJOR = 0, ORC_COL_MAJOR = 1 };
-enum { ORC_BF16 = 0, ORC_F32 = 1 };
+enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2 };
 enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4,
        ORC_EPI_SIGMOID = 5, ORC_EPI_TANH = 6, ORC_EPI_MISH = 7, ORC_EPI_HARDSWISH = 8, ORC_EPI_LEAKY_RELU = 9,
        ORC_EPI_ELU = 10, ORC_EPI_CLIP = 11 };
@@ -67,8 +67,22 @@ static double bf16_to_f64(uint16_t bits) {
     return (double)f;
 }
 
+/* IEEE binary16 -> fp64, exact: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double f16_to_f64(uint16_t bits) {
+    int sign = bits >> 15, e = (bits >> 10) & 0x1F, f = bits & 0x3FF;
+    double v;
+    if (e == 0) v = ldexp((double)f, -24);                       /* zero and subnormals: f * 2^-24 */
+    else if (e == 31) v = f ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)f / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
+/* The two 16-bit input formats (.with_dtype(input=bf16 | fp16, ...)). */
+static double in16_to_f64(uint16_t bits, int dtype) { return dtype == ORC_F16 ? f16_to_f64(bits) : bf16_to_f64(bits); }
+
 static double load_as_f64(const void* p, int dtype, int64_t idx) {
     if (dtype == ORC_BF16) return bf16_to_f64(((const uint16_t*)p)[idx]);
+    if (dtype == ORC_F16) return f16_to_f64(((const uint16_t*)p)[idx]);
     return (double)((const float*)p)[idx];
 }
 
@@ -127,14 +141,15 @@ typedef struct {
     double alpha, beta;
     int epi;
     double a0, a1;                               /* activation parameters */
+    int in_dtype;                                /* ORC_BF16 or ORC_F16: type of A, B and bias */
 } gemm_problem;
 
 /* One output element and, optionally, the magnitude sum used to scale fp32 tolerances. */
 static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* absacc) {
     double sum = 0.0, asum = 0.0;
     for (int64_t k = 0; k < g->K; ++k) {
-        double a = bf16_to_f64(g->layout_a == ORC_ROW_MAJOR ? g->A[i * g->lda + k] : g->A[k * g->lda + i]);
-        double b = bf16_to_f64(g->layout_b == ORC_ROW_MAJOR ? g->B[k * g->ldb + j] : g->B[j * g->ldb + k]);
+        double a = in16_to_f64(g->layout_a == ORC_ROW_MAJOR ? g->A[i * g->lda + k] : g->A[k * g->lda + i], g->in_dtype);
+        double b = in16_to_f64(g->layout_b == ORC_ROW_MAJOR ? g->B[k * g->ldb + j] : g->B[j * g->ldb + k], g->in_dtype);
         sum += a * b;
         asum += fabs(a * b);
     }
@@ -146,7 +161,7 @@ static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* 
         av += fabs(g->beta * c);
     }
     if (g->bias) {
-        double bj = bf16_to_f64(g->bias[j]);
+        double bj = in16_to_f64(g->bias[j], g->in_dtype);
         v += bj;
         av += fabs(bj);
     }
@@ -161,11 +176,11 @@ static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* 
 int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
              const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
              const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
-             double alpha, double beta, int epi, double a0, double a1,
+             double alpha, double beta, int epi, double a0, double a1, int in_dtype,
              int64_t row_begin, int64_t row_end, double* ref, double* absacc, int64_t ldr) {
     if (M < 0 || N < 0 || K < 0 || row_begin < 0 || row_end > M || row_begin > row_end) return 1;
     if (beta != 0.0 && !C) return 2;
-    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1};
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1, in_dtype};
 #pragma omp parallel for schedule(static)
     for (int64_t i = row_begin; i < row_end; ++i) {
         for (int64_t j = 0; j < N; ++j) {
@@ -182,10 +197,10 @@ int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
 int orc_gemm_points(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
                     const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
                     const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
-                    double alpha, double beta, int epi, double a0, double a1,
+                    double alpha, double beta, int epi, double a0, double a1, int in_dtype,
                     int64_t npts, const int64_t* pi, const int64_t* pj, double* ref, double* absacc) {
     if (beta != 0.0 && !C) return 2;
-    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1};
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1, in_dtype};
     for (int64_t t = 0; t < npts; ++t)
         if (pi[t] < 0 || pi[t] >= M || pj[t] < 0 || pj[t] >= N) return 1;
 #pragma omp parallel for schedule(static)
@@ -214,6 +229,7 @@ typedef struct {
     double alpha, beta;
     int epi;
     double a0, a1;
+    int in_dtype;
 } conv_problem;
 
 int64_t orc_conv_out_extent(int64_t in, int64_t pad, int64_t dil, int64_t filt, int64_t stride) {
@@ -233,7 +249,7 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
             const uint16_t* xp = cv->X + ((n * cv->H + h) * cv->W + w) * cv->C;
             const uint16_t* wp = cv->Wf + ((k * cv->R + r) * cv->S + s) * cv->C;
             for (int64_t c = 0; c < cv->C; ++c) {
-                double t = bf16_to_f64(xp[c]) * bf16_to_f64(wp[c]);
+                double t = in16_to_f64(xp[c], cv->in_dtype) * in16_to_f64(wp[c], cv->in_dtype);
                 sum += t;
                 asum += fabs(t);
             }
@@ -247,7 +263,7 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
         av += fabs(cv->beta * c);
     }
     if (cv->bias) {
-        double bk = bf16_to_f64(cv->bias[k]);
+        double bk = in16_to_f64(cv->bias[k], cv->in_dtype);
         v += bk;
         av += fabs(bk);
     }
@@ -257,7 +273,7 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
 
 static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, const uint16_t* Wf,
                       const void* Cin, int c_dtype, const uint16_t* bias, double alpha, double beta, int epi,
-                      double a0, double a1) {
+                      double a0, double a1, int in_dtype) {
     cv->N = d[0]; cv->H = d[1]; cv->W = d[2]; cv->C = d[3]; cv->K = d[4]; cv->R = d[5]; cv->S = d[6];
     cv->pad_h = d[7]; cv->pad_w = d[8]; cv->stride_h = d[9]; cv->stride_w = d[10];
     cv->dil_h = d[11]; cv->dil_w = d[12];
@@ -267,7 +283,7 @@ static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, con
     cv->P = orc_conv_out_extent(cv->H, cv->pad_h, cv->dil_h, cv->R, cv->stride_h);
     cv->Q = orc_conv_out_extent(cv->W, cv->pad_w, cv->dil_w, cv->S, cv->stride_w);
     cv->X = X; cv->Wf = Wf; cv->Cin = Cin; cv->c_dtype = c_dtype; cv->bias = bias;
-    cv->alpha = alpha; cv->beta = beta; cv->epi = epi; cv->a0 = a0; cv->a1 = a1;
+    cv->alpha = alpha; cv->beta = beta; cv->epi = epi; cv->a0 = a0; cv->a1 = a1; cv->in_dtype = in_dtype;
     return 0;
 }
 
@@ -278,10 +294,10 @@ static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, con
  */
 int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
                      const void* Cin, int c_dtype, const uint16_t* bias,
-                     double alpha, double beta, int epi, double a0, double a1,
+                     double alpha, double beta, int epi, double a0, double a1, int in_dtype,
                      int64_t pix_begin, int64_t pix_end, double* ref, double* absacc) {
     conv_problem cv;
-    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1);
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1, in_dtype);
     if (rc) return rc;
     if (pix_begin < 0 || pix_end > cv.N * cv.P * cv.Q || pix_begin > pix_end) return 1;
 #pragma omp parallel for schedule(static)
@@ -302,10 +318,10 @@ int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
 /* The listed (flattened pixel, output channel) pairs only. */
 int orc_conv2d_points(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
                       const void* Cin, int c_dtype, const uint16_t* bias,
-                      double alpha, double beta, int epi, double a0, double a1,
+                      double alpha, double beta, int epi, double a0, double a1, int in_dtype,
                       int64_t npts, const int64_t* ppix, const int64_t* pk, double* ref, double* absacc) {
     conv_problem cv;
-    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1);
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1, in_dtype);
     if (rc) return rc;
     for (int64_t t = 0; t < npts; ++t)
         if (ppix[t] < 0 || ppix[t] >= cv.N * cv.P * cv.Q || pk[t] < 0 || pk[t] >= cv.K) return 1;

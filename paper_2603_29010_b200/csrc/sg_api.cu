@@ -79,31 +79,31 @@ struct KernelEntry {
     int threads;
 };
 
-template <int BN, bool kPair, bool kF32, int kEpiWarps>
+template <int BN, bool kPair, int kOut, int kEpiWarps>
 KernelEntry entry() {
     using Cfg = Config<BN, kPair, kEpiWarps>;
-    return KernelEntry{contract_kernel<BN, kPair, kF32, kEpiWarps>, Cfg::SMEM_BYTES, Cfg::THREADS};
+    return KernelEntry{contract_kernel<BN, kPair, kOut, kEpiWarps>, Cfg::SMEM_BYTES, Cfg::THREADS};
 }
 
 template <int BN, int kEpiWarps>
-KernelEntry entry_for(bool pair, bool f32) {
-    return pair ? (f32 ? entry<BN, true, true, kEpiWarps>() : entry<BN, true, false, kEpiWarps>())
-                : (f32 ? entry<BN, false, true, kEpiWarps>() : entry<BN, false, false, kEpiWarps>());
+KernelEntry entry_for(bool pair, int out) {
+    if (pair) return out == 1 ? entry<BN, true, 1, kEpiWarps>() : (out == 2 ? entry<BN, true, 2, kEpiWarps>() : entry<BN, true, 0, kEpiWarps>());
+    return out == 1 ? entry<BN, false, 1, kEpiWarps>() : (out == 2 ? entry<BN, false, 2, kEpiWarps>() : entry<BN, false, 0, kEpiWarps>());
 }
 
-// tile width (64, 128, 256) x CTA pairing x output type x number of epilogue warps (4 or 8)
-KernelEntry kernel_for(int bn, bool pair, bool f32, int epi_warps) {
+// tile width (64, 128, 256) x CTA pairing x output type (0 bf16, 1 fp32, 2 fp16) x epilogue warps (4 or 8)
+KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps) {
     if (epi_warps == 8) {
         switch (bn) {
-            case 64: return entry_for<64, 8>(pair, f32);
-            case 128: return entry_for<128, 8>(pair, f32);
-            default: return entry_for<256, 8>(pair, f32);
+            case 64: return entry_for<64, 8>(pair, out);
+            case 128: return entry_for<128, 8>(pair, out);
+            default: return entry_for<256, 8>(pair, out);
         }
     }
     switch (bn) {
-        case 64: return entry_for<64, 4>(pair, f32);
-        case 128: return entry_for<128, 4>(pair, f32);
-        default: return entry_for<256, 4>(pair, f32);
+        case 64: return entry_for<64, 4>(pair, out);
+        case 128: return entry_for<128, 4>(pair, out);
+        default: return entry_for<256, 4>(pair, out);
     }
 }
 
@@ -150,15 +150,15 @@ sg_status_t device_state(DeviceState** out) {
             const int bns[3] = {64, 128, 256};
             for (int i = 0; i < 3 && d.init_status == SG_OK; ++i)
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
-                    for (int f32 = 0; f32 < 2 && d.init_status == SG_OK; ++f32)
+                    for (int f32 = 0; f32 < 3 && d.init_status == SG_OK; ++f32)
                         for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4) {
-                            KernelEntry k = kernel_for(bns[i], pair != 0, f32 != 0, ew);
+                            KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew);
                             e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
                             if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
                         }
             if (d.init_status == SG_OK) {
                 // how many 2-CTA clusters fit at once (some GPCs may not pair up all of their SMs)
-                KernelEntry k = kernel_for(256, true, false, 8);
+                KernelEntry k = kernel_for(256, true, 0, 8);
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3(2 * d.sm_count);
                 cfg.blockDim = dim3(k.threads);
@@ -211,12 +211,15 @@ sg_status_t make_tiled_map(CUtensorMap* map, CUtensorMapDataType dt, int esize, 
 struct Checked {
     bool f32_out;
     int esize_out;
+    int out_kind;                 // kernel template value: 0 bf16, 1 fp32, 2 fp16
+    bool in_f16;
+    CUtensorMapDataType tm_in, tm_out;
 };
 
 sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, float a0, float a1,
                          int32_t reserved, Checked* c) {
-    if (in_dtype != SG_BF16) return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: only SG_BF16 inputs are implemented", in_dtype);
-    if (out_dtype != SG_BF16 && out_dtype != SG_F32) return fail(SG_ERR_INVALID_ARG, "out_dtype %d is not a sg_dtype_t", out_dtype);
+    if (in_dtype != SG_BF16 && in_dtype != SG_F16) return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16 or SG_F16", in_dtype);
+    if (out_dtype != SG_BF16 && out_dtype != SG_F32 && out_dtype != SG_F16) return fail(SG_ERR_INVALID_ARG, "out_dtype %d is not a sg_dtype_t", out_dtype);
     if (epi < SG_EPI_NONE || epi > SG_EPI_CLIP) return fail(SG_ERR_INVALID_ARG, "epi %d is not a sg_epilogue_t", epi);
     if (!std::isfinite(alpha) || !std::isfinite(beta)) return fail(SG_ERR_INVALID_ARG, "alpha and beta must be finite");
     if ((epi == SG_EPI_LEAKY_RELU || epi == SG_EPI_ELU) && !std::isfinite(a0)) return fail(SG_ERR_INVALID_ARG, "epi_arg0 (slope) must be finite");
@@ -224,6 +227,11 @@ sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float
     if (reserved != 0) return fail(SG_ERR_INVALID_ARG, "reserved field must be 0");
     c->f32_out = (out_dtype == SG_F32);
     c->esize_out = c->f32_out ? 4 : 2;
+    c->out_kind = out_dtype == SG_F32 ? 1 : (out_dtype == SG_F16 ? 2 : 0);
+    c->in_f16 = (in_dtype == SG_F16);
+    c->tm_in = c->in_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    c->tm_out = out_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                    : (out_dtype == SG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     return SG_OK;
 }
 
@@ -396,8 +404,8 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
     }
 }
 
-sg_status_t launch(const DeviceState& d, const Shape& s, bool f32, const Params& p, cudaStream_t stream) {
-    KernelEntry k = kernel_for(s.bn, s.pair, f32, s.epi_warps);
+sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Params& p, cudaStream_t stream) {
+    KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;
     const int tiles = p.num_tiles < slots ? p.num_tiles : slots;
@@ -465,6 +473,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
 
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
+    p.in_f16 = c.in_f16 ? 1 : 0;
     const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
     Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
@@ -493,27 +502,27 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
         // K-contiguous operand: boxes of 64 k x tile rows.  M/N-contiguous operand (column-major A, row-major B):
         // the map is over [k][rows] and every load is a box of 64 rows x 64 k.
         if (p.a_mn_major)
-            st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->M, desc->K, batch, desc->lda, sA, 64, 64, "A");
+            st = make_tiled_map(&p.tmA, c.tm_in, 2, A, desc->M, desc->K, batch, desc->lda, sA, 64, 64, "A");
         else
-            st = make_tiled_map(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
+            st = make_tiled_map(&p.tmA, c.tm_in, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
         if (st != SG_OK) return st;
         if (p.b_mn_major) {
-            st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->N, desc->K, batch, desc->ldb, sB, 64, 64, "B");
+            st = make_tiled_map(&p.tmB, c.tm_in, 2, B, desc->N, desc->K, batch, desc->ldb, sB, 64, 64, "B");
             p.tmB2 = p.tmB;
         } else {
-            st = make_tiled_map(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+            st = make_tiled_map(&p.tmB, c.tm_in, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
                                 s.pair ? s.bn / 2 : s.bn, "B");
             if (st != SG_OK) return st;
-            st = make_tiled_map(&p.tmB2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+            st = make_tiled_map(&p.tmB2, c.tm_in, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
                                 (s.pair ? s.bn / 2 : s.bn) / p.split, "B (narrow)");
         }
         if (st != SG_OK) return st;
     }
-    st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, D,
+    st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, D,
                         desc->N, desc->M, batch, desc->ldd, sD, c.f32_out ? 32 : 64, 32, "D");
     if (st != SG_OK) return st;
     if (desc->K == 0) { p.tmA = p.tmD; p.tmB = p.tmD; p.tmB2 = p.tmD; }   // never used for loads; keeps the prefetch harmless
-    return launch(*d, s, c.f32_out, p, static_cast<cudaStream_t>(stream));
+    return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(stream));
 }
 
 // ------------------------------------------------------------------------------------------ grouped
@@ -705,6 +714,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
 
     Params p;
     base_params(&p, *d, common->alpha, common->beta, common->epi, common->epi_arg0, common->epi_arg1);
+    p.in_f16 = c.in_f16 ? 1 : 0;
     int64_t tiles = 0;
     for (int g = 0; g < groups; ++g) tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
@@ -730,23 +740,23 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
         tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
         const uint32_t b_box = static_cast<uint32_t>(s.pair ? s.bn / 2 : s.bn);
         if (common->K > 0) {
-            st = make_tiled_map(&maps[4 * g], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A_ptrs_host[g], common->K, rows[g], 1,
+            st = make_tiled_map(&maps[4 * g], c.tm_in, 2, A_ptrs_host[g], common->K, rows[g], 1,
                                 common->lda, 0, 64, 128, "A_g");
             if (st != SG_OK) return st;
             if (common->layout_b == SG_ROW_MAJOR) {
-                st = make_tiled_map(&maps[4 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->N, common->K, 1,
+                st = make_tiled_map(&maps[4 * g + 1], c.tm_in, 2, B_ptrs_host[g], common->N, common->K, 1,
                                     common->ldb, 0, 64, 64, "B_g");
                 maps[4 * g + 3] = maps[4 * g + 1];
             } else {
-                st = make_tiled_map(&maps[4 * g + 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                st = make_tiled_map(&maps[4 * g + 1], c.tm_in, 2, B_ptrs_host[g], common->K, common->N, 1,
                                     common->ldb, 0, 64, b_box, "B_g");
                 if (st != SG_OK) return st;
-                st = make_tiled_map(&maps[4 * g + 3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B_ptrs_host[g], common->K, common->N, 1,
+                st = make_tiled_map(&maps[4 * g + 3], c.tm_in, 2, B_ptrs_host[g], common->K, common->N, 1,
                                     common->ldb, 0, 64, b_box / p.split, "B_g (narrow)");
             }
             if (st != SG_OK) return st;
         }
-        st = make_tiled_map(&maps[4 * g + 2], c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+        st = make_tiled_map(&maps[4 * g + 2], c.tm_out,
                             c.esize_out, D_ptrs_host[g], common->N, rows[g], 1, common->ldd, 0, c.f32_out ? 32 : 64, 32, "D_g");
         if (st != SG_OK) return st;
     }
@@ -772,7 +782,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     p.batch = groups;
     p.tiles_n = tiles_n;
     p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
-    return launch(*d, s, c.f32_out, p, stream);
+    return launch(*d, s, c.out_kind, p, stream);
 }
 
 // ---- grouped GEMM without any device allocation by anyone -----------------------------------------------
@@ -847,6 +857,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     if (st != SG_OK) return st;
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
+    p.in_f16 = c.in_f16 ? 1 : 0;
     Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_CONV;
@@ -882,7 +893,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
         int upper[2] = {static_cast<int>(desc->pad_w - (desc->S - 1) * desc->dil_w),
                         static_cast<int>(desc->pad_h - (desc->R - 1) * desc->dil_h)};
         cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(desc->stride_w), static_cast<cuuint32_t>(desc->stride_h), 1};
-        CUresult r = g_encode_im2col(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(X), dims, strides, lower, upper,
+        CUresult r = g_encode_im2col(&p.tmA, c.tm_in, 4, const_cast<void*>(X), dims, strides, lower, upper,
                                      64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(X) failed with CUresult %d", static_cast<int>(r));
@@ -894,20 +905,20 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
         cuuint64_t strides[2] = {static_cast<cuuint64_t>(desc->C) * 2, static_cast<cuuint64_t>(Kg) * 2};
         cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(s.pair ? s.bn / 2 : s.bn)};
         cuuint32_t estr[3] = {1, 1, 1};
-        CUresult r = g_encode_tiled(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(Wf), dims, strides, box, estr,
+        CUresult r = g_encode_tiled(&p.tmB, c.tm_in, 3, const_cast<void*>(Wf), dims, strides, box, estr,
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
         box[2] /= static_cast<cuuint32_t>(p.split);
-        r = g_encode_tiled(&p.tmB2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(Wf), dims, strides, box, estr,
+        r = g_encode_tiled(&p.tmB2, c.tm_in, 3, const_cast<void*>(Wf), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf, narrow) failed with CUresult %d", static_cast<int>(r));
     }
-    st = make_tiled_map(&p.tmD, c.f32_out ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, c.esize_out, Y,
+    st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, Y,
                         desc->K, Mg, 1, desc->K, 0, c.f32_out ? 32 : 64, 32, "Y");
     if (st != SG_OK) return st;
-    return launch(*d, s, c.f32_out, p, static_cast<cudaStream_t>(cuda_stream));
+    return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
 }
 
 sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* out, void* cuda_stream) {

@@ -16,6 +16,7 @@
 // roles poll, lets outstanding copies land, frees TMEM and returns.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include "sg_ptx.cuh"
 
 namespace sg {
@@ -53,11 +54,38 @@ struct alignas(64) Params {
     float alpha, beta;
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
     int32_t epi, mode;
+    int32_t in_f16;                     // 1: A, B and bias are fp16 (else bf16)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
     uint32_t* status;                   // device status words (8 x u32)
     uint64_t timeout_ns;                // bound of every device-side wait
 };
+
+// 16-bit storage types: two packed values -> two floats and back (bf16 is the upper half of an fp32; fp16 converts)
+template <bool kF16>
+__device__ __forceinline__ void unpack2(uint32_t w, float& lo, float& hi) {
+    if constexpr (kF16) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        lo = f.x;
+        hi = f.y;
+    } else {
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xFFFF0000u);
+    }
+}
+template <bool kF16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    if constexpr (kF16) {
+        const __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&h);
+    } else {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&h);
+    }
+}
+__device__ __forceinline__ float half_bits_to_float(uint16_t b, bool f16) {
+    return f16 ? __half2float(__ushort_as_half(b)) : __uint_as_float(static_cast<uint32_t>(b) << 16);
+}
 
 // Experiments only (-DSG_DEBUG_STAMPS): CTA `SG_DEBUG_STAMPS - 1` records globaltimer values at a few points of
 // its life into the words after the status words.
@@ -285,11 +313,14 @@ struct Config {
     static_assert(SMEM_BYTES <= 227 * 1024, "configuration exceeds the shared memory of one CTA");
 };
 
-template <int BN, bool kPair, bool kOutF32, int kEpiWarps>
+// kOut: 0 = bf16 output, 1 = fp32, 2 = fp16 (C, when read, has the output's type)
+template <int BN, bool kPair, int kOut, int kEpiWarps>
 __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) contract_kernel(const __grid_constant__ Params p) {
     using Cfg = Config<BN, kPair, kEpiWarps>;
     constexpr int kCtas = Cfg::kCtas;
     constexpr int STAGES = Cfg::STAGES;
+    constexpr bool kOutF32 = (kOut == 1);
+    constexpr bool kOutF16 = (kOut == 2);
     constexpr int CH = kOutF32 ? 32 : 64;          // output columns per 128-byte staging row
 
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -459,7 +490,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
                 const Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
-                const uint32_t idesc = umma_idesc_bf16_f32(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0);
+                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0, p.in_f16 != 0);
                 const uint32_t a_step = p.a_mn_major ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
                 const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
                 const int acc = iter & 1;
@@ -511,6 +542,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         constexpr int kMyBiasSlots = ((BN / CH + kStep - 1) / kStep) * CH;     // columns of the chunks one warp handles
         const bool has_bias = (p.mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
         const bool has_c = (p.beta != 0.0f);
+        const bool in_f16 = (p.in_f16 != 0);
         const float alpha = p.alpha, beta = p.beta;
         const int epi = p.epi;
         int iter = 0, g_hint = 0, g_fenced = -1;
@@ -527,14 +559,14 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const int n0 = ti.n0;
             const int row0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32;
             const CUtensorMap* mapD = &p.tmD;
-            const __nv_bfloat16* bias_g = reinterpret_cast<const __nv_bfloat16*>(p.bias);
+            const uint16_t* bias_g = reinterpret_cast<const uint16_t*>(p.bias);
             const uint8_t* c_g = reinterpret_cast<const uint8_t*>(p.C);
             uint8_t* d_g = reinterpret_cast<uint8_t*>(p.D);
             int bz = ti.b;
             if (p.mode == MODE_GROUPED) {
                 mapD = p.gmaps + 4 * ti.b + 2;
                 bz = 0;
-                if (has_bias) bias_g = reinterpret_cast<const __nv_bfloat16*>(p.g_bias[ti.b]);
+                if (has_bias) bias_g = reinterpret_cast<const uint16_t*>(p.g_bias[ti.b]);
                 if (has_c) c_g = reinterpret_cast<const uint8_t*>(p.g_C[ti.b]);
                 d_g = reinterpret_cast<uint8_t*>(p.g_D[ti.b]);
                 if (g_fenced != ti.b) {
@@ -549,7 +581,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             if (has_bias) {
                 // every warp keeps its own copy of the tile's bias values, so no barrier between warps is needed
                 __syncwarp();
-                const uint16_t* bsrc = reinterpret_cast<const uint16_t*>(bias_g);
+                const uint16_t* bsrc = bias_g;
                 for (int i = lane; i < kMyBiasSlots; i += 32) {
                     const int n = n0 + ((i / CH) * kStep + half) * CH + (i % CH);     // column of local slot i
                     bias_w[i] = (n < p.N) ? bsrc[n] : static_cast<uint16_t>(0);
@@ -671,7 +703,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                             for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += beta * cp[i];
                         }
                     } else {
-                        const __nv_bfloat16* cp = reinterpret_cast<const __nv_bfloat16*>(c_g) + static_cast<int64_t>(row) * p.ldc + col0;
+                        const uint16_t* cp = reinterpret_cast<const uint16_t*>(c_g) + static_cast<int64_t>(row) * p.ldc + col0;
                         if (col0 + CH <= p.N) {
 #pragma unroll
                             for (int i = 0; i < CH; i += 8) {
@@ -679,12 +711,14 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                                 const uint32_t w[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) {
-                                    v[i + 2 * j] += beta * __uint_as_float(w[j] << 16);
-                                    v[i + 2 * j + 1] += beta * __uint_as_float(w[j] & 0xFFFF0000u);
+                                    float lo, hi;
+                                    unpack2<kOutF16>(w[j], lo, hi);
+                                    v[i + 2 * j] += beta * lo;
+                                    v[i + 2 * j + 1] += beta * hi;
                                 }
                             }
                         } else {
-                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += beta * __bfloat162float(cp[i]);
+                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += beta * half_bits_to_float(cp[i], kOutF16);
                         }
                     }
                 }
@@ -692,13 +726,15 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int i = 0; i < CH; i += 4) {
                         const uint2 b2 = *reinterpret_cast<const uint2*>(bias_w + (c / kStep) * CH + i);   // 4 bf16, broadcast read
-                        v[i] += __uint_as_float(b2.x << 16); v[i + 1] += __uint_as_float(b2.x & 0xFFFF0000u);
-                        v[i + 2] += __uint_as_float(b2.y << 16); v[i + 3] += __uint_as_float(b2.y & 0xFFFF0000u);
+                        float b0, b1, b2f, b3;
+                        if (in_f16) { unpack2<true>(b2.x, b0, b1); unpack2<true>(b2.y, b2f, b3); }
+                        else { unpack2<false>(b2.x, b0, b1); unpack2<false>(b2.y, b2f, b3); }
+                        v[i] += b0; v[i + 1] += b1; v[i + 2] += b2f; v[i + 3] += b3;
                     }
                 }
                 if (epi >= EPI_RELU) {
 #pragma unroll
-                    for (int i = 0; i < CH; ++i) v[i] = apply_act<!kOutF32>(v[i], epi, p.epi_arg0, p.epi_arg1);
+                    for (int i = 0; i < CH; ++i) v[i] = apply_act<kOut == 0>(v[i], epi, p.epi_arg0, p.epi_arg1);
                 }
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
@@ -711,8 +747,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                             float* dp = reinterpret_cast<float*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
                             for (int i = 0; i < CH; ++i) if (col0 + i < p.N) dp[i] = v[i];
                         } else {
-                            __nv_bfloat16* dp = reinterpret_cast<__nv_bfloat16*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
-                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) dp[i] = __float2bfloat16_rn(v[i]);
+                            uint16_t* dp = reinterpret_cast<uint16_t*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
+                            for (int i = 0; i < CH; ++i)
+                                if (col0 + i < p.N) dp[i] = static_cast<uint16_t>(pack2<kOutF16>(v[i], 0.0f) & 0xFFFFu);
                         }
                     }
                     __syncwarp();
@@ -736,12 +773,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         w0 = __float_as_uint(v[4 * j]); w1 = __float_as_uint(v[4 * j + 1]);
                         w2 = __float_as_uint(v[4 * j + 2]); w3 = __float_as_uint(v[4 * j + 3]);
                     } else {
-                        __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * j], v[8 * j + 1]);
-                        __nv_bfloat162 h1 = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
-                        __nv_bfloat162 h3 = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
-                        w0 = *reinterpret_cast<uint32_t*>(&h0); w1 = *reinterpret_cast<uint32_t*>(&h1);
-                        w2 = *reinterpret_cast<uint32_t*>(&h2); w3 = *reinterpret_cast<uint32_t*>(&h3);
+                        w0 = pack2<kOutF16>(v[8 * j], v[8 * j + 1]);
+                        w1 = pack2<kOutF16>(v[8 * j + 2], v[8 * j + 3]);
+                        w2 = pack2<kOutF16>(v[8 * j + 4], v[8 * j + 5]);
+                        w3 = pack2<kOutF16>(v[8 * j + 6], v[8 * j + 7]);
                     }
                     const uint32_t addr = row_addr + ((static_cast<uint32_t>(j) ^ (lane & 7u)) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");

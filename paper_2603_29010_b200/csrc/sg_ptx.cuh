@@ -274,11 +274,12 @@ __device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t smem_addr)
     return d;
 }
 
-// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, both K-major, no
-// negation, dense.  bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format,
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 or fp16 A and B, no negation, dense.  bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format,
 // 15 / 16 A / B major (0 = K), 17-22 N >> 3, 24-28 M >> 4.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n, bool a_mn_major = false, bool b_mn_major = false) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
+// in_f16 selects fp16 (format code 0) instead of bf16 (format code 1) for both A and B.
+__host__ __device__ constexpr uint32_t umma_idesc_f32acc(int m, int n, bool a_mn_major, bool b_mn_major, bool in_f16) {
+    const uint32_t fmt = in_f16 ? 0u : 1u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 

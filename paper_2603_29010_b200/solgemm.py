@@ -32,7 +32,7 @@ STATUS_NAMES = ["SG_OK", "SG_ERR_INVALID_ARG", "SG_ERR_NULL_POINTER", "SG_ERR_AL
 LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
-DTYPES = {torch.bfloat16: 0, torch.float32: 1}
+DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2}
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop",
@@ -179,8 +179,8 @@ def _ld(t: torch.Tensor) -> int:
 
 
 def _gemm_desc(M, N, K, lda, ldb, ldc, ldd, layout_a, layout_b, out_dtype, alpha, beta, epi,
-               epi_args=(0.0, 0.0)) -> GemmDesc:
-    return GemmDesc(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], lda, ldb, ldc, ldd, 0, DTYPES[out_dtype],
+               epi_args=(0.0, 0.0), in_dtype=torch.bfloat16) -> GemmDesc:
+    return GemmDesc(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], lda, ldb, ldc, ldd, DTYPES[in_dtype], DTYPES[out_dtype],
                     float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), 0)
 
 
@@ -202,7 +202,7 @@ def gemm(A: torch.Tensor, B: torch.Tensor, *, C: Optional[torch.Tensor] = None, 
     if out is None:
         out = torch.empty((M, N), dtype=out_dtype, device=A.device)
     desc = _gemm_desc(M, N, K, _ld(A), _ld(B), _ld(C) if C is not None else max(N, 1), _ld(out), layout_a, layout_b,
-                      out.dtype, alpha, beta, epi, epi_args)
+                      out.dtype, alpha, beta, epi, epi_args, A.dtype)
     _check(_lib.sg_gemm(ctypes.byref(desc), _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
     return out
 
@@ -221,7 +221,7 @@ def batched_gemm(A: torch.Tensor, B: torch.Tensor, *, C=None, bias=None, out=Non
             raise ValueError("batched operands must be 3-D with inner stride 1")
     sbias = 0 if bias is None or bias.dim() == 1 else bias.stride(0)
     desc = _gemm_desc(M, N, K, A.stride(1), B.stride(1), C.stride(1) if C is not None else max(N, 1), out.stride(1),
-                      layout_a, layout_b, out.dtype, alpha, beta, epi, epi_args)
+                      layout_a, layout_b, out.dtype, alpha, beta, epi, epi_args, A.dtype)
     _check(_lib.sg_batched_gemm(ctypes.byref(desc), batch, A.stride(0), B.stride(0),
                                 C.stride(0) if C is not None else 0, out.stride(0), sbias,
                                 _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
@@ -258,7 +258,7 @@ def grouped_gemm(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], *, Cs=N
         outs = [torch.empty((m, N), dtype=out_dtype, device=As[0].device) for m in Ms]
     ld = lambda ts, default: next((_ld(t) for t in ts if t.shape[0] > 1), default)
     desc = _gemm_desc(0, N, K, ld(As, max(K, 1)), ld(Bs, max(K, 1)), ld(Cs, max(N, 1)) if Cs is not None else max(N, 1),
-                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi, epi_args)
+                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi, epi_args, As[0].dtype)
     if workspace is None:
         workspace = torch.empty(grouped_workspace_size(groups), dtype=torch.uint8, device=As[0].device)
     m_arr = (ctypes.c_int64 * groups)(*Ms)
@@ -287,7 +287,7 @@ def grouped_gemm_static(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], 
     Ms = [(_mnk(a, b, layout_a, layout_b))[0] for a, b in zip(As, Bs)]
     ld = lambda ts, default: next((_ld(t) for t in ts if t.shape[0] > 1), default)
     desc = _gemm_desc(0, N, K, ld(As, max(K, 1)), ld(Bs, max(K, 1)), ld(Cs, max(N, 1)) if Cs is not None else max(N, 1),
-                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi, epi_args)
+                      ld(outs, max(N, 1)), layout_a, layout_b, outs[0].dtype, alpha, beta, epi, epi_args, As[0].dtype)
     m_arr = (ctypes.c_int64 * groups)(*Ms)
     _check(_lib.sg_grouped_gemm_static(ctypes.byref(desc), groups, m_arr, _ptr_array(As), _ptr_array(Bs),
                                        _ptr_array(Cs), _ptr_array(biases), _ptr_array(outs), _stream(stream)))
@@ -309,7 +309,8 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
     ensure_scratch()
     if out is None:
         out = torch.empty((N, P, Q, K), dtype=out_dtype, device=X.device)
-    desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], 0, DTYPES[out.dtype],
+    desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], DTYPES[X.dtype],
+                      DTYPES[out.dtype],
                       float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), 0)
     _check(_lib.sg_conv2d_fprop(ctypes.byref(desc), _ptr(X), _ptr(Wf), _ptr(Cin), _ptr(bias), _ptr(out), _stream(stream)))
     return out

@@ -1,6 +1,8 @@
 """Element-by-element comparison of a computed result with the oracle's fp64 reference.
 
 bf16 output:  |D - ref| <= 1e-2 + 1e-2 |ref|                      (every element)
+fp16 output:  |D - ref| <= 1e-3 + 1e-3 |ref| + 1e-4 * absacc      (one fp16 rounding is 2^-11 = 4.9e-4 relative;
+              the last term is the fp32 path's bound for the accumulation)
 fp32 output:  |D - ref| <= 1e-4 * absacc,  absacc = |alpha| sum|a||b| + |beta c| + |bias|
               (relative to the magnitude of the terms summed, so that results
               near zero from cancellation are judged on the dot product's scale)
@@ -17,6 +19,8 @@ F32_RTOL = 1e-4
 def allowed_error(ref: torch.Tensor, absacc: torch.Tensor, out_dtype: torch.dtype) -> torch.Tensor:
     if out_dtype == torch.bfloat16:
         return BF16_ATOL + BF16_RTOL * ref.abs()
+    if out_dtype == torch.float16:
+        return 1e-3 + 1e-3 * ref.abs() + F32_RTOL * absacc
     if out_dtype == torch.float32:
         return F32_RTOL * absacc
     raise ValueError(out_dtype)

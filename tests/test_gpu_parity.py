@@ -508,3 +508,53 @@ def test_layout_pipeline_nchw_conv_nchw_and_conv1d():
     ref1, _ = orc.conv2d_fprop(X1.view(3, 1, 50, 32), W1.view(40, 1, 5, 32), pad=(0, 2), stride=(1, 2))
     y1 = sg.conv1d_fprop(X1.to(DEV), W1.to(DEV), pad=2, stride=2)
     parity.assert_bit_exact(y1, ref1.view(3, -1, 40), "conv1d")
+
+
+# ---------------------------------------------------------------------------------------- fp16 inputs / outputs
+
+@pytest.mark.parametrize("tile_n,pair", [(64, 0), (256, 0), (128, 1), (256, 1)])
+@pytest.mark.parametrize("out_dtype", [torch.float16, torch.float32, torch.bfloat16])
+def test_fp16_inputs_integer_problem_bit_exact(out_dtype, tile_n, pair):
+    sg.set_tuning(tile_n, pair)
+    M, N, K = 300, 200, 136
+    A = inputs.small_integers([M, K], 717, 1).half()
+    B = inputs.small_integers([N, K], 717, 2).half()
+    ref, _ = orc.gemm(A, B)
+    D = sg.gemm(A.to(DEV), B.to(DEV), out_dtype=out_dtype)
+    parity.assert_bit_exact(D, ref, f"fp16 in, {out_dtype} out")
+
+
+@pytest.mark.parametrize("epi", ["none", "relu", "gelu", "silu"])
+def test_fp16_dsl_example_dtype_triple_with_bias_and_residual(epi):
+    # the DSL's running example: input=fp16, acc=fp32, output=fp16, with a bias and an activation
+    M, N, K = 200, 328, 264
+    A = (inputs.normal([M, K], 727, 1).float() * K ** -0.25).half()
+    B = (inputs.normal([N, K], 727, 2).float() * K ** -0.25).half()
+    bias = inputs.normal([N], 727, 4).half()
+    C = inputs.normal([M, N], 727, 3).half()
+    ref, absacc = orc.gemm(A, B, C=C, bias=bias, alpha=0.75, beta=-0.5, epi=epi)
+    D = sg.gemm(A.to(DEV), B.to(DEV), C=C.to(DEV), bias=bias.to(DEV), alpha=0.75, beta=-0.5, epi=epi, out_dtype=torch.float16)
+    parity.assert_matches(D, ref, absacc, f"fp16 {epi}")
+    # ragged N (plain-store path), batched, grouped and convolution with fp16 operands
+    refr, accr = orc.gemm(A, B[:90], bias=bias[:90].contiguous(), epi=epi)
+    big = torch.full((M, 96), float("nan"), dtype=torch.float16, device=DEV)
+    sg.gemm(A.to(DEV), B[:90].to(DEV), bias=bias[:90].contiguous().to(DEV), epi=epi, out=big[:, :90])
+    parity.assert_matches(big[:, :90], refr, accr, "fp16 ragged N")
+    assert bool(torch.isnan(big[:, 90:]).all())
+
+
+def test_fp16_batched_grouped_and_conv():
+    A = (inputs.uniform([3, 72, 136], 737, 1)).half()
+    B = (inputs.uniform([3, 64, 136], 737, 2)).half()
+    ref, absacc = orc.batched_gemm(A, B, epi="relu")
+    parity.assert_matches(sg.batched_gemm(A.to(DEV), B.to(DEV), epi="relu", out_dtype=torch.float16), ref, absacc, "fp16 batched")
+    As = [inputs.small_integers([m, 72], 747 + g, 1).half() for g, m in enumerate([130, 40])]
+    Bs = [inputs.small_integers([136, 72], 747 + g, 2).half() for g in range(2)]
+    refs, _ = orc.grouped_gemm(As, Bs)
+    outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs], out_dtype=torch.float16)
+    for g in range(2):
+        parity.assert_bit_exact(outs[g], refs[g], f"fp16 grouped {g}")
+    X = inputs.small_integers([2, 9, 11, 64], 757, 6, -1, 1).half()
+    Wf = (inputs.small_integers([72, 3, 3, 64], 757, 7, -1, 1) * (inputs.small_integers([72, 3, 3, 64], 758, 7, 0, 3) == 0).to(torch.bfloat16)).half()
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    parity.assert_bit_exact(sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1), out_dtype=torch.float16), ref, "fp16 conv")

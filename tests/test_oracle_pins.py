@@ -407,3 +407,35 @@ def test_transpose_matches_torch_permute_and_cast():
     padded[:, :, :29] = x32
     assert torch.equal(orc.transpose(padded[:, :, :29], torch.bfloat16), x32.permute(0, 2, 1).to(torch.bfloat16).double())
     assert orc.transpose_bytes(32, 256, 3136, 4, 2) == 32 * 256 * 3136 * 6
+
+
+# ---------------------------------------------------------------- fp16 inputs
+
+def test_fp16_inputs_are_widened_exactly():
+    # every one of the 65536 binary16 patterns, through the oracle's own decoder (a K = 1 product with 1.0)
+    bits = torch.arange(0, 65536, dtype=torch.int32).to(torch.int16).view(torch.float16)
+    finite = torch.isfinite(bits)
+    col = bits[finite].view(-1, 1)
+    one = torch.ones(1, 1, dtype=torch.float16)
+    ref, _ = orc.gemm(col, one)
+    assert torch.equal(ref.view(-1), col.double().view(-1))            # torch's own widening as the library pin
+    assert float(orc.gemm(torch.tensor([[6.103515625e-05]], dtype=torch.float16), one)[0]) == 2.0 ** -14
+    assert float(orc.gemm(torch.tensor([[5.960464477539063e-08]], dtype=torch.float16), one)[0]) == 2.0 ** -24   # smallest subnormal
+    assert float(orc.gemm(torch.tensor([[65504.0]], dtype=torch.float16), one)[0]) == 65504.0
+
+
+def test_fp16_gemm_and_conv_match_torch_fp64():
+    A = (inputs.uniform([23, 41], 31, 1).float() * 3.3).half()
+    Bt = (inputs.uniform([17, 41], 31, 2).float() * 0.7).half()
+    bias = inputs.normal([17], 31, 4).half()
+    C = inputs.normal([23, 17], 31, 3).half()
+    ref, _ = orc.gemm(A, Bt, C=C, bias=bias, alpha=0.5, beta=2.0, epi="bias")
+    want = 0.5 * (A.double() @ Bt.double().t()) + 2.0 * C.double() + bias.double()
+    assert torch.allclose(ref, want, rtol=0, atol=1e-12)
+    X = inputs.uniform([2, 6, 7, 5], 32, 6).half()
+    Wf = inputs.uniform([4, 3, 3, 5], 32, 7).half()
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    want = torch.nn.functional.conv2d(X.double().permute(0, 3, 1, 2), Wf.double().permute(0, 3, 1, 2), padding=1).permute(0, 2, 3, 1)
+    assert torch.allclose(ref, want, rtol=0, atol=1e-12)
+    with pytest.raises(ValueError):
+        orc.gemm(A, Bt.to(torch.bfloat16))
