@@ -21,6 +21,9 @@
  *    output D is bf16, fp16 or fp32 (`out_dtype`); C, when read, has the output's dtype and shape.
  *    Accumulation and the epilogue run in fp32; the result is rounded to nearest-even.
  *    (The DSL's .with_dtype(input, acc, output); its running example is input=fp16, acc=fp32, output=fp16.)
+ *    A and B (conv: X and Wf) may also be 8-bit floating point, SG_FP8_E4M3 or SG_FP8_E5M2 (both the same;
+ *    the DSL's fp8_e4m3 / fp8_e5m2 input types): K-contiguous layouts only, leading dimensions multiples of 16
+ *    elements; the bias then is bf16, the output bf16, fp16 or fp32.  Scale factors go through alpha.
  *  - Epilogue: v = alpha*acc (+ beta*C if beta != 0) (+ bias[j] if bias != NULL); D = act(v).
  *    bias holds one value per output column j (GEMM) or output channel (conv); it is NOT scaled
  *    by alpha.  SG_EPI_BIAS is the identity activation and requires bias != NULL; every other
@@ -59,7 +62,7 @@ typedef enum {
     SG_ERR_TIMEOUT = 8        /* a bounded device-side wait expired (see sg_poll_status) */
 } sg_status_t;
 
-typedef enum { SG_BF16 = 0, SG_F32 = 1, SG_F16 = 2 } sg_dtype_t;
+typedef enum { SG_BF16 = 0, SG_F32 = 1, SG_F16 = 2, SG_FP8_E4M3 = 3, SG_FP8_E5M2 = 4 } sg_dtype_t;
 typedef enum { SG_ROW_MAJOR = 0, SG_COL_MAJOR = 1 } sg_layout_t;
 typedef enum {
     SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4,
@@ -86,7 +89,7 @@ typedef struct sg_gemm_desc {
     int64_t M, N, K;
     int32_t layout_a, layout_b;   /* sg_layout_t */
     int64_t lda, ldb, ldc, ldd;
-    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype SG_BF16 or SG_F16 */
+    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype SG_BF16, SG_F16, SG_FP8_E4M3 or SG_FP8_E5M2 */
     float alpha, beta;
     int32_t epi;                  /* sg_epilogue_t */
     float epi_arg0, epi_arg1;     /* activation parameters (leaky_relu / elu slope, clip bounds); else ignored */
@@ -166,7 +169,8 @@ sg_status_t sg_grouped_gemm_static(const sg_gemm_desc_t* common, int32_t groups,
  *   Y[n,p,q,k] = act( alpha * sum_{r,s,c} X[n, p stride_h - pad_h + r dil_h, q stride_w - pad_w + s dil_w, c]
  *                                         * Wf[k,r,s,c]  + beta * Cin[n,p,q,k] + bias[k] ),
  *   taps outside the image contribute zero.  The im2col matrix is never materialised.
- * Requires C % 8 == 0 and K % 8 == 0 (16-byte rule) and pads / filter extents within the TMA
+ * Requires C * (input element size) and K * (output element size) to be multiples of 16 bytes (C % 8 == 0 and
+ * K % 8 == 0 for bf16; C % 16 == 0 for 8-bit inputs) and pads / filter extents within the TMA
  * im2col limits (pad <= 127, (R-1) dil_h <= 255, (S-1) dil_w <= 255), else SG_ERR_ALIGNMENT /
  * SG_ERR_UNSUPPORTED.
  */

@@ -32,8 +32,14 @@ _LIB = os.path.join(_HERE, "libsg_oracle.so")
 LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
-_DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2}
-_IN_DTYPES = (torch.bfloat16, torch.float16)
+_DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4}
+_IN_DTYPES = (torch.bfloat16, torch.float16, torch.float8_e4m3fn, torch.float8_e5m2)
+_FP8 = (torch.float8_e4m3fn, torch.float8_e5m2)
+
+
+def bias_dtype_for(in_dtype: torch.dtype) -> torch.dtype:
+    """The bias has the inputs' type, except that 8-bit inputs come with a bf16 bias."""
+    return torch.bfloat16 if in_dtype in _FP8 else in_dtype
 
 
 def build(force: bool = False) -> str:
@@ -59,17 +65,17 @@ def lib() -> ctypes.CDLL:
         L.orc_act2.restype = dbl
         L.orc_act2.argtypes = [ci, dbl, dbl, dbl]
         L.orc_gemm.restype = ci
-        L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl, ci,
+        L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, ci, dbl, dbl, ci, dbl, dbl, ci,
                                i64, i64, vp, vp, i64]
         L.orc_gemm_points.restype = ci
-        L.orc_gemm_points.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, dbl, dbl, ci, dbl, dbl, ci,
+        L.orc_gemm_points.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, ci, dbl, dbl, ci, dbl, dbl, ci,
                                       i64, vp, vp, vp, vp]
         L.orc_conv_out_extent.restype = i64
         L.orc_conv_out_extent.argtypes = [i64] * 5
         L.orc_conv2d_fprop.restype = ci
-        L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, ci, i64, i64, vp, vp]
+        L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, ci, dbl, dbl, ci, dbl, dbl, ci, i64, i64, vp, vp]
         L.orc_conv2d_points.restype = ci
-        L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, dbl, dbl, ci, dbl, dbl, ci, i64, vp, vp, vp, vp]
+        L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, ci, dbl, dbl, ci, dbl, dbl, ci, i64, vp, vp, vp, vp]
         L.orc_transpose.restype = ci
         L.orc_transpose.argtypes = [i64, i64, i64, vp, ci, i64, i64, ci, vp]
         L.orc_transpose_bytes.restype = i64
@@ -102,7 +108,7 @@ def _ptr(t: Optional[torch.Tensor]):
 
 def _check2d(t: torch.Tensor, name: str):
     if t.device.type != "cpu" or t.dim() != 2 or t.dtype not in _IN_DTYPES:
-        raise ValueError(f"{name}: want a 2-D CPU bf16 or fp16 tensor")
+        raise ValueError(f"{name}: want a 2-D CPU bf16, fp16 or fp8 tensor")
     if t.shape[1] > 1 and t.stride(1) != 1:
         raise ValueError(f"{name}: inner stride must be 1")
 
@@ -143,14 +149,14 @@ def gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a: str = "row", layout_b: s
          rows: Optional[Tuple[int, int]] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """act(alpha A.B + beta C + bias) for rows ``rows=(begin, end)`` (default: all)."""
     M, N, K, lda, ldb = _gemm_shapes(A, B, layout_a, layout_b)
-    _check_bias(bias, N, A.dtype)
+    _check_bias(bias, N, bias_dtype_for(A.dtype))
     C, c_dtype, ldc = _c_args(C, M, N)
     r0, r1 = rows if rows is not None else (0, M)
     ref = torch.empty((r1 - r0, N), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
-                        _ptr(C), c_dtype, ldc, _ptr(bias), float(alpha), float(beta), EPILOGUES[epi],
-                        float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], r0, r1, _ptr(ref), _ptr(absacc),
+                        _ptr(C), c_dtype, ldc, _ptr(bias), _DTYPES[bias_dtype_for(A.dtype)], float(alpha), float(beta),
+                        EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], r0, r1, _ptr(ref), _ptr(absacc),
                         max(N, 1))
     if rc:
         raise ValueError(f"orc_gemm rejected its arguments (code {rc})")
@@ -161,15 +167,15 @@ def gemm_points(A, B, pi: Sequence[int], pj: Sequence[int], *, layout_a="row", l
                 alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)) -> Tuple[torch.Tensor, torch.Tensor]:
     """The elements (pi[t], pj[t]) of the result only."""
     M, N, K, lda, ldb = _gemm_shapes(A, B, layout_a, layout_b)
-    _check_bias(bias, N, A.dtype)
+    _check_bias(bias, N, bias_dtype_for(A.dtype))
     C, c_dtype, ldc = _c_args(C, M, N)
     pi = torch.as_tensor(pi, dtype=torch.int64).contiguous()
     pj = torch.as_tensor(pj, dtype=torch.int64).contiguous()
     ref = torch.empty(pi.numel(), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm_points(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
-                               _ptr(C), c_dtype, ldc, _ptr(bias), float(alpha), float(beta), EPILOGUES[epi],
-                               float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], pi.numel(), _ptr(pi), _ptr(pj),
+                               _ptr(C), c_dtype, ldc, _ptr(bias), _DTYPES[bias_dtype_for(A.dtype)], float(alpha),
+                               float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], pi.numel(), _ptr(pi), _ptr(pj),
                                _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_gemm_points rejected its arguments (code {rc})")
@@ -206,7 +212,7 @@ def conv_out_extent(size: int, pad: int, dil: int, filt: int, stride: int) -> in
 
 def _conv_dims(X, Wf, pad, stride, dil):
     if X.device.type != "cpu" or X.dim() != 4 or X.dtype not in _IN_DTYPES or not X.is_contiguous():
-        raise ValueError("X: want a contiguous CPU bf16 or fp16 NHWC tensor")
+        raise ValueError("X: want a contiguous CPU bf16, fp16 or fp8 NHWC tensor")
     if Wf.device.type != "cpu" or Wf.dim() != 4 or Wf.dtype != X.dtype or not Wf.is_contiguous():
         raise ValueError("Wf: want a contiguous CPU KRSC tensor of X's dtype")
     N, H, W, C = X.shape
@@ -233,12 +239,12 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
                  pixels: Optional[Tuple[int, int]] = None):
     """Direct convolution; returns ``[N,P,Q,K]`` tensors, or ``[pixels, K]`` for a flattened pixel range."""
     d, N, P, Q, K = _conv_dims(X, Wf, pad, stride, dil)
-    _check_bias(bias, K, X.dtype)
+    _check_bias(bias, K, bias_dtype_for(X.dtype))
     Cin, c_dtype = _conv_c(Cin, N, P, Q, K)
     p0, p1 = pixels if pixels is not None else (0, N * P * Q)
     ref = torch.empty((p1 - p0, K), dtype=torch.float64)
     absacc = torch.empty_like(ref)
-    rc = lib().orc_conv2d_fprop(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
+    rc = lib().orc_conv2d_fprop(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias), _DTYPES[bias_dtype_for(X.dtype)],
                                 float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
                                 _DTYPES[X.dtype], p0, p1, _ptr(ref), _ptr(absacc))
     if rc:
@@ -252,14 +258,14 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
                   Cin=None, bias=None, alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0)):
     """The outputs (flattened pixel ppix[t], channel pk[t]) only."""
     d, N, P, Q, K = _conv_dims(X, Wf, pad, stride, dil)
-    _check_bias(bias, K, X.dtype)
+    _check_bias(bias, K, bias_dtype_for(X.dtype))
     Cin, c_dtype = _conv_c(Cin, N, P, Q, K)
     ppix = torch.as_tensor(ppix, dtype=torch.int64).contiguous()
     pk = torch.as_tensor(pk, dtype=torch.int64).contiguous()
     ref = torch.empty(ppix.numel(), dtype=torch.float64)
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_points(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
-                                 float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
+                                 _DTYPES[bias_dtype_for(X.dtype)], float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
                                  _DTYPES[X.dtype], ppix.numel(), _ptr(ppix), _ptr(pk), _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_points rejected its arguments (code {rc})")

@@ -45,7 +45,7 @@
 #endif
 
 enum { ORC_ROW_MAJOR = 0, ORC_COL_MAJOR = 1 };
-enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2 };
+enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2, ORC_FP8_E4M3 = 3, ORC_FP8_E5M2 = 4 };
 enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4,
        ORC_EPI_SIGMOID = 5, ORC_EPI_TANH = 6, ORC_EPI_MISH = 7, ORC_EPI_HARDSWISH = 8, ORC_EPI_LEAKY_RELU = 9,
        ORC_EPI_ELU = 10, ORC_EPI_CLIP = 11 };
@@ -77,8 +77,35 @@ static double f16_to_f64(uint16_t bits) {
     return sign ? -v : v;
 }
 
-/* The two 16-bit input formats (.with_dtype(input=bf16 | fp16, ...)). */
-static double in16_to_f64(uint16_t bits, int dtype) { return dtype == ORC_F16 ? f16_to_f64(bits) : bf16_to_f64(bits); }
+/* 8-bit floats (the DSL's fp8_e4m3 / fp8_e5m2).  e4m3 ("fn" flavour): 1 sign, 4 exponent (bias 7), 3 fraction
+ * bits, no infinities, only S.1111.111 is NaN, largest value 448.  e5m2: 1, 5 (bias 15), 2, IEEE-like with
+ * infinities and NaNs. */
+static double fp8_e4m3_to_f64(uint8_t bits) {
+    int sign = bits >> 7, e = (bits >> 3) & 0xF, f = bits & 0x7;
+    double v;
+    if (e == 15 && f == 7) v = NAN;
+    else if (e == 0) v = ldexp((double)f, -9);                    /* subnormals: f/8 * 2^-6 */
+    else v = ldexp(1.0 + (double)f / 8.0, e - 7);
+    return sign ? -v : v;
+}
+static double fp8_e5m2_to_f64(uint8_t bits) {
+    int sign = bits >> 7, e = (bits >> 2) & 0x1F, f = bits & 0x3;
+    double v;
+    if (e == 31) v = f ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)f, -16);                   /* subnormals: f/4 * 2^-14 */
+    else v = ldexp(1.0 + (double)f / 4.0, e - 15);
+    return sign ? -v : v;
+}
+
+/* Element idx of an input operand (.with_dtype(input=bf16 | fp16 | fp8_e4m3 | fp8_e5m2, ...)), widened exactly. */
+static double in_to_f64(const void* p, int dtype, int64_t idx) {
+    switch (dtype) {
+        case ORC_F16: return f16_to_f64(((const uint16_t*)p)[idx]);
+        case ORC_FP8_E4M3: return fp8_e4m3_to_f64(((const uint8_t*)p)[idx]);
+        case ORC_FP8_E5M2: return fp8_e5m2_to_f64(((const uint8_t*)p)[idx]);
+        default: return bf16_to_f64(((const uint16_t*)p)[idx]);
+    }
+}
 
 static double load_as_f64(const void* p, int dtype, int64_t idx) {
     if (dtype == ORC_BF16) return bf16_to_f64(((const uint16_t*)p)[idx]);
@@ -134,22 +161,22 @@ double orc_act(int epi, double x) { return orc_act2(epi, x, 0.0, 0.0); }
 typedef struct {
     int64_t M, N, K;
     int layout_a, layout_b;
-    const uint16_t* A; int64_t lda;
-    const uint16_t* B; int64_t ldb;
+    const void* A; int64_t lda;
+    const void* B; int64_t ldb;
     const void* C; int c_dtype; int64_t ldc;     /* read only when beta != 0 */
-    const uint16_t* bias;                        /* [N] or NULL */
+    const void* bias; int bias_dtype;            /* [N] or NULL */
     double alpha, beta;
     int epi;
     double a0, a1;                               /* activation parameters */
-    int in_dtype;                                /* ORC_BF16 or ORC_F16: type of A, B and bias */
+    int in_dtype;                                /* type of A and B */
 } gemm_problem;
 
 /* One output element and, optionally, the magnitude sum used to scale fp32 tolerances. */
 static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* absacc) {
     double sum = 0.0, asum = 0.0;
     for (int64_t k = 0; k < g->K; ++k) {
-        double a = in16_to_f64(g->layout_a == ORC_ROW_MAJOR ? g->A[i * g->lda + k] : g->A[k * g->lda + i], g->in_dtype);
-        double b = in16_to_f64(g->layout_b == ORC_ROW_MAJOR ? g->B[k * g->ldb + j] : g->B[j * g->ldb + k], g->in_dtype);
+        double a = in_to_f64(g->A, g->in_dtype, g->layout_a == ORC_ROW_MAJOR ? i * g->lda + k : k * g->lda + i);
+        double b = in_to_f64(g->B, g->in_dtype, g->layout_b == ORC_ROW_MAJOR ? k * g->ldb + j : j * g->ldb + k);
         sum += a * b;
         asum += fabs(a * b);
     }
@@ -161,7 +188,7 @@ static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* 
         av += fabs(g->beta * c);
     }
     if (g->bias) {
-        double bj = in16_to_f64(g->bias[j], g->in_dtype);
+        double bj = in_to_f64(g->bias, g->bias_dtype, j);
         v += bj;
         av += fabs(bj);
     }
@@ -174,13 +201,13 @@ static double gemm_element(const gemm_problem* g, int64_t i, int64_t j, double* 
  * (row_end-row_begin) x N values, row stride ldr, row 0 = row_begin.
  */
 int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
-             const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
-             const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
+             const void* A, int64_t lda, const void* B, int64_t ldb,
+             const void* C, int c_dtype, int64_t ldc, const void* bias, int bias_dtype,
              double alpha, double beta, int epi, double a0, double a1, int in_dtype,
              int64_t row_begin, int64_t row_end, double* ref, double* absacc, int64_t ldr) {
     if (M < 0 || N < 0 || K < 0 || row_begin < 0 || row_end > M || row_begin > row_end) return 1;
     if (beta != 0.0 && !C) return 2;
-    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1, in_dtype};
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, bias_dtype, alpha, beta, epi, a0, a1, in_dtype};
 #pragma omp parallel for schedule(static)
     for (int64_t i = row_begin; i < row_end; ++i) {
         for (int64_t j = 0; j < N; ++j) {
@@ -195,12 +222,12 @@ int orc_gemm(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
 
 /* The listed elements (pi[t], pj[t]) only: used to spot-check full-size problems. */
 int orc_gemm_points(int64_t M, int64_t N, int64_t K, int layout_a, int layout_b,
-                    const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb,
-                    const void* C, int c_dtype, int64_t ldc, const uint16_t* bias,
+                    const void* A, int64_t lda, const void* B, int64_t ldb,
+                    const void* C, int c_dtype, int64_t ldc, const void* bias, int bias_dtype,
                     double alpha, double beta, int epi, double a0, double a1, int in_dtype,
                     int64_t npts, const int64_t* pi, const int64_t* pj, double* ref, double* absacc) {
     if (beta != 0.0 && !C) return 2;
-    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, alpha, beta, epi, a0, a1, in_dtype};
+    gemm_problem g = {M, N, K, layout_a, layout_b, A, lda, B, ldb, C, c_dtype, ldc, bias, bias_dtype, alpha, beta, epi, a0, a1, in_dtype};
     for (int64_t t = 0; t < npts; ++t)
         if (pi[t] < 0 || pi[t] >= M || pj[t] < 0 || pj[t] >= N) return 1;
 #pragma omp parallel for schedule(static)
@@ -223,9 +250,9 @@ typedef struct {
     int64_t N, H, W, C, K, R, S;
     int64_t pad_h, pad_w, stride_h, stride_w, dil_h, dil_w;
     int64_t P, Q;
-    const uint16_t* X; const uint16_t* Wf;
+    const void* X; const void* Wf;
     const void* Cin; int c_dtype;
-    const uint16_t* bias;
+    const void* bias; int bias_dtype;
     double alpha, beta;
     int epi;
     double a0, a1;
@@ -246,10 +273,10 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
         for (int64_t s = 0; s < cv->S; ++s) {
             int64_t w = q * cv->stride_w - cv->pad_w + s * cv->dil_w;
             if (w < 0 || w >= cv->W) continue;
-            const uint16_t* xp = cv->X + ((n * cv->H + h) * cv->W + w) * cv->C;
-            const uint16_t* wp = cv->Wf + ((k * cv->R + r) * cv->S + s) * cv->C;
+            const int64_t xo = ((n * cv->H + h) * cv->W + w) * cv->C;
+            const int64_t wo = ((k * cv->R + r) * cv->S + s) * cv->C;
             for (int64_t c = 0; c < cv->C; ++c) {
-                double t = in16_to_f64(xp[c], cv->in_dtype) * in16_to_f64(wp[c], cv->in_dtype);
+                double t = in_to_f64(cv->X, cv->in_dtype, xo + c) * in_to_f64(cv->Wf, cv->in_dtype, wo + c);
                 sum += t;
                 asum += fabs(t);
             }
@@ -263,7 +290,7 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
         av += fabs(cv->beta * c);
     }
     if (cv->bias) {
-        double bk = in16_to_f64(cv->bias[k], cv->in_dtype);
+        double bk = in_to_f64(cv->bias, cv->bias_dtype, k);
         v += bk;
         av += fabs(bk);
     }
@@ -271,8 +298,8 @@ static double conv_element(const conv_problem* cv, int64_t n, int64_t p, int64_t
     return orc_act2(cv->epi, v, cv->a0, cv->a1);
 }
 
-static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, const uint16_t* Wf,
-                      const void* Cin, int c_dtype, const uint16_t* bias, double alpha, double beta, int epi,
+static int conv_setup(conv_problem* cv, const int64_t* d, const void* X, const void* Wf,
+                      const void* Cin, int c_dtype, const void* bias, int bias_dtype, double alpha, double beta, int epi,
                       double a0, double a1, int in_dtype) {
     cv->N = d[0]; cv->H = d[1]; cv->W = d[2]; cv->C = d[3]; cv->K = d[4]; cv->R = d[5]; cv->S = d[6];
     cv->pad_h = d[7]; cv->pad_w = d[8]; cv->stride_h = d[9]; cv->stride_w = d[10];
@@ -282,7 +309,7 @@ static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, con
     if (beta != 0.0 && !Cin) return 2;
     cv->P = orc_conv_out_extent(cv->H, cv->pad_h, cv->dil_h, cv->R, cv->stride_h);
     cv->Q = orc_conv_out_extent(cv->W, cv->pad_w, cv->dil_w, cv->S, cv->stride_w);
-    cv->X = X; cv->Wf = Wf; cv->Cin = Cin; cv->c_dtype = c_dtype; cv->bias = bias;
+    cv->X = X; cv->Wf = Wf; cv->Cin = Cin; cv->c_dtype = c_dtype; cv->bias = bias; cv->bias_dtype = bias_dtype;
     cv->alpha = alpha; cv->beta = beta; cv->epi = epi; cv->a0 = a0; cv->a1 = a1; cv->in_dtype = in_dtype;
     return 0;
 }
@@ -292,12 +319,12 @@ static int conv_setup(conv_problem* cv, const int64_t* d, const uint16_t* X, con
  * Output pixels [pix_begin, pix_end) in flattened (n,p,q) order; ref holds
  * (pix_end-pix_begin) x K values.
  */
-int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
-                     const void* Cin, int c_dtype, const uint16_t* bias,
+int orc_conv2d_fprop(const int64_t* dims, const void* X, const void* Wf,
+                     const void* Cin, int c_dtype, const void* bias, int bias_dtype,
                      double alpha, double beta, int epi, double a0, double a1, int in_dtype,
                      int64_t pix_begin, int64_t pix_end, double* ref, double* absacc) {
     conv_problem cv;
-    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1, in_dtype);
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, bias_dtype, alpha, beta, epi, a0, a1, in_dtype);
     if (rc) return rc;
     if (pix_begin < 0 || pix_end > cv.N * cv.P * cv.Q || pix_begin > pix_end) return 1;
 #pragma omp parallel for schedule(static)
@@ -316,12 +343,12 @@ int orc_conv2d_fprop(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
 }
 
 /* The listed (flattened pixel, output channel) pairs only. */
-int orc_conv2d_points(const int64_t* dims, const uint16_t* X, const uint16_t* Wf,
-                      const void* Cin, int c_dtype, const uint16_t* bias,
+int orc_conv2d_points(const int64_t* dims, const void* X, const void* Wf,
+                      const void* Cin, int c_dtype, const void* bias, int bias_dtype,
                       double alpha, double beta, int epi, double a0, double a1, int in_dtype,
                       int64_t npts, const int64_t* ppix, const int64_t* pk, double* ref, double* absacc) {
     conv_problem cv;
-    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, alpha, beta, epi, a0, a1, in_dtype);
+    int rc = conv_setup(&cv, dims, X, Wf, Cin, c_dtype, bias, bias_dtype, alpha, beta, epi, a0, a1, in_dtype);
     if (rc) return rc;
     for (int64_t t = 0; t < npts; ++t)
         if (ppix[t] < 0 || ppix[t] >= cv.N * cv.P * cv.Q || pk[t] < 0 || pk[t] >= cv.K) return 1;

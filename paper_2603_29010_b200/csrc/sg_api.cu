@@ -213,13 +213,18 @@ struct Checked {
     int esize_out;
     int out_kind;                 // kernel template value: 0 bf16, 1 fp32, 2 fp16
     bool in_f16;
+    int in_fp8;                   // 0 no, 1 e4m3, 2 e5m2
+    int esize_in, bk;             // bytes per input element; K elements per 128-byte stage row
     CUtensorMapDataType tm_in, tm_out;
 };
 
 sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, float a0, float a1,
                          int32_t reserved, Checked* c) {
-    if (in_dtype != SG_BF16 && in_dtype != SG_F16) return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16 or SG_F16", in_dtype);
-    if (out_dtype != SG_BF16 && out_dtype != SG_F32 && out_dtype != SG_F16) return fail(SG_ERR_INVALID_ARG, "out_dtype %d is not a sg_dtype_t", out_dtype);
+    if (in_dtype != SG_BF16 && in_dtype != SG_F16 && in_dtype != SG_FP8_E4M3 && in_dtype != SG_FP8_E5M2)
+        return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16, SG_F16, SG_FP8_E4M3 or SG_FP8_E5M2", in_dtype);
+    if (out_dtype != SG_BF16 && out_dtype != SG_F32 && out_dtype != SG_F16)
+        return fail(out_dtype == SG_FP8_E4M3 || out_dtype == SG_FP8_E5M2 ? SG_ERR_UNSUPPORTED : SG_ERR_INVALID_ARG,
+                    "out_dtype %d: outputs must be SG_BF16, SG_F16 or SG_F32", out_dtype);
     if (epi < SG_EPI_NONE || epi > SG_EPI_CLIP) return fail(SG_ERR_INVALID_ARG, "epi %d is not a sg_epilogue_t", epi);
     if (!std::isfinite(alpha) || !std::isfinite(beta)) return fail(SG_ERR_INVALID_ARG, "alpha and beta must be finite");
     if ((epi == SG_EPI_LEAKY_RELU || epi == SG_EPI_ELU) && !std::isfinite(a0)) return fail(SG_ERR_INVALID_ARG, "epi_arg0 (slope) must be finite");
@@ -229,7 +234,11 @@ sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float
     c->esize_out = c->f32_out ? 4 : 2;
     c->out_kind = out_dtype == SG_F32 ? 1 : (out_dtype == SG_F16 ? 2 : 0);
     c->in_f16 = (in_dtype == SG_F16);
-    c->tm_in = c->in_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    c->in_fp8 = in_dtype == SG_FP8_E4M3 ? 1 : (in_dtype == SG_FP8_E5M2 ? 2 : 0);
+    c->esize_in = c->in_fp8 ? 1 : 2;
+    c->bk = c->in_fp8 ? 128 : 64;
+    c->tm_in = c->in_fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                         : (c->in_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     c->tm_out = out_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                     : (out_dtype == SG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     return SG_OK;
@@ -256,7 +265,9 @@ sg_status_t check_gemm_desc(const sg_gemm_desc_t* d, bool grouped, Checked* c) {
         return fail(SG_ERR_INVALID_ARG, "ldb %lld is smaller than B's contiguous extent %lld", (long long)d->ldb, (long long)b_inner);
     if (d->ldd < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldd %lld < N %lld", (long long)d->ldd, (long long)d->N);
     if (d->beta != 0.0f && d->ldc < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldc %lld < N %lld", (long long)d->ldc, (long long)d->N);
-    if ((d->lda * 2) % 16 || (d->ldb * 2) % 16) return fail(SG_ERR_ALIGNMENT, "lda and ldb must be multiples of 8 elements (16 bytes)");
+    if ((d->lda * c->esize_in) % 16 || (d->ldb * c->esize_in) % 16) return fail(SG_ERR_ALIGNMENT, "lda and ldb must be multiples of 16 bytes");
+    if (c->in_fp8 && (d->layout_a != SG_ROW_MAJOR || d->layout_b != SG_COL_MAJOR))
+        return fail(SG_ERR_UNSUPPORTED, "8-bit inputs are implemented for the K-contiguous pair (A row-major, B column-major) only");
     if ((d->ldd * c->esize_out) % 16) return fail(SG_ERR_ALIGNMENT, "ldd must be a multiple of 16 bytes");
     if (d->beta != 0.0f && (d->ldc * c->esize_out) % 16) return fail(SG_ERR_ALIGNMENT, "ldc must be a multiple of 16 bytes");
     return SG_OK;
@@ -463,7 +474,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (st != SG_OK) return st;
     if (batch > 1) {
         if (sA < 0 || sB < 0 || sC < 0 || sD < 0 || sBias < 0) return fail(SG_ERR_INVALID_ARG, "%s: negative batch stride", who);
-        if ((sA * 2) % 16 || (sB * 2) % 16 || (sD * c.esize_out) % 16 || (desc->beta != 0.0f && (sC * c.esize_out) % 16))
+        if ((sA * c.esize_in) % 16 || (sB * c.esize_in) % 16 || (sD * c.esize_out) % 16 || (desc->beta != 0.0f && (sC * c.esize_out) % 16))
             return fail(SG_ERR_ALIGNMENT, "%s: batch strides must be multiples of 16 bytes", who);
         if (sD < (desc->M - 1) * desc->ldd + desc->N) return fail(SG_ERR_INVALID_ARG, "%s: strideD smaller than one output", who);
     }
@@ -474,6 +485,8 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
     p.in_f16 = c.in_f16 ? 1 : 0;
+    p.in_fp8 = c.in_fp8;
+    p.bk_elems = c.bk;
     const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
     Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
     const int tile_m = s.pair ? 256 : 128;
@@ -488,7 +501,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.tiles_n = static_cast<int32_t>((desc->N + s.bn - 1) / s.bn);
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n * batch;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
-    p.num_kb = static_cast<int32_t>((desc->K + 63) / 64);
+    p.num_kb = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
     plan_tail(*d, s, tiles, &p, min_b_rows);
     p.bias = bias;
     p.C = desc->beta != 0.0f ? C : nullptr;
@@ -502,18 +515,18 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
         // K-contiguous operand: boxes of 64 k x tile rows.  M/N-contiguous operand (column-major A, row-major B):
         // the map is over [k][rows] and every load is a box of 64 rows x 64 k.
         if (p.a_mn_major)
-            st = make_tiled_map(&p.tmA, c.tm_in, 2, A, desc->M, desc->K, batch, desc->lda, sA, 64, 64, "A");
+            st = make_tiled_map(&p.tmA, c.tm_in, c.esize_in, A, desc->M, desc->K, batch, desc->lda, sA, 64, 64, "A");
         else
-            st = make_tiled_map(&p.tmA, c.tm_in, 2, A, desc->K, desc->M, batch, desc->lda, sA, 64, 128, "A");
+            st = make_tiled_map(&p.tmA, c.tm_in, c.esize_in, A, desc->K, desc->M, batch, desc->lda, sA, c.bk, 128, "A");
         if (st != SG_OK) return st;
         if (p.b_mn_major) {
-            st = make_tiled_map(&p.tmB, c.tm_in, 2, B, desc->N, desc->K, batch, desc->ldb, sB, 64, 64, "B");
+            st = make_tiled_map(&p.tmB, c.tm_in, c.esize_in, B, desc->N, desc->K, batch, desc->ldb, sB, 64, 64, "B");
             p.tmB2 = p.tmB;
         } else {
-            st = make_tiled_map(&p.tmB, c.tm_in, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+            st = make_tiled_map(&p.tmB, c.tm_in, c.esize_in, B, desc->K, desc->N, batch, desc->ldb, sB, c.bk,
                                 s.pair ? s.bn / 2 : s.bn, "B");
             if (st != SG_OK) return st;
-            st = make_tiled_map(&p.tmB2, c.tm_in, 2, B, desc->K, desc->N, batch, desc->ldb, sB, 64,
+            st = make_tiled_map(&p.tmB2, c.tm_in, c.esize_in, B, desc->K, desc->N, batch, desc->ldb, sB, c.bk,
                                 (s.pair ? s.bn / 2 : s.bn) / p.split, "B (narrow)");
         }
         if (st != SG_OK) return st;
@@ -715,11 +728,13 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     Params p;
     base_params(&p, *d, common->alpha, common->beta, common->epi, common->epi_arg0, common->epi_arg1);
     p.in_f16 = c.in_f16 ? 1 : 0;
+    p.in_fp8 = c.in_fp8;
+    p.bk_elems = c.bk;
     int64_t tiles = 0;
     for (int g = 0; g < groups; ++g) tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: too many tiles");
     p.K = static_cast<int32_t>(common->K);
-    p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
+    p.num_kb = static_cast<int32_t>((common->K + c.bk - 1) / c.bk);
     plan_tail(*d, s, tiles, &p, min_b_rows);
 
     std::vector<uint8_t> host(L.total, 0);
@@ -740,19 +755,19 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
         tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
         const uint32_t b_box = static_cast<uint32_t>(s.pair ? s.bn / 2 : s.bn);
         if (common->K > 0) {
-            st = make_tiled_map(&maps[4 * g], c.tm_in, 2, A_ptrs_host[g], common->K, rows[g], 1,
-                                common->lda, 0, 64, 128, "A_g");
+            st = make_tiled_map(&maps[4 * g], c.tm_in, c.esize_in, A_ptrs_host[g], common->K, rows[g], 1,
+                                common->lda, 0, c.bk, 128, "A_g");
             if (st != SG_OK) return st;
             if (common->layout_b == SG_ROW_MAJOR) {
-                st = make_tiled_map(&maps[4 * g + 1], c.tm_in, 2, B_ptrs_host[g], common->N, common->K, 1,
+                st = make_tiled_map(&maps[4 * g + 1], c.tm_in, c.esize_in, B_ptrs_host[g], common->N, common->K, 1,
                                     common->ldb, 0, 64, 64, "B_g");
                 maps[4 * g + 3] = maps[4 * g + 1];
             } else {
-                st = make_tiled_map(&maps[4 * g + 1], c.tm_in, 2, B_ptrs_host[g], common->K, common->N, 1,
-                                    common->ldb, 0, 64, b_box, "B_g");
+                st = make_tiled_map(&maps[4 * g + 1], c.tm_in, c.esize_in, B_ptrs_host[g], common->K, common->N, 1,
+                                    common->ldb, 0, c.bk, b_box, "B_g");
                 if (st != SG_OK) return st;
-                st = make_tiled_map(&maps[4 * g + 3], c.tm_in, 2, B_ptrs_host[g], common->K, common->N, 1,
-                                    common->ldb, 0, 64, b_box / p.split, "B_g (narrow)");
+                st = make_tiled_map(&maps[4 * g + 3], c.tm_in, c.esize_in, B_ptrs_host[g], common->K, common->N, 1,
+                                    common->ldb, 0, c.bk, b_box / p.split, "B_g (narrow)");
             }
             if (st != SG_OK) return st;
         }
@@ -781,7 +796,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
     p.K = static_cast<int32_t>(common->K);
     p.batch = groups;
     p.tiles_n = tiles_n;
-    p.num_kb = static_cast<int32_t>((common->K + 63) / 64);
+    p.num_kb = static_cast<int32_t>((common->K + c.bk - 1) / c.bk);
     return launch(*d, s, c.out_kind, p, stream);
 }
 
@@ -842,7 +857,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     if (Mg == 0 || desc->K == 0) return SG_OK;
     if (Mg > INT32_MAX || desc->C * desc->R * desc->S > INT32_MAX || desc->K > INT32_MAX || desc->H > 65535 || desc->W > 65535)
         return fail(SG_ERR_UNSUPPORTED, "sg_conv2d_fprop: extents too large");
-    if (desc->C % 8 || desc->K % 8) return fail(SG_ERR_ALIGNMENT, "sg_conv2d_fprop: C and K must be multiples of 8 (16-byte rule)");
+    if ((desc->C * c.esize_in) % 16 || (desc->K * c.esize_out) % 16)
+        return fail(SG_ERR_ALIGNMENT, "sg_conv2d_fprop: C (input type) and K (output type) must span multiples of 16 bytes");
     if (desc->pad_h > 127 || desc->pad_w > 127 || (desc->R - 1) * desc->dil_h > 255 || (desc->S - 1) * desc->dil_w > 255 ||
         desc->pad_h - (desc->R - 1) * desc->dil_h < -128 || desc->pad_w - (desc->S - 1) * desc->dil_w < -128 ||
         desc->stride_h > 8 || desc->stride_w > 8)
@@ -858,6 +874,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     Params p;
     base_params(&p, *d, desc->alpha, desc->beta, desc->epi, desc->epi_arg0, desc->epi_arg1);
     p.in_f16 = c.in_f16 ? 1 : 0;
+    p.in_fp8 = c.in_fp8;
+    p.bk_elems = c.bk;
     Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_CONV;
@@ -867,7 +885,7 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     p.batch = 1;
     p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
     p.tiles_n = static_cast<int32_t>((desc->K + s.bn - 1) / s.bn);
-    p.cblocks = static_cast<int32_t>((desc->C + 63) / 64);
+    p.cblocks = static_cast<int32_t>((desc->C + c.bk - 1) / c.bk);
     p.num_kb = static_cast<int32_t>(desc->R * desc->S) * p.cblocks;
     plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p);
     p.bias = bias;
@@ -887,14 +905,15 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     {
         cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->W),
                               static_cast<cuuint64_t>(desc->H), static_cast<cuuint64_t>(desc->N)};
-        cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->C) * 2, static_cast<cuuint64_t>(desc->W * desc->C) * 2,
-                                 static_cast<cuuint64_t>(desc->H * desc->W * desc->C) * 2};
+        const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
+        cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->C) * es, static_cast<cuuint64_t>(desc->W * desc->C) * es,
+                                 static_cast<cuuint64_t>(desc->H * desc->W * desc->C) * es};
         int lower[2] = {-desc->pad_w, -desc->pad_h};
         int upper[2] = {static_cast<int>(desc->pad_w - (desc->S - 1) * desc->dil_w),
                         static_cast<int>(desc->pad_h - (desc->R - 1) * desc->dil_h)};
         cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(desc->stride_w), static_cast<cuuint32_t>(desc->stride_h), 1};
         CUresult r = g_encode_im2col(&p.tmA, c.tm_in, 4, const_cast<void*>(X), dims, strides, lower, upper,
-                                     64, 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     static_cast<cuuint32_t>(c.bk), 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(X) failed with CUresult %d", static_cast<int>(r));
     }
@@ -902,8 +921,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     {
         cuuint64_t dims[3] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->R * desc->S),
                               static_cast<cuuint64_t>(desc->K)};
-        cuuint64_t strides[2] = {static_cast<cuuint64_t>(desc->C) * 2, static_cast<cuuint64_t>(Kg) * 2};
-        cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(s.pair ? s.bn / 2 : s.bn)};
+        cuuint64_t strides[2] = {static_cast<cuuint64_t>(desc->C) * c.esize_in, static_cast<cuuint64_t>(Kg) * c.esize_in};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(c.bk), 1, static_cast<cuuint32_t>(s.pair ? s.bn / 2 : s.bn)};
         cuuint32_t estr[3] = {1, 1, 1};
         CUresult r = g_encode_tiled(&p.tmB, c.tm_in, 3, const_cast<void*>(Wf), dims, strides, box, estr,
                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,

@@ -54,7 +54,9 @@ struct alignas(64) Params {
     float alpha, beta;
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
     int32_t epi, mode;
-    int32_t in_f16;                     // 1: A, B and bias are fp16 (else bf16)
+    int32_t in_f16;                     // 1: the bias (and 16-bit A, B) are fp16, else bf16
+    int32_t in_fp8;                     // 0: 16-bit A and B; 1: e4m3; 2: e5m2 (the bias then is bf16 or fp16 as in_f16 says)
+    int32_t bk_elems;                   // elements of K per 128-byte stage row: 64 (16-bit) or 128 (8-bit)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
     uint32_t* status;                   // device status words (8 x u32)
@@ -195,6 +197,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Pa
     return wait_slow(bar, parity, p, role, tile, which);
 }
 
+
 __device__ __forceinline__ float tanh_approx(float x) {
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -210,52 +213,73 @@ __device__ __forceinline__ float tanh_approx(float x) {
 #ifndef SG_FAST_ACT
 #define SG_FAST_ACT 1
 #endif
-template <bool kFast>
-__device__ __forceinline__ float apply_act(float v, int epi, float a0, float a1) {
+template <bool kFast, int kEpi>
+__device__ __forceinline__ float act_one(float v, float a0, float a1) {
     constexpr bool fast = kFast && SG_FAST_ACT;
-    switch (epi) {
-        case EPI_RELU:
-            return fmaxf(v, 0.0f);
-        case EPI_GELU: {
-            const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
-            if constexpr (fast) {
-                const float h = 0.5f * v;
-                return fmaf(h, tanh_approx(u), h);
-            } else {
-                return __fdividef(v, 1.0f + __expf(-2.0f * u));
-            }
+    if constexpr (kEpi == EPI_RELU) {
+        return fmaxf(v, 0.0f);
+    } else if constexpr (kEpi == EPI_GELU) {
+        const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
+        if constexpr (fast) {
+            const float h = 0.5f * v;
+            return fmaf(h, tanh_approx(u), h);
+        } else {
+            return __fdividef(v, 1.0f + __expf(-2.0f * u));
         }
-        case EPI_SILU: {
-            if constexpr (fast) {
-                const float h = 0.5f * v;
-                return fmaf(h, tanh_approx(h), h);
-            } else {
-                return __fdividef(v, 1.0f + __expf(-v));
-            }
+    } else if constexpr (kEpi == EPI_SILU) {
+        if constexpr (fast) {
+            const float h = 0.5f * v;
+            return fmaf(h, tanh_approx(h), h);
+        } else {
+            return __fdividef(v, 1.0f + __expf(-v));
         }
-        case EPI_SIGMOID:
-            if constexpr (fast) return fmaf(0.5f, tanh_approx(0.5f * v), 0.5f);
-            else return __fdividef(1.0f, 1.0f + __expf(-v));
-        case EPI_TANH:
-            if constexpr (fast) return tanh_approx(v);
-            else return tanhf(v);
-        case EPI_MISH: {
-            // x tanh(softplus(x)); softplus(x) = x beyond 20 (e^-20 is below fp32 resolution next to x)
-            if constexpr (fast) return v * tanh_approx(v > 20.0f ? v : __logf(1.0f + __expf(v)));
-            else return v * tanhf(v > 20.0f ? v : log1pf(expf(v)));
-        }
-        case EPI_HARDSWISH:
-            return v * fminf(fmaxf(v + 3.0f, 0.0f), 6.0f) * (1.0f / 6.0f);
-        case EPI_LEAKY_RELU:
-            return v > 0.0f ? v : a0 * v;
-        case EPI_ELU:
-            if constexpr (fast) return v > 0.0f ? v : a0 * (__expf(v) - 1.0f);
-            else return v > 0.0f ? v : a0 * expm1f(v);
-        case EPI_CLIP:
-            return fminf(fmaxf(v, a0), a1);
-        default:
-            return v;
+    } else if constexpr (kEpi == EPI_SIGMOID) {
+        if constexpr (fast) return fmaf(0.5f, tanh_approx(0.5f * v), 0.5f);
+        else return __fdividef(1.0f, 1.0f + __expf(-v));
+    } else if constexpr (kEpi == EPI_TANH) {
+        if constexpr (fast) return tanh_approx(v);
+        else return tanhf(v);
+    } else if constexpr (kEpi == EPI_MISH) {
+        // x tanh(softplus(x)); softplus(x) = x beyond 20 (e^-20 is below fp32 resolution next to x)
+        if constexpr (fast) return v * tanh_approx(v > 20.0f ? v : __logf(1.0f + __expf(v)));
+        else return v * tanhf(v > 20.0f ? v : log1pf(expf(v)));
+    } else if constexpr (kEpi == EPI_HARDSWISH) {
+        return v * fminf(fmaxf(v + 3.0f, 0.0f), 6.0f) * (1.0f / 6.0f);
+    } else if constexpr (kEpi == EPI_LEAKY_RELU) {
+        return v > 0.0f ? v : a0 * v;
+    } else if constexpr (kEpi == EPI_ELU) {
+        if constexpr (fast) return v > 0.0f ? v : a0 * (__expf(v) - 1.0f);
+        else return v > 0.0f ? v : a0 * expm1f(v);
+    } else if constexpr (kEpi == EPI_CLIP) {
+        return fminf(fmaxf(v, a0), a1);
+    } else {
+        return v;
     }
+}
+
+// Applies the activation to a whole chunk of values: the (runtime) choice of the activation is taken once per
+// chunk, outside the element loop.
+template <bool kFast, int kN>
+__device__ __forceinline__ void apply_act_chunk(float (&v)[kN], int epi, float a0, float a1) {
+#define SG_ACT_CASE(E)                                                        \
+    case E:                                                                   \
+        _Pragma("unroll") for (int i = 0; i < kN; ++i) v[i] = act_one<kFast, E>(v[i], a0, a1); \
+        break;
+    switch (epi) {
+        SG_ACT_CASE(EPI_RELU)
+        SG_ACT_CASE(EPI_GELU)
+        SG_ACT_CASE(EPI_SILU)
+        SG_ACT_CASE(EPI_SIGMOID)
+        SG_ACT_CASE(EPI_TANH)
+        SG_ACT_CASE(EPI_MISH)
+        SG_ACT_CASE(EPI_HARDSWISH)
+        SG_ACT_CASE(EPI_LEAKY_RELU)
+        SG_ACT_CASE(EPI_ELU)
+        SG_ACT_CASE(EPI_CLIP)
+        default:
+            break;
+    }
+#undef SG_ACT_CASE
 }
 
 // Bounded wait until a global arrival counter (written by another CTA of this launch with a release pattern)
@@ -418,6 +442,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 const int nb0 = ti.n0 + static_cast<int>(cta_rank) * b_rows;
                 const uint32_t stage_tx = static_cast<uint32_t>(Cfg::A_BYTES + b_rows * Cfg::BK * 2) * kCtas;
                 const bool narrow = ti.width != BN;
+                const int bk_elems = p.bk_elems;
                 const CUtensorMap* mapA = &p.tmA;
                 const CUtensorMap* mapB = narrow ? &p.tmB2 : &p.tmB;
                 int bz = ti.b;
@@ -451,7 +476,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
                     if (p.mode == MODE_CONV) {
                         const int tap = kb / p.cblocks;
-                        const int c0 = (kb - tap * p.cblocks) * Cfg::BK;
+                        const int c0 = (kb - tap * p.cblocks) * bk_elems;
                         const int r = tap / p.S;
                         const int s = tap - r * p.S;
                         tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(s * p.dil_w),
@@ -462,15 +487,15 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                             // column-major A: boxes of 64 rows of the tile (contiguous) x 64 k, one per 64 tile rows
 #pragma unroll
                             for (int j = 0; j < Cfg::BM / 64; ++j)
-                                tma_load_3d<kPair>(a_dst + j * 8192, mapA, fb, m0 + j * 64, kb * Cfg::BK, bz);
+                                tma_load_3d<kPair>(a_dst + j * 8192, mapA, fb, m0 + j * 64, kb * Cfg::BK, bz);   // 16-bit only
                         } else {
-                            tma_load_3d<kPair>(a_dst, mapA, fb, kb * Cfg::BK, m0, bz);
+                            tma_load_3d<kPair>(a_dst, mapA, fb, kb * bk_elems, m0, bz);
                         }
                         if (p.b_mn_major) {
                             for (int j = 0; j < b_rows / 64; ++j)
                                 tma_load_3d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, kb * Cfg::BK, bz);
                         } else {
-                            tma_load_3d<kPair>(b_dst, mapB, fb, kb * Cfg::BK, nb0, bz);
+                            tma_load_3d<kPair>(b_dst, mapB, fb, kb * bk_elems, nb0, bz);
                         }
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -487,10 +512,15 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             uint32_t phase = 0;
             int iter = 0;
             int g_hint = 0;
+            const uint64_t a_desc0 = p.a_mn_major ? smem_desc_mn_major_sw128(smem_base) : smem_desc_k_major_sw128(smem_base);
+            const uint64_t b_desc0 = p.b_mn_major ? smem_desc_mn_major_sw128(smem_base + Cfg::A_BYTES)
+                                                  : smem_desc_k_major_sw128(smem_base + Cfg::A_BYTES);
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
                 const Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
-                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0, p.in_f16 != 0);
+                const bool fp8 = p.in_fp8 != 0;
+                const uint32_t in_fmt = fp8 ? static_cast<uint32_t>(p.in_fp8 - 1) : (p.in_f16 ? 0u : 1u);
+                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0, in_fmt);
                 const uint32_t a_step = p.a_mn_major ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
                 const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
                 const int acc = iter & 1;
@@ -503,15 +533,21 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     if (!wait_bar(full_bar(stage), phase, p, ROLE_MMA, t, stage)) { ok = false; break; }
                     if (t == first_tile && kb == ti.kb0) SG_STAMP(4);
                     tc_fence_after_sync();
-                    const uint32_t a_src = smem_base + stage * Cfg::STAGE_BYTES;
-                    const uint64_t a_desc = p.a_mn_major ? smem_desc_mn_major_sw128(a_src) : smem_desc_k_major_sw128(a_src);
-                    const uint64_t b_desc = p.b_mn_major ? smem_desc_mn_major_sw128(a_src + Cfg::A_BYTES)
-                                                         : smem_desc_k_major_sw128(a_src + Cfg::A_BYTES);
+                    // descriptors of this stage: those of stage 0 plus the stage offset in the 16-byte address field
+                    const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage * (Cfg::STAGE_BYTES >> 4));
+                    const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(stage * (Cfg::STAGE_BYTES >> 4));
+                    // One instruction-K step is 32 bytes along a K-major row (16 two-byte or 32 one-byte elements), or two
+                    // 1 KB k-groups of an MN-major tile; a 128-byte stage row holds four of them for either width.
+                    if (fp8) {
 #pragma unroll
-                    for (int kk = 0; kk < Cfg::BK / 16; ++kk) {
-                        // one K=16 step: 32 bytes along a K-major row, or two 1 KB k-groups of an MN-major tile
-                        umma_bf16<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
-                                         (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_fp8<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
+                                            (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_bf16<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
+                                             (kb != ti.kb0 || kk != 0) ? 1u : 0u);
                     }
                     umma_commit<kPair>(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -732,10 +768,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         v[i] += b0; v[i + 1] += b1; v[i + 2] += b2f; v[i + 3] += b3;
                     }
                 }
-                if (epi >= EPI_RELU) {
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) v[i] = apply_act<kOut == 0>(v[i], epi, p.epi_arg0, p.epi_arg1);
-                }
+                if (epi >= EPI_RELU) apply_act_chunk<kOut == 0, CH>(v, epi, p.epi_arg0, p.epi_arg1);
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
                 // the last, partial chunk is therefore written with plain stores so nothing beyond column N changes.

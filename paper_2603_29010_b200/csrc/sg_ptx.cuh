@@ -214,6 +214,30 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
             : "memory");
     }
 }
+// The same for 8-bit floating-point operands (e4m3 / e5m2): K = 32 per instruction.
+template <bool kPair>
+__device__ __forceinline__ void umma_fp8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    if constexpr (kPair) {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
 // Arrive on `bar` once every MMA issued so far by this thread has completed.  For a CTA pair the
 // arrival is delivered to the same barrier offset in both CTAs (mask 0b11).
 template <bool kPair>
@@ -276,9 +300,9 @@ __device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t smem_addr)
 
 // Instruction descriptor for kind::f16: fp32 accumulator, bf16 or fp16 A and B, no negation, dense.  bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format,
 // 15 / 16 A / B major (0 = K), 17-22 N >> 3, 24-28 M >> 4.
-// in_f16 selects fp16 (format code 0) instead of bf16 (format code 1) for both A and B.
-__host__ __device__ constexpr uint32_t umma_idesc_f32acc(int m, int n, bool a_mn_major, bool b_mn_major, bool in_f16) {
-    const uint32_t fmt = in_f16 ? 0u : 1u;
+// in_fmt: operand format code of both A and B.  kind::f16: 0 = fp16, 1 = bf16.  kind::f8f6f4: 0 = e4m3, 1 = e5m2.
+__host__ __device__ constexpr uint32_t umma_idesc_f32acc(int m, int n, bool a_mn_major, bool b_mn_major, uint32_t in_fmt) {
+    const uint32_t fmt = in_fmt;
     return (1u << 4) | (fmt << 7) | (fmt << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }

@@ -558,3 +558,49 @@ def test_fp16_batched_grouped_and_conv():
     Wf = (inputs.small_integers([72, 3, 3, 64], 757, 7, -1, 1) * (inputs.small_integers([72, 3, 3, 64], 758, 7, 0, 3) == 0).to(torch.bfloat16)).half()
     ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
     parity.assert_bit_exact(sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1), out_dtype=torch.float16), ref, "fp16 conv")
+
+
+# ---------------------------------------------------------------------------------------- fp8 inputs
+
+@pytest.mark.parametrize("dtype", [torch.float8_e4m3fn, torch.float8_e5m2])
+@pytest.mark.parametrize("tile_n,pair", [(64, 0), (128, 0), (256, 0), (128, 1), (256, 1)])
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (300, 200, 272), (1000, 520, 1040), (129, 72, 16)])
+def test_fp8_inputs_integer_problem_bit_exact(M, N, K, tile_n, pair, dtype):
+    sg.set_tuning(tile_n, pair)
+    A = inputs.small_integers([M, K], 818, 1, -1, 1).float().to(dtype)
+    B = inputs.small_integers([N, K], 818, 2, -1, 1).float().to(dtype)
+    ref, _ = orc.gemm(A, B)
+    assert float(ref.abs().max()) <= 256
+    D, whole = guarded((M, N), torch.bfloat16)
+    sg.gemm(A.to(DEV), B.to(DEV), out=D)
+    parity.assert_bit_exact(D, ref, f"fp8 {dtype} {M}x{N}x{K}")
+    assert guards_intact(whole, cols=N)
+
+
+def test_fp8_real_values_epilogue_batched_grouped_and_conv():
+    dt = torch.float8_e4m3fn
+    M, N, K = 200, 264, 528
+    A = (inputs.normal([M, K], 828, 1).float()).to(dt)
+    B = (inputs.normal([N, K], 828, 2).float()).to(dt)
+    bias = inputs.normal([N], 828, 4)
+    for out_dtype in (torch.bfloat16, torch.float32):
+        ref, absacc = orc.gemm(A, B, bias=bias, alpha=K ** -0.5, epi="gelu")
+        D = sg.gemm(A.to(DEV), B.to(DEV), bias=bias.to(DEV), alpha=K ** -0.5, epi="gelu", out_dtype=out_dtype)
+        parity.assert_matches(D, ref, absacc, f"fp8 gelu {out_dtype}")
+    Ab = inputs.small_integers([3, 72, 144], 838, 1, -1, 1).float().to(dt)
+    Bb = inputs.small_integers([3, 64, 144], 838, 2, -1, 1).float().to(dt)
+    ref, _ = orc.batched_gemm(Ab, Bb)
+    parity.assert_bit_exact(sg.batched_gemm(Ab.to(DEV), Bb.to(DEV)), ref, "fp8 batched")
+    As = [inputs.small_integers([m, 144], 848 + g, 1, -1, 1).float().to(dt) for g, m in enumerate([130, 40])]
+    Bs = [inputs.small_integers([136, 144], 848 + g, 2, -1, 1).float().to(dt) for g in range(2)]
+    refs, _ = orc.grouped_gemm(As, Bs)
+    outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs])
+    for g in range(2):
+        parity.assert_bit_exact(outs[g], refs[g], f"fp8 grouped {g}")
+    X = inputs.small_integers([2, 9, 11, 144], 858, 6, -1, 1).float().to(torch.float8_e5m2)
+    Wf = (inputs.small_integers([72, 3, 3, 144], 858, 7, -1, 1) * (inputs.small_integers([72, 3, 3, 144], 859, 7, 0, 3) == 0).to(torch.bfloat16)).float().to(torch.float8_e5m2)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    assert float(ref.abs().max()) <= 256
+    parity.assert_bit_exact(sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1)), ref, "fp8 conv")
+    with pytest.raises(sg.SolgemmError):                       # only the K-contiguous layouts with 8-bit inputs
+        sg.gemm(A.to(DEV), torch.zeros(K, N, device=DEV).to(dt), layout_b="row")

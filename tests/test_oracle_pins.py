@@ -439,3 +439,35 @@ def test_fp16_gemm_and_conv_match_torch_fp64():
     assert torch.allclose(ref, want, rtol=0, atol=1e-12)
     with pytest.raises(ValueError):
         orc.gemm(A, Bt.to(torch.bfloat16))
+
+
+# ---------------------------------------------------------------- 8-bit floating-point inputs
+
+@pytest.mark.parametrize("dtype", [torch.float8_e4m3fn, torch.float8_e5m2])
+def test_fp8_inputs_are_widened_exactly(dtype):
+    bits = torch.arange(0, 256, dtype=torch.int32).to(torch.uint8).view(dtype)
+    wide = bits.float().double()                                    # torch's widening as the library pin
+    finite = torch.isfinite(wide)
+    col = bits[finite].view(-1, 1)
+    ref, _ = orc.gemm(col, torch.ones(1, 1).to(dtype))
+    assert torch.equal(ref.view(-1), wide[finite])
+    # hand values: largest finite, smallest subnormal, 1.5
+    one = torch.ones(1, 1).to(dtype)
+    big, tiny = (448.0, 2.0 ** -9) if dtype == torch.float8_e4m3fn else (57344.0, 2.0 ** -16)
+    for v in (big, tiny, 1.5, -0.75):
+        assert float(orc.gemm(torch.tensor([[v]]).to(dtype), one)[0]) == v
+
+
+def test_fp8_gemm_with_bf16_bias_matches_torch_fp64():
+    A = (inputs.uniform([19, 48], 41, 1).float() * 3).to(torch.float8_e4m3fn)
+    Bt = (inputs.uniform([11, 48], 41, 2).float() * 2).to(torch.float8_e4m3fn)
+    bias = inputs.normal([11], 41, 4)                               # bf16 bias with 8-bit inputs
+    ref, _ = orc.gemm(A, Bt, bias=bias, alpha=0.25, epi="bias")
+    want = 0.25 * (A.float().double() @ Bt.float().double().t()) + bias.double()
+    assert torch.allclose(ref, want, rtol=0, atol=1e-12)
+    X = inputs.uniform([1, 5, 6, 16], 42, 6).to(torch.float8_e5m2)
+    Wf = inputs.uniform([4, 3, 3, 16], 42, 7).to(torch.float8_e5m2)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    want = torch.nn.functional.conv2d(X.float().double().permute(0, 3, 1, 2), Wf.float().double().permute(0, 3, 1, 2),
+                                      padding=1).permute(0, 2, 3, 1)
+    assert torch.allclose(ref, want, rtol=0, atol=1e-12)
