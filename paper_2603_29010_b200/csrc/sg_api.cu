@@ -38,7 +38,7 @@ sg_status_t fail(sg_status_t st, const char* fmt, ...) {
     } while (0)
 
 // ------------------------------------------------------------------------------------------ per-device state
-__device__ uint32_t g_status_words[8 + 32];   // 8 status words, then scratch for experimental time stamps
+__device__ uint32_t g_status_words[8 + 64];   // 8 status words, then scratch for experimental time stamps
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -415,7 +415,27 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
     }
 }
 
-sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Params& p, cudaStream_t stream) {
+// Magic numbers of sg::fast_div for a divisor 1 <= d < 2^31 (exact for dividends below 2^31: with
+// 2^sh = q d + r and mul = q + 1, n mul / 2^sh exceeds n / d by less than 2^-ceil(log2 d) <= 1 / d).
+FastDiv make_fastdiv(int64_t d) {
+    if (d < 1) d = 1;
+    int l = 0;
+    while ((int64_t{1} << l) < d) ++l;
+    FastDiv f;
+    f.sh = static_cast<uint32_t>(31 + l);
+    f.mul = static_cast<uint32_t>((uint64_t{1} << f.sh) / static_cast<uint64_t>(d) + 1);
+    return f;
+}
+
+sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Params& p_in, cudaStream_t stream) {
+    Params p = p_in;
+    p.split_log2 = p.split >= 4 ? 2 : (p.split >= 2 ? 1 : 0);
+    if (p.mode != MODE_GROUPED && p.tiles_m > 0 && p.band_m > p.tiles_m) p.band_m = p.tiles_m;   // same walk, one divisor
+    p.div_per = make_fastdiv(static_cast<int64_t>(p.tiles_m) * p.tiles_n);
+    p.div_band_tiles = make_fastdiv(static_cast<int64_t>(p.band_m) * p.tiles_n);
+    p.div_band_m = make_fastdiv(p.band_m);
+    p.div_pq = make_fastdiv(static_cast<int64_t>(p.P) * p.Q);
+    p.div_q = make_fastdiv(p.Q);
     KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;
@@ -607,12 +627,12 @@ const char* sg_last_error(void) { return t_err; }
 int64_t sg_launch_count(void) { return g_launches.load(); }
 
 #ifdef SG_DEBUG_STAMPS
-sg_status_t sg_debug_stamps(uint64_t* out16) {
+sg_status_t sg_debug_stamps(uint64_t* out32) {
     DeviceState* d = nullptr;
     sg_status_t st = device_state(&d);
     if (st != SG_OK) return st;
     SG_CUDA(cudaDeviceSynchronize());
-    SG_CUDA(cudaMemcpy(out16, d->status_dev + 8, 16 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    SG_CUDA(cudaMemcpy(out32, d->status_dev + 8, 32 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
     return SG_OK;
 }
 #endif

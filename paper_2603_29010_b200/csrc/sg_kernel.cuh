@@ -28,6 +28,16 @@ enum : int32_t { EPI_NONE = 0, EPI_BIAS = 1, EPI_RELU = 2, EPI_GELU = 3, EPI_SIL
 // status word 0: 0 = fine, else (role << 24 | detail); words 1..3 hold tile / barrier / block of the first failure
 enum : uint32_t { ROLE_PRODUCER = 1, ROLE_MMA = 2, ROLE_EPILOGUE = 3, ROLE_SETUP = 4 };
 
+// Division by a divisor fixed per launch: q = (n * mul) >> sh is floor(n / d) for every 0 <= n < 2^31 when
+// sh = 31 + ceil(log2 d) and mul = floor(2^sh / d) + 1 (the host fills these in).  A 32-bit integer division
+// is a chain of some thirty dependent instructions; the tile decode runs four of them before a CTA's first load.
+struct FastDiv {
+    uint32_t mul, sh;
+};
+__device__ __forceinline__ int fast_div(int n, FastDiv d) {
+    return static_cast<int>((static_cast<uint64_t>(static_cast<uint32_t>(n)) * d.mul) >> d.sh);
+}
+
 struct alignas(64) Params {
     CUtensorMap tmA, tmB, tmD;          // dense / batched / conv operands (3-D; conv A is a 4-D im2col map)
     CUtensorMap tmB2;                   // B with the narrower box of split tail tiles
@@ -45,7 +55,12 @@ struct alignas(64) Params {
     int32_t M, N, K, batch;             // batch = number of problems (dense) or groups (grouped)
     int32_t tiles_m, tiles_n, num_tiles, num_kb;
     int32_t split_begin, split;         // tiles at list positions >= split_begin are 1/split-wide column slices
+    int32_t split_log2;                 // log2(split)
     int32_t band_m;                     // raster: tiles are walked in bands of this many tile rows, column by column
+    FastDiv div_per;                    // dense / conv: by tiles_m * tiles_n (tiles of one problem)
+    FastDiv div_band_tiles;             // by band_m * tiles_n
+    FastDiv div_band_m;                 // by band_m (rows of every band but a shorter last one)
+    FastDiv div_pq, div_q;              // conv: by P * Q and by Q
     int32_t ksplit;                     // > 1: tail tiles are cut into this many K ranges instead (split is then 1)
     int32_t sk_arrivals;                // warp arrivals that complete one helper's partial tile (epilogue warps x CTAs)
     float* sk_partials;                 // K-split scratch: [tail tile][helper][CTA of the tile][128 rows][BN] fp32
@@ -113,10 +128,10 @@ struct Tile {
 // at the same time then share few A and B panels, and a band's A rows stay in L2 while its columns stream by.
 __device__ __forceinline__ void raster(const Params& p, int r, int tiles_m, int& tm, int& tn) {
     const int band_tiles = p.band_m * p.tiles_n;
-    const int band = r / band_tiles;
+    const int band = fast_div(r, p.div_band_tiles);
     const int in_band = r - band * band_tiles;
     const int band_rows = min(p.band_m, tiles_m - band * p.band_m);
-    tn = in_band / band_rows;
+    tn = band_rows == p.band_m ? fast_div(in_band, p.div_band_m) : in_band / band_rows;
     tm = band * p.band_m + (in_band - tn * band_rows);
 }
 
@@ -144,10 +159,10 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
             ti.kb0 = ti.part * base + min(ti.part, extra);
             ti.kb1 = ti.kb0 + base + (ti.part < extra ? 1 : 0);
         } else {
-            const int parent = u / p.split;
-            sub = u - parent * p.split;
+            const int parent = u >> p.split_log2;      // split is 1, 2 or 4
+            sub = u - (parent << p.split_log2);
             t = p.split_begin + parent;
-            ti.width = BN / p.split;
+            ti.width = BN >> p.split_log2;
         }
     }
     int tm, tn;
@@ -161,7 +176,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         raster(p, t - p.g_tile_start[g], (rows + TILE_M - 1) / TILE_M, tm, tn);
     } else {
         const int per = p.tiles_m * p.tiles_n;
-        ti.b = t / per;
+        ti.b = fast_div(t, p.div_per);
         ti.rows = p.M;
         raster(p, t - ti.b * per, p.tiles_m, tm, tn);
     }
@@ -219,7 +234,8 @@ __device__ __forceinline__ float act_one(float v, float a0, float a1) {
     if constexpr (kEpi == EPI_RELU) {
         return fmaxf(v, 0.0f);
     } else if constexpr (kEpi == EPI_GELU) {
-        const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
+        // u = sqrt(2/pi) (v + 0.044715 v^3) = v (c1 + c2 v^2)
+        const float u = v * fmaf(v * v, 0.7978845608028654f * 0.044715f, 0.7978845608028654f);
         if constexpr (fast) {
             const float h = 0.5f * v;
             return fmaf(h, tanh_approx(u), h);
@@ -422,6 +438,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     // on global memory is read and written: wait for the previous kernel, then let the next one start setting up.
     grid_dependency_wait();
     grid_launch_dependents();
+    if (threadIdx.x == 0) SG_STAMP(16);
 
     const int num_kb = p.num_kb;
     const int first_tile = blockIdx.x / kCtas;
@@ -437,6 +454,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
                 Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
+                if (t == first_tile) SG_STAMP(17);
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
                 const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
                 const int nb0 = ti.n0 + static_cast<int>(cta_rank) * b_rows;
@@ -460,28 +478,39 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 int cw = 0, ch = 0, cn = 0;
                 if (p.mode == MODE_CONV) {
                     const int pq = p.P * p.Q;
-                    cn = m0 / pq;
+                    cn = fast_div(m0, p.div_pq);
                     const int rem = m0 - cn * pq;
-                    const int op = rem / p.Q;
+                    const int op = fast_div(rem, p.div_q);
                     const int oq = rem - op * p.Q;
                     cw = oq * p.stride_w - p.pad_w;
                     ch = op * p.stride_h - p.pad_h;
                 }
+                // conv: filter tap (r, s) and channel block of the current k-block, advanced incrementally
+                int c_tap = 0, c_cb = 0, c_r = 0, c_s = 0;
+                if (p.mode == MODE_CONV) {
+                    c_tap = ti.kb0 / p.cblocks;
+                    c_cb = ti.kb0 - c_tap * p.cblocks;
+                    c_r = c_tap / p.S;
+                    c_s = c_tap - c_r * p.S;
+                }
                 for (int kb = ti.kb0; kb < ti.kb1; ++kb) {
                     if (!wait_bar(empty_bar(stage), phase ^ 1u, p, ROLE_PRODUCER, t, stage)) { ok = false; break; }
+                    if (t == first_tile && kb == ti.kb0) SG_STAMP(18);
                     const uint32_t a_dst = smem_base + stage * Cfg::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + Cfg::A_BYTES;
                     uint32_t fb = full_bar(stage);
                     if constexpr (kPair) fb = map_to_cta(fb, 0);
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
                     if (p.mode == MODE_CONV) {
-                        const int tap = kb / p.cblocks;
-                        const int c0 = (kb - tap * p.cblocks) * bk_elems;
-                        const int r = tap / p.S;
-                        const int s = tap - r * p.S;
-                        tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(s * p.dil_w),
-                                                  static_cast<uint16_t>(r * p.dil_h));
-                        tma_load_3d<kPair>(b_dst, mapB, fb, c0, tap, nb0);
+                        const int c0 = c_cb * bk_elems;
+                        tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(c_s * p.dil_w),
+                                                  static_cast<uint16_t>(c_r * p.dil_h));
+                        tma_load_3d<kPair>(b_dst, mapB, fb, c0, c_tap, nb0);
+                        if (++c_cb == p.cblocks) {
+                            c_cb = 0;
+                            ++c_tap;
+                            if (++c_s == p.S) { c_s = 0; ++c_r; }
+                        }
                     } else {
                         if (p.a_mn_major) {
                             // column-major A: boxes of 64 rows of the tile (contiguous) x 64 k, one per 64 tile rows
@@ -632,6 +661,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (!done) { ok = false; break; }
                 tc_fence_after_sync();
                 if (warp == 2 && lane == 0 && t == first_tile) SG_STAMP(7);
+                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(19);
             }
             const int ncols = min(ti.width, p.N - n0);
             const int nchunks = (ncols + CH - 1) / CH;
@@ -659,6 +689,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         uint32_t r1[32];
                         tmem_ld_32x32(t_row + c * CH + 32, r1);
                         tmem_ld_wait();
+                        if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(20 + 4 * (c / kStep > 0 ? 1 : 0));
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             v[i] = __uint_as_float(r0[i]);
@@ -723,8 +754,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     }
                 }
 
+                if (alpha != 1.0f) {
 #pragma unroll
-                for (int i = 0; i < CH; ++i) v[i] *= alpha;
+                    for (int i = 0; i < CH; ++i) v[i] *= alpha;
+                }
                 if (has_c && row < ti.rows) {
                     const int col0 = n0 + c * CH;
                     if constexpr (kOutF32) {
@@ -769,6 +802,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     }
                 }
                 if (epi >= EPI_RELU) apply_act_chunk<kOut == 0, CH>(v, epi, p.epi_arg0, p.epi_arg1);
+                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(21 + 4 * (c / kStep > 0 ? 1 : 0));
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
                 // the last, partial chunk is therefore written with plain stores so nothing beyond column N changes.
@@ -797,6 +831,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 ++chunk_ctr;
                 if (lane == 0) tma_store_wait_read<Cfg::STAGING_BUFS - 1>();   // the store that last read this block is done
                 __syncwarp();
+                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(22 + 4 * (c / kStep > 0 ? 1 : 0));
                 const uint32_t stg = smem_base + Cfg::OFF_STAGING + (ew * Cfg::STAGING_BUFS + sb) * 4096u;
                 const uint32_t row_addr = stg + lane * 128u;
 #pragma unroll
@@ -822,6 +857,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     tma_store_commit();
                 }
 #endif
+                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(23 + 4 * (c / kStep > 0 ? 1 : 0));
             }
             if (!ok) break;
             if (ti.nparts > 1) {
@@ -845,7 +881,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             }
         }
         if (warp == 2 && lane == 0) SG_STAMP(8);
-        if (lane == 0) tma_store_wait_all();
+        // the staging blocks must have been read before the CTA's shared memory goes away; the writes themselves
+        // complete with the grid
+        if (lane == 0) tma_store_wait_read<0>();
         if (warp == 2 && lane == 0) SG_STAMP(9);
         __syncwarp();
     }
