@@ -324,8 +324,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     per_launch = dt / args.steps
     achieved = flops / per_launch / 1e12
     # Denominator: the burst cuBLAS figure for short timed regions; the sustained one when the region ran long
-    # enough (>= 0.1 s of back-to-back launches) to be held at the board's power cap, as the clock record shows.
-    sustained = dt >= 0.1 and "sw_power_cap" in clocks["reasons"]
+    # enough (>= 0.1 s of back-to-back launches) to be held at the board's power cap.  Evidence of the cap: the
+    # driver's sw_power_cap reason, or (NVML on this pool reports the requested clock and no reason) the SM clock
+    # counted inside the kernel sitting below three quarters of the maximum.
+    in_kernel = clocks.get("sm_mhz_in_kernel") or 0.0
+    capped = "sw_power_cap" in clocks["reasons"] or (0.0 < in_kernel < 0.75 * float(clocks.get("sm_max_mhz") or 1965))
+    sustained = dt >= 0.1 and capped
     peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     sol_spec = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=SPEC_PEAK_FLOPS, peak_bytes_per_s=SPEC_PEAK_BW)
     sol_meas = sg.sol_bound("gemm", M=M, N=N, K=K, has_bias=1, peak_flops=peaks["bf16_tflops"] * 1e12,
