@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.orc_act.argtypes = [ci, dbl]
         L.orc_act2.restype = dbl
         L.orc_act2.argtypes = [ci, dbl, dbl, dbl]
+        L.orc_act_array.restype = None
+        L.orc_act_array.argtypes = [ci, dbl, dbl, i64, vp, vp]
         L.orc_gemm.restype = ci
         L.orc_gemm.argtypes = [i64, i64, i64, ci, ci, vp, i64, vp, i64, vp, ci, i64, vp, ci, dbl, dbl, ci, dbl, dbl, ci,
                                i64, i64, vp, vp, i64]
@@ -204,6 +206,68 @@ def grouped_gemm(As, Bs, *, layout_a="row", layout_b="col", Cs=None, biases=None
                         C=None if Cs is None else Cs[g], bias=None if biases is None else biases[g],
                         alpha=alpha, beta=beta, epi=epi, epi_args=epi_args))
     return [o[0] for o in out], [o[1] for o in out]
+
+
+def act_array(epi: str, x: torch.Tensor, args=(0.0, 0.0)) -> torch.Tensor:
+    """The activation applied to every element of an fp64 tensor."""
+    x = x.to(torch.float64).contiguous()
+    out = torch.empty_like(x)
+    lib().orc_act_array(EPILOGUES[epi], float(args[0]), float(args[1]), x.numel(), _ptr(x), _ptr(out))
+    return out
+
+
+def epilogue_chain(acc: torch.Tensor, absacc: torch.Tensor, *, alpha=1.0, beta=0.0, C=None, bias=None, epi="none",
+                   epi_args=(0.0, 0.0), row_scale=None, col_scale=None, row_bias=None, post_scale=1.0, aux_load=None):
+    """The extended epilogue chain (Table 1c built-ins per_row_scale, per_col_scale / per_channel_scale,
+    column_broadcast, scale, aux_store, aux_load) on a matrix of plain dot products, in the order the library fixes:
+
+        t   = alpha acc[i,j] row_scale[i] col_scale[j] + beta C[i,j] + bias[j] + row_bias[i]
+        aux = t                                   (what aux_store receives)
+        D   = post_scale act(t) + aux_load[i,j]
+
+    ``acc`` / ``absacc`` are sum a b and sum |a b| as fp64 [M, N]; every other tensor is widened to fp64 exactly.
+    Returns (D, aux, absacc_D, absacc_aux): the last two are the sums of the magnitudes of all terms that enter D
+    and aux (the scale of the fp32 tolerance)."""
+    f = lambda x: None if x is None else x.to(torch.float64)
+    M, N = acc.shape
+    t = float(alpha) * acc.to(torch.float64)
+    mag = abs(float(alpha)) * absacc.to(torch.float64)
+    if row_scale is not None:
+        t = t * f(row_scale).reshape(M, 1)
+        mag = mag * f(row_scale).abs().reshape(M, 1)
+    if col_scale is not None:
+        t = t * f(col_scale).reshape(1, N)
+        mag = mag * f(col_scale).abs().reshape(1, N)
+    if beta != 0.0:
+        t = t + float(beta) * f(C).reshape(M, N)
+        mag = mag + (float(beta) * f(C).reshape(M, N)).abs()
+    if bias is not None:
+        t = t + f(bias).reshape(1, N)
+        mag = mag + f(bias).abs().reshape(1, N)
+    if row_bias is not None:
+        t = t + f(row_bias).reshape(M, 1)
+        mag = mag + f(row_bias).abs().reshape(M, 1)
+    aux = t.clone()
+    d = float(post_scale) * act_array(epi, t, epi_args)
+    # the activations are 1-Lipschitz up to a small factor, so the magnitudes carry through scaled by post_scale
+    mag_d = abs(float(post_scale)) * mag
+    if aux_load is not None:
+        d = d + f(aux_load).reshape(M, N)
+        mag_d = mag_d + f(aux_load).abs().reshape(M, N)
+    return d, aux, mag_d, mag
+
+
+def gemm_ex(A, B, *, layout_a="row", layout_b="col", **chain):
+    """``epilogue_chain`` on the plain products of ``gemm`` (alpha = 1, no C, bias or activation there)."""
+    acc, absacc = gemm(A, B, layout_a=layout_a, layout_b=layout_b)
+    return epilogue_chain(acc, absacc, **chain)
+
+
+def conv2d_fprop_ex(X, Wf, *, pad=(0, 0), stride=(1, 1), dil=(1, 1), **chain):
+    """``epilogue_chain`` on the plain sums of ``conv2d_fprop``, rows = output pixels (n, p, q), columns = channels."""
+    acc, absacc = conv2d_fprop(X, Wf, pad=pad, stride=stride, dil=dil)
+    K = acc.shape[-1]
+    return epilogue_chain(acc.reshape(-1, K), absacc.reshape(-1, K), **chain)
 
 
 def conv_out_extent(size: int, pad: int, dil: int, filt: int, stride: int) -> int:

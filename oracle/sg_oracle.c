@@ -153,6 +153,11 @@ double orc_act2(int epi, double x, double a0, double a1) {
 
 double orc_act(int epi, double x) { return orc_act2(epi, x, 0.0, 0.0); }
 
+/* The activation applied to n values (used by the extended epilogue chain of oracle.py). */
+void orc_act_array(int epi, double a0, double a1, int64_t n, const double* in, double* out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_act2(epi, in[i], a0, a1);
+}
+
 /* -------------------------------------------------------------------------------------------
  * GEMM.   a(i,k) = A[i*lda + k] (row-major) or A[k*lda + i] (column-major)
  *         b(k,j) = B[k*ldb + j] (row-major) or B[j*ldb + k] (column-major)

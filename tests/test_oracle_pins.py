@@ -471,3 +471,78 @@ def test_fp8_gemm_with_bf16_bias_matches_torch_fp64():
     want = torch.nn.functional.conv2d(X.float().double().permute(0, 3, 1, 2), Wf.float().double().permute(0, 3, 1, 2),
                                       padding=1).permute(0, 2, 3, 1)
     assert torch.allclose(ref, want, rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------------------------------------------
+# Extended epilogue chain (Table 1c: per_row_scale, per_col_scale, column_broadcast, scale, aux_store, aux_load)
+# ------------------------------------------------------------------------------------------------
+
+def test_chain_hand_computed():
+    # A = [[1, 2], [3, 4]], B^T = [[1, 0], [1, 1]] (column-major B: rows are columns of B) -> A.B = [[1, 3], [3, 7]]
+    A = torch.tensor([[1., 2.], [3., 4.]]).to(torch.bfloat16)
+    Bt = torch.tensor([[1., 0.], [1., 1.]]).to(torch.bfloat16)
+    C = torch.tensor([[1., -1.], [2., 0.]])
+    bias = torch.tensor([0.5, -0.5]).to(torch.bfloat16)
+    R = torch.tensor([[10., 20.], [30., 40.]])
+    d, aux, mag_d, mag = orc.gemm_ex(A, Bt, alpha=2.0, beta=0.5, C=C, bias=bias, epi="relu",
+                                        row_scale=torch.tensor([1., -1.]), col_scale=torch.tensor([2., 0.5]),
+                                        row_bias=torch.tensor([0.25, 1.]), post_scale=3.0, aux_load=R)
+    # t[0,0] = 2*1*1*2 + 0.5*1 + 0.5 + 0.25 = 5.25      t[0,1] = 2*3*1*0.5 - 0.5 - 0.5 + 0.25 = 2.25
+    # t[1,0] = 2*3*(-1)*2 + 1 + 0.5 + 1 = -9.5           t[1,1] = 2*7*(-1)*0.5 + 0 - 0.5 + 1 = -6.5
+    assert aux.tolist() == [[5.25, 2.25], [-9.5, -6.5]]
+    # D = 3 relu(t) + R
+    assert d.tolist() == [[25.75, 26.75], [30.0, 40.0]]
+    assert mag.tolist() == [[5.25, 4.25], [14.5, 8.5]]
+    assert mag_d.tolist() == [[25.75, 32.75], [73.5, 65.5]]
+
+
+def test_chain_without_extras_is_the_plain_epilogue():
+    A, B, _ = inputs.make_gemm(37, 29, 50, "uniform", 1.0, seed=3)
+    C = inputs.uniform([37, 29], 3, 3).to(torch.float32)
+    bias = inputs.normal([29], 3, 4)
+    for epi in ("none", "gelu", "silu", "tanh"):
+        want, want_abs = orc.gemm(A, B, C=C, bias=bias, alpha=0.75, beta=-1.5, epi=epi)
+        d, aux, mag_d, mag = orc.gemm_ex(A, B, C=C, bias=bias, alpha=0.75, beta=-1.5, epi=epi)
+        torch.testing.assert_close(d, want, rtol=1e-13, atol=1e-13)
+        torch.testing.assert_close(mag_d, want_abs, rtol=1e-13, atol=1e-13)
+        lin, _ = orc.gemm(A, B, C=C, bias=bias, alpha=0.75, beta=-1.5)
+        torch.testing.assert_close(aux, lin, rtol=1e-13, atol=1e-13)
+
+
+def test_chain_scales_and_row_bias_reduce_to_plain_products():
+    M, N, K = 23, 19, 40
+    A, B, _ = inputs.make_gemm(M, N, K, "uniform", 1.0, seed=5)          # B is [N, K] (column-major)
+    # powers of two scale bf16 values exactly, so the scaled operands are again bf16 matrices
+    rs = torch.tensor([2.0 ** ((i % 5) - 2) for i in range(M)])
+    cs = torch.tensor([-(2.0 ** ((j % 3) - 1)) for j in range(N)])
+    d, _, _, _ = orc.gemm_ex(A, B, row_scale=rs, col_scale=cs)
+    As = (A.to(torch.float64) * rs.reshape(M, 1).double()).to(torch.bfloat16)
+    Bs = (B.to(torch.float64) * cs.reshape(N, 1).double()).to(torch.bfloat16)
+    want, _ = orc.gemm(As, Bs)
+    torch.testing.assert_close(d, want, rtol=1e-13, atol=1e-13)
+    # a per-row bias is one more k: A' = [A | r], B' = [B | 1]
+    r = inputs.uniform([M], 5, 9)                                         # bf16 values
+    d, _, _, _ = orc.gemm_ex(A, B, row_bias=r.to(torch.float32))
+    A1 = torch.cat([A, r.reshape(M, 1)], dim=1).contiguous()
+    B1 = torch.cat([B, torch.ones(N, 1, dtype=torch.bfloat16)], dim=1).contiguous()
+    want, _ = orc.gemm(A1, B1)
+    torch.testing.assert_close(d, want, rtol=1e-13, atol=1e-13)
+
+
+def test_chain_post_scale_and_aux_load_follow_the_activation():
+    A, B, _ = inputs.make_gemm(9, 11, 16, "uniform", 1.0, seed=8)
+    R = inputs.normal([9, 11], 8, 3)
+    base, _ = orc.gemm(A, B, epi="gelu")
+    d, aux, _, _ = orc.gemm_ex(A, B, epi="gelu", post_scale=-0.5, aux_load=R)
+    torch.testing.assert_close(d, -0.5 * base + R.double(), rtol=1e-13, atol=1e-13)
+    lin, _ = orc.gemm(A, B)
+    torch.testing.assert_close(aux, lin, rtol=0, atol=0)
+
+
+def test_chain_on_conv_rows_are_pixels_columns_are_channels():
+    X, Wf, _ = inputs.make_conv(2, 5, 4, 8, 6, 3, 3, "uniform", 1.0, seed=4)
+    cs = torch.tensor([2.0 ** (k % 3) for k in range(6)])
+    d, _, _, _ = orc.conv2d_fprop_ex(X, Wf, pad=(1, 1), col_scale=cs, epi="relu")
+    Ws = (Wf.to(torch.float64) * cs.reshape(6, 1, 1, 1).double()).to(torch.bfloat16)
+    want, _ = orc.conv2d_fprop(X, Ws, pad=(1, 1), epi="relu")
+    torch.testing.assert_close(d, want.reshape(-1, 6), rtol=1e-13, atol=1e-13)
