@@ -188,6 +188,41 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
                             const void* Cin, const void* bias, void* Y, void* cuda_stream);
 
 /*
+ * Extended epilogue chain: the remaining built-ins of the DSL's `>>` chain (Table 1c; Appendix A.1
+ * broadcast_op and fusion_op: per_row_scale, per_col_scale / per_channel_scale, column_broadcast,
+ * scale(alpha=), aux_store, aux_load).  The DSL lets these follow one another in any order; this library
+ * evaluates one fixed order (the order a dequantise - bias - activation - residual chain uses):
+ *
+ *   t          = alpha * acc[i][j] * row_scale[i] * col_scale[j] + beta * C[i][j] + bias[j] + row_bias[i]
+ *   aux_store[i][j] = t                        (cast to out_dtype; the value the activation sees)
+ *   D[i][j]    = post_scale * act(t) + aux_load[i][j]
+ *
+ * Every member is optional (NULL pointer / post_scale == 1 leaves its term out).
+ *   row_scale, row_bias   device, fp32, [M]   (conv: one per output pixel, [N*P*Q]); 4-byte aligned
+ *   col_scale             device, fp32, [N]   (conv: one per output channel, [K]);   16-byte aligned
+ *   aux_load, aux_store   device, out_dtype, row-major [M][ld] with ld >= N; base and ld multiples of 16 bytes;
+ *                         aux_store must not overlap D or any input; nothing beyond column N is read or written
+ * Errors as for sg_gemm / sg_conv2d_fprop, plus SG_ERR_ALIGNMENT / SG_ERR_INVALID_ARG for the rules above.
+ * ex == NULL makes the calls identical to sg_gemm / sg_conv2d_fprop.
+ */
+typedef struct sg_epilogue_ex {
+    const void* row_scale;
+    const void* col_scale;
+    const void* row_bias;
+    float post_scale;
+    int32_t reserved0;            /* must be 0 */
+    const void* aux_load;
+    int64_t ld_aux_load;          /* elements */
+    void* aux_store;
+    int64_t ld_aux_store;         /* elements */
+} sg_epilogue_ex_t;
+
+sg_status_t sg_gemm_ex(const sg_gemm_desc_t* desc, const sg_epilogue_ex_t* ex, const void* A, const void* B,
+                       const void* C, const void* bias, void* D, void* cuda_stream);
+sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_ex_t* ex, const void* X,
+                               const void* Wf, const void* Cin, const void* bias, void* Y, void* cuda_stream);
+
+/*
  * sg_transpose: out[b][c][r] = convert(in[b][r][c]) for b < batch, r < rows, c < cols -- the layout-transpose
  * stage with fused dtype conversion that the DSL's pipeline(transpose(...), kernel, transpose(...)) places
  * around a kernel (Section 3 "Multi-stage pipelines"; Appendix A.1 transpose_op: NCL <-> NLC, and

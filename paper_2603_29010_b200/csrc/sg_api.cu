@@ -481,9 +481,39 @@ void base_params(Params* p, const DeviceState& d, float alpha, float beta, int32
     p->timeout_ns = kWaitLimitNs;
 }
 
+// Validates the optional extended epilogue chain and copies it into the kernel parameters.
+sg_status_t apply_ex(Params* p, const sg_epilogue_ex_t* ex, int64_t N, int esize_out, const char* who) {
+    if (!ex) return SG_OK;
+    if (ex->reserved0 != 0) return fail(SG_ERR_INVALID_ARG, "%s: ex->reserved0 must be 0", who);
+    if (!std::isfinite(ex->post_scale)) return fail(SG_ERR_INVALID_ARG, "%s: post_scale must be finite", who);
+    if ((reinterpret_cast<uintptr_t>(ex->row_scale) | reinterpret_cast<uintptr_t>(ex->row_bias)) % 4)
+        return fail(SG_ERR_ALIGNMENT, "%s: row_scale and row_bias must be 4-byte aligned", who);
+    if (reinterpret_cast<uintptr_t>(ex->col_scale) % 16) return fail(SG_ERR_ALIGNMENT, "%s: col_scale must be 16-byte aligned", who);
+    if (ex->aux_load) {
+        if (ex->ld_aux_load < N) return fail(SG_ERR_INVALID_ARG, "%s: ld_aux_load smaller than N", who);
+        if (reinterpret_cast<uintptr_t>(ex->aux_load) % 16 || (ex->ld_aux_load * esize_out) % 16)
+            return fail(SG_ERR_ALIGNMENT, "%s: aux_load base and leading dimension must be multiples of 16 bytes", who);
+    }
+    if (ex->aux_store) {
+        if (ex->ld_aux_store < N) return fail(SG_ERR_INVALID_ARG, "%s: ld_aux_store smaller than N", who);
+        if (reinterpret_cast<uintptr_t>(ex->aux_store) % 16 || (ex->ld_aux_store * esize_out) % 16)
+            return fail(SG_ERR_ALIGNMENT, "%s: aux_store base and leading dimension must be multiples of 16 bytes", who);
+    }
+    p->row_scale = static_cast<const float*>(ex->row_scale);
+    p->col_scale = static_cast<const float*>(ex->col_scale);
+    p->row_bias = static_cast<const float*>(ex->row_bias);
+    p->post_scale = ex->post_scale;
+    p->aux_load = ex->aux_load;
+    p->ld_aux_load = ex->ld_aux_load;
+    p->aux_store = ex->aux_store;
+    p->ld_aux_store = ex->ld_aux_store;
+    p->ex_any = (ex->row_scale || ex->col_scale || ex->row_bias || ex->aux_load || ex->aux_store || ex->post_scale != 1.0f) ? 1 : 0;
+    return SG_OK;
+}
+
 sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int64_t sB, int64_t sC, int64_t sD,
                       int64_t sBias, const void* A, const void* B, const void* C, const void* bias, void* D,
-                      void* stream, const char* who) {
+                      void* stream, const char* who, const sg_epilogue_ex_t* ex = nullptr) {
     Checked c;
     sg_status_t st = check_gemm_desc(desc, false, &c);
     if (st != SG_OK) return st;
@@ -523,6 +553,8 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
     p.num_kb = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
     plan_tail(*d, s, tiles, &p, min_b_rows);
+    st = apply_ex(&p, ex, desc->N, c.esize_out, who);
+    if (st != SG_OK) return st;
     p.bias = bias;
     p.C = desc->beta != 0.0f ? C : nullptr;
     p.ldc = desc->ldc;
@@ -690,6 +722,11 @@ sg_status_t sg_set_tail_mode(int32_t mode) {
 sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C, const void* bias, void* D,
                     void* cuda_stream) {
     return run_dense(desc, 1, 0, 0, 0, 0, 0, A, B, C, bias, D, cuda_stream, "sg_gemm");
+}
+
+sg_status_t sg_gemm_ex(const sg_gemm_desc_t* desc, const sg_epilogue_ex_t* ex, const void* A, const void* B, const void* C,
+                       const void* bias, void* D, void* cuda_stream) {
+    return run_dense(desc, 1, 0, 0, 0, 0, 0, A, B, C, bias, D, cuda_stream, "sg_gemm_ex", ex);
 }
 
 sg_status_t sg_batched_gemm(const sg_gemm_desc_t* desc, int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
@@ -860,6 +897,11 @@ sg_status_t sg_grouped_gemm_static(const sg_gemm_desc_t* common, int32_t groups,
 
 sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const void* Wf, const void* Cin, const void* bias,
                             void* Y, void* cuda_stream) {
+    return sg_conv2d_fprop_ex(desc, nullptr, X, Wf, Cin, bias, Y, cuda_stream);
+}
+
+sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_ex_t* ex, const void* X, const void* Wf,
+                               const void* Cin, const void* bias, void* Y, void* cuda_stream) {
     if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
     Checked c;
     sg_status_t st = check_common(desc->in_dtype, desc->out_dtype, desc->epi, desc->alpha, desc->beta, desc->epi_arg0, desc->epi_arg1,
@@ -956,6 +998,8 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
     }
     st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, Y,
                         desc->K, Mg, 1, desc->K, 0, c.f32_out ? 32 : 64, 32, "Y");
+    if (st != SG_OK) return st;
+    st = apply_ex(&p, ex, desc->K, c.esize_out, "sg_conv2d_fprop_ex");
     if (st != SG_OK) return st;
     return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
 }

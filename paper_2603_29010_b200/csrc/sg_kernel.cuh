@@ -74,6 +74,17 @@ struct alignas(64) Params {
     int32_t bk_elems;                   // elements of K per 128-byte stage row: 64 (16-bit) or 128 (8-bit)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
+    // extended epilogue chain (all optional; ex_any = 1 when any of them is in use; dense and conv modes only):
+    //   t = alpha acc * row_scale[i] * col_scale[j] + beta C + bias[j] + row_bias[i];  aux_store[i][j] = t;
+    //   D = post_scale * act(t) + aux_load[i][j]
+    int32_t ex_any;
+    float post_scale;
+    const float* row_scale;             // fp32 [M]
+    const float* col_scale;             // fp32 [N]
+    const float* row_bias;              // fp32 [M]
+    const void* aux_load;               // out dtype, row-major, leading dimension ld_aux_load
+    void* aux_store;                    // out dtype, row-major, leading dimension ld_aux_store
+    int64_t ld_aux_load, ld_aux_store;  // elements
     uint32_t* status;                   // device status words (8 x u32)
     uint64_t timeout_ns;                // bound of every device-side wait
 };
@@ -758,6 +769,32 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int i = 0; i < CH; ++i) v[i] *= alpha;
                 }
+#ifdef SG_NO_EX
+                constexpr bool ex_any = false;       // experiments: the chain compiled out
+#else
+                const bool ex_any = p.ex_any != 0;
+#endif
+                if (ex_any) {
+                    if (p.row_scale != nullptr) {
+                        const float rs = row < ti.rows ? __ldg(p.row_scale + row) : 0.0f;
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) v[i] *= rs;
+                    }
+                    if (p.col_scale != nullptr) {
+                        // every lane reads the same addresses: one broadcast transaction per load
+                        const float* cs = p.col_scale + n0 + c * CH;
+                        if (n0 + (c + 1) * CH <= p.N) {
+#pragma unroll
+                            for (int i = 0; i < CH; i += 4) {
+                                const float4 s4 = __ldg(reinterpret_cast<const float4*>(cs + i));
+                                v[i] *= s4.x; v[i + 1] *= s4.y; v[i + 2] *= s4.z; v[i + 3] *= s4.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < CH; ++i) v[i] *= (n0 + c * CH + i < p.N) ? __ldg(cs + i) : 0.0f;
+                        }
+                    }
+                }
                 if (has_c && row < ti.rows) {
                     const int col0 = n0 + c * CH;
                     if constexpr (kOutF32) {
@@ -801,7 +838,80 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         v[i] += b0; v[i + 1] += b1; v[i + 2] += b2f; v[i + 3] += b3;
                     }
                 }
+                if (ex_any) {
+                    if (p.row_bias != nullptr) {
+                        const float rb = row < ti.rows ? __ldg(p.row_bias + row) : 0.0f;
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) v[i] += rb;
+                    }
+                    if (p.aux_store != nullptr && row < ti.rows) {
+                        // the value the activation is about to see, in the output's type; each lane owns one row
+                        const int col0 = n0 + c * CH;
+                        if constexpr (kOutF32) {
+                            float* ap = reinterpret_cast<float*>(p.aux_store) + static_cast<int64_t>(row) * p.ld_aux_store + col0;
+                            if (col0 + CH <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < CH; i += 4)
+                                    *reinterpret_cast<float4*>(ap + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                            } else {
+                                for (int i = 0; i < CH; ++i) if (col0 + i < p.N) ap[i] = v[i];
+                            }
+                        } else {
+                            uint16_t* ap = reinterpret_cast<uint16_t*>(p.aux_store) + static_cast<int64_t>(row) * p.ld_aux_store + col0;
+                            if (col0 + CH <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < CH; i += 8)
+                                    *reinterpret_cast<uint4*>(ap + i) =
+                                        make_uint4(pack2<kOutF16>(v[i], v[i + 1]), pack2<kOutF16>(v[i + 2], v[i + 3]),
+                                                   pack2<kOutF16>(v[i + 4], v[i + 5]), pack2<kOutF16>(v[i + 6], v[i + 7]));
+                            } else {
+                                for (int i = 0; i < CH; ++i)
+                                    if (col0 + i < p.N) ap[i] = static_cast<uint16_t>(pack2<kOutF16>(v[i], 0.0f) & 0xFFFFu);
+                            }
+                        }
+                    }
+                }
                 if (epi >= EPI_RELU) apply_act_chunk<kOut == 0, CH>(v, epi, p.epi_arg0, p.epi_arg1);
+                if (ex_any) {
+                    if (p.post_scale != 1.0f) {
+                        const float ps = p.post_scale;
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) v[i] *= ps;
+                    }
+                    if (p.aux_load != nullptr && row < ti.rows) {
+                        const int col0 = n0 + c * CH;
+                        if constexpr (kOutF32) {
+                            const float* rp = reinterpret_cast<const float*>(p.aux_load) + static_cast<int64_t>(row) * p.ld_aux_load + col0;
+                            if (col0 + CH <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < CH; i += 4) {
+                                    const float4 rv = *reinterpret_cast<const float4*>(rp + i);
+                                    v[i] += rv.x; v[i + 1] += rv.y; v[i + 2] += rv.z; v[i + 3] += rv.w;
+                                }
+                            } else {
+                                for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += rp[i];
+                            }
+                        } else {
+                            const uint16_t* rp = reinterpret_cast<const uint16_t*>(p.aux_load) + static_cast<int64_t>(row) * p.ld_aux_load + col0;
+                            if (col0 + CH <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < CH; i += 8) {
+                                    const uint4 rv = *reinterpret_cast<const uint4*>(rp + i);
+                                    const uint32_t w[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        float lo, hi;
+                                        unpack2<kOutF16>(w[j], lo, hi);
+                                        v[i + 2 * j] += lo;
+                                        v[i + 2 * j + 1] += hi;
+                                    }
+                                }
+                            } else {
+                                for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += half_bits_to_float(rp[i], kOutF16);
+                            }
+                        }
+                    }
+                }
                 if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(21 + 4 * (c / kStep > 0 ? 1 : 0));
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes

@@ -35,7 +35,7 @@ EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5
 DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4}
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
-            "sg_grouped_gemm_static", "sg_conv2d_fprop",
+            "sg_grouped_gemm_static", "sg_conv2d_fprop", "sg_gemm_ex", "sg_conv2d_fprop_ex",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
             "sg_last_kernel_clock", "sg_transpose"]
@@ -67,6 +67,13 @@ class Conv2dDesc(ctypes.Structure):
                 ("epi_arg0", ctypes.c_float), ("epi_arg1", ctypes.c_float), ("reserved", ctypes.c_int32)]
 
 
+class EpilogueEx(ctypes.Structure):
+    _fields_ = [("row_scale", ctypes.c_void_p), ("col_scale", ctypes.c_void_p), ("row_bias", ctypes.c_void_p),
+                ("post_scale", ctypes.c_float), ("reserved0", ctypes.c_int32),
+                ("aux_load", ctypes.c_void_p), ("ld_aux_load", ctypes.c_int64),
+                ("aux_store", ctypes.c_void_p), ("ld_aux_store", ctypes.c_int64)]
+
+
 class TransposeDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in ("batch", "rows", "cols", "ld_in", "ld_out", "stride_in", "stride_out")] + \
                [(n, ctypes.c_int32) for n in ("in_dtype", "out_dtype", "reserved", "reserved2")]
@@ -87,6 +94,10 @@ class Sol(ctypes.Structure):
 _vp, _i64, _i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
 _lib.sg_gemm.restype = ctypes.c_int
 _lib.sg_gemm.argtypes = [ctypes.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_gemm_ex.restype = ctypes.c_int
+_lib.sg_gemm_ex.argtypes = [ctypes.POINTER(GemmDesc), ctypes.POINTER(EpilogueEx), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_conv2d_fprop_ex.restype = ctypes.c_int
+_lib.sg_conv2d_fprop_ex.argtypes = [ctypes.POINTER(Conv2dDesc), ctypes.POINTER(EpilogueEx), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_batched_gemm.restype = ctypes.c_int
 _lib.sg_batched_gemm.argtypes = [ctypes.POINTER(GemmDesc), _i64, _i64, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_grouped_gemm_workspace_size.restype = ctypes.c_int
@@ -192,17 +203,53 @@ def _mnk(A, B, layout_a, layout_b):
     return M, N, K
 
 
+def _addr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _ex_struct(ex: Optional[dict]) -> Optional[EpilogueEx]:
+    """``ex``: dict with any of row_scale, col_scale, row_bias (fp32 vectors), post_scale (float), aux_load,
+    aux_store (2-D tensors of the output's type, inner stride 1) -> the C structure (None when ``ex`` is None)."""
+    if ex is None:
+        return None
+    unknown = set(ex) - {"row_scale", "col_scale", "row_bias", "post_scale", "aux_load", "aux_store"}
+    if unknown:
+        raise ValueError(f"unknown extended-epilogue members: {sorted(unknown)}")
+    for name in ("row_scale", "col_scale", "row_bias"):
+        t = ex.get(name)
+        if t is not None and (t.dtype != torch.float32 or not t.is_contiguous()):
+            raise ValueError(f"{name} must be a contiguous fp32 vector")
+    al, ast = ex.get("aux_load"), ex.get("aux_store")
+    def as2d(t, name):                      # conv: a contiguous [N, P, Q, K] tensor is the [NPQ, K] matrix
+        if t is None or t.dim() == 2:
+            return t
+        if not t.is_contiguous():
+            raise ValueError(f"{name} with more than two dimensions must be contiguous")
+        return t.view(-1, t.shape[-1])
+    al2, ast2 = as2d(al, "aux_load"), as2d(ast, "aux_store")
+    return EpilogueEx(_addr(ex.get("row_scale")), _addr(ex.get("col_scale")), _addr(ex.get("row_bias")),
+                      float(ex.get("post_scale", 1.0)), 0,
+                      _addr(al2), _ld(al2) if al2 is not None else 0, _addr(ast2), _ld(ast2) if ast2 is not None else 0)
+
+
 def gemm(A: torch.Tensor, B: torch.Tensor, *, C: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
          out: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.bfloat16, alpha: float = 1.0,
          beta: float = 0.0, epi: str = "none", epi_args=(0.0, 0.0), layout_a: str = "row", layout_b: str = "col",
-         stream=None) -> torch.Tensor:
-    """D = act(alpha A.B + beta C + bias) through ``sg_gemm``.  Returns D (``out`` if given)."""
+         stream=None, ex: Optional[dict] = None) -> torch.Tensor:
+    """D = act(alpha A.B + beta C + bias) through ``sg_gemm``.  Returns D (``out`` if given).
+
+    ``ex`` (see ``_ex_struct``) routes the call through ``sg_gemm_ex`` with the extended epilogue chain."""
     M, N, K = _mnk(A, B, layout_a, layout_b)
     ensure_scratch()
     if out is None:
         out = torch.empty((M, N), dtype=out_dtype, device=A.device)
     desc = _gemm_desc(M, N, K, _ld(A), _ld(B), _ld(C) if C is not None else max(N, 1), _ld(out), layout_a, layout_b,
                       out.dtype, alpha, beta, epi, epi_args, A.dtype)
+    if ex is not None:
+        exs = _ex_struct(ex)
+        _check(_lib.sg_gemm_ex(ctypes.byref(desc), ctypes.byref(exs), _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out),
+                               _stream(stream)))
+        return out
     _check(_lib.sg_gemm(ctypes.byref(desc), _ptr(A), _ptr(B), _ptr(C), _ptr(bias), _ptr(out), _stream(stream)))
     return out
 
@@ -296,8 +343,10 @@ def grouped_gemm_static(As: Sequence[torch.Tensor], Bs: Sequence[torch.Tensor], 
 
 def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1), dil=(1, 1), Cin=None, bias=None,
                  out=None, out_dtype=torch.bfloat16, alpha=1.0, beta=0.0, epi="none", epi_args=(0.0, 0.0),
-                 stream=None) -> torch.Tensor:
-    """NHWC x KRSC -> NPQK forward convolution through ``sg_conv2d_fprop`` (implicit GEMM, nothing materialised)."""
+                 stream=None, ex: Optional[dict] = None) -> torch.Tensor:
+    """NHWC x KRSC -> NPQK forward convolution through ``sg_conv2d_fprop`` (implicit GEMM, nothing materialised).
+
+    ``ex`` routes the call through ``sg_conv2d_fprop_ex`` (rows are output pixels, columns output channels)."""
     if X.dim() != 4 or Wf.dim() != 4 or not X.is_contiguous() or not Wf.is_contiguous():
         raise ValueError("X (NHWC) and Wf (KRSC) must be contiguous 4-D tensors")
     N, H, W, C = X.shape
@@ -312,6 +361,11 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
     desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], DTYPES[X.dtype],
                       DTYPES[out.dtype],
                       float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), 0)
+    if ex is not None:
+        exs = _ex_struct(ex)
+        _check(_lib.sg_conv2d_fprop_ex(ctypes.byref(desc), ctypes.byref(exs), _ptr(X), _ptr(Wf), _ptr(Cin), _ptr(bias),
+                                       _ptr(out), _stream(stream)))
+        return out
     _check(_lib.sg_conv2d_fprop(ctypes.byref(desc), _ptr(X), _ptr(Wf), _ptr(Cin), _ptr(bias), _ptr(out), _stream(stream)))
     return out
 

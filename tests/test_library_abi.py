@@ -33,6 +33,7 @@ def test_library_exports_every_declared_symbol(sg):
 def test_struct_layouts_match_the_header(sg):
     assert ctypes.sizeof(sg.GemmDesc) == 96 and ctypes.sizeof(sg.Conv2dDesc) == 112
     assert ctypes.sizeof(sg.Hw) == 48 and ctypes.sizeof(sg.Sol) == 80
+    assert ctypes.sizeof(sg.EpilogueEx) == 64
 
 
 def test_status_strings(sg):
