@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.orc_conv_out_extent.argtypes = [i64] * 5
         L.orc_conv2d_fprop.restype = ci
         L.orc_conv2d_fprop.argtypes = [vp, vp, vp, vp, ci, vp, ci, dbl, dbl, ci, dbl, dbl, ci, i64, i64, vp, vp]
+        L.orc_conv2d_dgrad.restype = ci
+        L.orc_conv2d_dgrad.argtypes = [vp, vp, vp, vp, ci, dbl, dbl, ci, i64, i64, vp, vp]
+        L.orc_conv2d_wgrad.restype = ci
+        L.orc_conv2d_wgrad.argtypes = [vp, vp, vp, vp, ci, dbl, dbl, ci, i64, i64, vp, vp]
         L.orc_conv2d_points.restype = ci
         L.orc_conv2d_points.argtypes = [vp, vp, vp, vp, ci, vp, ci, dbl, dbl, ci, dbl, dbl, ci, i64, vp, vp, vp, vp]
         L.orc_transpose.restype = ci
@@ -315,6 +319,63 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
         raise ValueError(f"orc_conv2d_fprop rejected its arguments (code {rc})")
     if pixels is None:
         return ref.view(N, P, Q, K), absacc.view(N, P, Q, K)
+    return ref, absacc
+
+
+def _grad_dims(N, H, W, C, K, R, S, pad, stride, dil):
+    d = torch.tensor([N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1]], dtype=torch.int64)
+    P = conv_out_extent(H, pad[0], dil[0], R, stride[0])
+    Q = conv_out_extent(W, pad[1], dil[1], S, stride[1])
+    return d, P, Q
+
+
+def _check_grad_operand(t, shape, name, dtype=None):
+    if t.device.type != "cpu" or tuple(t.shape) != tuple(shape) or not t.is_contiguous() \
+            or (dtype is not None and t.dtype != dtype) or (dtype is None and t.dtype not in (torch.bfloat16, torch.float16)):
+        raise ValueError(f"{name}: want a contiguous CPU tensor of shape {tuple(shape)} (bf16 or fp16)")
+
+
+def conv2d_dgrad(dY: torch.Tensor, Wf: torch.Tensor, hw: Tuple[int, int], *, pad=(0, 0), stride=(1, 1), dil=(1, 1),
+                 Cin=None, alpha=1.0, beta=0.0, pixels: Optional[Tuple[int, int]] = None):
+    """Gradient of the forward convolution with respect to its input: ``dY`` [N,P,Q,K], ``Wf`` [K,R,S,C] ->
+    [N,H,W,C] with ``hw = (H, W)`` (or ``[pixels, C]`` for a flattened range of (n,h,w))."""
+    K, R, S, C = Wf.shape
+    N = dY.shape[0]
+    H, W = hw
+    d, P, Q = _grad_dims(N, H, W, C, K, R, S, pad, stride, dil)
+    _check_grad_operand(dY, (N, P, Q, K), "dY")
+    _check_grad_operand(Wf, (K, R, S, C), "Wf", dY.dtype)
+    Cin, c_dtype = _conv_c(Cin, N, H, W, C)
+    p0, p1 = pixels if pixels is not None else (0, N * H * W)
+    ref = torch.empty((p1 - p0, C), dtype=torch.float64)
+    absacc = torch.empty_like(ref)
+    rc = lib().orc_conv2d_dgrad(_ptr(d), _ptr(dY), _ptr(Wf), _ptr(Cin), c_dtype, float(alpha), float(beta),
+                                _DTYPES[dY.dtype], p0, p1, _ptr(ref), _ptr(absacc))
+    if rc:
+        raise ValueError(f"orc_conv2d_dgrad rejected its arguments (code {rc})")
+    if pixels is None:
+        return ref.view(N, H, W, C), absacc.view(N, H, W, C)
+    return ref, absacc
+
+
+def conv2d_wgrad(dY: torch.Tensor, X: torch.Tensor, rs: Tuple[int, int], *, pad=(0, 0), stride=(1, 1), dil=(1, 1),
+                 Cin=None, alpha=1.0, beta=0.0, filters: Optional[Tuple[int, int]] = None):
+    """Gradient with respect to the filter: ``dY`` [N,P,Q,K], ``X`` [N,H,W,C] -> [K,R,S,C] with ``rs = (R, S)``
+    (or filters ``[k0, k1)`` only)."""
+    N, H, W, C = X.shape
+    K = dY.shape[3]
+    R, S = rs
+    d, P, Q = _grad_dims(N, H, W, C, K, R, S, pad, stride, dil)
+    _check_grad_operand(dY, (N, P, Q, K), "dY")
+    _check_grad_operand(X, (N, H, W, C), "X", dY.dtype)
+    Cin, c_dtype = _conv_c(Cin, K, R, S, C)
+    k0, k1 = filters if filters is not None else (0, K)
+    ref = torch.empty((k1 - k0, R, S, C), dtype=torch.float64)
+    absacc = torch.empty_like(ref)
+    rc = lib().orc_conv2d_wgrad(_ptr(d), _ptr(dY), _ptr(X), _ptr(Cin), c_dtype, float(alpha), float(beta),
+                                _DTYPES[dY.dtype], k0, k1, _ptr(ref), _ptr(absacc))
+    if rc:
+        raise ValueError(f"orc_conv2d_wgrad rejected its arguments (code {rc})")
     return ref, absacc
 
 

@@ -368,6 +368,92 @@ int orc_conv2d_points(const int64_t* dims, const void* X, const void* Wf,
 }
 
 /* -------------------------------------------------------------------------------------------
+ * conv2d data and weight gradients (the DSL's conv2d_dgrad / conv2d_wgrad operators, Appendix A.1): the two
+ * adjoints of the forward map  y[n,p,q,k] = sum_{r,s,c} x[n, p sh - ph + r dh, q sw - pw + s dw, c] w[k,r,s,c].
+ *   dgrad:  dx[n,h,w,c]  = alpha * sum over all (p,r), (q,s), k with  p sh - ph + r dh = h  and  q sw - pw + s dw = w
+ *                          of dy[n,p,q,k] w[k,r,s,c]                     + beta * Cin[n,h,w,c]
+ *   wgrad:  dw[k,r,s,c]  = alpha * sum_{n,p,q} dy[n,p,q,k] x[n, p sh - ph + r dh, q sw - pw + s dw, c]
+ *                          (taps outside the image contribute 0)        + beta * Cin[k,r,s,c]
+ * dims as for the forward convolution (N,H,W,C describe x / dx; K,R,S the filter); dy is [N,P,Q,K].
+ * ----------------------------------------------------------------------------------------- */
+int orc_conv2d_dgrad(const int64_t* dims, const void* dY, const void* Wf, const void* Cin, int c_dtype,
+                     double alpha, double beta, int in_dtype, int64_t pix_begin, int64_t pix_end,
+                     double* ref, double* absacc) {
+    conv_problem cv;
+    int rc = conv_setup(&cv, dims, NULL, Wf, Cin, c_dtype, NULL, 0, alpha, beta, 0, 0.0, 0.0, in_dtype);
+    if (rc) return rc;
+    if (pix_begin < 0 || pix_end > cv.N * cv.H * cv.W || pix_begin > pix_end) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t pix = pix_begin; pix < pix_end; ++pix) {
+        const int64_t n = pix / (cv.H * cv.W), h = (pix / cv.W) % cv.H, w = pix % cv.W;
+        for (int64_t c = 0; c < cv.C; ++c) {
+            double sum = 0.0, asum = 0.0;
+            for (int64_t p = 0; p < cv.P; ++p)
+                for (int64_t r = 0; r < cv.R; ++r) {
+                    if (p * cv.stride_h - cv.pad_h + r * cv.dil_h != h) continue;
+                    for (int64_t q = 0; q < cv.Q; ++q)
+                        for (int64_t s2 = 0; s2 < cv.S; ++s2) {
+                            if (q * cv.stride_w - cv.pad_w + s2 * cv.dil_w != w) continue;
+                            for (int64_t k = 0; k < cv.K; ++k) {
+                                double t = in_to_f64(dY, in_dtype, ((n * cv.P + p) * cv.Q + q) * cv.K + k) *
+                                           in_to_f64(Wf, in_dtype, ((k * cv.R + r) * cv.S + s2) * cv.C + c);
+                                sum += t;
+                                asum += fabs(t);
+                            }
+                        }
+                }
+            double v = alpha * sum, av = fabs(alpha) * asum;
+            if (beta != 0.0) {
+                double cc = load_as_f64(Cin, c_dtype, pix * cv.C + c);
+                v += beta * cc;
+                av += fabs(beta * cc);
+            }
+            ref[(pix - pix_begin) * cv.C + c] = v;
+            if (absacc) absacc[(pix - pix_begin) * cv.C + c] = av;
+        }
+    }
+    return 0;
+}
+
+/* Filters [k_begin, k_end): ref holds (k_end-k_begin) x R x S x C values. */
+int orc_conv2d_wgrad(const int64_t* dims, const void* dY, const void* X, const void* Cin, int c_dtype,
+                     double alpha, double beta, int in_dtype, int64_t k_begin, int64_t k_end,
+                     double* ref, double* absacc) {
+    conv_problem cv;
+    int rc = conv_setup(&cv, dims, X, NULL, Cin, c_dtype, NULL, 0, alpha, beta, 0, 0.0, 0.0, in_dtype);
+    if (rc) return rc;
+    if (k_begin < 0 || k_end > cv.K || k_begin > k_end) return 1;
+    const int64_t rsc = cv.R * cv.S * cv.C;
+#pragma omp parallel for schedule(static)
+    for (int64_t e = k_begin * rsc; e < k_end * rsc; ++e) {
+        const int64_t k = e / rsc, r = (e / (cv.S * cv.C)) % cv.R, s2 = (e / cv.C) % cv.S, c = e % cv.C;
+        double sum = 0.0, asum = 0.0;
+        for (int64_t n = 0; n < cv.N; ++n)
+            for (int64_t p = 0; p < cv.P; ++p) {
+                const int64_t h = p * cv.stride_h - cv.pad_h + r * cv.dil_h;
+                if (h < 0 || h >= cv.H) continue;
+                for (int64_t q = 0; q < cv.Q; ++q) {
+                    const int64_t w = q * cv.stride_w - cv.pad_w + s2 * cv.dil_w;
+                    if (w < 0 || w >= cv.W) continue;
+                    double t = in_to_f64(dY, in_dtype, ((n * cv.P + p) * cv.Q + q) * cv.K + k) *
+                               in_to_f64(X, in_dtype, ((n * cv.H + h) * cv.W + w) * cv.C + c);
+                    sum += t;
+                    asum += fabs(t);
+                }
+            }
+        double v = alpha * sum, av = fabs(alpha) * asum;
+        if (beta != 0.0) {
+            double cc = load_as_f64(Cin, c_dtype, e);
+            v += beta * cc;
+            av += fabs(beta * cc);
+        }
+        ref[e - k_begin * rsc] = v;
+        if (absacc) absacc[e - k_begin * rsc] = av;
+    }
+    return 0;
+}
+
+/* -------------------------------------------------------------------------------------------
  * Layout transpose with dtype conversion (the DSL's transpose(ref, L1, L2[, dt1, dt2]) stage, Appendix A.1):
  *   out[b][c][r] = convert(in[b][r][c]).  bf16 -> fp32 is exact; fp32 -> bf16 rounds to nearest, ties to even
  *   (the 16 discarded bits decide; a NaN stays a NaN).  The result is returned as fp64 holding the converted value.

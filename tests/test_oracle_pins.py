@@ -546,3 +546,74 @@ def test_chain_on_conv_rows_are_pixels_columns_are_channels():
     Ws = (Wf.to(torch.float64) * cs.reshape(6, 1, 1, 1).double()).to(torch.bfloat16)
     want, _ = orc.conv2d_fprop(X, Ws, pad=(1, 1), epi="relu")
     torch.testing.assert_close(d, want.reshape(-1, 6), rtol=1e-13, atol=1e-13)
+
+
+# ------------------------------------------------------------------------------------------------
+# conv2d_dgrad / conv2d_wgrad (Appendix A.1 operators): the adjoints of the forward convolution
+# ------------------------------------------------------------------------------------------------
+
+def test_dgrad_wgrad_hand_computed():
+    # N=1, H=W=2, C=K=1, 2x2 filter, no padding -> P=Q=1: y = sum x*w.
+    # dx = dy * w (elementwise over the window), dw = dy * x.
+    dY = bf([[[[3.0]]]])
+    Wf = bf([[[[1.0], [2.0]], [[-1.0], [0.5]]]])
+    X = bf([[[[1.0], [2.0]], [[4.0], [-2.0]]]])
+    dx, mag = orc.conv2d_dgrad(dY, Wf, (2, 2))
+    assert dx.reshape(2, 2).tolist() == [[3.0, 6.0], [-3.0, 1.5]]
+    assert mag.reshape(2, 2).tolist() == [[3.0, 6.0], [3.0, 1.5]]
+    dw, _ = orc.conv2d_wgrad(dY, X, (2, 2))
+    assert dw.reshape(2, 2).tolist() == [[3.0, 6.0], [12.0, -6.0]]
+    # 1x3 input, 1x2 filter, pad 1, stride 2 (W direction): outputs q=0 reads w in {-1,0}, q=1 reads w in {1,2}
+    dY = bf([[[[1.0], [10.0]]]])                    # [1,1,2,1]
+    Wf = bf([[[[2.0], [3.0]]]])                     # [1,1,2,1]
+    dx, _ = orc.conv2d_dgrad(dY, Wf, (1, 3), pad=(0, 1), stride=(1, 2))
+    assert dx.reshape(3).tolist() == [3.0, 20.0, 30.0]
+    X = bf([[[[5.0], [6.0], [7.0]]]])
+    dw, _ = orc.conv2d_wgrad(dY, X, (1, 2), pad=(0, 1), stride=(1, 2))
+    assert dw.reshape(2).tolist() == [60.0, 75.0]   # tap 0: 10*6 (q=0 is in the halo), tap 1: 1*5 + 10*7
+
+
+@pytest.mark.parametrize("pad,stride,dil,R,S", [((1, 1), (1, 1), (1, 1), 3, 3), ((0, 2), (2, 1), (1, 2), 2, 3),
+                                                ((2, 1), (2, 3), (2, 1), 3, 2), ((0, 0), (1, 1), (1, 1), 1, 1)])
+def test_dgrad_wgrad_are_the_adjoints_of_the_forward_oracle(pad, stride, dil, R, S):
+    # <conv(X, W), dY> = <X, dgrad(dY, W)> = <W, wgrad(dY, X)>, exactly on small integers
+    N_, H, W_, C, K = 2, 7, 6, 3, 4
+    X = randi([N_, H, W_, C], 21, 1)
+    Wf = randi([K, R, S, C], 21, 2)
+    y, _ = orc.conv2d_fprop(X, Wf, pad=pad, stride=stride, dil=dil)
+    dY = randi(list(y.shape), 21, 3)
+    lhs = float((y * dY.double()).sum())
+    dx, _ = orc.conv2d_dgrad(dY, Wf, (H, W_), pad=pad, stride=stride, dil=dil)
+    dw, _ = orc.conv2d_wgrad(dY, X, (R, S), pad=pad, stride=stride, dil=dil)
+    assert float((dx * X.double()).sum()) == lhs
+    assert float((dw * Wf.double()).sum()) == lhs
+
+
+@pytest.mark.parametrize("pad,stride,dil", [((1, 1), (1, 1), (1, 1)), ((1, 0), (2, 2), (1, 1)), ((2, 2), (1, 2), (2, 1))])
+def test_dgrad_wgrad_match_torch_library_gradients(pad, stride, dil):
+    N_, H, W_, C, K, R, S = 2, 8, 7, 5, 3, 3, 3
+    X, Wf, _ = inputs.make_conv(N_, H, W_, C, K, R, S, "uniform", 1.0, seed=22)
+    P = orc.conv_out_extent(H, pad[0], dil[0], R, stride[0])
+    Q = orc.conv_out_extent(W_, pad[1], dil[1], S, stride[1])
+    dY = inputs.uniform([N_, P, Q, K], 22, 3)
+    Cx = inputs.normal([N_, H, W_, C], 22, 4).to(torch.float32)
+    dx, _ = orc.conv2d_dgrad(dY, Wf, (H, W_), pad=pad, stride=stride, dil=dil, Cin=Cx, alpha=0.5, beta=2.0)
+    dw, _ = orc.conv2d_wgrad(dY, X, (R, S), pad=pad, stride=stride, dil=dil, alpha=-1.5)
+    g = dY.double().permute(0, 3, 1, 2)
+    want_dx = torch.nn.grad.conv2d_input((N_, C, H, W_), Wf.double().permute(0, 3, 1, 2), g, stride=stride, padding=pad,
+                                         dilation=dil).permute(0, 2, 3, 1)
+    want_dw = torch.nn.grad.conv2d_weight(X.double().permute(0, 3, 1, 2), (K, C, R, S), g, stride=stride, padding=pad,
+                                          dilation=dil).permute(0, 2, 3, 1)
+    torch.testing.assert_close(dx, 0.5 * want_dx + 2.0 * Cx.double(), rtol=1e-12, atol=1e-12)
+    torch.testing.assert_close(dw, -1.5 * want_dw, rtol=1e-12, atol=1e-12)
+
+
+def test_dgrad_wgrad_ranges_agree_with_full():
+    X, Wf, _ = inputs.make_conv(2, 5, 6, 4, 3, 3, 2, "uniform", 1.0, seed=23)
+    dY = inputs.uniform([2, 5, 7, 3], 23, 3)          # pad (1,1): P = 5, Q = 6 + 2 - 1 = 7
+    dx, ax = orc.conv2d_dgrad(dY, Wf, (5, 6), pad=(1, 1))
+    part, apart = orc.conv2d_dgrad(dY, Wf, (5, 6), pad=(1, 1), pixels=(7, 41))
+    assert torch.equal(part, dx.reshape(-1, 4)[7:41]) and torch.equal(apart, ax.reshape(-1, 4)[7:41])
+    dw, _ = orc.conv2d_wgrad(dY, X, (3, 2), pad=(1, 1))
+    part, _ = orc.conv2d_wgrad(dY, X, (3, 2), pad=(1, 1), filters=(1, 3))
+    assert torch.equal(part, dw[1:3])
