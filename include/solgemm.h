@@ -188,6 +188,29 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
                             const void* Cin, const void* bias, void* Y, void* cuda_stream);
 
 /*
+ * sg_conv2d_dgrad / sg_conv2d_wgrad: the gradients of sg_conv2d_fprop with respect to its input and its filter
+ * (paper: conv2d_dgrad(...), conv2d_wgrad(...), Appendix A.1 operator list).  `desc` describes the FORWARD problem
+ * (N,H,W,C input, K filters of R x S, pads, strides, dilations); P, Q are its output extents.
+ *   dgrad:  dX[n,h,w,c] = alpha * sum_{k,r,s} dY[n,p,q,k] * Wf[k,r,s,c]   over the (p,r), (q,s) with
+ *           p*stride_h - pad_h + r*dil_h == h and q*stride_w - pad_w + s*dil_w == w,       + beta * Cin[n,h,w,c]
+ *   wgrad:  dW[k,r,s,c] = alpha * sum_{n,p,q} dY[n,p,q,k] * X[n, p*stride_h - pad_h + r*dil_h, q*stride_w - pad_w + s*dil_w, c]
+ *           (taps outside the image contribute 0)                                         + beta * Cin[k,r,s,c]
+ *   dY   device, in_dtype (bf16 or fp16), [N,P,Q,K]        Wf  device, in_dtype, [K,R,S,C]       X  device, in_dtype, [N,H,W,C]
+ *   Cin  device, out_dtype, the output's shape; may be NULL when beta == 0
+ *   dX   device, out_dtype, [N,H,W,C], written in full     dW  device, out_dtype, [K,R,S,C], written in full
+ * Both run as implicit GEMMs in the forward kernel: dgrad contracts over (tap, k) with the filter read C-contiguous
+ * and its taps mirrored; wgrad is one product per tap, dY^T (K x NPQ) times the tap-shifted X (NPQ x C), whose long
+ * contraction is cut into K ranges through the scratch of sg_set_scratch when one is lent (few output tiles).
+ * desc->epi must be SG_EPI_NONE.  K and C must span multiples of 16 bytes in both types.
+ * SG_ERR_UNSUPPORTED: dgrad with a stride other than 1 or with pad > dil*(filter-1); 8-bit inputs.
+ * Empty outputs return SG_OK without a launch; an empty sum (no output pixels) gives beta * Cin.
+ */
+sg_status_t sg_conv2d_dgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* Wf, const void* Cin,
+                            void* dX, void* cuda_stream);
+sg_status_t sg_conv2d_wgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* X, const void* Cin,
+                            void* dW, void* cuda_stream);
+
+/*
  * Extended epilogue chain: the remaining built-ins of the DSL's `>>` chain (Table 1c; Appendix A.1
  * broadcast_op and fusion_op: per_row_scale, per_col_scale / per_channel_scale, column_broadcast,
  * scale(alpha=), aux_store, aux_load).  The DSL lets these follow one another in any order; this library

@@ -296,6 +296,18 @@ struct Shape {
 // (wide two-CTA tiles move the fewest operand bytes per FLOP; narrow tiles are bound by shared-memory
 // and L2 reads, not by the tensor pipe).  Two-CTA tiles pay a fixed cluster set-up cost, so they are
 // used only when the K loop is long and there is at least one full wave of them.
+// Modelled cost of sharing one tile's K loop between ks work items through the scratch (us): every part parks its
+// partial sums and finishes a share of the columns from the other parts' (measured: conv weight gradient and
+// skinny long-K products).
+inline double ksplit_exchange_us(int64_t ks) { return ks > 1 ? 6.0 + 0.5 * static_cast<double>(ks - 1) : 0.0; }
+constexpr double kUsPerKBlock = 0.25;      // one 64-deep k-block of a 128 x 256 tile per SM
+
+bool ksplit_allowed(const DeviceState& d) {
+    static const int env_k = getenv("SG_TAIL_KSPLIT") ? atoi(getenv("SG_TAIL_KSPLIT")) : -1;
+    const int tail_mode = g_tune_tail.load();
+    return d.scratch != nullptr && tail_mode != 0 && tail_mode != 1 && env_k != 0;
+}
+
 Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N,
                    int64_t K, int min_b_rows = 1) {
     const int force_bn = g_tune_tile_n.load();
@@ -307,7 +319,15 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
         for (int64_t r : rows_per_problem) tiles += ((r + tile_m - 1) / tile_m) * ((N + bn - 1) / bn);
         return tiles * batch_mult;
     };
-    const bool pair_worthwhile = K >= 1024 && d.max_pairs > 0 && tiles_for(256, 256) >= d.max_pairs;
+    int64_t max_rows = 0;
+    for (int64_t r : rows_per_problem) max_rows = r > max_rows ? r : max_rows;
+    const int64_t num_kb = (K + 63) / 64;
+    const bool can_split = ksplit_allowed(d) && num_kb >= 2;
+    const bool full_wave_of_pairs = d.max_pairs > 0 && tiles_for(256, 256) >= d.max_pairs;
+    // pairs: for long K loops, when there is a whole wave of 256 x 256 tiles -- or, for problems with less than a wave
+    // of tiles whose K loop can be shared between SMs, when a pair's 256 rows are not mostly padding
+    const bool pair_only = K >= 1024 && full_wave_of_pairs;
+    const bool pair_possible = pair_only || (K >= 1024 && d.max_pairs > 0 && can_split && max_rows > 128);
     // Eight epilogue warps drain an accumulator twice as fast; that pays when the K loop is too short to hide
     // the epilogue (short K, heavy activations) and costs a little when it is long.
     static const int forced_ew = getenv("SG_EPI_WARPS") ? atoi(getenv("SG_EPI_WARPS")) : 0;   // experiments: 4 or 8
@@ -315,16 +335,30 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
     Shape best{256, false, epi_warps};
     double best_cost = 1e300;
     for (int pi = 0; pi < 2; ++pi) {
-        if (force_pair >= 0 ? pi != force_pair : (pi == 1) != pair_worthwhile) continue;
+        if (force_pair >= 0 ? pi != force_pair : (pi == 1 ? !pair_possible : pair_only)) continue;
         for (int bi = 0; bi < 3; ++bi) {
             const int bn = bns[bi];
             if (force_bn > 0 && bn != force_bn) continue;
             if (bn / (pi ? 2 : 1) < min_b_rows) continue;       // an N-contiguous B is loaded in blocks of 64 rows
             const int64_t tiles = tiles_for(pi ? 256 : 128, bn);
             const int64_t slots = pi ? d.max_pairs : d.sm_count;
+            if (slots <= 0) continue;
             const int64_t waves = (tiles + slots - 1) / slots;
-            // the K-independent part of a tile (pipeline fill, epilogue drain) weighs more when K is short
-            const double cost = static_cast<double>(waves) * bn * (factor[pi][bi] + 96.0 / static_cast<double>(K > 64 ? K : 64));
+            // time of one k-block of a tile on its SM(s), and the K-independent part of a tile (pipeline fill,
+            // epilogue drain), which weighs more when K is short
+            const double t_kb = kUsPerKBlock * bn / 256.0 * factor[pi][bi];
+            const double t_fixed = kUsPerKBlock * bn / 256.0 * 96.0 / 64.0;
+            double cost = static_cast<double>(waves) * (t_kb * static_cast<double>(num_kb > 0 ? num_kb : 1) + t_fixed);
+            if (can_split && tiles * 2 <= slots) {
+                // less than half a wave: plan_tail may cut every tile's K loop into ranges run by different SMs
+                int64_t ks_max = slots / tiles;
+                if (ks_max > 16) ks_max = 16;
+                if (ks_max > num_kb) ks_max = num_kb;
+                for (int64_t ks = 2; ks <= ks_max; ++ks) {
+                    const double t = t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed + ksplit_exchange_us(ks);
+                    if (t < cost) cost = t;
+                }
+            }
             if (cost < best_cost) {
                 best_cost = cost;
                 best = Shape{bn, pi != 0, epi_warps};
@@ -363,11 +397,10 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
             best_split = (s.bn / forced >= 64 && s.bn / forced / (s.pair ? 2 : 1) >= min_b_rows) ? forced : 1;
             best = 0.9;
         }
-        // K ranges through the registered scratch: ksplit SM groups share one tail tile's K loop and the owner adds
-        // the helpers' fp32 partial tiles in its epilogue (this is also what serves skinny problems with a long K:
-        // when there is less than one wave of tiles, every tile is a "tail" tile).  Measured cost of the exchange:
-        // about 8 us for the dump, wait and first partial plus 1 us per further partial, whatever the tile's K; a
-        // k-block of a tile takes about 0.25 us.  A split is planned when it saves a fifth of the tail's time.
+        // K ranges through the registered scratch: ksplit SM groups share one tail tile's K loop; every part parks its
+        // fp32 partial sums and finishes a share of the tile's columns from all parts' sums (this is also what serves
+        // skinny problems with a long K: when there is less than one wave of tiles, every tile is a "tail" tile).
+        // A k-block of a tile takes about 0.25 us; a split is planned when it saves a fifth of the tail's time.
         if (d.scratch && forced_k != 0 && p->num_kb >= 2 && rem * 2 <= slots) {
             int64_t ks_max = slots / rem;
             if (ks_max > 16) ks_max = 16;
@@ -375,15 +408,15 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
             const size_t buf_bytes = static_cast<size_t>(s.pair ? 2 : 1) * 128 * s.bn * sizeof(float);
             size_t max_buffers = d.scratch_bytes > kScratchFlagBytes ? (d.scratch_bytes - kScratchFlagBytes) / buf_bytes : 0;
             if (max_buffers > static_cast<size_t>(kScratchMaxBuffers)) max_buffers = kScratchMaxBuffers;
-            while (ks_max >= 2 && static_cast<size_t>(rem * (ks_max - 1)) > max_buffers) --ks_max;
+            while (ks_max >= 2 && static_cast<size_t>(rem * ks_max) > max_buffers) --ks_max;      // every part parks a tile
             int64_t ks = 0;
             if (forced_k >= 2) {
                 ks = forced_k < ks_max ? forced_k : ks_max;
             } else if (rem <= kScratchMaxBuffers) {
-                const double t_tile = 0.25 * p->num_kb * best;      // us: the tail as planned so far (whole or sliced)
+                const double t_tile = kUsPerKBlock * p->num_kb * best;      // us: the tail as planned so far (whole or sliced)
                 double best_time = t_tile * 0.8;
                 for (int64_t k = 2; k <= ks_max; ++k) {
-                    const double t = 0.25 * p->num_kb / static_cast<double>(k) + 8.0 + 1.0 * static_cast<double>(k - 1);
+                    const double t = kUsPerKBlock * p->num_kb / static_cast<double>(k) + ksplit_exchange_us(k);
                     if (t < best_time) {
                         best_time = t;
                         ks = k;
@@ -1003,6 +1036,201 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
     if (st != SG_OK) return st;
     return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
 }
+
+}  // extern "C"
+
+namespace {
+
+// Checks shared by the two gradient entry points; P, Q are the forward output extents.
+sg_status_t grad_geometry(const sg_conv2d_desc_t* desc, const char* who, Checked* c, int64_t* P, int64_t* Q) {
+    if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
+    sg_status_t st = check_common(desc->in_dtype, desc->out_dtype, desc->epi, desc->alpha, desc->beta, desc->epi_arg0,
+                                  desc->epi_arg1, desc->reserved, c);
+    if (st != SG_OK) return st;
+    if (desc->epi != SG_EPI_NONE) return fail(SG_ERR_INVALID_ARG, "%s: epi must be SG_EPI_NONE", who);
+    if (c->in_fp8) return fail(SG_ERR_UNSUPPORTED, "%s: 8-bit inputs are not supported (an operand is read N-contiguous)", who);
+    if (desc->N < 0 || desc->H < 0 || desc->W < 0 || desc->C < 0 || desc->K < 0 || desc->R < 1 || desc->S < 1)
+        return fail(SG_ERR_INVALID_ARG, "%s: extents must be >= 0 and the filter at least 1x1", who);
+    if (desc->stride_h < 1 || desc->stride_w < 1 || desc->dil_h < 1 || desc->dil_w < 1 || desc->pad_h < 0 || desc->pad_w < 0)
+        return fail(SG_ERR_INVALID_ARG, "%s: strides and dilations must be >= 1, pads >= 0", who);
+    const int64_t span_h = desc->H + 2 * desc->pad_h - desc->dil_h * (desc->R - 1) - 1;
+    const int64_t span_w = desc->W + 2 * desc->pad_w - desc->dil_w * (desc->S - 1) - 1;
+    *P = span_h < 0 ? 0 : span_h / desc->stride_h + 1;
+    *Q = span_w < 0 ? 0 : span_w / desc->stride_w + 1;
+    if (desc->N * desc->H * desc->W > INT32_MAX || desc->N * *P * *Q > INT32_MAX || desc->C * desc->R * desc->S > INT32_MAX ||
+        desc->K * desc->R * desc->S > INT32_MAX || desc->H > 65535 || desc->W > 65535)
+        return fail(SG_ERR_UNSUPPORTED, "%s: extents too large", who);
+    if ((desc->R - 1) * desc->dil_h > 255 || (desc->S - 1) * desc->dil_w > 255 || desc->pad_h > 127 || desc->pad_w > 127 ||
+        desc->stride_h > 8 || desc->stride_w > 8)
+        return fail(SG_ERR_UNSUPPORTED, "%s: pad / filter extent / stride outside the im2col TMA limits", who);
+    return SG_OK;
+}
+
+}  // namespace
+
+extern "C" sg_status_t sg_conv2d_dgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* Wf, const void* Cin, void* dX,
+                                       void* cuda_stream) {
+    const char* who = "sg_conv2d_dgrad";
+    Checked c;
+    int64_t P = 0, Q = 0;
+    sg_status_t st = grad_geometry(desc, who, &c, &P, &Q);
+    if (st != SG_OK) return st;
+    if (desc->stride_h != 1 || desc->stride_w != 1)
+        return fail(SG_ERR_UNSUPPORTED, "%s: only stride 1 is implemented", who);
+    const int64_t pad_h = desc->dil_h * (desc->R - 1) - desc->pad_h, pad_w = desc->dil_w * (desc->S - 1) - desc->pad_w;
+    if (pad_h < 0 || pad_w < 0) return fail(SG_ERR_UNSUPPORTED, "%s: pad larger than the dilated filter extent", who);
+    if (pad_h > 127 || pad_w > 127) return fail(SG_ERR_UNSUPPORTED, "%s: filter extent outside the im2col TMA limits", who);
+    const int64_t Mg = desc->N * desc->H * desc->W;       // rows: input pixels
+    if (Mg == 0 || desc->C == 0) return SG_OK;
+    const int64_t Kg = desc->K * desc->R * desc->S;       // contraction: taps x output channels of the forward pass
+    if ((desc->K * c.esize_in) % 16 || (desc->C * c.esize_in) % 16 || (desc->C * c.esize_out) % 16)
+        return fail(SG_ERR_ALIGNMENT, "%s: K and C must span multiples of 16 bytes", who);
+    const bool empty = P == 0 || Q == 0 || desc->K == 0;  // nothing to sum: dX = beta * Cin
+    st = check_ptrs(dY, Wf, Cin, nullptr, dX, empty ? 0 : Kg, desc->beta, desc->epi, who);
+    if (st != SG_OK) return st;
+
+    DeviceState* d = nullptr;
+    st = device_state(&d);
+    if (st != SG_OK) return st;
+    Params p;
+    base_params(&p, *d, desc->alpha, desc->beta, desc->epi, 0.0f, 0.0f);
+    p.in_f16 = c.in_f16 ? 1 : 0;
+    p.bk_elems = c.bk;
+    Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->C, Kg, 64);
+    const int tile_m = s.pair ? 256 : 128;
+    p.mode = MODE_CONV;
+    p.b_mn_major = 1;
+    p.flip_taps = 1;
+    p.num_taps = static_cast<int32_t>(desc->R * desc->S);
+    p.M = static_cast<int32_t>(Mg);
+    p.N = static_cast<int32_t>(desc->C);
+    p.K = static_cast<int32_t>(Kg);
+    p.batch = 1;
+    p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
+    p.tiles_n = static_cast<int32_t>((desc->C + s.bn - 1) / s.bn);
+    p.cblocks = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
+    p.num_kb = empty ? 0 : p.num_taps * p.cblocks;
+    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p, 64);
+    p.C = desc->beta != 0.0f ? Cin : nullptr;
+    p.ldc = desc->C;
+    p.D = dX;
+    p.ldd = desc->C;
+    // the "image" the kernel walks is dY [N,P,Q,K]; its output pixels are the H x W pixels of dX
+    p.P = static_cast<int32_t>(desc->H);
+    p.Q = static_cast<int32_t>(desc->W);
+    p.stride_h = 1; p.stride_w = 1;
+    p.pad_h = static_cast<int32_t>(pad_h); p.pad_w = static_cast<int32_t>(pad_w);
+    p.dil_h = desc->dil_h; p.dil_w = desc->dil_w;
+    p.S = static_cast<int32_t>(desc->S);
+    st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, dX, desc->C, Mg, 1, desc->C, 0, c.f32_out ? 32 : 64, 32, "dX");
+    if (st != SG_OK) return st;
+    if (empty) {
+        p.tmA = p.tmD; p.tmB = p.tmD; p.tmB2 = p.tmD;
+    } else {
+        cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->K), static_cast<cuuint64_t>(Q), static_cast<cuuint64_t>(P),
+                              static_cast<cuuint64_t>(desc->N)};
+        const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
+        cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->K) * es, static_cast<cuuint64_t>(Q * desc->K) * es,
+                                 static_cast<cuuint64_t>(P * Q * desc->K) * es};
+        int lower[2] = {static_cast<int>(-pad_w), static_cast<int>(-pad_h)};
+        int upper[2] = {static_cast<int>(pad_w - (desc->S - 1) * desc->dil_w), static_cast<int>(pad_h - (desc->R - 1) * desc->dil_h)};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        CUresult r = g_encode_im2col(&p.tmA, c.tm_in, 4, const_cast<void*>(dY), dims, strides, lower, upper,
+                                     static_cast<cuuint32_t>(c.bk), 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(dY) failed with CUresult %d", static_cast<int>(r));
+        // filter [K][R*S][C] read with C contiguous: boxes of 64 c x 1 tap x 64 k
+        cuuint64_t fdims[3] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->R * desc->S),
+                               static_cast<cuuint64_t>(desc->K)};
+        cuuint64_t fstrides[2] = {static_cast<cuuint64_t>(desc->C) * es, static_cast<cuuint64_t>(desc->C * desc->R * desc->S) * es};
+        cuuint32_t box[3] = {64, 1, 64};
+        cuuint32_t e3[3] = {1, 1, 1};
+        r = g_encode_tiled(&p.tmB, c.tm_in, 3, const_cast<void*>(Wf), fdims, fstrides, box, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
+        p.tmB2 = p.tmB;
+    }
+    return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" sg_status_t sg_conv2d_wgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* X, const void* Cin, void* dW,
+                                       void* cuda_stream) {
+    const char* who = "sg_conv2d_wgrad";
+    Checked c;
+    int64_t P = 0, Q = 0;
+    sg_status_t st = grad_geometry(desc, who, &c, &P, &Q);
+    if (st != SG_OK) return st;
+    if (desc->K == 0 || desc->C == 0) return SG_OK;
+    const int64_t taps = desc->R * desc->S;
+    const int64_t pixels = desc->N * P * Q;               // contraction: output pixels of the forward pass
+    if ((desc->K * c.esize_in) % 16 || (desc->C * c.esize_in) % 16 || (desc->C * c.esize_out) % 16)
+        return fail(SG_ERR_ALIGNMENT, "%s: K and C must span multiples of 16 bytes", who);
+    if (desc->pad_h - (desc->R - 1) * desc->dil_h < -128 || desc->pad_w - (desc->S - 1) * desc->dil_w < -128)
+        return fail(SG_ERR_UNSUPPORTED, "%s: filter extent outside the im2col TMA limits", who);
+    st = check_ptrs(dY, X, Cin, nullptr, dW, pixels, desc->beta, desc->epi, who);
+    if (st != SG_OK) return st;
+
+    DeviceState* d = nullptr;
+    st = device_state(&d);
+    if (st != SG_OK) return st;
+    Params p;
+    base_params(&p, *d, desc->alpha, desc->beta, desc->epi, 0.0f, 0.0f);
+    p.in_f16 = c.in_f16 ? 1 : 0;
+    p.bk_elems = c.bk;
+    // one product per filter tap: dW[:, tap, :] (K x C) = dY^T (K x pixels) . X shifted by the tap (pixels x C)
+    Shape s = choose_shape(*d, std::vector<int64_t>{desc->K}, taps, desc->C, pixels, 64);
+    const int tile_m = s.pair ? 256 : 128;
+    p.mode = MODE_WGRAD;
+    p.a_mn_major = 1;
+    p.b_mn_major = 1;
+    p.num_taps = static_cast<int32_t>(taps);
+    p.M = static_cast<int32_t>(desc->K);
+    p.N = static_cast<int32_t>(desc->C);
+    p.K = static_cast<int32_t>(pixels);
+    p.batch = static_cast<int32_t>(taps);
+    p.tiles_m = static_cast<int32_t>((desc->K + tile_m - 1) / tile_m);
+    p.tiles_n = static_cast<int32_t>((desc->C + s.bn - 1) / s.bn);
+    p.num_kb = static_cast<int32_t>((pixels + 63) / 64);
+    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n * taps, &p, 64);
+    p.C = desc->beta != 0.0f ? Cin : nullptr;
+    p.ldc = taps * desc->C;
+    p.strideC = desc->C;
+    p.D = dW;
+    p.ldd = taps * desc->C;
+    p.strideD = desc->C;
+    p.P = static_cast<int32_t>(P);
+    p.Q = static_cast<int32_t>(Q);
+    p.stride_h = desc->stride_h; p.stride_w = desc->stride_w;
+    p.pad_h = desc->pad_h; p.pad_w = desc->pad_w;
+    p.dil_h = desc->dil_h; p.dil_w = desc->dil_w;
+    p.S = static_cast<int32_t>(desc->S);
+    st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, dW, desc->C, desc->K, taps, taps * desc->C, desc->C,
+                        c.f32_out ? 32 : 64, 32, "dW");
+    if (st != SG_OK) return st;
+    if (pixels == 0) {
+        p.tmA = p.tmD; p.tmB = p.tmD; p.tmB2 = p.tmD;
+    } else {
+        st = make_tiled_map(&p.tmA, c.tm_in, c.esize_in, dY, desc->K, pixels, 1, desc->K, 0, 64, 64, "dY");
+        if (st != SG_OK) return st;
+        cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->W), static_cast<cuuint64_t>(desc->H),
+                              static_cast<cuuint64_t>(desc->N)};
+        const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
+        cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->C) * es, static_cast<cuuint64_t>(desc->W * desc->C) * es,
+                                 static_cast<cuuint64_t>(desc->H * desc->W * desc->C) * es};
+        int lower[2] = {-desc->pad_w, -desc->pad_h};
+        int upper[2] = {static_cast<int>(desc->pad_w - (desc->S - 1) * desc->dil_w),
+                        static_cast<int>(desc->pad_h - (desc->R - 1) * desc->dil_h)};
+        cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(desc->stride_w), static_cast<cuuint32_t>(desc->stride_h), 1};
+        CUresult r = g_encode_im2col(&p.tmB, c.tm_in, 4, const_cast<void*>(X), dims, strides, lower, upper, 64, 64, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(X) failed with CUresult %d", static_cast<int>(r));
+        p.tmB2 = p.tmB;
+    }
+    return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" {
 
 sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* out, void* cuda_stream) {
     if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");

@@ -21,7 +21,7 @@
 
 namespace sg {
 
-enum : int32_t { MODE_DENSE = 0, MODE_GROUPED = 1, MODE_CONV = 2 };
+enum : int32_t { MODE_DENSE = 0, MODE_GROUPED = 1, MODE_CONV = 2, MODE_WGRAD = 3 };
 enum : int32_t { EPI_NONE = 0, EPI_BIAS = 1, EPI_RELU = 2, EPI_GELU = 3, EPI_SILU = 4, EPI_SIGMOID = 5, EPI_TANH = 6,
                  EPI_MISH = 7, EPI_HARDSWISH = 8, EPI_LEAKY_RELU = 9, EPI_ELU = 10, EPI_CLIP = 11 };
 
@@ -62,9 +62,9 @@ struct alignas(64) Params {
     FastDiv div_band_m;                 // by band_m (rows of every band but a shorter last one)
     FastDiv div_pq, div_q;              // conv: by P * Q and by Q
     int32_t ksplit;                     // > 1: tail tiles are cut into this many K ranges instead (split is then 1)
-    int32_t sk_arrivals;                // warp arrivals that complete one helper's partial tile (epilogue warps x CTAs)
-    float* sk_partials;                 // K-split scratch: [tail tile][helper][CTA of the tile][128 rows][BN] fp32
-    uint32_t* sk_flags;                 // K-split scratch: [buffer] arrival counters, then [tail tile] consumed counters
+    int32_t sk_arrivals;                // warp arrivals that complete one part's parked tile (epilogue warps x CTAs)
+    float* sk_partials;                 // K-split scratch: [tail tile][part][CTA of the tile][128 rows][BN] fp32
+    uint32_t* sk_flags;                 // K-split scratch: [tail tile][part] arrival counters, then [tail tile] done counters
     int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
     float alpha, beta;
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
@@ -74,6 +74,8 @@ struct alignas(64) Params {
     int32_t bk_elems;                   // elements of K per 128-byte stage row: 64 (16-bit) or 128 (8-bit)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
+    int32_t flip_taps;                  // conv (data gradient): the filter tap of B is RS - 1 - (tap of A)
+    int32_t num_taps;                   // conv: R * S
     // extended epilogue chain (all optional; ex_any = 1 when any of them is in use; dense and conv modes only):
     //   t = alpha acc * row_scale[i] * col_scale[j] + beta C + bias[j] + row_bias[i];  aux_store[i][j] = t;
     //   D = post_scale * act(t) + aux_load[i][j]
@@ -131,7 +133,7 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t b, bool f16) {
 struct Tile {
     int m0, n0, b, rows, width;   // first row / column, problem index, valid rows of the problem, tile width in columns
     int kb0, kb1;                 // k-blocks [kb0, kb1) this work item contracts (the whole K unless the tile is K-split)
-    int part, nparts, tail;       // K-split: part 0 owns (finishes) the tile, parts 1.. help; index of the tail tile
+    int part, nparts, tail;       // K-split: this item is part `part` of `nparts` sharing the tile's K range; index of the tail tile
 };
 
 // Tile r of one problem -> (tile row, tile column).  Tiles are walked in horizontal bands of band_m tile
@@ -161,7 +163,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
     if (t >= p.split_begin) {
         const int u = t - p.split_begin;
         if (p.ksplit > 1) {
-            // the tile's K range is shared by ksplit work items: part 0 owns the tile, the others help
+            // the tile's K range is shared by ksplit work items
             ti.nparts = p.ksplit;
             ti.tail = u / p.ksplit;
             ti.part = u - ti.tail * p.ksplit;
@@ -449,7 +451,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     // on global memory is read and written: wait for the previous kernel, then let the next one start setting up.
     grid_dependency_wait();
     grid_launch_dependents();
-    if (threadIdx.x == 0) SG_STAMP(16);
 
     const int num_kb = p.num_kb;
     const int first_tile = blockIdx.x / kCtas;
@@ -465,7 +466,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
                 Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
-                if (t == first_tile) SG_STAMP(17);
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
                 const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
                 const int nb0 = ti.n0 + static_cast<int>(cta_rank) * b_rows;
@@ -504,9 +504,20 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     c_r = c_tap / p.S;
                     c_s = c_tap - c_r * p.S;
                 }
+                // weight gradient: the problem index is the filter tap, the contraction runs over output pixels;
+                // (w_n, w_p, w_q) is the first pixel of the current k-block
+                int w_n = 0, w_p = 0, w_q = 0;
+                if (p.mode == MODE_WGRAD) {
+                    c_r = ti.b / p.S;
+                    c_s = ti.b - c_r * p.S;
+                    const int pix = ti.kb0 * Cfg::BK;
+                    w_n = fast_div(pix, p.div_pq);
+                    const int rem = pix - w_n * (p.P * p.Q);
+                    w_p = fast_div(rem, p.div_q);
+                    w_q = rem - w_p * p.Q;
+                }
                 for (int kb = ti.kb0; kb < ti.kb1; ++kb) {
                     if (!wait_bar(empty_bar(stage), phase ^ 1u, p, ROLE_PRODUCER, t, stage)) { ok = false; break; }
-                    if (t == first_tile && kb == ti.kb0) SG_STAMP(18);
                     const uint32_t a_dst = smem_base + stage * Cfg::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + Cfg::A_BYTES;
                     uint32_t fb = full_bar(stage);
@@ -516,11 +527,33 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         const int c0 = c_cb * bk_elems;
                         tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(c_s * p.dil_w),
                                                   static_cast<uint16_t>(c_r * p.dil_h));
-                        tma_load_3d<kPair>(b_dst, mapB, fb, c0, c_tap, nb0);
+                        if (p.b_mn_major) {
+                            // data gradient: the filter [k][tap][c] is read with c contiguous, 64 k x 64 c per box
+                            const int tap_b = p.flip_taps ? p.num_taps - 1 - c_tap : c_tap;
+                            for (int j = 0; j < b_rows / 64; ++j)
+                                tma_load_3d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, tap_b, c0);
+                        } else {
+                            tma_load_3d<kPair>(b_dst, mapB, fb, c0, c_tap, nb0);
+                        }
                         if (++c_cb == p.cblocks) {
                             c_cb = 0;
                             ++c_tap;
                             if (++c_s == p.S) { c_s = 0; ++c_r; }
+                        }
+                    } else if (p.mode == MODE_WGRAD) {
+                        // A = dY^T: [pixels][filters] read with the filter index contiguous; B = the 64 pixels of
+                        // this k-block shifted by the tap, 64 channels per box (im2col addressing)
+#pragma unroll
+                        for (int j = 0; j < Cfg::BM / 64; ++j)
+                            tma_load_3d<kPair>(a_dst + j * 8192, mapA, fb, m0 + j * 64, kb * Cfg::BK, 0);
+                        for (int j = 0; j < b_rows / 64; ++j)
+                            tma_load_im2col_4d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, w_q * p.stride_w - p.pad_w,
+                                                      w_p * p.stride_h - p.pad_h, w_n, static_cast<uint16_t>(c_s * p.dil_w),
+                                                      static_cast<uint16_t>(c_r * p.dil_h));
+                        w_q += Cfg::BK;
+                        while (w_q >= p.Q) {
+                            w_q -= p.Q;
+                            if (++w_p == p.P) { w_p = 0; ++w_n; }
                         }
                     } else {
                         if (p.a_mn_major) {
@@ -672,7 +705,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (!done) { ok = false; break; }
                 tc_fence_after_sync();
                 if (warp == 2 && lane == 0 && t == first_tile) SG_STAMP(7);
-                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(19);
             }
             const int ncols = min(ti.width, p.N - n0);
             const int nchunks = (ncols + CH - 1) / CH;
@@ -680,8 +712,16 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
             const int row = row0 + lane;
 
-            bool sk_waited = false;
-            if (num_kb > 0 && half >= nchunks) {
+            // K-split tile: the tile's K range is shared by nparts work items.  Every part parks its raw fp32 sums of
+            // the column chunks it does not finish in the scratch (pass 0), then finishes the chunks it owns
+            // from its own accumulator plus the other parts' parked sums
+            // (pass 1), so the exchange is spread over all parts instead of serialised in one.  The unit of ownership
+            // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
+            const bool ksplit_tile = ti.nparts > 1;
+            // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
+            auto owned = [&](int c) { return (c + (BN / CH) * (q * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
+            const int passes = ksplit_tile ? 2 : 1;
+            if (num_kb > 0 && half >= nchunks && !ksplit_tile) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
                 tc_fence_before_sync();
                 __syncwarp();
@@ -691,7 +731,30 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
             }
 #pragma unroll 1
+            for (int pass = 0; pass < passes && ok; ++pass) {
+            if (ksplit_tile && pass == 1) {
+                // this warp's share of the parked sums is complete: publish it, then wait for the other parts
+                __threadfence();
+                __syncwarp();
+                uint32_t okw = 1;
+                if (lane == 0) {
+                    uint32_t* flags = p.sk_flags + ti.tail * p.ksplit;
+                    atomicAdd(flags + ti.part, 1u);
+                    bool owns = false;
+                    for (int c = half; c < nchunks; c += kStep) owns = owns || owned(c);
+                    if (owns && rows_live) {
+                        for (int h = 0; h < ti.nparts && okw; ++h)
+                            if (h != ti.part)
+                                okw = wait_counter(flags + h, static_cast<uint32_t>(p.sk_arrivals), p, t) ? 1u : 0u;
+                    }
+                }
+                okw = __shfl_sync(0xFFFFFFFFu, okw, 0);
+                if (!okw) { ok = false; break; }
+                __threadfence();
+            }
+#pragma unroll 1
             for (int c = half; c < nchunks; c += kStep) {
+                if (ksplit_tile && owned(c) != (pass == 1)) continue;
                 float v[CH];
                 if (num_kb > 0) {
                     uint32_t r0[32];
@@ -700,7 +763,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         uint32_t r1[32];
                         tmem_ld_32x32(t_row + c * CH + 32, r1);
                         tmem_ld_wait();
-                        if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(20 + 4 * (c / kStep > 0 ? 1 : 0));
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             v[i] = __uint_as_float(r0[i]);
@@ -711,7 +773,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
                     }
-                    if (c + kStep >= nchunks) {
+                    if (c + kStep >= nchunks && !ksplit_tile) {
                         // this warp has read its last columns of the accumulator: hand its share back to the MMA warp
                         tc_fence_before_sync();
                         __syncwarp();
@@ -726,37 +788,25 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 if (!rows_live) continue;       // nothing of this warp's 32 rows exists (ragged last tile)
 
-                if (ti.nparts > 1) {
-                    // K-split tail tile.  Helpers park their raw fp32 partial sums in the scratch; the owner adds
-                    // them to its own (always in the order own + helper 1 + helper 2 ..., so results are reproducible).
-                    // Scratch layout of one CTA's partial tile: [group of 4 columns][row] float4, so that the 32
+                if (ksplit_tile) {
+                    // Scratch layout of one CTA's parked tile: [group of 4 columns][row] float4, so that the 32
                     // lanes (= rows) of a warp touch 512 contiguous bytes per access.
                     const size_t tile_elems = static_cast<size_t>(Cfg::BM) * BN;
                     const size_t my_off = static_cast<size_t>(cta_rank) * tile_elems +
                                           (static_cast<size_t>(c * (CH / 4)) * Cfg::BM + static_cast<size_t>(q * 32 + lane)) * 4;
-                    if (ti.part > 0) {
-                        float* pb = p.sk_partials +
-                                    static_cast<size_t>(ti.tail * (p.ksplit - 1) + ti.part - 1) * kCtas * tile_elems + my_off;
+                    float* tile_bufs = p.sk_partials + static_cast<size_t>(ti.tail) * p.ksplit * kCtas * tile_elems;
+                    if (pass == 0) {
+                        float* pb = tile_bufs + static_cast<size_t>(ti.part) * kCtas * tile_elems + my_off;
 #pragma unroll
                         for (int i = 0; i < CH; i += 4)
                             __stcg(reinterpret_cast<float4*>(pb + static_cast<size_t>(i) * Cfg::BM),
                                    make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
                         continue;
                     }
-                    if (!sk_waited) {
-                        uint32_t okw = 1;
-                        if (lane == 0) {
-                            for (int h = 0; h < ti.nparts - 1 && okw; ++h)
-                                okw = wait_counter(p.sk_flags + ti.tail * (p.ksplit - 1) + h, static_cast<uint32_t>(p.sk_arrivals), p, t) ? 1u : 0u;
-                        }
-                        okw = __shfl_sync(0xFFFFFFFFu, okw, 0);
-                        if (!okw) { ok = false; break; }
-                        __threadfence();
-                        sk_waited = true;
-                    }
-                    for (int h = 0; h < ti.nparts - 1; ++h) {
-                        const float* pb = p.sk_partials +
-                                          static_cast<size_t>(ti.tail * (p.ksplit - 1) + h) * kCtas * tile_elems + my_off;
+                    // own sums first, then the other parts' in increasing order: reproducible for a given plan
+                    for (int h = 0; h < ti.nparts; ++h) {
+                        if (h == ti.part) continue;
+                        const float* pb = tile_bufs + static_cast<size_t>(h) * kCtas * tile_elems + my_off;
 #pragma unroll
                         for (int i = 0; i < CH; i += 4) {
                             const float4 x = __ldcg(reinterpret_cast<const float4*>(pb + static_cast<size_t>(i) * Cfg::BM));
@@ -912,7 +962,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         }
                     }
                 }
-                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(21 + 4 * (c / kStep > 0 ? 1 : 0));
 
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
                 // the last, partial chunk is therefore written with plain stores so nothing beyond column N changes.
@@ -941,7 +990,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 ++chunk_ctr;
                 if (lane == 0) tma_store_wait_read<Cfg::STAGING_BUFS - 1>();   // the store that last read this block is done
                 __syncwarp();
-                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(22 + 4 * (c / kStep > 0 ? 1 : 0));
                 const uint32_t stg = smem_base + Cfg::OFF_STAGING + (ew * Cfg::STAGING_BUFS + sb) * 4096u;
                 const uint32_t row_addr = stg + lane * 128u;
 #pragma unroll
@@ -967,25 +1015,25 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     tma_store_commit();
                 }
 #endif
-                if (warp == 2 && lane == 0 && t + tile_step >= p.num_tiles) SG_STAMP(23 + 4 * (c / kStep > 0 ? 1 : 0));
             }
             if (!ok) break;
-            if (ti.nparts > 1) {
-                // K-split bookkeeping, once per warp and tile whether or not the warp had columns or live rows
+            }   // passes
+            if (!ok) break;
+            if (ksplit_tile) {
+                // the accumulator was read in both passes: hand it back now; then count this warp as done with the
+                // tile's scratch -- the last warp of all parts leaves every counter at zero for the next launch
+                tc_fence_before_sync();
                 __threadfence();
                 __syncwarp();
                 if (lane == 0) {
-                    uint32_t* flags = p.sk_flags + ti.tail * (p.ksplit - 1);
-                    if (ti.part > 0) {
-                        atomicAdd(flags + ti.part - 1, 1u);                      // this warp's share of the partial is visible
-                    } else {
-                        uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
-                        if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals) - 1u) {
-                            // last warp of the owner: every partial has been read; leave the counters at zero for the next launch
-                            for (int h = 0; h < ti.nparts - 1; ++h) flags[h] = 0u;
-                            *consumed = 0u;
-                            __threadfence();
-                        }
+                    if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
+                    else mbar_arrive(tempty_remote[acc]);
+                    uint32_t* flags = p.sk_flags + ti.tail * p.ksplit;
+                    uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
+                    if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals * ti.nparts) - 1u) {
+                        for (int h = 0; h < ti.nparts; ++h) flags[h] = 0u;
+                        *consumed = 0u;
+                        __threadfence();
                     }
                 }
             }

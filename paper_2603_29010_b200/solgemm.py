@@ -36,6 +36,7 @@ DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop", "sg_gemm_ex", "sg_conv2d_fprop_ex",
+            "sg_conv2d_dgrad", "sg_conv2d_wgrad",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
             "sg_last_kernel_clock", "sg_transpose"]
@@ -98,6 +99,10 @@ _lib.sg_gemm_ex.restype = ctypes.c_int
 _lib.sg_gemm_ex.argtypes = [ctypes.POINTER(GemmDesc), ctypes.POINTER(EpilogueEx), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_conv2d_fprop_ex.restype = ctypes.c_int
 _lib.sg_conv2d_fprop_ex.argtypes = [ctypes.POINTER(Conv2dDesc), ctypes.POINTER(EpilogueEx), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_conv2d_dgrad.restype = ctypes.c_int
+_lib.sg_conv2d_dgrad.argtypes = [ctypes.POINTER(Conv2dDesc), _vp, _vp, _vp, _vp, _vp]
+_lib.sg_conv2d_wgrad.restype = ctypes.c_int
+_lib.sg_conv2d_wgrad.argtypes = [ctypes.POINTER(Conv2dDesc), _vp, _vp, _vp, _vp, _vp]
 _lib.sg_batched_gemm.restype = ctypes.c_int
 _lib.sg_batched_gemm.argtypes = [ctypes.POINTER(GemmDesc), _i64, _i64, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_grouped_gemm_workspace_size.restype = ctypes.c_int
@@ -367,6 +372,44 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
                                        _ptr(out), _stream(stream)))
         return out
     _check(_lib.sg_conv2d_fprop(ctypes.byref(desc), _ptr(X), _ptr(Wf), _ptr(Cin), _ptr(bias), _ptr(out), _stream(stream)))
+    return out
+
+
+def conv2d_dgrad(dY: torch.Tensor, Wf: torch.Tensor, hw, *, pad=(0, 0), stride=(1, 1), dil=(1, 1), Cin=None, out=None,
+                 out_dtype=torch.bfloat16, alpha=1.0, beta=0.0, stream=None) -> torch.Tensor:
+    """Gradient of ``conv2d_fprop`` with respect to its input through ``sg_conv2d_dgrad``: ``dY`` [N,P,Q,K],
+    ``Wf`` [K,R,S,C] -> [N,H,W,C] with ``hw = (H, W)`` of the forward input."""
+    if dY.dim() != 4 or Wf.dim() != 4 or not dY.is_contiguous() or not Wf.is_contiguous():
+        raise ValueError("dY (NPQK) and Wf (KRSC) must be contiguous 4-D tensors")
+    N, K = dY.shape[0], dY.shape[3]
+    Kw, R, S, C = Wf.shape
+    if K != Kw:
+        raise ValueError("dY and Wf disagree on K")
+    H, W = hw
+    ensure_scratch()
+    if out is None:
+        out = torch.empty((N, H, W, C), dtype=out_dtype, device=dY.device)
+    desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], DTYPES[dY.dtype],
+                      DTYPES[out.dtype], float(alpha), float(beta), EPILOGUES["none"], 0.0, 0.0, 0)
+    _check(_lib.sg_conv2d_dgrad(ctypes.byref(desc), _ptr(dY), _ptr(Wf), _ptr(Cin), _ptr(out), _stream(stream)))
+    return out
+
+
+def conv2d_wgrad(dY: torch.Tensor, X: torch.Tensor, rs, *, pad=(0, 0), stride=(1, 1), dil=(1, 1), Cin=None, out=None,
+                 out_dtype=torch.float32, alpha=1.0, beta=0.0, stream=None) -> torch.Tensor:
+    """Gradient of ``conv2d_fprop`` with respect to its filter through ``sg_conv2d_wgrad``: ``dY`` [N,P,Q,K],
+    ``X`` [N,H,W,C] -> [K,R,S,C] with ``rs = (R, S)``."""
+    if dY.dim() != 4 or X.dim() != 4 or not dY.is_contiguous() or not X.is_contiguous():
+        raise ValueError("dY (NPQK) and X (NHWC) must be contiguous 4-D tensors")
+    N, H, W, C = X.shape
+    K = dY.shape[3]
+    R, S = rs
+    ensure_scratch()
+    if out is None:
+        out = torch.empty((K, R, S, C), dtype=out_dtype, device=dY.device)
+    desc = Conv2dDesc(N, H, W, C, K, R, S, pad[0], pad[1], stride[0], stride[1], dil[0], dil[1], DTYPES[dY.dtype],
+                      DTYPES[out.dtype], float(alpha), float(beta), EPILOGUES["none"], 0.0, 0.0, 0)
+    _check(_lib.sg_conv2d_wgrad(ctypes.byref(desc), _ptr(dY), _ptr(X), _ptr(Cin), _ptr(out), _stream(stream)))
     return out
 
 
