@@ -64,7 +64,7 @@ struct alignas(64) Params {
     int32_t ksplit;                     // > 1: tail tiles are cut into this many K ranges instead (split is then 1)
     int32_t sk_arrivals;                // warp arrivals that complete one part's parked tile (epilogue warps x CTAs)
     float* sk_partials;                 // K-split scratch: [tail tile][part][CTA of the tile][128 rows][BN] fp32
-    uint32_t* sk_flags;                 // K-split scratch: [tail tile][part] arrival counters, then [tail tile] done counters
+    uint32_t* sk_flags;                 // K-split scratch: [tail tile] arrival counters, then [tail tile] done counters
     int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
     float alpha, beta;
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
@@ -360,7 +360,7 @@ struct Config {
     static constexpr int OFF_BIAS = OFF_STAGING + STAGING_BYTES;
     static constexpr int BIAS_SLOTS = BN / CHUNK_STEP < 64 ? 64 : BN / CHUNK_STEP;   // per warp: bf16 bias of its chunks
     static constexpr int OFF_BAR = OFF_BIAS + EPI_WARPS * BIAS_SLOTS * 2;
-    static constexpr int NUM_BARS = 2 * STAGES + 5;                // full, empty, tmem_full[2], tmem_empty[2], drain
+    static constexpr int NUM_BARS = 2 * STAGES + 5 + EPI_WARPS;    // full, empty, tmem_full[2], tmem_empty[2], drain, K-split fetch per warp
     static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
     static_assert(SMEM_BYTES <= 227 * 1024, "configuration exceeds the shared memory of one CTA");
@@ -389,6 +389,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
     const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 4);
+    auto fetch_bar = [&](int w) { return bar_base + 8u * (2 * STAGES + 5 + w); };
     const uint32_t tmem_slot = bar_base + 8u * Cfg::NUM_BARS;
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem + Cfg::OFF_BAR + 8 * Cfg::NUM_BARS);
 
@@ -426,6 +427,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             mbar_init(tempty_bar(a), Cfg::EPI_WARPS * kCtas);
         }
         mbar_init(drain_bar, 1);
+        for (int w = 0; w < Cfg::EPI_WARPS; ++w) mbar_init(fetch_bar(w), 1);
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -647,6 +649,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         const int half = ew >> 2;             // which chunks of a tile this warp takes (always 0 with four warps)
         constexpr int kStep = Cfg::CHUNK_STEP;
         uint32_t chunk_ctr = 0;
+        uint32_t fetch_phase = 0;             // phase of this warp's K-split fetch barrier
         uint16_t* bias_w = reinterpret_cast<uint16_t*>(smem + Cfg::OFF_BIAS) + ew * Cfg::BIAS_SLOTS;   // bf16 bias of its chunks
         constexpr int kMyBiasSlots = ((BN / CH + kStep - 1) / kStep) * CH;     // columns of the chunks one warp handles
         const bool has_bias = (p.mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
@@ -719,7 +722,23 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
             const bool ksplit_tile = ti.nparts > 1;
             // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
-            auto owned = [&](int c) { return (c + (BN / CH) * (q * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
+            auto owned_by = [&](int c, int qq) { return (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
+            auto owned = [&](int c) { return owned_by(c, q); };
+            // how many epilogue warps of this CTA finish at least one unit, and this warp's rank among them: the
+            // stage ring (idle by then) is divided between them as the landing zone of the other parts' sums
+            int fetch_owners = 0, fetch_rank = 0;
+            if (ksplit_tile) {
+                for (int w = 0; w < Cfg::EPI_WARPS; ++w) {
+                    const int qq = (w + 2) & 3;
+                    bool o = false;
+                    for (int c = w >> 2; c < nchunks; c += kStep) o = o || owned_by(c, qq);
+                    o = o && (ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + qq * 32 < ti.rows);
+                    if (o) {
+                        if (w < ew) ++fetch_rank;
+                        ++fetch_owners;
+                    }
+                }
+            }
             const int passes = ksplit_tile ? 2 : 1;
             if (num_kb > 0 && half >= nchunks && !ksplit_tile) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
@@ -734,23 +753,22 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int pass = 0; pass < passes && ok; ++pass) {
             if (ksplit_tile && pass == 1) {
                 // this warp's share of the parked sums is complete: publish it, then wait for the other parts
+                // (the readers fetch it with bulk copies, i.e. through the asynchronous proxy)
                 __threadfence();
+                fence_proxy_async_all();
                 __syncwarp();
                 uint32_t okw = 1;
+                bool owns = false;
+                for (int c = half; c < nchunks; c += kStep) owns = owns || owned(c);
+                owns = owns && rows_live;
                 if (lane == 0) {
-                    uint32_t* flags = p.sk_flags + ti.tail * p.ksplit;
-                    atomicAdd(flags + ti.part, 1u);
-                    bool owns = false;
-                    for (int c = half; c < nchunks; c += kStep) owns = owns || owned(c);
-                    if (owns && rows_live) {
-                        for (int h = 0; h < ti.nparts && okw; ++h)
-                            if (h != ti.part)
-                                okw = wait_counter(flags + h, static_cast<uint32_t>(p.sk_arrivals), p, t) ? 1u : 0u;
-                    }
+                    uint32_t* arrived = p.sk_flags + ti.tail;       // one counter per tile: every warp of every part
+                    atomicAdd(arrived, 1u);
+                    if (owns) okw = wait_counter(arrived, static_cast<uint32_t>(p.sk_arrivals * ti.nparts), p, t) ? 1u : 0u;
                 }
                 okw = __shfl_sync(0xFFFFFFFFu, okw, 0);
                 if (!okw) { ok = false; break; }
-                __threadfence();
+                if (owns) __threadfence();      // the other parts' sums are read after their flags
             }
 #pragma unroll 1
             for (int c = half; c < nchunks; c += kStep) {
@@ -789,28 +807,83 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (!rows_live) continue;       // nothing of this warp's 32 rows exists (ragged last tile)
 
                 if (ksplit_tile) {
-                    // Scratch layout of one CTA's parked tile: [group of 4 columns][row] float4, so that the 32
-                    // lanes (= rows) of a warp touch 512 contiguous bytes per access.
+                    // Scratch layout of one CTA's parked tile: [chunk][lane quarter][group of 4 columns][32 rows] float4:
+                    // a unit (one warp's rows of one chunk) is one contiguous block of CH x 128 bytes, and the 32 lanes
+                    // (= rows) of a warp touch 512 contiguous bytes per access.
+                    constexpr uint32_t kUnitBytes = CH * 128u;
                     const size_t tile_elems = static_cast<size_t>(Cfg::BM) * BN;
-                    const size_t my_off = static_cast<size_t>(cta_rank) * tile_elems +
-                                          (static_cast<size_t>(c * (CH / 4)) * Cfg::BM + static_cast<size_t>(q * 32 + lane)) * 4;
+                    const size_t unit_off = static_cast<size_t>(cta_rank) * tile_elems +
+                                            static_cast<size_t>(c * 4 + q) * (kUnitBytes / 4);
                     float* tile_bufs = p.sk_partials + static_cast<size_t>(ti.tail) * p.ksplit * kCtas * tile_elems;
                     if (pass == 0) {
-                        float* pb = tile_bufs + static_cast<size_t>(ti.part) * kCtas * tile_elems + my_off;
+                        float* pb = tile_bufs + static_cast<size_t>(ti.part) * kCtas * tile_elems + unit_off + lane * 4;
 #pragma unroll
                         for (int i = 0; i < CH; i += 4)
-                            __stcg(reinterpret_cast<float4*>(pb + static_cast<size_t>(i) * Cfg::BM),
-                                   make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
+                            __stcg(reinterpret_cast<float4*>(pb + i * 32), make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]));
                         continue;
                     }
-                    // own sums first, then the other parts' in increasing order: reproducible for a given plan
-                    for (int h = 0; h < ti.nparts; ++h) {
-                        if (h == ti.part) continue;
-                        const float* pb = tile_bufs + static_cast<size_t>(h) * kCtas * tile_elems + my_off;
+                    // Own sums first, then the other parts' in increasing order: reproducible for a given plan.
+                    // The other parts' units are fetched with bulk copies, several at a time, into this warp's share
+                    // of the stage ring (idle by now: a K-split item is the last work of its CTA, its MMAs are done),
+                    // so the latency of the exchange is paid once per batch of parts rather than once per part.
+                    const uint32_t fetch_bytes = static_cast<uint32_t>(STAGES * Cfg::STAGE_BYTES) /
+                                                 static_cast<uint32_t>(fetch_owners > 0 ? fetch_owners : 1) / kUnitBytes * kUnitBytes;
+                    const int kBatch = static_cast<int>(fetch_bytes / kUnitBytes);
+                    const bool ring_idle = t + tile_step >= p.num_tiles;
+                    if (kEpiWarps == 4 && kBatch >= 2 && ring_idle) {    // (8-warp kernels serve short K: registers are scarce there)
+                        const uint32_t fetch_base = smem_base + static_cast<uint32_t>(fetch_rank) * fetch_bytes;
+                        int h = 0;
+                        while (h < ti.nparts && ok) {
+                            int n = 0;
+                            if (lane == 0) {
+                                fence_proxy_async_all();
+                                int hh = h;
+                                for (; hh < ti.nparts && n < kBatch; ++hh)
+                                    if (hh != ti.part) ++n;
+                                if (n > 0) {
+                                    mbar_arrive_expect_tx(fetch_bar(ew), static_cast<uint32_t>(n) * kUnitBytes);
+                                    int k = 0;
+                                    for (int g = h; g < hh; ++g) {
+                                        if (g == ti.part) continue;
+                                        bulk_load_1d(fetch_base + static_cast<uint32_t>(k) * kUnitBytes,
+                                                     tile_bufs + static_cast<size_t>(g) * kCtas * tile_elems + unit_off, kUnitBytes,
+                                                     fetch_bar(ew));
+                                        ++k;
+                                    }
+                                }
+                                h = hh;
+                            }
+                            n = __shfl_sync(0xFFFFFFFFu, n, 0);
+                            h = __shfl_sync(0xFFFFFFFFu, h, 0);
+                            if (n == 0) continue;
+                            uint32_t got = 1;
+                            if (lane == 0) got = wait_bar(fetch_bar(ew), fetch_phase, p, ROLE_EPILOGUE, t, 400 + ew) ? 1u : 0u;
+                            got = __shfl_sync(0xFFFFFFFFu, got, 0);
+                            if (!got) { ok = false; break; }
+                            fetch_phase ^= 1u;
+                            for (int k = 0; k < n; ++k) {
+                                const uint32_t ub = fetch_base + static_cast<uint32_t>(k) * kUnitBytes + lane * 16u;
 #pragma unroll
-                        for (int i = 0; i < CH; i += 4) {
-                            const float4 x = __ldcg(reinterpret_cast<const float4*>(pb + static_cast<size_t>(i) * Cfg::BM));
-                            v[i] += x.x; v[i + 1] += x.y; v[i + 2] += x.z; v[i + 3] += x.w;
+                                for (int i = 0; i < CH; i += 4) {
+                                    float4 x;
+                                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                                 : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
+                                                 : "r"(ub + static_cast<uint32_t>(i) * 128u));
+                                    v[i] += x.x; v[i + 1] += x.y; v[i + 2] += x.z; v[i + 3] += x.w;
+                                }
+                            }
+                            __syncwarp();      // every lane has read the batch before lane 0 refills the buffer
+                        }
+                        if (!ok) break;
+                    } else {
+                        for (int h = 0; h < ti.nparts; ++h) {
+                            if (h == ti.part) continue;
+                            const float* pb = tile_bufs + static_cast<size_t>(h) * kCtas * tile_elems + unit_off + lane * 4;
+#pragma unroll
+                            for (int i = 0; i < CH; i += 4) {
+                                const float4 x = __ldcg(reinterpret_cast<const float4*>(pb + i * 32));
+                                v[i] += x.x; v[i + 1] += x.y; v[i + 2] += x.z; v[i + 3] += x.w;
+                            }
                         }
                     }
                 }
@@ -1023,15 +1096,14 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 // the accumulator was read in both passes: hand it back now; then count this warp as done with the
                 // tile's scratch -- the last warp of all parts leaves every counter at zero for the next launch
                 tc_fence_before_sync();
-                __threadfence();
                 __syncwarp();
                 if (lane == 0) {
                     if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
                     else mbar_arrive(tempty_remote[acc]);
-                    uint32_t* flags = p.sk_flags + ti.tail * p.ksplit;
+                    uint32_t* arrived = p.sk_flags + ti.tail;
                     uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
                     if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals * ti.nparts) - 1u) {
-                        for (int h = 0; h < ti.nparts; ++h) flags[h] = 0u;
+                        *arrived = 0u;
                         *consumed = 0u;
                         __threadfence();
                     }

@@ -134,6 +134,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
             : "memory");
     }
 }
+// Untiled bulk copy global -> shared memory of this CTA, completing `bytes` on an mbarrier of this CTA.
+// Both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// Orders this thread's earlier generic-proxy accesses (all state spaces) before later asynchronous-proxy ones.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 // im2col 4-D load: coordinates {c, w, h, n} of the first base pixel, filter-tap offsets {w_off, h_off}.
 template <bool kPair>
 __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const void* tmap, uint32_t bar, int c, int w, int h,
