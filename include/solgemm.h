@@ -277,7 +277,9 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
  *   t_compute = flops / eff_peak, t_mem = bytes / eff_bandwidth, t_sol = max of the two;
  *   ai = flops / bytes, ridge = eff_peak / eff_bandwidth, compute_bound = ai > ridge.
  *   op                SG_OP_GEMM / SG_OP_BATCHED / SG_OP_GROUPED: desc is sg_gemm_desc_t;
- *                     SG_OP_CONV2D: desc is sg_conv2d_desc_t; SG_OP_TRANSPOSE: desc is sg_transpose_desc_t
+ *                     SG_OP_CONV2D, SG_OP_CONV2D_DGRAD, SG_OP_CONV2D_WGRAD: desc is sg_conv2d_desc_t (the forward
+ *                     problem; the gradients execute the same 2*NPQ*K*CRS FLOPs and move dY + Wf + dX, resp. dY + X + dW);
+ *                     SG_OP_TRANSPOSE: desc is sg_transpose_desc_t
  *                     (flops = 0; element sizes come from its dtypes, elem_bytes_* are ignored).
  *   batch_or_groups   batch count (BATCHED), group count (GROUPED), ignored otherwise.
  *   M_host            [groups] for GROUPED (desc->M ignored), else may be NULL.
@@ -295,7 +297,8 @@ typedef struct sg_sol {
     int32_t reserved;
 } sg_sol_t;
 
-typedef enum { SG_OP_GEMM = 0, SG_OP_BATCHED = 1, SG_OP_GROUPED = 2, SG_OP_CONV2D = 3, SG_OP_TRANSPOSE = 4 } sg_op_t;
+typedef enum { SG_OP_GEMM = 0, SG_OP_BATCHED = 1, SG_OP_GROUPED = 2, SG_OP_CONV2D = 3, SG_OP_TRANSPOSE = 4,
+               SG_OP_CONV2D_DGRAD = 5, SG_OP_CONV2D_WGRAD = 6 } sg_op_t;
 
 sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, const int64_t* M_host,
                          int32_t elem_bytes_in, int32_t elem_bytes_out, int32_t has_bias,

@@ -94,6 +94,8 @@ def lib() -> ctypes.CDLL:
         L.orc_conv_flops.argtypes = [vp]
         L.orc_conv_bytes.restype = i64
         L.orc_conv_bytes.argtypes = [vp, i64, i64, ci, ci]
+        L.orc_conv_grad_bytes.restype = i64
+        L.orc_conv_grad_bytes.argtypes = [vp, ci, i64, i64, ci]
         L.orc_sol_bound.restype = ci
         L.orc_sol_bound.argtypes = [i64, i64, vp, vp]
         _lib = L
@@ -439,6 +441,13 @@ def conv_bytes(N, H, W, C, K, R, S, pad=(0, 0), stride=(1, 1), dil=(1, 1), eb_in
                has_c=False, has_bias=False) -> int:
     d = _dims13(N, H, W, C, K, R, S, pad, stride, dil)
     return int(lib().orc_conv_bytes(_ptr(d), eb_in, eb_out, int(has_c), int(has_bias)))
+
+
+def conv_grad_bytes(which: str, N, H, W, C, K, R, S, pad=(0, 0), stride=(1, 1), dil=(1, 1), eb_in=2, eb_out=2,
+                    has_c: bool = False) -> int:
+    """Best-case bytes of ``which`` = "dgrad" (dY + Wf read, dX written) or "wgrad" (dY + X read, dW written)."""
+    d = _dims13(N, H, W, C, K, R, S, pad, stride, dil)
+    return int(lib().orc_conv_grad_bytes(_ptr(d), {"dgrad": 0, "wgrad": 1}[which], eb_in, eb_out, int(has_c)))
 
 
 def sol_bound(flops: int, bytes_: int, peak_flops: float, peak_bytes_per_s: float,

@@ -526,6 +526,19 @@ int64_t orc_conv_bytes(const int64_t* dims, int64_t eb_in, int64_t eb_out, int h
     return bytes;
 }
 
+/* Best-case bytes of the two gradients: which = 0 data gradient (reads dy and w, writes dx),
+ * which = 1 weight gradient (reads dy and x, writes dw); has_c adds one read of the written tensor. */
+int64_t orc_conv_grad_bytes(const int64_t* dims, int which, int64_t eb_in, int64_t eb_out, int has_c) {
+    int64_t P = orc_conv_out_extent(dims[1], dims[7], dims[11], dims[5], dims[9]);
+    int64_t Q = orc_conv_out_extent(dims[2], dims[8], dims[12], dims[6], dims[10]);
+    int64_t x = dims[0] * dims[1] * dims[2] * dims[3];
+    int64_t w = dims[4] * dims[5] * dims[6] * dims[3];
+    int64_t y = dims[0] * P * Q * dims[4];
+    int64_t rd = which == 0 ? y + w : y + x;
+    int64_t wr = which == 0 ? x : w;
+    return rd * eb_in + wr * eb_out * (has_c ? 2 : 1);
+}
+
 /*
  * hw = {peak_flops, peak_bytes_per_s, sm_clock, sm_clock_max, mem_clock, mem_clock_max}
  *      (a zero clock or zero max clock means "do not scale": ratio 1).

@@ -1319,7 +1319,7 @@ sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, 
             if (has_bias == 2) elems_in += g->N;
             elems_out = b * g->M * g->N * (reads_c ? 2 : 1);
         }
-    } else if (op == SG_OP_CONV2D) {
+    } else if (op == SG_OP_CONV2D || op == SG_OP_CONV2D_DGRAD || op == SG_OP_CONV2D_WGRAD) {
         const sg_conv2d_desc_t* cv = static_cast<const sg_conv2d_desc_t*>(desc);
         if (cv->N < 0 || cv->H < 0 || cv->W < 0 || cv->C < 0 || cv->K < 0 || cv->R < 1 || cv->S < 1 || cv->stride_h < 1 ||
             cv->stride_w < 1 || cv->dil_h < 1 || cv->dil_w < 1 || cv->pad_h < 0 || cv->pad_w < 0)
@@ -1329,8 +1329,18 @@ sg_status_t sg_sol_bound(int32_t op, const void* desc, int64_t batch_or_groups, 
         const int64_t P = sh < 0 ? 0 : sh / cv->stride_h + 1;
         const int64_t Q = sw < 0 ? 0 : sw / cv->stride_w + 1;
         macs = cv->N * P * Q * cv->K * cv->C * cv->R * cv->S;
-        elems_in = cv->N * cv->H * cv->W * cv->C + cv->K * cv->R * cv->S * cv->C + (has_bias ? cv->K : 0);
-        elems_out = cv->N * P * Q * cv->K * (cv->beta != 0.0f ? 2 : 1);
+        const int64_t x = cv->N * cv->H * cv->W * cv->C, w = cv->K * cv->R * cv->S * cv->C, y = cv->N * P * Q * cv->K;
+        const int64_t rw = cv->beta != 0.0f ? 2 : 1;            // the output tensor is also read when beta != 0
+        if (op == SG_OP_CONV2D) {
+            elems_in = x + w + (has_bias ? cv->K : 0);
+            elems_out = y * rw;
+        } else if (op == SG_OP_CONV2D_DGRAD) {                   // reads dY and the filter, writes dX
+            elems_in = y + w;
+            elems_out = x * rw;
+        } else {                                                 // reads dY and X, writes dW
+            elems_in = y + x;
+            elems_out = w * rw;
+        }
     } else if (op == SG_OP_TRANSPOSE) {
         const sg_transpose_desc_t* t = static_cast<const sg_transpose_desc_t*>(desc);
         if (t->batch < 0 || t->rows < 0 || t->cols < 0) return fail(SG_ERR_INVALID_ARG, "sg_sol_bound: negative extent");

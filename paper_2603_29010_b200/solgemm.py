@@ -33,7 +33,7 @@ LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
 DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4}
-OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4}
+OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4, "conv2d_dgrad": 5, "conv2d_wgrad": 6}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop", "sg_gemm_ex", "sg_conv2d_fprop_ex",
             "sg_conv2d_dgrad", "sg_conv2d_wgrad",
@@ -487,7 +487,7 @@ def sol_bound(op: str, *, M=0, N=0, K=0, batch_or_groups=1, Ms: Optional[Sequenc
     if op == "transpose":
         b, r, c_ = transpose_shape
         desc = TransposeDesc(b, r, c_, c_, r, r * c_, r * c_, DTYPES[transpose_dtypes[0]], DTYPES[transpose_dtypes[1]], 0, 0)
-    elif op == "conv2d":
+    elif op in ("conv2d", "conv2d_dgrad", "conv2d_wgrad"):
         c = conv
         desc = Conv2dDesc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], *c.get("pad", (0, 0)),
                           *c.get("stride", (1, 1)), *c.get("dil", (1, 1)), 0, 0, 1.0, float(beta), 0, 0.0, 0.0, 0)

@@ -154,6 +154,14 @@ def test_sol_bound_counts_for_every_operation(sg):
     r = sg.sol_bound("conv2d", conv=conv, has_bias=1, **hw)
     assert (r["flops"], r["bytes"]) == (118_380_036_096, 103_940_608)
     assert r["flops"] == orc.conv_flops(**conv) and r["bytes"] == orc.conv_bytes(**conv, has_bias=True)
+    # the gradients execute the forward problem's FLOPs; bytes: dY + Wf + dX and dY + X + dW (hand counts:
+    # x = y = 25,690,112 elements, w = 589,824 elements; dW kept in fp32)
+    r = sg.sol_bound("conv2d_dgrad", conv=conv, **hw)
+    assert (r["flops"], r["bytes"]) == (118_380_036_096, 2 * (25_690_112 + 589_824) + 2 * 25_690_112)
+    assert r["bytes"] == orc.conv_grad_bytes("dgrad", **conv)
+    r = sg.sol_bound("conv2d_wgrad", conv=conv, elem_bytes_out=4, beta=1.0, **hw)
+    assert (r["flops"], r["bytes"]) == (118_380_036_096, 2 * 2 * 25_690_112 + 2 * 4 * 589_824)
+    assert r["bytes"] == orc.conv_grad_bytes("wgrad", **conv, eb_out=4, has_c=True)
     Ms = [128, 4096, 1000, 0]
     r = sg.sol_bound("grouped", N=4096, K=4096, batch_or_groups=4, Ms=Ms, **hw)
     assert r["flops"] == 33_554_432 * sum(Ms) and r["bytes"] == 16_384 * sum(Ms) + 4 * 33_554_432
