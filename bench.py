@@ -248,6 +248,91 @@ def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int) -> dict:
     return out
 
 
+def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
+    """Kernel-only timings of the rows built beyond the five configurations: residual and extended epilogues, other
+    input types and operand layouts, skinny long-K shapes, the transpose stage and the convolution gradients."""
+    out = {}
+    hw = dict(peak_flops=peaks["bf16_tflops"] * 1e12, peak_bytes_per_s=peaks["hbm_gbs"] * 1e9)
+
+    def timed(name, fns, sol_kw, reps=20, note=None):
+        for f in fns[:2]:
+            f()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for f in fns:
+                f()
+        graph.replay()
+        torch.cuda.synchronize()
+        dt = time_steps(lambda i: graph.replay(), reps, torch) / (reps * len(fns))
+        sol = sg.sol_bound(**sol_kw, **hw)
+        out[name] = {"us": round(dt * 1e6, 2), "tflops": round(sol["flops"] / dt / 1e12, 1), "gbs": round(sol["bytes"] / dt / 1e9),
+                     "frac_of_sol_measured_bf16_peaks": round(sol["t_sol_s"] / dt, 3), "plan": sg.last_launch_plan()}
+        if note:
+            out[name]["note"] = note
+
+    n = 4096
+    sets = 7
+    bf = torch.bfloat16
+    data = [inputs.make_gemm(n, n, n, "normal", 1 / 64., bias=True, seed=i, device=dev) for i in range(sets)]
+    outs = [torch.empty(n, n, dtype=bf, device=dev) for _ in range(sets)]
+    res = [inputs.normal([n, n], 90 + i, 3, device=dev) for i in range(2)]
+    gemm_sol = dict(op="gemm", M=n, N=n, K=n, has_bias=1)
+    timed("gemm4096_bias_relu", [(lambda i=i: sg.gemm(*data[i][:2], bias=data[i][2], out=outs[i], epi="relu")) for i in range(sets)],
+          gemm_sol)
+    timed("gemm4096_bias_relu_residual_beta1",
+          [(lambda i=i: sg.gemm(*data[i][:2], bias=data[i][2], C=res[i % 2], beta=1.0, out=outs[i], epi="relu")) for i in range(sets)],
+          dict(gemm_sol, beta=1.0))
+    rs = torch.rand(n, device=dev) + 0.5
+    cs = torch.rand(n, device=dev) + 0.5
+    aux = torch.empty(n, n, dtype=bf, device=dev)
+    timed("gemm4096_ex_scales_gelu_auxstore_residual",
+          [(lambda i=i: sg.gemm(*data[i][:2], bias=data[i][2], out=outs[i], epi="gelu",
+                                ex=dict(row_scale=rs, col_scale=cs, aux_store=aux, aux_load=res[i % 2], post_scale=0.5)))
+           for i in range(sets)], gemm_sol, note="bytes of the scales and aux tensors not counted in the bound")
+    for la, lb in (("col", "col"), ("row", "row"), ("col", "row")):
+        timed(f"gemm4096_layout_A{la}_B{lb}",
+              [(lambda i=i: sg.gemm(data[i][0], data[i][1], out=outs[i], layout_a=la, layout_b=lb)) for i in range(sets)],
+              dict(op="gemm", M=n, N=n, K=n))
+    h16 = [(data[i][0].to(torch.float16), data[i][1].to(torch.float16)) for i in range(sets)]
+    o16 = [torch.empty(n, n, dtype=torch.float16, device=dev) for _ in range(2)]
+    timed("gemm4096_fp16_in_fp16_out", [(lambda i=i: sg.gemm(*h16[i], out=o16[i % 2])) for i in range(sets)], dict(op="gemm", M=n, N=n, K=n))
+    del h16, o16
+    for dt8, nm in ((torch.float8_e4m3fn, "e4m3"), (torch.float8_e5m2, "e5m2")):
+        q = [(data[i][0].float().mul(64).to(dt8), data[i][1].float().mul(64).to(dt8)) for i in range(sets)]
+        timed(f"gemm4096_fp8_{nm}_in_bf16_out", [(lambda i=i: sg.gemm(*q[i], out=outs[i])) for i in range(sets)],
+              dict(op="gemm", M=n, N=n, K=n, elem_bytes_in=1), note="fraction against the bf16 peak: above 1 is expected")
+        del q
+    del data, outs, res, aux
+    for (M, N, K) in ((256, 256, 32768), (512, 512, 16384), (128, 4096, 16384), (2048, 4096, 8192), (8192, 8192, 8192)):
+        A = inputs.normal([M, K], 1, 1, K ** -0.5, device=dev)
+        B = inputs.normal([N, K], 1, 2, 1.0, device=dev)
+        O = torch.empty(M, N, dtype=bf, device=dev)
+        timed(f"gemm_{M}x{N}x{K}", [lambda: sg.gemm(A, B, out=O)], dict(op="gemm", M=M, N=N, K=K), reps=10,
+              note="one buffer set (operands may stay in L2)")
+        del A, B, O
+    for (b, r, c_) in ((32, 256, 3136), (8, 4096, 4096)):
+        for di, do in ((torch.float32, bf), (bf, bf)):
+            xs = [torch.randn(b, r, c_, device=dev).to(di) for _ in range(4)]
+            ys = [torch.empty(b, c_, r, dtype=do, device=dev) for _ in range(4)]
+            timed(f"transpose_{b}x{r}x{c_}_{str(di)[6:]}_to_{str(do)[6:]}", [(lambda i=i: sg.transpose(xs[i], out=ys[i])) for i in range(4)],
+                  dict(op="transpose", transpose_shape=(b, r, c_), transpose_dtypes=(di, do)))
+            del xs, ys
+    cv = inputs.CONFIGS["c4_conv_32x56x56x256_k256_3x3_bias_relu"]
+    geo = {k: cv[k] for k in ("N", "H", "W", "C", "K", "R", "S", "pad")}
+    X = [inputs.normal([cv["N"], cv["H"], cv["W"], cv["C"]], 70 + i, 1, device=dev) for i in range(4)]
+    dY = [inputs.normal([cv["N"], 56, 56, cv["K"]], 70 + i, 3, device=dev) for i in range(4)]
+    Wf = inputs.normal([cv["K"], cv["R"], cv["S"], cv["C"]], 70, 2, 1 / 48., device=dev)
+    dX = [torch.empty(cv["N"], cv["H"], cv["W"], cv["C"], dtype=bf, device=dev) for _ in range(4)]
+    dW = torch.empty(cv["K"], cv["R"], cv["S"], cv["C"], dtype=torch.float32, device=dev)
+    timed("conv2d_dgrad_32x56x56x256_k256_3x3", [(lambda i=i: sg.conv2d_dgrad(dY[i], Wf, (56, 56), pad=(1, 1), out=dX[i])) for i in range(4)],
+          dict(op="conv2d_dgrad", conv=geo))
+    timed("conv2d_wgrad_32x56x56x256_k256_3x3_fp32_dW",
+          [(lambda i=i: sg.conv2d_wgrad(dY[i], X[i], (3, 3), pad=(1, 1), out=dW)) for i in range(4)],
+          dict(op="conv2d_wgrad", conv=geo, elem_bytes_out=4))
+    return out
+
+
 def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     import torch
     import torch.distributed as dist
@@ -387,6 +472,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         torch.cuda.synchronize()
         got = outs[0][:rows].cpu().double()
         line["parity_sample_ok"] = bool(((got - ref).abs() <= 1e-2 + 1e-2 * ref.abs()).all())
+        if args.widened:
+            line["widened"] = bench_widened(sg, inputs, torch, dev, peaks)
         if args.all_configs:
             line["per_config"] = bench_extra_configs(sg, inputs, torch, dev, peaks, args.steps)
             if args.torch_ref:
@@ -410,6 +497,9 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (N=1 only)")
+    ap.add_argument("--widened", action="store_true",
+                    help="also time the rows built beyond the five configurations (epilogue chain, dtypes, layouts, "
+                         "skinny shapes, transpose, conv gradients; N=1 only)")
     ap.add_argument("--torch-ref", action="store_true", help="with --all-configs: also time torch's library kernels")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernel)")
