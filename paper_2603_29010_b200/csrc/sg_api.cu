@@ -555,6 +555,11 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (desc->M == 0 || desc->N == 0 || batch == 0) return SG_OK;
     st = check_ptrs(A, B, C, bias, D, desc->K, desc->beta, desc->epi, who);
     if (st != SG_OK) return st;
+    {
+        Params scratch_params;          // the chain's rules are checked before any device is touched
+        st = apply_ex(&scratch_params, ex, desc->N, c.esize_out, who);
+        if (st != SG_OK) return st;
+    }
     if (batch > 1) {
         if (sA < 0 || sB < 0 || sC < 0 || sD < 0 || sBias < 0) return fail(SG_ERR_INVALID_ARG, "%s: negative batch stride", who);
         if ((sA * c.esize_in) % 16 || (sB * c.esize_in) % 16 || (sD * c.esize_out) % 16 || (desc->beta != 0.0f && (sC * c.esize_out) % 16))
@@ -961,6 +966,11 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
     const int64_t Kg = desc->C * desc->R * desc->S;
     st = check_ptrs(X, Wf, Cin, bias, Y, Kg, desc->beta, desc->epi, "sg_conv2d_fprop");
     if (st != SG_OK) return st;
+    {
+        Params scratch_params;
+        st = apply_ex(&scratch_params, ex, desc->K, c.esize_out, "sg_conv2d_fprop_ex");
+        if (st != SG_OK) return st;
+    }
     if (desc->C == 0) return fail(SG_ERR_UNSUPPORTED, "sg_conv2d_fprop: C == 0");
 
     DeviceState* d = nullptr;

@@ -1,9 +1,11 @@
 """Host-side partitioning of the four operations across GPUs (one process per GPU).
 
-Every operation of the library decomposes into independent units -- rows of A/D for a GEMM,
+Every forward operation of the library decomposes into independent units -- rows of A/D for a GEMM,
 batch entries, whole groups, images of a convolution -- so a multi-GPU run needs no exchange
-step on the data path: each rank runs the single-GPU kernel on its shard.  The functions here
+step on the data path: each rank runs the single-GPU kernel on its shard.  The partition functions
 are pure integer arithmetic (no tensors, no CUDA) so they can be tested with CPU process groups.
+The one operation with a real exchange step is the data-parallel weight gradient: its sum runs over
+the images, so the ranks' partial dW are added with an all-reduce (``reduce_weight_gradient``).
 """
 from __future__ import annotations
 
@@ -49,3 +51,11 @@ def assign_groups(Ms: Sequence[int], world: int) -> List[List[int]]:
     for lst in owned:
         lst.sort()
     return owned
+
+
+def reduce_weight_gradient(dW, group=None):
+    """Data-parallel ``conv2d_wgrad``: every rank has summed over its own images (``conv_images``); the filter
+    gradient is the sum over all images, i.e. an all-reduce of the ranks' dW (NCCL on GPUs, gloo on CPU), in place."""
+    import torch.distributed as dist
+    dist.all_reduce(dW, op=dist.ReduceOp.SUM, group=group)
+    return dW

@@ -125,6 +125,26 @@ def test_grouped_and_conv_validation(sg):
     assert sg.STATUS_NAMES[call(conv(), X=None)] == "SG_ERR_NULL_POINTER"
     assert call(conv(N=0)) == 0 and call(conv(H=1, W=1, pad_h=0, pad_w=0)) == 0      # empty output
 
+    # gradients: checked before any device is touched
+    dgrad = lambda d, dY=0x1000: lib.sg_conv2d_dgrad(ctypes.byref(d), dY, 0x2000, None, 0x3000, None)
+    wgrad = lambda d, dY=0x1000: lib.sg_conv2d_wgrad(ctypes.byref(d), dY, 0x2000, None, 0x3000, None)
+    assert sg.STATUS_NAMES[dgrad(conv(stride_h=2))] == "SG_ERR_UNSUPPORTED"          # strided data gradient
+    assert sg.STATUS_NAMES[dgrad(conv(pad_h=3))] == "SG_ERR_UNSUPPORTED"             # pad beyond the filter extent
+    assert sg.STATUS_NAMES[dgrad(conv(epi=2))] == "SG_ERR_INVALID_ARG"               # no activation on a gradient
+    assert sg.STATUS_NAMES[wgrad(conv(in_dtype=3))] == "SG_ERR_UNSUPPORTED"          # fp8 inputs
+    assert sg.STATUS_NAMES[wgrad(conv(C=20))] == "SG_ERR_ALIGNMENT"
+    assert sg.STATUS_NAMES[dgrad(conv(K=12))] == "SG_ERR_ALIGNMENT"
+    assert sg.STATUS_NAMES[wgrad(conv(dil_w=0))] == "SG_ERR_INVALID_ARG"
+    assert sg.STATUS_NAMES[lib.sg_conv2d_wgrad(None, 0x1000, 0x2000, None, 0x3000, None)] == "SG_ERR_NULL_POINTER"
+    assert dgrad(conv(N=0)) == 0 and wgrad(conv(K=0)) == 0                           # empty outputs
+
+    # extended epilogue: the chain's own rules
+    ex = sg.EpilogueEx(None, 0x5004, None, 1.0, 0, None, 0, None, 0)
+    call_ex = lambda e: lib.sg_gemm_ex(ctypes.byref(_desc(sg)), ctypes.byref(e), 0x1000, 0x2000, None, None, 0x3000, None)
+    assert sg.STATUS_NAMES[call_ex(ex)] == "SG_ERR_ALIGNMENT"                        # col_scale not 16-byte aligned
+    assert sg.STATUS_NAMES[call_ex(sg.EpilogueEx(None, None, None, 1.0, 7, None, 0, None, 0))] == "SG_ERR_INVALID_ARG"
+    assert sg.STATUS_NAMES[call_ex(sg.EpilogueEx(None, None, None, 1.0, 0, 0x6000, 64, None, 0))] == "SG_ERR_INVALID_ARG"  # ld < N
+
 
 def test_sol_bound_matches_the_printed_report_and_the_oracle(sg, golden_dir):
     g = load_golden(os.path.join(golden_dir, "sol_report_gemm4096.txt"))

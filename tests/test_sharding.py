@@ -71,3 +71,30 @@ def test_two_ranks_partition_every_operation_over_gloo():
     world = 2
     Ms = inputs.grouped_sizes(16, 128, 4096)
     mp.spawn(_worker, args=(world, _free_port(), 4096, 128, Ms), nprocs=world, join=True)
+
+
+def _wgrad_worker(rank, world, port):
+    from oracle import oracle as orc
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        N, H, W, C, K, R, S = 5, 6, 7, 8, 8, 3, 3
+        X = inputs.small_integers([N, H, W, C], 51, 1, -2, 2)
+        dY = inputs.small_integers([N, H, W, K], 51, 3, -2, 2)
+        n0, n1 = sharding.conv_images(N, world, rank)
+        part, _ = orc.conv2d_wgrad(dY[n0:n1].contiguous(), X[n0:n1].contiguous(), (R, S), pad=(1, 1))
+        dW = part.to(torch.float32)               # integers: exact in fp32
+        sharding.reduce_weight_gradient(dW)
+        full, _ = orc.conv2d_wgrad(dY, X, (R, S), pad=(1, 1))
+        assert torch.equal(dW.double(), full)
+        # the data gradient needs no exchange: each rank's images are its own rows of dX
+        Wf = inputs.small_integers([K, R, S, C], 51, 2, -2, 2)
+        mine, _ = orc.conv2d_dgrad(dY[n0:n1].contiguous(), Wf, (H, W), pad=(1, 1))
+        whole, _ = orc.conv2d_dgrad(dY, Wf, (H, W), pad=(1, 1))
+        assert torch.equal(mine, whole[n0:n1])
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_data_parallel_conv_gradients_over_gloo():
+    mp.spawn(_wgrad_worker, args=(2, _free_port()), nprocs=2, join=True)
