@@ -114,3 +114,25 @@ def test_c5_grouped_silu():
         pi, pj = sample_points(m, c["N"], 256, 100 + g)
         ref, absacc = orc.gemm_points(hA, hB, pi, pj, epi=c["epi"])
         check_points(outs[g], ref, absacc, pi, pj, f"c5 group {g} sampled")
+
+
+def test_c4_sized_conv_gradients():
+    # the gradients of the benchmark convolution at its full size, in the configuration bench.py --widened times
+    c = CFG["c4_conv_32x56x56x256_k256_3x3_bias_relu"]
+    N_, H, W, C, K, R, S = c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"]
+    X = inputs.normal([N_, H, W, C], 70, 1, device=DEV)
+    dY = inputs.normal([N_, H, W, K], 70, 3, 1 / 16., device=DEV)
+    Wf = inputs.normal([K, R, S, C], 70, 2, 1 / 48., device=DEV)
+    hX, hdY, hW = X.cpu(), dY.cpu(), Wf.cpu()
+    dX = sg.conv2d_dgrad(dY, Wf, (H, W), pad=c["pad"])
+    assert bool(torch.isfinite(dX).all())
+    PQ = H * W
+    dXf = dX.view(-1, C)
+    for p0 in (0, 52, 124, PQ - 6, 9 * PQ + 1500, N_ * PQ - 8):      # corners, a tile edge, an image boundary, the end
+        ref, absacc = orc.conv2d_dgrad(hdY, hW, (H, W), pad=c["pad"], pixels=(p0, p0 + 8))
+        parity.assert_matches(dXf[p0:p0 + 8], ref, absacc, f"c4 dgrad pixels {p0}")
+    dW = sg.conv2d_wgrad(dY, X, (R, S), pad=c["pad"])                  # fp32, K ranges through the scratch
+    assert sg.last_launch_plan()["tail_split"] < 0 and bool(torch.isfinite(dW).all())
+    for k0 in (0, 131, K - 1):                                          # first tile, across the pair's second CTA, last row
+        ref, absacc = orc.conv2d_wgrad(hdY, hX, (R, S), pad=c["pad"], filters=(k0, k0 + 1))
+        parity.assert_matches(dW[k0:k0 + 1].reshape(-1, C), ref.reshape(-1, C), absacc.reshape(-1, C), f"c4 wgrad filter {k0}")
