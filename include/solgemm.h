@@ -340,15 +340,18 @@ sg_status_t sg_last_kernel_clock(double* sm_mhz, void* cuda_stream);
 sg_status_t sg_set_tail_mode(int32_t mode);
 
 /*
- * sg_set_scratch: lends the library a device buffer (current device) that later contraction calls may use to
- * balance their last, partial wave of tiles: several SM groups then share one output tile's K loop and exchange
- * fp32 partial sums through the buffer ("stream-K" for the tail; paper: scheduler tile=stream_k, Appendix A.1).
- * Optional: without a scratch the tail tiles are cut into column slices instead, and results are the same up to
- * fp32 summation order.  (As measured so far the exchange costs about as much as it saves, so the planner
- * prefers column slices; sg_set_tail_mode(2) forces the K ranges.)  256-byte aligned; SG_SCRATCH_BYTES_RECOMMENDED covers every shape; the first 8 KB are
- * cleared synchronously by this call.  The caller keeps ownership and must keep the buffer alive and untouched
- * until it calls sg_set_scratch(NULL, 0).  All calls on the device share it: work that overlaps on the GPU
- * (several streams) must not use it concurrently -- unregister it, or serialise such calls.
+ * sg_set_scratch: lends the library a device buffer (current device) through which several SM groups can share
+ * one output tile's K loop: every group parks its fp32 partial sums in the buffer and finishes a share of the tile
+ * from all groups' sums (the DSL's split-K / tile=stream_k knobs, Appendix A.1).  With a scratch lent the planner
+ * uses K ranges for problems with few output tiles and a long K -- skinny GEMMs, the convolution weight gradient --
+ * where they are several times faster than whole tiles on a few SMs; for the last partial wave of large problems it
+ * keeps column slices (as measured the exchange costs what it saves there; sg_set_tail_mode(2) forces K ranges).
+ * Optional: without a scratch every tile runs its whole K loop; results agree up to fp32 summation order, and are
+ * reproducible for a given shape and scratch.  256-byte aligned, at least 1 MB + 8 KB; SG_SCRATCH_BYTES_RECOMMENDED
+ * covers every shape; the first 8 KB (counters) are cleared synchronously by this call and left at zero by every
+ * launch.  The caller keeps ownership and must keep the buffer alive and untouched until it calls
+ * sg_set_scratch(NULL, 0).  All calls on the device share it: work that overlaps on the GPU (several streams) must
+ * not use it concurrently -- unregister it, or serialise such calls.
  */
 #define SG_SCRATCH_BYTES_RECOMMENDED (32u << 20)
 sg_status_t sg_set_scratch(void* scratch_dev, size_t bytes);
