@@ -131,6 +131,7 @@ def test_c4_sized_conv_gradients():
     for p0 in (0, 52, 124, PQ - 6, 9 * PQ + 1500, N_ * PQ - 8):      # corners, a tile edge, an image boundary, the end
         ref, absacc = orc.conv2d_dgrad(hdY, hW, (H, W), pad=c["pad"], pixels=(p0, p0 + 8))
         parity.assert_matches(dXf[p0:p0 + 8], ref, absacc, f"c4 dgrad pixels {p0}")
+    sg.enable_scratch(True)                                             # (the environment may have turned lending off)
     dW = sg.conv2d_wgrad(dY, X, (R, S), pad=c["pad"])                  # fp32, K ranges through the scratch
     assert sg.last_launch_plan()["tail_split"] < 0 and bool(torch.isfinite(dW).all())
     for k0 in (0, 131, K - 1):                                          # first tile, across the pair's second CTA, last row
