@@ -199,10 +199,12 @@ sg_status_t sg_conv2d_fprop(const sg_conv2d_desc_t* desc, const void* X, const v
  *   Cin  device, out_dtype, the output's shape; may be NULL when beta == 0
  *   dX   device, out_dtype, [N,H,W,C], written in full     dW  device, out_dtype, [K,R,S,C], written in full
  * Both run as implicit GEMMs in the forward kernel: dgrad contracts over (tap, k) with the filter read C-contiguous
- * and its taps mirrored; wgrad is one product per tap, dY^T (K x NPQ) times the tap-shifted X (NPQ x C), whose long
- * contraction is cut into K ranges through the scratch of sg_set_scratch when one is lent (few output tiles).
+ * and its taps mirrored -- with a stride, one launch per output phase (h mod stride_h, w mod stride_w), each a
+ * stride-1 problem over the taps that reach that phase, its rows scattered to their pixels of dX; wgrad is one
+ * product per tap, dY^T (K x NPQ) times the tap-shifted X (NPQ x C), whose long contraction is cut into K ranges
+ * through the scratch of sg_set_scratch when one is lent (few output tiles).
  * desc->epi must be SG_EPI_NONE.  K and C must span multiples of 16 bytes in both types.
- * SG_ERR_UNSUPPORTED: dgrad with a stride other than 1 or with pad > dil*(filter-1); 8-bit inputs.
+ * SG_ERR_UNSUPPORTED: 8-bit inputs; strides above 8 or filter extents beyond the im2col TMA limits.
  * Empty outputs return SG_OK without a launch; an empty sum (no output pixels) gives beta * Cin.
  */
 sg_status_t sg_conv2d_dgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* Wf, const void* Cin,

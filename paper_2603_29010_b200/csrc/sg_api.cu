@@ -313,7 +313,10 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
     const int force_bn = g_tune_tile_n.load();
     const int force_pair = g_tune_pair.load();
     const int bns[3] = {256, 128, 64};
-    const double factor[2][3] = {{1.18, 1.30, 1.89}, {1.00, 1.26, 2.57}};   // [pair][bn index], relative time per output area
+    // [pair][bn index]: time per output area relative to two-CTA 256-wide tiles, measured on the 4096^3 GEMM and the
+    // benchmark convolution with every tiling forced (narrow tiles re-read the A panel for fewer columns and are bound
+    // by operand traffic)
+    const double factor[2][3] = {{1.18, 1.56, 2.90}, {1.00, 1.50, 3.30}};
     auto tiles_for = [&](int tile_m, int bn) {
         int64_t tiles = 0;
         for (int64_t r : rows_per_problem) tiles += ((r + tile_m - 1) / tile_m) * ((N + bn - 1) / bn);
@@ -1078,6 +1081,41 @@ sg_status_t grad_geometry(const sg_conv2d_desc_t* desc, const char* who, Checked
 
 }  // namespace
 
+namespace {
+
+// One spatial dimension of one output phase of the data gradient.  Output positions h = a + stride * i (i < out_n)
+// receive the filter taps r with (a + pad - r * dil) divisible by the stride; for those p = i + (a + pad - r * dil) /
+// stride.  The taps form an arithmetic progression; walked from the largest r down, the offsets grow by dd per tap,
+// i.e. the phase is a stride-1 correlation of dY with a mirrored, thinned filter:
+//   p = i + lower + m * dd,   filter tap r = tap_hi - m * tap_step,   m = 0 .. taps - 1.
+struct PhaseDim {
+    int64_t out_n = 0;
+    int taps = 0, tap_hi = 0, tap_step = 1, dd = 1;
+    int64_t lower = 0;
+};
+PhaseDim phase_dim(int64_t a, int64_t extent, int64_t pad, int64_t dil, int64_t filt, int64_t stride) {
+    PhaseDim d;
+    d.out_n = a < extent ? (extent - a + stride - 1) / stride : 0;
+    int first = -1, second = -1, last = -1;
+    for (int r = 0; r < filt; ++r) {
+        const int64_t x = a + pad - r * dil;
+        if (((x % stride) + stride) % stride != 0) continue;
+        if (first < 0) first = r;
+        else if (second < 0) second = r;
+        last = r;
+        ++d.taps;
+    }
+    if (d.taps == 0) return d;
+    d.tap_hi = last;
+    d.tap_step = d.taps > 1 ? second - first : 1;
+    d.dd = d.taps > 1 ? static_cast<int>(dil * d.tap_step / stride) : 1;
+    const int64_t x = a + pad - static_cast<int64_t>(last) * dil;       // divisible by the stride
+    d.lower = x >= 0 ? x / stride : -((-x) / stride);
+    return d;
+}
+
+}  // namespace
+
 extern "C" sg_status_t sg_conv2d_dgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* Wf, const void* Cin, void* dX,
                                        void* cuda_stream) {
     const char* who = "sg_conv2d_dgrad";
@@ -1085,82 +1123,116 @@ extern "C" sg_status_t sg_conv2d_dgrad(const sg_conv2d_desc_t* desc, const void*
     int64_t P = 0, Q = 0;
     sg_status_t st = grad_geometry(desc, who, &c, &P, &Q);
     if (st != SG_OK) return st;
-    if (desc->stride_h != 1 || desc->stride_w != 1)
-        return fail(SG_ERR_UNSUPPORTED, "%s: only stride 1 is implemented", who);
-    const int64_t pad_h = desc->dil_h * (desc->R - 1) - desc->pad_h, pad_w = desc->dil_w * (desc->S - 1) - desc->pad_w;
-    if (pad_h < 0 || pad_w < 0) return fail(SG_ERR_UNSUPPORTED, "%s: pad larger than the dilated filter extent", who);
-    if (pad_h > 127 || pad_w > 127) return fail(SG_ERR_UNSUPPORTED, "%s: filter extent outside the im2col TMA limits", who);
-    const int64_t Mg = desc->N * desc->H * desc->W;       // rows: input pixels
-    if (Mg == 0 || desc->C == 0) return SG_OK;
-    const int64_t Kg = desc->K * desc->R * desc->S;       // contraction: taps x output channels of the forward pass
+    if (desc->N * desc->H * desc->W == 0 || desc->C == 0) return SG_OK;
     if ((desc->K * c.esize_in) % 16 || (desc->C * c.esize_in) % 16 || (desc->C * c.esize_out) % 16)
         return fail(SG_ERR_ALIGNMENT, "%s: K and C must span multiples of 16 bytes", who);
-    const bool empty = P == 0 || Q == 0 || desc->K == 0;  // nothing to sum: dX = beta * Cin
-    st = check_ptrs(dY, Wf, Cin, nullptr, dX, empty ? 0 : Kg, desc->beta, desc->epi, who);
+    const bool no_sum = P == 0 || Q == 0 || desc->K == 0;       // nothing to sum anywhere: dX = beta * Cin
+    st = check_ptrs(dY, Wf, Cin, nullptr, dX, no_sum ? 0 : desc->K, desc->beta, desc->epi, who);
     if (st != SG_OK) return st;
+    const bool strided = desc->stride_h != 1 || desc->stride_w != 1;
+    // every output phase (h mod stride_h, w mod stride_w) is one launch; a stride-1 gradient has one phase
+    std::vector<std::pair<PhaseDim, PhaseDim>> phases;
+    std::vector<std::pair<int, int>> phase_ab;
+    for (int a = 0; a < desc->stride_h; ++a)
+        for (int b = 0; b < desc->stride_w; ++b) {
+            PhaseDim ph = phase_dim(a, desc->H, desc->pad_h, desc->dil_h, desc->R, desc->stride_h);
+            PhaseDim pw = phase_dim(b, desc->W, desc->pad_w, desc->dil_w, desc->S, desc->stride_w);
+            if (ph.out_n == 0 || pw.out_n == 0) continue;
+            for (const PhaseDim* d : {&ph, &pw}) {
+                const int64_t in_extent = d == &ph ? P : Q;
+                const int64_t upper = d->out_n - in_extent + d->lower;
+                if (d->taps > 0 && (d->lower < -128 || d->lower > 127 || upper < -128 || upper > 127 ||
+                                    static_cast<int64_t>(d->taps - 1) * d->dd > 255))
+                    return fail(SG_ERR_UNSUPPORTED, "%s: pad / filter extent / stride outside the im2col TMA limits", who);
+            }
+            phases.emplace_back(ph, pw);
+            phase_ab.emplace_back(a, b);
+        }
 
     DeviceState* d = nullptr;
     st = device_state(&d);
     if (st != SG_OK) return st;
-    Params p;
-    base_params(&p, *d, desc->alpha, desc->beta, desc->epi, 0.0f, 0.0f);
-    p.in_f16 = c.in_f16 ? 1 : 0;
-    p.bk_elems = c.bk;
-    Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->C, Kg, 64);
-    const int tile_m = s.pair ? 256 : 128;
-    p.mode = MODE_CONV;
-    p.b_mn_major = 1;
-    p.flip_taps = 1;
-    p.num_taps = static_cast<int32_t>(desc->R * desc->S);
-    p.M = static_cast<int32_t>(Mg);
-    p.N = static_cast<int32_t>(desc->C);
-    p.K = static_cast<int32_t>(Kg);
-    p.batch = 1;
-    p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
-    p.tiles_n = static_cast<int32_t>((desc->C + s.bn - 1) / s.bn);
-    p.cblocks = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
-    p.num_kb = empty ? 0 : p.num_taps * p.cblocks;
-    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p, 64);
-    p.C = desc->beta != 0.0f ? Cin : nullptr;
-    p.ldc = desc->C;
-    p.D = dX;
-    p.ldd = desc->C;
-    // the "image" the kernel walks is dY [N,P,Q,K]; its output pixels are the H x W pixels of dX
-    p.P = static_cast<int32_t>(desc->H);
-    p.Q = static_cast<int32_t>(desc->W);
-    p.stride_h = 1; p.stride_w = 1;
-    p.pad_h = static_cast<int32_t>(pad_h); p.pad_w = static_cast<int32_t>(pad_w);
-    p.dil_h = desc->dil_h; p.dil_w = desc->dil_w;
-    p.S = static_cast<int32_t>(desc->S);
-    st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, dX, desc->C, Mg, 1, desc->C, 0, c.f32_out ? 32 : 64, 32, "dX");
-    if (st != SG_OK) return st;
-    if (empty) {
-        p.tmA = p.tmD; p.tmB = p.tmD; p.tmB2 = p.tmD;
-    } else {
-        cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->K), static_cast<cuuint64_t>(Q), static_cast<cuuint64_t>(P),
-                              static_cast<cuuint64_t>(desc->N)};
-        const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
-        cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->K) * es, static_cast<cuuint64_t>(Q * desc->K) * es,
-                                 static_cast<cuuint64_t>(P * Q * desc->K) * es};
-        int lower[2] = {static_cast<int>(-pad_w), static_cast<int>(-pad_h)};
-        int upper[2] = {static_cast<int>(pad_w - (desc->S - 1) * desc->dil_w), static_cast<int>(pad_h - (desc->R - 1) * desc->dil_h)};
-        cuuint32_t estr[4] = {1, 1, 1, 1};
-        CUresult r = g_encode_im2col(&p.tmA, c.tm_in, 4, const_cast<void*>(dY), dims, strides, lower, upper,
-                                     static_cast<cuuint32_t>(c.bk), 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(dY) failed with CUresult %d", static_cast<int>(r));
-        // filter [K][R*S][C] read with C contiguous: boxes of 64 c x 1 tap x 64 k
-        cuuint64_t fdims[3] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->R * desc->S),
-                               static_cast<cuuint64_t>(desc->K)};
-        cuuint64_t fstrides[2] = {static_cast<cuuint64_t>(desc->C) * es, static_cast<cuuint64_t>(desc->C * desc->R * desc->S) * es};
-        cuuint32_t box[3] = {64, 1, 64};
-        cuuint32_t e3[3] = {1, 1, 1};
-        r = g_encode_tiled(&p.tmB, c.tm_in, 3, const_cast<void*>(Wf), fdims, fstrides, box, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
-        p.tmB2 = p.tmB;
+    for (size_t i = 0; i < phases.size(); ++i) {
+        const PhaseDim& ph = phases[i].first;
+        const PhaseDim& pw = phases[i].second;
+        const int64_t Mg = desc->N * ph.out_n * pw.out_n;       // rows: this phase's input pixels
+        const int64_t taps = static_cast<int64_t>(ph.taps) * pw.taps;
+        const bool empty = no_sum || taps == 0;
+        const int64_t Kg = desc->K * (taps > 0 ? taps : 1);     // contraction: taps x output channels of the forward pass
+        Params p;
+        base_params(&p, *d, desc->alpha, desc->beta, desc->epi, 0.0f, 0.0f);
+        p.in_f16 = c.in_f16 ? 1 : 0;
+        p.bk_elems = c.bk;
+        Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->C, Kg, 64);
+        const int tile_m = s.pair ? 256 : 128;
+        p.mode = MODE_CONV;
+        p.b_mn_major = 1;
+        p.num_taps = static_cast<int32_t>(taps);
+        p.tapb_r0 = ph.tap_hi; p.tapb_rs = -ph.tap_step;
+        p.tapb_s0 = pw.tap_hi; p.tapb_ss = -pw.tap_step;
+        p.filt_s = static_cast<int32_t>(desc->S);
+        p.M = static_cast<int32_t>(Mg);
+        p.N = static_cast<int32_t>(desc->C);
+        p.K = static_cast<int32_t>(Kg);
+        p.batch = 1;
+        p.tiles_m = static_cast<int32_t>((Mg + tile_m - 1) / tile_m);
+        p.tiles_n = static_cast<int32_t>((desc->C + s.bn - 1) / s.bn);
+        p.cblocks = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
+        p.num_kb = empty ? 0 : p.num_taps * p.cblocks;
+        plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p, 64);
+        p.C = desc->beta != 0.0f ? Cin : nullptr;
+        p.ldc = desc->C;
+        p.D = dX;
+        p.ldd = desc->C;
+        // the "image" the kernel walks is dY [N,P,Q,K]; its output pixels are this phase's pixels of dX
+        p.P = static_cast<int32_t>(ph.out_n);
+        p.Q = static_cast<int32_t>(pw.out_n);
+        p.stride_h = 1; p.stride_w = 1;
+        p.pad_h = static_cast<int32_t>(-ph.lower); p.pad_w = static_cast<int32_t>(-pw.lower);
+        p.dil_h = ph.dd; p.dil_w = pw.dd;
+        p.S = pw.taps > 0 ? pw.taps : 1;
+        if (strided) {
+            p.d_remap = 1;
+            p.remap_h0 = phase_ab[i].first; p.remap_sh = desc->stride_h;
+            p.remap_w0 = phase_ab[i].second; p.remap_sw = desc->stride_w;
+            p.remap_H = static_cast<int32_t>(desc->H); p.remap_W = static_cast<int32_t>(desc->W);
+        }
+        st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, dX, desc->C, desc->N * desc->H * desc->W, 1, desc->C, 0,
+                            c.f32_out ? 32 : 64, 32, "dX");
+        if (st != SG_OK) return st;
+        if (empty) {
+            p.tmA = p.tmD; p.tmB = p.tmD; p.tmB2 = p.tmD;
+        } else {
+            cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->K), static_cast<cuuint64_t>(Q), static_cast<cuuint64_t>(P),
+                                  static_cast<cuuint64_t>(desc->N)};
+            const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
+            cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->K) * es, static_cast<cuuint64_t>(Q * desc->K) * es,
+                                     static_cast<cuuint64_t>(P * Q * desc->K) * es};
+            int lower[2] = {static_cast<int>(pw.lower), static_cast<int>(ph.lower)};
+            int upper[2] = {static_cast<int>(pw.out_n - Q + pw.lower), static_cast<int>(ph.out_n - P + ph.lower)};
+            cuuint32_t estr[4] = {1, 1, 1, 1};
+            CUresult r = g_encode_im2col(&p.tmA, c.tm_in, 4, const_cast<void*>(dY), dims, strides, lower, upper,
+                                         static_cast<cuuint32_t>(c.bk), 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS)
+                return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(dY) failed with CUresult %d (corners %d..%d, %d..%d)",
+                            static_cast<int>(r), lower[0], upper[0], lower[1], upper[1]);
+            // filter [K][R*S][C] read with C contiguous: boxes of 64 c x 1 tap x 64 k
+            cuuint64_t fdims[3] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->R * desc->S),
+                                   static_cast<cuuint64_t>(desc->K)};
+            cuuint64_t fstrides[2] = {static_cast<cuuint64_t>(desc->C) * es, static_cast<cuuint64_t>(desc->C * desc->R * desc->S) * es};
+            cuuint32_t box[3] = {64, 1, 64};
+            cuuint32_t e3[3] = {1, 1, 1};
+            r = g_encode_tiled(&p.tmB, c.tm_in, 3, const_cast<void*>(Wf), fdims, fstrides, box, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
+            p.tmB2 = p.tmB;
+        }
+        st = launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
+        if (st != SG_OK) return st;
     }
-    return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
+    return SG_OK;
 }
 
 extern "C" sg_status_t sg_conv2d_wgrad(const sg_conv2d_desc_t* desc, const void* dY, const void* X, const void* Cin, void* dW,

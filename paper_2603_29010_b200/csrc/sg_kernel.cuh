@@ -74,8 +74,13 @@ struct alignas(64) Params {
     int32_t bk_elems;                   // elements of K per 128-byte stage row: 64 (16-bit) or 128 (8-bit)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
-    int32_t flip_taps;                  // conv (data gradient): the filter tap of B is RS - 1 - (tap of A)
-    int32_t num_taps;                   // conv: R * S
+    int32_t num_taps;                   // conv: taps walked by the K loop
+    // conv (data gradient): the filter tap B reads for A's tap (c_r, c_s) is row tapb_r0 + tapb_rs * c_r, column
+    // tapb_s0 + tapb_ss * c_s of the full R x S filter (mirrored, and for a strided gradient a subset), filt_s = S
+    int32_t tapb_r0, tapb_rs, tapb_s0, tapb_ss, filt_s;
+    // conv (strided data gradient): row m = (n, i, j) of this launch's output is pixel (n, remap_h0 + remap_sh * i,
+    // remap_w0 + remap_sw * j) of the remap_H x remap_W image that C and D address; 0 = rows are stored as they come
+    int32_t d_remap, remap_h0, remap_sh, remap_w0, remap_sw, remap_H, remap_W;
     // extended epilogue chain (all optional; ex_any = 1 when any of them is in use; dense and conv modes only):
     //   t = alpha acc * row_scale[i] * col_scale[j] + beta C + bias[j] + row_bias[i];  aux_store[i][j] = t;
     //   D = post_scale * act(t) + aux_load[i][j]
@@ -562,7 +567,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                                                   static_cast<uint16_t>(c_r * p.dil_h));
                         if (p.b_mn_major) {
                             // data gradient: the filter [k][tap][c] is read with c contiguous, 64 k x 64 c per box
-                            const int tap_b = p.flip_taps ? p.num_taps - 1 - c_tap : c_tap;
+                            const int tap_b = (p.tapb_r0 + p.tapb_rs * c_r) * p.filt_s + p.tapb_s0 + p.tapb_ss * c_s;
                             for (int j = 0; j < b_rows / 64; ++j)
                                 tma_load_3d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, tap_b, c0);
                         } else {
@@ -745,6 +750,17 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const bool rows_live = row0 < ti.rows;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
             const int row = row0 + lane;
+            // row of C and D in memory: the row itself, or for a strided data gradient the pixel it stands for
+            int64_t mem_row = row;
+            if (p.d_remap && row < ti.rows) {
+                const int pq = p.P * p.Q;
+                const int n_img = fast_div(row, p.div_pq);
+                const int rem = row - n_img * pq;
+                const int pi = fast_div(rem, p.div_q);
+                const int pj = rem - pi * p.Q;
+                mem_row = (static_cast<int64_t>(n_img) * p.remap_H + p.remap_h0 + p.remap_sh * pi) * p.remap_W + p.remap_w0 +
+                          p.remap_sw * pj;
+            }
 
             // K-split tile: the tile's K range is shared by nparts work items.  Every part parks its raw fp32 sums of
             // the column chunks it does not finish in the scratch (pass 0), then finishes the chunks it owns
@@ -952,7 +968,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (has_c && row < ti.rows) {
                     const int col0 = n0 + c * CH;
                     if constexpr (kOutF32) {
-                        const float* cp = reinterpret_cast<const float*>(c_g) + static_cast<int64_t>(row) * p.ldc + col0;
+                        const float* cp = reinterpret_cast<const float*>(c_g) + mem_row * p.ldc + col0;
                         if (col0 + CH <= p.N) {
 #pragma unroll
                             for (int i = 0; i < CH; i += 4) {
@@ -963,7 +979,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                             for (int i = 0; i < CH; ++i) if (col0 + i < p.N) v[i] += beta * cp[i];
                         }
                     } else {
-                        const uint16_t* cp = reinterpret_cast<const uint16_t*>(c_g) + static_cast<int64_t>(row) * p.ldc + col0;
+                        const uint16_t* cp = reinterpret_cast<const uint16_t*>(c_g) + mem_row * p.ldc + col0;
                         if (col0 + CH <= p.N) {
 #pragma unroll
                             for (int i = 0; i < CH; i += 8) {
@@ -1067,19 +1083,39 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     }
                 }
 
-                // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes
-                // the last, partial chunk is therefore written with plain stores so nothing beyond column N changes.
+                // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes the
+                // last, partial chunk is therefore written with plain stores so nothing beyond column N changes; a
+                // strided data gradient, whose rows are scattered over the image, is always stored this way.
                 constexpr int kElemsPer16B = kOutF32 ? 4 : 8;
-                if (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0) {
+                if (p.d_remap || (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0)) {
                     if (row < ti.rows) {
                         const int col0 = n0 + c * CH;
+                        const int valid = min(CH, p.N - col0);
                         if constexpr (kOutF32) {
-                            float* dp = reinterpret_cast<float*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
-                            for (int i = 0; i < CH; ++i) if (col0 + i < p.N) dp[i] = v[i];
+                            float* dp = reinterpret_cast<float*>(d_g) + mem_row * p.ldd + col0;
+#pragma unroll
+                            for (int i = 0; i < CH; i += 4) {
+                                if (i + 4 <= valid) {
+                                    *reinterpret_cast<float4*>(dp + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) if (i + j < valid) dp[i + j] = v[i + j];
+                                }
+                            }
                         } else {
-                            uint16_t* dp = reinterpret_cast<uint16_t*>(d_g) + static_cast<int64_t>(row) * p.ldd + col0;
-                            for (int i = 0; i < CH; ++i)
-                                if (col0 + i < p.N) dp[i] = static_cast<uint16_t>(pack2<kOutF16>(v[i], 0.0f) & 0xFFFFu);
+                            uint16_t* dp = reinterpret_cast<uint16_t*>(d_g) + mem_row * p.ldd + col0;
+#pragma unroll
+                            for (int i = 0; i < CH; i += 8) {
+                                if (i + 8 <= valid) {
+                                    *reinterpret_cast<uint4*>(dp + i) =
+                                        make_uint4(pack2<kOutF16>(v[i], v[i + 1]), pack2<kOutF16>(v[i + 2], v[i + 3]),
+                                                   pack2<kOutF16>(v[i + 4], v[i + 5]), pack2<kOutF16>(v[i + 6], v[i + 7]));
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j)
+                                        if (i + j < valid) dp[i + j] = static_cast<uint16_t>(pack2<kOutF16>(v[i + j], 0.0f) & 0xFFFFu);
+                                }
+                            }
                         }
                     }
                     __syncwarp();

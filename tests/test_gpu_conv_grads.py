@@ -41,9 +41,15 @@ GRAD_CASES = [
     (2, 11, 13, 64, 96, 3, 2, (2, 0), (1, 1), (2, 1)),      # dilation, asymmetric pads
     (2, 16, 16, 200, 72, 5, 5, (2, 2), (1, 1), (1, 1)),
 ]
-WGRAD_ONLY = [
+STRIDED = [
     (2, 15, 14, 64, 64, 3, 3, (1, 1), (2, 2), (1, 1)),      # stride 2
     (1, 13, 21, 136, 72, 3, 3, (0, 1), (2, 1), (1, 2)),
+    (2, 16, 16, 64, 64, 1, 1, (0, 0), (2, 2), (1, 1)),      # 1x1 stride 2: three of the four output phases get no tap
+    (1, 17, 19, 64, 72, 3, 3, (0, 0), (2, 2), (1, 1)),      # the last input row / column is outside every window
+    (2, 20, 18, 64, 64, 5, 4, (2, 1), (3, 2), (1, 1)),      # stride 3 x 2
+    (1, 21, 20, 72, 64, 3, 3, (2, 2), (2, 2), (2, 2)),      # stride and dilation share a factor
+    (1, 23, 9, 64, 64, 4, 2, (1, 0), (4, 1), (1, 1)),       # stride as large as the filter
+    (1, 6, 7, 64, 64, 3, 3, (3, 3), (1, 1), (1, 1)),        # pad beyond the filter extent: border windows see padding only
 ]
 
 
@@ -61,7 +67,7 @@ def _problem(case, seed, integer):
 
 
 @pytest.mark.parametrize("pair", [0, 1])
-@pytest.mark.parametrize("case", GRAD_CASES)
+@pytest.mark.parametrize("case", GRAD_CASES + STRIDED)
 def test_dgrad_integer_inputs_bit_exact(case, pair):
     sg.set_tuning(-1, pair)
     N_, H, W, C, K, R, S, pad, stride, dil = case
@@ -75,7 +81,7 @@ def test_dgrad_integer_inputs_bit_exact(case, pair):
 
 @pytest.mark.parametrize("scratch", [False, True])
 @pytest.mark.parametrize("pair", [0, 1])
-@pytest.mark.parametrize("case", GRAD_CASES + WGRAD_ONLY)
+@pytest.mark.parametrize("case", GRAD_CASES + STRIDED)
 def test_wgrad_integer_inputs_bit_exact(case, pair, scratch):
     sg.enable_scratch(scratch)
     sg.set_tuning(-1, pair)
@@ -118,10 +124,12 @@ def test_grads_are_adjoint_to_the_forward_kernel_on_the_gpu():
 
 
 def test_grad_argument_errors_and_empty_sums():
-    dY = torch.zeros((1, 4, 4, 64), dtype=torch.bfloat16, device=DEV)
     Wf = torch.zeros((64, 3, 3, 64), dtype=torch.bfloat16, device=DEV)
     with pytest.raises(sg.SolgemmError, match="SG_ERR_UNSUPPORTED"):
-        sg.conv2d_dgrad(dY, Wf, (8, 8), pad=(1, 1), stride=(2, 2))
+        sg.conv2d_dgrad(torch.zeros((1, 1, 1, 64), dtype=torch.bfloat16, device=DEV), Wf, (9, 9), stride=(9, 9))
+    with pytest.raises(sg.SolgemmError, match="SG_ERR_INVALID_ARG"):
+        sg.conv2d_wgrad(torch.zeros((1, 4, 4, 64), dtype=torch.bfloat16, device=DEV),
+                        torch.zeros((1, 4, 4, 64), dtype=torch.bfloat16, device=DEV), (3, 3), pad=(1, 1), dil=(0, 1))
     # an image smaller than the filter has no output pixels: the gradients are beta * Cin
     X = inputs.normal([1, 2, 2, 64], 35, 1).to(DEV)
     dY0 = torch.zeros((1, 0, 0, 64), dtype=torch.bfloat16, device=DEV)
@@ -146,3 +154,16 @@ def test_wgrad_long_pixel_contraction_is_cut_into_k_ranges():
     ref, mag = orc.conv2d_wgrad(dYr, Xr, (R, S), pad=pad)
     out = sg.conv2d_wgrad(dYr.to(DEV), Xr.to(DEV), (R, S), pad=pad)
     parity.assert_matches(out.reshape(-1, C), ref.reshape(-1, C), mag.reshape(-1, C), "wgrad k ranges real")
+
+
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_strided_dgrad_real_values_with_residual(out_dtype):
+    # stride 2: four launches, each writing its own pixels of dX (and reading the same pixels of Cin)
+    case = (2, 19, 18, 72, 80, 3, 3, (1, 1), (2, 2), (1, 1))
+    N_, H, W, C, K, R, S, pad, stride, dil = case
+    X, Wf, dY = _problem(case, 38, False)
+    Cx = inputs.normal([N_, H, W, C], 38, 5).to(out_dtype)
+    ref, mag = orc.conv2d_dgrad(dY, Wf, (H, W), pad=pad, stride=stride, Cin=Cx, alpha=1.5, beta=0.5)
+    out = torch.full((N_, H, W, C), float("nan"), dtype=out_dtype, device=DEV)
+    sg.conv2d_dgrad(dY.to(DEV), Wf.to(DEV), (H, W), pad=pad, stride=stride, Cin=Cx.to(DEV), alpha=1.5, beta=0.5, out=out)
+    parity.assert_matches(out.reshape(-1, C), ref.reshape(-1, C), mag.reshape(-1, C), "strided dgrad")
