@@ -333,6 +333,55 @@ def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
     return out
 
 
+def profile_config(args) -> None:
+    """A few kernel-only launches of one of the configurations c3, c4, c5 inside a cudaProfilerStart/Stop bracket, so that
+    `ncu --profile-from-start off` captures that configuration's kernel alone (the default run profiles c2)."""
+    import torch
+    from paper_2603_29010_b200 import inputs, solgemm as sg
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    C = inputs.CONFIGS
+    name = {"c3": "c3_batched_128x256x256x512_gelu", "c4": "c4_conv_32x56x56x256_k256_3x3_bias_relu",
+            "c5": "c5_grouped_16xMx4096x4096_silu"}[args.profile_config]
+    c = C[name]
+    if args.profile_config == "c3":
+        sets = 4
+        data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev, batch=c["batch"]) for i in range(sets)]
+        outs = [torch.empty(c["batch"], c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        step = lambda i: sg.batched_gemm(data[i % sets][0], data[i % sets][1], out=outs[i % sets], epi=c["epi"])
+    elif args.profile_config == "c4":
+        sets = 4
+        data = [inputs.make_conv(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["dist"], c["scale"], bias=True, seed=i,
+                                 device=dev) for i in range(sets)]
+        outs = [torch.empty(c["N"], 56, 56, c["K"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        step = lambda i: sg.conv2d_fprop(data[i % sets][0], data[i % sets][1], pad=c["pad"], bias=data[i % sets][2],
+                                         out=outs[i % sets], epi=c["epi"])
+    else:
+        Ms = inputs.grouped_sizes(c["groups"], c["M_lo"], c["M_hi"])
+        As, Bs = inputs.make_grouped(Ms, c["N"], c["K"], c["dist"], c["scale"], device=dev)
+        outs = [torch.empty(m, c["N"], dtype=torch.bfloat16, device=dev) for m in Ms]
+        ws = torch.empty(sg.grouped_workspace_size(len(Ms)), dtype=torch.uint8, device=dev)
+        step = lambda i: sg.grouped_gemm(As, Bs, outs=outs, epi=c["epi"], workspace=ws)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than L2: every timed launch starts cold
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    times = []
+    torch.cuda.profiler.start()
+    for i in range(args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step(i)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3)
+    torch.cuda.profiler.stop()
+    sg.poll_status()
+    print(json.dumps({"profile_config": name, "launches": args.steps, "us_per_launch_single_cold": times,
+                      "plan": sg.last_launch_plan()}), flush=True)
+
+
 def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     import torch
     import torch.distributed as dist
@@ -500,6 +549,8 @@ def main() -> None:
     ap.add_argument("--widened", action="store_true",
                     help="also time the rows built beyond the five configurations (epilogue chain, dtypes, layouts, "
                          "skinny shapes, transpose, conv gradients; N=1 only)")
+    ap.add_argument("--profile-config", choices=["c3", "c4", "c5"], default=None,
+                    help="only run a few launches of that configuration inside the profiler bracket (for ncu)")
     ap.add_argument("--torch-ref", action="store_true", help="with --all-configs: also time torch's library kernels")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernel)")
@@ -514,6 +565,11 @@ def main() -> None:
         cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
                "--master-addr", "127.0.0.1", "--master-port", port, os.path.abspath(__file__)] + sys.argv[1:]
         sys.exit(subprocess.call(cmd))
+    if args.profile_config:
+        if world > 1 or args.impl != "ours":
+            raise SystemExit("--profile-config is a single-GPU mode of the CUDA arm")
+        profile_config(args)
+        return
     if args.impl == "reference":
         if args.steps < 1:
             args.steps = 1
