@@ -455,27 +455,60 @@ def conv1d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=0, stride=1, dil=1, *
     return y.view(n, y.shape[2], k)
 
 
+_side_streams = {}      # device index -> (copy-in stream, copy-out stream)
+
+
 def gemm_host(A_host: torch.Tensor, B_host: torch.Tensor, out_host: torch.Tensor, *, bias_host=None, epi="none",
-              alpha=1.0, device="cuda", scratch: Optional[dict] = None, stream=None) -> torch.Tensor:
+              alpha=1.0, device="cuda", scratch: Optional[dict] = None, stream=None, chunks: int = 4) -> torch.Tensor:
     """End-to-end GEMM for callers whose data lives in (pinned) host memory.
 
-    Copies A, B (and bias) to the device, runs ``sg_gemm`` and copies D back into ``out_host``,
-    all on one stream.  ``scratch`` may hold preallocated device buffers ("A", "B", "bias", "D").
+    Copies A, B (and bias) to the device, runs ``sg_gemm`` and copies D back into ``out_host``.  The rows of A and D
+    are cut into ``chunks`` blocks: while the copy engine brings in block i+1, the kernel works on block i and the
+    other copy engine takes block i-1 of D back, so the call costs about the larger of the two transfers instead of
+    their sum.  Everything is ordered against ``stream`` (default: the current stream): the call starts after the
+    work already on it and the stream continues only when ``out_host`` is complete.  ``scratch`` may hold
+    preallocated device buffers ("A", "B", "bias", "D"); it is filled on first use.
     """
     scratch = {} if scratch is None else scratch
-    dev = {}
-    for name, t in (("A", A_host), ("B", B_host), ("bias", bias_host)):
-        if t is None:
-            dev[name] = None
-            continue
-        if name not in scratch:
-            scratch[name] = torch.empty(t.shape, dtype=t.dtype, device=device)
-        scratch[name].copy_(t, non_blocking=True)
-        dev[name] = scratch[name]
-    if "D" not in scratch:
-        scratch["D"] = torch.empty(out_host.shape, dtype=out_host.dtype, device=device)
-    gemm(dev["A"], dev["B"], bias=dev["bias"], out=scratch["D"], alpha=alpha, epi=epi, stream=stream)
-    out_host.copy_(scratch["D"], non_blocking=True)
+    dev = torch.device(device)
+    if dev.index is None:
+        dev = torch.device("cuda", torch.cuda.current_device())
+    main = torch.cuda.current_stream(dev) if stream is None else stream
+    for name, t in (("A", A_host), ("B", B_host), ("bias", bias_host), ("D", out_host)):
+        if t is not None and name not in scratch:
+            scratch[name] = torch.empty(t.shape, dtype=t.dtype, device=dev)
+    if dev.index not in _side_streams:
+        _side_streams[dev.index] = (torch.cuda.Stream(dev), torch.cuda.Stream(dev))
+    s_in, s_out = _side_streams[dev.index]
+    M = A_host.shape[0]
+    rows = max(256, -(-M // max(chunks, 1) // 256) * 256)        # block height: a multiple of the 256-row tile
+    blocks = [(r, min(r + rows, M)) for r in range(0, M, rows)]
+    fork = torch.cuda.Event()
+    fork.record(main)
+    s_in.wait_event(fork)           # the device buffers may still be in use by work enqueued before this call
+    s_out.wait_event(fork)
+    arrived = []
+    with torch.cuda.stream(s_in):
+        scratch["B"].copy_(B_host, non_blocking=True)
+        if bias_host is not None:
+            scratch["bias"].copy_(bias_host, non_blocking=True)
+        for r0, r1 in blocks:
+            scratch["A"][r0:r1].copy_(A_host[r0:r1], non_blocking=True)
+            ev = torch.cuda.Event()
+            ev.record(s_in)
+            arrived.append(ev)
+    for (r0, r1), ev in zip(blocks, arrived):
+        main.wait_event(ev)
+        gemm(scratch["A"][r0:r1], scratch["B"], bias=scratch.get("bias") if bias_host is not None else None,
+             out=scratch["D"][r0:r1], alpha=alpha, epi=epi, stream=main)
+        done = torch.cuda.Event()
+        done.record(main)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(done)
+            out_host[r0:r1].copy_(scratch["D"][r0:r1], non_blocking=True)
+    back = torch.cuda.Event()
+    back.record(s_out)
+    main.wait_event(back)
     return out_host
 
 

@@ -604,3 +604,18 @@ def test_fp8_real_values_epilogue_batched_grouped_and_conv():
     parity.assert_bit_exact(sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1)), ref, "fp8 conv")
     with pytest.raises(sg.SolgemmError):                       # only the K-contiguous layouts with 8-bit inputs
         sg.gemm(A.to(DEV), torch.zeros(K, N, device=DEV).to(dt), layout_b="row")
+
+
+@pytest.mark.parametrize("M,chunks", [(1000, 8), (256, 8), (2304, 3), (64, 1)])
+def test_gemm_host_pipelined_copies_match_the_oracle(M, chunks):
+    N, K = 264, 200
+    A, B, bias = inputs.make_gemm(M, N, K, "uniform", 1.0, bias=True, seed=61)
+    ref, absacc = orc.gemm(A, B, bias=bias, epi="relu")
+    hA, hB, hb = A.pin_memory(), B.pin_memory(), bias.pin_memory()
+    hD = torch.full((M, N), float("nan"), dtype=torch.bfloat16).pin_memory()
+    scratch = {}
+    for _ in range(2):                      # the second call reuses the device buffers of the first
+        hD.fill_(float("nan"))
+        sg.gemm_host(hA, hB, hD, bias_host=hb, epi="relu", scratch=scratch, chunks=chunks)
+        torch.cuda.current_stream().synchronize()
+        parity.assert_matches(hD, ref, absacc, f"gemm_host M={M} chunks={chunks}")
