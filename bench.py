@@ -177,7 +177,7 @@ def time_steps(fn, steps: int, torch) -> float:
     return start.elapsed_time(stop) * 1e-3
 
 
-def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int) -> dict:
+def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int, torch_ref: bool = False) -> dict:
     """Kernel-only timings of the other four configurations (reported inside the one JSON line)."""
     out = {}
     hw = dict(peak_flops=peaks["bf16_tflops"] * 1e12, peak_bytes_per_s=peaks["hbm_gbs"] * 1e9)
@@ -211,18 +211,19 @@ def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int) -> dict:
     C = inputs.CONFIGS
     c = C["c1_gemm_256"]
     sets = 64
-    data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev) for i in range(4)]
+    data_c1 = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev) for i in range(4)]
     outs = [torch.empty(c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
-    record("c1_gemm_256", lambda i: (lambda: sg.gemm(data[i % 4][0], data[i % 4][1], out=outs[i])), sets,
+    record("c1_gemm_256", lambda i: (lambda: sg.gemm(data_c1[i % 4][0], data_c1[i % 4][1], out=outs[i])), sets,
            dict(op="gemm", M=c["M"], N=c["N"], K=c["K"]), max(steps, 200))
 
     c = C["c3_batched_128x256x256x512_gelu"]
     sets = 8      # 8 x 84 MB > L2
-    data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev, batch=c["batch"])
-            for i in range(sets)]
-    outs = [torch.empty(c["batch"], c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+    data_c3 = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev, batch=c["batch"])
+               for i in range(sets)]
+    outs3 = [torch.empty(c["batch"], c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+    c3 = c
     record("c3_batched_128x256x256x512_gelu",
-           lambda i: (lambda: sg.batched_gemm(data[i][0], data[i][1], out=outs[i], epi=c["epi"])), sets,
+           lambda i: (lambda: sg.batched_gemm(data_c3[i][0], data_c3[i][1], out=outs3[i], epi=c3["epi"])), sets,
            dict(op="batched", M=c["M"], N=c["N"], K=c["K"], batch_or_groups=c["batch"]), max(steps, 200))
 
     c4 = C["c4_conv_32x56x56x256_k256_3x3_bias_relu"]
@@ -245,6 +246,30 @@ def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int) -> dict:
            lambda i: (lambda: sg.grouped_gemm(As, Bs, outs=outs5, epi=c5["epi"], workspace=ws)), 1,
            dict(op="grouped", N=c5["N"], K=c5["K"], batch_or_groups=len(Ms), Ms=Ms), max(steps // 10, 20))
     out["c5_grouped_16xMx4096x4096_silu"]["M_i"] = Ms
+    if torch_ref:
+        # the same problems through torch's library kernels (separate epilogue kernels where torch has no fusion):
+        # context for the table, not a target
+        import torch.nn.functional as F
+
+        def lib_time(name, fn, reps):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fn()
+            graph.replay()
+            torch.cuda.synchronize()
+            out[name]["torch_library_us"] = time_steps(lambda i: graph.replay(), reps, torch) / reps * 1e6
+
+        a1, b1 = data_c1[0][0], data_c1[0][1]
+        lib_time("c1_gemm_256", lambda: torch.matmul(a1, b1.t()), 200)
+        a3, b3 = data_c3[0][0], data_c3[0][1]
+        lib_time("c3_batched_128x256x256x512_gelu", lambda: F.gelu(torch.bmm(a3, b3.transpose(1, 2)), approximate="tanh"), 100)
+        x4 = data4[0][0].permute(0, 3, 1, 2)                      # NCHW view of the NHWC buffer = channels_last
+        w4 = data4[0][1].permute(0, 3, 1, 2)
+        lib_time("c4_conv_32x56x56x256_k256_3x3_bias_relu", lambda: torch.relu(F.conv2d(x4, w4, data4[0][2], padding=1)), 50)
+        lib_time("c5_grouped_16xMx4096x4096_silu", lambda: [F.silu(a @ b.t()) for a, b in zip(As, Bs)], 10)
     return out
 
 
@@ -524,7 +549,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         if args.widened:
             line["widened"] = bench_widened(sg, inputs, torch, dev, peaks)
         if args.all_configs:
-            line["per_config"] = bench_extra_configs(sg, inputs, torch, dev, peaks, args.steps)
+            line["per_config"] = bench_extra_configs(sg, inputs, torch, dev, peaks, args.steps, args.torch_ref)
             if args.torch_ref:
                 A, B, bias = data[0]
                 f = lambda i: torch.relu(torch.addmm(bias, data[i % sets][0], data[i % sets][1].t()))
