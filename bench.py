@@ -355,6 +355,17 @@ def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
     timed("conv2d_wgrad_32x56x56x256_k256_3x3_fp32_dW",
           [(lambda i=i: sg.conv2d_wgrad(dY[i], X[i], (3, 3), pad=(1, 1), out=dW)) for i in range(4)],
           dict(op="conv2d_wgrad", conv=geo, elem_bytes_out=4))
+    # a strided layer: 32x56x56x256 -> 512 filters 3x3 stride 2 (output 28x28)
+    geo2 = dict(N=32, H=56, W=56, C=256, K=512, R=3, S=3, pad=(1, 1), stride=(2, 2))
+    dY2 = [inputs.normal([32, 28, 28, 512], 80 + i, 3, device=dev) for i in range(4)]
+    Wf2 = inputs.normal([512, 3, 3, 256], 80, 2, 1 / 48., device=dev)
+    dW2 = torch.empty(512, 3, 3, 256, dtype=torch.float32, device=dev)
+    timed("conv2d_dgrad_32x56x56x256_k512_3x3_stride2",
+          [(lambda i=i: sg.conv2d_dgrad(dY2[i], Wf2, (56, 56), pad=(1, 1), stride=(2, 2), out=dX[i])) for i in range(4)],
+          dict(op="conv2d_dgrad", conv=geo2), note="four output phases in one launch")
+    timed("conv2d_wgrad_32x56x56x256_k512_3x3_stride2_fp32_dW",
+          [(lambda i=i: sg.conv2d_wgrad(dY2[i], X[i], (3, 3), pad=(1, 1), stride=(2, 2), out=dW2)) for i in range(4)],
+          dict(op="conv2d_wgrad", conv=geo2, elem_bytes_out=4))
     return out
 
 

@@ -10,6 +10,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <algorithm>
 #include <vector>
 
 #include "solgemm.h"
@@ -375,7 +376,7 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
 // cut into `split` column slices so that the idle SMs of that wave take a share.  Narrow slices cost more
 // per output area (same factors as in choose_shape), so a split is used only when it shortens the tail.
 // Sets p->split_begin, p->split and p->num_tiles (the length of the tile list) from the full-width count.
-void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1) {
+void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1, bool allow_ksplit = true) {
     const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
     int best_split = 1, best_ksplit = 1;
@@ -404,7 +405,7 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
         // fp32 partial sums and finishes a share of the tile's columns from all parts' sums (this is also what serves
         // skinny problems with a long K: when there is less than one wave of tiles, every tile is a "tail" tile).
         // A k-block of a tile takes about 0.25 us; a split is planned when it saves a fifth of the tail's time.
-        if (d.scratch && forced_k != 0 && p->num_kb >= 2 && rem * 2 <= slots) {
+        if (allow_ksplit && d.scratch && forced_k != 0 && p->num_kb >= 2 && rem * 2 <= slots) {
             int64_t ks_max = slots / rem;
             if (ks_max > 16) ks_max = 16;
             if (ks_max > p->num_kb) ks_max = p->num_kb;
@@ -1152,6 +1153,105 @@ extern "C" sg_status_t sg_conv2d_dgrad(const sg_conv2d_desc_t* desc, const void*
     DeviceState* d = nullptr;
     st = device_state(&d);
     if (st != SG_OK) return st;
+    if (strided && !no_sum && phases.size() >= 2 && phases.size() <= static_cast<size_t>(kMaxPhases)) {
+        // All phases in one launch: their tiles are one list (longest K loops first), so the phases share the waves
+        // of the machine instead of each paying its own partial last wave and its own launch.
+        std::vector<size_t> order(phases.size());
+        for (size_t i = 0; i < order.size(); ++i) order[i] = i;
+        std::sort(order.begin(), order.end(), [&](size_t x, size_t y) {
+            const int64_t kx = static_cast<int64_t>(phases[x].first.taps) * phases[x].second.taps;
+            const int64_t ky = static_cast<int64_t>(phases[y].first.taps) * phases[y].second.taps;
+            return kx != ky ? kx > ky : x < y;
+        });
+        std::vector<int64_t> rows;
+        int64_t k_sum = 0;
+        for (size_t i : order) {
+            rows.push_back(desc->N * phases[i].first.out_n * phases[i].second.out_n);
+            k_sum += desc->K * std::max<int64_t>(1, static_cast<int64_t>(phases[i].first.taps) * phases[i].second.taps);
+        }
+        Params p;
+        base_params(&p, *d, desc->alpha, desc->beta, desc->epi, 0.0f, 0.0f);
+        p.in_f16 = c.in_f16 ? 1 : 0;
+        p.bk_elems = c.bk;
+        Shape s = choose_shape(*d, rows, 1, desc->C, k_sum / static_cast<int64_t>(order.size()), 64);
+        const int tile_m = s.pair ? 256 : 128;
+        p.mode = MODE_CONV;
+        p.b_mn_major = 1;
+        p.filt_s = static_cast<int32_t>(desc->S);
+        p.N = static_cast<int32_t>(desc->C);
+        p.batch = 1;
+        p.tiles_m = 1;
+        p.tiles_n = static_cast<int32_t>((desc->C + s.bn - 1) / s.bn);
+        p.cblocks = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
+        p.stride_h = 1; p.stride_w = 1;
+        p.d_remap = 1;
+        p.remap_sh = desc->stride_h; p.remap_sw = desc->stride_w;
+        p.remap_H = static_cast<int32_t>(desc->H); p.remap_W = static_cast<int32_t>(desc->W);
+        p.C = desc->beta != 0.0f ? Cin : nullptr;
+        p.ldc = desc->C;
+        p.D = dX;
+        p.ldd = desc->C;
+        st = make_tiled_map(&p.tmD, c.tm_out, c.esize_out, dX, desc->C, desc->N * desc->H * desc->W, 1, desc->C, 0,
+                            c.f32_out ? 32 : 64, 32, "dX");
+        if (st != SG_OK) return st;
+        p.nphases = static_cast<int32_t>(order.size());
+        int64_t tiles = 0;
+        for (size_t j = 0; j < order.size(); ++j) {
+            const PhaseDim& ph = phases[order[j]].first;
+            const PhaseDim& pw = phases[order[j]].second;
+            ConvPhase& f = p.ph[j];
+            const int64_t taps = static_cast<int64_t>(ph.taps) * pw.taps;
+            f.tile_start = static_cast<int32_t>(tiles);
+            f.M = static_cast<int32_t>(rows[j]);
+            f.num_kb = static_cast<int32_t>(taps * p.cblocks);
+            f.P = static_cast<int32_t>(ph.out_n); f.Q = static_cast<int32_t>(pw.out_n);
+            f.pad_h = static_cast<int32_t>(-ph.lower); f.pad_w = static_cast<int32_t>(-pw.lower);
+            f.dil_h = ph.dd; f.dil_w = pw.dd;
+            f.S = pw.taps > 0 ? pw.taps : 1;
+            f.tapb_r0 = ph.tap_hi; f.tapb_rs = -ph.tap_step;
+            f.tapb_s0 = pw.tap_hi; f.tapb_ss = -pw.tap_step;
+            f.remap_h0 = phase_ab[order[j]].first; f.remap_w0 = phase_ab[order[j]].second;
+            f.div_pq = make_fastdiv(ph.out_n * pw.out_n);
+            f.div_q = make_fastdiv(pw.out_n);
+            tiles += ((rows[j] + tile_m - 1) / tile_m) * p.tiles_n;
+            if (f.num_kb > p.num_kb) p.num_kb = f.num_kb;
+            if (f.M > p.M) p.M = f.M;
+            if (taps == 0) {
+                p.tmPh[j] = p.tmD;
+                continue;
+            }
+            cuuint64_t dims[4] = {static_cast<cuuint64_t>(desc->K), static_cast<cuuint64_t>(Q), static_cast<cuuint64_t>(P),
+                                  static_cast<cuuint64_t>(desc->N)};
+            const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
+            cuuint64_t strides[3] = {static_cast<cuuint64_t>(desc->K) * es, static_cast<cuuint64_t>(Q * desc->K) * es,
+                                     static_cast<cuuint64_t>(P * Q * desc->K) * es};
+            int lower[2] = {static_cast<int>(pw.lower), static_cast<int>(ph.lower)};
+            int upper[2] = {static_cast<int>(pw.out_n - Q + pw.lower), static_cast<int>(ph.out_n - P + ph.lower)};
+            cuuint32_t estr[4] = {1, 1, 1, 1};
+            CUresult r = g_encode_im2col(&p.tmPh[j], c.tm_in, 4, const_cast<void*>(dY), dims, strides, lower, upper,
+                                         static_cast<cuuint32_t>(c.bk), 128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeIm2col(dY) failed with CUresult %d", static_cast<int>(r));
+        }
+        if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
+        p.K = p.num_kb * c.bk;
+        p.tmA = p.tmPh[0];
+        {
+            const cuuint64_t es = static_cast<cuuint64_t>(c.esize_in);
+            cuuint64_t fdims[3] = {static_cast<cuuint64_t>(desc->C), static_cast<cuuint64_t>(desc->R * desc->S),
+                                   static_cast<cuuint64_t>(desc->K)};
+            cuuint64_t fstrides[2] = {static_cast<cuuint64_t>(desc->C) * es, static_cast<cuuint64_t>(desc->C * desc->R * desc->S) * es};
+            cuuint32_t box[3] = {64, 1, 64};
+            cuuint32_t e3[3] = {1, 1, 1};
+            CUresult r = g_encode_tiled(&p.tmB, c.tm_in, 3, const_cast<void*>(Wf), fdims, fstrides, box, e3, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(Wf) failed with CUresult %d", static_cast<int>(r));
+            p.tmB2 = p.tmB;
+        }
+        plan_tail(*d, s, tiles, &p, 64, false);
+        return launch(*d, s, c.out_kind, p, static_cast<cudaStream_t>(cuda_stream));
+    }
     for (size_t i = 0; i < phases.size(); ++i) {
         const PhaseDim& ph = phases[i].first;
         const PhaseDim& pw = phases[i].second;

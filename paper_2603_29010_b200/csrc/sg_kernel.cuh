@@ -38,6 +38,18 @@ __device__ __forceinline__ int fast_div(int n, FastDiv d) {
     return static_cast<int>((static_cast<uint64_t>(static_cast<uint32_t>(n)) * d.mul) >> d.sh);
 }
 
+// One output phase of a strided convolution data gradient run inside one launch (see sg_conv2d_dgrad): the phases are
+// consecutive ranges of the tile list, each with its own rows, K loop, im2col window and pixel map.
+struct ConvPhase {
+    int32_t tile_start;                 // first (full-width) tile of the phase in the tile list
+    int32_t M, num_kb;                  // rows (pixels of the phase) and k-blocks (taps x channel blocks)
+    int32_t P, Q, pad_h, pad_w, dil_h, dil_w, S;
+    int32_t tapb_r0, tapb_rs, tapb_s0, tapb_ss;
+    int32_t remap_h0, remap_w0;
+    FastDiv div_pq, div_q;
+};
+constexpr int kMaxPhases = 4;
+
 struct alignas(64) Params {
     CUtensorMap tmA, tmB, tmD;          // dense / batched / conv operands (3-D; conv A is a 4-D im2col map)
     CUtensorMap tmB2;                   // B with the narrower box of split tail tiles
@@ -81,6 +93,9 @@ struct alignas(64) Params {
     // conv (strided data gradient): row m = (n, i, j) of this launch's output is pixel (n, remap_h0 + remap_sh * i,
     // remap_w0 + remap_sw * j) of the remap_H x remap_W image that C and D address; 0 = rows are stored as they come
     int32_t d_remap, remap_h0, remap_sh, remap_w0, remap_sw, remap_H, remap_W;
+    int32_t nphases;                    // > 1: the tile list is the concatenation of ph[0 .. nphases), A maps in tmPh
+    ConvPhase ph[kMaxPhases];
+    CUtensorMap tmPh[kMaxPhases];
     // extended epilogue chain (all optional; ex_any = 1 when any of them is in use; dense and conv modes only):
     //   t = alpha acc * row_scale[i] * col_scale[j] + beta C + bias[j] + row_bias[i];  aux_store[i][j] = t;
     //   D = post_scale * act(t) + aux_load[i][j]
@@ -141,6 +156,26 @@ struct Tile {
     int part, nparts, tail;       // K-split: this item is part `part` of `nparts` sharing the tile's K range; index of the tail tile
 };
 
+// The convolution geometry a tile works with: the launch's own, or its phase's.
+struct ConvView {
+    int P, Q, pad_h, pad_w, dil_h, dil_w, S, tapb_r0, tapb_rs, tapb_s0, tapb_ss, remap_h0, remap_w0;
+    FastDiv div_pq, div_q;
+};
+__device__ __forceinline__ ConvView conv_view(const Params& p, int phase) {
+    ConvView v;
+    if (p.nphases > 1) {
+        const ConvPhase& f = p.ph[phase];
+        v.P = f.P; v.Q = f.Q; v.pad_h = f.pad_h; v.pad_w = f.pad_w; v.dil_h = f.dil_h; v.dil_w = f.dil_w; v.S = f.S;
+        v.tapb_r0 = f.tapb_r0; v.tapb_rs = f.tapb_rs; v.tapb_s0 = f.tapb_s0; v.tapb_ss = f.tapb_ss;
+        v.remap_h0 = f.remap_h0; v.remap_w0 = f.remap_w0; v.div_pq = f.div_pq; v.div_q = f.div_q;
+    } else {
+        v.P = p.P; v.Q = p.Q; v.pad_h = p.pad_h; v.pad_w = p.pad_w; v.dil_h = p.dil_h; v.dil_w = p.dil_w; v.S = p.S;
+        v.tapb_r0 = p.tapb_r0; v.tapb_rs = p.tapb_rs; v.tapb_s0 = p.tapb_s0; v.tapb_ss = p.tapb_ss;
+        v.remap_h0 = p.remap_h0; v.remap_w0 = p.remap_w0; v.div_pq = p.div_pq; v.div_q = p.div_q;
+    }
+    return v;
+}
+
 // Tile r of one problem -> (tile row, tile column).  Tiles are walked in horizontal bands of band_m tile
 // rows; inside a band the walk goes down a column of the band, then to the next column.  The tiles running
 // at the same time then share few A and B panels, and a band's A rows stay in L2 while its columns stream by.
@@ -192,6 +227,16 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         ti.b = g;
         ti.rows = rows;
         raster(p, t - p.g_tile_start[g], (rows + TILE_M - 1) / TILE_M, tm, tn);
+    } else if (p.nphases > 1) {
+        int ph = 0;
+        while (ph + 1 < p.nphases && t >= p.ph[ph + 1].tile_start) ++ph;
+        const int local = t - p.ph[ph].tile_start;
+        ti.b = ph;
+        ti.rows = p.ph[ph].M;
+        ti.kb1 = p.ph[ph].num_kb;
+        const int tm_count = (ti.rows + TILE_M - 1) / TILE_M;
+        tn = local / tm_count;                  // down a column of tiles, then the next column
+        tm = local - tn * tm_count;
     } else {
         const int per = p.tiles_m * p.tiles_n;
         ti.b = fast_div(t, p.div_per);
@@ -520,22 +565,25 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     }
                 }
                 int cw = 0, ch = 0, cn = 0;
+                ConvView cv = {};
                 if (p.mode == MODE_CONV) {
-                    const int pq = p.P * p.Q;
-                    cn = fast_div(m0, p.div_pq);
+                    cv = conv_view(p, ti.b);
+                    if (p.nphases > 1) mapA = &p.tmPh[ti.b];
+                    const int pq = cv.P * cv.Q;
+                    cn = fast_div(m0, cv.div_pq);
                     const int rem = m0 - cn * pq;
-                    const int op = fast_div(rem, p.div_q);
-                    const int oq = rem - op * p.Q;
-                    cw = oq * p.stride_w - p.pad_w;
-                    ch = op * p.stride_h - p.pad_h;
+                    const int op = fast_div(rem, cv.div_q);
+                    const int oq = rem - op * cv.Q;
+                    cw = oq * p.stride_w - cv.pad_w;
+                    ch = op * p.stride_h - cv.pad_h;
                 }
                 // conv: filter tap (r, s) and channel block of the current k-block, advanced incrementally
                 int c_tap = 0, c_cb = 0, c_r = 0, c_s = 0;
                 if (p.mode == MODE_CONV) {
                     c_tap = ti.kb0 / p.cblocks;
                     c_cb = ti.kb0 - c_tap * p.cblocks;
-                    c_r = c_tap / p.S;
-                    c_s = c_tap - c_r * p.S;
+                    c_r = c_tap / cv.S;
+                    c_s = c_tap - c_r * cv.S;
                 }
                 // weight gradient: the problem index is the filter tap, the contraction runs over output pixels;
                 // (w_n, w_p, w_q) is the first pixel of the current k-block
@@ -563,11 +611,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
                     if (p.mode == MODE_CONV) {
                         const int c0 = c_cb * bk_elems;
-                        tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(c_s * p.dil_w),
-                                                  static_cast<uint16_t>(c_r * p.dil_h));
+                        tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(c_s * cv.dil_w),
+                                                  static_cast<uint16_t>(c_r * cv.dil_h));
                         if (p.b_mn_major) {
                             // data gradient: the filter [k][tap][c] is read with c contiguous, 64 k x 64 c per box
-                            const int tap_b = (p.tapb_r0 + p.tapb_rs * c_r) * p.filt_s + p.tapb_s0 + p.tapb_ss * c_s;
+                            const int tap_b = (cv.tapb_r0 + cv.tapb_rs * c_r) * p.filt_s + cv.tapb_s0 + cv.tapb_ss * c_s;
                             for (int j = 0; j < b_rows / 64; ++j)
                                 tma_load_3d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, tap_b, c0);
                         } else {
@@ -576,7 +624,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         if (++c_cb == p.cblocks) {
                             c_cb = 0;
                             ++c_tap;
-                            if (++c_s == p.S) { c_s = 0; ++c_r; }
+                            if (++c_s == cv.S) { c_s = 0; ++c_r; }
                         }
                     } else if (p.mode == MODE_WGRAD) {
                         // A = dY^T: [pixels][filters] read with the filter index contiguous; B = the 64 pixels of
@@ -629,6 +677,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
                 const Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
+                if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
                 const bool fp8 = p.in_fp8 != 0;
                 const uint32_t in_fmt = fp8 ? static_cast<uint32_t>(p.in_fp8 - 1) : (p.in_f16 ? 0u : 1u);
                 const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0, in_fmt);
@@ -701,9 +750,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         for (int t = first_tile; t < p.num_tiles && ok; t += tile_step) {
             Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
             if (ti.n0 >= p.N) continue;
+            const bool has_k = num_kb > 0 && ti.kb1 > ti.kb0;   // else the tile is the empty sum: no accumulator is involved
             const int acc = iter & 1;
             const uint32_t acc_phase = (iter >> 1) & 1u;
-            ++iter;
+            if (has_k) ++iter;
             const int n0 = ti.n0;
             const int row0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32;
             const CUtensorMap* mapD = &p.tmD;
@@ -736,7 +786,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 __syncwarp();
             }
-            if (num_kb > 0) {
+            if (has_k) {
                 // one lane polls; the other 31 wait at the warp barrier without issuing instructions
                 uint32_t done = 1;
                 if (lane == 0) done = wait_bar(tfull_bar(acc), acc_phase, p, ROLE_EPILOGUE, t, 200 + acc) ? 1u : 0u;
@@ -753,12 +803,13 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // row of C and D in memory: the row itself, or for a strided data gradient the pixel it stands for
             int64_t mem_row = row;
             if (p.d_remap && row < ti.rows) {
-                const int pq = p.P * p.Q;
-                const int n_img = fast_div(row, p.div_pq);
+                const ConvView cv = conv_view(p, ti.b);
+                const int pq = cv.P * cv.Q;
+                const int n_img = fast_div(row, cv.div_pq);
                 const int rem = row - n_img * pq;
-                const int pi = fast_div(rem, p.div_q);
-                const int pj = rem - pi * p.Q;
-                mem_row = (static_cast<int64_t>(n_img) * p.remap_H + p.remap_h0 + p.remap_sh * pi) * p.remap_W + p.remap_w0 +
+                const int pi = fast_div(rem, cv.div_q);
+                const int pj = rem - pi * cv.Q;
+                mem_row = (static_cast<int64_t>(n_img) * p.remap_H + cv.remap_h0 + p.remap_sh * pi) * p.remap_W + cv.remap_w0 +
                           p.remap_sw * pj;
             }
 
@@ -787,7 +838,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
             }
             const int passes = ksplit_tile ? 2 : 1;
-            if (num_kb > 0 && half >= nchunks && !ksplit_tile) {
+            if (has_k && half >= nchunks && !ksplit_tile) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
                 tc_fence_before_sync();
                 __syncwarp();
@@ -821,7 +872,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int c = half; c < nchunks; c += kStep) {
                 if (ksplit_tile && owned(c) != (pass == 1)) continue;
                 float v[CH];
-                if (num_kb > 0) {
+                if (has_k) {
                     uint32_t r0[32];
                     tmem_ld_32x32(t_row + c * CH, r0);
                     if constexpr (!kOutF32) {
