@@ -80,32 +80,41 @@ struct KernelEntry {
     int threads;
 };
 
-template <int BN, bool kPair, int kOut, int kEpiWarps>
+template <int BN, bool kPair, int kOut, int kEpiWarps, bool kLean>
 KernelEntry entry() {
     using Cfg = Config<BN, kPair, kEpiWarps>;
-    return KernelEntry{contract_kernel<BN, kPair, kOut, kEpiWarps>, Cfg::SMEM_BYTES, Cfg::THREADS};
+    return KernelEntry{contract_kernel<BN, kPair, kOut, kEpiWarps, kLean>, Cfg::SMEM_BYTES, Cfg::THREADS};
 }
 
-template <int BN, int kEpiWarps>
+template <int BN, int kEpiWarps, bool kLean>
 KernelEntry entry_for(bool pair, int out) {
-    if (pair) return out == 1 ? entry<BN, true, 1, kEpiWarps>() : (out == 2 ? entry<BN, true, 2, kEpiWarps>() : entry<BN, true, 0, kEpiWarps>());
-    return out == 1 ? entry<BN, false, 1, kEpiWarps>() : (out == 2 ? entry<BN, false, 2, kEpiWarps>() : entry<BN, false, 0, kEpiWarps>());
+    if (pair)
+        return out == 1 ? entry<BN, true, 1, kEpiWarps, kLean>()
+                        : (out == 2 ? entry<BN, true, 2, kEpiWarps, kLean>() : entry<BN, true, 0, kEpiWarps, kLean>());
+    return out == 1 ? entry<BN, false, 1, kEpiWarps, kLean>()
+                    : (out == 2 ? entry<BN, false, 2, kEpiWarps, kLean>() : entry<BN, false, 0, kEpiWarps, kLean>());
 }
 
-// tile width (64, 128, 256) x CTA pairing x output type (0 bf16, 1 fp32, 2 fp16) x epilogue warps (4 or 8)
-KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps) {
+template <bool kLean>
+KernelEntry kernel_for_lean(int bn, bool pair, int out, int epi_warps) {
     if (epi_warps == 8) {
         switch (bn) {
-            case 64: return entry_for<64, 8>(pair, out);
-            case 128: return entry_for<128, 8>(pair, out);
-            default: return entry_for<256, 8>(pair, out);
+            case 64: return entry_for<64, 8, kLean>(pair, out);
+            case 128: return entry_for<128, 8, kLean>(pair, out);
+            default: return entry_for<256, 8, kLean>(pair, out);
         }
     }
     switch (bn) {
-        case 64: return entry_for<64, 4>(pair, out);
-        case 128: return entry_for<128, 4>(pair, out);
-        default: return entry_for<256, 4>(pair, out);
+        case 64: return entry_for<64, 4, kLean>(pair, out);
+        case 128: return entry_for<128, 4, kLean>(pair, out);
+        default: return entry_for<256, 4, kLean>(pair, out);
     }
+}
+
+// tile width (64, 128, 256) x CTA pairing x output type (0 bf16, 1 fp32, 2 fp16) x epilogue warps (4 or 8) x
+// lean (plain dense problems only, the other modes compiled out) or full
+KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, bool lean = false) {
+    return lean ? kernel_for_lean<true>(bn, pair, out, epi_warps) : kernel_for_lean<false>(bn, pair, out, epi_warps);
 }
 
 sg_status_t device_state(DeviceState** out) {
@@ -152,11 +161,12 @@ sg_status_t device_state(DeviceState** out) {
             for (int i = 0; i < 3 && d.init_status == SG_OK; ++i)
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
                     for (int f32 = 0; f32 < 3 && d.init_status == SG_OK; ++f32)
-                        for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4) {
-                            KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew);
-                            e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
-                            if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
-                        }
+                        for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4)
+                            for (int lean = 0; lean < 2 && d.init_status == SG_OK; ++lean) {
+                                KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew, lean != 0);
+                                e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
+                                if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
+                            }
             if (d.init_status == SG_OK) {
                 // how many 2-CTA clusters fit at once (some GPCs may not pair up all of their SMs)
                 KernelEntry k = kernel_for(256, true, 0, 8);
@@ -473,7 +483,11 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     p.div_band_m = make_fastdiv(p.band_m);
     p.div_pq = make_fastdiv(static_cast<int64_t>(p.P) * p.Q);
     p.div_q = make_fastdiv(p.Q);
-    KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps);
+    // plain dense problems run the lean variant of the kernel (same instructions, the other modes compiled out)
+    static const bool no_lean = getenv("SG_NO_LEAN") && atoi(getenv("SG_NO_LEAN")) != 0;      // experiments
+    const bool lean = !no_lean && p.mode == MODE_DENSE && !p.a_mn_major && !p.b_mn_major && !p.in_fp8 && !p.ex_any &&
+                      p.ksplit <= 1 && !p.d_remap && p.nphases <= 1;
+    KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps, lean);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;
     const int tiles = p.num_tiles < slots ? p.num_tiles : slots;

@@ -190,7 +190,7 @@ __device__ __forceinline__ void raster(const Params& p, int r, int tiles_m, int&
 
 // Position t of the tile list -> tile.  The list holds the full-width tiles of all complete waves first;
 // the tiles of the last, partial wave follow as `split` column slices each, so that more SMs share them.
-template <int TILE_M, int BN>
+template <int TILE_M, int BN, bool kLean = false>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint) {
     Tile ti;
     int sub = 0;
@@ -202,7 +202,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
     ti.tail = 0;
     if (t >= p.split_begin) {
         const int u = t - p.split_begin;
-        if (p.ksplit > 1) {
+        if (!kLean && p.ksplit > 1) {
             // the tile's K range is shared by ksplit work items
             ti.nparts = p.ksplit;
             ti.tail = u / p.ksplit;
@@ -219,7 +219,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         }
     }
     int tm, tn;
-    if (p.mode == MODE_GROUPED) {
+    if (!kLean && p.mode == MODE_GROUPED) {
         int g = g_hint;
         while (t >= p.g_tile_start[g + 1]) ++g;      // tiles are visited in increasing order
         g_hint = g;
@@ -227,7 +227,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         ti.b = g;
         ti.rows = rows;
         raster(p, t - p.g_tile_start[g], (rows + TILE_M - 1) / TILE_M, tm, tn);
-    } else if (p.nphases > 1) {
+    } else if (!kLean && p.nphases > 1) {
         int ph = 0;
         while (ph + 1 < p.nphases && t >= p.ph[ph + 1].tile_start) ++ph;
         const int local = t - p.ph[ph].tile_start;
@@ -417,9 +417,18 @@ struct Config {
 };
 
 // kOut: 0 = bf16 output, 1 = fp32, 2 = fp16 (C, when read, has the output's type)
-template <int BN, bool kPair, int kOut, int kEpiWarps>
+// kLean: the variant for plain dense problems (K-contiguous 16-bit operands, no K ranges, no extended epilogue chain):
+// the other modes and options are compiled out.  The instructions are the same; the code is a quarter smaller, and a
+// launch that runs each piece of code once or twice (c1, c3) spends measurably less time fetching it.
+template <int BN, bool kPair, int kOut, int kEpiWarps, bool kLean = false>
 __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) contract_kernel(const __grid_constant__ Params p) {
     using Cfg = Config<BN, kPair, kEpiWarps>;
+    // options the lean variant folds away at compile time
+    const int32_t mode = kLean ? MODE_DENSE : p.mode;
+    const bool a_mn = kLean ? false : p.a_mn_major != 0;
+    const bool b_mn = kLean ? false : p.b_mn_major != 0;
+    const bool d_remap = kLean ? false : p.d_remap != 0;
+    const bool phased = kLean ? false : p.nphases > 1;
     constexpr int kCtas = Cfg::kCtas;
     constexpr int STAGES = Cfg::STAGES;
     constexpr bool kOutF32 = (kOut == 1);
@@ -486,10 +495,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     // tile's first stages right away, before the rest of the set-up; the producer loop skips those k-blocks.
     int early_kb = 0;
     if constexpr (!kPair) {
-        if (p.mode == MODE_DENSE && !p.a_mn_major && !p.b_mn_major && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
+        if (mode == MODE_DENSE && !a_mn && !b_mn && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
             static_cast<int>(blockIdx.x) < p.num_tiles) {
             int g_hint0 = 0;
-            const Tile t0 = decode_tile<Cfg::TILE_M, BN>(p, static_cast<int>(blockIdx.x), g_hint0);
+            const Tile t0 = decode_tile<Cfg::TILE_M, BN, kLean>(p, static_cast<int>(blockIdx.x), g_hint0);
             if (t0.n0 < p.N) {
                 early_kb = min(STAGES, t0.kb1 - t0.kb0);
                 if (threadIdx.x == 0) {
@@ -510,7 +519,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         tmem_alloc<kPair>(tmem_slot, Cfg::TMEM_COLS);
         tmem_relinquish<kPair>();
     }
-    if (warp == 0 && lane == 0 && p.mode != MODE_GROUPED) {
+    if (warp == 0 && lane == 0 && mode != MODE_GROUPED) {
         prefetch_tensormap(&p.tmA);
         prefetch_tensormap(&p.tmB);
         prefetch_tensormap(&p.tmD);
@@ -542,7 +551,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             uint32_t phase = 0;
             int g_hint = 0, g_fenced = -1;
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
+                Tile ti = decode_tile<Cfg::TILE_M, BN, kLean>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
                 const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
@@ -553,7 +562,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 const CUtensorMap* mapA = &p.tmA;
                 const CUtensorMap* mapB = narrow ? &p.tmB2 : &p.tmB;
                 int bz = ti.b;
-                if (p.mode == MODE_GROUPED) {
+                if (mode == MODE_GROUPED) {
                     mapA = p.gmaps + 4 * ti.b;
                     mapB = mapA + (narrow ? 3 : 1);
                     bz = 0;
@@ -566,9 +575,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 int cw = 0, ch = 0, cn = 0;
                 ConvView cv = {};
-                if (p.mode == MODE_CONV) {
+                if (mode == MODE_CONV) {
                     cv = conv_view(p, ti.b);
-                    if (p.nphases > 1) mapA = &p.tmPh[ti.b];
+                    if (phased) mapA = &p.tmPh[ti.b];
                     const int pq = cv.P * cv.Q;
                     cn = fast_div(m0, cv.div_pq);
                     const int rem = m0 - cn * pq;
@@ -579,7 +588,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 // conv: filter tap (r, s) and channel block of the current k-block, advanced incrementally
                 int c_tap = 0, c_cb = 0, c_r = 0, c_s = 0;
-                if (p.mode == MODE_CONV) {
+                if (mode == MODE_CONV) {
                     c_tap = ti.kb0 / p.cblocks;
                     c_cb = ti.kb0 - c_tap * p.cblocks;
                     c_r = c_tap / cv.S;
@@ -588,7 +597,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 // weight gradient: the problem index is the filter tap, the contraction runs over output pixels;
                 // (w_n, w_p, w_q) is the first pixel of the current k-block
                 int w_n = 0, w_p = 0, w_q = 0;
-                if (p.mode == MODE_WGRAD) {
+                if (mode == MODE_WGRAD) {
                     c_r = ti.b / p.S;
                     c_s = ti.b - c_r * p.S;
                     const int pix = ti.kb0 * Cfg::BK;
@@ -609,11 +618,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     uint32_t fb = full_bar(stage);
                     if constexpr (kPair) fb = map_to_cta(fb, 0);
                     if (leader) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
-                    if (p.mode == MODE_CONV) {
+                    if (mode == MODE_CONV) {
                         const int c0 = c_cb * bk_elems;
                         tma_load_im2col_4d<kPair>(a_dst, mapA, fb, c0, cw, ch, cn, static_cast<uint16_t>(c_s * cv.dil_w),
                                                   static_cast<uint16_t>(c_r * cv.dil_h));
-                        if (p.b_mn_major) {
+                        if (b_mn) {
                             // data gradient: the filter [k][tap][c] is read with c contiguous, 64 k x 64 c per box
                             const int tap_b = (cv.tapb_r0 + cv.tapb_rs * c_r) * p.filt_s + cv.tapb_s0 + cv.tapb_ss * c_s;
                             for (int j = 0; j < b_rows / 64; ++j)
@@ -626,7 +635,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                             ++c_tap;
                             if (++c_s == cv.S) { c_s = 0; ++c_r; }
                         }
-                    } else if (p.mode == MODE_WGRAD) {
+                    } else if (mode == MODE_WGRAD) {
                         // A = dY^T: [pixels][filters] read with the filter index contiguous; B = the 64 pixels of
                         // this k-block shifted by the tap, 64 channels per box (im2col addressing)
 #pragma unroll
@@ -642,7 +651,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                             if (++w_p == p.P) { w_p = 0; ++w_n; }
                         }
                     } else {
-                        if (p.a_mn_major) {
+                        if (a_mn) {
                             // column-major A: boxes of 64 rows of the tile (contiguous) x 64 k, one per 64 tile rows
 #pragma unroll
                             for (int j = 0; j < Cfg::BM / 64; ++j)
@@ -650,7 +659,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         } else {
                             tma_load_3d<kPair>(a_dst, mapA, fb, kb * bk_elems, m0, bz);
                         }
-                        if (p.b_mn_major) {
+                        if (b_mn) {
                             for (int j = 0; j < b_rows / 64; ++j)
                                 tma_load_3d<kPair>(b_dst + j * 8192, mapB, fb, nb0 + j * 64, kb * Cfg::BK, bz);
                         } else {
@@ -671,18 +680,18 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             uint32_t phase = 0;
             int iter = 0;
             int g_hint = 0;
-            const uint64_t a_desc0 = p.a_mn_major ? smem_desc_mn_major_sw128(smem_base) : smem_desc_k_major_sw128(smem_base);
-            const uint64_t b_desc0 = p.b_mn_major ? smem_desc_mn_major_sw128(smem_base + Cfg::A_BYTES)
+            const uint64_t a_desc0 = a_mn ? smem_desc_mn_major_sw128(smem_base) : smem_desc_k_major_sw128(smem_base);
+            const uint64_t b_desc0 = b_mn ? smem_desc_mn_major_sw128(smem_base + Cfg::A_BYTES)
                                                   : smem_desc_k_major_sw128(smem_base + Cfg::A_BYTES);
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                const Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
+                const Tile ti = decode_tile<Cfg::TILE_M, BN, kLean>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
                 if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
-                const bool fp8 = p.in_fp8 != 0;
+                const bool fp8 = kLean ? false : p.in_fp8 != 0;
                 const uint32_t in_fmt = fp8 ? static_cast<uint32_t>(p.in_fp8 - 1) : (p.in_f16 ? 0u : 1u);
-                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, p.a_mn_major != 0, p.b_mn_major != 0, in_fmt);
-                const uint32_t a_step = p.a_mn_major ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
-                const uint32_t b_step = p.b_mn_major ? (2048u >> 4) : (32u >> 4);
+                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, a_mn, b_mn, in_fmt);
+                const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
+                const uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
                 const int acc = iter & 1;
                 const uint32_t acc_phase = (iter >> 1) & 1u;
                 ++iter;
@@ -737,7 +746,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         uint32_t fetch_phase = 0;             // phase of this warp's K-split fetch barrier
         uint16_t* bias_w = reinterpret_cast<uint16_t*>(smem + Cfg::OFF_BIAS) + ew * Cfg::BIAS_SLOTS;   // bf16 bias of its chunks
         constexpr int kMyBiasSlots = ((BN / CH + kStep - 1) / kStep) * CH;     // columns of the chunks one warp handles
-        const bool has_bias = (p.mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
+        const bool has_bias = (mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
         const bool has_c = (p.beta != 0.0f);
         const bool in_f16 = (p.in_f16 != 0);
         const float alpha = p.alpha, beta = p.beta;
@@ -748,7 +757,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         for (int a = 0; a < 2; ++a) tempty_remote[a] = kPair ? map_to_cta(tempty_bar(a), 0) : tempty_bar(a);
 
         for (int t = first_tile; t < p.num_tiles && ok; t += tile_step) {
-            Tile ti = decode_tile<Cfg::TILE_M, BN>(p, t, g_hint);
+            Tile ti = decode_tile<Cfg::TILE_M, BN, kLean>(p, t, g_hint);
             if (ti.n0 >= p.N) continue;
             const bool has_k = num_kb > 0 && ti.kb1 > ti.kb0;   // else the tile is the empty sum: no accumulator is involved
             const int acc = iter & 1;
@@ -761,7 +770,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const uint8_t* c_g = reinterpret_cast<const uint8_t*>(p.C);
             uint8_t* d_g = reinterpret_cast<uint8_t*>(p.D);
             int bz = ti.b;
-            if (p.mode == MODE_GROUPED) {
+            if (mode == MODE_GROUPED) {
                 mapD = p.gmaps + 4 * ti.b + 2;
                 bz = 0;
                 if (has_bias) bias_g = reinterpret_cast<const uint16_t*>(p.g_bias[ti.b]);
@@ -802,7 +811,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const int row = row0 + lane;
             // row of C and D in memory: the row itself, or for a strided data gradient the pixel it stands for
             int64_t mem_row = row;
-            if (p.d_remap && row < ti.rows) {
+            if (d_remap && row < ti.rows) {
                 const ConvView cv = conv_view(p, ti.b);
                 const int pq = cv.P * cv.Q;
                 const int n_img = fast_div(row, cv.div_pq);
@@ -818,7 +827,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // from its own accumulator plus the other parts' parked sums
             // (pass 1), so the exchange is spread over all parts instead of serialised in one.  The unit of ownership
             // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
-            const bool ksplit_tile = ti.nparts > 1;
+            const bool ksplit_tile = kLean ? false : ti.nparts > 1;
             // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
             auto owned_by = [&](int c, int qq) { return (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
             auto owned = [&](int c) { return owned_by(c, q); };
@@ -990,11 +999,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int i = 0; i < CH; ++i) v[i] *= alpha;
                 }
-#ifdef SG_NO_EX
-                constexpr bool ex_any = false;       // experiments: the chain compiled out
-#else
-                const bool ex_any = p.ex_any != 0;
-#endif
+                const bool ex_any = kLean ? false : p.ex_any != 0;
                 if (ex_any) {
                     if (p.row_scale != nullptr) {
                         const float rs = row < ti.rows ? __ldg(p.row_scale + row) : 0.0f;
@@ -1138,7 +1143,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 // last, partial chunk is therefore written with plain stores so nothing beyond column N changes; a
                 // strided data gradient, whose rows are scattered over the image, is always stored this way.
                 constexpr int kElemsPer16B = kOutF32 ? 4 : 8;
-                if (p.d_remap || (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0)) {
+                if (d_remap || (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0)) {
                     if (row < ti.rows) {
                         const int col0 = n0 + c * CH;
                         const int valid = min(CH, p.N - col0);
