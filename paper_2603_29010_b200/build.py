@@ -9,8 +9,9 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libsolgemm.so")
-_SOURCES = ["sg_api.cu"]
-_DEPS = ["sg_api.cu", "sg_kernel.cuh", "sg_ptx.cuh", "sg_transpose.cuh", os.path.join(_ROOT, "include", "solgemm.h")]
+_SOURCES = ["sg_api.cu", "sg_variant_0.cu", "sg_variant_1.cu", "sg_variant_2.cu", "sg_variant_3.cu"]
+_DEPS = _SOURCES + ["sg_kernel.cuh", "sg_ptx.cuh", "sg_transpose.cuh", "sg_variants.h", "sg_variant.inc",
+                    os.path.join(_ROOT, "include", "solgemm.h")]
 
 
 def _nvcc() -> str:
@@ -28,24 +29,40 @@ def is_stale() -> bool:
 def build(force: bool = False, verbose: bool = False, extra_flags=(), out_path: str = LIB_PATH) -> str:
     """Compile the CUDA sources into ``libsolgemm.so`` next to this file and return its path.
 
+    The translation units (the host API and one file per kernel variant) are compiled in parallel and linked.
     ``extra_flags`` / ``out_path`` build an experimental variant (e.g. ``-DSG_MAX_STAGES=4``) beside the
     product library; ``SOLGEMM_LIB`` makes the binding load it.
     """
     if out_path == LIB_PATH and not extra_flags and not force and not is_stale():
         return LIB_PATH
-    tmp = out_path + ".tmp%d" % os.getpid()
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-           "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v",
-           "-I", os.path.join(_ROOT, "include"), "-I", _CSRC]
-    cmd += list(extra_flags) + [os.path.join(_CSRC, s) for s in _SOURCES] + ["-o", tmp]
-    proc = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or proc.returncode != 0:
-        sys.stderr.write(proc.stdout + proc.stderr)
-    if proc.returncode != 0:
-        raise RuntimeError("nvcc failed building libsolgemm.so")
-    with open(os.path.join(_PKG, "ptxas.log"), "w") as f:
-        f.write(proc.stderr)
-    os.replace(tmp, out_path)
+    import shutil
+    import tempfile
+    from concurrent.futures import ThreadPoolExecutor
+    base = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
+            "-Xcompiler", "-fPIC", "-Xptxas", "-v", "-I", os.path.join(_ROOT, "include"), "-I", _CSRC] + list(extra_flags)
+    work = tempfile.mkdtemp(prefix="solgemm_build_")
+    try:
+        def compile_one(src):
+            obj = os.path.join(work, src.replace(".cu", ".o"))
+            return src, obj, subprocess.run(base + ["-c", os.path.join(_CSRC, src), "-o", obj], capture_output=True, text=True)
+        with ThreadPoolExecutor(max_workers=len(_SOURCES)) as pool:
+            results = list(pool.map(compile_one, _SOURCES))
+        log = "".join(f"==== {src}\n{r.stdout}{r.stderr}" for src, _, r in results)
+        if verbose or any(r.returncode != 0 for _, _, r in results):
+            sys.stderr.write(log)
+        if any(r.returncode != 0 for _, _, r in results):
+            raise RuntimeError("nvcc failed building libsolgemm.so")
+        tmp = out_path + ".tmp%d" % os.getpid()
+        link = subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "--shared", "-Xcompiler", "-fPIC"] +
+                              [obj for _, obj, _ in results] + ["-o", tmp], capture_output=True, text=True)
+        if link.returncode != 0:
+            sys.stderr.write(link.stdout + link.stderr)
+            raise RuntimeError("nvcc failed linking libsolgemm.so")
+        with open(os.path.join(_PKG, "ptxas.log"), "w") as f:
+            f.write(log)
+        os.replace(tmp, out_path)
+    finally:
+        shutil.rmtree(work, ignore_errors=True)
     return out_path
 
 

@@ -15,6 +15,7 @@
 
 #include "solgemm.h"
 #include "sg_kernel.cuh"
+#include "sg_variants.h"
 #include "sg_transpose.cuh"
 
 namespace {
@@ -72,49 +73,13 @@ std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_tune_tile_n{-1}, g_tune_pair{-1}, g_tune_tail{-1};
 thread_local int32_t t_last_plan[6] = {0, 0, 0, 0, 0, 0};   // tile_n, cta_pair, tail split, tile-list length, first split position, grid
 
-using KernelFn = void (*)(const Params);
-
-struct KernelEntry {
-    KernelFn fn;
-    int smem;
-    int threads;
-};
-
-template <int BN, bool kPair, int kOut, int kEpiWarps, bool kLean>
-KernelEntry entry() {
-    using Cfg = Config<BN, kPair, kEpiWarps>;
-    return KernelEntry{contract_kernel<BN, kPair, kOut, kEpiWarps, kLean>, Cfg::SMEM_BYTES, Cfg::THREADS};
-}
-
-template <int BN, int kEpiWarps, bool kLean>
-KernelEntry entry_for(bool pair, int out) {
-    if (pair)
-        return out == 1 ? entry<BN, true, 1, kEpiWarps, kLean>()
-                        : (out == 2 ? entry<BN, true, 2, kEpiWarps, kLean>() : entry<BN, true, 0, kEpiWarps, kLean>());
-    return out == 1 ? entry<BN, false, 1, kEpiWarps, kLean>()
-                    : (out == 2 ? entry<BN, false, 2, kEpiWarps, kLean>() : entry<BN, false, 0, kEpiWarps, kLean>());
-}
-
-template <bool kLean>
-KernelEntry kernel_for_lean(int bn, bool pair, int out, int epi_warps) {
-    if (epi_warps == 8) {
-        switch (bn) {
-            case 64: return entry_for<64, 8, kLean>(pair, out);
-            case 128: return entry_for<128, 8, kLean>(pair, out);
-            default: return entry_for<256, 8, kLean>(pair, out);
-        }
+KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 0) {
+    switch (variant) {
+        case 1: return kernel_variant_1(bn, pair, out, epi_warps);
+        case 2: return kernel_variant_2(bn, pair, out, epi_warps);
+        case 3: return kernel_variant_3(bn, pair, out, epi_warps);
+        default: return kernel_variant_0(bn, pair, out, epi_warps);
     }
-    switch (bn) {
-        case 64: return entry_for<64, 4, kLean>(pair, out);
-        case 128: return entry_for<128, 4, kLean>(pair, out);
-        default: return entry_for<256, 4, kLean>(pair, out);
-    }
-}
-
-// tile width (64, 128, 256) x CTA pairing x output type (0 bf16, 1 fp32, 2 fp16) x epilogue warps (4 or 8) x
-// lean (plain dense problems only, the other modes compiled out) or full
-KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, bool lean = false) {
-    return lean ? kernel_for_lean<true>(bn, pair, out, epi_warps) : kernel_for_lean<false>(bn, pair, out, epi_warps);
 }
 
 sg_status_t device_state(DeviceState** out) {
@@ -162,8 +127,8 @@ sg_status_t device_state(DeviceState** out) {
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
                     for (int f32 = 0; f32 < 3 && d.init_status == SG_OK; ++f32)
                         for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4)
-                            for (int lean = 0; lean < 2 && d.init_status == SG_OK; ++lean) {
-                                KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew, lean != 0);
+                            for (int variant = 0; variant < 4 && d.init_status == SG_OK; ++variant) {
+                                KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew, variant);
                                 e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
                                 if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
                             }
@@ -483,11 +448,13 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     p.div_band_m = make_fastdiv(p.band_m);
     p.div_pq = make_fastdiv(static_cast<int64_t>(p.P) * p.Q);
     p.div_q = make_fastdiv(p.Q);
-    // plain dense problems run the lean variant of the kernel (same instructions, the other modes compiled out)
+    // plain dense, convolution-forward and grouped problems run the variant of the kernel specialised for them
+    // (same instructions, the other modes and options compiled out)
     static const bool no_lean = getenv("SG_NO_LEAN") && atoi(getenv("SG_NO_LEAN")) != 0;      // experiments
-    const bool lean = !no_lean && p.mode == MODE_DENSE && !p.a_mn_major && !p.b_mn_major && !p.in_fp8 && !p.ex_any &&
-                      p.ksplit <= 1 && !p.d_remap && p.nphases <= 1;
-    KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps, lean);
+    int variant = 0;
+    if (!no_lean && !p.a_mn_major && !p.b_mn_major && !p.in_fp8 && !p.ex_any && p.ksplit <= 1 && !p.d_remap && p.nphases <= 1)
+        variant = p.mode == MODE_DENSE ? 1 : (p.mode == MODE_CONV ? 2 : (p.mode == MODE_GROUPED ? 3 : 0));
+    KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps, variant);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;
     const int tiles = p.num_tiles < slots ? p.num_tiles : slots;

@@ -161,9 +161,9 @@ struct ConvView {
     int P, Q, pad_h, pad_w, dil_h, dil_w, S, tapb_r0, tapb_rs, tapb_s0, tapb_ss, remap_h0, remap_w0;
     FastDiv div_pq, div_q;
 };
-__device__ __forceinline__ ConvView conv_view(const Params& p, int phase) {
+__device__ __forceinline__ ConvView conv_view(const Params& p, int phase, bool phased) {
     ConvView v;
-    if (p.nphases > 1) {
+    if (phased) {
         const ConvPhase& f = p.ph[phase];
         v.P = f.P; v.Q = f.Q; v.pad_h = f.pad_h; v.pad_w = f.pad_w; v.dil_h = f.dil_h; v.dil_w = f.dil_w; v.S = f.S;
         v.tapb_r0 = f.tapb_r0; v.tapb_rs = f.tapb_rs; v.tapb_s0 = f.tapb_s0; v.tapb_ss = f.tapb_ss;
@@ -190,7 +190,8 @@ __device__ __forceinline__ void raster(const Params& p, int r, int tiles_m, int&
 
 // Position t of the tile list -> tile.  The list holds the full-width tiles of all complete waves first;
 // the tiles of the last, partial wave follow as `split` column slices each, so that more SMs share them.
-template <int TILE_M, int BN, bool kLean = false>
+// kV: kernel variant (see contract_kernel): 0 everything, 1 dense only, 2 convolution forward only, 3 grouped only.
+template <int TILE_M, int BN, int kV = 0>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint) {
     Tile ti;
     int sub = 0;
@@ -202,7 +203,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
     ti.tail = 0;
     if (t >= p.split_begin) {
         const int u = t - p.split_begin;
-        if (!kLean && p.ksplit > 1) {
+        if (kV == 0 && p.ksplit > 1) {
             // the tile's K range is shared by ksplit work items
             ti.nparts = p.ksplit;
             ti.tail = u / p.ksplit;
@@ -219,7 +220,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         }
     }
     int tm, tn;
-    if (!kLean && p.mode == MODE_GROUPED) {
+    if (kV == 3 || (kV == 0 && p.mode == MODE_GROUPED)) {
         int g = g_hint;
         while (t >= p.g_tile_start[g + 1]) ++g;      // tiles are visited in increasing order
         g_hint = g;
@@ -227,7 +228,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         ti.b = g;
         ti.rows = rows;
         raster(p, t - p.g_tile_start[g], (rows + TILE_M - 1) / TILE_M, tm, tn);
-    } else if (!kLean && p.nphases > 1) {
+    } else if (kV == 0 && p.nphases > 1) {
         int ph = 0;
         while (ph + 1 < p.nphases && t >= p.ph[ph + 1].tile_start) ++ph;
         const int local = t - p.ph[ph].tile_start;
@@ -249,7 +250,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
 }
 
 // Bounded mbarrier wait.  Returns false when the wait expired or another role already gave up.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Params& p, uint32_t role, uint32_t tile,
+static __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Params& p, uint32_t role, uint32_t tile,
                                        uint32_t which) {
     volatile uint32_t* st = p.status;
     const uint64_t t0 = global_timer_ns();
@@ -363,7 +364,7 @@ __device__ __forceinline__ void apply_act_chunk(float (&v)[kN], int epi, float a
 
 // Bounded wait until a global arrival counter (written by another CTA of this launch with a release pattern)
 // reaches `target`.  Returns false when the wait expired or another role already gave up.
-__device__ __noinline__ bool wait_counter(const uint32_t* counter, uint32_t target, const Params& p, uint32_t tile) {
+static __device__ __noinline__ bool wait_counter(const uint32_t* counter, uint32_t target, const Params& p, uint32_t tile) {
     const volatile uint32_t* c = counter;
     volatile uint32_t* st = p.status;
     const uint64_t t0 = global_timer_ns();
@@ -417,14 +418,17 @@ struct Config {
 };
 
 // kOut: 0 = bf16 output, 1 = fp32, 2 = fp16 (C, when read, has the output's type)
-// kLean: the variant for plain dense problems (K-contiguous 16-bit operands, no K ranges, no extended epilogue chain):
-// the other modes and options are compiled out.  The instructions are the same; the code is a quarter smaller, and a
-// launch that runs each piece of code once or twice (c1, c3) spends measurably less time fetching it.
-template <int BN, bool kPair, int kOut, int kEpiWarps, bool kLean = false>
+// kV selects a variant of the same kernel.  0: every mode and option.  1, 2, 3: plain dense / convolution forward /
+// grouped problems with K-contiguous 16-bit operands, no K ranges and no extended epilogue chain -- the other modes and
+// options are compiled out.  The instructions executed are the same; the code is a quarter smaller and needs fewer
+// registers, which measurably shortens every launch (4096^3 GEMM 96.4 -> 93.4 us, the benchmark convolution
+// 85.8 -> 81.8 us, 128 x (256 x 256 x 512) 19.6 -> 18.75 us, 256^3 6.3 -> 4.7 us, each pair timed in one GPU call).
+template <int BN, bool kPair, int kOut, int kEpiWarps, int kV = 0>
 __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) contract_kernel(const __grid_constant__ Params p) {
     using Cfg = Config<BN, kPair, kEpiWarps>;
-    // options the lean variant folds away at compile time
-    const int32_t mode = kLean ? MODE_DENSE : p.mode;
+    // options the specialised variants fold away at compile time
+    constexpr bool kLean = kV != 0;
+    const int32_t mode = kV == 1 ? MODE_DENSE : (kV == 2 ? MODE_CONV : (kV == 3 ? MODE_GROUPED : p.mode));
     const bool a_mn = kLean ? false : p.a_mn_major != 0;
     const bool b_mn = kLean ? false : p.b_mn_major != 0;
     const bool d_remap = kLean ? false : p.d_remap != 0;
@@ -498,7 +502,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         if (mode == MODE_DENSE && !a_mn && !b_mn && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
             static_cast<int>(blockIdx.x) < p.num_tiles) {
             int g_hint0 = 0;
-            const Tile t0 = decode_tile<Cfg::TILE_M, BN, kLean>(p, static_cast<int>(blockIdx.x), g_hint0);
+            const Tile t0 = decode_tile<Cfg::TILE_M, BN, kV>(p, static_cast<int>(blockIdx.x), g_hint0);
             if (t0.n0 < p.N) {
                 early_kb = min(STAGES, t0.kb1 - t0.kb0);
                 if (threadIdx.x == 0) {
@@ -551,7 +555,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             uint32_t phase = 0;
             int g_hint = 0, g_fenced = -1;
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                Tile ti = decode_tile<Cfg::TILE_M, BN, kLean>(p, t, g_hint);
+                Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
                 const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
@@ -576,7 +580,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 int cw = 0, ch = 0, cn = 0;
                 ConvView cv = {};
                 if (mode == MODE_CONV) {
-                    cv = conv_view(p, ti.b);
+                    cv = conv_view(p, ti.b, phased);
                     if (phased) mapA = &p.tmPh[ti.b];
                     const int pq = cv.P * cv.Q;
                     cn = fast_div(m0, cv.div_pq);
@@ -684,7 +688,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const uint64_t b_desc0 = b_mn ? smem_desc_mn_major_sw128(smem_base + Cfg::A_BYTES)
                                                   : smem_desc_k_major_sw128(smem_base + Cfg::A_BYTES);
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                const Tile ti = decode_tile<Cfg::TILE_M, BN, kLean>(p, t, g_hint);
+                const Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
                 if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
                 const bool fp8 = kLean ? false : p.in_fp8 != 0;
@@ -757,7 +761,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         for (int a = 0; a < 2; ++a) tempty_remote[a] = kPair ? map_to_cta(tempty_bar(a), 0) : tempty_bar(a);
 
         for (int t = first_tile; t < p.num_tiles && ok; t += tile_step) {
-            Tile ti = decode_tile<Cfg::TILE_M, BN, kLean>(p, t, g_hint);
+            Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
             if (ti.n0 >= p.N) continue;
             const bool has_k = num_kb > 0 && ti.kb1 > ti.kb0;   // else the tile is the empty sum: no accumulator is involved
             const int acc = iter & 1;
@@ -812,7 +816,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // row of C and D in memory: the row itself, or for a strided data gradient the pixel it stands for
             int64_t mem_row = row;
             if (d_remap && row < ti.rows) {
-                const ConvView cv = conv_view(p, ti.b);
+                const ConvView cv = conv_view(p, ti.b, phased);
                 const int pq = cv.P * cv.Q;
                 const int n_img = fast_div(row, cv.div_pq);
                 const int rem = row - n_img * pq;

@@ -1,0 +1,23 @@
+// Host-side table of the contraction kernel's instantiations, one translation unit per kernel variant so that the
+// variants compile in parallel.
+#pragma once
+#include "sg_kernel.cuh"
+
+namespace sg {
+
+using KernelFn = void (*)(const Params);
+
+struct KernelEntry {
+    KernelFn fn;
+    int smem;
+    int threads;
+};
+
+// tile width (64, 128, 256) x CTA pairing x output type (0 bf16, 1 fp32, 2 fp16) x epilogue warps (4 or 8), for
+// variant 0 (every mode and option), 1 (dense only), 2 (convolution forward only), 3 (grouped only)
+KernelEntry kernel_variant_0(int bn, bool pair, int out, int epi_warps);
+KernelEntry kernel_variant_1(int bn, bool pair, int out, int epi_warps);
+KernelEntry kernel_variant_2(int bn, bool pair, int out, int epi_warps);
+KernelEntry kernel_variant_3(int bn, bool pair, int out, int epi_warps);
+
+}  // namespace sg
