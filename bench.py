@@ -42,7 +42,7 @@ SPEC_PEAK_BW = 8000e9          # NVIDIA B200 HBM3e (datasheet)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the
 # ncu capture summarised under profiles/ (read + write of one c2 launch).
-NCU_DRAM_BYTES_PER_LAUNCH = 73_634_048 + 15_962_368   # profiles/contract_kernel_c2_gemm4096_ncu.md
+NCU_DRAM_BYTES_PER_LAUNCH = 73_352_448 + 16_339_456   # profiles/contract_kernel_c2_gemm4096_ncu.md
 
 
 def measured_peaks():
