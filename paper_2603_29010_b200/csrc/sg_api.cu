@@ -78,6 +78,8 @@ KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 
         case 1: return kernel_variant_1(bn, pair, out, epi_warps);
         case 2: return kernel_variant_2(bn, pair, out, epi_warps);
         case 3: return kernel_variant_3(bn, pair, out, epi_warps);
+        case 4: return kernel_variant_4(bn, pair, out, epi_warps);
+        case 5: return kernel_variant_5(bn, pair, out, epi_warps);
         default: return kernel_variant_0(bn, pair, out, epi_warps);
     }
 }
@@ -127,7 +129,7 @@ sg_status_t device_state(DeviceState** out) {
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
                     for (int f32 = 0; f32 < 3 && d.init_status == SG_OK; ++f32)
                         for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4)
-                            for (int variant = 0; variant < 4 && d.init_status == SG_OK; ++variant) {
+                            for (int variant = 0; variant < 6 && d.init_status == SG_OK; ++variant) {
                                 KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew, variant);
                                 e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
                                 if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
@@ -452,8 +454,13 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     // (same instructions, the other modes and options compiled out)
     static const bool no_lean = getenv("SG_NO_LEAN") && atoi(getenv("SG_NO_LEAN")) != 0;      // experiments
     int variant = 0;
-    if (!no_lean && !p.a_mn_major && !p.b_mn_major && !p.in_fp8 && !p.ex_any && p.ksplit <= 1 && !p.d_remap && p.nphases <= 1)
-        variant = p.mode == MODE_DENSE ? 1 : (p.mode == MODE_CONV ? 2 : (p.mode == MODE_GROUPED ? 3 : 0));
+    if (!no_lean && !p.in_fp8) {
+        const bool plain = !p.a_mn_major && !p.b_mn_major && p.ksplit <= 1 && !p.d_remap && p.nphases <= 1;
+        if (p.mode == MODE_DENSE && plain) variant = p.ex_any ? 4 : 1;
+        else if (p.mode == MODE_CONV && plain && !p.ex_any) variant = 2;
+        else if (p.mode == MODE_GROUPED && plain && !p.ex_any) variant = 3;
+        else if (p.mode == MODE_CONV && !p.a_mn_major && p.b_mn_major && p.ksplit <= 1 && !p.ex_any) variant = 5;
+    }
     KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps, variant);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;

@@ -190,7 +190,7 @@ __device__ __forceinline__ void raster(const Params& p, int r, int tiles_m, int&
 
 // Position t of the tile list -> tile.  The list holds the full-width tiles of all complete waves first;
 // the tiles of the last, partial wave follow as `split` column slices each, so that more SMs share them.
-// kV: kernel variant (see contract_kernel): 0 everything, 1 dense only, 2 convolution forward only, 3 grouped only.
+// kV: kernel variant (see contract_kernel).
 template <int TILE_M, int BN, int kV = 0>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint) {
     Tile ti;
@@ -228,7 +228,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
         ti.b = g;
         ti.rows = rows;
         raster(p, t - p.g_tile_start[g], (rows + TILE_M - 1) / TILE_M, tm, tn);
-    } else if (kV == 0 && p.nphases > 1) {
+    } else if ((kV == 0 || kV == 5) && p.nphases > 1) {
         int ph = 0;
         while (ph + 1 < p.nphases && t >= p.ph[ph + 1].tile_start) ++ph;
         const int local = t - p.ph[ph].tile_start;
@@ -418,9 +418,10 @@ struct Config {
 };
 
 // kOut: 0 = bf16 output, 1 = fp32, 2 = fp16 (C, when read, has the output's type)
-// kV selects a variant of the same kernel.  0: every mode and option.  1, 2, 3: plain dense / convolution forward /
-// grouped problems with K-contiguous 16-bit operands, no K ranges and no extended epilogue chain -- the other modes and
-// options are compiled out.  The instructions executed are the same; the code is a quarter smaller and needs fewer
+// kV selects a variant of the same kernel.  0: every mode and option.  The others keep one path and compile the rest
+// out (16-bit operands throughout): 1 dense, 2 convolution forward, 3 grouped -- K-contiguous operands, no K ranges, no
+// extended epilogue chain; 4 dense with the extended chain; 5 convolution data gradient (filter read C-contiguous,
+// phase table and pixel scatter).  (A weight-gradient variant measured no faster than variant 0.)  The instructions executed are the same; the code is a quarter smaller and needs fewer
 // registers, which measurably shortens every launch (4096^3 GEMM 96.4 -> 93.4 us, the benchmark convolution
 // 85.8 -> 81.8 us, 128 x (256 x 256 x 512) 19.6 -> 18.75 us, 256^3 6.3 -> 4.7 us, each pair timed in one GPU call).
 template <int BN, bool kPair, int kOut, int kEpiWarps, int kV = 0>
@@ -428,11 +429,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     using Cfg = Config<BN, kPair, kEpiWarps>;
     // options the specialised variants fold away at compile time
     constexpr bool kLean = kV != 0;
-    const int32_t mode = kV == 1 ? MODE_DENSE : (kV == 2 ? MODE_CONV : (kV == 3 ? MODE_GROUPED : p.mode));
+    const int32_t mode = (kV == 1 || kV == 4) ? MODE_DENSE : ((kV == 2 || kV == 5) ? MODE_CONV : (kV == 3 ? MODE_GROUPED : p.mode));
     const bool a_mn = kLean ? false : p.a_mn_major != 0;
-    const bool b_mn = kLean ? false : p.b_mn_major != 0;
-    const bool d_remap = kLean ? false : p.d_remap != 0;
-    const bool phased = kLean ? false : p.nphases > 1;
+    const bool b_mn = kLean ? kV == 5 : p.b_mn_major != 0;
+    const bool d_remap = (kV == 0 || kV == 5) ? p.d_remap != 0 : false;
+    const bool phased = (kV == 0 || kV == 5) ? p.nphases > 1 : false;
     constexpr int kCtas = Cfg::kCtas;
     constexpr int STAGES = Cfg::STAGES;
     constexpr bool kOutF32 = (kOut == 1);
@@ -831,7 +832,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // from its own accumulator plus the other parts' parked sums
             // (pass 1), so the exchange is spread over all parts instead of serialised in one.  The unit of ownership
             // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
-            const bool ksplit_tile = kLean ? false : ti.nparts > 1;
+            const bool ksplit_tile = kV == 0 ? ti.nparts > 1 : false;
             // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
             auto owned_by = [&](int c, int qq) { return (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
             auto owned = [&](int c) { return owned_by(c, q); };
@@ -1003,7 +1004,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int i = 0; i < CH; ++i) v[i] *= alpha;
                 }
-                const bool ex_any = kLean ? false : p.ex_any != 0;
+                const bool ex_any = (kV == 0 || kV == 4) ? p.ex_any != 0 : false;
                 if (ex_any) {
                     if (p.row_scale != nullptr) {
                         const float rs = row < ti.rows ? __ldg(p.row_scale + row) : 0.0f;

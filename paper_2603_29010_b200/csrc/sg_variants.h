@@ -14,10 +14,13 @@ struct KernelEntry {
 };
 
 // tile width (64, 128, 256) x CTA pairing x output type (0 bf16, 1 fp32, 2 fp16) x epilogue warps (4 or 8), for
-// variant 0 (every mode and option), 1 (dense only), 2 (convolution forward only), 3 (grouped only)
+// variant 0 (every mode and option), 1 dense, 2 convolution forward, 3 grouped, 4 dense with the extended epilogue
+// chain, 5 convolution data gradient
 KernelEntry kernel_variant_0(int bn, bool pair, int out, int epi_warps);
 KernelEntry kernel_variant_1(int bn, bool pair, int out, int epi_warps);
 KernelEntry kernel_variant_2(int bn, bool pair, int out, int epi_warps);
 KernelEntry kernel_variant_3(int bn, bool pair, int out, int epi_warps);
+KernelEntry kernel_variant_4(int bn, bool pair, int out, int epi_warps);
+KernelEntry kernel_variant_5(int bn, bool pair, int out, int epi_warps);
 
 }  // namespace sg
