@@ -33,13 +33,18 @@ LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
 _DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4}
-_IN_DTYPES = (torch.bfloat16, torch.float16, torch.float8_e4m3fn, torch.float8_e5m2)
+_IN_DTYPES = (torch.bfloat16, torch.float16, torch.float8_e4m3fn, torch.float8_e5m2, torch.float32)
 _FP8 = (torch.float8_e4m3fn, torch.float8_e5m2)
 
 
 def bias_dtype_for(in_dtype: torch.dtype) -> torch.dtype:
     """The bias has the inputs' type, except that 8-bit inputs come with a bf16 bias."""
     return torch.bfloat16 if in_dtype in _FP8 else in_dtype
+
+
+def _in_code(dtype: torch.dtype) -> int:
+    """Type code of A / B (X / Wf): fp32 operands are read as tf32 (their low 13 fraction bits do not take part)."""
+    return 5 if dtype == torch.float32 else _DTYPES[dtype]
 
 
 def build(force: bool = False) -> str:
@@ -164,7 +169,7 @@ def gemm(A: torch.Tensor, B: torch.Tensor, *, layout_a: str = "row", layout_b: s
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
                         _ptr(C), c_dtype, ldc, _ptr(bias), _DTYPES[bias_dtype_for(A.dtype)], float(alpha), float(beta),
-                        EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], r0, r1, _ptr(ref), _ptr(absacc),
+                        EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), _in_code(A.dtype), r0, r1, _ptr(ref), _ptr(absacc),
                         max(N, 1))
     if rc:
         raise ValueError(f"orc_gemm rejected its arguments (code {rc})")
@@ -183,7 +188,7 @@ def gemm_points(A, B, pi: Sequence[int], pj: Sequence[int], *, layout_a="row", l
     absacc = torch.empty_like(ref)
     rc = lib().orc_gemm_points(M, N, K, LAYOUTS[layout_a], LAYOUTS[layout_b], _ptr(A), lda, _ptr(B), ldb,
                                _ptr(C), c_dtype, ldc, _ptr(bias), _DTYPES[bias_dtype_for(A.dtype)], float(alpha),
-                               float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), _DTYPES[A.dtype], pi.numel(), _ptr(pi), _ptr(pj),
+                               float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]), _in_code(A.dtype), pi.numel(), _ptr(pi), _ptr(pj),
                                _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_gemm_points rejected its arguments (code {rc})")
@@ -316,7 +321,7 @@ def conv2d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=(0, 0), stride=(1, 1)
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_fprop(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias), _DTYPES[bias_dtype_for(X.dtype)],
                                 float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
-                                _DTYPES[X.dtype], p0, p1, _ptr(ref), _ptr(absacc))
+                                _in_code(X.dtype), p0, p1, _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_fprop rejected its arguments (code {rc})")
     if pixels is None:
@@ -393,7 +398,7 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
     absacc = torch.empty_like(ref)
     rc = lib().orc_conv2d_points(_ptr(d), _ptr(X), _ptr(Wf), _ptr(Cin), c_dtype, _ptr(bias),
                                  _DTYPES[bias_dtype_for(X.dtype)], float(alpha), float(beta), EPILOGUES[epi], float(epi_args[0]), float(epi_args[1]),
-                                 _DTYPES[X.dtype], ppix.numel(), _ptr(ppix), _ptr(pk), _ptr(ref), _ptr(absacc))
+                                 _in_code(X.dtype), ppix.numel(), _ptr(ppix), _ptr(pk), _ptr(ref), _ptr(absacc))
     if rc:
         raise ValueError(f"orc_conv2d_points rejected its arguments (code {rc})")
     return ref, absacc

@@ -45,7 +45,7 @@
 #endif
 
 enum { ORC_ROW_MAJOR = 0, ORC_COL_MAJOR = 1 };
-enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2, ORC_FP8_E4M3 = 3, ORC_FP8_E5M2 = 4 };
+enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2, ORC_FP8_E4M3 = 3, ORC_FP8_E5M2 = 4, ORC_TF32 = 5 };
 enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4,
        ORC_EPI_SIGMOID = 5, ORC_EPI_TANH = 6, ORC_EPI_MISH = 7, ORC_EPI_HARDSWISH = 8, ORC_EPI_LEAKY_RELU = 9,
        ORC_EPI_ELU = 10, ORC_EPI_CLIP = 11 };
@@ -97,9 +97,22 @@ static double fp8_e5m2_to_f64(uint8_t bits) {
     return sign ? -v : v;
 }
 
-/* Element idx of an input operand (.with_dtype(input=bf16 | fp16 | fp8_e4m3 | fp8_e5m2, ...)), widened exactly. */
+/* fp32 storage used as a tf32 operand (the DSL's input=fp32 problems run on TF32 tensor cores, Appendix A.2 "TF32
+ * note"): 1 sign, 8 exponent and the upper 10 fraction bits take part, the lower 13 fraction bits are ignored. */
+static double tf32_to_f64(float f) {
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    u &= 0xFFFFE000u;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Element idx of an input operand (.with_dtype(input=bf16 | fp16 | fp8_e4m3 | fp8_e5m2 | fp32-as-tf32, ...)), widened
+ * exactly (for tf32: after dropping the bits the tensor core does not read). */
 static double in_to_f64(const void* p, int dtype, int64_t idx) {
     switch (dtype) {
+        case ORC_TF32: return tf32_to_f64(((const float*)p)[idx]);
+        case ORC_F32: return (double)((const float*)p)[idx];
         case ORC_F16: return f16_to_f64(((const uint16_t*)p)[idx]);
         case ORC_FP8_E4M3: return fp8_e4m3_to_f64(((const uint8_t*)p)[idx]);
         case ORC_FP8_E5M2: return fp8_e5m2_to_f64(((const uint8_t*)p)[idx]);

@@ -617,3 +617,42 @@ def test_dgrad_wgrad_ranges_agree_with_full():
     dw, _ = orc.conv2d_wgrad(dY, X, (3, 2), pad=(1, 1))
     part, _ = orc.conv2d_wgrad(dY, X, (3, 2), pad=(1, 1), filters=(1, 3))
     assert torch.equal(part, dw[1:3])
+
+
+# ------------------------------------------------------------------------------------------------
+# fp32 operands read as tf32 (Appendix A.2: FP32 problems run on TF32 tensor cores)
+# ------------------------------------------------------------------------------------------------
+
+def test_tf32_operands_drop_their_low_13_fraction_bits():
+    # 1 + 2^-11 + 2^-12 sits above the half-way point between the tf32 neighbours 1 and 1 + 2^-10: a rounding
+    # conversion would give 1 + 2^-10, the tensor core's reading (the low 13 bits do not take part) gives 1.
+    x = 1.0 + 2.0 ** -11 + 2.0 ** -12
+    A = torch.tensor([[x, 1.0 + 2.0 ** -10, -x, 3.0]], dtype=torch.float32)
+    B = torch.eye(4, dtype=torch.float32)                        # column-major identity: picks the elements of A
+    ref, _ = orc.gemm(A, B)
+    assert ref.tolist() == [[1.0, 1.0 + 2.0 ** -10, -1.0, 3.0]]
+    # both operands are read that way; the bias (fp32) is used exactly
+    bias = torch.tensor([x], dtype=torch.float32)
+    ref, _ = orc.gemm(torch.tensor([[x]], dtype=torch.float32), torch.tensor([[x]], dtype=torch.float32), bias=bias)
+    assert ref.item() == 1.0 + float(torch.tensor(x, dtype=torch.float32))
+
+
+def test_tf32_representable_operands_give_the_plain_product():
+    A16, B16, _ = inputs.make_gemm(19, 23, 40, "uniform", 1.0, seed=41)       # bf16 values are tf32 values
+    want, want_abs = orc.gemm(A16, B16, alpha=0.5, epi="gelu")
+    got, got_abs = orc.gemm(A16.float(), B16.float(), alpha=0.5, epi="gelu")
+    assert torch.equal(got, want) and torch.equal(got_abs, want_abs)
+    X16, W16, _ = inputs.make_conv(2, 6, 5, 4, 3, 3, 3, "uniform", 1.0, seed=42)
+    want, _ = orc.conv2d_fprop(X16, W16, pad=(1, 1))
+    got, _ = orc.conv2d_fprop(X16.float(), W16.float(), pad=(1, 1))
+    assert torch.equal(got, want)
+
+
+def test_tf32_gemm_matches_torch_fp64_on_masked_operands():
+    g = torch.Generator().manual_seed(7)
+    A = torch.randn(17, 33, generator=g)
+    B = torch.randn(21, 33, generator=g)
+    mask = lambda t: (t.view(torch.int32) & -8192).view(torch.float32)     # clear the low 13 bits
+    ref, _ = orc.gemm(A, B)
+    torch.testing.assert_close(ref, mask(A).double() @ mask(B).double().t(), rtol=1e-13, atol=1e-13)
+    assert not torch.allclose(ref, A.double() @ B.double().t(), rtol=0, atol=1e-6)   # the dropped bits are visible
