@@ -323,6 +323,13 @@ def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
     o16 = [torch.empty(n, n, dtype=torch.float16, device=dev) for _ in range(2)]
     timed("gemm4096_fp16_in_fp16_out", [(lambda i=i: sg.gemm(*h16[i], out=o16[i % 2])) for i in range(sets)], dict(op="gemm", M=n, N=n, K=n))
     del h16, o16
+    f32 = [(data[i][0].float(), data[i][1].float()) for i in range(4)]
+    o32 = [torch.empty(n, n, dtype=torch.float32, device=dev) for _ in range(2)]
+    timed("gemm4096_fp32_in_tf32_fp32_out", [(lambda i=i: sg.gemm(*f32[i], out=o32[i % 2])) for i in range(4)],
+          dict(op="gemm", M=n, N=n, K=n, elem_bytes_in=4, elem_bytes_out=4),
+          note="the paper's worked SOL example (4096^3, fp32 tensors, TF32 tensor cores); fraction against the bf16 peak: "
+               "the tf32 rate is half of it")
+    del f32, o32
     for dt8, nm in ((torch.float8_e4m3fn, "e4m3"), (torch.float8_e5m2, "e5m2")):
         q = [(data[i][0].float().mul(64).to(dt8), data[i][1].float().mul(64).to(dt8)) for i in range(sets)]
         timed(f"gemm4096_fp8_{nm}_in_bf16_out", [(lambda i=i: sg.gemm(*q[i], out=outs[i])) for i in range(sets)],

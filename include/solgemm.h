@@ -24,6 +24,10 @@
  *    A and B (conv: X and Wf) may also be 8-bit floating point, SG_FP8_E4M3 or SG_FP8_E5M2 (both the same;
  *    the DSL's fp8_e4m3 / fp8_e5m2 input types): K-contiguous layouts only, leading dimensions multiples of 16
  *    elements; the bias then is bf16, the output bf16, fp16 or fp32.  Scale factors go through alpha.
+ *    in_dtype SG_F32: A and B are fp32 in memory and are contracted on the TF32 tensor-core path (the paper's FP32
+ *    problems with TF32 throughput, Appendix A.2): of every operand element the sign, the exponent and the upper 10
+ *    fraction bits take part, the lower 13 fraction bits are ignored; accumulation is fp32.  K-contiguous layouts
+ *    only, leading dimensions multiples of 4 elements; the bias then is fp32 (4-byte aligned).
  *  - Epilogue: v = alpha*acc (+ beta*C if beta != 0) (+ bias[j] if bias != NULL); D = act(v).
  *    bias holds one value per output column j (GEMM) or output channel (conv); it is NOT scaled
  *    by alpha.  SG_EPI_BIAS is the identity activation and requires bias != NULL; every other
@@ -89,7 +93,7 @@ typedef struct sg_gemm_desc {
     int64_t M, N, K;
     int32_t layout_a, layout_b;   /* sg_layout_t */
     int64_t lda, ldb, ldc, ldd;
-    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype SG_BF16, SG_F16, SG_FP8_E4M3 or SG_FP8_E5M2 */
+    int32_t in_dtype, out_dtype;  /* sg_dtype_t; in_dtype SG_BF16, SG_F16, SG_F32 (tf32), SG_FP8_E4M3 or SG_FP8_E5M2 */
     float alpha, beta;
     int32_t epi;                  /* sg_epilogue_t */
     float epi_arg0, epi_arg1;     /* activation parameters (leaky_relu / elu slope, clip bounds); else ignored */

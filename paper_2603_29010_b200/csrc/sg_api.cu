@@ -191,15 +191,15 @@ struct Checked {
     int esize_out;
     int out_kind;                 // kernel template value: 0 bf16, 1 fp32, 2 fp16
     bool in_f16;
-    int in_fp8;                   // 0 no, 1 e4m3, 2 e5m2
+    int in_fp8;                   // operand kind: 0 sixteen-bit, 1 e4m3, 2 e5m2, 3 fp32 storage read as tf32
     int esize_in, bk;             // bytes per input element; K elements per 128-byte stage row
     CUtensorMapDataType tm_in, tm_out;
 };
 
 sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, float a0, float a1,
                          int32_t reserved, Checked* c) {
-    if (in_dtype != SG_BF16 && in_dtype != SG_F16 && in_dtype != SG_FP8_E4M3 && in_dtype != SG_FP8_E5M2)
-        return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16, SG_F16, SG_FP8_E4M3 or SG_FP8_E5M2", in_dtype);
+    if (in_dtype != SG_BF16 && in_dtype != SG_F16 && in_dtype != SG_FP8_E4M3 && in_dtype != SG_FP8_E5M2 && in_dtype != SG_F32)
+        return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16, SG_F16, SG_F32 (tf32), SG_FP8_E4M3 or SG_FP8_E5M2", in_dtype);
     if (out_dtype != SG_BF16 && out_dtype != SG_F32 && out_dtype != SG_F16)
         return fail(out_dtype == SG_FP8_E4M3 || out_dtype == SG_FP8_E5M2 ? SG_ERR_UNSUPPORTED : SG_ERR_INVALID_ARG,
                     "out_dtype %d: outputs must be SG_BF16, SG_F16 or SG_F32", out_dtype);
@@ -212,11 +212,12 @@ sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float
     c->esize_out = c->f32_out ? 4 : 2;
     c->out_kind = out_dtype == SG_F32 ? 1 : (out_dtype == SG_F16 ? 2 : 0);
     c->in_f16 = (in_dtype == SG_F16);
-    c->in_fp8 = in_dtype == SG_FP8_E4M3 ? 1 : (in_dtype == SG_FP8_E5M2 ? 2 : 0);
-    c->esize_in = c->in_fp8 ? 1 : 2;
-    c->bk = c->in_fp8 ? 128 : 64;
-    c->tm_in = c->in_fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
-                         : (c->in_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    c->in_fp8 = in_dtype == SG_FP8_E4M3 ? 1 : (in_dtype == SG_FP8_E5M2 ? 2 : (in_dtype == SG_F32 ? 3 : 0));
+    c->esize_in = c->in_fp8 == 3 ? 4 : (c->in_fp8 ? 1 : 2);
+    c->bk = 128 / c->esize_in;                      // one 128-byte swizzled row of K per stage row
+    c->tm_in = c->in_fp8 == 3 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                              : (c->in_fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                           : (c->in_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16));
     c->tm_out = out_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
                                     : (out_dtype == SG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
     return SG_OK;
@@ -245,7 +246,7 @@ sg_status_t check_gemm_desc(const sg_gemm_desc_t* d, bool grouped, Checked* c) {
     if (d->beta != 0.0f && d->ldc < (d->N > 1 ? d->N : 1)) return fail(SG_ERR_INVALID_ARG, "ldc %lld < N %lld", (long long)d->ldc, (long long)d->N);
     if ((d->lda * c->esize_in) % 16 || (d->ldb * c->esize_in) % 16) return fail(SG_ERR_ALIGNMENT, "lda and ldb must be multiples of 16 bytes");
     if (c->in_fp8 && (d->layout_a != SG_ROW_MAJOR || d->layout_b != SG_COL_MAJOR))
-        return fail(SG_ERR_UNSUPPORTED, "8-bit inputs are implemented for the K-contiguous pair (A row-major, B column-major) only");
+        return fail(SG_ERR_UNSUPPORTED, "8-bit and tf32 inputs are implemented for the K-contiguous pair (A row-major, B column-major) only");
     if ((d->ldd * c->esize_out) % 16) return fail(SG_ERR_ALIGNMENT, "ldd must be a multiple of 16 bytes");
     if (d->beta != 0.0f && (d->ldc * c->esize_out) % 16) return fail(SG_ERR_ALIGNMENT, "ldc must be a multiple of 16 bytes");
     return SG_OK;
@@ -547,6 +548,8 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (desc->M == 0 || desc->N == 0 || batch == 0) return SG_OK;
     st = check_ptrs(A, B, C, bias, D, desc->K, desc->beta, desc->epi, who);
     if (st != SG_OK) return st;
+    if (c.in_fp8 == 3 && bias && (reinterpret_cast<uintptr_t>(bias) & 3u))
+        return fail(SG_ERR_ALIGNMENT, "%s: an fp32 bias must be 4-byte aligned", who);
     {
         Params scratch_params;          // the chain's rules are checked before any device is touched
         st = apply_ex(&scratch_params, ex, desc->N, c.esize_out, who);
@@ -958,6 +961,8 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
     const int64_t Kg = desc->C * desc->R * desc->S;
     st = check_ptrs(X, Wf, Cin, bias, Y, Kg, desc->beta, desc->epi, "sg_conv2d_fprop");
     if (st != SG_OK) return st;
+    if (c.in_fp8 == 3 && bias && (reinterpret_cast<uintptr_t>(bias) & 3u))
+        return fail(SG_ERR_ALIGNMENT, "sg_conv2d_fprop: an fp32 bias must be 4-byte aligned");
     {
         Params scratch_params;
         st = apply_ex(&scratch_params, ex, desc->K, c.esize_out, "sg_conv2d_fprop_ex");
@@ -1050,7 +1055,7 @@ sg_status_t grad_geometry(const sg_conv2d_desc_t* desc, const char* who, Checked
                                   desc->epi_arg1, desc->reserved, c);
     if (st != SG_OK) return st;
     if (desc->epi != SG_EPI_NONE) return fail(SG_ERR_INVALID_ARG, "%s: epi must be SG_EPI_NONE", who);
-    if (c->in_fp8) return fail(SG_ERR_UNSUPPORTED, "%s: 8-bit inputs are not supported (an operand is read N-contiguous)", who);
+    if (c->in_fp8) return fail(SG_ERR_UNSUPPORTED, "%s: 8-bit and tf32 inputs are not supported (an operand is read N-contiguous)", who);
     if (desc->N < 0 || desc->H < 0 || desc->W < 0 || desc->C < 0 || desc->K < 0 || desc->R < 1 || desc->S < 1)
         return fail(SG_ERR_INVALID_ARG, "%s: extents must be >= 0 and the filter at least 1x1", who);
     if (desc->stride_h < 1 || desc->stride_w < 1 || desc->dil_h < 1 || desc->dil_w < 1 || desc->pad_h < 0 || desc->pad_w < 0)

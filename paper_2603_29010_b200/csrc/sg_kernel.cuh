@@ -82,7 +82,8 @@ struct alignas(64) Params {
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
     int32_t epi, mode;
     int32_t in_f16;                     // 1: the bias (and 16-bit A, B) are fp16, else bf16
-    int32_t in_fp8;                     // 0: 16-bit A and B; 1: e4m3; 2: e5m2 (the bias then is bf16 or fp16 as in_f16 says)
+    int32_t in_fp8;                     // operand kind: 0 sixteen-bit A and B; 1 e4m3; 2 e5m2 (bias bf16 or fp16 as in_f16 says);
+                                        // 3 fp32 storage read as tf32 (bias fp32)
     int32_t bk_elems;                   // elements of K per 128-byte stage row: 64 (16-bit) or 128 (8-bit)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
@@ -692,8 +693,8 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 const Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
                 if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
-                const bool fp8 = kLean ? false : p.in_fp8 != 0;
-                const uint32_t in_fmt = fp8 ? static_cast<uint32_t>(p.in_fp8 - 1) : (p.in_f16 ? 0u : 1u);
+                const int in_kind = kLean ? 0 : p.in_fp8;          // 0 sixteen-bit, 1 / 2 fp8, 3 tf32
+                const uint32_t in_fmt = in_kind == 3 ? 2u : (in_kind ? static_cast<uint32_t>(in_kind - 1) : (p.in_f16 ? 0u : 1u));
                 const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, a_mn, b_mn, in_fmt);
                 const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
                 const uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
@@ -712,7 +713,12 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(stage * (Cfg::STAGE_BYTES >> 4));
                     // One instruction-K step is 32 bytes along a K-major row (16 two-byte or 32 one-byte elements), or two
                     // 1 KB k-groups of an MN-major tile; a 128-byte stage row holds four of them for either width.
-                    if (fp8) {
+                    if (in_kind == 3) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_tf32<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
+                                             (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                    } else if (in_kind != 0) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             umma_fp8<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
@@ -752,6 +758,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         uint16_t* bias_w = reinterpret_cast<uint16_t*>(smem + Cfg::OFF_BIAS) + ew * Cfg::BIAS_SLOTS;   // bf16 bias of its chunks
         constexpr int kMyBiasSlots = ((BN / CH + kStep - 1) / kStep) * CH;     // columns of the chunks one warp handles
         const bool has_bias = (mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
+        const bool bias_f32 = kLean ? false : p.in_fp8 == 3;       // tf32 operands come with an fp32 bias, read directly
         const bool has_c = (p.beta != 0.0f);
         const bool in_f16 = (p.in_f16 != 0);
         const float alpha = p.alpha, beta = p.beta;
@@ -790,7 +797,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (has_c) c_g += static_cast<int64_t>(ti.b) * p.strideC * (kOutF32 ? 4 : 2);
                 d_g += static_cast<int64_t>(ti.b) * p.strideD * (kOutF32 ? 4 : 2);
             }
-            if (has_bias) {
+            if (has_bias && !bias_f32) {
                 // every warp keeps its own copy of the tile's bias values, so no barrier between warps is needed
                 __syncwarp();
                 const uint16_t* bsrc = bias_g;
@@ -1059,7 +1066,13 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         }
                     }
                 }
-                if (has_bias) {
+                if (has_bias && bias_f32) {
+                    // every lane reads the same addresses: broadcast loads
+                    const float* bf = reinterpret_cast<const float*>(mode == MODE_GROUPED ? p.g_bias[ti.b] : p.bias) +
+                                      (mode == MODE_GROUPED ? 0 : static_cast<int64_t>(ti.b) * p.strideBias) + n0 + c * CH;
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) v[i] += (n0 + c * CH + i < p.N) ? __ldg(bf + i) : 0.0f;
+                } else if (has_bias) {
 #pragma unroll
                     for (int i = 0; i < CH; i += 4) {
                         const uint2 b2 = *reinterpret_cast<const uint2*>(bias_w + (c / kStep) * CH + i);   // 4 bf16, broadcast read

@@ -248,6 +248,30 @@ __device__ __forceinline__ void umma_fp8(uint32_t d_tmem, uint64_t a_desc, uint6
             : "memory");
     }
 }
+// The same for fp32 storage read as tf32 (the low 13 fraction bits do not take part): K = 8 per instruction.
+template <bool kPair>
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    if constexpr (kPair) {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
 // Arrive on `bar` once every MMA issued so far by this thread has completed.  For a CTA pair the
 // arrival is delivered to the same barrier offset in both CTAs (mask 0b11).
 template <bool kPair>

@@ -68,7 +68,9 @@ def _call_gemm(sg, desc, A=0x1000, B=0x2000, C=None, bias=None, D=0x3000):
     (dict(), dict(A=None), "SG_ERR_NULL_POINTER"),
     (dict(beta=1.0), {}, "SG_ERR_NULL_POINTER"),         # beta != 0 without C
     (dict(epi=1), {}, "SG_ERR_NULL_POINTER"),            # SG_EPI_BIAS without bias
-    (dict(in_dtype=1), {}, "SG_ERR_UNSUPPORTED"),
+    (dict(in_dtype=9), {}, "SG_ERR_UNSUPPORTED"),
+    (dict(in_dtype=1, layout_a=1), {}, "SG_ERR_UNSUPPORTED"),      # fp32 (tf32) operands: K-contiguous only
+    (dict(in_dtype=1, lda=130), {}, "SG_ERR_ALIGNMENT"),           # 130 fp32 elements = 520 bytes
     (dict(layout_a=1, lda=64), {}, "SG_ERR_INVALID_ARG"),       # column-major A: lda must cover M = 128
     (dict(layout_b=7), {}, "SG_ERR_INVALID_ARG"),
 ])
