@@ -33,17 +33,19 @@ LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
 _DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4}
-_IN_DTYPES = (torch.bfloat16, torch.float16, torch.float8_e4m3fn, torch.float8_e5m2, torch.float32)
+_IN_DTYPES = (torch.bfloat16, torch.float16, torch.float8_e4m3fn, torch.float8_e5m2, torch.float32, torch.int8)
 _FP8 = (torch.float8_e4m3fn, torch.float8_e5m2)
 
 
 def bias_dtype_for(in_dtype: torch.dtype) -> torch.dtype:
-    """The bias has the inputs' type, except that 8-bit inputs come with a bf16 bias."""
-    return torch.bfloat16 if in_dtype in _FP8 else in_dtype
+    """The bias has the inputs' type, except that 8-bit inputs (fp8, int8) come with a bf16 bias."""
+    return torch.bfloat16 if in_dtype in _FP8 or in_dtype == torch.int8 else in_dtype
 
 
 def _in_code(dtype: torch.dtype) -> int:
     """Type code of A / B (X / Wf): fp32 operands are read as tf32 (their low 13 fraction bits do not take part)."""
+    if dtype == torch.int8:
+        return 6
     return 5 if dtype == torch.float32 else _DTYPES[dtype]
 
 

@@ -45,7 +45,7 @@
 #endif
 
 enum { ORC_ROW_MAJOR = 0, ORC_COL_MAJOR = 1 };
-enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2, ORC_FP8_E4M3 = 3, ORC_FP8_E5M2 = 4, ORC_TF32 = 5 };
+enum { ORC_BF16 = 0, ORC_F32 = 1, ORC_F16 = 2, ORC_FP8_E4M3 = 3, ORC_FP8_E5M2 = 4, ORC_TF32 = 5, ORC_INT8 = 6 };
 enum { ORC_EPI_NONE = 0, ORC_EPI_BIAS = 1, ORC_EPI_RELU = 2, ORC_EPI_GELU = 3, ORC_EPI_SILU = 4,
        ORC_EPI_SIGMOID = 5, ORC_EPI_TANH = 6, ORC_EPI_MISH = 7, ORC_EPI_HARDSWISH = 8, ORC_EPI_LEAKY_RELU = 9,
        ORC_EPI_ELU = 10, ORC_EPI_CLIP = 11 };
@@ -112,6 +112,7 @@ static double tf32_to_f64(float f) {
 static double in_to_f64(const void* p, int dtype, int64_t idx) {
     switch (dtype) {
         case ORC_TF32: return tf32_to_f64(((const float*)p)[idx]);
+        case ORC_INT8: return (double)((const int8_t*)p)[idx];       /* the DSL's int8 / s8 input type */
         case ORC_F32: return (double)((const float*)p)[idx];
         case ORC_F16: return f16_to_f64(((const uint16_t*)p)[idx]);
         case ORC_FP8_E4M3: return fp8_e4m3_to_f64(((const uint8_t*)p)[idx]);

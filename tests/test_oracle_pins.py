@@ -656,3 +656,23 @@ def test_tf32_gemm_matches_torch_fp64_on_masked_operands():
     ref, _ = orc.gemm(A, B)
     torch.testing.assert_close(ref, mask(A).double() @ mask(B).double().t(), rtol=1e-13, atol=1e-13)
     assert not torch.allclose(ref, A.double() @ B.double().t(), rtol=0, atol=1e-6)   # the dropped bits are visible
+
+
+def test_int8_operands_are_plain_integers():
+    # hand case incl. the extremes of the type: [[-128, 127]] . [[127], [-128]] = -128*127 + 127*(-128) = -32512
+    A = torch.tensor([[-128, 127], [1, 2]], dtype=torch.int8)
+    Bt = torch.tensor([[127, -128], [3, -4]], dtype=torch.int8)        # column-major B: rows are columns of B
+    ref, absacc = orc.gemm(A, Bt)
+    assert ref.tolist() == [[-32512.0, -892.0], [-129.0, -5.0]]
+    assert absacc.tolist() == [[32512.0, 892.0], [383.0, 11.0]]
+    g = torch.Generator().manual_seed(3)
+    A = torch.randint(-128, 128, (13, 40), generator=g, dtype=torch.int8)
+    B = torch.randint(-128, 128, (9, 40), generator=g, dtype=torch.int8)
+    bias = inputs.normal([9], 3, 4)
+    ref, _ = orc.gemm(A, B, bias=bias, alpha=0.5)
+    torch.testing.assert_close(ref, 0.5 * (A.double() @ B.double().t()) + bias.double(), rtol=0, atol=0)
+    X = torch.randint(-128, 128, (1, 5, 4, 16), generator=g, dtype=torch.int8)
+    Wf = torch.randint(-128, 128, (3, 3, 3, 16), generator=g, dtype=torch.int8)
+    y, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+    want = torch.nn.functional.conv2d(X.double().permute(0, 3, 1, 2), Wf.double().permute(0, 3, 1, 2), padding=1)
+    torch.testing.assert_close(y, want.permute(0, 2, 3, 1), rtol=0, atol=0)
