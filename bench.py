@@ -335,6 +335,11 @@ def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
         timed(f"gemm4096_fp8_{nm}_in_bf16_out", [(lambda i=i: sg.gemm(*q[i], out=outs[i])) for i in range(sets)],
               dict(op="gemm", M=n, N=n, K=n, elem_bytes_in=1), note="fraction against the bf16 peak: above 1 is expected")
         del q
+    q8 = [(data[i][0].float().mul(2048).clamp(-127, 127).to(torch.int8), data[i][1].float().mul(2048).clamp(-127, 127).to(torch.int8))
+          for i in range(sets)]
+    timed("gemm4096_int8_in_bf16_out", [(lambda i=i: sg.gemm(*q8[i], out=outs[i], alpha=2.0 ** -22)) for i in range(sets)],
+          dict(op="gemm", M=n, N=n, K=n, elem_bytes_in=1), note="integer tensor-core path; fraction against the bf16 peak")
+    del q8
     del data, outs, res, aux
     for (M, N, K) in ((256, 256, 32768), (512, 512, 16384), (128, 4096, 16384), (2048, 4096, 8192), (8192, 8192, 8192)):
         A = inputs.normal([M, K], 1, 1, K ** -0.5, device=dev)

@@ -28,6 +28,9 @@
  *    problems with TF32 throughput, Appendix A.2): of every operand element the sign, the exponent and the upper 10
  *    fraction bits take part, the lower 13 fraction bits are ignored; accumulation is fp32.  K-contiguous layouts
  *    only, leading dimensions multiples of 4 elements; the bias then is fp32 (4-byte aligned).
+ *    in_dtype SG_INT8 (the DSL's int8 / s8): signed 8-bit A and B, exact 32-bit integer accumulation; the accumulator
+ *    is converted to fp32 (exact below 2^24) and goes through the same floating-point epilogue (alpha and the scale
+ *    vectors of the extended chain dequantise); rules as for the 8-bit floats (K-contiguous, bf16 bias).
  *  - Epilogue: v = alpha*acc (+ beta*C if beta != 0) (+ bias[j] if bias != NULL); D = act(v).
  *    bias holds one value per output column j (GEMM) or output channel (conv); it is NOT scaled
  *    by alpha.  SG_EPI_BIAS is the identity activation and requires bias != NULL; every other
@@ -66,7 +69,7 @@ typedef enum {
     SG_ERR_TIMEOUT = 8        /* a bounded device-side wait expired (see sg_poll_status) */
 } sg_status_t;
 
-typedef enum { SG_BF16 = 0, SG_F32 = 1, SG_F16 = 2, SG_FP8_E4M3 = 3, SG_FP8_E5M2 = 4 } sg_dtype_t;
+typedef enum { SG_BF16 = 0, SG_F32 = 1, SG_F16 = 2, SG_FP8_E4M3 = 3, SG_FP8_E5M2 = 4, SG_INT8 = 5 } sg_dtype_t;
 typedef enum { SG_ROW_MAJOR = 0, SG_COL_MAJOR = 1 } sg_layout_t;
 typedef enum {
     SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4,

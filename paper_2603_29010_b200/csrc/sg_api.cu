@@ -191,17 +191,18 @@ struct Checked {
     int esize_out;
     int out_kind;                 // kernel template value: 0 bf16, 1 fp32, 2 fp16
     bool in_f16;
-    int in_fp8;                   // operand kind: 0 sixteen-bit, 1 e4m3, 2 e5m2, 3 fp32 storage read as tf32
+    int in_fp8;                   // operand kind: 0 sixteen-bit, 1 e4m3, 2 e5m2, 3 fp32 storage read as tf32, 4 int8
     int esize_in, bk;             // bytes per input element; K elements per 128-byte stage row
     CUtensorMapDataType tm_in, tm_out;
 };
 
 sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float alpha, float beta, float a0, float a1,
                          int32_t reserved, Checked* c) {
-    if (in_dtype != SG_BF16 && in_dtype != SG_F16 && in_dtype != SG_FP8_E4M3 && in_dtype != SG_FP8_E5M2 && in_dtype != SG_F32)
-        return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16, SG_F16, SG_F32 (tf32), SG_FP8_E4M3 or SG_FP8_E5M2", in_dtype);
+    if (in_dtype != SG_BF16 && in_dtype != SG_F16 && in_dtype != SG_FP8_E4M3 && in_dtype != SG_FP8_E5M2 && in_dtype != SG_F32 &&
+        in_dtype != SG_INT8)
+        return fail(SG_ERR_UNSUPPORTED, "in_dtype %d: inputs must be SG_BF16, SG_F16, SG_F32 (tf32), SG_FP8_E4M3, SG_FP8_E5M2 or SG_INT8", in_dtype);
     if (out_dtype != SG_BF16 && out_dtype != SG_F32 && out_dtype != SG_F16)
-        return fail(out_dtype == SG_FP8_E4M3 || out_dtype == SG_FP8_E5M2 ? SG_ERR_UNSUPPORTED : SG_ERR_INVALID_ARG,
+        return fail(out_dtype == SG_FP8_E4M3 || out_dtype == SG_FP8_E5M2 || out_dtype == SG_INT8 ? SG_ERR_UNSUPPORTED : SG_ERR_INVALID_ARG,
                     "out_dtype %d: outputs must be SG_BF16, SG_F16 or SG_F32", out_dtype);
     if (epi < SG_EPI_NONE || epi > SG_EPI_CLIP) return fail(SG_ERR_INVALID_ARG, "epi %d is not a sg_epilogue_t", epi);
     if (!std::isfinite(alpha) || !std::isfinite(beta)) return fail(SG_ERR_INVALID_ARG, "alpha and beta must be finite");
@@ -212,7 +213,7 @@ sg_status_t check_common(int32_t in_dtype, int32_t out_dtype, int32_t epi, float
     c->esize_out = c->f32_out ? 4 : 2;
     c->out_kind = out_dtype == SG_F32 ? 1 : (out_dtype == SG_F16 ? 2 : 0);
     c->in_f16 = (in_dtype == SG_F16);
-    c->in_fp8 = in_dtype == SG_FP8_E4M3 ? 1 : (in_dtype == SG_FP8_E5M2 ? 2 : (in_dtype == SG_F32 ? 3 : 0));
+    c->in_fp8 = in_dtype == SG_FP8_E4M3 ? 1 : (in_dtype == SG_FP8_E5M2 ? 2 : (in_dtype == SG_F32 ? 3 : (in_dtype == SG_INT8 ? 4 : 0)));
     c->esize_in = c->in_fp8 == 3 ? 4 : (c->in_fp8 ? 1 : 2);
     c->bk = 128 / c->esize_in;                      // one 128-byte swizzled row of K per stage row
     c->tm_in = c->in_fp8 == 3 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32

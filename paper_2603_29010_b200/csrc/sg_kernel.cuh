@@ -83,7 +83,7 @@ struct alignas(64) Params {
     int32_t epi, mode;
     int32_t in_f16;                     // 1: the bias (and 16-bit A, B) are fp16, else bf16
     int32_t in_fp8;                     // operand kind: 0 sixteen-bit A and B; 1 e4m3; 2 e5m2 (bias bf16 or fp16 as in_f16 says);
-                                        // 3 fp32 storage read as tf32 (bias fp32)
+                                        // 3 fp32 storage read as tf32 (bias fp32); 4 signed int8 with int32 accumulators (bias bf16)
     int32_t bk_elems;                   // elements of K per 128-byte stage row: 64 (16-bit) or 128 (8-bit)
     int32_t a_mn_major, b_mn_major;     // 1: the operand is stored with M (resp. N) contiguous: column-major A, row-major B
     int32_t P, Q, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, S, cblocks;   // conv
@@ -693,9 +693,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 const Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
                 if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
-                const int in_kind = kLean ? 0 : p.in_fp8;          // 0 sixteen-bit, 1 / 2 fp8, 3 tf32
-                const uint32_t in_fmt = in_kind == 3 ? 2u : (in_kind ? static_cast<uint32_t>(in_kind - 1) : (p.in_f16 ? 0u : 1u));
-                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, a_mn, b_mn, in_fmt);
+                const int in_kind = kLean ? 0 : p.in_fp8;          // 0 sixteen-bit, 1 / 2 fp8, 3 tf32, 4 int8
+                const uint32_t in_fmt = in_kind == 4 ? 1u
+                                        : (in_kind == 3 ? 2u : (in_kind ? static_cast<uint32_t>(in_kind - 1) : (p.in_f16 ? 0u : 1u)));
+                const uint32_t idesc = umma_idesc_f32acc(Cfg::TILE_M, ti.width, a_mn, b_mn, in_fmt, in_kind == 4);
                 const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);    // descriptor address units per K=16
                 const uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
                 const int acc = iter & 1;
@@ -713,7 +714,12 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(stage * (Cfg::STAGE_BYTES >> 4));
                     // One instruction-K step is 32 bytes along a K-major row (16 two-byte or 32 one-byte elements), or two
                     // 1 KB k-groups of an MN-major tile; a 128-byte stage row holds four of them for either width.
-                    if (in_kind == 3) {
+                    if (in_kind == 4) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_i8<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
+                                           (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                    } else if (in_kind == 3) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             umma_tf32<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
@@ -759,6 +765,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         constexpr int kMyBiasSlots = ((BN / CH + kStep - 1) / kStep) * CH;     // columns of the chunks one warp handles
         const bool has_bias = (mode == MODE_GROUPED) ? (p.g_bias != nullptr) : (p.bias != nullptr);
         const bool bias_f32 = kLean ? false : p.in_fp8 == 3;       // tf32 operands come with an fp32 bias, read directly
+        const bool acc_s32 = kLean ? false : p.in_fp8 == 4;        // int8 operands accumulate in 32-bit integers
         const bool has_c = (p.beta != 0.0f);
         const bool in_f16 = (p.in_f16 != 0);
         const float alpha = p.alpha, beta = p.beta;
@@ -902,13 +909,14 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         tmem_ld_wait();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
-                            v[i] = __uint_as_float(r0[i]);
-                            v[32 + i] = __uint_as_float(r1[i]);
+                            v[i] = acc_s32 ? static_cast<float>(static_cast<int32_t>(r0[i])) : __uint_as_float(r0[i]);
+                            v[32 + i] = acc_s32 ? static_cast<float>(static_cast<int32_t>(r1[i])) : __uint_as_float(r1[i]);
                         }
                     } else {
                         tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+                        for (int i = 0; i < 32; ++i)
+                            v[i] = acc_s32 ? static_cast<float>(static_cast<int32_t>(r0[i])) : __uint_as_float(r0[i]);
                     }
                     if (c + kStep >= nchunks && !ksplit_tile) {
                         // this warp has read its last columns of the accumulator: hand its share back to the MMA warp

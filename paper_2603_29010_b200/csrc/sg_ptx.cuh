@@ -272,6 +272,30 @@ __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint
             : "memory");
     }
 }
+// The same for signed 8-bit integer operands with 32-bit integer accumulators: K = 32 per instruction.
+template <bool kPair>
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    if constexpr (kPair) {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n"
+            "}\n"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
 // Arrive on `bar` once every MMA issued so far by this thread has completed.  For a CTA pair the
 // arrival is delivered to the same barrier offset in both CTAs (mask 0b11).
 template <bool kPair>
@@ -334,10 +358,12 @@ __device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t smem_addr)
 
 // Instruction descriptor for kind::f16: fp32 accumulator, bf16 or fp16 A and B, no negation, dense.  bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format,
 // 15 / 16 A / B major (0 = K), 17-22 N >> 3, 24-28 M >> 4.
-// in_fmt: operand format code of both A and B.  kind::f16: 0 = fp16, 1 = bf16.  kind::f8f6f4: 0 = e4m3, 1 = e5m2.
-__host__ __device__ constexpr uint32_t umma_idesc_f32acc(int m, int n, bool a_mn_major, bool b_mn_major, uint32_t in_fmt) {
+// in_fmt: operand format code of both A and B.  kind::f16: 0 = fp16, 1 = bf16.  kind::tf32: 2.  kind::f8f6f4: 0 = e4m3,
+// 1 = e5m2.  kind::i8: 1 = signed.  acc_s32: the accumulator is a 32-bit integer (kind::i8) instead of fp32.
+__host__ __device__ constexpr uint32_t umma_idesc_f32acc(int m, int n, bool a_mn_major, bool b_mn_major, uint32_t in_fmt,
+                                                         bool acc_s32 = false) {
     const uint32_t fmt = in_fmt;
-    return (1u << 4) | (fmt << 7) | (fmt << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
+    return ((acc_s32 ? 2u : 1u) << 4) | (fmt << 7) | (fmt << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 

@@ -32,7 +32,7 @@ STATUS_NAMES = ["SG_OK", "SG_ERR_INVALID_ARG", "SG_ERR_NULL_POINTER", "SG_ERR_AL
 LAYOUTS = {"row": 0, "col": 1}
 EPILOGUES = {"none": 0, "bias": 1, "relu": 2, "gelu": 3, "silu": 4, "sigmoid": 5, "tanh": 6, "mish": 7,
              "hardswish": 8, "leaky_relu": 9, "elu": 10, "clip": 11}
-DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4}
+DTYPES = {torch.bfloat16: 0, torch.float32: 1, torch.float16: 2, torch.float8_e4m3fn: 3, torch.float8_e5m2: 4, torch.int8: 5}
 OPS = {"gemm": 0, "batched": 1, "grouped": 2, "conv2d": 3, "transpose": 4, "conv2d_dgrad": 5, "conv2d_wgrad": 6}
 EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_grouped_gemm",
             "sg_grouped_gemm_static", "sg_conv2d_fprop", "sg_gemm_ex", "sg_conv2d_fprop_ex",

@@ -59,7 +59,8 @@ def _call_gemm(sg, desc, A=0x1000, B=0x2000, C=None, bias=None, D=0x3000):
     (dict(epi=12), {}, "SG_ERR_INVALID_ARG"),
     (dict(epi=11, epi_arg0=1.0, epi_arg1=0.0), {}, "SG_ERR_INVALID_ARG"),      # clip with min > max
     (dict(epi=9, epi_arg0=float("nan")), {}, "SG_ERR_INVALID_ARG"),
-    (dict(out_dtype=5), {}, "SG_ERR_INVALID_ARG"),
+    (dict(out_dtype=9), {}, "SG_ERR_INVALID_ARG"),
+    (dict(out_dtype=5), {}, "SG_ERR_UNSUPPORTED"),          # SG_INT8 is an input type only
     (dict(reserved=1), {}, "SG_ERR_INVALID_ARG"),
     (dict(lda=132), {}, "SG_ERR_ALIGNMENT"),             # 264 bytes: not a multiple of 16
     (dict(ldd=129), {}, "SG_ERR_ALIGNMENT"),
