@@ -288,8 +288,21 @@ bool ksplit_allowed(const DeviceState& d) {
     return d.scratch != nullptr && tail_mode != 0 && tail_mode != 1 && env_k != 0;
 }
 
+// What choose_shape needs to know for problems bound by memory traffic rather than by the tensor pipe: operand and
+// output element sizes and whether the activation is one of the transcendental ones (epi < 0: terms not applied).
+struct MemHint {
+    int epi = -1;
+    int esize_in = 2;
+    int esize_out = 2;
+};
+
+inline bool heavy_activation(int epi) {
+    return epi == SG_EPI_GELU || epi == SG_EPI_SILU || epi == SG_EPI_SIGMOID || epi == SG_EPI_TANH || epi == SG_EPI_MISH ||
+           epi == SG_EPI_ELU;
+}
+
 Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N,
-                   int64_t K, int min_b_rows = 1) {
+                   int64_t K, int min_b_rows = 1, MemHint mem = MemHint{}) {
     const int force_bn = g_tune_tile_n.load();
     const int force_pair = g_tune_pair.load();
     const int bns[3] = {256, 128, 64};
@@ -341,6 +354,23 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
                     const double t = t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed + ksplit_exchange_us(ks);
                     if (t < cost) cost = t;
                 }
+            }
+            if (mem.epi >= 0 && !pi && tiles_for(128, 256) >= d.sm_count) {
+                // Memory-bound problems with at least a wave of tiles (short K, many small problems): the time is the traffic -- each operand once
+                // from HBM (~7 TB/s), every tile's operand panels from the L2 (~14 TB/s over all SMs) -- plus what
+                // cannot overlap with it: the last tile's epilogue (measured: 1.7 us for a 128 x 256 tile under a
+                // transcendental activation, 0.5 us otherwise) and ~0.2 us per tile an SM walks through.  Narrower
+                // tiles shorten that end; measured on 128 problems of 256 x 256 x 512 with GELU: 18.8 us with 256-wide
+                // tiles, 17.7 us with 128-wide ones (19.8 with 64: L2 traffic), and the reverse order without activation.
+                double hbm_bytes = 0.0;
+                for (int64_t r : rows_per_problem)
+                    hbm_bytes += static_cast<double>(r + N) * static_cast<double>(K) * mem.esize_in +
+                                 static_cast<double>(r) * static_cast<double>(N) * mem.esize_out;
+                hbm_bytes *= static_cast<double>(batch_mult);
+                const double l2_bytes = static_cast<double>(tiles) * (128.0 + bn) * static_cast<double>(K) * mem.esize_in;
+                const double t_traffic = std::max(hbm_bytes / 7.0e6, l2_bytes / 14.0e6);
+                const double t_end = (heavy_activation(mem.epi) ? 1.7 : 0.5) * bn / 256.0 + 0.2 * static_cast<double>(waves);
+                if (t_traffic + t_end > cost) cost = t_traffic + t_end;
             }
             if (cost < best_cost) {
                 best_cost = cost;
@@ -572,7 +602,8 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.in_fp8 = c.in_fp8;
     p.bk_elems = c.bk;
     const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
-    Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows);
+    Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows,
+                           MemHint{desc->epi, c.esize_in, c.esize_out});
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_DENSE;
     p.a_mn_major = desc->layout_a == SG_COL_MAJOR ? 1 : 0;
