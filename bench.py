@@ -348,6 +348,15 @@ def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
         timed(f"gemm_{M}x{N}x{K}", [lambda: sg.gemm(A, B, out=O)], dict(op="gemm", M=M, N=N, K=K), reps=10,
               note="one buffer set (operands may stay in L2)")
         del A, B, O
+    # matrix-vector products (N = 1): a stream over the matrix, several matrices in turn so that none stays in the L2
+    for (R, K) in ((4096, 4096), (11008, 4096), (8192, 8192), (256, 131072), (16384, 16384)):
+        nset = max(2, min(12, int(400e6 // (R * K * 2)) + 1))
+        Ws = [torch.randn(R, K, device=dev).to(bf) for _ in range(nset)]
+        x = torch.randn(1, K, device=dev).to(bf)
+        ys = [torch.empty(R, 1, dtype=bf, device=dev) for _ in range(nset)]
+        timed(f"gemv_{R}x{K}", [(lambda i=i: sg.gemm(Ws[i], x, out=ys[i])) for i in range(nset)], dict(op="gemm", M=R, N=1, K=K),
+              note="plan: rows per CTA in 'tiles', K ranges in 'tail_split' (negative), CTAs in 'grid'")
+        del Ws, x, ys
     for (b, r, c_) in ((32, 256, 3136), (8, 4096, 4096)):
         for di, do in ((torch.float32, bf), (bf, bf)):
             xs = [torch.randn(b, r, c_, device=dev).to(di) for _ in range(4)]

@@ -17,6 +17,7 @@
 #include "sg_kernel.cuh"
 #include "sg_variants.h"
 #include "sg_transpose.cuh"
+#include "sg_gemv.cuh"
 
 namespace {
 
@@ -699,6 +700,125 @@ sg_status_t upload(const std::vector<uint8_t>& host, void* dev, cudaStream_t str
     return SG_OK;
 }
 
+// ------------------------------------------------------------------------------------------ matrix-vector products
+// A GEMM with N = 1 (the matrix is A) or M = 1 (the matrix is B) whose matrix is K-contiguous and whose vector is
+// contiguous runs as a stream over the matrix (sg_gemv.cuh) instead of through the tensor-core tiles.  *taken is false
+// when the call does not have that form (the general path then validates and runs it).
+template <typename T>
+cudaError_t launch_gemv(const GemvParams& gp, int rb, int ctas, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(gp.ksplit);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    switch (rb) {
+        case 4: return cudaLaunchKernelEx(&cfg, gemv_kernel<T, 4>, gp);
+        case 2: return cudaLaunchKernelEx(&cfg, gemv_kernel<T, 2>, gp);
+        default: return cudaLaunchKernelEx(&cfg, gemv_kernel<T, 1>, gp);
+    }
+}
+
+sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C, const void* bias, void* D,
+                     void* stream, bool* taken) {
+    *taken = false;
+    if (!desc || desc->K < 1 || desc->K > INT32_MAX || desc->M < 1 || desc->N < 1) return SG_OK;
+    static const bool off = getenv("SG_NO_GEMV") != nullptr;     // tests: the same product through the tiles
+    if (off) return SG_OK;
+    const bool mat_a = desc->N == 1;
+    if (!mat_a && desc->M != 1) return SG_OK;
+    if (desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F16 && desc->in_dtype != SG_F32) return SG_OK;
+    const int es = desc->in_dtype == SG_F32 ? 4 : 2;
+    // the matrix K-contiguous, the vector contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
+    const bool a_kc = desc->layout_a == SG_ROW_MAJOR, b_kc = desc->layout_b == SG_COL_MAJOR;
+    const void* W = mat_a ? A : B;
+    const void* x = mat_a ? B : A;
+    const int64_t ld = mat_a ? desc->lda : desc->ldb;
+    const int64_t R = mat_a ? desc->M : desc->N;
+    if (mat_a ? !(a_kc && (b_kc || desc->ldb == 1)) : !(b_kc && (a_kc || desc->lda == 1))) return SG_OK;
+    if (R > INT32_MAX || ld < desc->K || (ld * es) % 16 || !W || !x || !aligned16(W) || !aligned16(x)) return SG_OK;
+    *taken = true;
+
+    Checked c;
+    sg_status_t st = check_common(desc->in_dtype, desc->out_dtype, desc->epi, desc->alpha, desc->beta, desc->epi_arg0,
+                                  desc->epi_arg1, desc->reserved, &c);
+    if (st != SG_OK) return st;
+    if (desc->layout_a != SG_ROW_MAJOR && desc->layout_a != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_a %d is not a sg_layout_t", desc->layout_a);
+    if (desc->layout_b != SG_ROW_MAJOR && desc->layout_b != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_b %d is not a sg_layout_t", desc->layout_b);
+    if (!D) return fail(SG_ERR_NULL_POINTER, "sg_gemm: D is NULL");
+    if (desc->beta != 0.0f && !C) return fail(SG_ERR_NULL_POINTER, "sg_gemm: beta != 0 needs C");
+    if (desc->epi == SG_EPI_BIAS && !bias) return fail(SG_ERR_NULL_POINTER, "sg_gemm: SG_EPI_BIAS needs bias");
+    if (desc->ldd < desc->N) return fail(SG_ERR_INVALID_ARG, "ldd %lld < N %lld", (long long)desc->ldd, (long long)desc->N);
+    if (desc->beta != 0.0f && desc->ldc < desc->N) return fail(SG_ERR_INVALID_ARG, "ldc %lld < N %lld", (long long)desc->ldc, (long long)desc->N);
+    const uintptr_t out_mask = static_cast<uintptr_t>(c.esize_out - 1), in_mask = static_cast<uintptr_t>(es - 1);
+    if ((reinterpret_cast<uintptr_t>(D) & out_mask) || (desc->beta != 0.0f && (reinterpret_cast<uintptr_t>(C) & out_mask)) ||
+        (bias && (reinterpret_cast<uintptr_t>(bias) & in_mask)))
+        return fail(SG_ERR_ALIGNMENT, "sg_gemm: D, C and bias must be aligned to their element size");
+    DeviceState* d = nullptr;
+    st = device_state(&d);
+    if (st != SG_OK) return st;
+
+    GemvParams gp;
+    memset(&gp, 0, sizeof gp);
+    gp.W = W;
+    gp.x = x;
+    gp.C = desc->beta != 0.0f ? C : nullptr;
+    gp.bias = bias;
+    gp.D = D;
+    gp.ld = ld;
+    gp.c_stride = mat_a ? desc->ldc : 1;
+    gp.d_stride = mat_a ? desc->ldd : 1;
+    gp.R = static_cast<int32_t>(R);
+    gp.K = static_cast<int32_t>(desc->K);
+    gp.bias_stride = mat_a ? 0 : 1;
+    gp.out_kind = c.out_kind;
+    gp.epi = desc->epi;
+    gp.alpha = desc->alpha;
+    gp.beta = desc->beta;
+    gp.a0 = desc->epi_arg0;
+    gp.a1 = desc->epi_arg1;
+    // Geometry: at least two CTAs per SM where the problem has that much work; K ranges (CTAs of one cluster, at
+    // most 8) when the rows alone do not give that many, each range at least two sweeps of the 256 threads.
+    const int64_t sweep = 256 * (16 / es);
+    const int64_t ks_max = std::max<int64_t>(1, std::min<int64_t>(8, desc->K / (2 * sweep)));
+    const int64_t want = 2 * static_cast<int64_t>(d->sm_count);
+    static const int forced_rb = getenv("SG_GEMV_RB") ? atoi(getenv("SG_GEMV_RB")) : 0;    // experiments: 1, 2, 4
+    int rb = (forced_rb == 1 || forced_rb == 2 || forced_rb == 4) ? forced_rb : 4;
+    int64_t ks = 1;
+    for (;; rb >>= 1) {
+        const int64_t blocks = (R + rb - 1) / rb;
+        ks = std::min<int64_t>(ks_max, std::max<int64_t>(1, (want + blocks - 1) / blocks));
+        if (blocks * ks >= want || rb == 1 || forced_rb > 0) break;
+    }
+    int64_t kchunk = (desc->K + ks - 1) / ks;
+    kchunk = (kchunk + sweep - 1) / sweep * sweep;
+    ks = (desc->K + kchunk - 1) / kchunk;
+    gp.kchunk = static_cast<int32_t>(kchunk);
+    gp.ksplit = static_cast<int32_t>(ks);
+    const int64_t ctas = (R + rb - 1) / rb * ks;
+    if (ctas > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many rows for the matrix-vector path");
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    cudaError_t e = desc->in_dtype == SG_F32   ? launch_gemv<float>(gp, rb, static_cast<int>(ctas), cs)
+                    : desc->in_dtype == SG_F16 ? launch_gemv<__half>(gp, rb, static_cast<int>(ctas), cs)
+                                               : launch_gemv<__nv_bfloat16>(gp, rb, static_cast<int>(ctas), cs);
+    if (e != cudaSuccess) return fail(SG_ERR_CUDA, "matrix-vector kernel launch: %s", cudaGetErrorString(e));
+    g_launches.fetch_add(1);
+    t_last_plan[0] = 0;              // no tensor-core tiles: rows per CTA and K ranges instead
+    t_last_plan[1] = 0;
+    t_last_plan[2] = -static_cast<int32_t>(ks);
+    t_last_plan[3] = rb;
+    t_last_plan[4] = 0;
+    t_last_plan[5] = static_cast<int32_t>(ctas);
+    return SG_OK;
+}
+
+
 }  // namespace
 
 // ============================================================================================ C ABI
@@ -786,6 +906,9 @@ sg_status_t sg_set_tail_mode(int32_t mode) {
 
 sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C, const void* bias, void* D,
                     void* cuda_stream) {
+    bool taken = false;
+    const sg_status_t st = try_gemv(desc, A, B, C, bias, D, cuda_stream, &taken);
+    if (taken) return st;
     return run_dense(desc, 1, 0, 0, 0, 0, 0, A, B, C, bias, D, cuda_stream, "sg_gemm");
 }
 

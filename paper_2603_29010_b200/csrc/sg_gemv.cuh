@@ -1,0 +1,186 @@
+// Matrix-vector product with the fused epilogue: out[r] = act(alpha * sum_k W[r][k] x[k] + beta * C[r] + bias[r]).
+// The GEMM with N = 1 (or M = 1) of the paper's workload list (single-token decode): every matrix element is used
+// once, so the kernel is a stream over W bound by HBM, and the tensor cores have nothing to offer.
+//
+// Work split: a CTA of 256 threads takes RB consecutive rows and one K range; each thread walks the range in
+// 16-byte vectors (one vector of x serves RB vectors of W, so RB independent loads are in flight per thread and
+// iteration), sums in fp32, and the CTA reduces with shuffles and shared memory.  K ranges of one row block are the
+// CTAs of one thread-block cluster: rank 0 adds the other ranks' partial sums in rank order through distributed
+// shared memory (no global scratch, no atomics; the result depends only on the launch geometry).
+#pragma once
+#include <cooperative_groups.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cstdint>
+
+namespace sg {
+
+struct GemvParams {
+    const void* W;        // [R][ld], K contiguous
+    const void* x;        // [K], contiguous
+    const void* C;        // residual (output type) or null
+    const void* bias;     // input type (fp32 for fp32 inputs) or null
+    void* D;
+    int64_t ld;           // elements between rows of W
+    int64_t c_stride, d_stride;   // elements between consecutive rows' entries of C and D
+    int32_t R, K;
+    int32_t kchunk;       // K elements per cluster rank (a multiple of 256 vectors)
+    int32_t ksplit;       // CTAs per cluster
+    int32_t bias_stride;  // 0: one bias for all rows (N = 1), 1: one per row (M = 1)
+    int32_t out_kind;     // 0 bf16, 1 fp32, 2 fp16
+    int32_t epi;
+    float alpha, beta, a0, a1;
+};
+
+__device__ __forceinline__ uint4 ldg_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 16 bytes of input elements as fp32 values; fp32 inputs are read the way the tensor cores read them (tf32: the low
+// 13 fraction bits dropped), so that both paths of the library compute the same product.
+template <typename T> struct GemvVec;
+template <> struct GemvVec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void cvt(const uint4& u, float (&f)[8]) {
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    static __device__ __forceinline__ float one(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ float exact(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+};
+template <> struct GemvVec<__half> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void cvt(const uint4& u, float (&f)[8]) {
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            f[2 * i] = v.x;
+            f[2 * i + 1] = v.y;
+        }
+    }
+    static __device__ __forceinline__ float one(const __half* p) { return __half2float(*p); }
+    static __device__ __forceinline__ float exact(const __half* p) { return __half2float(*p); }
+};
+template <> struct GemvVec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void cvt(const uint4& u, float (&f)[4]) {
+        f[0] = __uint_as_float(u.x & 0xFFFFE000u);
+        f[1] = __uint_as_float(u.y & 0xFFFFE000u);
+        f[2] = __uint_as_float(u.z & 0xFFFFE000u);
+        f[3] = __uint_as_float(u.w & 0xFFFFE000u);
+    }
+    static __device__ __forceinline__ float one(const float* p) { return __uint_as_float(__float_as_uint(*p) & 0xFFFFE000u); }
+    static __device__ __forceinline__ float exact(const float* p) { return *p; }      // the bias is not an MMA operand
+};
+
+__device__ __forceinline__ float gemv_load_out(const void* base, int64_t i, int out_kind) {
+    if (out_kind == 1) return reinterpret_cast<const float*>(base)[i];
+    if (out_kind == 2) return __half2float(reinterpret_cast<const __half*>(base)[i]);
+    return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[i]);
+}
+__device__ __forceinline__ void gemv_store_out(void* base, int64_t i, int out_kind, float v) {
+    if (out_kind == 1) reinterpret_cast<float*>(base)[i] = v;
+    else if (out_kind == 2) reinterpret_cast<__half*>(base)[i] = __float2half_rn(v);
+    else reinterpret_cast<__nv_bfloat16*>(base)[i] = __float2bfloat16_rn(v);
+}
+
+// Four rows per CTA and a register budget that lets four CTAs of 16-bit inputs share an SM measured best (more,
+// smaller CTAs balance better over the SMs than eight rows per CTA; deeper unrolling did not help).
+template <typename T, int RB>
+__global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4) ? 4 : 1) gemv_kernel(const GemvParams p) {
+    namespace cg = cooperative_groups;
+    constexpr int V = GemvVec<T>::N;
+    constexpr int WARPS = 8;
+    __shared__ float warp_part[WARPS][RB];
+    __shared__ float cta_part[RB];
+
+    const int ks = p.ksplit;
+    const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));      // = rank in the (ks, 1, 1) cluster
+    const int64_t r0 = static_cast<int64_t>(blockIdx.x / static_cast<unsigned>(ks)) * RB;
+    const int kbeg = rank * p.kchunk;
+    const int kend = min(p.K, kbeg + p.kchunk);
+    const int kvec_end = kbeg < kend ? kbeg + ((kend - kbeg) / V) * V : kbeg;
+
+    const T* x = reinterpret_cast<const T*>(p.x);
+    const T* w[RB];
+#pragma unroll
+    for (int i = 0; i < RB; ++i) {
+        // rows past the end read the last row again (a valid address); their sums are never stored
+        const int64_t r = min(r0 + i, static_cast<int64_t>(p.R) - 1);
+        w[i] = reinterpret_cast<const T*>(p.W) + r * p.ld;
+    }
+    float acc[RB];
+#pragma unroll
+    for (int i = 0; i < RB; ++i) acc[i] = 0.0f;
+
+#pragma unroll 2
+    for (int k = kbeg + static_cast<int>(threadIdx.x) * V; k < kvec_end; k += 256 * V) {
+        uint4 wv[RB];
+#pragma unroll
+        for (int i = 0; i < RB; ++i) wv[i] = ldg_stream16(w[i] + k);
+        float xf[V];
+        GemvVec<T>::cvt(__ldg(reinterpret_cast<const uint4*>(x + k)), xf);
+#pragma unroll
+        for (int i = 0; i < RB; ++i) {
+            float wf[V];
+            GemvVec<T>::cvt(wv[i], wf);
+#pragma unroll
+            for (int j = 0; j < V; ++j) acc[i] = fmaf(wf[j], xf[j], acc[i]);
+        }
+    }
+    // the last K % V elements (only the last rank has any)
+    {
+        const int kt = kvec_end + static_cast<int>(threadIdx.x);
+        if (kt < kend) {
+            const float xv = GemvVec<T>::one(x + kt);
+#pragma unroll
+            for (int i = 0; i < RB; ++i) acc[i] = fmaf(GemvVec<T>::one(w[i] + kt), xv, acc[i]);
+        }
+    }
+
+#pragma unroll
+    for (int i = 0; i < RB; ++i) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc[i] += __shfl_xor_sync(0xFFFFFFFFu, acc[i], off);
+    }
+    const int warp = static_cast<int>(threadIdx.x) >> 5, lane = static_cast<int>(threadIdx.x) & 31;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < RB; ++i) warp_part[warp][i] = acc[i];
+    }
+    __syncthreads();
+    if (threadIdx.x < RB) {
+        float s = 0.0f;
+#pragma unroll
+        for (int wi = 0; wi < WARPS; ++wi) s += warp_part[wi][threadIdx.x];
+        cta_part[threadIdx.x] = s;
+    }
+    if (ks > 1) cg::this_cluster().sync();
+    if (rank == 0 && threadIdx.x < RB) {
+        float s = cta_part[threadIdx.x];
+        if (ks > 1) {
+            cg::cluster_group cluster = cg::this_cluster();
+            for (int r = 1; r < ks; ++r) s += *cluster.map_shared_rank(&cta_part[threadIdx.x], r);
+        }
+        const int64_t row = r0 + threadIdx.x;
+        if (row < p.R) {
+            float v[1] = {p.alpha * s};
+            if (p.beta != 0.0f) v[0] = fmaf(p.beta, gemv_load_out(p.C, row * p.c_stride, p.out_kind), v[0]);
+            if (p.bias != nullptr) v[0] += GemvVec<T>::exact(reinterpret_cast<const T*>(p.bias) + row * p.bias_stride);
+            if (p.epi >= EPI_RELU) apply_act_chunk<false, 1>(v, p.epi, p.a0, p.a1);
+            gemv_store_out(p.D, row * p.d_stride, p.out_kind, v[0]);
+        }
+    }
+    if (ks > 1) cg::this_cluster().sync();      // keep every rank's shared memory alive until rank 0 has read it
+}
+
+}  // namespace sg

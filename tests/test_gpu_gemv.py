@@ -1,0 +1,110 @@
+"""GPU parity of matrix-vector products (a GEMM with N = 1 or M = 1), which run as a stream over the matrix."""
+import pytest
+import torch
+
+from paper_2603_29010_b200 import inputs
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+from oracle import oracle as orc                      # noqa: E402
+from paper_2603_29010_b200 import solgemm as sg       # noqa: E402
+
+DEV = "cuda"
+
+
+@pytest.fixture(autouse=True)
+def _clean_status():
+    sg.set_tuning(-1, -1)
+    yield
+    torch.cuda.synchronize()
+    sg.poll_status()
+
+
+def _took_vector_path():
+    return sg.last_launch_plan()["tile_n"] == 0
+
+
+# rows x K: many rows, few rows with a long K (K ranges over a cluster), ragged row blocks, one row, tiny
+SHAPES = [(4096, 4096), (64, 65536), (1003, 1024), (8, 40000), (1, 4096), (3, 8), (300, 2056), (7, 262144)]
+
+
+@pytest.mark.parametrize("R,K", SHAPES)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
+def test_matrix_times_vector_integer_values_bit_exact(R, K, dtype):
+    # small integers: every partial sum is exact in fp32 whatever the order, so the result must match to the bit
+    W = inputs.small_integers([R, K], 90, 1, lo=-2, hi=2).to(dtype)
+    x = inputs.small_integers([1, K], 90, 2, lo=-2, hi=2).to(dtype)
+    ref, _ = orc.gemm(W, x)
+    D = torch.full((R, 1), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(W.to(DEV), x.to(DEV), out=D)
+    assert _took_vector_path()
+    parity.assert_bit_exact(D, ref, f"gemv {R}x{K} {dtype}")
+    # the vector on the left: (1 x K) . (R x K)^T
+    ref_t, _ = orc.gemm(x, W)
+    Dt = torch.full((1, R), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(x.to(DEV), W.to(DEV), out=Dt)
+    assert _took_vector_path()
+    parity.assert_bit_exact(Dt, ref_t, f"vector-matrix {R}x{K} {dtype}")
+
+
+@pytest.mark.parametrize("R,K", [(4096, 4096), (257, 33000), (5, 100008)])
+@pytest.mark.parametrize("dtype,out_dtype", [(torch.bfloat16, torch.bfloat16), (torch.float16, torch.float16),
+                                             (torch.float32, torch.float32), (torch.bfloat16, torch.float32)])
+@pytest.mark.parametrize("epi", ["none", "gelu", "relu"])
+def test_matrix_times_vector_real_values_with_epilogue(R, K, dtype, out_dtype, epi):
+    g = torch.Generator().manual_seed(R + K)
+    W = (torch.randn(R, K, generator=g) / 8).to(dtype)
+    x = (torch.randn(1, K, generator=g) / 8).to(dtype)
+    C = torch.randn(R, 1, generator=g).to(out_dtype)
+    bias1 = torch.randn(1, generator=g).to(dtype)
+    ref, absacc = orc.gemm(W, x, C=C, bias=bias1, alpha=0.75, beta=0.5, epi=epi)
+    D = sg.gemm(W.to(DEV), x.to(DEV), C=C.to(DEV), bias=bias1.to(DEV), alpha=0.75, beta=0.5, epi=epi, out_dtype=out_dtype)
+    assert _took_vector_path()
+    parity.assert_matches(D, ref, absacc, f"gemv {R}x{K} {dtype} {epi}")
+    # vector on the left: the bias is per output column, the residual a row
+    biasR = torch.randn(R, generator=g).to(dtype)
+    Ct = torch.randn(1, R, generator=g).to(out_dtype)
+    ref, absacc = orc.gemm(x, W, C=Ct, bias=biasR, alpha=-1.25, beta=2.0, epi=epi)
+    D = sg.gemm(x.to(DEV), W.to(DEV), C=Ct.to(DEV), bias=biasR.to(DEV), alpha=-1.25, beta=2.0, epi=epi, out_dtype=out_dtype)
+    assert _took_vector_path()
+    parity.assert_matches(D, ref, absacc, f"vector-matrix {R}x{K} {dtype} {epi}")
+
+
+def test_padded_rows_strided_outputs_and_a_column_vector_operand():
+    g = torch.Generator().manual_seed(11)
+    R, K, ld = 517, 1003, 1008                         # K is no multiple of a 16-byte vector; rows padded to one
+    Wp = (torch.randn(R, ld, generator=g) / 4).to(torch.bfloat16)
+    W = Wp[:, :K]
+    xcol = (torch.randn(K, 1, generator=g) / 4).to(torch.bfloat16)     # a K x 1 row-major B
+    Cp = torch.randn(R, 4, generator=g).to(torch.bfloat16)
+    ref, absacc = orc.gemm(W, xcol, layout_b="row", C=Cp[:, :1], beta=1.0, epi="silu")
+    Dp = torch.full((R, 3), 7.0, dtype=torch.bfloat16, device=DEV)
+    sg.gemm(Wp.to(DEV)[:, :K], xcol.to(DEV), layout_b="row", C=Cp.to(DEV)[:, :1], beta=1.0,
+            epi="silu", out=Dp[:, :1])
+    assert _took_vector_path()
+    parity.assert_matches(Dp[:, :1], ref, absacc, "padded gemv")
+    assert bool((Dp[:, 1:] == 7.0).all()), "the neighbours of a strided output column were written"
+
+
+def test_results_do_not_depend_on_the_run():
+    g = torch.Generator().manual_seed(3)
+    W = torch.randn(100, 70000, generator=g).to(torch.bfloat16).to(DEV)
+    x = torch.randn(1, 70000, generator=g).to(torch.bfloat16).to(DEV)
+    first = sg.gemm(W, x, out_dtype=torch.float32).clone()
+    for _ in range(5):
+        assert torch.equal(sg.gemm(W, x, out_dtype=torch.float32), first)
+
+
+def test_other_forms_still_go_through_the_tiles():
+    g = torch.Generator().manual_seed(4)
+    A = torch.randn(256, 64, generator=g).to(torch.bfloat16)
+    B2 = torch.randn(2, 64, generator=g).to(torch.bfloat16)
+    out = torch.empty(256, 8, dtype=torch.bfloat16, device=DEV)
+    sg.gemm(A.to(DEV), B2.to(DEV), out=out[:, :2])
+    assert not _took_vector_path()
+    ref, absacc = orc.gemm(A, B2)
+    parity.assert_matches(out[:, :2], ref, absacc, "N = 2")
