@@ -110,12 +110,13 @@ typedef struct sg_gemm_desc {
  *   bias   device, in_dtype, [N]; may be NULL unless epi == SG_EPI_BIAS.
  *   D      device, out_dtype, [M,N] row-major; written in full (all M x N elements).
  * M == 0 or N == 0: SG_OK, nothing is launched.  K == 0: D = act(beta*C + bias).
- * Matrix-vector form (the workload list's single-token decode product): when N == 1 (or M == 1), the matrix operand is
+ * Matrix-vector form (the workload list's single-token decode product): when N <= 4 (or M <= 4), the matrix operand is
  *   K-contiguous (A row-major, resp. B column-major) and 16-byte aligned with a leading dimension that is a multiple
- *   of 16 bytes, the vector operand is contiguous and 16-byte aligned (either layout, with a leading dimension of 1
- *   when it is stored as K x 1), and in_dtype is SG_BF16, SG_F16 or SG_F32, the product runs as one pass over the
- *   matrix at HBM speed instead of through tensor-core tiles.  In that form ldc and ldd may be any value >= N
- *   (no 16-byte rule) and C, D and bias need only their element alignment; results are reproducible from run to run.
+ *   of 16 bytes, the vectors are K-contiguous, 16-byte aligned and a multiple of 16 bytes apart (a single vector may
+ *   also be stored as K x 1 with a leading dimension of 1), and in_dtype is SG_BF16, SG_F16 or SG_F32, the product
+ *   runs as one pass over the matrix at HBM speed instead of through tensor-core tiles.  In that form ldc and ldd may
+ *   be any value >= N (no 16-byte rule) and C, D and bias need only their element alignment; results are reproducible
+ *   from run to run.
  */
 sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C,
                     const void* bias, void* D, void* cuda_stream);

@@ -346,13 +346,29 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
             const double t_kb = kUsPerKBlock * bn / 256.0 * factor[pi][bi];
             const double t_fixed = kUsPerKBlock * bn / 256.0 * 96.0 / 64.0;
             double cost = static_cast<double>(waves) * (t_kb * static_cast<double>(num_kb > 0 ? num_kb : 1) + t_fixed);
+            // One row of tiles (M <= 128: a weight matrix streamed past a few activations): what bounds the time is
+            // how many of B's bytes are in flight -- `active` CTAs x stages x the B share of a stage -- against the
+            // memory latency under load (~1.9 us); the A share of every stage is mostly padding.  Parts of a K-split
+            // tile stream at ~4.7 TB/s at best and start ~2 us later.  Fitted to 8..128 x {2048..14336} x {4096..14336}
+            // with every tiling forced, e.g. 16 x 8192 x 8192: 256-wide tiles in 4 column slices 45 us, in 4 K ranges
+            // 36 us, 128-wide 35 us, 64-wide 31 us.
+            auto stream_us = [&](int64_t active, bool k_ranges) {
+                const double stages = std::min(8.0, std::floor(192.0 * 1024.0 / (16384.0 + 128.0 * bn)));
+                const double in_flight = static_cast<double>(std::min<int64_t>(active, slots)) * stages * 128.0 * bn;
+                const double b_bytes = static_cast<double>(N) * static_cast<double>(K) * mem.esize_in * static_cast<double>(batch_mult) *
+                                       static_cast<double>(rows_per_problem.size());
+                return b_bytes / std::min(k_ranges ? 4.7e6 : 7.0e6, in_flight / 1.9) + (k_ranges ? 2.0 : 0.0);
+            };
+            const bool one_tile_row = mem.epi >= 0 && !pi && max_rows <= 128;
+            if (one_tile_row) cost = std::max(cost, stream_us(tiles, false));
             if (can_split && tiles * 2 <= slots) {
                 // less than half a wave: plan_tail may cut every tile's K loop into ranges run by different SMs
                 int64_t ks_max = slots / tiles;
                 if (ks_max > 16) ks_max = 16;
                 if (ks_max > num_kb) ks_max = num_kb;
                 for (int64_t ks = 2; ks <= ks_max; ++ks) {
-                    const double t = t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed + ksplit_exchange_us(ks);
+                    double t = t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed + ksplit_exchange_us(ks);
+                    if (one_tile_row) t = std::max(t, stream_us(tiles * ks, true) + ksplit_exchange_us(ks));
                     if (t < cost) cost = t;
                 }
             }
@@ -701,7 +717,7 @@ sg_status_t upload(const std::vector<uint8_t>& host, void* dev, cudaStream_t str
 }
 
 // ------------------------------------------------------------------------------------------ matrix-vector products
-// A GEMM with N = 1 (the matrix is A) or M = 1 (the matrix is B) whose matrix is K-contiguous and whose vector is
+// A GEMM with N <= 4 (the matrix is A) or M <= 4 (the matrix is B) whose matrix is K-contiguous and whose vectors are
 // contiguous runs as a stream over the matrix (sg_gemv.cuh) instead of through the tensor-core tiles.  *taken is false
 // when the call does not have that form (the general path then validates and runs it).
 template <typename T>
@@ -718,11 +734,19 @@ cudaError_t launch_gemv(const GemvParams& gp, int rb, int ctas, cudaStream_t str
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    const int nv = gp.nvec <= 1 ? 1 : (gp.nvec == 2 ? 2 : 4);
+#define SG_GEMV_CASE(RB_)                                                             \
+    case RB_:                                                                         \
+        return nv == 1   ? cudaLaunchKernelEx(&cfg, gemv_kernel<T, RB_, 1>, gp)       \
+               : nv == 2 ? cudaLaunchKernelEx(&cfg, gemv_kernel<T, RB_, 2>, gp)       \
+                         : cudaLaunchKernelEx(&cfg, gemv_kernel<T, RB_, 4>, gp);
     switch (rb) {
-        case 4: return cudaLaunchKernelEx(&cfg, gemv_kernel<T, 4>, gp);
-        case 2: return cudaLaunchKernelEx(&cfg, gemv_kernel<T, 2>, gp);
-        default: return cudaLaunchKernelEx(&cfg, gemv_kernel<T, 1>, gp);
+        SG_GEMV_CASE(4)
+        SG_GEMV_CASE(2)
+        default:
+            SG_GEMV_CASE(1)
     }
+#undef SG_GEMV_CASE
 }
 
 sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C, const void* bias, void* D,
@@ -731,18 +755,22 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     if (!desc || desc->K < 1 || desc->K > INT32_MAX || desc->M < 1 || desc->N < 1) return SG_OK;
     static const bool off = getenv("SG_NO_GEMV") != nullptr;     // tests: the same product through the tiles
     if (off) return SG_OK;
-    const bool mat_a = desc->N == 1;
-    if (!mat_a && desc->M != 1) return SG_OK;
+    // up to four vectors; the matrix is the operand with more rows
+    const bool mat_a = desc->N <= 4 && desc->M >= desc->N;
+    if (!mat_a && desc->M > 4) return SG_OK;
     if (desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F16 && desc->in_dtype != SG_F32) return SG_OK;
     const int es = desc->in_dtype == SG_F32 ? 4 : 2;
-    // the matrix K-contiguous, the vector contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
+    // the matrix K-contiguous, the vectors contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
     const bool a_kc = desc->layout_a == SG_ROW_MAJOR, b_kc = desc->layout_b == SG_COL_MAJOR;
     const void* W = mat_a ? A : B;
     const void* x = mat_a ? B : A;
     const int64_t ld = mat_a ? desc->lda : desc->ldb;
     const int64_t R = mat_a ? desc->M : desc->N;
-    if (mat_a ? !(a_kc && (b_kc || desc->ldb == 1)) : !(b_kc && (a_kc || desc->lda == 1))) return SG_OK;
+    const int64_t nvec = mat_a ? desc->N : desc->M;
+    const int64_t x_stride = mat_a ? desc->ldb : desc->lda;
+    if (mat_a ? !(a_kc && (b_kc || (nvec == 1 && desc->ldb == 1))) : !(b_kc && (a_kc || (nvec == 1 && desc->lda == 1)))) return SG_OK;
     if (R > INT32_MAX || ld < desc->K || (ld * es) % 16 || !W || !x || !aligned16(W) || !aligned16(x)) return SG_OK;
+    if (nvec > 1 && (x_stride < desc->K || (x_stride * es) % 16)) return SG_OK;
     *taken = true;
 
     Checked c;
@@ -772,11 +800,16 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     gp.bias = bias;
     gp.D = D;
     gp.ld = ld;
-    gp.c_stride = mat_a ? desc->ldc : 1;
-    gp.d_stride = mat_a ? desc->ldd : 1;
+    gp.x_stride = x_stride;
+    gp.c_row_stride = mat_a ? desc->ldc : 1;
+    gp.c_vec_stride = mat_a ? 1 : desc->ldc;
+    gp.d_row_stride = mat_a ? desc->ldd : 1;
+    gp.d_vec_stride = mat_a ? 1 : desc->ldd;
     gp.R = static_cast<int32_t>(R);
     gp.K = static_cast<int32_t>(desc->K);
-    gp.bias_stride = mat_a ? 0 : 1;
+    gp.nvec = static_cast<int32_t>(nvec);
+    gp.bias_row_stride = mat_a ? 0 : 1;
+    gp.bias_vec_stride = mat_a ? 1 : 0;
     gp.out_kind = c.out_kind;
     gp.epi = desc->epi;
     gp.alpha = desc->alpha;

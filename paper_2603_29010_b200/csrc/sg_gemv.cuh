@@ -1,6 +1,7 @@
-// Matrix-vector product with the fused epilogue: out[r] = act(alpha * sum_k W[r][k] x[k] + beta * C[r] + bias[r]).
-// The GEMM with N = 1 (or M = 1) of the paper's workload list (single-token decode): every matrix element is used
-// once, so the kernel is a stream over W bound by HBM, and the tensor cores have nothing to offer.
+// Matrix-vector product with the fused epilogue: out[r] = act(alpha * sum_k W[r][k] x[k] + beta * C[r] + bias[r]),
+// for up to four vectors x at once.  The GEMM with N <= 4 (or M <= 4) of the paper's workload list (single-token
+// decode): every matrix element is used once per vector, so the kernel is a stream over W bound by HBM, and the
+// tensor cores (128-row tiles for at most four useful rows) have nothing to offer.
 //
 // Work split: a CTA of 256 threads takes RB consecutive rows and one K range; each thread walks the range in
 // 16-byte vectors (one vector of x serves RB vectors of W, so RB independent loads are in flight per thread and
@@ -17,16 +18,18 @@ namespace sg {
 
 struct GemvParams {
     const void* W;        // [R][ld], K contiguous
-    const void* x;        // [K], contiguous
+    const void* x;        // nvec vectors [K], contiguous, x_stride elements apart
     const void* C;        // residual (output type) or null
     const void* bias;     // input type (fp32 for fp32 inputs) or null
     void* D;
     int64_t ld;           // elements between rows of W
-    int64_t c_stride, d_stride;   // elements between consecutive rows' entries of C and D
+    int64_t x_stride;
+    int64_t c_row_stride, c_vec_stride, d_row_stride, d_vec_stride;   // element (row r, vector v) of C and D
     int32_t R, K;
+    int32_t nvec;         // 1..4
     int32_t kchunk;       // K elements per cluster rank (a multiple of 256 vectors)
     int32_t ksplit;       // CTAs per cluster
-    int32_t bias_stride;  // 0: one bias for all rows (N = 1), 1: one per row (M = 1)
+    int32_t bias_row_stride, bias_vec_stride;   // (0, 1): one bias per vector (the matrix is A); (1, 0): one per row
     int32_t out_kind;     // 0 bf16, 1 fp32, 2 fp16
     int32_t epi;
     float alpha, beta, a0, a1;
@@ -95,13 +98,17 @@ __device__ __forceinline__ void gemv_store_out(void* base, int64_t i, int out_ki
 
 // Four rows per CTA and a register budget that lets four CTAs of 16-bit inputs share an SM measured best (more,
 // smaller CTAs balance better over the SMs than eight rows per CTA; deeper unrolling did not help).
-template <typename T, int RB>
-__global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4) ? 4 : 1) gemv_kernel(const GemvParams p) {
+// NV = vectors handled at once (1, 2 or 4; three vectors run as four with the last one repeated and not stored);
+// with several vectors a budget of 85 registers (three CTAs per SM) measured best: two leave too few loads in
+// flight, four spill.
+template <typename T, int RB, int NV>
+__global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4 && NV == 1) ? 4 : (NV > 1 ? 3 : 1)) gemv_kernel(const GemvParams p) {
     namespace cg = cooperative_groups;
     constexpr int V = GemvVec<T>::N;
     constexpr int WARPS = 8;
-    __shared__ float warp_part[WARPS][RB];
-    __shared__ float cta_part[RB];
+    constexpr int NACC = RB * NV;
+    __shared__ float warp_part[WARPS][NACC];
+    __shared__ float cta_part[NACC];
 
     const int ks = p.ksplit;
     const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));      // = rank in the (ks, 1, 1) cluster
@@ -110,7 +117,9 @@ __global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4) ? 4 : 1) gemv
     const int kend = min(p.K, kbeg + p.kchunk);
     const int kvec_end = kbeg < kend ? kbeg + ((kend - kbeg) / V) * V : kbeg;
 
-    const T* x = reinterpret_cast<const T*>(p.x);
+    const T* x[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) x[v] = reinterpret_cast<const T*>(p.x) + static_cast<int64_t>(min(v, p.nvec - 1)) * p.x_stride;
     const T* w[RB];
 #pragma unroll
     for (int i = 0; i < RB; ++i) {
@@ -118,66 +127,86 @@ __global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4) ? 4 : 1) gemv
         const int64_t r = min(r0 + i, static_cast<int64_t>(p.R) - 1);
         w[i] = reinterpret_cast<const T*>(p.W) + r * p.ld;
     }
-    float acc[RB];
+    float acc[RB][NV];
 #pragma unroll
-    for (int i = 0; i < RB; ++i) acc[i] = 0.0f;
+    for (int i = 0; i < RB; ++i) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) acc[i][v] = 0.0f;
+    }
 
 #pragma unroll 2
     for (int k = kbeg + static_cast<int>(threadIdx.x) * V; k < kvec_end; k += 256 * V) {
-        uint4 wv[RB];
+        uint4 wv[RB], xv[NV];
 #pragma unroll
         for (int i = 0; i < RB; ++i) wv[i] = ldg_stream16(w[i] + k);
-        float xf[V];
-        GemvVec<T>::cvt(__ldg(reinterpret_cast<const uint4*>(x + k)), xf);
 #pragma unroll
-        for (int i = 0; i < RB; ++i) {
-            float wf[V];
-            GemvVec<T>::cvt(wv[i], wf);
+        for (int v = 0; v < NV; ++v) xv[v] = __ldg(reinterpret_cast<const uint4*>(x[v] + k));
+        float wf[RB][V];
 #pragma unroll
-            for (int j = 0; j < V; ++j) acc[i] = fmaf(wf[j], xf[j], acc[i]);
+        for (int i = 0; i < RB; ++i) GemvVec<T>::cvt(wv[i], wf[i]);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            float xf[V];
+            GemvVec<T>::cvt(xv[v], xf);
+#pragma unroll
+            for (int i = 0; i < RB; ++i) {
+#pragma unroll
+                for (int j = 0; j < V; ++j) acc[i][v] = fmaf(wf[i][j], xf[j], acc[i][v]);
+            }
         }
     }
     // the last K % V elements (only the last rank has any)
     {
         const int kt = kvec_end + static_cast<int>(threadIdx.x);
         if (kt < kend) {
-            const float xv = GemvVec<T>::one(x + kt);
 #pragma unroll
-            for (int i = 0; i < RB; ++i) acc[i] = fmaf(GemvVec<T>::one(w[i] + kt), xv, acc[i]);
+            for (int v = 0; v < NV; ++v) {
+                const float xv = GemvVec<T>::one(x[v] + kt);
+#pragma unroll
+                for (int i = 0; i < RB; ++i) acc[i][v] = fmaf(GemvVec<T>::one(w[i] + kt), xv, acc[i][v]);
+            }
         }
     }
 
 #pragma unroll
     for (int i = 0; i < RB; ++i) {
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc[i] += __shfl_xor_sync(0xFFFFFFFFu, acc[i], off);
+        for (int v = 0; v < NV; ++v) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc[i][v] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][v], off);
+        }
     }
     const int warp = static_cast<int>(threadIdx.x) >> 5, lane = static_cast<int>(threadIdx.x) & 31;
     if (lane == 0) {
 #pragma unroll
-        for (int i = 0; i < RB; ++i) warp_part[warp][i] = acc[i];
+        for (int i = 0; i < RB; ++i) {
+#pragma unroll
+            for (int v = 0; v < NV; ++v) warp_part[warp][i * NV + v] = acc[i][v];
+        }
     }
     __syncthreads();
-    if (threadIdx.x < RB) {
+    if (threadIdx.x < NACC) {
         float s = 0.0f;
 #pragma unroll
         for (int wi = 0; wi < WARPS; ++wi) s += warp_part[wi][threadIdx.x];
         cta_part[threadIdx.x] = s;
     }
     if (ks > 1) cg::this_cluster().sync();
-    if (rank == 0 && threadIdx.x < RB) {
+    if (rank == 0 && threadIdx.x < NACC) {
         float s = cta_part[threadIdx.x];
         if (ks > 1) {
             cg::cluster_group cluster = cg::this_cluster();
             for (int r = 1; r < ks; ++r) s += *cluster.map_shared_rank(&cta_part[threadIdx.x], r);
         }
-        const int64_t row = r0 + threadIdx.x;
-        if (row < p.R) {
+        const int64_t row = r0 + static_cast<int>(threadIdx.x) / NV;
+        const int vec = static_cast<int>(threadIdx.x) % NV;
+        if (row < p.R && vec < p.nvec) {
             float v[1] = {p.alpha * s};
-            if (p.beta != 0.0f) v[0] = fmaf(p.beta, gemv_load_out(p.C, row * p.c_stride, p.out_kind), v[0]);
-            if (p.bias != nullptr) v[0] += GemvVec<T>::exact(reinterpret_cast<const T*>(p.bias) + row * p.bias_stride);
+            if (p.beta != 0.0f) v[0] = fmaf(p.beta, gemv_load_out(p.C, row * p.c_row_stride + vec * p.c_vec_stride, p.out_kind), v[0]);
+            if (p.bias != nullptr)
+                v[0] += GemvVec<T>::exact(reinterpret_cast<const T*>(p.bias) + row * p.bias_row_stride + vec * p.bias_vec_stride);
             if (p.epi >= EPI_RELU) apply_act_chunk<false, 1>(v, p.epi, p.a0, p.a1);
-            gemv_store_out(p.D, row * p.d_stride, p.out_kind, v[0]);
+            gemv_store_out(p.D, row * p.d_row_stride + vec * p.d_vec_stride, p.out_kind, v[0]);
         }
     }
     if (ks > 1) cg::this_cluster().sync();      // keep every rank's shared memory alive until rank 0 has read it

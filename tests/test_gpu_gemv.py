@@ -74,6 +74,37 @@ def test_matrix_times_vector_real_values_with_epilogue(R, K, dtype, out_dtype, e
     parity.assert_matches(D, ref, absacc, f"vector-matrix {R}x{K} {dtype} {epi}")
 
 
+@pytest.mark.parametrize("nvec", [2, 3, 4])
+@pytest.mark.parametrize("R,K", [(4096, 4096), (130, 66000), (5, 1000)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
+def test_up_to_four_vectors_in_one_pass(R, K, nvec, dtype):
+    g = torch.Generator().manual_seed(R + K + nvec)
+    out_dtype = torch.float32 if dtype == torch.float32 else dtype
+    W = (torch.randn(R, K, generator=g) / 8).to(dtype)
+    X = (torch.randn(nvec, K, generator=g) / 8).to(dtype)
+    # matrix on the left: D [R, nvec], bias per vector
+    C = torch.randn(R, nvec, generator=g).to(out_dtype)
+    bias = torch.randn(nvec, generator=g).to(dtype)
+    ref, absacc = orc.gemm(W, X, C=C, bias=bias, alpha=0.5, beta=-1.0, epi="tanh")
+    D = sg.gemm(W.to(DEV), X.to(DEV), C=C.to(DEV), bias=bias.to(DEV), alpha=0.5, beta=-1.0, epi="tanh", out_dtype=out_dtype)
+    assert _took_vector_path()
+    parity.assert_matches(D, ref, absacc, f"{R}x{K} times {nvec} vectors {dtype}")
+    # vectors on the left (a decode batch): D [nvec, R], bias per matrix row
+    Ct = torch.randn(nvec, R, generator=g).to(out_dtype)
+    biasR = torch.randn(R, generator=g).to(dtype)
+    ref, absacc = orc.gemm(X, W, C=Ct, bias=biasR, beta=0.5, epi="silu")
+    D = sg.gemm(X.to(DEV), W.to(DEV), C=Ct.to(DEV), bias=biasR.to(DEV), beta=0.5, epi="silu", out_dtype=out_dtype)
+    assert _took_vector_path()
+    parity.assert_matches(D, ref, absacc, f"{nvec} vectors times {R}x{K} {dtype}")
+    # small integers: exact
+    Wi = inputs.small_integers([R, K], 91, 1, lo=-2, hi=2).to(dtype)
+    Xi = inputs.small_integers([nvec, K], 91, 2, lo=-2, hi=2).to(dtype)
+    ref, _ = orc.gemm(Xi, Wi)
+    Di = torch.full((nvec, R), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(Xi.to(DEV), Wi.to(DEV), out=Di)
+    parity.assert_bit_exact(Di, ref, f"{nvec} integer vectors times {R}x{K} {dtype}")
+
+
 def test_padded_rows_strided_outputs_and_a_column_vector_operand():
     g = torch.Generator().manual_seed(11)
     R, K, ld = 517, 1003, 1008                         # K is no multiple of a 16-byte vector; rows padded to one
@@ -102,9 +133,15 @@ def test_results_do_not_depend_on_the_run():
 def test_other_forms_still_go_through_the_tiles():
     g = torch.Generator().manual_seed(4)
     A = torch.randn(256, 64, generator=g).to(torch.bfloat16)
-    B2 = torch.randn(2, 64, generator=g).to(torch.bfloat16)
+    B5 = torch.randn(5, 64, generator=g).to(torch.bfloat16)
     out = torch.empty(256, 8, dtype=torch.bfloat16, device=DEV)
-    sg.gemm(A.to(DEV), B2.to(DEV), out=out[:, :2])
+    sg.gemm(A.to(DEV), B5.to(DEV), out=out[:, :5])
     assert not _took_vector_path()
-    ref, absacc = orc.gemm(A, B2)
-    parity.assert_matches(out[:, :2], ref, absacc, "N = 2")
+    ref, absacc = orc.gemm(A, B5)
+    parity.assert_matches(out[:, :5], ref, absacc, "N = 5")
+    # a K x 2 row-major B is not a pair of contiguous vectors
+    Brow = torch.randn(64, 8, generator=g).to(torch.bfloat16)
+    sg.gemm(A.to(DEV), Brow.to(DEV)[:, :2], layout_b="row", out=out[:, :2])
+    assert not _took_vector_path()
+    ref, absacc = orc.gemm(A, Brow[:, :2], layout_b="row")
+    parity.assert_matches(out[:, :2], ref, absacc, "N = 2, row-major B")
