@@ -81,6 +81,8 @@ KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 
         case 3: return kernel_variant_3(bn, pair, out, epi_warps);
         case 4: return kernel_variant_4(bn, pair, out, epi_warps);
         case 5: return kernel_variant_5(bn, pair, out, epi_warps);
+        case 6: return kernel_variant_6(bn, pair, out, epi_warps);
+        case 7: return kernel_variant_7(bn, pair, out, epi_warps);
         default: return kernel_variant_0(bn, pair, out, epi_warps);
     }
 }
@@ -130,7 +132,8 @@ sg_status_t device_state(DeviceState** out) {
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
                     for (int f32 = 0; f32 < 3 && d.init_status == SG_OK; ++f32)
                         for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4)
-                            for (int variant = 0; variant < 6 && d.init_status == SG_OK; ++variant) {
+                            for (int variant = 0; variant < 8 && d.init_status == SG_OK; ++variant) {
+                                if (variant >= 6 && pair) continue;      // the short-A variants have no two-CTA form
                                 KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew, variant);
                                 e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
                                 if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
@@ -353,7 +356,9 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
             // with every tiling forced, e.g. 16 x 8192 x 8192: 256-wide tiles in 4 column slices 45 us, in 4 K ranges
             // 36 us, 128-wide 35 us, 64-wide 31 us.
             auto stream_us = [&](int64_t active, bool k_ranges) {
-                const double stages = std::min(8.0, std::floor(192.0 * 1024.0 / (16384.0 + 128.0 * bn)));
+                // with at most 64 (32) rows only that many rows of A are loaded per stage, and up to 16 stages fit
+                const double a_bytes = k_ranges || max_rows > 64 ? 16384.0 : (max_rows > 32 ? 8192.0 : 4096.0);
+                const double stages = std::min(a_bytes < 16384.0 ? 16.0 : 8.0, std::floor(192.0 * 1024.0 / (a_bytes + 128.0 * bn)));
                 const double in_flight = static_cast<double>(std::min<int64_t>(active, slots)) * stages * 128.0 * bn;
                 const double b_bytes = static_cast<double>(N) * static_cast<double>(K) * mem.esize_in * static_cast<double>(batch_mult) *
                                        static_cast<double>(rows_per_problem.size());
@@ -505,7 +510,7 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     int variant = 0;
     if (!no_lean && !p.in_fp8) {
         const bool plain = !p.a_mn_major && !p.b_mn_major && p.ksplit <= 1 && !p.d_remap && p.nphases <= 1;
-        if (p.mode == MODE_DENSE && plain) variant = p.ex_any ? 4 : 1;
+        if (p.mode == MODE_DENSE && plain) variant = p.ex_any ? 4 : (p.a_rows == 64 ? 6 : (p.a_rows == 32 ? 7 : 1));
         else if (p.mode == MODE_CONV && plain && !p.ex_any) variant = 2;
         else if (p.mode == MODE_GROUPED && plain && !p.ex_any) variant = 3;
         else if (p.mode == MODE_CONV && !p.a_mn_major && p.b_mn_major && p.ksplit <= 1 && !p.ex_any) variant = 5;
@@ -637,6 +642,12 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     plan_tail(*d, s, tiles, &p, min_b_rows);
     st = apply_ex(&p, ex, desc->N, c.esize_out, who);
     if (st != SG_OK) return st;
+    // a few rows against a large matrix: load only 32 or 64 rows of A per stage (kernel variants 6 and 7), which
+    // leaves room for more stages of B
+    static const bool no_short_a = getenv("SG_NO_SHORT_A") != nullptr;      // experiments
+    p.a_rows = 128;
+    if (!no_short_a && !s.pair && !p.in_fp8 && !p.a_mn_major && !p.b_mn_major && p.ksplit <= 1 && !p.ex_any && desc->M <= 64)
+        p.a_rows = desc->M <= 32 ? 32 : 64;
     p.bias = bias;
     p.C = desc->beta != 0.0f ? C : nullptr;
     p.ldc = desc->ldc;
@@ -651,7 +662,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
         if (p.a_mn_major)
             st = make_tiled_map(&p.tmA, c.tm_in, c.esize_in, A, desc->M, desc->K, batch, desc->lda, sA, 64, 64, "A");
         else
-            st = make_tiled_map(&p.tmA, c.tm_in, c.esize_in, A, desc->K, desc->M, batch, desc->lda, sA, c.bk, 128, "A");
+            st = make_tiled_map(&p.tmA, c.tm_in, c.esize_in, A, desc->K, desc->M, batch, desc->lda, sA, c.bk, p.a_rows, "A");
         if (st != SG_OK) return st;
         if (p.b_mn_major) {
             st = make_tiled_map(&p.tmB, c.tm_in, c.esize_in, B, desc->N, desc->K, batch, desc->ldb, sB, 64, 64, "B");

@@ -94,6 +94,7 @@ struct alignas(64) Params {
     // conv (strided data gradient): row m = (n, i, j) of this launch's output is pixel (n, remap_h0 + remap_sh * i,
     // remap_w0 + remap_sw * j) of the remap_H x remap_W image that C and D address; 0 = rows are stored as they come
     int32_t d_remap, remap_h0, remap_sh, remap_w0, remap_sw, remap_H, remap_W;
+    int32_t a_rows;                     // rows of A loaded per tile (128; 64 or 32 in the short-A variants)
     int32_t nphases;                    // > 1: the tile list is the concatenation of ph[0 .. nphases), A maps in tmPh
     ConvPhase ph[kMaxPhases];
     CUtensorMap tmPh[kMaxPhases];
@@ -387,22 +388,28 @@ static __device__ __noinline__ bool wait_counter(const uint32_t* counter, uint32
     return true;
 }
 
-template <int BN, bool kPair, int kEpiWarps = 4>
+// A_ROWS: rows of the A tile that are loaded.  128 = the whole tile; 64 or 32 when the problem has no more rows than
+// that (a few activations against a large weight matrix): the A share of a stage shrinks to those rows, so more
+// stages fit and more of B is in flight.  The MMA still reads 128 rows from the stage's A address -- the rows past
+// A_ROWS are whatever follows in shared memory (the stage's B tile, later stages, the staging area: always inside the
+// CTA's allocation) and produce accumulator rows past M, which no store ever writes.
+template <int BN, bool kPair, int kEpiWarps = 4, int A_ROWS = 128>
 struct Config {
     static constexpr int kCtas = kPair ? 2 : 1;
     static constexpr int BM = 128;                 // rows per CTA (= TMEM lanes)
     static constexpr int TILE_M = BM * kCtas;      // rows per tile
     static constexpr int BK = 64;                  // 64 bf16 = one 128-byte swizzled row
     static constexpr int B_ROWS = BN / kCtas;      // rows of the B tile this CTA loads
-    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int A_BYTES = A_ROWS * BK * 2;
     static constexpr int B_BYTES = B_ROWS * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES_RAW = (192 * 1024) / STAGE_BYTES;
 #ifdef SG_MAX_STAGES
     static constexpr int STAGES = STAGES_RAW > SG_MAX_STAGES ? SG_MAX_STAGES : STAGES_RAW;   // experiments only
 #else
-    static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+    static constexpr int STAGES = STAGES_RAW > (A_ROWS < 128 ? 16 : 8) ? (A_ROWS < 128 ? 16 : 8) : STAGES_RAW;
 #endif
+    static_assert(A_ROWS == 128 || !kPair, "short A tiles are for single-CTA tiles");
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;   // BN in {64,128,256} -> power of two
     static constexpr int EPI_WARPS = kEpiWarps;                    // 4: one per TMEM lane quarter; 8: two, alternating chunks
     static constexpr int CHUNK_STEP = EPI_WARPS / 4;
@@ -427,14 +434,17 @@ struct Config {
 // 85.8 -> 81.8 us, 128 x (256 x 256 x 512) 19.6 -> 18.75 us, 256^3 6.3 -> 4.7 us, each pair timed in one GPU call).
 template <int BN, bool kPair, int kOut, int kEpiWarps, int kV = 0>
 __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) contract_kernel(const __grid_constant__ Params p) {
-    using Cfg = Config<BN, kPair, kEpiWarps>;
+    // variants 6 and 7 are variant 1 with an A tile of 64 resp. 32 loaded rows
+    constexpr int kARows = kV == 6 ? 64 : (kV == 7 ? 32 : 128);
+    constexpr int kVB = kV >= 6 ? 1 : kV;
+    using Cfg = Config<BN, kPair, kEpiWarps, kARows>;
     // options the specialised variants fold away at compile time
-    constexpr bool kLean = kV != 0;
-    const int32_t mode = (kV == 1 || kV == 4) ? MODE_DENSE : ((kV == 2 || kV == 5) ? MODE_CONV : (kV == 3 ? MODE_GROUPED : p.mode));
+    constexpr bool kLean = kVB != 0;
+    const int32_t mode = (kVB == 1 || kVB == 4) ? MODE_DENSE : ((kVB == 2 || kVB == 5) ? MODE_CONV : (kVB == 3 ? MODE_GROUPED : p.mode));
     const bool a_mn = kLean ? false : p.a_mn_major != 0;
-    const bool b_mn = kLean ? kV == 5 : p.b_mn_major != 0;
-    const bool d_remap = (kV == 0 || kV == 5) ? p.d_remap != 0 : false;
-    const bool phased = (kV == 0 || kV == 5) ? p.nphases > 1 : false;
+    const bool b_mn = kLean ? kVB == 5 : p.b_mn_major != 0;
+    const bool d_remap = (kVB == 0 || kVB == 5) ? p.d_remap != 0 : false;
+    const bool phased = (kVB == 0 || kVB == 5) ? p.nphases > 1 : false;
     constexpr int kCtas = Cfg::kCtas;
     constexpr int STAGES = Cfg::STAGES;
     constexpr bool kOutF32 = (kOut == 1);
@@ -504,7 +514,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         if (mode == MODE_DENSE && !a_mn && !b_mn && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
             static_cast<int>(blockIdx.x) < p.num_tiles) {
             int g_hint0 = 0;
-            const Tile t0 = decode_tile<Cfg::TILE_M, BN, kV>(p, static_cast<int>(blockIdx.x), g_hint0);
+            const Tile t0 = decode_tile<Cfg::TILE_M, BN, kVB>(p, static_cast<int>(blockIdx.x), g_hint0);
             if (t0.n0 < p.N) {
                 early_kb = min(STAGES, t0.kb1 - t0.kb0);
                 if (threadIdx.x == 0) {
@@ -557,7 +567,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             uint32_t phase = 0;
             int g_hint = 0, g_fenced = -1;
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
+                Tile ti = decode_tile<Cfg::TILE_M, BN, kVB>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
                 const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
@@ -690,7 +700,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const uint64_t b_desc0 = b_mn ? smem_desc_mn_major_sw128(smem_base + Cfg::A_BYTES)
                                                   : smem_desc_k_major_sw128(smem_base + Cfg::A_BYTES);
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                const Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
+                const Tile ti = decode_tile<Cfg::TILE_M, BN, kVB>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
                 if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
                 const int in_kind = kLean ? 0 : p.in_fp8;          // 0 sixteen-bit, 1 / 2 fp8, 3 tf32, 4 int8
@@ -776,7 +786,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         for (int a = 0; a < 2; ++a) tempty_remote[a] = kPair ? map_to_cta(tempty_bar(a), 0) : tempty_bar(a);
 
         for (int t = first_tile; t < p.num_tiles && ok; t += tile_step) {
-            Tile ti = decode_tile<Cfg::TILE_M, BN, kV>(p, t, g_hint);
+            Tile ti = decode_tile<Cfg::TILE_M, BN, kVB>(p, t, g_hint);
             if (ti.n0 >= p.N) continue;
             const bool has_k = num_kb > 0 && ti.kb1 > ti.kb0;   // else the tile is the empty sum: no accumulator is involved
             const int acc = iter & 1;
@@ -846,7 +856,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // from its own accumulator plus the other parts' parked sums
             // (pass 1), so the exchange is spread over all parts instead of serialised in one.  The unit of ownership
             // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
-            const bool ksplit_tile = kV == 0 ? ti.nparts > 1 : false;
+            const bool ksplit_tile = kVB == 0 ? ti.nparts > 1 : false;
             // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
             auto owned_by = [&](int c, int qq) { return (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
             auto owned = [&](int c) { return owned_by(c, q); };
@@ -1019,7 +1029,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int i = 0; i < CH; ++i) v[i] *= alpha;
                 }
-                const bool ex_any = (kV == 0 || kV == 4) ? p.ex_any != 0 : false;
+                const bool ex_any = (kVB == 0 || kVB == 4) ? p.ex_any != 0 : false;
                 if (ex_any) {
                     if (p.row_scale != nullptr) {
                         const float rs = row < ti.rows ? __ldg(p.row_scale + row) : 0.0f;
