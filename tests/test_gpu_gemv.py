@@ -145,3 +145,41 @@ def test_other_forms_still_go_through_the_tiles():
     assert not _took_vector_path()
     ref, absacc = orc.gemm(A, Brow[:, :2], layout_b="row")
     parity.assert_matches(out[:, :2], ref, absacc, "N = 2, row-major B")
+
+
+@pytest.mark.parametrize("M", [5, 16, 32, 33, 64, 65])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_few_rows_against_a_large_matrix_on_the_tiles(M, dtype):
+    # 5..64 rows: the tensor-core tiles with only 32 or 64 rows of A loaded per stage; 65: the full A tile
+    g = torch.Generator().manual_seed(100 + M)
+    N, K = 1080, 2056
+    A = (torch.randn(M, K, generator=g) / 8).to(dtype)
+    W = (torch.randn(N, K, generator=g) / 8).to(dtype)
+    C = torch.randn(M, N, generator=g).to(dtype)
+    bias = torch.randn(N, generator=g).to(dtype)
+    ref, absacc = orc.gemm(A, W, C=C, bias=bias, alpha=1.5, beta=0.5, epi="gelu")
+    D = sg.gemm(A.to(DEV), W.to(DEV), C=C.to(DEV), bias=bias.to(DEV), alpha=1.5, beta=0.5, epi="gelu", out_dtype=dtype)
+    assert not _took_vector_path()
+    parity.assert_matches(D, ref, absacc, f"{M} rows x {N} x {K} {dtype}")
+    # exact on integers, through every tile width
+    Ai = inputs.small_integers([M, K], 92, 1).to(dtype)
+    Wi = inputs.small_integers([N, K], 92, 2).to(dtype)
+    refi, _ = orc.gemm(Ai, Wi)
+    for tile_n in (64, 128, 256):
+        sg.set_tuning(tile_n, 0)
+        Di = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+        sg.gemm(Ai.to(DEV), Wi.to(DEV), out=Di)
+        parity.assert_bit_exact(Di, refi, f"{M} integer rows, tile width {tile_n}")
+    sg.set_tuning(-1, -1)
+
+
+def test_few_rows_batched():
+    g = torch.Generator().manual_seed(77)
+    batch, M, N, K = 3, 20, 200, 264
+    A = (torch.randn(batch, M, K, generator=g) / 4).to(torch.bfloat16)
+    W = (torch.randn(batch, N, K, generator=g) / 4).to(torch.bfloat16)
+    bias = torch.randn(batch, N, generator=g).to(torch.bfloat16)
+    D = sg.batched_gemm(A.to(DEV), W.to(DEV), bias=bias.to(DEV), epi="relu")
+    for b in range(batch):
+        ref, absacc = orc.gemm(A[b], W[b], bias=bias[b], epi="relu")
+        parity.assert_matches(D[b], ref, absacc, f"few rows, batch {b}")

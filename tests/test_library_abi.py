@@ -74,6 +74,14 @@ def _call_gemm(sg, desc, A=0x1000, B=0x2000, C=None, bias=None, D=0x3000):
     (dict(in_dtype=1, lda=130), {}, "SG_ERR_ALIGNMENT"),           # 130 fp32 elements = 520 bytes
     (dict(layout_a=1, lda=64), {}, "SG_ERR_INVALID_ARG"),       # column-major A: lda must cover M = 128
     (dict(layout_b=7), {}, "SG_ERR_INVALID_ARG"),
+    # matrix-vector form (N <= 4 or M <= 4): its own, relaxed checks, still before any launch
+    (dict(N=1, ldd=1), dict(D=None), "SG_ERR_NULL_POINTER"),
+    (dict(N=1, ldd=1, ldc=1, beta=1.0), {}, "SG_ERR_NULL_POINTER"),
+    (dict(M=1, epi=1), {}, "SG_ERR_NULL_POINTER"),
+    (dict(N=3, ldd=3, out_dtype=5), {}, "SG_ERR_UNSUPPORTED"),
+    (dict(N=2, ldd=1), {}, "SG_ERR_INVALID_ARG"),                       # ldd < N
+    (dict(N=1, ldd=1), dict(D=0x3001), "SG_ERR_ALIGNMENT"),              # a bf16 output on an odd address
+    (dict(N=1, ldd=1, lda=132), {}, "SG_ERR_ALIGNMENT"),                 # rows not 16-byte multiples: general path's rule
 ])
 def test_gemm_rejects_bad_arguments_before_any_launch(sg, kw, ptrs, want):
     before = sg.launch_count()
