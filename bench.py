@@ -273,6 +273,61 @@ def bench_extra_configs(sg, inputs, torch, dev, peaks, steps: int, torch_ref: bo
     return out
 
 
+def bench_shape_sweep(sg, torch, dev) -> dict:
+    """The GEMM shape classes of the paper's workload list (square, LLM-like, small and large K, irregular, tall-skinny,
+    matrix-vector, a few rows against a weight matrix, batched) through this library and, for context, through
+    torch.matmul / torch.bmm (library kernels), each as one CUDA graph over rotating buffer sets."""
+    bf = torch.bfloat16
+    out = {}
+
+    def time_graph(fns, reps=10):
+        for f in fns[:2]:
+            f()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for f in fns:
+                f()
+        graph.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(3):
+            best = min(best, time_steps(lambda i: graph.replay(), reps, torch) / (reps * len(fns)))
+        return best
+
+    def run(M, N, K, batch=1):
+        nbytes = batch * (M * K + N * K + M * N) * 2
+        sets = max(1, min(8, int(300e6 // nbytes) + 1))
+        shape = (lambda r, c: (r, c)) if batch == 1 else (lambda r, c: (batch, r, c))
+        As = [torch.randn(*shape(M, K), device=dev).to(bf) for _ in range(sets)]
+        Bs = [torch.randn(*shape(N, K), device=dev).to(bf) for _ in range(sets)]
+        Os = [torch.empty(*shape(M, N), dtype=bf, device=dev) for _ in range(sets)]
+        if batch == 1:
+            t = time_graph([(lambda i=i: sg.gemm(As[i], Bs[i], out=Os[i])) for i in range(sets)])
+            plan = sg.last_launch_plan()
+            tl = time_graph([(lambda i=i: torch.matmul(As[i], Bs[i].t(), out=Os[i])) for i in range(sets)])
+        else:
+            t = time_graph([(lambda i=i: sg.batched_gemm(As[i], Bs[i], out=Os[i])) for i in range(sets)])
+            plan = sg.last_launch_plan()
+            tl = time_graph([(lambda i=i: torch.bmm(As[i], Bs[i].transpose(1, 2), out=Os[i])) for i in range(sets)])
+        flops = 2.0 * batch * M * N * K
+        out[f"b{batch}_{M}x{N}x{K}"] = {"us": round(t * 1e6, 2), "tflops": round(flops / t / 1e12, 1), "gbs": round(nbytes / t / 1e9),
+                                        "library_us": round(tl * 1e6, 2), "library_over_ours": round(tl / t, 2),
+                                        "buffer_sets": sets, "plan": plan}
+
+    for shp in [(4096, 4096, 4096), (2048, 4096, 8192), (8192, 8192, 8192), (16384, 16384, 32), (16384, 16384, 64), (8192, 8192, 128),
+                (8192, 8192, 256), (256, 256, 131072), (4096, 4096, 14336), (4096, 14336, 4096), (2047, 2040, 2056), (1000, 1000, 1000),
+                (3000, 5000, 7000), (32768, 64, 4096), (32768, 128, 1024), (64, 32768, 4096), (512, 512, 512), (1024, 1024, 1024),
+                (2048, 2048, 2048), (8192, 1024, 8192), (1024, 8192, 8192),
+                (8192, 1, 8192), (4096, 1, 4096), (1, 8192, 8192), (1, 11008, 4096), (2, 8192, 8192), (4, 8192, 8192), (4, 4096, 14336),
+                (8, 4096, 14336), (16, 8192, 8192), (32, 4096, 4096), (64, 8192, 8192), (64, 14336, 4096), (128, 8192, 8192)]:
+        run(*shp)
+    for shp in [(512, 512, 64, 128), (512, 64, 512, 128), (2048, 2048, 128, 32), (2048, 128, 2048, 32), (128, 128, 128, 1024),
+                (1024, 1024, 1024, 16)]:
+        run(*shp)
+    return out
+
+
 def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
     """Kernel-only timings of the rows built beyond the five configurations: residual and extended epilogues, other
     input types and operand layouts, skinny long-K shapes, the transpose stage and the convolution gradients."""
@@ -580,6 +635,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         line["parity_sample_ok"] = bool(((got - ref).abs() <= 1e-2 + 1e-2 * ref.abs()).all())
         if args.widened:
             line["widened"] = bench_widened(sg, inputs, torch, dev, peaks)
+        if args.shape_sweep:
+            line["shape_sweep"] = bench_shape_sweep(sg, torch, dev)
         if args.all_configs:
             line["per_config"] = bench_extra_configs(sg, inputs, torch, dev, peaks, args.steps, args.torch_ref)
             if args.torch_ref:
@@ -603,6 +660,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--all-configs", action="store_true", help="also time the other four configurations (N=1 only)")
+    ap.add_argument("--shape-sweep", action="store_true",
+                    help="also time the workload list's GEMM shape classes, with torch's library kernels beside them")
     ap.add_argument("--widened", action="store_true",
                     help="also time the rows built beyond the five configurations (epilogue chain, dtypes, layouts, "
                          "skinny shapes, transpose, conv gradients; N=1 only)")
