@@ -110,7 +110,8 @@ typedef struct sg_gemm_desc {
  *   bias   device, in_dtype, [N]; may be NULL unless epi == SG_EPI_BIAS.
  *   D      device, out_dtype, [M,N] row-major; written in full (all M x N elements).
  * M == 0 or N == 0: SG_OK, nothing is launched.  K == 0: D = act(beta*C + bias).
- * Matrix-vector form (the workload list's single-token decode product): when N <= 4 (or M <= 4), the matrix operand is
+ * Matrix-vector form (the workload list's single-token decode product): when N <= 8 (or M <= 8; 4 for SG_F32 inputs or
+ *   when K is no multiple of 8), the matrix operand is
  *   K-contiguous (A row-major, resp. B column-major) and 16-byte aligned with a leading dimension that is a multiple
  *   of 16 bytes, the vectors are K-contiguous, 16-byte aligned and a multiple of 16 bytes apart (a single vector may
  *   also be stored as K x 1 with a leading dimension of 1), and in_dtype is SG_BF16, SG_F16 or SG_F32, the product

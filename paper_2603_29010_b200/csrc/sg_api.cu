@@ -728,7 +728,7 @@ sg_status_t upload(const std::vector<uint8_t>& host, void* dev, cudaStream_t str
 }
 
 // ------------------------------------------------------------------------------------------ matrix-vector products
-// A GEMM with N <= 4 (the matrix is A) or M <= 4 (the matrix is B) whose matrix is K-contiguous and whose vectors are
+// A GEMM with N <= 8 (the matrix is A) or M <= 8 (the matrix is B; fp32 inputs: 4) whose matrix is K-contiguous and whose vectors are
 // contiguous runs as a stream over the matrix (sg_gemv.cuh) instead of through the tensor-core tiles.  *taken is false
 // when the call does not have that form (the general path then validates and runs it).
 template <typename T>
@@ -766,11 +766,13 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     if (!desc || desc->K < 1 || desc->K > INT32_MAX || desc->M < 1 || desc->N < 1) return SG_OK;
     static const bool off = getenv("SG_NO_GEMV") != nullptr;     // tests: the same product through the tiles
     if (off) return SG_OK;
-    // up to four vectors; the matrix is the operand with more rows
-    const bool mat_a = desc->N <= 4 && desc->M >= desc->N;
-    if (!mat_a && desc->M > 4) return SG_OK;
+    // up to eight vectors of 16-bit inputs (four of fp32); the matrix is the operand with more rows
     if (desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F16 && desc->in_dtype != SG_F32) return SG_OK;
     const int es = desc->in_dtype == SG_F32 ? 4 : 2;
+    static const bool no_mma = getenv("SG_GEMV_NO_MMA") != nullptr;      // experiments: FMA kernel only (<= 4 vectors)
+    const int64_t max_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? 8 : 4;
+    const bool mat_a = desc->N <= max_vec && desc->M >= desc->N;
+    if (!mat_a && desc->M > max_vec) return SG_OK;
     // the matrix K-contiguous, the vectors contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
     const bool a_kc = desc->layout_a == SG_ROW_MAJOR, b_kc = desc->layout_b == SG_COL_MAJOR;
     const void* W = mat_a ? A : B;
@@ -827,11 +829,61 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     gp.beta = desc->beta;
     gp.a0 = desc->epi_arg0;
     gp.a1 = desc->epi_arg1;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const int64_t want = 2 * static_cast<int64_t>(d->sm_count);
+    if (es == 2 && !no_mma && desc->K % 8 == 0 && nvec >= 2) {
+        // two to eight vectors: warp-level MMAs, 16 rows per CTA, K ranges in units of 256 elements (one step of
+        // the CTA's eight warps), at least four steps per warp and rank
+        const int64_t blocks = (R + 15) / 16;
+        const int64_t ks_max = std::max<int64_t>(1, std::min<int64_t>(8, desc->K / 1024));
+        // K ranges only until there are two CTAs per SM: more (to even out the 16-row units over the SMs) measured
+        // slower (8192 x 8192: 30 -> 33 us)
+        static const int64_t per_sm = getenv("SG_GEMV_MMA_PER_SM") ? atoi(getenv("SG_GEMV_MMA_PER_SM")) : 2;    // experiments
+        const int64_t want_mma = per_sm * static_cast<int64_t>(d->sm_count);
+        int64_t ks = 1;
+        while (ks < 8 && ks * 2 <= ks_max && blocks * ks < want_mma) ks *= 2;
+        static const bool no_wide = getenv("SG_GEMV_NO_WIDE") != nullptr;      // experiments
+        const bool wide = !no_wide && desc->K % 16 == 0 && (ld * 2) % 32 == 0 && (x_stride * 2) % 32 == 0 &&
+                          reinterpret_cast<uintptr_t>(W) % 32 == 0 && reinterpret_cast<uintptr_t>(x) % 32 == 0;
+        const int64_t unit = wide ? 512 : 256;      // K elements per step of the CTA's eight warps
+        int64_t kchunk = (desc->K + ks - 1) / ks;
+        kchunk = (kchunk + unit - 1) / unit * unit;
+        ks = (desc->K + kchunk - 1) / kchunk;
+        gp.kchunk = static_cast<int32_t>(kchunk);
+        gp.ksplit = static_cast<int32_t>(ks);
+        const int64_t ctas = blocks * ks;
+        if (ctas > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many rows for the matrix-vector path");
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = cs;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = static_cast<unsigned>(ks);
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = desc->in_dtype == SG_F16
+                            ? (wide ? cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__half, true>, gp)
+                                    : cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__half, false>, gp))
+                            : (wide ? cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__nv_bfloat16, true>, gp)
+                                    : cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__nv_bfloat16, false>, gp));
+        if (e != cudaSuccess) return fail(SG_ERR_CUDA, "matrix-vector (MMA) kernel launch: %s", cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+        t_last_plan[0] = 0;
+        t_last_plan[1] = 0;
+        t_last_plan[2] = -static_cast<int32_t>(ks);
+        t_last_plan[3] = 16;
+        t_last_plan[4] = 0;
+        t_last_plan[5] = static_cast<int32_t>(ctas);
+        return SG_OK;
+    }
     // Geometry: at least two CTAs per SM where the problem has that much work; K ranges (CTAs of one cluster, at
     // most 8) when the rows alone do not give that many, each range at least two sweeps of the 256 threads.
     const int64_t sweep = 256 * (16 / es);
     const int64_t ks_max = std::max<int64_t>(1, std::min<int64_t>(8, desc->K / (2 * sweep)));
-    const int64_t want = 2 * static_cast<int64_t>(d->sm_count);
     static const int forced_rb = getenv("SG_GEMV_RB") ? atoi(getenv("SG_GEMV_RB")) : 0;    // experiments: 1, 2, 4
     int rb = (forced_rb == 1 || forced_rb == 2 || forced_rb == 4) ? forced_rb : 4;
     int64_t ks = 1;
@@ -847,7 +899,6 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     gp.ksplit = static_cast<int32_t>(ks);
     const int64_t ctas = (R + rb - 1) / rb * ks;
     if (ctas > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many rows for the matrix-vector path");
-    cudaStream_t cs = static_cast<cudaStream_t>(stream);
     cudaError_t e = desc->in_dtype == SG_F32   ? launch_gemv<float>(gp, rb, static_cast<int>(ctas), cs)
                     : desc->in_dtype == SG_F16 ? launch_gemv<__half>(gp, rb, static_cast<int>(ctas), cs)
                                                : launch_gemv<__nv_bfloat16>(gp, rb, static_cast<int>(ctas), cs);

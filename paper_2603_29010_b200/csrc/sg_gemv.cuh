@@ -212,4 +212,172 @@ __global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4 && NV == 1) ? 
     if (ks > 1) cg::this_cluster().sync();      // keep every rank's shared memory alive until rank 0 has read it
 }
 
+// Two to eight vectors of 16-bit inputs: the multiply-adds of the kernel above would saturate the FMA pipe (8 vectors =
+// 64 FMAs per 16 bytes of W), so the products go through warp-level tensor-core MMAs (m16n8k16, fp32 accumulation):
+// a warp owns 16 rows x 8 vectors, needs four accumulator registers per thread, and one MMA consumes what 16 rows x
+// 16 k took 256 FMAs-lanes.  tcgen05 has no shape for this (its tiles are 64 or 128 rows fed from shared memory);
+// the kernel stays a stream over W bound by HBM.
+// Fragment trick: the MMA sums over k, so any permutation of k applied to both operands gives the same result.  Thread
+// (g = lane / 4, t = lane % 4) loads 16 bytes = 8 consecutive k of rows g and g + 8 and of vector g, all at
+// k0 + 8 t, and feeds word pairs (0, 1) and (2, 3) of those loads to two MMAs: the MMA's "k = 2t, 2t+1" and
+// "k = 2t+8, 2t+9" slots then hold the same physical k on the A and on the B side.  The four lanes of a row read 64
+// contiguous bytes; the eight warps of a CTA interleave their steps, so a CTA reads 512 contiguous bytes per row.
+template <typename T> struct GemvMma;
+template <> struct GemvMma<__nv_bfloat16> {
+    static __device__ __forceinline__ void mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+};
+template <> struct GemvMma<__half> {
+    static __device__ __forceinline__ void mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+};
+
+// 256-bit global load (sm_100): 32 contiguous bytes per thread, so the four lanes of a row fetch a whole 128-byte line
+// with one instruction (with 16-byte loads a warp-wide load covers 16 row pieces of 64 bytes: twice the number of
+// memory transactions per byte).
+struct U8 {
+    uint32_t w[8];
+};
+__device__ __forceinline__ U8 ldg_stream32(const void* p) {
+    U8 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ U8 ldg_cached32(const void* p) {
+    U8 v;
+    asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])
+                 : "l"(p));
+    return v;
+}
+
+// kWide = false: 16-byte pieces; requires K % 8 == 0 and kchunk % 256 == 0.
+// kWide = true: 32-byte pieces; requires K % 16 == 0, kchunk % 512 == 0 and 32-byte aligned rows and vectors.
+// Grid: ceil(R / 16) row blocks x ksplit ranks.
+template <typename T, bool kWide>
+__global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
+    namespace cg = cooperative_groups;
+    constexpr int WARPS = 8;
+    constexpr int PE = kWide ? 16 : 8;        // elements per thread and step
+    constexpr int U = kWide ? 2 : 4;          // steps in flight per warp
+    constexpr int STEP = 4 * PE;              // elements of K a warp covers per step
+    __shared__ float warp_part[WARPS][128];   // 16 rows x 8 vectors per warp
+    __shared__ float cta_part[128];
+
+    const int ks = p.ksplit;
+    const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));
+    const int64_t r0 = static_cast<int64_t>(blockIdx.x / static_cast<unsigned>(ks)) * 16;
+    const int kbeg = rank * p.kchunk;
+    const int kend = min(p.K, kbeg + p.kchunk);
+    const int warp = static_cast<int>(threadIdx.x) >> 5, lane = static_cast<int>(threadIdx.x) & 31;
+    const int g = lane >> 2, t = lane & 3;
+
+    const T* wlo = reinterpret_cast<const T*>(p.W) + min(r0 + g, static_cast<int64_t>(p.R) - 1) * p.ld;
+    const T* whi = reinterpret_cast<const T*>(p.W) + min(r0 + g + 8, static_cast<int64_t>(p.R) - 1) * p.ld;
+    const T* xv = reinterpret_cast<const T*>(p.x) + static_cast<int64_t>(min(g, p.nvec - 1)) * p.x_stride;
+    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+
+    // The loop bounds are the same for all lanes of a warp (mma.sync must be executed by the whole warp).  Main loop:
+    // U steps whose pieces all lie inside the K range, loads without conditions; then single steps in which a lane
+    // whose piece lies past the end contributes zeros.
+    int kw = kbeg + warp * STEP;
+    for (; kw + (U - 1) * WARPS * STEP + STEP <= kend; kw += U * WARPS * STEP) {
+        const int k0 = kw + t * PE;
+        if constexpr (kWide) {
+            U8 lo[U], hi[U], xx[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                lo[u] = ldg_stream32(wlo + k0 + u * WARPS * STEP);
+                hi[u] = ldg_stream32(whi + k0 + u * WARPS * STEP);
+                xx[u] = ldg_cached32(xv + k0 + u * WARPS * STEP);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    GemvMma<T>::mma(c, lo[u].w[2 * j], hi[u].w[2 * j], lo[u].w[2 * j + 1], hi[u].w[2 * j + 1], xx[u].w[2 * j],
+                                    xx[u].w[2 * j + 1]);
+            }
+        } else {
+            uint4 lo[U], hi[U], xx[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                lo[u] = ldg_stream16(wlo + k0 + u * WARPS * STEP);
+                hi[u] = ldg_stream16(whi + k0 + u * WARPS * STEP);
+                xx[u] = __ldg(reinterpret_cast<const uint4*>(xv + k0 + u * WARPS * STEP));
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                GemvMma<T>::mma(c, lo[u].x, hi[u].x, lo[u].y, hi[u].y, xx[u].x, xx[u].y);
+                GemvMma<T>::mma(c, lo[u].z, hi[u].z, lo[u].w, hi[u].w, xx[u].z, xx[u].w);
+            }
+        }
+    }
+    for (; kw < kend; kw += WARPS * STEP) {
+        const int k = kw + t * PE;
+        const bool valid = k < kend;        // pieces are whole: K, kbeg and k are multiples of PE
+        if constexpr (kWide) {
+            U8 lo, hi, xx;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) lo.w[j] = hi.w[j] = xx.w[j] = 0u;
+            if (valid) {
+                lo = ldg_stream32(wlo + k);
+                hi = ldg_stream32(whi + k);
+                xx = ldg_cached32(xv + k);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                GemvMma<T>::mma(c, lo.w[2 * j], hi.w[2 * j], lo.w[2 * j + 1], hi.w[2 * j + 1], xx.w[2 * j], xx.w[2 * j + 1]);
+        } else {
+            uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo, xx = lo;
+            if (valid) {
+                lo = ldg_stream16(wlo + k);
+                hi = ldg_stream16(whi + k);
+                xx = __ldg(reinterpret_cast<const uint4*>(xv + k));
+            }
+            GemvMma<T>::mma(c, lo.x, hi.x, lo.y, hi.y, xx.x, xx.y);
+            GemvMma<T>::mma(c, lo.z, hi.z, lo.w, hi.w, xx.z, xx.w);
+        }
+    }
+    // accumulator fragment: c0 (row g, vector 2t), c1 (g, 2t+1), c2 (g+8, 2t), c3 (g+8, 2t+1)
+    warp_part[warp][g * 8 + 2 * t] = c[0];
+    warp_part[warp][g * 8 + 2 * t + 1] = c[1];
+    warp_part[warp][(g + 8) * 8 + 2 * t] = c[2];
+    warp_part[warp][(g + 8) * 8 + 2 * t + 1] = c[3];
+    __syncthreads();
+    if (threadIdx.x < 128) {
+        float s = 0.0f;
+#pragma unroll
+        for (int wi = 0; wi < WARPS; ++wi) s += warp_part[wi][threadIdx.x];
+        cta_part[threadIdx.x] = s;
+    }
+    if (ks > 1) cg::this_cluster().sync();
+    if (rank == 0 && threadIdx.x < 128) {
+        float s = cta_part[threadIdx.x];
+        if (ks > 1) {
+            cg::cluster_group cluster = cg::this_cluster();
+            for (int r = 1; r < ks; ++r) s += *cluster.map_shared_rank(&cta_part[threadIdx.x], r);
+        }
+        const int64_t row = r0 + static_cast<int>(threadIdx.x) / 8;
+        const int vec = static_cast<int>(threadIdx.x) % 8;
+        if (row < p.R && vec < p.nvec) {
+            float v[1] = {p.alpha * s};
+            if (p.beta != 0.0f) v[0] = fmaf(p.beta, gemv_load_out(p.C, row * p.c_row_stride + vec * p.c_vec_stride, p.out_kind), v[0]);
+            if (p.bias != nullptr)
+                v[0] += GemvVec<T>::exact(reinterpret_cast<const T*>(p.bias) + row * p.bias_row_stride + vec * p.bias_vec_stride);
+            if (p.epi >= EPI_RELU) apply_act_chunk<false, 1>(v, p.epi, p.a0, p.a1);
+            gemv_store_out(p.D, row * p.d_row_stride + vec * p.d_vec_stride, p.out_kind, v[0]);
+        }
+    }
+    if (ks > 1) cg::this_cluster().sync();
+}
+
 }  // namespace sg

@@ -74,10 +74,13 @@ def test_matrix_times_vector_real_values_with_epilogue(R, K, dtype, out_dtype, e
     parity.assert_matches(D, ref, absacc, f"vector-matrix {R}x{K} {dtype} {epi}")
 
 
-@pytest.mark.parametrize("nvec", [2, 3, 4])
-@pytest.mark.parametrize("R,K", [(4096, 4096), (130, 66000), (5, 1000)])
+@pytest.mark.parametrize("nvec", [2, 3, 4, 5, 8])
+@pytest.mark.parametrize("R,K", [(4096, 4096), (130, 66000), (5, 1000), (37, 264)])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16, torch.float32])
-def test_up_to_four_vectors_in_one_pass(R, K, nvec, dtype):
+def test_several_vectors_in_one_pass(R, K, nvec, dtype):
+    # 16-bit inputs: up to eight vectors (warp-level MMAs); fp32 inputs: up to four (FMA kernel)
+    if dtype == torch.float32 and nvec > 4:
+        pytest.skip("more than four fp32 vectors run on the tiles")
     g = torch.Generator().manual_seed(R + K + nvec)
     out_dtype = torch.float32 if dtype == torch.float32 else dtype
     W = (torch.randn(R, K, generator=g) / 8).to(dtype)
@@ -103,6 +106,18 @@ def test_up_to_four_vectors_in_one_pass(R, K, nvec, dtype):
     Di = torch.full((nvec, R), float("nan"), dtype=torch.float32, device=DEV)
     sg.gemm(Xi.to(DEV), Wi.to(DEV), out=Di)
     parity.assert_bit_exact(Di, ref, f"{nvec} integer vectors times {R}x{K} {dtype}")
+
+
+def test_several_vectors_with_a_ragged_k():
+    # K is no multiple of 8: the FMA kernel (up to four vectors), rows padded to 16 bytes
+    g = torch.Generator().manual_seed(21)
+    R, K, ld = 300, 1003, 1008
+    Wp = (torch.randn(R, ld, generator=g) / 4).to(torch.bfloat16)
+    Xp = (torch.randn(3, ld, generator=g) / 4).to(torch.bfloat16)
+    ref, absacc = orc.gemm(Xp[:, :K], Wp[:, :K], epi="relu")
+    D = sg.gemm(Xp.to(DEV)[:, :K], Wp.to(DEV)[:, :K], epi="relu")
+    assert _took_vector_path()
+    parity.assert_matches(D, ref, absacc, "three vectors, K = 1003")
 
 
 def test_padded_rows_strided_outputs_and_a_column_vector_operand():
@@ -133,12 +148,12 @@ def test_results_do_not_depend_on_the_run():
 def test_other_forms_still_go_through_the_tiles():
     g = torch.Generator().manual_seed(4)
     A = torch.randn(256, 64, generator=g).to(torch.bfloat16)
-    B5 = torch.randn(5, 64, generator=g).to(torch.bfloat16)
-    out = torch.empty(256, 8, dtype=torch.bfloat16, device=DEV)
-    sg.gemm(A.to(DEV), B5.to(DEV), out=out[:, :5])
+    B9 = torch.randn(9, 64, generator=g).to(torch.bfloat16)
+    out = torch.empty(256, 16, dtype=torch.bfloat16, device=DEV)
+    sg.gemm(A.to(DEV), B9.to(DEV), out=out[:, :9])
     assert not _took_vector_path()
-    ref, absacc = orc.gemm(A, B5)
-    parity.assert_matches(out[:, :5], ref, absacc, "N = 5")
+    ref, absacc = orc.gemm(A, B9)
+    parity.assert_matches(out[:, :9], ref, absacc, "N = 9")
     # a K x 2 row-major B is not a pair of contiguous vectors
     Brow = torch.randn(64, 8, generator=g).to(torch.bfloat16)
     sg.gemm(A.to(DEV), Brow.to(DEV)[:, :2], layout_b="row", out=out[:, :2])
@@ -147,10 +162,10 @@ def test_other_forms_still_go_through_the_tiles():
     parity.assert_matches(out[:, :2], ref, absacc, "N = 2, row-major B")
 
 
-@pytest.mark.parametrize("M", [5, 16, 32, 33, 64, 65])
+@pytest.mark.parametrize("M", [9, 16, 32, 33, 64, 65])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
 def test_few_rows_against_a_large_matrix_on_the_tiles(M, dtype):
-    # 5..64 rows: the tensor-core tiles with only 32 or 64 rows of A loaded per stage; 65: the full A tile
+    # 9..64 rows: the tensor-core tiles with only 32 or 64 rows of A loaded per stage; 65: the full A tile
     g = torch.Generator().manual_seed(100 + M)
     N, K = 1080, 2056
     A = (torch.randn(M, K, generator=g) / 8).to(dtype)
@@ -183,3 +198,23 @@ def test_few_rows_batched():
     for b in range(batch):
         ref, absacc = orc.gemm(A[b], W[b], bias=bias[b], epi="relu")
         parity.assert_matches(D[b], ref, absacc, f"few rows, batch {b}")
+
+
+@pytest.mark.parametrize("K", [8, 24, 200, 1000, 1016, 4104])
+@pytest.mark.parametrize("nvec", [3, 8])
+@pytest.mark.parametrize("R", [1, 17, 100])
+def test_several_vectors_k_not_a_multiple_of_a_warp_step(R, K, nvec):
+    # K % 32 != 0: the last step of a warp is partly past the end of the row (lanes there must contribute zeros
+    # while the whole warp still executes the tensor-core instruction)
+    W = inputs.small_integers([R, K], 93, 1, lo=-2, hi=2)
+    X = inputs.small_integers([nvec, K], 93, 2, lo=-2, hi=2)
+    ref, _ = orc.gemm(X, W)
+    D = torch.full((nvec, R), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(X.to(DEV), W.to(DEV), out=D)
+    assert _took_vector_path()
+    parity.assert_bit_exact(D, ref, f"{nvec} vectors times {R}x{K}")
+    ref, _ = orc.gemm(W, X)
+    D = torch.full((R, nvec), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(W.to(DEV), X.to(DEV), out=D)
+    assert _took_vector_path()
+    parity.assert_bit_exact(D, ref, f"{R}x{K} times {nvec} vectors")
