@@ -403,6 +403,14 @@ def bench_widened(sg, inputs, torch, dev, peaks) -> dict:
         timed(f"gemm_{M}x{N}x{K}", [lambda: sg.gemm(A, B, out=O)], dict(op="gemm", M=M, N=N, K=K), reps=10,
               note="one buffer set (operands may stay in L2)")
         del A, B, O
+    # the three-stage layout pipeline around the benchmark convolution: fp32 NCHW in, fp32 NCHW out
+    xs = [torch.randn(32, 256, 56, 56, device=dev) / 48 for _ in range(3)]
+    wf = inputs.make_conv(32, 56, 56, 256, 256, 3, 3, "normal", 1 / 48.0, bias=True, seed=3, device=dev)
+    timed("pipeline_nchw_fp32_conv3x3_nchw_fp32_32x256x56x56",
+          [(lambda i=i: sg.conv2d_fprop_nchw(xs[i], wf[1], pad=(1, 1), bias=wf[2], epi="relu")) for i in range(3)],
+          dict(op="conv2d", conv=dict(N=32, H=56, W=56, C=256, K=256, R=3, S=3, pad=(1, 1))),
+          note="three launches (transpose + convert, convolution, transpose + convert); the bound is the convolution's alone")
+    del xs, wf
     # matrix-vector products (N = 1): a stream over the matrix, several matrices in turn so that none stays in the L2
     for (R, K) in ((4096, 4096), (11008, 4096), (8192, 8192), (256, 131072), (16384, 16384)):
         nset = max(2, min(12, int(400e6 // (R * K * 2)) + 1))

@@ -447,6 +447,19 @@ def nhwc_to_nchw(x: torch.Tensor, out_dtype: Optional[torch.dtype] = None) -> to
     return transpose(x.reshape(n, h * w, c), out_dtype=out_dtype).view(n, c, h, w)
 
 
+def conv2d_fprop_nchw(x: torch.Tensor, Wf: torch.Tensor, *, compute_dtype: torch.dtype = torch.bfloat16,
+                      out_dtype: Optional[torch.dtype] = None, stream=None, **conv_kw) -> torch.Tensor:
+    """The DSL's three-stage pipeline (Appendix A.1) for a framework that keeps NCHW tensors:
+    ``pipeline(transpose(input, NCHW, NHWC, dtype, compute_dtype), conv2d_fprop(...), transpose(output, NHWC, NCHW,
+    compute_dtype, out_dtype))`` -- three launches on one stream, no host work in between.  ``x`` is [N, C, H, W]
+    (fp32 or bf16), ``Wf`` is [K, R, S, C] in the compute type; ``conv_kw`` goes to ``conv2d_fprop``."""
+    n, c, h, w = x.shape
+    x_nhwc = transpose(x.reshape(n, c, h * w), out_dtype=compute_dtype, stream=stream).view(n, h, w, c)
+    y = conv2d_fprop(x_nhwc, Wf, stream=stream, **conv_kw)
+    _, p, q, k = y.shape
+    return transpose(y.reshape(n, p * q, k), out_dtype=out_dtype or x.dtype, stream=stream).view(n, k, p, q)
+
+
 def conv1d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=0, stride=1, dil=1, **kw) -> torch.Tensor:
     """1-D convolution lowered to ``sg_conv2d_fprop`` with H = 1 (the paper's Table 1a note): X [N, L, C], Wf [K, S, C]."""
     n, l, c = X.shape

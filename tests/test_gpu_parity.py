@@ -502,6 +502,16 @@ def test_layout_pipeline_nchw_conv_nchw_and_conv1d():
     y_nchw = sg.nhwc_to_nchw(y, out_dtype=torch.float32)
     ref, _ = orc.conv2d_fprop(x_nchw.permute(0, 2, 3, 1).contiguous().to(torch.bfloat16), Wf, pad=(1, 1), epi="relu")
     parity.assert_bit_exact(y_nchw.permute(0, 2, 3, 1), ref, "NCHW -> conv -> NCHW")
+    # the same three stages through the pipeline driver, with a bias and on a side stream
+    bias = inputs.small_integers([K], 628, 8, -2, 2)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        y2 = sg.conv2d_fprop_nchw(x_nchw.to(DEV), Wf.to(DEV), pad=(1, 1), bias=bias.to(DEV), epi="relu", stream=side)
+    side.synchronize()
+    assert y2.dtype == torch.float32 and tuple(y2.shape) == (N, K, H, W)
+    ref2, _ = orc.conv2d_fprop(x_nchw.permute(0, 2, 3, 1).contiguous().to(torch.bfloat16), Wf, pad=(1, 1), bias=bias, epi="relu")
+    parity.assert_bit_exact(y2.permute(0, 2, 3, 1), ref2, "pipeline driver")
     # conv1d lowered to conv2d with H = 1
     X1 = inputs.small_integers([3, 50, 32], 636, 6, -1, 1)
     W1 = inputs.small_integers([40, 5, 32], 636, 7, -1, 1) * (inputs.small_integers([40, 5, 32], 637, 7, 0, 2) == 0).to(torch.bfloat16)
