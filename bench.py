@@ -462,9 +462,17 @@ def profile_config(args) -> None:
     torch.cuda.set_device(dev)
     C = inputs.CONFIGS
     name = {"c3": "c3_batched_128x256x256x512_gelu", "c4": "c4_conv_32x56x56x256_k256_3x3_bias_relu",
-            "c5": "c5_grouped_16xMx4096x4096_silu"}[args.profile_config]
-    c = C[name]
-    if args.profile_config == "c3":
+            "c5": "c5_grouped_16xMx4096x4096_silu", "gemv1": "matrix_vector_8192x8192_1_vector",
+            "gemv8": "matrix_vector_8192x8192_8_vectors"}[args.profile_config]
+    c = C.get(name)
+    if args.profile_config in ("gemv1", "gemv8"):
+        nvec = 1 if args.profile_config == "gemv1" else 8
+        sets = 3
+        Ws = [torch.randn(8192, 8192, device=dev).to(torch.bfloat16) for _ in range(sets)]
+        x = torch.randn(nvec, 8192, device=dev).to(torch.bfloat16)
+        outs = [torch.empty(8192, nvec, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        step = lambda i: sg.gemm(Ws[i % sets], x, out=outs[i % sets])
+    elif args.profile_config == "c3":
         sets = 4
         data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev, batch=c["batch"]) for i in range(sets)]
         outs = [torch.empty(c["batch"], c["M"], c["N"], dtype=torch.bfloat16, device=dev) for _ in range(sets)]
@@ -673,7 +681,7 @@ def main() -> None:
     ap.add_argument("--widened", action="store_true",
                     help="also time the rows built beyond the five configurations (epilogue chain, dtypes, layouts, "
                          "skinny shapes, transpose, conv gradients; N=1 only)")
-    ap.add_argument("--profile-config", choices=["c3", "c4", "c5"], default=None,
+    ap.add_argument("--profile-config", choices=["c3", "c4", "c5", "gemv1", "gemv8"], default=None,
                     help="only run a few launches of that configuration inside the profiler bracket (for ncu)")
     ap.add_argument("--torch-ref", action="store_true", help="with --all-configs: also time torch's library kernels")
     ap.add_argument("--kernel-only", action="store_true",
