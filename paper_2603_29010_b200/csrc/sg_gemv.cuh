@@ -1,12 +1,14 @@
-// Matrix-vector product with the fused epilogue: out[r] = act(alpha * sum_k W[r][k] x[k] + beta * C[r] + bias[r]),
-// for up to four vectors x at once.  The GEMM with N <= 4 (or M <= 4) of the paper's workload list (single-token
-// decode): every matrix element is used once per vector, so the kernel is a stream over W bound by HBM, and the
-// tensor cores (128-row tiles for at most four useful rows) have nothing to offer.
+// Matrix-vector products with the fused epilogue: out[r][v] = act(alpha * sum_k W[r][k] x_v[k] + beta * C + bias), for
+// up to eight vectors x_v at once.  The GEMM with N <= 8 (or M <= 8) of the paper's workload list (single-token
+// decode): every matrix element is used once per vector, so the kernels are a stream over W bound by HBM, and the
+// tcgen05 tiles (128 rows for at most eight useful ones, operands staged in shared memory) have nothing to offer.
+// Two kernels: gemv_kernel (CUDA-core FMAs: one vector; fp32 inputs or a ragged K: up to four) and gemv_mma_kernel
+// (warp-level MMAs: two to eight vectors of 16-bit inputs).
 //
-// Work split: a CTA of 256 threads takes RB consecutive rows and one K range; each thread walks the range in
-// 16-byte vectors (one vector of x serves RB vectors of W, so RB independent loads are in flight per thread and
-// iteration), sums in fp32, and the CTA reduces with shuffles and shared memory.  K ranges of one row block are the
-// CTAs of one thread-block cluster: rank 0 adds the other ranks' partial sums in rank order through distributed
+// Work split of gemv_kernel: a CTA of 256 threads takes RB consecutive rows and one K range; each thread walks the
+// range in 16-byte vectors (one vector of x serves RB vectors of W, so RB independent loads are in flight per thread
+// and iteration), sums in fp32, and the CTA reduces with shuffles and shared memory.  K ranges of one row block are
+// the CTAs of one thread-block cluster: rank 0 adds the other ranks' partial sums in rank order through distributed
 // shared memory (no global scratch, no atomics; the result depends only on the launch geometry).
 #pragma once
 #include <cooperative_groups.h>
@@ -26,7 +28,7 @@ struct GemvParams {
     int64_t x_stride;
     int64_t c_row_stride, c_vec_stride, d_row_stride, d_vec_stride;   // element (row r, vector v) of C and D
     int32_t R, K;
-    int32_t nvec;         // 1..4
+    int32_t nvec;         // 1..8 (gemv_kernel: 1..4)
     int32_t kchunk;       // K elements per cluster rank (a multiple of 256 vectors)
     int32_t ksplit;       // CTAs per cluster
     int32_t bias_row_stride, bias_vec_stride;   // (0, 1): one bias per vector (the matrix is A); (1, 0): one per row
