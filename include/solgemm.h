@@ -160,11 +160,14 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
  * device) is forbidden.  (The paper has no counterpart: its generated wrappers allocate their workspace.)
  *   The per-group tensor maps and the tile table go into a fixed scratch array that is part of the library
  *   image (about 36 KB of device memory on every GPU that loads the library, held until the process exits),
- *   so the call takes no workspace arguments and performs no device allocation of any kind.  Inputs and
+ *   so the call takes no workspace arguments and (after the first call on a device, see below) allocates nothing.  Inputs and
  *   outputs are still the caller's buffers; all other arguments and the result are those of sg_grouped_gemm.
  *   groups > SG_STATIC_MAX_GROUPS           -> SG_ERR_WORKSPACE, nothing is launched.
  *   The first call on a device looks up the array's device address (once per device, with that device
- *   current); make that first call outside any stream capture.
+ *   current).  That look-up, like the first use of any kernel of the library, makes the CUDA runtime load the
+ *   library's device code, which itself takes device memory and may synchronise: make the first call on each
+ *   device early -- before the GPU's memory is handed to the pool -- and outside any stream capture.  From the
+ *   second call on nothing is allocated or loaded.
  *   All calls on a device share the one array and it keeps the previous call's tables until they are
  *   overwritten: every call rewrites all entries it uses before its kernel reads them, but two calls whose
  *   work overlaps on the GPU (different streams, or the same stream from two threads) race on it.  Serialise
@@ -329,7 +332,10 @@ const char* sg_last_error(void);
  * sg_poll_status: reads (and clears) the device-side status word of the current device.  Call it
  * after synchronising the stream(s) the work was enqueued on; `cuda_stream` is used for the read.
  * SG_OK, or SG_ERR_TIMEOUT with the role / tile / barrier that gave up in sg_last_error().  While
- * the word is set, later kernels of this library return at once without computing.
+ * the word is set, later launches of the tensor-core contraction kernel (every entry point above except the
+ * matrix-vector form of sg_gemm and sg_transpose, whose kernels contain no waits and do not read the word) return
+ * at once without computing and leave their outputs untouched; the poll that reports the word also clears it and
+ * the K-range counters of a lent scratch, after which calls compute again.
  */
 sg_status_t sg_poll_status(void* cuda_stream);
 
@@ -344,7 +350,7 @@ sg_status_t sg_set_tuning(int32_t tile_n, int32_t cta_pair);
  * sg_last_kernel_clock: the SM clock (MHz) at which the most recent contraction kernel on the current device
  * actually ran, measured inside the kernel (cycle counter over nanosecond timer of its first CTA).  Under a
  * board power cap this is what the paper's clock-aware Speed-of-Light rule should scale the peak by (Section 4.1,
- * "hardware limits ... scaled by the current clock"); management libraries may report the requested clock instead.
+ * hardware-limits step); management libraries may report the requested clock instead.
  * Synchronises `cuda_stream`.  0 if no kernel has run yet.
  */
 sg_status_t sg_last_kernel_clock(double* sm_mhz, void* cuda_stream);
@@ -372,6 +378,37 @@ sg_status_t sg_set_tail_mode(int32_t mode);
  */
 #define SG_SCRATCH_BYTES_RECOMMENDED (32u << 20)
 sg_status_t sg_set_scratch(void* scratch_dev, size_t bytes);
+
+/*
+ * sg_set_option: planner and launch overrides for measurements and tests (never needed for correct use; they apply to
+ * later calls from any thread).  value -1 restores the default.  (The paper's DSL exposes such choices as explicit
+ * clauses -- .with_tile, .with_stages, .with_scheduler, splits=, Table 1b; here a host heuristic takes them and these
+ * knobs pin it.)
+ */
+typedef enum {
+    SG_OPT_EPI_WARPS = 0,       /* 4 or 8 epilogue warps per CTA (default: 8 when K <= 1024) */
+    SG_OPT_TAIL_SPLIT = 1,      /* 1, 2 or 4: column slices per tile of the last partial wave */
+    SG_OPT_TAIL_KSPLIT = 2,     /* 0: never cut a K loop into ranges; k >= 2: k ranges where ranges are possible */
+    SG_OPT_BAND_M = 3,          /* tile rows per raster band */
+    SG_OPT_GENERAL_KERNEL = 4,  /* 1: always run the all-options kernel variant instead of the specialised ones */
+    SG_OPT_NO_PDL = 5,          /* 1: launch without programmatic dependent launch */
+    SG_OPT_NO_SHORT_A = 6,      /* 1: no short-A tiles for M <= 64 */
+    SG_OPT_NO_GEMV = 7,         /* 1: matrix-vector shaped calls go through the tensor-core tiles */
+    SG_OPT_GEMV_NO_MMA = 8,     /* 1: several vectors on the FMA matrix-vector kernel (<= 4 vectors) */
+    SG_OPT_GEMV_NO_WIDE = 9,    /* 1: 16-byte loads only in the multi-vector kernel */
+    SG_OPT_GEMV_ROWS = 10,      /* 1, 2 or 4 matrix rows per CTA in the single-vector kernel */
+    SG_OPT_WAIT_LIMIT_NS = 11,  /* bound of every device-side wait in nanoseconds (default 2 s); tests shorten it to
+                                   see the kernel give up, record where, and return */
+    SG_OPT_COUNT_ = 12
+} sg_option_t;
+sg_status_t sg_set_option(int32_t option, int64_t value);
+
+/*
+ * sg_test_set_status_word: TEST HOOK.  Writes `value` into the device-side status word of the current device (what a
+ * kernel whose wait ran out would do) and synchronises `cuda_stream`, so that the containment path -- later launches
+ * are no-ops, sg_poll_status reports and clears -- can be exercised without any kernel waiting on anything.
+ */
+sg_status_t sg_test_set_status_word(uint32_t value, void* cuda_stream);
 
 /* Number of kernel launches this library has enqueued from this process (monotonic). */
 int64_t sg_launch_count(void);

@@ -72,6 +72,12 @@ EncodeTiledFn g_encode_tiled = nullptr;
 EncodeIm2colFn g_encode_im2col = nullptr;
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_tune_tile_n{-1}, g_tune_pair{-1}, g_tune_tail{-1};
+// sg_set_option: planner overrides for measurements and tests (-1 = the planner decides / the default)
+std::atomic<int64_t> g_opt[SG_OPT_COUNT_];
+struct OptInit {
+    OptInit() { for (auto& o : g_opt) o.store(-1); }
+} g_opt_init;
+inline int64_t opt(int which) { return g_opt[which].load(std::memory_order_relaxed); }
 thread_local int32_t t_last_plan[6] = {0, 0, 0, 0, 0, 0};   // tile_n, cta_pair, tail split, tile-list length, first split position, grid
 
 KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 0) {
@@ -287,9 +293,8 @@ inline double ksplit_exchange_us(int64_t ks) { return ks > 1 ? 6.0 + 0.5 * stati
 constexpr double kUsPerKBlock = 0.25;      // one 64-deep k-block of a 128 x 256 tile per SM
 
 bool ksplit_allowed(const DeviceState& d) {
-    static const int env_k = getenv("SG_TAIL_KSPLIT") ? atoi(getenv("SG_TAIL_KSPLIT")) : -1;
     const int tail_mode = g_tune_tail.load();
-    return d.scratch != nullptr && tail_mode != 0 && tail_mode != 1 && env_k != 0;
+    return d.scratch != nullptr && tail_mode != 0 && tail_mode != 1 && opt(SG_OPT_TAIL_KSPLIT) != 0;
 }
 
 // What choose_shape needs to know for problems bound by memory traffic rather than by the tensor pipe: operand and
@@ -330,8 +335,8 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
     const bool pair_possible = pair_only || (K >= 1024 && d.max_pairs > 0 && can_split && max_rows > 128);
     // Eight epilogue warps drain an accumulator twice as fast; that pays when the K loop is too short to hide
     // the epilogue (short K, heavy activations) and costs a little when it is long.
-    static const int forced_ew = getenv("SG_EPI_WARPS") ? atoi(getenv("SG_EPI_WARPS")) : 0;   // experiments: 4 or 8
-    const int epi_warps = (forced_ew == 4 || forced_ew == 8) ? forced_ew : (K <= 1024 ? 8 : 4);
+    const int64_t forced_ew = opt(SG_OPT_EPI_WARPS);
+    const int epi_warps = (forced_ew == 4 || forced_ew == 8) ? static_cast<int>(forced_ew) : (K <= 1024 ? 8 : 4);
     Shape best{256, false, epi_warps};
     double best_cost = 1e300;
     for (int pi = 0; pi < 2; ++pi) {
@@ -412,8 +417,8 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
     int best_split = 1, best_ksplit = 1;
     const int64_t rem = full_tiles % slots;
-    static const int forced = getenv("SG_TAIL_SPLIT") ? atoi(getenv("SG_TAIL_SPLIT")) : 0;   // experiments: 1, 2 or 4
-    static const int env_k = getenv("SG_TAIL_KSPLIT") ? atoi(getenv("SG_TAIL_KSPLIT")) : -1;   // experiments: 0 = off
+    const int forced = static_cast<int>(opt(SG_OPT_TAIL_SPLIT));      // 1, 2 or 4
+    const int env_k = static_cast<int>(opt(SG_OPT_TAIL_KSPLIT));      // 0 = off, >= 2: that many K ranges
     const int tail_mode = g_tune_tail.load();      // -1 auto, 0 none, 1 column slices, 2 K ranges
     const int forced_k = tail_mode == 2 ? 4 : (tail_mode == 0 || tail_mode == 1 ? 0 : env_k);
     if (rem != 0 && tail_mode != 0) {
@@ -467,7 +472,7 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
     // raster bands: keep a band's A panels (band_m x TILE_M rows x K) within about 32 MB of L2
     const int64_t panel_bytes = static_cast<int64_t>(s.pair ? 256 : 128) * (p->K > 0 ? p->K : 1) * 2;
     int64_t band = (32ll << 20) / panel_bytes;
-    static const int forced_band = getenv("SG_BAND_M") ? atoi(getenv("SG_BAND_M")) : 0;   // experiments
+    const int64_t forced_band = opt(SG_OPT_BAND_M);
     if (forced_band > 0) band = forced_band;
     p->band_m = static_cast<int32_t>(band < 1 ? 1 : (band > 4096 ? 4096 : band));
     const int parts = best_ksplit > 1 ? best_ksplit : best_split;
@@ -506,7 +511,7 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     p.div_q = make_fastdiv(p.Q);
     // plain dense, convolution-forward and grouped problems run the variant of the kernel specialised for them
     // (same instructions, the other modes and options compiled out)
-    static const bool no_lean = getenv("SG_NO_LEAN") && atoi(getenv("SG_NO_LEAN")) != 0;      // experiments
+    const bool no_lean = opt(SG_OPT_GENERAL_KERNEL) > 0;
     int variant = 0;
     if (!no_lean && !p.in_fp8) {
         const bool plain = !p.a_mn_major && !p.b_mn_major && p.ksplit <= 1 && !p.d_remap && p.nphases <= 1;
@@ -531,7 +536,7 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     attr[0].val.clusterDim.z = 1;
     // programmatic dependent launch: this kernel's set-up may overlap the previous kernel's tail (the kernel
     // itself waits for that kernel before it touches global memory)
-    static const bool pdl = !(getenv("SG_NO_PDL") && atoi(getenv("SG_NO_PDL")) != 0);
+    const bool pdl = !(opt(SG_OPT_NO_PDL) > 0);
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
@@ -557,7 +562,8 @@ void base_params(Params* p, const DeviceState& d, float alpha, float beta, int32
     p->epi_arg0 = a0;
     p->epi_arg1 = a1;
     p->status = d.status_dev;
-    p->timeout_ns = kWaitLimitNs;
+    const int64_t limit = opt(SG_OPT_WAIT_LIMIT_NS);
+    p->timeout_ns = limit > 0 ? static_cast<uint64_t>(limit) : kWaitLimitNs;
 }
 
 // Validates the optional extended epilogue chain and copies it into the kernel parameters.
@@ -644,7 +650,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (st != SG_OK) return st;
     // a few rows against a large matrix: load only 32 or 64 rows of A per stage (kernel variants 6 and 7), which
     // leaves room for more stages of B
-    static const bool no_short_a = getenv("SG_NO_SHORT_A") != nullptr;      // experiments
+    const bool no_short_a = opt(SG_OPT_NO_SHORT_A) > 0;
     p.a_rows = 128;
     if (!no_short_a && !s.pair && !p.in_fp8 && !p.a_mn_major && !p.b_mn_major && p.ksplit <= 1 && !p.ex_any && desc->M <= 64)
         p.a_rows = desc->M <= 32 ? 32 : 64;
@@ -764,12 +770,11 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
                      void* stream, bool* taken) {
     *taken = false;
     if (!desc || desc->K < 1 || desc->K > INT32_MAX || desc->M < 1 || desc->N < 1) return SG_OK;
-    static const bool off = getenv("SG_NO_GEMV") != nullptr;     // tests: the same product through the tiles
-    if (off) return SG_OK;
+    if (opt(SG_OPT_NO_GEMV) > 0) return SG_OK;      // tests: the same product through the tiles
     // up to eight vectors of 16-bit inputs (four of fp32); the matrix is the operand with more rows
     if (desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F16 && desc->in_dtype != SG_F32) return SG_OK;
     const int es = desc->in_dtype == SG_F32 ? 4 : 2;
-    static const bool no_mma = getenv("SG_GEMV_NO_MMA") != nullptr;      // experiments: FMA kernel only (<= 4 vectors)
+    const bool no_mma = opt(SG_OPT_GEMV_NO_MMA) > 0;      // FMA kernel only (<= 4 vectors)
     const int64_t max_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? 8 : 4;
     const bool mat_a = desc->N <= max_vec && desc->M >= desc->N;
     if (!mat_a && desc->M > max_vec) return SG_OK;
@@ -838,11 +843,10 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         const int64_t ks_max = std::max<int64_t>(1, std::min<int64_t>(8, desc->K / 1024));
         // K ranges only until there are two CTAs per SM: more (to even out the 16-row units over the SMs) measured
         // slower (8192 x 8192: 30 -> 33 us)
-        static const int64_t per_sm = getenv("SG_GEMV_MMA_PER_SM") ? atoi(getenv("SG_GEMV_MMA_PER_SM")) : 2;    // experiments
-        const int64_t want_mma = per_sm * static_cast<int64_t>(d->sm_count);
+        const int64_t want_mma = 2 * static_cast<int64_t>(d->sm_count);
         int64_t ks = 1;
         while (ks < 8 && ks * 2 <= ks_max && blocks * ks < want_mma) ks *= 2;
-        static const bool no_wide = getenv("SG_GEMV_NO_WIDE") != nullptr;      // experiments
+        const bool no_wide = opt(SG_OPT_GEMV_NO_WIDE) > 0;
         const bool wide = !no_wide && desc->K % 16 == 0 && (ld * 2) % 32 == 0 && (x_stride * 2) % 32 == 0 &&
                           reinterpret_cast<uintptr_t>(W) % 32 == 0 && reinterpret_cast<uintptr_t>(x) % 32 == 0;
         const int64_t unit = wide ? 512 : 256;      // K elements per step of the CTA's eight warps
@@ -884,8 +888,8 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     // most 8) when the rows alone do not give that many, each range at least two sweeps of the 256 threads.
     const int64_t sweep = 256 * (16 / es);
     const int64_t ks_max = std::max<int64_t>(1, std::min<int64_t>(8, desc->K / (2 * sweep)));
-    static const int forced_rb = getenv("SG_GEMV_RB") ? atoi(getenv("SG_GEMV_RB")) : 0;    // experiments: 1, 2, 4
-    int rb = (forced_rb == 1 || forced_rb == 2 || forced_rb == 4) ? forced_rb : 4;
+    const int64_t forced_rb = opt(SG_OPT_GEMV_ROWS);    // 1, 2, 4
+    int rb = (forced_rb == 1 || forced_rb == 2 || forced_rb == 4) ? static_cast<int>(forced_rb) : 4;
     int64_t ks = 1;
     for (;; rb >>= 1) {
         const int64_t blocks = (R + rb - 1) / rb;
@@ -938,7 +942,26 @@ const char* sg_last_error(void) { return t_err; }
 
 int64_t sg_launch_count(void) { return g_launches.load(); }
 
+sg_status_t sg_set_option(int32_t option, int64_t value) {
+    if (option < 0 || option >= SG_OPT_COUNT_) return fail(SG_ERR_INVALID_ARG, "sg_set_option: option %d is not a sg_option_t", option);
+    if (value < -1) return fail(SG_ERR_INVALID_ARG, "sg_set_option: value must be >= -1");
+    g_opt[option].store(value);
+    return SG_OK;
+}
+
+sg_status_t sg_test_set_status_word(uint32_t value, void* cuda_stream) {
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    SG_CUDA(cudaMemcpyAsync(d->status_dev, &value, sizeof value, cudaMemcpyHostToDevice, stream));
+    SG_CUDA(cudaStreamSynchronize(stream));
+    return SG_OK;
+}
+
 #ifdef SG_DEBUG_STAMPS
+// Diagnostic builds only (-DSG_DEBUG_STAMPS=<n>, never the product library, hence not in solgemm.h): copies out the 32
+// time-stamp words that CTA n - 1 of the last launch recorded.
 sg_status_t sg_debug_stamps(uint64_t* out32) {
     DeviceState* d = nullptr;
     sg_status_t st = device_state(&d);

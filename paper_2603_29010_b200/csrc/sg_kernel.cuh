@@ -139,8 +139,10 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t b, bool f16) {
     return f16 ? __half2float(__ushort_as_half(b)) : __uint_as_float(static_cast<uint32_t>(b) << 16);
 }
 
-// Experiments only (-DSG_DEBUG_STAMPS): CTA `SG_DEBUG_STAMPS - 1` records globaltimer values at a few points of
-// its life into the words after the status words.
+// Diagnostic build (-DSG_DEBUG_STAMPS=<n>, off in the product library): CTA n - 1 records %globaltimer values at a
+// few points of its life (entry, set-up done, first load issued, first MMA, accumulator ready, last store, exit) into
+// the words after the status words; sg_debug_stamps() reads them back.  This is how the per-role time lines of a
+// launch's start and end were measured.
 #ifdef SG_DEBUG_STAMPS
 #define SG_STAMP(slot)                                                                           \
     do {                                                                                         \
@@ -1214,9 +1216,6 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     continue;
                 }
 
-#if defined(SG_DEBUG_SKIP) && (SG_DEBUG_SKIP & 4)
-                if (v[0] != 12345.678f) continue;
-#endif
                 // stage the 32 x 128-byte block (row = lane) in the swizzled layout the store map expects
                 const uint32_t sb = chunk_ctr % Cfg::STAGING_BUFS;
                 ++chunk_ctr;
@@ -1241,12 +1240,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
-#if !(defined(SG_DEBUG_SKIP) && (SG_DEBUG_SKIP & 1))
                 if (lane == 0) {
                     tma_store_3d(mapD, stg, n0 + c * CH, row0, bz);
                     tma_store_commit();
                 }
-#endif
             }
             if (!ok) break;
             }   // passes

@@ -39,7 +39,9 @@ EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_
             "sg_conv2d_dgrad", "sg_conv2d_wgrad",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
-            "sg_last_kernel_clock", "sg_transpose"]
+            "sg_last_kernel_clock", "sg_transpose", "sg_set_option", "sg_test_set_status_word"]
+OPTIONS = {"epi_warps": 0, "tail_split": 1, "tail_ksplit": 2, "band_m": 3, "general_kernel": 4, "no_pdl": 5, "no_short_a": 6,
+           "no_gemv": 7, "gemv_no_mma": 8, "gemv_no_wide": 9, "gemv_rows": 10, "wait_limit_ns": 11}
 
 
 class SolgemmError(RuntimeError):
@@ -133,6 +135,10 @@ _lib.sg_set_scratch.restype = ctypes.c_int
 _lib.sg_set_scratch.argtypes = [_vp, ctypes.c_size_t]
 _lib.sg_last_launch_plan.restype = ctypes.c_int
 _lib.sg_last_launch_plan.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+_lib.sg_set_option.restype = ctypes.c_int
+_lib.sg_set_option.argtypes = [_i32, _i64]
+_lib.sg_test_set_status_word.restype = ctypes.c_int
+_lib.sg_test_set_status_word.argtypes = [ctypes.c_uint32, _vp]
 
 
 SCRATCH_BYTES = 32 << 20
@@ -568,6 +574,19 @@ def last_kernel_clock_mhz(stream=None) -> float:
 def set_tail_mode(mode: int = -1) -> None:
     """-1 planner's choice, 0 whole tail tiles, 1 column slices, 2 K ranges through the scratch."""
     _check(_lib.sg_set_tail_mode(mode))
+
+
+def set_option(name: str, value: int = -1) -> None:
+    """``sg_set_option``: pin one of the planner's choices (see ``OPTIONS``); -1 restores the default."""
+    _check(_lib.sg_set_option(OPTIONS[name], int(value)))
+
+
+def test_set_status_word(value: int, stream=None) -> None:
+    """``sg_test_set_status_word`` (test hook): write the device status word as an expired wait would."""
+    _check(_lib.sg_test_set_status_word(int(value), _stream(stream)))
+
+
+test_set_status_word.__test__ = False      # not a pytest test, whatever module imports it
 
 
 def launch_count() -> int:

@@ -1,10 +1,10 @@
-"""GPU parity on the five benchmark configurations at their full sizes.
+"""GPU parity on the five benchmark configurations at their full sizes, in the launch configuration bench.py times.
 
-Small configurations are compared on every element.  For the large ones the
-oracle computes every row next to a tile edge of the first / last tiles plus
-seeded random points spread over the whole output (never a prefix), and the
-whole output is additionally checked for finiteness and against a tighter
-self-imposed bound on the sampled points.
+c1, c2, c3 and c4 are compared with the oracle on EVERY output element (the oracle runs once per configuration and
+serves both output types).  c5 (about 1.1e12 MACs) is compared on every row within one row of a group edge or of a
+128-row tile edge, plus a seeded 2 % sample of each group's rows spread over the whole group -- never a prefix.
+On top of the stated tolerance every compared element must meet a tighter self-imposed bound (one rounding of the
+result in the output type plus fp32 accumulation noise), because config 2's products are small against its bias.
 """
 import pytest
 import torch
@@ -38,13 +38,29 @@ def sample_points(rows, cols, count, seed):
     return pi, pj
 
 
+def assert_tight(got, ref, absacc, what):
+    """Tighter than the stated tolerance: one rounding of the result in the output type (2^-8 relative for bf16; the fp32
+    path is already judged on that scale) plus fp32 accumulation noise on the scale of the terms summed."""
+    parity.assert_matches(got, ref, absacc, what)
+    err = (got.detach().cpu().double().reshape(ref.shape) - ref).abs()
+    tight = 2.0 ** -8 * ref.abs() + 1e-4 * absacc + 1e-30
+    bad = err > tight
+    assert not bool(bad.any()), f"{what}: {int(bad.sum())} of {bad.numel()} elements outside the tight bound"
+
+
 def check_points(D, ref, absacc, pi, pj, what):
     got = D[torch.as_tensor(pi, device=D.device), torch.as_tensor(pj, device=D.device)]
-    parity.assert_matches(got, ref, absacc, what)
-    # tighter than the stated tolerance: one bf16 rounding of the result plus fp32 accumulation noise
-    err = (got.cpu().double() - ref).abs()
-    tight = 2.0 ** -8 * ref.abs() + 1e-4 * absacc + 1e-30
-    assert bool((err <= tight).all()), f"{what}: sampled points outside the tight bound"
+    assert_tight(got, ref, absacc, what)
+
+
+_REFS = {}
+
+
+def reference(name, fn):
+    """One oracle run per configuration and test session (the reference does not depend on the output type)."""
+    if name not in _REFS:
+        _REFS[name] = fn()
+    return _REFS[name]
 
 
 def test_c1_gemm_256_every_element():
@@ -60,14 +76,11 @@ def test_c2_gemm_4096_bias_relu(out_dtype):
     c = CFG["c2_gemm_4096_bias_relu"]
     A, B, bias = inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], bias=True, device=DEV)
     D = sg.gemm(A, B, bias=bias, epi=c["epi"], out_dtype=out_dtype)
+    plan = sg.last_launch_plan()
+    assert plan["tile_n"] == 256 and plan["cta_pair"] == 1          # the configuration bench.py times
     assert bool(torch.isfinite(D).all()) and bool((D >= 0).all())
-    hA, hB, hb = A.cpu(), B.cpu(), bias.cpu()
-    for r0 in (0, 120, 2040, 4088):                      # rows on both sides of tile edges, first and last tiles
-        ref, absacc = orc.gemm(hA, hB, bias=hb, epi=c["epi"], rows=(r0, r0 + 8))
-        parity.assert_matches(D[r0:r0 + 8], ref, absacc, f"c2 rows {r0}")
-    pi, pj = sample_points(c["M"], c["N"], 4096, 7)
-    ref, absacc = orc.gemm_points(hA, hB, pi, pj, bias=hb, epi=c["epi"])
-    check_points(D, ref, absacc, pi, pj, "c2 sampled")
+    ref, absacc = reference("c2", lambda: orc.gemm(A.cpu(), B.cpu(), bias=bias.cpu(), epi=c["epi"]))
+    assert_tight(D, ref, absacc, f"c2 every element, {out_dtype}")
 
 
 def test_c3_batched_gelu_every_element():
@@ -80,22 +93,15 @@ def test_c3_batched_gelu_every_element():
     parity.assert_matches(D32, ref, absacc, "c3 fp32 out")
 
 
-def test_c4_conv_bias_relu():
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_c4_conv_bias_relu(out_dtype):
     c = CFG["c4_conv_32x56x56x256_k256_3x3_bias_relu"]
     X, Wf, bias = inputs.make_conv(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], c["dist"], c["scale"],
                                    bias=True, device=DEV)
-    Y = sg.conv2d_fprop(X, Wf, pad=c["pad"], bias=bias, epi=c["epi"])
+    Y = sg.conv2d_fprop(X, Wf, pad=c["pad"], bias=bias, epi=c["epi"], out_dtype=out_dtype)
     assert bool(torch.isfinite(Y).all()) and bool((Y >= 0).all())
-    hX, hW, hb = X.cpu(), Wf.cpu(), bias.cpu()
-    PQ = 56 * 56
-    Yf = Y.view(-1, c["K"])
-    # image corners and borders, a tile edge (pixel 128), an image boundary, the very last pixels
-    for p0 in (0, 50, 120, PQ - 8, PQ + 48, 17 * PQ + 1000, 32 * PQ - 16):
-        ref, absacc = orc.conv2d_fprop(hX, hW, pad=c["pad"], bias=hb, epi=c["epi"], pixels=(p0, p0 + 16))
-        parity.assert_matches(Yf[p0:p0 + 16], ref, absacc, f"c4 pixels {p0}")
-    ppix, pk = sample_points(32 * PQ, c["K"], 2048, 9)
-    ref, absacc = orc.conv2d_points(hX, hW, ppix, pk, pad=c["pad"], bias=hb, epi=c["epi"])
-    check_points(Yf, ref, absacc, ppix, pk, "c4 sampled")
+    ref, absacc = reference("c4", lambda: orc.conv2d_fprop(X.cpu(), Wf.cpu(), pad=c["pad"], bias=bias.cpu(), epi=c["epi"]))
+    assert_tight(Y.view(-1, c["K"]), ref.reshape(-1, c["K"]), absacc.reshape(-1, c["K"]), f"c4 every element, {out_dtype}")
 
 
 def test_c5_grouped_silu():
@@ -104,16 +110,19 @@ def test_c5_grouped_silu():
     assert all(c["M_lo"] <= m <= c["M_hi"] for m in Ms)
     As, Bs = inputs.make_grouped(Ms, c["N"], c["K"], c["dist"], c["scale"], device=DEV)
     outs = sg.grouped_gemm(As, Bs, epi=c["epi"])
+    compared = 0
     for g, m in enumerate(Ms):
         assert outs[g].shape == (m, c["N"]) and bool(torch.isfinite(outs[g]).all())
-        hA, hB = As[g].cpu(), Bs[g].cpu()
-        last = max(m - 4, 0)
-        for r0, r1 in ((0, 2), (last, m)):               # first rows and the ragged last rows of every group
-            ref, absacc = orc.gemm(hA, hB, epi=c["epi"], rows=(r0, r1))
-            parity.assert_matches(outs[g][r0:r1], ref, absacc, f"c5 group {g} rows {r0}:{r1}")
-        pi, pj = sample_points(m, c["N"], 256, 100 + g)
-        ref, absacc = orc.gemm_points(hA, hB, pi, pj, epi=c["epi"])
-        check_points(outs[g], ref, absacc, pi, pj, f"c5 group {g} sampled")
+        # every row within one row of the group's edges and of every 128-row tile edge ...
+        rows = {r for r in range(m) if r % 128 in (0, 1, 127)} | {0, 1, m - 2, m - 1}
+        # ... plus a seeded 2 % of the group's rows, spread over the whole group
+        rows |= set(inputs.integers(max(1, (m + 49) // 50), 300 + g, 13, 0, m - 1))
+        idx = torch.tensor(sorted(r for r in rows if 0 <= r < m))
+        compared += len(idx)
+        # the oracle's product of the selected rows of A_g with B_g (each output row depends on its own row of A only)
+        ref, absacc = orc.gemm(As[g].cpu()[idx].contiguous(), Bs[g].cpu(), epi=c["epi"])
+        assert_tight(outs[g][idx.to(DEV)], ref, absacc, f"c5 group {g}: {len(idx)} rows at tile and group edges + sample")
+    assert compared >= sum(Ms) // 25
 
 
 def test_c4_sized_conv_gradients():

@@ -36,10 +36,18 @@ def _compare(Ms, N, K, seed, epi):
     As, Bs, biases = _problem(Ms, N, K, seed)
     want = sg.grouped_gemm(As, Bs, biases=biases, epi=epi)                  # caller-provided workspace
     outs = [torch.full((m, N), float("nan"), dtype=torch.bfloat16, device=DEV) for m in Ms]
-    before = torch.cuda.memory_allocated()
-    got = sg.grouped_gemm_static(As, Bs, biases=biases, outs=outs, epi=epi)  # tables in the library's own array
-    assert torch.cuda.memory_allocated() == before                         # the wrapper allocated nothing either
+    # The first call on a device makes the CUDA runtime load the library's device code (documented: do it early);
+    # from then on nothing may be taken from the device, neither through torch's allocator nor behind its back.
+    sg.grouped_gemm_static(As, Bs, biases=biases, outs=outs, epi=epi)
     torch.cuda.synchronize()
+    for o in outs:
+        o.fill_(float("nan"))
+    torch.cuda.synchronize()
+    before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+    got = sg.grouped_gemm_static(As, Bs, biases=biases, outs=outs, epi=epi)  # tables in the library's own array
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before                         # the wrapper allocated nothing either
+    assert torch.cuda.mem_get_info()[0] >= free_before                     # and no cudaMalloc happened underneath it
     sg.poll_status()
     for g, m in enumerate(Ms):
         w, o = want[g].float(), got[g].float()
