@@ -414,6 +414,15 @@ sg_status_t sg_test_set_status_word(uint32_t value, void* cuda_stream);
 int64_t sg_launch_count(void);
 
 /*
+ * sg_last_kernel_name: the device function the calling thread's most recent compute launch ran, as the library's
+ * own record (e.g. "sg::contract_kernel<256, true, 0, 4, 1>": tile width, two-CTA tiles, output type, epilogue
+ * warps, variant).  Benchmarks list it next to their timings so that a reader can see that no vendor-library kernel
+ * stands behind a number -- the check the paper's integrity pipeline makes on profiler kernel names (Section 4.4,
+ * PyTorch-only detector).  Thread-local text, valid until the thread's next launch; "" before the first.
+ */
+const char* sg_last_kernel_name(void);
+
+/*
  * How the calling thread's most recent contraction launch was tiled, for tests and benchmark records:
  *   plan6[0] tile width in columns, [1] 1 for two-CTA tiles, [2] tail split (the tiles of the last,
  *   partial wave are cut into this many column slices; 1 = none; a negative value -k means they are

@@ -78,6 +78,13 @@ struct OptInit {
     OptInit() { for (auto& o : g_opt) o.store(-1); }
 } g_opt_init;
 inline int64_t opt(int which) { return g_opt[which].load(std::memory_order_relaxed); }
+thread_local char t_last_kernel[128] = "";      // the kernel function this thread launched last (sg_last_kernel_name)
+void note_kernel(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_last_kernel, sizeof t_last_kernel, fmt, ap);
+    va_end(ap);
+}
 thread_local int32_t t_last_plan[6] = {0, 0, 0, 0, 0, 0};   // tile_n, cta_pair, tail split, tile-list length, first split position, grid
 
 KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 0) {
@@ -543,6 +550,7 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     cfg.numAttrs = pdl ? 2 : 1;
     SG_CUDA(cudaLaunchKernelEx(&cfg, k.fn, p));
     g_launches.fetch_add(1);
+    note_kernel("sg::contract_kernel<%d, %s, %d, %d, %d>", s.bn, s.pair ? "true" : "false", out_kind, s.epi_warps, variant);
     t_last_plan[0] = s.bn;
     t_last_plan[1] = s.pair ? 1 : 0;
     t_last_plan[2] = p.ksplit > 1 ? -p.ksplit : p.split;
@@ -876,6 +884,7 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
                                     : cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__nv_bfloat16, false>, gp));
         if (e != cudaSuccess) return fail(SG_ERR_CUDA, "matrix-vector (MMA) kernel launch: %s", cudaGetErrorString(e));
         g_launches.fetch_add(1);
+        note_kernel("sg::gemv_mma_kernel<%s, %s>", desc->in_dtype == SG_F16 ? "__half" : "__nv_bfloat16", wide ? "true" : "false");
         t_last_plan[0] = 0;
         t_last_plan[1] = 0;
         t_last_plan[2] = -static_cast<int32_t>(ks);
@@ -908,6 +917,8 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
                                                : launch_gemv<__nv_bfloat16>(gp, rb, static_cast<int>(ctas), cs);
     if (e != cudaSuccess) return fail(SG_ERR_CUDA, "matrix-vector kernel launch: %s", cudaGetErrorString(e));
     g_launches.fetch_add(1);
+    note_kernel("sg::gemv_kernel<%s, %d, %d>", desc->in_dtype == SG_F32 ? "float" : (desc->in_dtype == SG_F16 ? "__half" : "__nv_bfloat16"),
+                rb, static_cast<int>(nvec <= 1 ? 1 : (nvec == 2 ? 2 : 4)));
     t_last_plan[0] = 0;              // no tensor-core tiles: rows per CTA and K ranges instead
     t_last_plan[1] = 0;
     t_last_plan[2] = -static_cast<int32_t>(ks);
@@ -941,6 +952,8 @@ const char* sg_status_string(sg_status_t s) {
 const char* sg_last_error(void) { return t_err; }
 
 int64_t sg_launch_count(void) { return g_launches.load(); }
+
+const char* sg_last_kernel_name(void) { return t_last_kernel; }
 
 sg_status_t sg_set_option(int32_t option, int64_t value) {
     if (option < 0 || option >= SG_OPT_COUNT_) return fail(SG_ERR_INVALID_ARG, "sg_set_option: option %d is not a sg_option_t", option);
@@ -1718,6 +1731,8 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
     else transpose_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(tp);
     SG_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
+    note_kernel("sg::transpose_kernel<%s, %s>", desc->in_dtype == SG_F32 ? "float" : "__nv_bfloat16",
+                desc->out_dtype == SG_F32 ? "float" : "__nv_bfloat16");
     return SG_OK;
 }
 

@@ -39,7 +39,8 @@ EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_
             "sg_conv2d_dgrad", "sg_conv2d_wgrad",
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
-            "sg_last_kernel_clock", "sg_transpose", "sg_set_option", "sg_test_set_status_word"]
+            "sg_last_kernel_clock", "sg_transpose", "sg_set_option", "sg_test_set_status_word",
+            "sg_last_kernel_name"]
 OPTIONS = {"epi_warps": 0, "tail_split": 1, "tail_ksplit": 2, "band_m": 3, "general_kernel": 4, "no_pdl": 5, "no_short_a": 6,
            "no_gemv": 7, "gemv_no_mma": 8, "gemv_no_wide": 9, "gemv_rows": 10, "wait_limit_ns": 11}
 
@@ -135,6 +136,7 @@ _lib.sg_set_scratch.restype = ctypes.c_int
 _lib.sg_set_scratch.argtypes = [_vp, ctypes.c_size_t]
 _lib.sg_last_launch_plan.restype = ctypes.c_int
 _lib.sg_last_launch_plan.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+_lib.sg_last_kernel_name.restype = ctypes.c_char_p
 _lib.sg_set_option.restype = ctypes.c_int
 _lib.sg_set_option.argtypes = [_i32, _i64]
 _lib.sg_test_set_status_word.restype = ctypes.c_int
@@ -591,6 +593,11 @@ test_set_status_word.__test__ = False      # not a pytest test, whatever module 
 
 def launch_count() -> int:
     return int(_lib.sg_launch_count())
+
+
+def last_kernel_name() -> str:
+    """``sg_last_kernel_name``: the device function this thread's most recent launch ran (the library's own record)."""
+    return _lib.sg_last_kernel_name().decode()
 
 
 def last_launch_plan() -> dict:
