@@ -399,7 +399,9 @@ typedef enum {
     SG_OPT_GEMV_ROWS = 10,      /* 1, 2 or 4 matrix rows per CTA in the single-vector kernel */
     SG_OPT_WAIT_LIMIT_NS = 11,  /* bound of every device-side wait in nanoseconds (default 2 s); tests shorten it to
                                    see the kernel give up, record where, and return */
-    SG_OPT_COUNT_ = 12
+    SG_OPT_L2_WARM_KBLOCKS = 12, /* k-blocks of every CTA's first tile prefetched into the L2 at kernel entry, before the
+                                   launch dependency is waited for (default: 4 when the K loop has at most 16 k-blocks, else 0) */
+    SG_OPT_COUNT_ = 13
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

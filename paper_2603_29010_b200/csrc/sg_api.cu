@@ -527,6 +527,10 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
         else if (p.mode == MODE_GROUPED && plain && !p.ex_any) variant = 3;
         else if (p.mode == MODE_CONV && !p.a_mn_major && p.b_mn_major && p.ksplit <= 1 && !p.ex_any) variant = 5;
     }
+    // L2 warm-up at kernel entry: measured to pay for short K loops, where a launch is mostly its start and its end
+    // (128 problems of 256 x 256 x 512: 17.6 -> 17.1 us with 4 k-blocks), and to cost a little on long ones
+    // (4096^3: 94.6 -> 95.3 us with 8)
+    if (p.warm_kb < 0) p.warm_kb = p.num_kb <= 16 ? 4 : 0;
     KernelEntry k = kernel_for(s.bn, s.pair, out_kind, s.epi_warps, variant);
     const int ctas_per_tile = s.pair ? 2 : 1;
     const int slots = s.pair ? d.max_pairs : d.sm_count;
@@ -570,6 +574,8 @@ void base_params(Params* p, const DeviceState& d, float alpha, float beta, int32
     p->epi_arg0 = a0;
     p->epi_arg1 = a1;
     p->status = d.status_dev;
+    const int64_t warm = opt(SG_OPT_L2_WARM_KBLOCKS);
+    p->warm_kb = warm >= 0 ? static_cast<int32_t>(warm > 64 ? 64 : warm) : -1;      // -1: launch() decides from the K loop's length
     const int64_t limit = opt(SG_OPT_WAIT_LIMIT_NS);
     p->timeout_ns = limit > 0 ? static_cast<uint64_t>(limit) : kWaitLimitNs;
 }
@@ -973,8 +979,17 @@ sg_status_t sg_test_set_status_word(uint32_t value, void* cuda_stream) {
 }
 
 #ifdef SG_DEBUG_STAMPS
-// Diagnostic builds only (-DSG_DEBUG_STAMPS=<n>, never the product library, hence not in solgemm.h): copies out the 32
-// time-stamp words that CTA n - 1 of the last launch recorded.
+// Diagnostic builds only (-DSG_DEBUG_STAMPS, never the product library, hence not in solgemm.h): choose the CTA that
+// records time stamps in later launches, and copy out the 32 time-stamp words it recorded in the last one.
+sg_status_t sg_debug_select_cta(uint32_t cta) {
+    DeviceState* d = nullptr;
+    sg_status_t st = device_state(&d);
+    if (st != SG_OK) return st;
+    const uint64_t v = cta;
+    SG_CUDA(cudaDeviceSynchronize());
+    SG_CUDA(cudaMemcpy(reinterpret_cast<uint64_t*>(d->status_dev + 8) + 31, &v, sizeof v, cudaMemcpyHostToDevice));
+    return SG_OK;
+}
 sg_status_t sg_debug_stamps(uint64_t* out32) {
     DeviceState* d = nullptr;
     sg_status_t st = device_state(&d);

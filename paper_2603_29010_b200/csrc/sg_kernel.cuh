@@ -95,6 +95,7 @@ struct alignas(64) Params {
     // remap_w0 + remap_sw * j) of the remap_H x remap_W image that C and D address; 0 = rows are stored as they come
     int32_t d_remap, remap_h0, remap_sh, remap_w0, remap_sw, remap_H, remap_W;
     int32_t a_rows;                     // rows of A loaded per tile (128; 64 or 32 in the short-A variants)
+    int32_t warm_kb;                    // k-blocks of a CTA's first tile prefetched into the L2 at kernel entry
     int32_t nphases;                    // > 1: the tile list is the concatenation of ph[0 .. nphases), A maps in tmPh
     ConvPhase ph[kMaxPhases];
     CUtensorMap tmPh[kMaxPhases];
@@ -139,14 +140,15 @@ __device__ __forceinline__ float half_bits_to_float(uint16_t b, bool f16) {
     return f16 ? __half2float(__ushort_as_half(b)) : __uint_as_float(static_cast<uint32_t>(b) << 16);
 }
 
-// Diagnostic build (-DSG_DEBUG_STAMPS=<n>, off in the product library): CTA n - 1 records %globaltimer values at a
-// few points of its life (entry, set-up done, first load issued, first MMA, accumulator ready, last store, exit) into
-// the words after the status words; sg_debug_stamps() reads them back.  This is how the per-role time lines of a
-// launch's start and end were measured.
+// Diagnostic build (-DSG_DEBUG_STAMPS, off in the product library): one CTA -- its index is the 64-bit word 31 of the
+// stamp area, written by sg_debug_select_cta() -- records %globaltimer values at a few points of its life (entry,
+// set-up done, first load issued, first MMA, accumulator ready, last store, exit) into the words after the status
+// words; sg_debug_stamps() reads them back.  This is how the per-role time lines of a launch's start and end were
+// measured.
 #ifdef SG_DEBUG_STAMPS
 #define SG_STAMP(slot)                                                                           \
     do {                                                                                         \
-        if (blockIdx.x == (SG_DEBUG_STAMPS - 1)) {                                               \
+        if (blockIdx.x == sg_stamp_cta) {                                                        \
             reinterpret_cast<volatile uint64_t*>(p.status + 8)[slot] = global_timer_ns();        \
         }                                                                                        \
     } while (0)
@@ -470,7 +472,16 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     const uint32_t tmem_slot = bar_base + 8u * Cfg::NUM_BARS;
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem + Cfg::OFF_BAR + 8 * Cfg::NUM_BARS);
 
+#ifdef SG_DEBUG_STAMPS
+    const uint32_t sg_stamp_cta = static_cast<uint32_t>(reinterpret_cast<volatile uint64_t*>(p.status + 8)[31]);
+#endif
     if (threadIdx.x == 0) SG_STAMP(0);
+    // The first operand tile cannot arrive before the TMA unit holds the tensor maps: fetch them at once, from a warp
+    // that has nothing else to do yet, while thread 0 sets the barriers up.
+    if (threadIdx.x == 64 && p.mode != MODE_GROUPED) {
+        prefetch_tensormap(&p.tmA);
+        prefetch_tensormap(&p.tmB);
+    }
     // CTA 0 measures the SM clock this launch actually ran at (cycle counter against the nanosecond timer);
     // the host reads it through sg_last_kernel_clock for clock-scaled Speed-of-Light figures.
     uint64_t clk0 = 0, ns0 = 0;
@@ -479,7 +490,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         ns0 = global_timer_ns();
     }
 #ifdef SG_DEBUG_STAMPS
-    if (threadIdx.x == 32 && blockIdx.x == (SG_DEBUG_STAMPS - 1)) {
+    if (threadIdx.x == 32 && blockIdx.x == sg_stamp_cta) {
         reinterpret_cast<volatile uint64_t*>(p.status + 8)[11] = clock64();
         reinterpret_cast<volatile uint64_t*>(p.status + 8)[13] = global_timer_ns();
     }
@@ -507,21 +518,37 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         for (int w = 0; w < Cfg::EPI_WARPS; ++w) mbar_init(fetch_bar(w), 1);
         fence_barrier_init();
     }
-    // Early start: a launch spends its first microsecond and a half between kernel entry and its first TMA load
-    // (TMEM allocation, the set-up barrier, first execution of the producer's code).  For plain K-contiguous dense
-    // problems on single-CTA tiles the thread that initialised the barriers therefore issues the loads of the first
-    // tile's first stages right away, before the rest of the set-up; the producer loop skips those k-blocks.
+    // Start of a launch.  Between kernel entry and the first operand bytes in shared memory lie the set-up (TMEM
+    // allocation, barriers), the first execution of the producer's code and a DRAM round trip; under programmatic
+    // dependent launch a CTA may also sit for a microsecond or two waiting for the previous kernel in the stream to
+    // finish.  For plain K-contiguous dense problems two things shorten that:
+    //  * L2 warm-up: an otherwise idle thread asks the TMA unit to PREFETCH the first k-blocks of the CTA's first
+    //    tile into the L2 -- before the launch dependency is waited for (nothing reaches the SM, and the L2 is the
+    //    point of coherence, so this is safe even if the previous kernel is still writing those very lines);
+    //  * early start (single-CTA tiles): the thread that initialised the barriers issues the loads of the first
+    //    tile's first stages itself, before the set-up barrier; the producer loop skips those k-blocks.
     int early_kb = 0;
-    if constexpr (!kPair) {
-        if (mode == MODE_DENSE && !a_mn && !b_mn && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
-            static_cast<int>(blockIdx.x) < p.num_tiles) {
-            int g_hint0 = 0;
-            const Tile t0 = decode_tile<Cfg::TILE_M, BN, kVB>(p, static_cast<int>(blockIdx.x), g_hint0);
-            if (t0.n0 < p.N) {
+    if (mode == MODE_DENSE && !a_mn && !b_mn && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
+        static_cast<int>(blockIdx.x) / kCtas < p.num_tiles) {
+        int g_hint0 = 0;
+        const Tile t0 = decode_tile<Cfg::TILE_M, BN, kVB>(p, static_cast<int>(blockIdx.x) / kCtas, g_hint0);
+        if (t0.n0 < p.N) {
+            const CUtensorMap* mapB0 = (t0.width != BN) ? &p.tmB2 : &p.tmB;
+            const int b_rows0 = t0.width / kCtas;
+            const int m00 = t0.m0 + static_cast<int>(cta_rank) * Cfg::BM;
+            const int nb00 = t0.n0 + static_cast<int>(cta_rank) * b_rows0;
+            if (threadIdx.x == 96) {
+                const int npf = min(p.warm_kb, t0.kb1 - t0.kb0);
+                for (int j = 0; j < npf; ++j) {
+                    tma_prefetch_3d(&p.tmA, (t0.kb0 + j) * p.bk_elems, m00, t0.b);
+                    tma_prefetch_3d(mapB0, (t0.kb0 + j) * p.bk_elems, nb00, t0.b);
+                }
+            }
+            if constexpr (!kPair) {
                 early_kb = min(STAGES, t0.kb1 - t0.kb0);
                 if (threadIdx.x == 0) {
                     grid_dependency_wait();
-                    const CUtensorMap* mapB0 = (t0.width != BN) ? &p.tmB2 : &p.tmB;
+                    SG_STAMP(2);
                     const uint32_t tx0 = static_cast<uint32_t>(Cfg::A_BYTES + t0.width * Cfg::BK * 2);
                     for (int j = 0; j < early_kb; ++j) {
                         const uint32_t a_dst = smem_base + j * Cfg::STAGE_BYTES;
@@ -537,11 +564,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         tmem_alloc<kPair>(tmem_slot, Cfg::TMEM_COLS);
         tmem_relinquish<kPair>();
     }
-    if (warp == 0 && lane == 0 && mode != MODE_GROUPED) {
-        prefetch_tensormap(&p.tmA);
-        prefetch_tensormap(&p.tmB);
-        prefetch_tensormap(&p.tmD);
-    }
+    if (warp == 0 && lane == 0 && mode != MODE_GROUPED) prefetch_tensormap(&p.tmD);
     tc_fence_before_sync();
     const bool dead = __syncthreads_or(bad != 0u) != 0;
     if constexpr (kPair) {
@@ -1302,7 +1325,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     }
     if (threadIdx.x == 32) SG_STAMP(10);
 #ifdef SG_DEBUG_STAMPS
-    if (threadIdx.x == 32 && blockIdx.x == (SG_DEBUG_STAMPS - 1)) {
+    if (threadIdx.x == 32 && blockIdx.x == sg_stamp_cta) {
         reinterpret_cast<volatile uint64_t*>(p.status + 8)[12] = clock64();
         reinterpret_cast<volatile uint64_t*>(p.status + 8)[14] = global_timer_ns();
     }

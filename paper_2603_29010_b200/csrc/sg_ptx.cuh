@@ -134,6 +134,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
             : "memory");
     }
 }
+// Tiled 3-D prefetch global -> L2 of the box a later tma_load_3d with the same map and coordinates will read.  Nothing
+// reaches the SM, so it may be issued before a programmatic launch dependency has resolved: the L2 is the point of
+// coherence, later writes of the previous kernel update the prefetched lines.
+__device__ __forceinline__ void tma_prefetch_3d(const void* tmap, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(tmap), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
 // Untiled bulk copy global -> shared memory of this CTA, completing `bytes` on an mbarrier of this CTA.
 // Both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
