@@ -274,6 +274,9 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
  *   out  device, out_dtype (bf16 or fp32), [batch][cols][rows], row stride ld_out, batch stride stride_out
  *   fp32 -> bf16 rounds to nearest even; bf16 -> fp32 is exact.  in and out must not overlap.
  * Base pointers 16-byte aligned, ld and strides multiples of 16 bytes, ld_in >= cols, ld_out >= rows.
+ * When rows and cols both span multiples of 16 bytes (in the output resp. input type) the stage runs as a persistent
+ * kernel that streams tiles through shared memory with TMA loads and stores; other extents take a plain-store kernel
+ * with element-wise edges.  Either way nothing outside out[b][c][0 .. rows) is written.
  * An empty extent returns SG_OK without a launch.  A memory-bound kernel: its Speed-of-Light time is
  * batch*rows*cols*(input + output element bytes) / bandwidth (sg_sol_bound, SG_OP_TRANSPOSE).
  */
@@ -401,7 +404,8 @@ typedef enum {
                                    see the kernel give up, record where, and return */
     SG_OPT_L2_WARM_KBLOCKS = 12, /* k-blocks of every CTA's first tile prefetched into the L2 at kernel entry, before the
                                    launch dependency is waited for (default: 4 when the K loop has at most 16 k-blocks, else 0) */
-    SG_OPT_COUNT_ = 13
+    SG_OPT_TRANSPOSE_PLAIN = 13, /* 1: sg_transpose always runs its plain-store kernel (the one ragged extents take) */
+    SG_OPT_COUNT_ = 14
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

@@ -152,6 +152,20 @@ sg_status_t device_state(DeviceState** out) {
                                 if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
                             }
             if (d.init_status == SG_OK) {
+                cudaError_t e2 = cudaFuncSetAttribute(transpose_tma_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                      TransposeCfg<float, float>::SMEM_BYTES);
+                if (e2 == cudaSuccess)
+                    e2 = cudaFuncSetAttribute(transpose_tma_kernel<float, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              TransposeCfg<float, __nv_bfloat16>::SMEM_BYTES);
+                if (e2 == cudaSuccess)
+                    e2 = cudaFuncSetAttribute(transpose_tma_kernel<__nv_bfloat16, float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              TransposeCfg<__nv_bfloat16, float>::SMEM_BYTES);
+                if (e2 == cudaSuccess)
+                    e2 = cudaFuncSetAttribute(transpose_tma_kernel<__nv_bfloat16, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              TransposeCfg<__nv_bfloat16, __nv_bfloat16>::SMEM_BYTES);
+                if (e2 != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(transpose shared memory)", cudaGetErrorString(e2));
+            }
+            if (d.init_status == SG_OK) {
                 // how many 2-CTA clusters fit at once (some GPCs may not pair up all of their SMs)
                 KernelEntry k = kernel_for(256, true, 0, 8);
                 cudaLaunchConfig_t cfg = {};
@@ -186,14 +200,15 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // 3-D tiled map over a row-major [batch][rows][inner] tensor with 128-byte swizzled boxes.
 sg_status_t make_tiled_map(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base, uint64_t inner,
                            uint64_t rows, uint64_t batch, uint64_t row_stride_elems, uint64_t batch_stride_elems,
-                           uint32_t box_inner, uint32_t box_rows, const char* what) {
+                           uint32_t box_inner, uint32_t box_rows, const char* what,
+                           CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     cuuint64_t dims[3] = {inner, rows, batch};
     cuuint64_t strides[2] = {row_stride_elems * esize, batch_stride_elems * esize};
     if (batch <= 1) strides[1] = strides[0] * (rows > 0 ? rows : 1);
     cuuint32_t box[3] = {box_inner, box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = g_encode_tiled(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(SG_ERR_CUDA, "cuTensorMapEncodeTiled(%s) failed with CUresult %d (dims %llu x %llu x %llu, strides %llu, %llu)",
@@ -1731,6 +1746,62 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
     DeviceState* d = nullptr;
     sg_status_t st = device_state(&d);
     if (st != SG_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // Extents that are multiples of 16 bytes in both types (every tile edge then falls on a 16-byte boundary of its
+    // row): the persistent TMA kernel.  Ragged extents take the plain-store kernel below.
+    if ((desc->cols * es_in) % 16 == 0 && (desc->rows * es_out) % 16 == 0 && desc->rows <= INT32_MAX && desc->cols <= INT32_MAX &&
+        desc->batch <= INT32_MAX && opt(SG_OPT_TRANSPOSE_PLAIN) <= 0) {
+        const int vi = 16 / es_in, vo = 16 / es_out;
+        const int TR = 16 * vo, TC = 16 * vi;
+        const int64_t tr = (desc->rows + TR - 1) / TR, tc = (desc->cols + TC - 1) / TC;
+        if (tr * tc * desc->batch > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_transpose: too many tiles");
+        TransposeTmaParams tp;
+        memset(&tp, 0, sizeof tp);
+        const CUtensorMapDataType dt_in = desc->in_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+        const CUtensorMapDataType dt_out = desc->out_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+        st = make_tiled_map(&tp.tm_in, dt_in, es_in, in, desc->cols, desc->rows, desc->batch, desc->ld_in, desc->stride_in, TC, TR,
+                            "transpose input", CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (st != SG_OK) return st;
+        st = make_tiled_map(&tp.tm_out, dt_out, es_out, out, desc->rows, desc->cols, desc->batch, desc->ld_out, desc->stride_out, TR, TC,
+                            "transpose output", CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (st != SG_OK) return st;
+        tp.tiles_r = static_cast<int32_t>(tr);
+        tp.tiles_c = static_cast<int32_t>(tc);
+        tp.num_tiles = static_cast<int32_t>(tr * tc * desc->batch);
+        tp.status = d->status_dev;
+        const int64_t limit = opt(SG_OPT_WAIT_LIMIT_NS);
+        tp.timeout_ns = limit > 0 ? static_cast<uint64_t>(limit) : kWaitLimitNs;
+        cudaLaunchConfig_t cfg = {};
+        const int64_t slots = static_cast<int64_t>(d->sm_count) *
+                              (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32 ? TransposeCfg<float, float>::CTAS_PER_SM : 1);
+        cfg.gridDim = dim3(static_cast<unsigned>(tp.num_tiles < slots ? tp.num_tiles : slots));
+        cfg.blockDim = dim3(288);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = opt(SG_OPT_NO_PDL) > 0 ? 0 : 1;
+        cudaError_t e;
+        if (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32) {
+            cfg.dynamicSmemBytes = TransposeCfg<float, float>::SMEM_BYTES;
+            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<float, float>, tp);
+        } else if (desc->in_dtype == SG_F32) {
+            cfg.dynamicSmemBytes = TransposeCfg<float, __nv_bfloat16>::SMEM_BYTES;
+            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<float, __nv_bfloat16>, tp);
+        } else if (desc->out_dtype == SG_F32) {
+            cfg.dynamicSmemBytes = TransposeCfg<__nv_bfloat16, float>::SMEM_BYTES;
+            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<__nv_bfloat16, float>, tp);
+        } else {
+            cfg.dynamicSmemBytes = TransposeCfg<__nv_bfloat16, __nv_bfloat16>::SMEM_BYTES;
+            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<__nv_bfloat16, __nv_bfloat16>, tp);
+        }
+        if (e != cudaSuccess) return fail(SG_ERR_CUDA, "transpose kernel launch: %s", cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+        note_kernel("sg::transpose_tma_kernel<%s, %s>", desc->in_dtype == SG_F32 ? "float" : "__nv_bfloat16",
+                    desc->out_dtype == SG_F32 ? "float" : "__nv_bfloat16");
+        return SG_OK;
+    }
     TransposeParams tp;
     tp.in = in;
     tp.out = out;
@@ -1739,7 +1810,6 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
     tp.stride_in = desc->stride_in; tp.stride_out = desc->stride_out;
     tp.tiles_r = static_cast<int32_t>(tiles_r); tp.tiles_c = static_cast<int32_t>(tiles_c);
     const dim3 grid(static_cast<unsigned>(tiles_r * tiles_c * desc->batch));
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32) transpose_kernel<float, float><<<grid, 256, 0, stream>>>(tp);
     else if (desc->in_dtype == SG_F32) transpose_kernel<float, __nv_bfloat16><<<grid, 256, 0, stream>>>(tp);
     else if (desc->out_dtype == SG_F32) transpose_kernel<__nv_bfloat16, float><<<grid, 256, 0, stream>>>(tp);

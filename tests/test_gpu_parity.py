@@ -491,6 +491,30 @@ def test_transpose_with_dtype_conversion_bit_exact(shape, in_dtype, out_dtype):
         assert torch.equal(sg.transpose(x.to(DEV), out_dtype=out_dtype).cpu(), x.permute(0, 2, 1).to(out_dtype))
 
 
+@pytest.mark.parametrize("in_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_transpose_many_tiles_per_cta_and_both_kernels(in_dtype, out_dtype):
+    # Far more tiles than SMs x ring stages: every CTA of the persistent TMA kernel wraps its stage ring and reuses both
+    # output tiles several times; rows and columns end inside a tile (clipped loads and stores).
+    batch, rows, cols = 6, 1000, 2072
+    x = (inputs.normal([batch, rows, cols], 717, 1).float() * 1.37).to(in_dtype)
+    want = orc.transpose(x, out_dtype)
+    dx = x.to(DEV)
+    out, whole = guarded((batch, cols, rows), out_dtype)
+    sg.transpose(dx, out=out)
+    assert sg.last_kernel_name().startswith("sg::transpose_tma_kernel")
+    parity.assert_bit_exact(out, want, f"TMA transpose {in_dtype}->{out_dtype}")
+    assert guards_intact(whole)
+    try:
+        sg.set_option("transpose_plain", 1)                  # the kernel ragged extents take, on the same problem
+        out2 = torch.full((batch, cols, rows), float("nan"), dtype=out_dtype, device=DEV)
+        sg.transpose(dx, out=out2)
+        assert sg.last_kernel_name().startswith("sg::transpose_kernel")
+    finally:
+        sg.set_option("transpose_plain", -1)
+    assert torch.equal(out2, out)
+
+
 def test_layout_pipeline_nchw_conv_nchw_and_conv1d():
     # pipeline(transpose(input, NCHW, NHWC, fp32, bf16), conv2d_fprop, transpose(output, NHWC, NCHW, bf16, fp32))
     N, C, H, W, K = 2, 64, 10, 12, 72
