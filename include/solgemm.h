@@ -405,7 +405,9 @@ typedef enum {
     SG_OPT_L2_WARM_KBLOCKS = 12, /* k-blocks of every CTA's first tile prefetched into the L2 at kernel entry, before the
                                    launch dependency is waited for (default: 4 when the K loop has at most 16 k-blocks, else 0) */
     SG_OPT_TRANSPOSE_PLAIN = 13, /* 1: sg_transpose always runs its plain-store kernel (the one ragged extents take) */
-    SG_OPT_COUNT_ = 14
+    SG_OPT_EARLY_DONORS = 14,   /* K ranges for the last partial wave with the donor ranges run first (needs a scratch):
+                                   0 never, k = 2..4 that many ranges per tile (default: the planner's estimate) */
+    SG_OPT_COUNT_ = 15
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

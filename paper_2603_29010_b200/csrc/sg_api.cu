@@ -96,6 +96,8 @@ KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 
         case 5: return kernel_variant_5(bn, pair, out, epi_warps);
         case 6: return kernel_variant_6(bn, pair, out, epi_warps);
         case 7: return kernel_variant_7(bn, pair, out, epi_warps);
+        case 8: return kernel_variant_8(bn, pair, out, epi_warps);
+        case 9: return kernel_variant_9(bn, pair, out, epi_warps);
         default: return kernel_variant_0(bn, pair, out, epi_warps);
     }
 }
@@ -145,8 +147,8 @@ sg_status_t device_state(DeviceState** out) {
                 for (int pair = 0; pair < 2 && d.init_status == SG_OK; ++pair)
                     for (int f32 = 0; f32 < 3 && d.init_status == SG_OK; ++f32)
                         for (int ew = 4; ew <= 8 && d.init_status == SG_OK; ew += 4)
-                            for (int variant = 0; variant < 8 && d.init_status == SG_OK; ++variant) {
-                                if (variant >= 6 && pair) continue;      // the short-A variants have no two-CTA form
+                            for (int variant = 0; variant < 10 && d.init_status == SG_OK; ++variant) {
+                                if ((variant == 6 || variant == 7) && pair) continue;      // the short-A variants have no two-CTA form
                                 KernelEntry k = kernel_for(bns[i], pair != 0, f32, ew, variant);
                                 e = cudaFuncSetAttribute(k.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem);
                                 if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
@@ -437,7 +439,7 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
 void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1, bool allow_ksplit = true) {
     const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
-    int best_split = 1, best_ksplit = 1;
+    int best_split = 1, best_ksplit = 1, early_ks = 0;
     const int64_t rem = full_tiles % slots;
     const int forced = static_cast<int>(opt(SG_OPT_TAIL_SPLIT));      // 1, 2 or 4
     const int env_k = static_cast<int>(opt(SG_OPT_TAIL_KSPLIT));      // 0 = off, >= 2: that many K ranges
@@ -490,6 +492,44 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
                 best_split = 1;
             }
         }
+        // K ranges with early donors (see decode_tile): with at least one whole wave before the partial one, the tiles
+        // of the last wave are cut into ks K ranges of which all but the last run FIRST, on CTAs of their own, and park
+        // their sums; the CTA that runs the last range at the very end has them put into its accumulator beforehand, by
+        // epilogue warps that would otherwise idle.  Nobody waits for a peer and nothing is exchanged after the last MMA,
+        // so the tail costs 1 / ks of a tile -- against column slices, which are bound by operand traffic and take
+        // almost a whole tile's time however narrow they are.  (Needs two whole waves: the accumulator is filled while
+        // the CTA works on the item before the last.)
+        const int early_opt = static_cast<int>(opt(SG_OPT_EARLY_DONORS));      // -1 auto, 0 off, k >= 2: k ranges
+        const int64_t waves = full_tiles / slots;
+        if (allow_ksplit && d.scratch && tail_mode != 0 && tail_mode != 1 && early_opt != 0 && forced_k <= 0 && waves >= 2 &&
+            rem * 2 <= slots && p->num_kb >= 16) {
+            const size_t buf_bytes = static_cast<size_t>(s.pair ? 2 : 1) * 128 * s.bn * sizeof(float);
+            size_t max_buffers = d.scratch_bytes > kScratchFlagBytes ? (d.scratch_bytes - kScratchFlagBytes) / buf_bytes : 0;
+            if (max_buffers > static_cast<size_t>(kScratchMaxBuffers)) max_buffers = kScratchMaxBuffers;
+            int64_t ks_max = slots / rem;
+            if (ks_max > 4) ks_max = 4;
+            while (ks_max >= 2 && (p->num_kb / ks_max < 8 || static_cast<size_t>(rem * ks_max) > max_buffers)) --ks_max;
+            const double t_tile = kUsPerKBlock * p->num_kb * (s.bn / 256.0) * (s.pair ? 1.5 : 1.18);      // one whole tile, us
+            double best_time = t_tile * (best_ksplit > 1 ? 1.0 / best_ksplit : best) + (best_ksplit > 1 ? ksplit_exchange_us(best_ksplit) : 0.0);
+            int64_t ks = 0;
+            // Measured against column slices (the kernel variant that keeps the K-range code in runs its tiles 2 - 3 %
+            // slower than the plain one, which eats the better balance on short K loops): 4096 x 4096 x 8192 188.7 ->
+            // 184.2 us, 2560 x 4096 x 8192 123.2 -> 120.1, 4096^3 93.4 -> 93.8, 4096 x 4096 x 2048 49.2 -> 49.9.  So the
+            // planner takes this road for K loops of 96 k-blocks or more only.
+            for (int64_t k = 2; k <= ks_max && p->num_kb >= 96; ++k) {
+                const double t = t_tile / static_cast<double>(k) + 0.5;
+                if (t < best_time * 0.9) {
+                    best_time = t;
+                    ks = k;
+                }
+            }
+            if (early_opt >= 2 && early_opt <= ks_max) ks = early_opt;
+            if (ks >= 2 && rem <= kScratchMaxBuffers) {
+                early_ks = static_cast<int>(ks);
+                best_ksplit = early_ks;
+                best_split = 1;
+            }
+        }
     }
     // raster bands: keep a band's A panels (band_m x TILE_M rows x K) within about 32 MB of L2
     const int64_t panel_bytes = static_cast<int64_t>(s.pair ? 256 : 128) * (p->K > 0 ? p->K : 1) * 2;
@@ -502,6 +542,13 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
     p->ksplit = best_ksplit;
     p->split_begin = static_cast<int32_t>(parts > 1 ? full_tiles - rem : full_tiles);
     p->num_tiles = static_cast<int32_t>(parts > 1 ? full_tiles - rem + rem * parts : full_tiles);
+    p->sk_early = 0;
+    if (early_ks > 1) {
+        // list: R (ks - 1) donor parts, the whole waves' tiles, R owner parts
+        p->sk_early = static_cast<int32_t>(rem * (early_ks - 1));
+        p->split_begin = static_cast<int32_t>(p->sk_early + (full_tiles - rem));
+        p->num_tiles = static_cast<int32_t>(p->split_begin + rem);
+    }
     if (best_ksplit > 1) {
         p->sk_flags = static_cast<uint32_t*>(d.scratch);
         p->sk_consumed_off = kScratchMaxBuffers;
@@ -536,9 +583,12 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     const bool no_lean = opt(SG_OPT_GENERAL_KERNEL) > 0;
     int variant = 0;
     if (!no_lean && !p.in_fp8) {
-        const bool plain = !p.a_mn_major && !p.b_mn_major && p.ksplit <= 1 && !p.d_remap && p.nphases <= 1;
+        const bool plain_k = !p.a_mn_major && !p.b_mn_major && !p.d_remap && p.nphases <= 1;
+        const bool plain = plain_k && p.ksplit <= 1;
         if (p.mode == MODE_DENSE && plain) variant = p.ex_any ? 4 : (p.a_rows == 64 ? 6 : (p.a_rows == 32 ? 7 : 1));
         else if (p.mode == MODE_CONV && plain && !p.ex_any) variant = 2;
+        else if (p.mode == MODE_DENSE && plain_k && !p.ex_any && p.a_rows == 128) variant = 8;      // dense with K ranges
+        else if (p.mode == MODE_CONV && plain_k && !p.ex_any) variant = 9;                          // convolution with K ranges
         else if (p.mode == MODE_GROUPED && plain && !p.ex_any) variant = 3;
         else if (p.mode == MODE_CONV && !p.a_mn_major && p.b_mn_major && p.ksplit <= 1 && !p.ex_any) variant = 5;
     }

@@ -78,6 +78,7 @@ struct alignas(64) Params {
     float* sk_partials;                 // K-split scratch: [tail tile][part][CTA of the tile][128 rows][BN] fp32
     uint32_t* sk_flags;                 // K-split scratch: [tail tile] arrival counters, then [tail tile] done counters
     int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
+    int32_t sk_early;                   // > 0: "early donors" (see decode_tile); the number of donor items at the list's head
     float alpha, beta;
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
     int32_t epi, mode;
@@ -197,7 +198,16 @@ __device__ __forceinline__ void raster(const Params& p, int r, int tiles_m, int&
 // Position t of the tile list -> tile.  The list holds the full-width tiles of all complete waves first;
 // the tiles of the last, partial wave follow as `split` column slices each, so that more SMs share them.
 // kV: kernel variant (see contract_kernel).
-template <int TILE_M, int BN, int kV = 0>
+//
+// K ranges with early donors (p.sk_early > 0; problems with whole waves of tiles plus a partial last wave): each of the
+// R tiles of the last wave has its K loop cut into ksplit ranges.  The first ksplit - 1 of them ("donor" parts) are the
+// very FIRST items of R (ksplit - 1) CTAs (list positions 0 .. sk_early), which park their raw sums in the scratch and
+// go on to their full tiles; the last range (the "owner" part) is the very LAST item of another R CTAs (positions
+// split_begin ..).  Long before an owner part starts, the epilogue warps of its CTA -- idle between two epilogues -- add
+// the donors' parked sums up and write them into the TMEM accumulator the part will use (tcgen05.st); its MMAs then
+// accumulate on top of them and its epilogue is an ordinary one.  Nobody waits for a peer that runs at the same time,
+// nothing is fetched after the last MMA, and every CTA gets the same amount of work to within one K range.
+template <int TILE_M, int BN, int kV = 0, bool kSplitK = (kV == 0)>
 __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint) {
     Tile ti;
     int sub = 0;
@@ -207,9 +217,27 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, int t, int& g_hint)
     ti.part = 0;
     ti.nparts = 1;
     ti.tail = 0;
-    if (t >= p.split_begin) {
+    if (kSplitK && p.sk_early > 0) {
+        const int first_tail = p.split_begin - p.sk_early;     // id of the first tile of the last wave
+        if (t < p.sk_early || t >= p.split_begin) {
+            ti.nparts = p.ksplit;
+            if (t < p.sk_early) {
+                ti.tail = t / (p.ksplit - 1);
+                ti.part = t - ti.tail * (p.ksplit - 1);
+            } else {
+                ti.tail = t - p.split_begin;
+                ti.part = p.ksplit - 1;
+            }
+            t = first_tail + ti.tail;
+            const int base = p.num_kb / p.ksplit, extra = p.num_kb - base * p.ksplit;
+            ti.kb0 = ti.part * base + min(ti.part, extra);
+            ti.kb1 = ti.kb0 + base + (ti.part < extra ? 1 : 0);
+        } else {
+            t -= p.sk_early;
+        }
+    } else if (t >= p.split_begin) {
         const int u = t - p.split_begin;
-        if (kV == 0 && p.ksplit > 1) {
+        if (kSplitK && p.ksplit > 1) {
             // the tile's K range is shared by ksplit work items
             ti.nparts = p.ksplit;
             ti.tail = u / p.ksplit;
@@ -440,7 +468,9 @@ template <int BN, bool kPair, int kOut, int kEpiWarps, int kV = 0>
 __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) contract_kernel(const __grid_constant__ Params p) {
     // variants 6 and 7 are variant 1 with an A tile of 64 resp. 32 loaded rows
     constexpr int kARows = kV == 6 ? 64 : (kV == 7 ? 32 : 128);
-    constexpr int kVB = kV >= 6 ? 1 : kV;
+    // variants 8 and 9 are variants 1 and 2 (dense, convolution forward) with the K-range code kept in
+    constexpr int kVB = kV >= 8 ? kV - 7 : (kV >= 6 ? 1 : kV);
+    constexpr bool kSplitK = (kV == 0 || kV >= 8);
     using Cfg = Config<BN, kPair, kEpiWarps, kARows>;
     // options the specialised variants fold away at compile time
     constexpr bool kLean = kVB != 0;
@@ -531,7 +561,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
     if (mode == MODE_DENSE && !a_mn && !b_mn && (smem_base & 1023u) == 0u && p.num_kb > 0 &&
         static_cast<int>(blockIdx.x) / kCtas < p.num_tiles) {
         int g_hint0 = 0;
-        const Tile t0 = decode_tile<Cfg::TILE_M, BN, kVB>(p, static_cast<int>(blockIdx.x) / kCtas, g_hint0);
+        const Tile t0 = decode_tile<Cfg::TILE_M, BN, kVB, kSplitK>(p, static_cast<int>(blockIdx.x) / kCtas, g_hint0);
         if (t0.n0 < p.N) {
             const CUtensorMap* mapB0 = (t0.width != BN) ? &p.tmB2 : &p.tmB;
             const int b_rows0 = t0.width / kCtas;
@@ -592,7 +622,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             uint32_t phase = 0;
             int g_hint = 0, g_fenced = -1;
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                Tile ti = decode_tile<Cfg::TILE_M, BN, kVB>(p, t, g_hint);
+                Tile ti = decode_tile<Cfg::TILE_M, BN, kVB, kSplitK>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;                       // a column slice past the last column: no work
                 const int m0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM;
                 const int b_rows = ti.width / kCtas;              // rows of B this CTA loads
@@ -725,7 +755,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const uint64_t b_desc0 = b_mn ? smem_desc_mn_major_sw128(smem_base + Cfg::A_BYTES)
                                                   : smem_desc_k_major_sw128(smem_base + Cfg::A_BYTES);
             for (int t = first_tile; t < p.num_tiles && ok && num_kb > 0; t += tile_step) {
-                const Tile ti = decode_tile<Cfg::TILE_M, BN, kVB>(p, t, g_hint);
+                const Tile ti = decode_tile<Cfg::TILE_M, BN, kVB, kSplitK>(p, t, g_hint);
                 if (ti.n0 >= p.N) continue;
                 if (ti.kb1 <= ti.kb0) continue;                  // a phase no filter tap reaches: the epilogue writes beta C
                 const int in_kind = kLean ? 0 : p.in_fp8;          // 0 sixteen-bit, 1 / 2 fp8, 3 tf32, 4 int8
@@ -737,6 +767,8 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 const int acc = iter & 1;
                 const uint32_t acc_phase = (iter >> 1) & 1u;
                 ++iter;
+                // an owner part of the early-donor scheme finds the donors' sums in its accumulator: add to them
+                const bool preloaded = kSplitK ? (p.sk_early > 0 && ti.nparts > 1 && ti.part == ti.nparts - 1) : false;
                 if (!wait_bar(tempty_bar(acc), acc_phase ^ 1u, p, ROLE_MMA, t, 100 + acc)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
@@ -753,22 +785,22 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             umma_i8<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
-                                           (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                                           (kb != ti.kb0 || kk != 0 || preloaded) ? 1u : 0u);
                     } else if (in_kind == 3) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             umma_tf32<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
-                                             (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                                             (kb != ti.kb0 || kk != 0 || preloaded) ? 1u : 0u);
                     } else if (in_kind != 0) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             umma_fp8<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
-                                            (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                                            (kb != ti.kb0 || kk != 0 || preloaded) ? 1u : 0u);
                     } else {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
                             umma_bf16<kPair>(d_tmem, a_desc + a_step * kk, b_desc + b_step * kk, idesc,
-                                             (kb != ti.kb0 || kk != 0) ? 1u : 0u);
+                                             (kb != ti.kb0 || kk != 0 || preloaded) ? 1u : 0u);
                     }
                     umma_commit<kPair>(empty_bar(stage));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -811,12 +843,19 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
         for (int a = 0; a < 2; ++a) tempty_remote[a] = kPair ? map_to_cta(tempty_bar(a), 0) : tempty_bar(a);
 
         for (int t = first_tile; t < p.num_tiles && ok; t += tile_step) {
-            Tile ti = decode_tile<Cfg::TILE_M, BN, kVB>(p, t, g_hint);
+            Tile ti = decode_tile<Cfg::TILE_M, BN, kVB, kSplitK>(p, t, g_hint);
             if (ti.n0 >= p.N) continue;
             const bool has_k = num_kb > 0 && ti.kb1 > ti.kb0;   // else the tile is the empty sum: no accumulator is involved
             const int acc = iter & 1;
             const uint32_t acc_phase = (iter >> 1) & 1u;
             if (has_k) ++iter;
+            // K ranges with early donors: an owner part (list positions from split_begin on) finds the donors' sums in
+            // its accumulator, so its epilogue is an ordinary one; and the item that used that accumulator buffer before
+            // it -- two items earlier in this CTA's walk -- keeps the buffer until it has put them there.
+            const bool early = kSplitK ? p.sk_early > 0 : false;
+            const bool early_owner = early && ti.nparts > 1 && ti.part == ti.nparts - 1;
+            const int t_next2 = t + 2 * tile_step;
+            const bool preload_next = early && has_k && t_next2 >= p.split_begin && t_next2 < p.num_tiles;
             const int n0 = ti.n0;
             const int row0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32;
             const CUtensorMap* mapD = &p.tmD;
@@ -881,9 +920,12 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // from its own accumulator plus the other parts' parked sums
             // (pass 1), so the exchange is spread over all parts instead of serialised in one.  The unit of ownership
             // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
-            const bool ksplit_tile = kVB == 0 ? ti.nparts > 1 : false;
+            const bool ksplit_tile = kSplitK ? (ti.nparts > 1 && !early_owner) : false;
             // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
-            auto owned_by = [&](int c, int qq) { return (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part; };
+            // (early donors park every unit: nothing is theirs to finish)
+            auto owned_by = [&](int c, int qq) {
+                return early ? false : (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part;
+            };
             auto owned = [&](int c) { return owned_by(c, q); };
             // how many epilogue warps of this CTA finish at least one unit, and this warp's rank among them: the
             // stage ring (idle by then) is divided between them as the landing zone of the other parts' sums
@@ -901,7 +943,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
             }
             const int passes = ksplit_tile ? 2 : 1;
-            if (has_k && half >= nchunks && !ksplit_tile) {
+            if (has_k && half >= nchunks && !ksplit_tile && !preload_next) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
                 tc_fence_before_sync();
                 __syncwarp();
@@ -953,7 +995,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         for (int i = 0; i < 32; ++i)
                             v[i] = acc_s32 ? static_cast<float>(static_cast<int32_t>(r0[i])) : __uint_as_float(r0[i]);
                     }
-                    if (c + kStep >= nchunks && !ksplit_tile) {
+                    if (c + kStep >= nchunks && !ksplit_tile && !preload_next) {
                         // this warp has read its last columns of the accumulator: hand its share back to the MMA warp
                         tc_fence_before_sync();
                         __syncwarp();
@@ -1279,9 +1321,72 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (lane == 0) {
                     if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
                     else mbar_arrive(tempty_remote[acc]);
-                    uint32_t* arrived = p.sk_flags + ti.tail;
-                    uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
-                    if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals * ti.nparts) - 1u) {
+                    if (!early) {       // (with early donors the owner's CTA resets the counters)
+                        uint32_t* arrived = p.sk_flags + ti.tail;
+                        uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
+                        if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals * ti.nparts) - 1u) {
+                            *arrived = 0u;
+                            *consumed = 0u;
+                            __threadfence();
+                        }
+                    }
+                }
+            }
+            if (kSplitK && preload_next) {
+                // The item two further on is an owner part and will accumulate in the buffer this item just used: wait
+                // for the donors of its tile (they ran at the very start of the launch), add their parked sums up, write
+                // them into the buffer, and only then hand the buffer back to the MMA warp.
+                int g_hint2 = 0;
+                const Tile tn = decode_tile<Cfg::TILE_M, BN, kVB, kSplitK>(p, t_next2, g_hint2);
+                uint32_t* arrived = p.sk_flags + tn.tail;
+                uint32_t okw = 1;
+                if (lane == 0) okw = wait_counter(arrived, static_cast<uint32_t>(p.sk_arrivals * (tn.nparts - 1)), p, t_next2) ? 1u : 0u;
+                okw = __shfl_sync(0xFFFFFFFFu, okw, 0);
+                if (!okw) { ok = false; break; }
+                __threadfence();                // the donors' sums are read after their arrivals
+                if (tn.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32 < tn.rows) {
+                    constexpr uint32_t kUnitBytes = CH * 128u;
+                    const size_t tile_elems = static_cast<size_t>(Cfg::BM) * BN;
+                    const float* bufs = p.sk_partials + static_cast<size_t>(tn.tail) * p.ksplit * kCtas * tile_elems +
+                                        static_cast<size_t>(cta_rank) * tile_elems + lane * 4;
+                    const int nchunks2 = (min(tn.width, p.N - tn.n0) + CH - 1) / CH;
+#pragma unroll 1
+                    for (int c = half; c < nchunks2; c += kStep) {
+                        uint32_t w[CH];
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) w[i] = 0u;
+                        for (int g = 0; g < tn.nparts - 1; ++g) {
+                            const float* pb = bufs + static_cast<size_t>(g) * kCtas * tile_elems + static_cast<size_t>(c * 4 + q) * (kUnitBytes / 4);
+#pragma unroll
+                            for (int i = 0; i < CH; i += 4) {
+                                const float4 x = __ldcg(reinterpret_cast<const float4*>(pb + i * 32));
+                                w[i] = __float_as_uint(__uint_as_float(w[i]) + x.x);
+                                w[i + 1] = __float_as_uint(__uint_as_float(w[i + 1]) + x.y);
+                                w[i + 2] = __float_as_uint(__uint_as_float(w[i + 2]) + x.z);
+                                w[i + 3] = __float_as_uint(__uint_as_float(w[i + 3]) + x.w);
+                            }
+                        }
+                        uint32_t lo[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) lo[i] = w[i];
+                        tmem_st_32x32(t_row + c * CH, lo);
+                        if constexpr (!kOutF32) {
+                            uint32_t hi[32];
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) hi[i] = w[32 + i];
+                            tmem_st_32x32(t_row + c * CH + 32, hi);
+                        }
+                    }
+                    tmem_st_wait();
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
+                    else mbar_arrive(tempty_remote[acc]);
+                    // this warp is done with the tile's scratch: the last warp of the owner's CTAs leaves the counters at zero
+                    uint32_t* consumed = p.sk_flags + p.sk_consumed_off + tn.tail;
+                    if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals) - 1u) {
                         *arrived = 0u;
                         *consumed = 0u;
                         __threadfence();

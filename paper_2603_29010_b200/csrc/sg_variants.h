@@ -24,5 +24,7 @@ KernelEntry kernel_variant_4(int bn, bool pair, int out, int epi_warps);
 KernelEntry kernel_variant_5(int bn, bool pair, int out, int epi_warps);
 KernelEntry kernel_variant_6(int bn, bool pair, int out, int epi_warps);   // dense, 64 rows of A loaded (single-CTA tiles)
 KernelEntry kernel_variant_7(int bn, bool pair, int out, int epi_warps);   // dense, 32 rows of A loaded
+KernelEntry kernel_variant_8(int bn, bool pair, int out, int epi_warps);   // dense, K ranges kept in
+KernelEntry kernel_variant_9(int bn, bool pair, int out, int epi_warps);   // convolution forward, K ranges kept in
 
 }  // namespace sg

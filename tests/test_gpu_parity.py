@@ -226,6 +226,64 @@ def test_gemm_tail_wave_is_shared_between_sms(tile_n, pair, M, N, K, scratch):
         assert guards_intact(whole, cols=N)
 
 
+@pytest.mark.parametrize("tile_n,pair,M,N,K,ks", [
+    (256, 1, 256 * 150, 256, 1024, 2),         # 150 pair tiles on 74 pairs: two waves + 2 tiles, 2 ranges of 8 k-blocks
+    (256, 1, 256 * 149 + 77, 200, 2048, 4),    # ragged rows and columns, 4 ranges of 8 k-blocks
+    (256, 1, 256 * 79, 512, 1536, 3),          # 158 tiles: two waves + 10 tiles, 3 ranges
+    (128, 0, 128 * 149, 256, 1024, 2),         # single-CTA tiles: 298 tiles on 148 SMs
+    (128, 0, 128 * 149 + 5, 200, 2056, 3),     # 150 x 2 = 300 tiles on 148 SMs, ragged rows and columns, K tail of 8
+    (64, 1, 256 * 150, 64, 1024, 2),           # narrow pair tiles
+])
+def test_k_ranges_with_early_donors_bit_exact(tile_n, pair, M, N, K, ks):
+    # The tiles of the last, partial wave have their K loop cut into ks ranges; the first ks - 1 ranges run as the very
+    # first items of CTAs of their own and park their sums, which the CTA that runs the last range at the end finds in
+    # its accumulator.
+    # Integer inputs and fp32 output: whatever the summation order, the result must be exact.  Twice in a row: the
+    # arrival counters must be back at zero after a launch.
+    sg.set_tuning(tile_n, pair)
+    sg.set_option("early_donors", ks)
+    try:
+        A = inputs.small_integers([M, K], 343, 1)
+        B = inputs.small_integers([N, K], 343, 2)
+        bias = inputs.small_integers([N], 343, 4, -3, 3)
+        ref, _ = orc.gemm(A, B, bias=bias, alpha=2.0, epi="relu")
+        dA, dB, db = A.to(DEV), B.to(DEV), bias.to(DEV)
+        D, whole = guarded((M, N), torch.float32)
+        for _ in range(2):
+            D.fill_(float("nan"))
+            sg.gemm(dA, dB, bias=db, alpha=2.0, epi="relu", out=D)
+            plan = sg.last_launch_plan()
+            assert plan["tail_split"] == -ks, plan
+            assert plan["split_begin"] > plan["tiles"] - plan["split_begin"], plan      # owner parts sit at the list's end
+            parity.assert_bit_exact(D, ref, f"early donors {plan}")
+            assert guards_intact(whole, cols=N)
+    finally:
+        sg.set_option("early_donors", -1)
+
+
+def test_k_ranges_with_early_donors_conv_and_real_values():
+    # the convolution path (151 pair tiles of 256 pixels x 256 filters on 74 pairs; 18 k-blocks in 2 ranges) ...
+    sg.set_tuning(256, 1)
+    sg.set_option("early_donors", 2)
+    try:
+        X = inputs.small_integers([4, 98, 98, 128], 353, 6, -1, 1)
+        Wf = inputs.small_integers([256, 3, 3, 128], 353, 7, -1, 1) * (inputs.small_integers([256, 3, 3, 128], 354, 7, 0, 2) == 0).to(torch.bfloat16)
+        ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+        Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1), out_dtype=torch.float32)
+        assert sg.last_launch_plan()["tail_split"] == -2 and sg.last_kernel_name().endswith(", 9>")
+        parity.assert_bit_exact(Y.view(-1, 256), ref.reshape(-1, 256), "conv early donors")
+        # ... and a dense problem with real values, residual, bias and GELU in bf16
+        M, N, K = 256 * 75, 320, 1544                     # 75 x 2 = 150 tiles
+        A, B, bias = inputs.make_gemm(M, N, K, "normal", K ** -0.25, bias=True, seed=363)
+        C = inputs.normal([M, N], 363, 3)
+        ref, absacc = orc.gemm(A, B, C=C, bias=bias, alpha=1.25, beta=0.5, epi="gelu")
+        D = sg.gemm(A.to(DEV), B.to(DEV), C=C.to(DEV), bias=bias.to(DEV), alpha=1.25, beta=0.5, epi="gelu")
+        assert sg.last_launch_plan()["tail_split"] == -2
+        parity.assert_matches(D, ref, absacc, "early donors, real values")
+    finally:
+        sg.set_option("early_donors", -1)
+
+
 def test_k_split_tail_with_full_epilogue_matches_oracle():
     sg.set_tuning(256, 1)
     sg.set_tail_mode(2)
