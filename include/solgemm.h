@@ -407,7 +407,11 @@ typedef enum {
     SG_OPT_TRANSPOSE_PLAIN = 13, /* 1: sg_transpose always runs its plain-store kernel (the one ragged extents take) */
     SG_OPT_EARLY_DONORS = 14,   /* K ranges for the last partial wave with the donor ranges run first (needs a scratch):
                                    0 never, k = 2..4 that many ranges per tile (default: the planner's estimate) */
-    SG_OPT_COUNT_ = 15
+    SG_OPT_TWO_PASS_SPLIT_K = 15, /* problems with fewer tiles than half the SMs and a long K loop: 0 = never cut the K loop
+                                   into ranges summed by a second kernel, k >= 2 = at most k ranges (default: as many as
+                                   there are SMs to go round) */
+    SG_OPT_SPLIT_K_REDUCE_WARPS = 16, /* second pass of a two-pass K split: 1, 2, 4 or 8 warps share the parts of a column slice */
+    SG_OPT_COUNT_ = 17
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

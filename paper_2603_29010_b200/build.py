@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libsolgemm.so")
 _SOURCES = ["sg_api.cu"] + [f"sg_variant_{v}.cu" for v in range(10)]
-_DEPS = _SOURCES + ["sg_kernel.cuh", "sg_ptx.cuh", "sg_transpose.cuh", "sg_gemv.cuh", "sg_variants.h", "sg_variant.inc",
+_DEPS = _SOURCES + ["sg_kernel.cuh", "sg_ptx.cuh", "sg_transpose.cuh", "sg_gemv.cuh", "sg_splitk.cuh", "sg_variants.h", "sg_variant.inc",
                     os.path.join(_ROOT, "include", "solgemm.h")]
 
 

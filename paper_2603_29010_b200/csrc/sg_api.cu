@@ -18,6 +18,7 @@
 #include "sg_variants.h"
 #include "sg_transpose.cuh"
 #include "sg_gemv.cuh"
+#include "sg_splitk.cuh"
 
 namespace {
 
@@ -314,6 +315,19 @@ struct Shape {
 // partial sums and finishes a share of the columns from the other parts' (measured: conv weight gradient and
 // skinny long-K products).
 inline double ksplit_exchange_us(int64_t ks) { return ks > 1 ? 6.0 + 0.5 * static_cast<double>(ks - 1) : 0.0; }
+// The same for the two-pass form (every part parks all its sums and exits; a second kernel adds them up): flat in ks.
+constexpr int kTwoPassMinKb = 4;           // k-blocks per part at least
+// Modelled time (us) of a two-pass K split with `ks` parts per tile: the longer of the parts' tensor time and of streaming
+// the operands from HBM (a CTA pulls about 38 GB/s, all of them together about 5.5 TB/s), plus a fixed 3 us for the
+// second kernel, plus writing and re-reading the parked sums.  Fitted to 256 x 256 x {8192 .. 131072}, 512 x 512 x 16384,
+// 1024 x 1024 x 8192 and 128 x 4096 x 16384 with the number of parts forced to 2 .. 74.
+inline double two_pass_us(int64_t tiles, int64_t ks, int bn, bool pair, int64_t num_kb, double t_kb, double t_fixed,
+                          double operand_bytes) {
+    const double ctas = static_cast<double>(tiles * ks * (pair ? 2 : 1));
+    const double rate = std::min(5.5e6, ctas * 0.038e6);                     // bytes per us
+    const double parked = static_cast<double>(tiles * ks) * (pair ? 2.0 : 1.0) * 128.0 * bn * 4.0;
+    return std::max(t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed, operand_bytes / rate) + 3.0 + 2.0 * parked / 8.0e6;
+}
 constexpr double kUsPerKBlock = 0.25;      // one 64-deep k-block of a 128 x 256 tile per SM
 
 bool ksplit_allowed(const DeviceState& d) {
@@ -327,6 +341,7 @@ struct MemHint {
     int epi = -1;
     int esize_in = 2;
     int esize_out = 2;
+    double operand_bytes = 0.0;      // bytes of A and B as stored (0: (rows + N) K esize_in per problem)
 };
 
 inline bool heavy_activation(int epi) {
@@ -335,7 +350,7 @@ inline bool heavy_activation(int epi) {
 }
 
 Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_problem, int64_t batch_mult, int64_t N,
-                   int64_t K, int min_b_rows = 1, MemHint mem = MemHint{}) {
+                   int64_t K, int min_b_rows = 1, MemHint mem = MemHint{}, bool two_pass_ok = false) {
     const int force_bn = g_tune_tile_n.load();
     const int force_pair = g_tune_pair.load();
     const int bns[3] = {256, 128, 64};
@@ -397,12 +412,23 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
             if (one_tile_row) cost = std::max(cost, stream_us(tiles, false));
             if (can_split && tiles * 2 <= slots) {
                 // less than half a wave: plan_tail may cut every tile's K loop into ranges run by different SMs
+                const bool two_pass = two_pass_ok && opt(SG_OPT_TWO_PASS_SPLIT_K) != 0;
                 int64_t ks_max = slots / tiles;
-                if (ks_max > 16) ks_max = 16;
-                if (ks_max > num_kb) ks_max = num_kb;
+                if (!two_pass && ks_max > 16) ks_max = 16;
+                if (ks_max > num_kb / (two_pass ? kTwoPassMinKb : 1)) ks_max = num_kb / (two_pass ? kTwoPassMinKb : 1);
+                double operand_bytes = mem.operand_bytes;
+                if (operand_bytes <= 0.0) {
+                    for (int64_t r : rows_per_problem) operand_bytes += static_cast<double>(r + N) * static_cast<double>(K) * mem.esize_in;
+                    operand_bytes *= static_cast<double>(batch_mult);
+                }
                 for (int64_t ks = 2; ks <= ks_max; ++ks) {
-                    double t = t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed + ksplit_exchange_us(ks);
-                    if (one_tile_row) t = std::max(t, stream_us(tiles * ks, true) + ksplit_exchange_us(ks));
+                    double t;
+                    if (two_pass) {
+                        t = two_pass_us(tiles, ks, bn, pi != 0, num_kb, t_kb, t_fixed, operand_bytes);
+                    } else {
+                        t = t_kb * static_cast<double>((num_kb + ks - 1) / ks) + t_fixed + ksplit_exchange_us(ks);
+                        if (one_tile_row) t = std::max(t, stream_us(tiles * ks, true) + ksplit_exchange_us(ks));
+                    }
                     if (t < cost) cost = t;
                 }
             }
@@ -436,7 +462,8 @@ Shape choose_shape(const DeviceState& d, const std::vector<int64_t>& rows_per_pr
 // cut into `split` column slices so that the idle SMs of that wave take a share.  Narrow slices cost more
 // per output area (same factors as in choose_shape), so a split is used only when it shortens the tail.
 // Sets p->split_begin, p->split and p->num_tiles (the length of the tile list) from the full-width count.
-void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1, bool allow_ksplit = true) {
+void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, int min_b_rows = 1, bool allow_ksplit = true,
+               bool two_pass_ok = false, double operand_bytes = 0.0) {
     const int64_t slots = s.pair ? d.max_pairs : d.sm_count;
     const double factor[2][3] = {{1.00, 1.10, 1.60}, {1.00, 1.26, 2.57}};   // relative to the full width: [pair][log2(split)]
     int best_split = 1, best_ksplit = 1, early_ks = 0;
@@ -543,6 +570,50 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
     p->split_begin = static_cast<int32_t>(parts > 1 ? full_tiles - rem : full_tiles);
     p->num_tiles = static_cast<int32_t>(parts > 1 ? full_tiles - rem + rem * parts : full_tiles);
     p->sk_early = 0;
+    p->sk_park_all = 0;
+    // Two-pass K split: fewer tiles than half the SMs (a skinny problem with a long K loop).  Every tile's K loop is cut
+    // into as many ranges as there are SMs to go round; each part parks its sums and exits, a second kernel adds them up
+    // and runs the epilogue (launch() enqueues it).  No part waits for another, and the cost of the exchange does not grow
+    // with the number of parts.
+    if (two_pass_ok && allow_ksplit && d.scratch && opt(SG_OPT_TWO_PASS_SPLIT_K) != 0 && tail_mode != 0 && tail_mode != 1 &&
+        tail_mode != 2 && forced_k <= 0 && full_tiles * 2 <= slots && p->num_kb >= 2 * kTwoPassMinKb) {
+        const size_t buf_bytes = static_cast<size_t>(s.pair ? 2 : 1) * 128 * s.bn * sizeof(float);
+        size_t max_buffers = d.scratch_bytes > kScratchFlagBytes ? (d.scratch_bytes - kScratchFlagBytes) / buf_bytes : 0;
+        int64_t ks_max = slots / full_tiles;
+        if (ks_max > p->num_kb / kTwoPassMinKb) ks_max = p->num_kb / kTwoPassMinKb;
+        while (ks_max >= 2 && static_cast<size_t>(full_tiles * ks_max) > max_buffers) --ks_max;
+        if (operand_bytes <= 0.0)
+            operand_bytes = (static_cast<double>(p->M) + p->N) * static_cast<double>(p->K) * (128.0 / p->bk_elems) *
+                            static_cast<double>(p->batch > 0 ? p->batch : 1);
+        const int pi = s.pair ? 1 : 0, bi = s.bn == 256 ? 0 : (s.bn == 128 ? 1 : 2);
+        const double shape_factor[2][3] = {{1.18, 1.56, 2.90}, {1.00, 1.50, 3.30}};      // as in choose_shape
+        const double t_kb = kUsPerKBlock * s.bn / 256.0 * shape_factor[pi][bi];
+        const double t_fixed = kUsPerKBlock * s.bn / 256.0 * 96.0 / 64.0;
+        int64_t ks = 0;
+        double best_t = 1e300;
+        for (int64_t k = 2; k <= ks_max; ++k) {
+            const double t = two_pass_us(full_tiles, k, s.bn, s.pair, p->num_kb, t_kb, t_fixed, operand_bytes);
+            if (t < best_t) {
+                best_t = t;
+                ks = k;
+            }
+        }
+        const int64_t forced_parts = opt(SG_OPT_TWO_PASS_SPLIT_K);
+        if (forced_parts >= 2) ks = forced_parts < ks_max ? forced_parts : ks_max;
+        if (ks >= 2) {
+            p->sk_park_all = 1;
+            p->split = 1;
+            p->ksplit = static_cast<int32_t>(ks);
+            p->split_begin = 0;
+            p->num_tiles = static_cast<int32_t>(full_tiles * ks);
+            p->band_m = INT32_MAX;      // tiles in plain column-major order: the second pass decodes them the same way
+            p->sk_partials = reinterpret_cast<float*>(static_cast<uint8_t*>(d.scratch) + kScratchFlagBytes);
+            p->sk_flags = static_cast<uint32_t*>(d.scratch);
+            p->sk_consumed_off = kScratchMaxBuffers;
+            p->sk_arrivals = s.epi_warps * (s.pair ? 2 : 1);
+            return;
+        }
+    }
     if (early_ks > 1) {
         // list: R (ks - 1) donor parts, the whole waves' tiles, R owner parts
         p->sk_early = static_cast<int32_t>(rem * (early_ks - 1));
@@ -620,6 +691,49 @@ sg_status_t launch(const DeviceState& d, const Shape& s, int out_kind, const Par
     SG_CUDA(cudaLaunchKernelEx(&cfg, k.fn, p));
     g_launches.fetch_add(1);
     note_kernel("sg::contract_kernel<%d, %s, %d, %d, %d>", s.bn, s.pair ? "true" : "false", out_kind, s.epi_warps, variant);
+    if (p.sk_park_all) {
+        // second pass of a two-pass K split: add the parked parts up and run the epilogue
+        SplitKReduceParams r;
+        memset(&r, 0, sizeof r);
+        r.partials = p.sk_partials;
+        r.status = p.status;
+        r.nparts = p.ksplit;
+        r.kctas = ctas_per_tile;
+        r.bn = s.bn;
+        r.tiles_m = p.tiles_m;
+        r.tiles_n = p.tiles_n;
+        r.M = p.M;
+        r.N = p.N;
+        r.batch = p.batch;
+        r.D = p.D;
+        r.C = p.C;
+        r.bias = p.bias;
+        r.ldd = p.ldd; r.strideD = p.strideD; r.ldc = p.ldc; r.strideC = p.strideC; r.strideBias = p.strideBias;
+        r.alpha = p.alpha; r.beta = p.beta; r.epi_arg0 = p.epi_arg0; r.epi_arg1 = p.epi_arg1;
+        r.epi = p.epi;
+        r.in_f16 = p.in_f16;
+        r.bias_f32 = p.in_fp8 == 3 ? 1 : 0;
+        const int ch = out_kind == 1 ? 32 : 64;
+        const int64_t full_tiles = static_cast<int64_t>(p.num_tiles) / p.ksplit;
+        cudaLaunchConfig_t rc = {};
+        r.pw = p.ksplit <= 4 ? 1 : (p.ksplit <= 8 ? 2 : (p.ksplit <= 16 ? 4 : 8));
+        const int64_t forced_pw = opt(SG_OPT_SPLIT_K_REDUCE_WARPS);
+        if (forced_pw == 1 || forced_pw == 2 || forced_pw == 4 || forced_pw == 8) r.pw = static_cast<int32_t>(forced_pw);
+        rc.gridDim = dim3(static_cast<unsigned>(full_tiles * ctas_per_tile * (s.bn / ch) * 4 * r.pw));
+        rc.blockDim = dim3(256);
+        rc.stream = stream;
+        rc.attrs = &attr[1];
+        rc.numAttrs = pdl ? 1 : 0;
+        using ReduceFn = void (*)(const SplitKReduceParams);
+        static const ReduceFn reduce_fns[3][4] = {
+            {splitk_reduce_kernel<0, 1>, splitk_reduce_kernel<0, 2>, splitk_reduce_kernel<0, 4>, splitk_reduce_kernel<0, 8>},
+            {splitk_reduce_kernel<1, 1>, splitk_reduce_kernel<1, 2>, splitk_reduce_kernel<1, 4>, splitk_reduce_kernel<1, 8>},
+            {splitk_reduce_kernel<2, 1>, splitk_reduce_kernel<2, 2>, splitk_reduce_kernel<2, 4>, splitk_reduce_kernel<2, 8>}};
+        const int pwi = r.pw == 1 ? 0 : (r.pw == 2 ? 1 : (r.pw == 4 ? 2 : 3));
+        cudaError_t e = cudaLaunchKernelEx(&rc, reduce_fns[out_kind][pwi], r);
+        if (e != cudaSuccess) return fail(SG_ERR_CUDA, "split-K second pass launch: %s", cudaGetErrorString(e));
+        g_launches.fetch_add(1);
+    }
     t_last_plan[0] = s.bn;
     t_last_plan[1] = s.pair ? 1 : 0;
     t_last_plan[2] = p.ksplit > 1 ? -p.ksplit : p.split;
@@ -688,10 +802,13 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     if (st != SG_OK) return st;
     if (c.in_fp8 == 3 && bias && (reinterpret_cast<uintptr_t>(bias) & 3u))
         return fail(SG_ERR_ALIGNMENT, "%s: an fp32 bias must be 4-byte aligned", who);
+    bool ex_any = false;
     {
         Params scratch_params;          // the chain's rules are checked before any device is touched
+        scratch_params.ex_any = 0;
         st = apply_ex(&scratch_params, ex, desc->N, c.esize_out, who);
         if (st != SG_OK) return st;
+        ex_any = ex != nullptr && scratch_params.ex_any != 0;
     }
     if (batch > 1) {
         if (sA < 0 || sB < 0 || sC < 0 || sD < 0 || sBias < 0) return fail(SG_ERR_INVALID_ARG, "%s: negative batch stride", who);
@@ -710,7 +827,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     p.bk_elems = c.bk;
     const int min_b_rows = desc->layout_b == SG_ROW_MAJOR ? 64 : 1;
     Shape s = choose_shape(*d, std::vector<int64_t>{desc->M}, batch, desc->N, desc->K, min_b_rows,
-                           MemHint{desc->epi, c.esize_in, c.esize_out});
+                           MemHint{desc->epi, c.esize_in, c.esize_out}, !ex_any);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_DENSE;
     p.a_mn_major = desc->layout_a == SG_COL_MAJOR ? 1 : 0;
@@ -724,7 +841,7 @@ sg_status_t run_dense(const sg_gemm_desc_t* desc, int64_t batch, int64_t sA, int
     const int64_t tiles = static_cast<int64_t>(p.tiles_m) * p.tiles_n * batch;
     if (tiles > INT32_MAX / 4) return fail(SG_ERR_UNSUPPORTED, "%s: too many tiles", who);
     p.num_kb = static_cast<int32_t>((desc->K + c.bk - 1) / c.bk);
-    plan_tail(*d, s, tiles, &p, min_b_rows);
+    plan_tail(*d, s, tiles, &p, min_b_rows, true, !ex_any);
     st = apply_ex(&p, ex, desc->N, c.esize_out, who);
     if (st != SG_OK) return st;
     // a few rows against a large matrix: load only 32 or 64 rows of A per stage (kernel variants 6 and 7), which
@@ -1329,10 +1446,13 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
     if (st != SG_OK) return st;
     if (c.in_fp8 == 3 && bias && (reinterpret_cast<uintptr_t>(bias) & 3u))
         return fail(SG_ERR_ALIGNMENT, "sg_conv2d_fprop: an fp32 bias must be 4-byte aligned");
+    bool ex_any = false;
     {
         Params scratch_params;
+        scratch_params.ex_any = 0;
         st = apply_ex(&scratch_params, ex, desc->K, c.esize_out, "sg_conv2d_fprop_ex");
         if (st != SG_OK) return st;
+        ex_any = ex != nullptr && scratch_params.ex_any != 0;
     }
     if (desc->C == 0) return fail(SG_ERR_UNSUPPORTED, "sg_conv2d_fprop: C == 0");
 
@@ -1344,7 +1464,10 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
     p.in_f16 = c.in_f16 ? 1 : 0;
     p.in_fp8 = c.in_fp8;
     p.bk_elems = c.bk;
-    Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg);
+    const double conv_bytes = (static_cast<double>(desc->N) * desc->H * desc->W * desc->C + static_cast<double>(desc->K) * Kg) * c.esize_in;
+    MemHint conv_hint;
+    conv_hint.operand_bytes = conv_bytes;
+    Shape s = choose_shape(*d, std::vector<int64_t>{Mg}, 1, desc->K, Kg, 1, conv_hint, !ex_any);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_CONV;
     p.M = static_cast<int32_t>(Mg);
@@ -1355,7 +1478,7 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
     p.tiles_n = static_cast<int32_t>((desc->K + s.bn - 1) / s.bn);
     p.cblocks = static_cast<int32_t>((desc->C + c.bk - 1) / c.bk);
     p.num_kb = static_cast<int32_t>(desc->R * desc->S) * p.cblocks;
-    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p);
+    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n, &p, 1, true, !ex_any, conv_bytes);
     p.bias = bias;
     p.C = desc->beta != 0.0f ? Cin : nullptr;
     p.ldc = desc->K;
@@ -1719,7 +1842,10 @@ extern "C" sg_status_t sg_conv2d_wgrad(const sg_conv2d_desc_t* desc, const void*
     p.in_f16 = c.in_f16 ? 1 : 0;
     p.bk_elems = c.bk;
     // one product per filter tap: dW[:, tap, :] (K x C) = dY^T (K x pixels) . X shifted by the tap (pixels x C)
-    Shape s = choose_shape(*d, std::vector<int64_t>{desc->K}, taps, desc->C, pixels, 64);
+    const double wgrad_bytes = (static_cast<double>(pixels) * desc->K + static_cast<double>(desc->N) * desc->H * desc->W * desc->C) * c.esize_in;
+    MemHint wgrad_hint;
+    wgrad_hint.operand_bytes = wgrad_bytes;
+    Shape s = choose_shape(*d, std::vector<int64_t>{desc->K}, taps, desc->C, pixels, 64, wgrad_hint, true);
     const int tile_m = s.pair ? 256 : 128;
     p.mode = MODE_WGRAD;
     p.a_mn_major = 1;
@@ -1732,7 +1858,7 @@ extern "C" sg_status_t sg_conv2d_wgrad(const sg_conv2d_desc_t* desc, const void*
     p.tiles_m = static_cast<int32_t>((desc->K + tile_m - 1) / tile_m);
     p.tiles_n = static_cast<int32_t>((desc->C + s.bn - 1) / s.bn);
     p.num_kb = static_cast<int32_t>((pixels + 63) / 64);
-    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n * taps, &p, 64);
+    plan_tail(*d, s, static_cast<int64_t>(p.tiles_m) * p.tiles_n * taps, &p, 64, true, true, wgrad_bytes);
     p.C = desc->beta != 0.0f ? Cin : nullptr;
     p.ldc = taps * desc->C;
     p.strideC = desc->C;

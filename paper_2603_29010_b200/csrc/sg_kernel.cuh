@@ -79,6 +79,7 @@ struct alignas(64) Params {
     uint32_t* sk_flags;                 // K-split scratch: [tail tile] arrival counters, then [tail tile] done counters
     int32_t sk_consumed_off;            // index of the first consumed counter inside sk_flags
     int32_t sk_early;                   // > 0: "early donors" (see decode_tile); the number of donor items at the list's head
+    int32_t sk_park_all;                // 1: two-pass K split: every part parks all its sums, a second kernel adds them up
     float alpha, beta;
     float epi_arg0, epi_arg1;           // activation parameters (leaky_relu / elu slope, clip bounds)
     int32_t epi, mode;
@@ -922,9 +923,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             // is one warp's 32 rows x one column chunk of one CTA: unit u belongs to part u mod nparts.
             const bool ksplit_tile = kSplitK ? (ti.nparts > 1 && !early_owner) : false;
             // chunk index first: one warp's chunks then go to different parts, and so do one chunk's warps
-            // (early donors park every unit: nothing is theirs to finish)
+            // (early donors, and the parts of a two-pass K split, park every unit: nothing is theirs to finish)
+            const bool two_pass = kSplitK ? p.sk_park_all != 0 : false;
             auto owned_by = [&](int c, int qq) {
-                return early ? false : (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part;
+                return (early || two_pass) ? false : (c + (BN / CH) * (qq * kCtas + static_cast<int>(cta_rank))) % ti.nparts == ti.part;
             };
             auto owned = [&](int c) { return owned_by(c, q); };
             // how many epilogue warps of this CTA finish at least one unit, and this warp's rank among them: the
@@ -942,7 +944,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     }
                 }
             }
-            const int passes = ksplit_tile ? 2 : 1;
+            const int passes = (ksplit_tile && !two_pass) ? 2 : 1;      // (two-pass: the kernel's end publishes the sums)
             if (has_k && half >= nchunks && !ksplit_tile && !preload_next) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
                 tc_fence_before_sync();
@@ -1321,7 +1323,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (lane == 0) {
                     if constexpr (kPair) mbar_arrive_cluster(tempty_remote[acc]);
                     else mbar_arrive(tempty_remote[acc]);
-                    if (!early) {       // (with early donors the owner's CTA resets the counters)
+                    if (!early && !two_pass) {       // (with early donors the owner's CTA resets the counters)
                         uint32_t* arrived = p.sk_flags + ti.tail;
                         uint32_t* consumed = p.sk_flags + p.sk_consumed_off + ti.tail;
                         if (atomicAdd(consumed, 1u) == static_cast<uint32_t>(p.sk_arrivals * ti.nparts) - 1u) {

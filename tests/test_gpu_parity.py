@@ -284,6 +284,55 @@ def test_k_ranges_with_early_donors_conv_and_real_values():
         sg.set_option("early_donors", -1)
 
 
+@pytest.mark.parametrize("tile_n,pair", [(-1, -1), (64, 0), (128, 0), (256, 0), (128, 1), (256, 1)])
+@pytest.mark.parametrize("batch,M,N,K", [(1, 256, 256, 8192), (1, 300, 200, 4104), (3, 130, 72, 2048), (1, 17, 264, 16384)])
+def test_two_pass_split_k_bit_exact(batch, M, N, K, tile_n, pair):
+    # A few tiles and a long K loop: the K loop is cut into many ranges, every part parks its sums, and a second kernel
+    # adds them up and runs the epilogue.  Integer inputs with sparse A so that every sum stays exact in bf16 too.
+    sg.set_tuning(tile_n, pair)
+    A = inputs.small_integers([batch, M, K], 373, 1) * (inputs.small_integers([batch, M, K], 374, 1, 0, 31) == 0).to(torch.bfloat16)
+    B = inputs.small_integers([batch, N, K], 373, 2)
+    bias = inputs.small_integers([N], 373, 4, -3, 3)
+    C = inputs.small_integers([batch, M, N], 373, 3, -2, 2)
+    for out_dtype in (torch.bfloat16, torch.float32):
+        ref = torch.stack([orc.gemm(A[b], B[b], C=C[b].to(out_dtype), bias=bias, alpha=2.0, beta=1.0, epi="relu")[0] for b in range(batch)])
+        assert float(ref.abs().max()) <= 256
+        D, whole = guarded((batch, M, N) if N % 8 == 0 else (M, N), out_dtype)
+        if batch > 1 or N % 8 == 0:
+            for _ in range(2):
+                D.fill_(float("nan"))
+                if batch == 1:
+                    sg.gemm(A[0].to(DEV), B[0].to(DEV), C=C[0].to(out_dtype).to(DEV), bias=bias.to(DEV), alpha=2.0, beta=1.0,
+                            epi="relu", out=D[0] if D.dim() == 3 else D)
+                else:
+                    sg.batched_gemm(A.to(DEV), B.to(DEV), C=C.to(out_dtype).to(DEV), bias=bias.to(DEV), alpha=2.0, beta=1.0,
+                                    epi="relu", out=D)
+                plan = sg.last_launch_plan()
+                assert plan["tail_split"] < -1, plan
+                parity.assert_bit_exact(D, ref, f"two-pass split-K {plan}")
+                assert guards_intact(whole, cols=N)
+
+
+def test_two_pass_split_k_real_values_and_part_counts():
+    # real values, GELU, fp32 and bf16 outputs, and the number of parts pinned to 2, 5 and "as many as fit"
+    M, N, K = 256, 384, 16384 + 8
+    A, B, bias = inputs.make_gemm(M, N, K, "normal", K ** -0.25, bias=True, seed=383)
+    ref, absacc = orc.gemm(A, B, bias=bias, alpha=0.75, epi="gelu")
+    try:
+        for parts in (2, 5, -1):
+            sg.set_option("two_pass_split_k", parts)
+            for out_dtype in (torch.bfloat16, torch.float32):
+                D = sg.gemm(A.to(DEV), B.to(DEV), bias=bias.to(DEV), alpha=0.75, epi="gelu", out_dtype=out_dtype)
+                plan = sg.last_launch_plan()
+                assert plan["tail_split"] < -1 and (parts < 0 or plan["tail_split"] == -parts), plan
+                parity.assert_matches(D, ref, absacc, f"two-pass {parts} parts {out_dtype}")
+        sg.set_option("two_pass_split_k", 0)            # off: the one-kernel exchange through the scratch
+        D = sg.gemm(A.to(DEV), B.to(DEV), bias=bias.to(DEV), alpha=0.75, epi="gelu")
+        parity.assert_matches(D, ref, absacc, "one-kernel K ranges")
+    finally:
+        sg.set_option("two_pass_split_k", -1)
+
+
 def test_k_split_tail_with_full_epilogue_matches_oracle():
     sg.set_tuning(256, 1)
     sg.set_tail_mode(2)
