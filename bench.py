@@ -51,8 +51,9 @@ PER_CLOCK_FLOPS = 8192.0 * 148  # dense bf16 FLOP per SM clock of the whole chip
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from one ncu capture of
 # the timed launch (read + write of one c2 launch); not re-measured by this script.
-NCU_DRAM_BYTES_PER_LAUNCH = 73_352_448 + 16_339_456
-NCU_DRAM_SOURCE = "one ncu capture of one launch of this kernel on this problem (an earlier build of the same tiling), not this run"
+NCU_DRAM_BYTES_PER_LAUNCH = 71_833_344 + 15_188_736
+NCU_DRAM_SOURCE = ("one ncu capture (--metrics dram__bytes_read.sum,dram__bytes_write.sum, one launch) of this kernel, "
+                   "sg::contract_kernel<256, true, 0, 4, 1>, on this problem; not re-measured by this run")
 
 
 def measured_peaks():

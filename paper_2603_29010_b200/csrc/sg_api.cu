@@ -589,8 +589,10 @@ void plan_tail(const DeviceState& d, Shape& s, int64_t full_tiles, Params* p, in
         const double shape_factor[2][3] = {{1.18, 1.56, 2.90}, {1.00, 1.50, 3.30}};      // as in choose_shape
         const double t_kb = kUsPerKBlock * s.bn / 256.0 * shape_factor[pi][bi];
         const double t_fixed = kUsPerKBlock * s.bn / 256.0 * 96.0 / 64.0;
+        // the unsplit launch as the yardstick: a split has to be a tenth faster to be taken
+        const double ctas1 = static_cast<double>(full_tiles * (s.pair ? 2 : 1));
         int64_t ks = 0;
-        double best_t = 1e300;
+        double best_t = 0.9 * std::max(t_kb * static_cast<double>(p->num_kb) + t_fixed, operand_bytes / std::min(5.5e6, ctas1 * 0.038e6));
         for (int64_t k = 2; k <= ks_max; ++k) {
             const double t = two_pass_us(full_tiles, k, s.bn, s.pair, p->num_kb, t_kb, t_fixed, operand_bytes);
             if (t < best_t) {
