@@ -98,3 +98,63 @@ def _wgrad_worker(rank, world, port):
 
 def test_two_ranks_data_parallel_conv_gradients_over_gloo():
     mp.spawn(_wgrad_worker, args=(2, _free_port()), nprocs=2, join=True)
+
+
+def _shard_worker(rank, world, port):
+    """Each rank computes its shard of a small GEMM, batched GEMM, convolution and grouped GEMM (the oracle stands in for
+    the per-rank kernel); gathered over gloo, the shards must reproduce the whole problem exactly."""
+    from oracle import oracle as orc
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        def gather(mine, full_rows):
+            # pad every rank's rows to the same count so that all_gather applies, then cut the padding off again
+            pad = torch.zeros((full_rows,) + tuple(mine.shape[1:]), dtype=torch.float64)
+            pad[:mine.shape[0]] = mine
+            outs = [torch.zeros_like(pad) for _ in range(world)]
+            dist.all_gather(outs, pad)
+            return outs
+        # GEMM: rows of A and D (cuts on the 256-row tile)
+        M, N, K = 700, 40, 24
+        A, B = inputs.small_integers([M, K], 61, 1), inputs.small_integers([N, K], 61, 2)
+        whole, _ = orc.gemm(A, B, epi="relu")
+        r0, r1 = sharding.gemm_rows(M, world, rank, 256)
+        mine, _ = orc.gemm(A[r0:r1].contiguous(), B, epi="relu")
+        parts = gather(mine, M)
+        cuts = [sharding.gemm_rows(M, world, r, 256) for r in range(world)]
+        assert torch.equal(torch.cat([parts[r][:c1 - c0] for r, (c0, c1) in enumerate(cuts)]), whole)
+        # batched: batch entries
+        Ab, Bb = inputs.small_integers([5, 16, 8], 62, 1), inputs.small_integers([5, 24, 8], 62, 2)
+        wholeb, _ = orc.batched_gemm(Ab, Bb)
+        b0, b1 = sharding.batch_entries(5, world, rank)
+        mineb, _ = orc.batched_gemm(Ab[b0:b1].contiguous(), Bb[b0:b1].contiguous())
+        partsb = gather(mineb, 5)
+        cutsb = [sharding.batch_entries(5, world, r) for r in range(world)]
+        assert torch.equal(torch.cat([partsb[r][:c1 - c0] for r, (c0, c1) in enumerate(cutsb)]), wholeb)
+        # convolution: images
+        X, Wf = inputs.small_integers([3, 6, 5, 8], 63, 6), inputs.small_integers([8, 3, 3, 8], 63, 7)
+        wholec, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1))
+        n0, n1 = sharding.conv_images(3, world, rank)
+        minec, _ = orc.conv2d_fprop(X[n0:n1].contiguous(), Wf, pad=(1, 1))
+        partsc = gather(minec, 3)
+        cutsc = [sharding.conv_images(3, world, r) for r in range(world)]
+        assert torch.equal(torch.cat([partsc[r][:c1 - c0] for r, (c0, c1) in enumerate(cutsc)]), wholec)
+        # grouped: whole groups; every group is computed by exactly one rank
+        Ms = [5, 0, 17, 9, 3]
+        As = [inputs.small_integers([m, 8], 64 + g, 1) for g, m in enumerate(Ms)]
+        Bs = [inputs.small_integers([12, 8], 64 + g, 2) for g in range(len(Ms))]
+        owned = sharding.assign_groups(Ms, world)
+        flags = torch.zeros(len(Ms))
+        for g in owned[rank]:
+            flags[g] = 1
+        dist.all_reduce(flags)
+        assert bool((flags == 1).all())
+        for g in owned[rank]:
+            if Ms[g]:
+                assert torch.equal(orc.gemm(As[g], Bs[g])[0], orc.grouped_gemm(As, Bs)[0][g])
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_shards_concatenate_to_the_whole_problem():
+    mp.spawn(_shard_worker, args=(2, _free_port()), nprocs=2, join=True)
