@@ -857,6 +857,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             const bool early_owner = early && ti.nparts > 1 && ti.part == ti.nparts - 1;
             const int t_next2 = t + 2 * tile_step;
             const bool preload_next = early && has_k && t_next2 >= p.split_begin && t_next2 < p.num_tiles;
+            // The accumulator buffer is handed back to the MMA warp only if a later item of this CTA will use it: at most
+            // the item after next can (the next one takes the other buffer).  On a CTA pair the hand-back is an arrival with
+            // cluster-scope release on the leader's barrier, about a microsecond -- in the middle of the one epilogue of
+            // the launch that nothing overlaps with.
+            const bool handback = t_next2 < p.num_tiles;
             const int n0 = ti.n0;
             const int row0 = ti.m0 + static_cast<int>(cta_rank) * Cfg::BM + q * 32;
             const CUtensorMap* mapD = &p.tmD;
@@ -945,7 +950,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 }
             }
             const int passes = (ksplit_tile && !two_pass) ? 2 : 1;      // (two-pass: the kernel's end publishes the sums)
-            if (has_k && half >= nchunks && !ksplit_tile && !preload_next) {
+            if (has_k && half >= nchunks && !ksplit_tile && !preload_next && handback) {
                 // no chunk of this tile is this warp's: it still has to hand the accumulator back
                 tc_fence_before_sync();
                 __syncwarp();
@@ -979,6 +984,10 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
             for (int c = half; c < nchunks; c += kStep) {
                 if (ksplit_tile && owned(c) != (pass == 1)) continue;
                 float v[CH];
+#ifdef SG_DEBUG_STAMPS
+                const bool stamp_chunk = warp == 2 && lane == 0 && t + tile_step >= p.num_tiles && c < 4;
+                if (stamp_chunk) SG_STAMP(16 + 3 * c);
+#endif
                 if (has_k) {
                     uint32_t r0[32];
                     tmem_ld_32x32(t_row + c * CH, r0);
@@ -997,7 +1006,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         for (int i = 0; i < 32; ++i)
                             v[i] = acc_s32 ? static_cast<float>(static_cast<int32_t>(r0[i])) : __uint_as_float(r0[i]);
                     }
-                    if (c + kStep >= nchunks && !ksplit_tile && !preload_next) {
+                    if (c + kStep >= nchunks && !ksplit_tile && !preload_next && handback) {
                         // this warp has read its last columns of the accumulator: hand its share back to the MMA warp
                         tc_fence_before_sync();
                         __syncwarp();
@@ -1094,6 +1103,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     }
                 }
 
+#ifdef SG_DEBUG_STAMPS
+                if (stamp_chunk) SG_STAMP(17 + 3 * c);
+#endif
                 if (alpha != 1.0f) {
 #pragma unroll
                     for (int i = 0; i < CH; ++i) v[i] *= alpha;
@@ -1283,6 +1295,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     continue;
                 }
 
+#ifdef SG_DEBUG_STAMPS
+                if (stamp_chunk) SG_STAMP(18 + 3 * c);
+#endif
                 // stage the 32 x 128-byte block (row = lane) in the swizzled layout the store map expects
                 const uint32_t sb = chunk_ctr % Cfg::STAGING_BUFS;
                 ++chunk_ctr;
