@@ -123,6 +123,28 @@ sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, co
                     const void* bias, void* D, void* cuda_stream);
 
 /*
+ * sg_gemm_host: sg_gemm for callers whose operands and result live in HOST memory (the end-to-end form the paper's
+ * generated wrappers have around a kernel: move the operands in, launch, hand the result back; Section 3, PyTorch wrapper).
+ *   A_host, B_host, C_host, bias_host, D_host   host pointers laid out exactly as `desc` says (same leading dimensions);
+ *                    pinned memory lets the copies overlap the kernel, pageable memory works but serialises them.
+ *                    Element alignment is enough.  C_host may be NULL when beta == 0, bias_host unless SG_EPI_BIAS.
+ *   staging_dev      device buffer lent by the caller, 256-byte aligned, at least sg_gemm_host_staging_size(desc)
+ *                    bytes: device copies of A, B, bias, C and D with the host's geometry.  The library allocates none.
+ *   chunks           the rows of A, C and D are cut into this many blocks (multiples of 256 rows; 0 = 4, at most 16):
+ *                    while one copy engine brings in block i+1 the kernel works on block i and the other copy engine
+ *                    takes block i-1 of D back, so the call costs about the larger of the two transfers, not their sum.
+ * Everything is ordered against `cuda_stream`: the call's work starts after what is already on it, and the stream
+ * continues only when D_host is complete; the call itself returns without synchronising.  The first call on a device
+ * creates two internal streams and a few events (not inside a stream capture).  Calls on one device share them: two
+ * calls may be in flight at once only on the same stream.
+ * Errors as for sg_gemm, SG_ERR_WORKSPACE for the staging buffer.  M == 0 or N == 0: SG_OK, nothing is enqueued.
+ */
+sg_status_t sg_gemm_host_staging_size(const sg_gemm_desc_t* desc, size_t* bytes);
+sg_status_t sg_gemm_host(const sg_gemm_desc_t* desc, const void* A_host, const void* B_host, const void* C_host,
+                         const void* bias_host, void* D_host, void* staging_dev, size_t staging_bytes, int32_t chunks,
+                         void* cuda_stream);
+
+/*
  * sg_batched_gemm: the same product for b = 0 .. batch-1, operand X of problem b starting at
  * X + b*strideX elements.                                      (paper: batched_gemm(), Appendix A.1)
  *   strideBias == 0 shares one bias vector between all problems.

@@ -1242,6 +1242,143 @@ sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, co
     return run_dense(desc, 1, 0, 0, 0, 0, 0, A, B, C, bias, D, cuda_stream, "sg_gemm");
 }
 
+// ---- sg_gemm with operands in host memory -------------------------------------------------------------------
+namespace {
+constexpr int kHostMaxChunks = 16;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t fork = nullptr, back = nullptr, arrived[kHostMaxChunks] = {}, done[kHostMaxChunks] = {};
+};
+HostPipe g_host_pipe[kMaxDevices];
+
+struct HostLayout {
+    size_t off_a, off_b, off_bias, off_c, off_d, total;
+    int64_t a_outer, b_outer;      // rows of the stored A / B arrays (the non-contiguous extent)
+};
+HostLayout host_layout(const sg_gemm_desc_t* d, const Checked& c) {
+    HostLayout L;
+    L.a_outer = d->layout_a == SG_ROW_MAJOR ? d->M : d->K;
+    L.b_outer = d->layout_b == SG_COL_MAJOR ? d->N : d->K;
+    size_t o = 0;
+    L.off_a = o;    o = round_up(o + static_cast<size_t>(L.a_outer) * d->lda * c.esize_in, 256);
+    L.off_b = o;    o = round_up(o + static_cast<size_t>(L.b_outer) * d->ldb * c.esize_in, 256);
+    L.off_bias = o; o = round_up(o + static_cast<size_t>(d->N) * 4, 256);
+    L.off_c = o;    o = round_up(o + (d->beta != 0.0f ? static_cast<size_t>(d->M) * d->ldc * c.esize_out : 0), 256);
+    L.off_d = o;    o = round_up(o + static_cast<size_t>(d->M) * d->ldd * c.esize_out, 256);
+    L.total = o;
+    return L;
+}
+}  // namespace
+
+sg_status_t sg_gemm_host_staging_size(const sg_gemm_desc_t* desc, size_t* bytes) {
+    if (!bytes) return fail(SG_ERR_NULL_POINTER, "bytes is NULL");
+    Checked c;
+    sg_status_t st = check_gemm_desc(desc, false, &c);
+    if (st != SG_OK) return st;
+    *bytes = host_layout(desc, c).total;
+    return SG_OK;
+}
+
+sg_status_t sg_gemm_host(const sg_gemm_desc_t* desc, const void* A_host, const void* B_host, const void* C_host,
+                         const void* bias_host, void* D_host, void* staging_dev, size_t staging_bytes, int32_t chunks,
+                         void* cuda_stream) {
+    Checked c;
+    sg_status_t st = check_gemm_desc(desc, false, &c);
+    if (st != SG_OK) return st;
+    if (desc->M == 0 || desc->N == 0) return SG_OK;
+    if (!D_host || (desc->K > 0 && (!A_host || !B_host))) return fail(SG_ERR_NULL_POINTER, "sg_gemm_host: A_host, B_host or D_host is NULL");
+    if (desc->beta != 0.0f && !C_host) return fail(SG_ERR_NULL_POINTER, "sg_gemm_host: beta != 0 needs C_host");
+    if (desc->epi == SG_EPI_BIAS && !bias_host) return fail(SG_ERR_NULL_POINTER, "sg_gemm_host: SG_EPI_BIAS needs bias_host");
+    const HostLayout L = host_layout(desc, c);
+    if (!staging_dev) return fail(SG_ERR_WORKSPACE, "sg_gemm_host: staging_dev is NULL");
+    if (reinterpret_cast<uintptr_t>(staging_dev) & 255u) return fail(SG_ERR_WORKSPACE, "sg_gemm_host: staging_dev must be 256-byte aligned");
+    if (staging_bytes < L.total) return fail(SG_ERR_WORKSPACE, "sg_gemm_host: staging has %zu bytes, %zu needed", staging_bytes, L.total);
+    if (chunks <= 0) chunks = 4;
+    if (chunks > kHostMaxChunks) chunks = kHostMaxChunks;
+
+    int dev = 0;
+    SG_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(SG_ERR_CUDA, "device index %d out of range", dev);
+    HostPipe& hp = g_host_pipe[dev];
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!hp.ready) {
+            SG_CUDA(cudaStreamCreateWithFlags(&hp.s_in, cudaStreamNonBlocking));
+            SG_CUDA(cudaStreamCreateWithFlags(&hp.s_out, cudaStreamNonBlocking));
+            SG_CUDA(cudaEventCreateWithFlags(&hp.fork, cudaEventDisableTiming));
+            SG_CUDA(cudaEventCreateWithFlags(&hp.back, cudaEventDisableTiming));
+            for (int i = 0; i < kHostMaxChunks; ++i) {
+                SG_CUDA(cudaEventCreateWithFlags(&hp.arrived[i], cudaEventDisableTiming));
+                SG_CUDA(cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming));
+            }
+            hp.ready = true;
+        }
+    }
+    cudaStream_t main_stream = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(staging_dev);
+    uint8_t* dA = base + L.off_a;
+    uint8_t* dB = base + L.off_b;
+    uint8_t* dBias = base + L.off_bias;
+    uint8_t* dC = base + L.off_c;
+    uint8_t* dD = base + L.off_d;
+    const size_t es_in = static_cast<size_t>(c.esize_in), es_out = static_cast<size_t>(c.esize_out);
+    const size_t bias_es = c.in_fp8 == 3 ? 4 : 2;
+    // row blocks of A and D: multiples of the 256-row tile
+    int64_t rows = (desc->M + chunks - 1) / chunks;
+    rows = (rows + 255) / 256 * 256;
+    if (rows < 256) rows = 256;
+    const int nblocks = static_cast<int>((desc->M + rows - 1) / rows);
+
+    // the staging buffers may still be in use by work enqueued on the caller's stream before this call
+    SG_CUDA(cudaEventRecord(hp.fork, main_stream));
+    SG_CUDA(cudaStreamWaitEvent(hp.s_in, hp.fork, 0));
+    SG_CUDA(cudaStreamWaitEvent(hp.s_out, hp.fork, 0));
+    if (desc->K > 0) {
+        const size_t b_inner = static_cast<size_t>(desc->layout_b == SG_COL_MAJOR ? desc->K : desc->N) * es_in;
+        SG_CUDA(cudaMemcpy2DAsync(dB, desc->ldb * es_in, B_host, desc->ldb * es_in, b_inner, static_cast<size_t>(L.b_outer),
+                                  cudaMemcpyHostToDevice, hp.s_in));
+    }
+    if (bias_host) SG_CUDA(cudaMemcpyAsync(dBias, bias_host, static_cast<size_t>(desc->N) * bias_es, cudaMemcpyHostToDevice, hp.s_in));
+    for (int i = 0; i < nblocks; ++i) {
+        const int64_t r0 = i * rows, r1 = std::min<int64_t>(desc->M, r0 + rows);
+        if (desc->K > 0) {
+            if (desc->layout_a == SG_ROW_MAJOR) {
+                SG_CUDA(cudaMemcpy2DAsync(dA + r0 * desc->lda * es_in, desc->lda * es_in,
+                                          static_cast<const uint8_t*>(A_host) + r0 * desc->lda * es_in, desc->lda * es_in,
+                                          static_cast<size_t>(desc->K) * es_in, static_cast<size_t>(r1 - r0), cudaMemcpyHostToDevice, hp.s_in));
+            } else {
+                SG_CUDA(cudaMemcpy2DAsync(dA + r0 * es_in, desc->lda * es_in, static_cast<const uint8_t*>(A_host) + r0 * es_in,
+                                          desc->lda * es_in, static_cast<size_t>(r1 - r0) * es_in, static_cast<size_t>(desc->K),
+                                          cudaMemcpyHostToDevice, hp.s_in));
+            }
+        }
+        if (desc->beta != 0.0f)
+            SG_CUDA(cudaMemcpy2DAsync(dC + r0 * desc->ldc * es_out, desc->ldc * es_out,
+                                      static_cast<const uint8_t*>(C_host) + r0 * desc->ldc * es_out, desc->ldc * es_out,
+                                      static_cast<size_t>(desc->N) * es_out, static_cast<size_t>(r1 - r0), cudaMemcpyHostToDevice, hp.s_in));
+        SG_CUDA(cudaEventRecord(hp.arrived[i], hp.s_in));
+    }
+    for (int i = 0; i < nblocks; ++i) {
+        const int64_t r0 = i * rows, r1 = std::min<int64_t>(desc->M, r0 + rows);
+        SG_CUDA(cudaStreamWaitEvent(main_stream, hp.arrived[i], 0));
+        sg_gemm_desc_t blk = *desc;
+        blk.M = r1 - r0;
+        const uint8_t* a_blk = dA + (desc->layout_a == SG_ROW_MAJOR ? r0 * desc->lda : r0) * es_in;
+        st = sg_gemm(&blk, a_blk, dB, desc->beta != 0.0f ? dC + r0 * desc->ldc * es_out : nullptr, bias_host ? dBias : nullptr,
+                     dD + r0 * desc->ldd * es_out, main_stream);
+        if (st != SG_OK) return st;
+        SG_CUDA(cudaEventRecord(hp.done[i], main_stream));
+        SG_CUDA(cudaStreamWaitEvent(hp.s_out, hp.done[i], 0));
+        SG_CUDA(cudaMemcpy2DAsync(static_cast<uint8_t*>(D_host) + r0 * desc->ldd * es_out, desc->ldd * es_out,
+                                  dD + r0 * desc->ldd * es_out, desc->ldd * es_out, static_cast<size_t>(desc->N) * es_out,
+                                  static_cast<size_t>(r1 - r0), cudaMemcpyDeviceToHost, hp.s_out));
+    }
+    SG_CUDA(cudaEventRecord(hp.back, hp.s_out));
+    SG_CUDA(cudaStreamWaitEvent(main_stream, hp.back, 0));
+    return SG_OK;
+}
+
 sg_status_t sg_gemm_ex(const sg_gemm_desc_t* desc, const sg_epilogue_ex_t* ex, const void* A, const void* B, const void* C,
                        const void* bias, void* D, void* cuda_stream) {
     return run_dense(desc, 1, 0, 0, 0, 0, 0, A, B, C, bias, D, cuda_stream, "sg_gemm_ex", ex);

@@ -40,7 +40,7 @@ EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_
             "sg_sol_bound", "sg_status_string", "sg_last_error", "sg_poll_status", "sg_set_tuning", "sg_launch_count",
             "sg_last_launch_plan", "sg_set_scratch", "sg_set_tail_mode",
             "sg_last_kernel_clock", "sg_transpose", "sg_set_option", "sg_test_set_status_word",
-            "sg_last_kernel_name"]
+            "sg_last_kernel_name", "sg_gemm_host", "sg_gemm_host_staging_size"]
 OPTIONS = {"epi_warps": 0, "tail_split": 1, "tail_ksplit": 2, "band_m": 3, "general_kernel": 4, "no_pdl": 5, "no_short_a": 6,
            "no_gemv": 7, "gemv_no_mma": 8, "gemv_no_wide": 9, "gemv_rows": 10, "wait_limit_ns": 11, "l2_warm_kblocks": 12, "transpose_plain": 13, "early_donors": 14,
            "two_pass_split_k": 15, "split_k_reduce_warps": 16}
@@ -138,6 +138,10 @@ _lib.sg_set_scratch.argtypes = [_vp, ctypes.c_size_t]
 _lib.sg_last_launch_plan.restype = ctypes.c_int
 _lib.sg_last_launch_plan.argtypes = [ctypes.POINTER(ctypes.c_int32)]
 _lib.sg_last_kernel_name.restype = ctypes.c_char_p
+_lib.sg_gemm_host_staging_size.restype = ctypes.c_int
+_lib.sg_gemm_host_staging_size.argtypes = [ctypes.POINTER(GemmDesc), ctypes.POINTER(ctypes.c_size_t)]
+_lib.sg_gemm_host.restype = ctypes.c_int
+_lib.sg_gemm_host.argtypes = [ctypes.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _i32, _vp]
 _lib.sg_set_option.restype = ctypes.c_int
 _lib.sg_set_option.argtypes = [_i32, _i64]
 _lib.sg_test_set_status_word.restype = ctypes.c_int
@@ -477,60 +481,32 @@ def conv1d_fprop(X: torch.Tensor, Wf: torch.Tensor, *, pad=0, stride=1, dil=1, *
     return y.view(n, y.shape[2], k)
 
 
-_side_streams = {}      # device index -> (copy-in stream, copy-out stream)
+def gemm_host(A_host: torch.Tensor, B_host: torch.Tensor, out_host: torch.Tensor, *, C_host=None, bias_host=None, epi="none",
+              alpha=1.0, beta=0.0, device="cuda", scratch: Optional[dict] = None, stream=None, chunks: int = 4,
+              layout_a: str = "row", layout_b: str = "col") -> torch.Tensor:
+    """``sg_gemm_host``: GEMM for callers whose data lives in (pinned) host memory.
 
-
-def gemm_host(A_host: torch.Tensor, B_host: torch.Tensor, out_host: torch.Tensor, *, bias_host=None, epi="none",
-              alpha=1.0, device="cuda", scratch: Optional[dict] = None, stream=None, chunks: int = 4) -> torch.Tensor:
-    """End-to-end GEMM for callers whose data lives in (pinned) host memory.
-
-    Copies A, B (and bias) to the device, runs ``sg_gemm`` and copies D back into ``out_host``.  The rows of A and D
-    are cut into ``chunks`` blocks: while the copy engine brings in block i+1, the kernel works on block i and the
-    other copy engine takes block i-1 of D back, so the call costs about the larger of the two transfers instead of
-    their sum.  Everything is ordered against ``stream`` (default: the current stream): the call starts after the
-    work already on it and the stream continues only when ``out_host`` is complete.  ``scratch`` may hold
-    preallocated device buffers ("A", "B", "bias", "D"); it is filled on first use.
+    The library copies A, B (C, bias) to a device staging buffer, runs ``sg_gemm`` and copies D back into ``out_host``,
+    pipelined over ``chunks`` row blocks on its own copy streams; everything is ordered against ``stream`` (default: the
+    current stream).  ``scratch`` may hold the staging tensor ("staging") between calls; torch owns that memory.
     """
     scratch = {} if scratch is None else scratch
     dev = torch.device(device)
     if dev.index is None:
         dev = torch.device("cuda", torch.cuda.current_device())
-    main = torch.cuda.current_stream(dev) if stream is None else stream
-    for name, t in (("A", A_host), ("B", B_host), ("bias", bias_host), ("D", out_host)):
-        if t is not None and name not in scratch:
-            scratch[name] = torch.empty(t.shape, dtype=t.dtype, device=dev)
-    if dev.index not in _side_streams:
-        _side_streams[dev.index] = (torch.cuda.Stream(dev), torch.cuda.Stream(dev))
-    s_in, s_out = _side_streams[dev.index]
-    M = A_host.shape[0]
-    rows = max(256, -(-M // max(chunks, 1) // 256) * 256)        # block height: a multiple of the 256-row tile
-    blocks = [(r, min(r + rows, M)) for r in range(0, M, rows)]
-    fork = torch.cuda.Event()
-    fork.record(main)
-    s_in.wait_event(fork)           # the device buffers may still be in use by work enqueued before this call
-    s_out.wait_event(fork)
-    arrived = []
-    with torch.cuda.stream(s_in):
-        scratch["B"].copy_(B_host, non_blocking=True)
-        if bias_host is not None:
-            scratch["bias"].copy_(bias_host, non_blocking=True)
-        for r0, r1 in blocks:
-            scratch["A"][r0:r1].copy_(A_host[r0:r1], non_blocking=True)
-            ev = torch.cuda.Event()
-            ev.record(s_in)
-            arrived.append(ev)
-    for (r0, r1), ev in zip(blocks, arrived):
-        main.wait_event(ev)
-        gemm(scratch["A"][r0:r1], scratch["B"], bias=scratch.get("bias") if bias_host is not None else None,
-             out=scratch["D"][r0:r1], alpha=alpha, epi=epi, stream=main)
-        done = torch.cuda.Event()
-        done.record(main)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(done)
-            out_host[r0:r1].copy_(scratch["D"][r0:r1], non_blocking=True)
-    back = torch.cuda.Event()
-    back.record(s_out)
-    main.wait_event(back)
+    M, N, K = _mnk(A_host, B_host, layout_a, layout_b)
+    desc = _gemm_desc(M, N, K, _ld(A_host), _ld(B_host), _ld(C_host) if C_host is not None else max(N, 1), _ld(out_host),
+                      layout_a, layout_b, out_host.dtype, alpha, beta, epi, in_dtype=A_host.dtype)
+    need = ctypes.c_size_t(0)
+    _check(_lib.sg_gemm_host_staging_size(ctypes.byref(desc), ctypes.byref(need)))
+    st = scratch.get("staging")
+    if st is None or st.numel() < need.value or st.device != dev:
+        st = scratch["staging"] = torch.empty(max(need.value, 256), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        ensure_scratch()
+        s = torch.cuda.current_stream(dev) if stream is None else stream
+        _check(_lib.sg_gemm_host(ctypes.byref(desc), _ptr(A_host), _ptr(B_host), _ptr(C_host), _ptr(bias_host), _ptr(out_host),
+                                 _ptr(st), st.numel(), int(chunks), ctypes.c_void_p(s.cuda_stream)))
     return out_host
 
 

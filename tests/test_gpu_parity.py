@@ -760,3 +760,23 @@ def test_gemm_host_pipelined_copies_match_the_oracle(M, chunks):
         sg.gemm_host(hA, hB, hD, bias_host=hb, epi="relu", scratch=scratch, chunks=chunks)
         torch.cuda.current_stream().synchronize()
         parity.assert_matches(hD, ref, absacc, f"gemm_host M={M} chunks={chunks}")
+
+
+def test_gemm_host_residual_other_layouts_padded_rows_and_pageable_memory():
+    # column-major A and row-major B with padded leading dimensions, a residual C, fp32 output, small integers (exact);
+    # once from pinned and once from pageable host memory; the padding of D_host must stay untouched
+    M, N, K = 700, 136, 72
+    Ast = inputs.small_integers([K, M + 28], 71, 1)                 # A column-major: [K, M] with lda = M + 28
+    Bst = inputs.small_integers([K, N + 8], 71, 2)                  # B row-major:    [K, N] with ldb = N + 8
+    C = inputs.small_integers([M, N + 4], 71, 3, -2, 2).float()
+    bias = inputs.small_integers([N], 71, 4, -3, 3)
+    ref, _ = orc.gemm(Ast[:, :M], Bst[:, :N], C=C[:, :N], bias=bias, alpha=2.0, beta=1.0, layout_a="col", layout_b="row")
+    for pin in (True, False):
+        place = (lambda t: t.pin_memory()) if pin else (lambda t: t.clone())
+        hA, hB, hC, hb = place(Ast), place(Bst), place(C), place(bias)
+        hD = place(torch.full((M, N + 12), float("nan"), dtype=torch.float32))
+        sg.gemm_host(hA[:, :M], hB[:, :N], hD[:, :N], C_host=hC[:, :N], bias_host=hb, alpha=2.0, beta=1.0, layout_a="col",
+                     layout_b="row", chunks=3)
+        torch.cuda.current_stream().synchronize()
+        parity.assert_bit_exact(hD[:, :N], ref, f"gemm_host layouts pinned={pin}")
+        assert bool(torch.isnan(hD[:, N:]).all())

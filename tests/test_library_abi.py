@@ -203,3 +203,18 @@ def test_sol_bound_counts_for_every_operation(sg):
     assert sg.sol_bound("batched", M=8, N=8, K=8, batch_or_groups=3, has_bias=1, **hw)["bytes"] == 3 * 384 + 48
     with pytest.raises(sg.SolgemmError):
         sg.sol_bound("gemm", M=8, N=8, K=8, peak_flops=0.0, peak_bytes_per_s=1.0)
+
+
+def test_gemm_host_rejects_a_missing_or_short_staging_buffer_before_touching_a_device(sg):
+    lib = sg.raw_lib()
+    desc = sg.GemmDesc(512, 64, 64, 0, 1, 64, 64, 64, 64, 0, 0, 1.0, 0.0, 0, 0.0, 0.0, 0)
+    need = ctypes.c_size_t(0)
+    assert lib.sg_gemm_host_staging_size(ctypes.byref(desc), ctypes.byref(need)) == 0
+    assert need.value >= (512 * 64 + 64 * 64 + 512 * 64) * 2
+    host = ctypes.c_void_p(0x1000)
+    st = lib.sg_gemm_host(ctypes.byref(desc), host, host, None, None, host, None, 0, 4, None)
+    assert sg.STATUS_NAMES[st] == "SG_ERR_WORKSPACE"
+    st = lib.sg_gemm_host(ctypes.byref(desc), host, host, None, None, host, ctypes.c_void_p(0x10000), need.value - 1, 4, None)
+    assert sg.STATUS_NAMES[st] == "SG_ERR_WORKSPACE" and str(need.value) in lib.sg_last_error().decode()
+    st = lib.sg_gemm_host(ctypes.byref(desc), None, host, None, None, host, ctypes.c_void_p(0x10000), need.value, 4, None)
+    assert sg.STATUS_NAMES[st] == "SG_ERR_NULL_POINTER"
