@@ -780,3 +780,31 @@ def test_gemm_host_residual_other_layouts_padded_rows_and_pageable_memory():
         torch.cuda.current_stream().synchronize()
         parity.assert_bit_exact(hD[:, :N], ref, f"gemm_host layouts pinned={pin}")
         assert bool(torch.isnan(hD[:, N:]).all())
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.float8_e4m3fn, torch.float8_e5m2, torch.int8, torch.float32])
+def test_two_pass_split_k_other_input_types_bit_exact(dtype):
+    # the K ranges of a skinny problem through the everything-in-one kernel variant: fp16, fp8, int8 (integer accumulators,
+    # converted before they are parked) and fp32-as-tf32 operands; small integers, exact in every type involved
+    M, N, K = 200, 264, 8192
+    A = (inputs.small_integers([M, K], 393, 1) * (inputs.small_integers([M, K], 394, 1, 0, 15) == 0).to(torch.bfloat16)).float().to(dtype)
+    B = inputs.small_integers([N, K], 393, 2).float().to(dtype)
+    bias = inputs.small_integers([N], 393, 4, -3, 3).to(orc.bias_dtype_for(dtype))
+    ref, _ = orc.gemm(A, B, bias=bias, epi="relu")
+    assert float(ref.abs().max()) <= 256
+    for out_dtype in (torch.bfloat16, torch.float32):
+        D = sg.gemm(A.to(DEV), B.to(DEV), bias=bias.to(DEV), epi="relu", out_dtype=out_dtype)
+        assert sg.last_launch_plan()["tail_split"] < -1, sg.last_launch_plan()
+        parity.assert_bit_exact(D, ref, f"two-pass {dtype} -> {out_dtype}")
+
+
+def test_two_pass_split_k_skinny_convolution():
+    # a convolution with few output pixels and many input channels: 128 pixels x 136 filters, K = 3 * 3 * 1024
+    X = inputs.small_integers([2, 8, 8, 1024], 403, 6, -1, 1) * (inputs.small_integers([2, 8, 8, 1024], 404, 6, 0, 7) == 0).to(torch.bfloat16)
+    Wf = inputs.small_integers([136, 3, 3, 1024], 403, 7, -1, 1)
+    bias = inputs.small_integers([136], 403, 4, -2, 2)
+    ref, _ = orc.conv2d_fprop(X, Wf, pad=(1, 1), bias=bias, epi="relu")
+    assert float(ref.abs().max()) <= 256
+    Y = sg.conv2d_fprop(X.to(DEV), Wf.to(DEV), pad=(1, 1), bias=bias.to(DEV), epi="relu")
+    assert sg.last_launch_plan()["tail_split"] < -1, sg.last_launch_plan()
+    parity.assert_bit_exact(Y, ref, "two-pass conv")
