@@ -559,7 +559,8 @@ def profile_config(args) -> None:
     C = inputs.CONFIGS
     name = {"c3": "c3_batched_128x256x256x512_gelu", "c4": "c4_conv_32x56x56x256_k256_3x3_bias_relu",
             "c5": "c5_grouped_16xMx4096x4096_silu", "gemv1": "matrix_vector_8192x8192_1_vector",
-            "gemv8": "matrix_vector_8192x8192_8_vectors"}[args.profile_config]
+            "gemv8": "matrix_vector_8192x8192_8_vectors", "transpose": "transpose_8x4096x4096_bf16_to_bf16",
+            "splitk": "gemm_256x256x32768_two_pass_split_k"}[args.profile_config]
     c = C.get(name)
     if args.profile_config in ("gemv1", "gemv8"):
         nvec = 1 if args.profile_config == "gemv1" else 8
@@ -568,6 +569,17 @@ def profile_config(args) -> None:
         x = torch.randn(nvec, 8192, device=dev).to(torch.bfloat16)
         outs = [torch.empty(8192, nvec, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
         step = lambda i: sg.gemm(Ws[i % sets], x, out=outs[i % sets])
+    elif args.profile_config == "transpose":
+        sets = 3
+        xs = [torch.randn(8, 4096, 4096, device=dev).to(torch.bfloat16) for _ in range(sets)]
+        ys = [torch.empty(8, 4096, 4096, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        step = lambda i: sg.transpose(xs[i % sets], out=ys[i % sets])
+    elif args.profile_config == "splitk":
+        sets = 8
+        As = [torch.randn(256, 32768, device=dev).to(torch.bfloat16) for _ in range(sets)]
+        Bs = [torch.randn(256, 32768, device=dev).to(torch.bfloat16) for _ in range(sets)]
+        outs = [torch.empty(256, 256, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        step = lambda i: sg.gemm(As[i % sets], Bs[i % sets], out=outs[i % sets])
     elif args.profile_config == "c3":
         sets = 4
         data = [inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"], seed=i, device=dev, batch=c["batch"]) for i in range(sets)]
@@ -603,7 +615,7 @@ def profile_config(args) -> None:
     torch.cuda.profiler.stop()
     sg.poll_status()
     print(json.dumps({"profile_config": name, "launches": args.steps, "us_per_launch_single_cold": times,
-                      "plan": sg.last_launch_plan()}), flush=True)
+                      "plan": sg.last_launch_plan(), "kernel": sg.last_kernel_name()}), flush=True)
 
 
 def spread_rows(M: int, count: int, tile_m: int = 256):
@@ -848,7 +860,7 @@ def main() -> None:
     ap.add_argument("--widened", action="store_true",
                     help="also time the rows built beyond the five configurations (epilogue chain, dtypes, layouts, "
                          "skinny shapes, transpose, conv gradients; N=1 only)")
-    ap.add_argument("--profile-config", choices=["c3", "c4", "c5", "gemv1", "gemv8"], default=None,
+    ap.add_argument("--profile-config", choices=["c3", "c4", "c5", "gemv1", "gemv8", "transpose", "splitk"], default=None,
                     help="only run a few launches of that configuration inside the profiler bracket (for ncu)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures of the timed kernel)")

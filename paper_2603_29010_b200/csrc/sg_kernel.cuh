@@ -809,6 +809,9 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (!ok) break;
                 umma_commit<kPair>(tfull_bar(acc));
                 if (t == first_tile) SG_STAMP(5);
+#ifdef SG_DEBUG_STAMPS
+                if (iter <= 8) SG_STAMP(21 + iter);      // last MMA of this CTA's iter-th item issued
+#endif
             }
             SG_STAMP(6);
             if (!ok) {
@@ -985,7 +988,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 if (ksplit_tile && owned(c) != (pass == 1)) continue;
                 float v[CH];
 #ifdef SG_DEBUG_STAMPS
-                const bool stamp_chunk = warp == 2 && lane == 0 && t + tile_step >= p.num_tiles && c < 4;
+                const bool stamp_chunk = warp == 2 && lane == 0 && t + tile_step >= p.num_tiles && c < 2;
                 if (stamp_chunk) SG_STAMP(16 + 3 * c);
 #endif
                 if (has_k) {
