@@ -292,9 +292,10 @@ sg_status_t sg_conv2d_fprop_ex(const sg_conv2d_desc_t* desc, const sg_epilogue_e
  * stage with fused dtype conversion that the DSL's pipeline(transpose(...), kernel, transpose(...)) places
  * around a kernel (Section 3 "Multi-stage pipelines"; Appendix A.1 transpose_op: NCL <-> NLC, and
  * NCHW <-> NHWC "implemented by flattening HW": batch = N, rows = C, cols = H*W or the reverse).
- *   in   device, in_dtype (bf16 or fp32; fp16 is not implemented here), [batch][rows][cols], row stride ld_in, batch stride stride_in (elements)
- *   out  device, out_dtype (bf16 or fp32), [batch][cols][rows], row stride ld_out, batch stride stride_out
- *   fp32 -> bf16 rounds to nearest even; bf16 -> fp32 is exact.  in and out must not overlap.
+ *   in   device, in_dtype (bf16, fp16 or fp32), [batch][rows][cols], row stride ld_in, batch stride stride_in (elements)
+ *   out  device, out_dtype (bf16, fp16 or fp32), [batch][cols][rows], row stride ld_out, batch stride stride_out
+ *   A conversion to a narrower significand (fp32 -> bf16 / fp16, bf16 <-> fp16) rounds to nearest even; widening is
+ *   exact.  in and out must not overlap.
  * Base pointers 16-byte aligned, ld and strides multiples of 16 bytes, ld_in >= cols, ld_out >= rows.
  * When rows and cols both span multiples of 16 bytes (in the output resp. input type) the stage runs as a persistent
  * kernel that streams tiles through shared memory with TMA loads and stores; other extents take a plain-store kernel

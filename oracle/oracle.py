@@ -409,7 +409,7 @@ def conv2d_points(X, Wf, ppix: Sequence[int], pk: Sequence[int], *, pad=(0, 0), 
 def transpose(x: torch.Tensor, out_dtype: torch.dtype) -> torch.Tensor:
     """out[b, c, r] = convert(x[b, r, c]) as fp64 values of the converted result; x is [batch, rows, cols]."""
     if x.device.type != "cpu" or x.dim() != 3 or x.dtype not in _DTYPES or (x.shape[2] > 1 and x.stride(2) != 1):
-        raise ValueError("x: want a CPU [batch, rows, cols] bf16 or fp32 tensor with inner stride 1")
+        raise ValueError("x: want a CPU [batch, rows, cols] bf16, fp16 or fp32 tensor with inner stride 1")
     batch, rows, cols = x.shape
     out = torch.empty((batch, cols, rows), dtype=torch.float64)
     rc = lib().orc_transpose(batch, rows, cols, _ptr(x), _DTYPES[x.dtype], x.stride(1) if rows > 1 else max(cols, 1),

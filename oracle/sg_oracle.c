@@ -469,8 +469,8 @@ int orc_conv2d_wgrad(const int64_t* dims, const void* dY, const void* X, const v
 
 /* -------------------------------------------------------------------------------------------
  * Layout transpose with dtype conversion (the DSL's transpose(ref, L1, L2[, dt1, dt2]) stage, Appendix A.1):
- *   out[b][c][r] = convert(in[b][r][c]).  bf16 -> fp32 is exact; fp32 -> bf16 rounds to nearest, ties to even
- *   (the 16 discarded bits decide; a NaN stays a NaN).  The result is returned as fp64 holding the converted value.
+ *   out[b][c][r] = convert(in[b][r][c]).  bf16 / fp16 -> fp32 is exact; a conversion to bf16 or fp16 rounds the (exactly
+ *   widened) value to nearest, ties to even; a NaN stays a NaN.  The result is returned as fp64 holding the converted value.
  * ----------------------------------------------------------------------------------------- */
 static double round_f32_to_bf16(float f) {
     uint32_t u;
@@ -487,6 +487,24 @@ static double round_f32_to_bf16(float f) {
     return (double)r;
 }
 
+/* fp32 -> fp16 (IEEE binary16: 5 exponent bits, 10 fraction bits), round to nearest, ties to even, written out
+ * from the definition: values of 65520 and above go to infinity, values below 2^-14 land on the subnormal grid of
+ * spacing 2^-24, a NaN stays a NaN.  Every bf16 and every fp32 input is a binary32 value, so this one rounding
+ * covers bf16 -> fp16 as well. */
+static double round_f32_to_f16(float f) {
+    if (f != f) return (double)f;                               /* NaN */
+    double x = (double)f, a = fabs(x), sign = (x < 0.0 || (x == 0.0 && 1.0 / x < 0.0)) ? -1.0 : 1.0;
+    if (a == 0.0) return x;
+    if (a >= 65520.0) return sign * INFINITY;                   /* the midpoint between 65504 and 2^16 rounds up (to even) */
+    int e;
+    (void)frexp(a, &e);                                         /* a = m 2^e, 0.5 <= m < 1: the leading bit has weight 2^(e-1) */
+    int ulp_exp = (e - 1 < -14 ? -14 : e - 1) - 10;             /* spacing of fp16 values around a */
+    double q = ldexp(a, -ulp_exp);                              /* a in units of that spacing: below 2^11, exact in fp64 */
+    double fl = floor(q), frac = q - fl;
+    if (frac > 0.5 || (frac == 0.5 && fmod(fl, 2.0) == 1.0)) fl += 1.0;
+    return sign * ldexp(fl, ulp_exp);
+}
+
 int orc_transpose(int64_t batch, int64_t rows, int64_t cols, const void* in, int in_dtype, int64_t ld_in,
                   int64_t stride_in, int out_dtype, double* out) {
     if (batch < 0 || rows < 0 || cols < 0) return 1;
@@ -494,7 +512,9 @@ int orc_transpose(int64_t batch, int64_t rows, int64_t cols, const void* in, int
         for (int64_t r = 0; r < rows; ++r)
             for (int64_t c = 0; c < cols; ++c) {
                 double v = load_as_f64(in, in_dtype, b * stride_in + r * ld_in + c);
-                if (out_dtype == ORC_BF16 && in_dtype == ORC_F32) v = round_f32_to_bf16((float)v);
+                /* every 16-bit input value is exact in fp32; only a conversion to a narrower significand rounds */
+                if (out_dtype == ORC_BF16 && in_dtype != ORC_BF16) v = round_f32_to_bf16((float)v);
+                if (out_dtype == ORC_F16 && in_dtype != ORC_F16) v = round_f32_to_f16((float)v);
                 out[(b * cols + c) * rows + r] = v;
             }
     return 0;

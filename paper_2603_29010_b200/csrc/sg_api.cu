@@ -103,6 +103,30 @@ KernelEntry kernel_for(int bn, bool pair, int out, int epi_warps, int variant = 
     }
 }
 
+// transpose kernels by (input, output) type: 0 fp32, 1 bf16, 2 fp16
+struct TransposeEntry {
+    void (*tma)(const TransposeTmaParams);
+    void (*plain)(const TransposeParams);
+    int smem, ctas_per_sm;
+    const char* in_name;
+    const char* out_name;
+};
+template <typename TI, typename TO>
+TransposeEntry transpose_entry_for(const char* in_name, const char* out_name) {
+    return TransposeEntry{transpose_tma_kernel<TI, TO>, transpose_kernel<TI, TO>, TransposeCfg<TI, TO>::SMEM_BYTES,
+                          TransposeCfg<TI, TO>::CTAS_PER_SM, in_name, out_name};
+}
+TransposeEntry transpose_entry(int ti, int to) {
+#define SG_TR_ROW(TI, NI)                                                                                   \
+    return to == 0 ? transpose_entry_for<TI, float>(NI, "float")                                            \
+                   : (to == 1 ? transpose_entry_for<TI, __nv_bfloat16>(NI, "__nv_bfloat16") : transpose_entry_for<TI, __half>(NI, "__half"));
+    if (ti == 0) { SG_TR_ROW(float, "float") }
+    if (ti == 1) { SG_TR_ROW(__nv_bfloat16, "__nv_bfloat16") }
+    SG_TR_ROW(__half, "__half")
+#undef SG_TR_ROW
+}
+inline int transpose_type_index(int32_t dt) { return dt == SG_F32 ? 0 : (dt == SG_BF16 ? 1 : 2); }
+
 sg_status_t device_state(DeviceState** out) {
     int dev = 0;
     SG_CUDA(cudaGetDevice(&dev));
@@ -155,17 +179,12 @@ sg_status_t device_state(DeviceState** out) {
                                 if (e != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(shared memory)", cudaGetErrorString(e));
                             }
             if (d.init_status == SG_OK) {
-                cudaError_t e2 = cudaFuncSetAttribute(transpose_tma_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                      TransposeCfg<float, float>::SMEM_BYTES);
-                if (e2 == cudaSuccess)
-                    e2 = cudaFuncSetAttribute(transpose_tma_kernel<float, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              TransposeCfg<float, __nv_bfloat16>::SMEM_BYTES);
-                if (e2 == cudaSuccess)
-                    e2 = cudaFuncSetAttribute(transpose_tma_kernel<__nv_bfloat16, float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              TransposeCfg<__nv_bfloat16, float>::SMEM_BYTES);
-                if (e2 == cudaSuccess)
-                    e2 = cudaFuncSetAttribute(transpose_tma_kernel<__nv_bfloat16, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              TransposeCfg<__nv_bfloat16, __nv_bfloat16>::SMEM_BYTES);
+                cudaError_t e2 = cudaSuccess;
+                for (int ti = 0; ti < 3 && e2 == cudaSuccess; ++ti)
+                    for (int to = 0; to < 3 && e2 == cudaSuccess; ++to) {
+                        const TransposeEntry te = transpose_entry(ti, to);
+                        e2 = cudaFuncSetAttribute(te.tma, cudaFuncAttributeMaxDynamicSharedMemorySize, te.smem);
+                    }
                 if (e2 != cudaSuccess) bad(SG_ERR_CUDA, "cudaFuncSetAttribute(transpose shared memory)", cudaGetErrorString(e2));
             }
             if (d.init_status == SG_OK) {
@@ -2041,8 +2060,10 @@ extern "C" {
 sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* out, void* cuda_stream) {
     if (!desc) return fail(SG_ERR_NULL_POINTER, "desc is NULL");
     if (desc->reserved != 0 || desc->reserved2 != 0) return fail(SG_ERR_INVALID_ARG, "reserved fields must be 0");
-    if ((desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F32) || (desc->out_dtype != SG_BF16 && desc->out_dtype != SG_F32))
-        return fail(SG_ERR_INVALID_ARG, "sg_transpose: dtypes must be SG_BF16 or SG_F32");
+    if ((desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F32 && desc->in_dtype != SG_F16) ||
+        (desc->out_dtype != SG_BF16 && desc->out_dtype != SG_F32 && desc->out_dtype != SG_F16))
+        return fail(SG_ERR_INVALID_ARG, "sg_transpose: dtypes must be SG_BF16, SG_F16 or SG_F32");
+    const TransposeEntry te = transpose_entry(transpose_type_index(desc->in_dtype), transpose_type_index(desc->out_dtype));
     if (desc->batch < 0 || desc->rows < 0 || desc->cols < 0) return fail(SG_ERR_INVALID_ARG, "sg_transpose: extents must be >= 0");
     if (desc->batch == 0 || desc->rows == 0 || desc->cols == 0) return SG_OK;
     const int es_in = desc->in_dtype == SG_F32 ? 4 : 2, es_out = desc->out_dtype == SG_F32 ? 4 : 2;
@@ -2072,8 +2093,10 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
         if (tr * tc * desc->batch > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_transpose: too many tiles");
         TransposeTmaParams tp;
         memset(&tp, 0, sizeof tp);
-        const CUtensorMapDataType dt_in = desc->in_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-        const CUtensorMapDataType dt_out = desc->out_dtype == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+        auto map_type = [](int32_t dt) {
+            return dt == SG_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : (dt == SG_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+        };
+        const CUtensorMapDataType dt_in = map_type(desc->in_dtype), dt_out = map_type(desc->out_dtype);
         st = make_tiled_map(&tp.tm_in, dt_in, es_in, in, desc->cols, desc->rows, desc->batch, desc->ld_in, desc->stride_in, TC, TR,
                             "transpose input", CU_TENSOR_MAP_SWIZZLE_NONE);
         if (st != SG_OK) return st;
@@ -2087,8 +2110,7 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
         const int64_t limit = opt(SG_OPT_WAIT_LIMIT_NS);
         tp.timeout_ns = limit > 0 ? static_cast<uint64_t>(limit) : kWaitLimitNs;
         cudaLaunchConfig_t cfg = {};
-        const int64_t slots = static_cast<int64_t>(d->sm_count) *
-                              (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32 ? TransposeCfg<float, float>::CTAS_PER_SM : 1);
+        const int64_t slots = static_cast<int64_t>(d->sm_count) * te.ctas_per_sm;
         cfg.gridDim = dim3(static_cast<unsigned>(tp.num_tiles < slots ? tp.num_tiles : slots));
         cfg.blockDim = dim3(288);
         cfg.stream = stream;
@@ -2097,24 +2119,11 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = opt(SG_OPT_NO_PDL) > 0 ? 0 : 1;
-        cudaError_t e;
-        if (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32) {
-            cfg.dynamicSmemBytes = TransposeCfg<float, float>::SMEM_BYTES;
-            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<float, float>, tp);
-        } else if (desc->in_dtype == SG_F32) {
-            cfg.dynamicSmemBytes = TransposeCfg<float, __nv_bfloat16>::SMEM_BYTES;
-            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<float, __nv_bfloat16>, tp);
-        } else if (desc->out_dtype == SG_F32) {
-            cfg.dynamicSmemBytes = TransposeCfg<__nv_bfloat16, float>::SMEM_BYTES;
-            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<__nv_bfloat16, float>, tp);
-        } else {
-            cfg.dynamicSmemBytes = TransposeCfg<__nv_bfloat16, __nv_bfloat16>::SMEM_BYTES;
-            e = cudaLaunchKernelEx(&cfg, transpose_tma_kernel<__nv_bfloat16, __nv_bfloat16>, tp);
-        }
+        cfg.dynamicSmemBytes = te.smem;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, te.tma, tp);
         if (e != cudaSuccess) return fail(SG_ERR_CUDA, "transpose kernel launch: %s", cudaGetErrorString(e));
         g_launches.fetch_add(1);
-        note_kernel("sg::transpose_tma_kernel<%s, %s>", desc->in_dtype == SG_F32 ? "float" : "__nv_bfloat16",
-                    desc->out_dtype == SG_F32 ? "float" : "__nv_bfloat16");
+        note_kernel("sg::transpose_tma_kernel<%s, %s>", te.in_name, te.out_name);
         return SG_OK;
     }
     TransposeParams tp;
@@ -2125,14 +2134,10 @@ sg_status_t sg_transpose(const sg_transpose_desc_t* desc, const void* in, void* 
     tp.stride_in = desc->stride_in; tp.stride_out = desc->stride_out;
     tp.tiles_r = static_cast<int32_t>(tiles_r); tp.tiles_c = static_cast<int32_t>(tiles_c);
     const dim3 grid(static_cast<unsigned>(tiles_r * tiles_c * desc->batch));
-    if (desc->in_dtype == SG_F32 && desc->out_dtype == SG_F32) transpose_kernel<float, float><<<grid, 256, 0, stream>>>(tp);
-    else if (desc->in_dtype == SG_F32) transpose_kernel<float, __nv_bfloat16><<<grid, 256, 0, stream>>>(tp);
-    else if (desc->out_dtype == SG_F32) transpose_kernel<__nv_bfloat16, float><<<grid, 256, 0, stream>>>(tp);
-    else transpose_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, stream>>>(tp);
+    te.plain<<<grid, 256, 0, stream>>>(tp);
     SG_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
-    note_kernel("sg::transpose_kernel<%s, %s>", desc->in_dtype == SG_F32 ? "float" : "__nv_bfloat16",
-                desc->out_dtype == SG_F32 ? "float" : "__nv_bfloat16");
+    note_kernel("sg::transpose_kernel<%s, %s>", te.in_name, te.out_name);
     return SG_OK;
 }
 

@@ -580,8 +580,8 @@ def test_conv_delta_filter_reproduces_input_on_gpu():
 
 # ---------------------------------------------------------------------------------------- transpose stage
 
-@pytest.mark.parametrize("in_dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("in_dtype", [torch.float32, torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16, torch.float16])
 @pytest.mark.parametrize("shape", [(1, 64, 64), (3, 100, 72), (2, 37, 200), (4, 256, 196), (1, 1, 8), (2, 129, 4)])
 def test_transpose_with_dtype_conversion_bit_exact(shape, in_dtype, out_dtype):
     batch, rows, cols = shape
@@ -598,8 +598,8 @@ def test_transpose_with_dtype_conversion_bit_exact(shape, in_dtype, out_dtype):
         assert torch.equal(sg.transpose(x.to(DEV), out_dtype=out_dtype).cpu(), x.permute(0, 2, 1).to(out_dtype))
 
 
-@pytest.mark.parametrize("in_dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("in_dtype", [torch.float32, torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16, torch.float16])
 def test_transpose_many_tiles_per_cta_and_both_kernels(in_dtype, out_dtype):
     # Far more tiles than SMs x ring stages: every CTA of the persistent TMA kernel wraps its stage ring and reuses both
     # output tiles several times; rows and columns end inside a tile (clipped loads and stores).

@@ -396,6 +396,35 @@ def test_transpose_hand_cases_and_rounding_ties():
     assert math.isnan(float(nan))
 
 
+def test_transpose_fp16_conversions_hand_cases_all_codes_and_library():
+    # hand cases of fp32 -> fp16 (11 significant bits, ties to even, subnormal grid 2^-24, overflow at 65520)
+    cases = torch.tensor([[[1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 1.0 + 2.0 ** -11 + 2.0 ** -20, -(1.0 + 2.0 ** -11),
+                            65519.99, 65520.0, 65504.0, 2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0001, 3 * 2.0 ** -25,
+                            2.0 ** -14 - 2.0 ** -25, 0.0]]], dtype=torch.float32)
+    got = orc.transpose(cases, torch.float16).view(-1).tolist()
+    assert got[:4] == [1.0, 1.0 + 2.0 ** -9, 1.0 + 2.0 ** -10, -1.0]
+    assert got[4] == 65504.0 and got[5] == float("inf") and got[6] == 65504.0
+    assert got[7] == 2.0 ** -24 and got[8] == 0.0 and got[9] == 2.0 ** -24 and got[10] == 2.0 ** -23       # ties to even on the subnormal grid
+    assert got[11] == 2.0 ** -14 and got[12] == 0.0
+    assert math.isnan(float(orc.transpose(torch.tensor([[[float("nan")]]]), torch.float16)))
+    # every fp16 code: widening is exact, so fp16 -> fp32 -> fp16 must give the code's own value back
+    codes = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.float16).view(1, 256, 256)
+    finite = torch.isfinite(codes.float())
+    widened = orc.transpose(codes, torch.float32)                       # [1, 256, 256] transposed
+    assert torch.equal(widened.permute(0, 2, 1)[finite], codes.double()[finite])
+    back = orc.transpose(codes.float(), torch.float16)
+    assert torch.equal(back.permute(0, 2, 1)[finite], codes.double()[finite])
+    # every bf16 code through bf16 -> fp16 and every fp16 code through fp16 -> bf16 against torch's casts (an unrelated
+    # library routine), and random fp32 values through fp32 -> fp16
+    bcodes = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.bfloat16).view(1, 256, 256)
+    bfin = torch.isfinite(bcodes.float())
+    assert torch.equal(orc.transpose(bcodes, torch.float16).permute(0, 2, 1)[bfin], bcodes.to(torch.float16).double()[bfin])
+    assert torch.equal(orc.transpose(codes, torch.bfloat16).permute(0, 2, 1)[finite], codes.to(torch.bfloat16).double()[finite])
+    g = torch.Generator().manual_seed(5)
+    x = torch.randn(2, 64, 48, generator=g) * torch.tensor([1e-7, 1e-3, 1.0, 300.0, 7e4, 1e-5]).repeat(8)
+    assert torch.equal(orc.transpose(x, torch.float16), x.permute(0, 2, 1).to(torch.float16).double())
+
+
 def test_transpose_matches_torch_permute_and_cast():
     x32 = inputs.normal([3, 37, 29], 21, 1).float() * 1.2345 + torch.rand(3, 37, 29, generator=torch.Generator().manual_seed(1)) * 1e-3
     xbf = inputs.uniform([3, 37, 29], 21, 2)
