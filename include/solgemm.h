@@ -89,7 +89,8 @@ typedef enum {
  *   b(k,j) = B[k*ldb + j] (row-major) or B[j*ldb + k] (column-major)
  *   C and D are row-major with leading dimensions ldc, ldd.  All ld* are in ELEMENTS.
  *   All four A/B layout pairs are implemented; the K-contiguous pair (A row-major, B column-major) is the
- *   tuned one.  (sg_grouped_gemm accepts a row-major A only: SG_ERR_UNSUPPORTED otherwise.)
+ *   tuned one.  (sg_grouped_gemm with a column-major A: every A_g is stored [K][M_g] with the one leading dimension
+ *   lda >= max M_g.)
  * Enum-valued fields are int32_t so that the layout is the same from C, C++ and ctypes.
  */
 typedef struct sg_gemm_desc {

@@ -287,8 +287,6 @@ sg_status_t check_gemm_desc(const sg_gemm_desc_t* d, bool grouped, Checked* c) {
         return fail(SG_ERR_UNSUPPORTED, "extents above 2^31-1 are not supported");
     if (d->layout_a != SG_ROW_MAJOR && d->layout_a != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_a %d is not a sg_layout_t", d->layout_a);
     if (d->layout_b != SG_ROW_MAJOR && d->layout_b != SG_COL_MAJOR) return fail(SG_ERR_INVALID_ARG, "layout_b %d is not a sg_layout_t", d->layout_b);
-    if (grouped && d->layout_a == SG_COL_MAJOR)
-        return fail(SG_ERR_UNSUPPORTED, "sg_grouped_gemm: a column-major A (one leading dimension for groups of different M) is not implemented");
     const int64_t M = grouped ? 1 : d->M;
     // leading dimension >= the contiguous extent: K for a K-contiguous operand, M (resp. N) otherwise
     const int64_t a_inner = d->layout_a == SG_ROW_MAJOR ? d->K : M;
@@ -1486,8 +1484,15 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
         tiles += ((rows[g] + tile_m - 1) / tile_m) * tiles_n;
         const uint32_t b_box = static_cast<uint32_t>(s.pair ? s.bn / 2 : s.bn);
         if (common->K > 0) {
-            st = make_tiled_map(&maps[4 * g], c.tm_in, c.esize_in, A_ptrs_host[g], common->K, rows[g], 1,
-                                common->lda, 0, c.bk, 128, "A_g");
+            if (common->layout_a == SG_COL_MAJOR) {
+                // A_g stored [K][M_g] with the common leading dimension: 64 x 64 boxes, consumed M-contiguous
+                if (common->lda < rows[g]) return fail(SG_ERR_INVALID_ARG, "sg_grouped_gemm: lda %lld is smaller than M[%d] = %lld",
+                                                       (long long)common->lda, g, (long long)rows[g]);
+                st = make_tiled_map(&maps[4 * g], c.tm_in, c.esize_in, A_ptrs_host[g], rows[g], common->K, 1, common->lda, 0, 64, 64, "A_g");
+            } else {
+                st = make_tiled_map(&maps[4 * g], c.tm_in, c.esize_in, A_ptrs_host[g], common->K, rows[g], 1,
+                                    common->lda, 0, c.bk, 128, "A_g");
+            }
             if (st != SG_OK) return st;
             if (common->layout_b == SG_ROW_MAJOR) {
                 st = make_tiled_map(&maps[4 * g + 1], c.tm_in, c.esize_in, B_ptrs_host[g], common->N, common->K, 1,
@@ -1514,6 +1519,7 @@ sg_status_t sg_grouped_gemm(const sg_gemm_desc_t* common, int32_t groups, const 
 
     uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
     p.mode = MODE_GROUPED;
+    p.a_mn_major = common->layout_a == SG_COL_MAJOR ? 1 : 0;
     p.b_mn_major = common->layout_b == SG_ROW_MAJOR ? 1 : 0;
     p.gmaps = reinterpret_cast<const CUtensorMap*>(ws + L.off_maps);
     p.g_tile_start = reinterpret_cast<const int32_t*>(ws + L.off_tile_start);

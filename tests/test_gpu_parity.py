@@ -121,6 +121,14 @@ def test_other_layouts_with_padded_leading_dimensions_batched_and_grouped():
     outs = sg.grouped_gemm([a.to(DEV) for a in As], [b.to(DEV) for b in Bs], layout_a="row", layout_b="row")
     for g in range(len(Ms)):
         parity.assert_bit_exact(outs[g], refs[g], f"grouped row/row group {g}")
+    # grouped: column-major A (every A_g stored [K, M_g] with one common leading dimension), both B layouts
+    lda = 264
+    Acs = [inputs.small_integers([K, lda], 141 + g, 1) for g in range(len(Ms))]
+    for lb, Bg in (("row", Bs), ("col", [b.t().contiguous() for b in Bs])):
+        refs, _ = orc.grouped_gemm([a[:, :m] for a, m in zip(Acs, Ms)], Bg, layout_a="col", layout_b=lb)
+        outs = sg.grouped_gemm([a.to(DEV)[:, :m] for a, m in zip(Acs, Ms)], [b.to(DEV) for b in Bg], layout_a="col", layout_b=lb)
+        for g in range(len(Ms)):
+            parity.assert_bit_exact(outs[g], refs[g], f"grouped col/{lb} group {g}")
 
 
 @pytest.mark.parametrize("pair", [0, 1])
