@@ -138,6 +138,25 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
         return *reinterpret_cast<const uint32_t*>(&h);
     }
 }
+// The same conversion with the ReLU folded in (negative values and -0 become +0): one instruction for both.
+template <bool kF16>
+__device__ __forceinline__ uint32_t pack2_relu(float lo, float hi) {
+    uint32_t w;
+    if constexpr (kF16) asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(hi), "f"(lo));
+    return w;
+}
+// v0 += low half, v1 += high half of a packed pair of 16-bit values: the mixed-precision add widens the 16-bit operand
+// exactly, so the sums are those of unpack2 followed by two fp32 adds, without the two unpacking instructions.
+template <bool kF16>
+__device__ __forceinline__ void add_pair(uint32_t w, float& v0, float& v1) {
+    if constexpr (kF16)
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; add.rn.f32.f16 %0, lo, %0; add.rn.f32.f16 %1, hi, %1; }"
+            : "+f"(v0), "+f"(v1) : "r"(w));
+    else
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; add.rn.f32.bf16 %0, lo, %0; add.rn.f32.bf16 %1, hi, %1; }"
+            : "+f"(v0), "+f"(v1) : "r"(w));
+}
 __device__ __forceinline__ float half_bits_to_float(uint16_t b, bool f16) {
     return f16 ? __half2float(__ushort_as_half(b)) : __uint_as_float(static_cast<uint32_t>(b) << 16);
 }
@@ -1178,10 +1197,16 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
 #pragma unroll
                     for (int i = 0; i < CH; i += 4) {
                         const uint2 b2 = *reinterpret_cast<const uint2*>(bias_w + (c / kStep) * CH + i);   // 4 bf16, broadcast read
-                        float b0, b1, b2f, b3;
-                        if (in_f16) { unpack2<true>(b2.x, b0, b1); unpack2<true>(b2.y, b2f, b3); }
-                        else { unpack2<false>(b2.x, b0, b1); unpack2<false>(b2.y, b2f, b3); }
-                        v[i] += b0; v[i + 1] += b1; v[i + 2] += b2f; v[i + 3] += b3;
+                        if constexpr (kEpiWarps == 4) {
+                            // (the instantiations of long K loops; in the others the shorter code measured slower)
+                            if (in_f16) { add_pair<true>(b2.x, v[i], v[i + 1]); add_pair<true>(b2.y, v[i + 2], v[i + 3]); }
+                            else { add_pair<false>(b2.x, v[i], v[i + 1]); add_pair<false>(b2.y, v[i + 2], v[i + 3]); }
+                        } else {
+                            float b0, b1, b2f, b3;
+                            if (in_f16) { unpack2<true>(b2.x, b0, b1); unpack2<true>(b2.y, b2f, b3); }
+                            else { unpack2<false>(b2.x, b0, b1); unpack2<false>(b2.y, b2f, b3); }
+                            v[i] += b0; v[i + 1] += b1; v[i + 2] += b2f; v[i + 3] += b3;
+                        }
                     }
                 }
                 if (ex_any) {
@@ -1217,7 +1242,14 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                         }
                     }
                 }
-                if (epi >= EPI_RELU) apply_act_chunk<kOut == 0, CH>(v, epi, p.epi_arg0, p.epi_arg1);
+                // A plain ReLU in front of a 16-bit output that goes out through the staging block is folded into the
+                // conversion below (one instruction per pair instead of two half-rate max operations and one).
+                constexpr int kElemsPer16B = kOutF32 ? 4 : 8;
+                const bool plain_store = d_remap || (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0);
+                // (Only in the four-epilogue-warp instantiations, the ones long K loops run in: the second copy of the
+                // staging loop lengthens the code a short launch has to fetch once per SM -- 256^3 3.6 -> 3.8 us.)
+                const bool relu_in_cvt = !kOutF32 && kEpiWarps == 4 && epi == EPI_RELU && !ex_any && !plain_store;
+                if (epi >= EPI_RELU && !relu_in_cvt) apply_act_chunk<kOut == 0, CH>(v, epi, p.epi_arg0, p.epi_arg1);
                 if (ex_any) {
                     if (p.post_scale != 1.0f) {
                         const float ps = p.post_scale;
@@ -1262,8 +1294,7 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                 // A TMA store clips at 16-byte granularity along the row.  When N is not a multiple of 16 bytes the
                 // last, partial chunk is therefore written with plain stores so nothing beyond column N changes; a
                 // strided data gradient, whose rows are scattered over the image, is always stored this way.
-                constexpr int kElemsPer16B = kOutF32 ? 4 : 8;
-                if (d_remap || (n0 + (c + 1) * CH > p.N && (p.N % kElemsPer16B) != 0)) {
+                if (plain_store) {
                     if (row < ti.rows) {
                         const int col0 = n0 + c * CH;
                         const int valid = min(CH, p.N - col0);
@@ -1314,6 +1345,11 @@ __global__ void __launch_bounds__(Config<BN, kPair, kEpiWarps>::THREADS, 1) cont
                     if constexpr (kOutF32) {
                         w0 = __float_as_uint(v[4 * j]); w1 = __float_as_uint(v[4 * j + 1]);
                         w2 = __float_as_uint(v[4 * j + 2]); w3 = __float_as_uint(v[4 * j + 3]);
+                    } else if (relu_in_cvt) {
+                        w0 = pack2_relu<kOutF16>(v[8 * j], v[8 * j + 1]);
+                        w1 = pack2_relu<kOutF16>(v[8 * j + 2], v[8 * j + 3]);
+                        w2 = pack2_relu<kOutF16>(v[8 * j + 4], v[8 * j + 5]);
+                        w3 = pack2_relu<kOutF16>(v[8 * j + 6], v[8 * j + 7]);
                     } else {
                         w0 = pack2<kOutF16>(v[8 * j], v[8 * j + 1]);
                         w1 = pack2<kOutF16>(v[8 * j + 2], v[8 * j + 3]);
