@@ -204,7 +204,9 @@ def _ld(t: torch.Tensor) -> int:
     """Leading dimension of a 2-D operand as stored (outer stride; the row length if there is one row)."""
     if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
         raise ValueError("operands must be 2-D with inner stride 1")
-    return t.stride(0) if t.shape[0] > 1 else max(t.shape[1], 1)
+    if t.shape[0] > 1 or t.stride(0) >= max(t.shape[1], 1):
+        return t.stride(0)            # (a one-row view of a padded buffer keeps the buffer's row pitch)
+    return max(t.shape[1], 1)
 
 
 def _gemm_desc(M, N, K, lda, ldb, ldc, ldd, layout_a, layout_b, out_dtype, alpha, beta, epi,
