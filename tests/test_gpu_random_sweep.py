@@ -241,3 +241,59 @@ def test_random_conv2d_wgrad(case):
     what = f"wgrad case {case}: N{N} {H}x{W} C{C} K{K} {R}x{S} pad{pad} stride{stride} dil{dil}"
     parity.assert_matches(out, ref, absacc, what)
     assert bool(torch.isnan(whole[:4]).all()) and bool(torch.isnan(whole[-4:]).all()), what
+
+
+@pytest.mark.parametrize("case", range(40))
+def test_random_skinny_long_k(case):
+    # few output tiles and a long contraction: the planner's K-range forms (two-pass, early donors), the short-A
+    # variants and the matrix-vector kernels (at most eight rows or columns) on extents nobody picked by hand
+    rng = random.Random(13000 + case)
+    seed = 13000 + case
+    M = rng.choice([1, 2, 3, 5, 8, 9, 16, 31, 64, 100, 128, 129, 200, 256, 260])
+    N = rng.choice([1, 2, 4, 7, 8, 9, 24, 64, 72, 128, 136, 256, 264])
+    K = 8 * rng.randint(250, 4100)
+    in_dtype = rng.choice([torch.bfloat16, torch.float16])
+    out_dtype = rng.choice([torch.bfloat16, torch.float32])
+    A = _operand(M, K, _pad8(K, rng), seed, 1, in_dtype)
+    B = _operand(N, K, _pad8(K, rng), seed, 2, in_dtype)
+    bias = inputs.uniform([N], seed, 4).to(in_dtype) if rng.random() < 0.5 else None
+    epi = rng.choice(["none", "relu", "gelu"])
+    alpha = rng.choice([1.0, 2.0 ** -5])
+    ref, absacc = orc.gemm(A, B, bias=bias, alpha=alpha, epi=epi)
+    out, whole, pr = _guarded_out(M, N, _pad8(N, rng), out_dtype)
+    sg.gemm(_dev(A), _dev(B), bias=_dev(bias), out=out, alpha=alpha, epi=epi)
+    plan = sg.last_launch_plan()
+    what = f"skinny case {case}: {M}x{N}x{K} {in_dtype}->{out_dtype} alpha={alpha} bias={bias is not None} epi={epi} plan={plan}"
+    parity.assert_matches(out, ref, absacc, what)
+    assert _guards_ok(whole, pr, N), what
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_multi_wave(case):
+    # more tiles than SMs, under the planner's own choice or a forced tile shape and tail mode: the persistent tile walk,
+    # the raster, tail slices and K ranges on ragged extents
+    rng = random.Random(14000 + case)
+    seed = 14000 + case
+    M, N = rng.randint(700, 2000), rng.randint(700, 2000)
+    K = 8 * rng.randint(8, 140)
+    la, lb = rng.choice([("row", "col"), ("row", "col"), ("col", "col"), ("row", "row"), ("col", "row")])
+    out_dtype = rng.choice([torch.bfloat16, torch.float32])
+    a_shape = (M, K) if la == "row" else (K, M)
+    b_shape = (N, K) if lb == "col" else (K, N)
+    A = _operand(a_shape[0], a_shape[1], _pad8(a_shape[1], rng), seed, 1, torch.bfloat16)
+    B = _operand(b_shape[0], b_shape[1], _pad8(b_shape[1], rng), seed, 2, torch.bfloat16)
+    bias = inputs.uniform([N], seed, 4) if rng.random() < 0.5 else None
+    beta = rng.choice([0.0, 1.0])
+    C = _operand(M, N, _pad8(N, rng), seed, 3, out_dtype) if beta != 0.0 else None
+    epi = rng.choice(["none", "relu", "silu"])
+    tile_n, pair = rng.choice([(-1, -1), (-1, -1), (64, 0), (128, 0), (256, 0), (128, 1), (256, 1)])
+    tail = rng.choice([-1, -1, 0, 1, 2])
+    sg.set_tuning(tile_n, pair)
+    sg.set_tail_mode(tail)
+    ref, absacc = orc.gemm(A, B, layout_a=la, layout_b=lb, C=C, bias=bias, beta=beta, epi=epi)
+    out, whole, pr = _guarded_out(M, N, _pad8(N, rng), out_dtype)
+    sg.gemm(_dev(A), _dev(B), C=_dev(C), bias=_dev(bias), out=out, beta=beta, epi=epi, layout_a=la, layout_b=lb)
+    what = f"multi-wave case {case}: {M}x{N}x{K} {la}/{lb} ->{out_dtype} beta={beta} bias={bias is not None} epi={epi} " \
+           f"forced tile {tile_n}/{pair} tail {tail} plan={sg.last_launch_plan()}"
+    parity.assert_matches(out, ref, absacc, what)
+    assert _guards_ok(whole, pr, N), what
