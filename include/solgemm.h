@@ -73,6 +73,7 @@ typedef enum { SG_BF16 = 0, SG_F32 = 1, SG_F16 = 2, SG_FP8_E4M3 = 3, SG_FP8_E5M2
 typedef enum { SG_ROW_MAJOR = 0, SG_COL_MAJOR = 1 } sg_layout_t;
 typedef enum {
     SG_EPI_NONE = 0, SG_EPI_BIAS = 1, SG_EPI_RELU = 2, SG_EPI_GELU = 3, SG_EPI_SILU = 4,
+    /* (SG_EPI_RELU is max(x, 0); where x is NaN the result is NaN or +0, depending on the kernel variant that runs) */
     /* further built-ins of the paper's Table 1c; epi_arg0 / epi_arg1 carry their parameters */
     SG_EPI_SIGMOID = 5,     /* 1 / (1 + e^-x) */
     SG_EPI_TANH = 6,
