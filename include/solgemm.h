@@ -113,7 +113,8 @@ typedef struct sg_gemm_desc {
  *   D      device, out_dtype, [M,N] row-major; written in full (all M x N elements).
  * M == 0 or N == 0: SG_OK, nothing is launched.  K == 0: D = act(beta*C + bias).
  * Matrix-vector form (the workload list's single-token decode product): when N <= 8 (or M <= 8; 4 for SG_F32 inputs or
- *   when K is no multiple of 8), the matrix operand is
+ *   when K is no multiple of 8; also 9..32 for 16-bit inputs against a matrix of at most 48 MB, 12 MB from 17 vectors
+ *   on, where the tiles' fixed cost would decide the time), the matrix operand is
  *   K-contiguous (A row-major, resp. B column-major) and 16-byte aligned with a leading dimension that is a multiple
  *   of 16 bytes, the vectors are K-contiguous, 16-byte aligned and a multiple of 16 bytes apart (a single vector may
  *   also be stored as K x 1 with a leading dimension of 1), and in_dtype is SG_BF16, SG_F16 or SG_F32, the product
@@ -436,7 +437,8 @@ typedef enum {
                                    into ranges summed by a second kernel, k >= 2 = at most k ranges (default: as many as
                                    there are SMs to go round) */
     SG_OPT_SPLIT_K_REDUCE_WARPS = 16, /* second pass of a two-pass K split: 1, 2, 4 or 8 warps share the parts of a column slice */
-    SG_OPT_COUNT_ = 17
+    SG_OPT_GEMV_MAX_VECTORS = 17, /* most vectors (4..32) the matrix-vector kernels take before the tiles do; default 32 */
+    SG_OPT_COUNT_ = 18
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

@@ -986,11 +986,12 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     *taken = false;
     if (!desc || desc->K < 1 || desc->K > INT32_MAX || desc->M < 1 || desc->N < 1) return SG_OK;
     if (opt(SG_OPT_NO_GEMV) > 0) return SG_OK;      // tests: the same product through the tiles
-    // up to eight vectors of 16-bit inputs (four of fp32); the matrix is the operand with more rows
+    // up to 32 vectors of 16-bit inputs (four of fp32); the matrix is the operand with more rows
     if (desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F16 && desc->in_dtype != SG_F32) return SG_OK;
     const int es = desc->in_dtype == SG_F32 ? 4 : 2;
     const bool no_mma = opt(SG_OPT_GEMV_NO_MMA) > 0;      // FMA kernel only (<= 4 vectors)
-    const int64_t max_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? 8 : 4;
+    const int64_t mma_vec = opt(SG_OPT_GEMV_MAX_VECTORS) > 0 ? std::min<int64_t>(32, opt(SG_OPT_GEMV_MAX_VECTORS)) : 32;
+    const int64_t max_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? std::max<int64_t>(mma_vec, 4) : 4;
     const bool mat_a = desc->N <= max_vec && desc->M >= desc->N;
     if (!mat_a && desc->M > max_vec) return SG_OK;
     // the matrix K-contiguous, the vectors contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
@@ -1004,6 +1005,14 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     if (mat_a ? !(a_kc && (b_kc || (nvec == 1 && desc->ldb == 1))) : !(b_kc && (a_kc || (nvec == 1 && desc->lda == 1)))) return SG_OK;
     if (R > INT32_MAX || ld < desc->K || (ld * es) % 16 || !W || !x || !aligned16(W) || !aligned16(x)) return SG_OK;
     if (nvec > 1 && (x_stride < desc->K || (x_stride * es) % 16)) return SG_OK;
+    if (nvec > 8 && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0) {
+        // Nine to 32 vectors: every CTA re-reads its K range of all vectors from the L2 and holds fewer matrix loads in
+        // flight, so the stream over a large matrix is slower than the tiles' (16 x 8192 x 8192: 33 against 28 us); what
+        // this path saves is the tiles' fixed cost, which decides small problems (16 x 1024 x 1024: 2.6 against 6.4 us,
+        // 32 x 2048 x 2048: 6.7 against 10.2, 12 x 4096 x 4096: 13.5 against 20.5).  Measured crossovers:
+        const double w_bytes = static_cast<double>(R) * static_cast<double>(desc->K) * es;
+        if (w_bytes > (nvec <= 16 ? 48.0e6 : 12.0e6)) return SG_OK;
+    }
     *taken = true;
 
     Checked c;
@@ -1052,7 +1061,7 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int64_t want = 2 * static_cast<int64_t>(d->sm_count);
     if (es == 2 && !no_mma && desc->K % 8 == 0 && nvec >= 2) {
-        // two to eight vectors: warp-level MMAs, 16 rows per CTA, K ranges in units of 256 elements (one step of
+        // two to 32 vectors: warp-level MMAs, 16 rows per CTA, K ranges in units of 256 elements (one step of
         // the CTA's eight warps), at least four steps per warp and rank
         const int64_t blocks = (R + 15) / 16;
         const int64_t ks_max = std::max<int64_t>(1, std::min<int64_t>(8, desc->K / 1024));
@@ -1084,14 +1093,18 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        cudaError_t e = desc->in_dtype == SG_F16
-                            ? (wide ? cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__half, true>, gp)
-                                    : cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__half, false>, gp))
-                            : (wide ? cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__nv_bfloat16, true>, gp)
-                                    : cudaLaunchKernelEx(&cfg, gemv_mma_kernel<__nv_bfloat16, false>, gp));
+        using GemvMmaFn = void (*)(const GemvParams);
+        static const GemvMmaFn table[2][2][3] = {
+            {{gemv_mma_kernel<__nv_bfloat16, false, 1>, gemv_mma_kernel<__nv_bfloat16, false, 2>, gemv_mma_kernel<__nv_bfloat16, false, 4>},
+             {gemv_mma_kernel<__nv_bfloat16, true, 1>, gemv_mma_kernel<__nv_bfloat16, true, 2>, gemv_mma_kernel<__nv_bfloat16, true, 4>}},
+            {{gemv_mma_kernel<__half, false, 1>, gemv_mma_kernel<__half, false, 2>, gemv_mma_kernel<__half, false, 4>},
+             {gemv_mma_kernel<__half, true, 1>, gemv_mma_kernel<__half, true, 2>, gemv_mma_kernel<__half, true, 4>}}};
+        const int nvb = nvec <= 8 ? 0 : (nvec <= 16 ? 1 : 2);        // blocks of eight vectors: 1, 2 or 4
+        cudaError_t e = cudaLaunchKernelEx(&cfg, table[desc->in_dtype == SG_F16 ? 1 : 0][wide ? 1 : 0][nvb], gp);
         if (e != cudaSuccess) return fail(SG_ERR_CUDA, "matrix-vector (MMA) kernel launch: %s", cudaGetErrorString(e));
         g_launches.fetch_add(1);
-        note_kernel("sg::gemv_mma_kernel<%s, %s>", desc->in_dtype == SG_F16 ? "__half" : "__nv_bfloat16", wide ? "true" : "false");
+        note_kernel("sg::gemv_mma_kernel<%s, %s, %d>", desc->in_dtype == SG_F16 ? "__half" : "__nv_bfloat16", wide ? "true" : "false",
+                    1 << nvb);
         t_last_plan[0] = 0;
         t_last_plan[1] = 0;
         t_last_plan[2] = -static_cast<int32_t>(ks);

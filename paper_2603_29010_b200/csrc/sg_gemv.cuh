@@ -1,9 +1,10 @@
 // Matrix-vector products with the fused epilogue: out[r][v] = act(alpha * sum_k W[r][k] x_v[k] + beta * C + bias), for
-// up to eight vectors x_v at once.  The GEMM with N <= 8 (or M <= 8) of the paper's workload list (single-token
+// up to 32 vectors x_v at once.  The GEMM with N <= 8 (or M <= 8) of the paper's workload list (single-token
 // decode): every matrix element is used once per vector, so the kernels are a stream over W bound by HBM, and the
 // tcgen05 tiles (128 rows for at most eight useful ones, operands staged in shared memory) have nothing to offer.
 // Two kernels: gemv_kernel (CUDA-core FMAs: one vector; fp32 inputs or a ragged K: up to four) and gemv_mma_kernel
-// (warp-level MMAs: two to eight vectors of 16-bit inputs).
+// (warp-level MMAs: two to eight vectors of 16-bit inputs, and nine to 32 against matrices small enough that the
+// tiles' fixed cost would decide the time).
 //
 // Work split of gemv_kernel: a CTA of 256 threads takes RB consecutive rows and one K range; each thread walks the
 // range in 16-byte vectors (one vector of x serves RB vectors of W, so RB independent loads are in flight per thread
@@ -28,7 +29,7 @@ struct GemvParams {
     int64_t x_stride;
     int64_t c_row_stride, c_vec_stride, d_row_stride, d_vec_stride;   // element (row r, vector v) of C and D
     int32_t R, K;
-    int32_t nvec;         // 1..8 (gemv_kernel: 1..4)
+    int32_t nvec;         // 1..32 (gemv_kernel: 1..4)
     int32_t kchunk;       // K elements per cluster rank (a multiple of 256 vectors)
     int32_t ksplit;       // CTAs per cluster
     int32_t bias_row_stride, bias_vec_stride;   // (0, 1): one bias per vector (the matrix is A); (1, 0): one per row
@@ -263,16 +264,19 @@ __device__ __forceinline__ U8 ldg_cached32(const void* p) {
 
 // kWide = false: 16-byte pieces; requires K % 8 == 0 and kchunk % 256 == 0.
 // kWide = true: 32-byte pieces; requires K % 16 == 0, kchunk % 512 == 0 and 32-byte aligned rows and vectors.
+// NVB: blocks of eight vectors (1, 2 or 4: up to 8, 16 or 32 vectors).  Every block is one more MMA per piece of W on
+// the same A fragment and four more accumulator registers; thread group g loads vectors g, g + 8, g + 16, g + 24.
 // Grid: ceil(R / 16) row blocks x ksplit ranks.
-template <typename T, bool kWide>
+template <typename T, bool kWide, int NVB = 1>
 __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     namespace cg = cooperative_groups;
     constexpr int WARPS = 8;
     constexpr int PE = kWide ? 16 : 8;        // elements per thread and step
-    constexpr int U = kWide ? 2 : 4;          // steps in flight per warp
+    constexpr int U = (kWide ? 2 : 4) / (NVB == 4 ? 2 : 1);   // steps in flight per warp (fewer with 32 vectors: registers)
     constexpr int STEP = 4 * PE;              // elements of K a warp covers per step
-    __shared__ float warp_part[WARPS][128];   // 16 rows x 8 vectors per warp
-    __shared__ float cta_part[128];
+    constexpr int NV = 8 * NVB;               // vector slots
+    __shared__ float warp_part[WARPS][16 * NV];   // 16 rows x NV vectors per warp
+    __shared__ float cta_part[16 * NV];
 
     const int ks = p.ksplit;
     const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));
@@ -284,8 +288,13 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
 
     const T* wlo = reinterpret_cast<const T*>(p.W) + min(r0 + g, static_cast<int64_t>(p.R) - 1) * p.ld;
     const T* whi = reinterpret_cast<const T*>(p.W) + min(r0 + g + 8, static_cast<int64_t>(p.R) - 1) * p.ld;
-    const T* xv = reinterpret_cast<const T*>(p.x) + static_cast<int64_t>(min(g, p.nvec - 1)) * p.x_stride;
-    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    const T* xv[NVB];
+    float c[NVB][4];
+#pragma unroll
+    for (int j = 0; j < NVB; ++j) {
+        xv[j] = reinterpret_cast<const T*>(p.x) + static_cast<int64_t>(min(g + 8 * j, p.nvec - 1)) * p.x_stride;
+        c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.0f;
+    }
 
     // The loop bounds are the same for all lanes of a warp (mma.sync must be executed by the whole warp).  Main loop:
     // U steps whose pieces all lie inside the K range, loads without conditions; then single steps in which a lane
@@ -294,32 +303,40 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     for (; kw + (U - 1) * WARPS * STEP + STEP <= kend; kw += U * WARPS * STEP) {
         const int k0 = kw + t * PE;
         if constexpr (kWide) {
-            U8 lo[U], hi[U], xx[U];
+            U8 lo[U], hi[U], xx[U][NVB];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 lo[u] = ldg_stream32(wlo + k0 + u * WARPS * STEP);
                 hi[u] = ldg_stream32(whi + k0 + u * WARPS * STEP);
-                xx[u] = ldg_cached32(xv + k0 + u * WARPS * STEP);
+#pragma unroll
+                for (int b = 0; b < NVB; ++b) xx[u][b] = ldg_cached32(xv[b] + k0 + u * WARPS * STEP);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    GemvMma<T>::mma(c, lo[u].w[2 * j], hi[u].w[2 * j], lo[u].w[2 * j + 1], hi[u].w[2 * j + 1], xx[u].w[2 * j],
-                                    xx[u].w[2 * j + 1]);
+                for (int b = 0; b < NVB; ++b) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        GemvMma<T>::mma(c[b], lo[u].w[2 * j], hi[u].w[2 * j], lo[u].w[2 * j + 1], hi[u].w[2 * j + 1],
+                                        xx[u][b].w[2 * j], xx[u][b].w[2 * j + 1]);
+                }
             }
         } else {
-            uint4 lo[U], hi[U], xx[U];
+            uint4 lo[U], hi[U], xx[U][NVB];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 lo[u] = ldg_stream16(wlo + k0 + u * WARPS * STEP);
                 hi[u] = ldg_stream16(whi + k0 + u * WARPS * STEP);
-                xx[u] = __ldg(reinterpret_cast<const uint4*>(xv + k0 + u * WARPS * STEP));
+#pragma unroll
+                for (int b = 0; b < NVB; ++b) xx[u][b] = __ldg(reinterpret_cast<const uint4*>(xv[b] + k0 + u * WARPS * STEP));
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                GemvMma<T>::mma(c, lo[u].x, hi[u].x, lo[u].y, hi[u].y, xx[u].x, xx[u].y);
-                GemvMma<T>::mma(c, lo[u].z, hi[u].z, lo[u].w, hi[u].w, xx[u].z, xx[u].w);
+#pragma unroll
+                for (int b = 0; b < NVB; ++b) {
+                    GemvMma<T>::mma(c[b], lo[u].x, hi[u].x, lo[u].y, hi[u].y, xx[u][b].x, xx[u][b].y);
+                    GemvMma<T>::mma(c[b], lo[u].z, hi[u].z, lo[u].w, hi[u].w, xx[u][b].z, xx[u][b].w);
+                }
             }
         }
     }
@@ -327,49 +344,66 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
         const int k = kw + t * PE;
         const bool valid = k < kend;        // pieces are whole: K, kbeg and k are multiples of PE
         if constexpr (kWide) {
-            U8 lo, hi, xx;
+            U8 lo, hi, xx[NVB];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) lo.w[j] = hi.w[j] = xx.w[j] = 0u;
+            for (int j = 0; j < 8; ++j) {
+                lo.w[j] = hi.w[j] = 0u;
+#pragma unroll
+                for (int b = 0; b < NVB; ++b) xx[b].w[j] = 0u;
+            }
             if (valid) {
                 lo = ldg_stream32(wlo + k);
                 hi = ldg_stream32(whi + k);
-                xx = ldg_cached32(xv + k);
+#pragma unroll
+                for (int b = 0; b < NVB; ++b) xx[b] = ldg_cached32(xv[b] + k);
             }
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                GemvMma<T>::mma(c, lo.w[2 * j], hi.w[2 * j], lo.w[2 * j + 1], hi.w[2 * j + 1], xx.w[2 * j], xx.w[2 * j + 1]);
+            for (int b = 0; b < NVB; ++b) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    GemvMma<T>::mma(c[b], lo.w[2 * j], hi.w[2 * j], lo.w[2 * j + 1], hi.w[2 * j + 1], xx[b].w[2 * j], xx[b].w[2 * j + 1]);
+            }
         } else {
-            uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo, xx = lo;
+            uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo, xx[NVB];
+#pragma unroll
+            for (int b = 0; b < NVB; ++b) xx[b] = lo;
             if (valid) {
                 lo = ldg_stream16(wlo + k);
                 hi = ldg_stream16(whi + k);
-                xx = __ldg(reinterpret_cast<const uint4*>(xv + k));
+#pragma unroll
+                for (int b = 0; b < NVB; ++b) xx[b] = __ldg(reinterpret_cast<const uint4*>(xv[b] + k));
             }
-            GemvMma<T>::mma(c, lo.x, hi.x, lo.y, hi.y, xx.x, xx.y);
-            GemvMma<T>::mma(c, lo.z, hi.z, lo.w, hi.w, xx.z, xx.w);
+#pragma unroll
+            for (int b = 0; b < NVB; ++b) {
+                GemvMma<T>::mma(c[b], lo.x, hi.x, lo.y, hi.y, xx[b].x, xx[b].y);
+                GemvMma<T>::mma(c[b], lo.z, hi.z, lo.w, hi.w, xx[b].z, xx[b].w);
+            }
         }
     }
-    // accumulator fragment: c0 (row g, vector 2t), c1 (g, 2t+1), c2 (g+8, 2t), c3 (g+8, 2t+1)
-    warp_part[warp][g * 8 + 2 * t] = c[0];
-    warp_part[warp][g * 8 + 2 * t + 1] = c[1];
-    warp_part[warp][(g + 8) * 8 + 2 * t] = c[2];
-    warp_part[warp][(g + 8) * 8 + 2 * t + 1] = c[3];
+    // accumulator fragment of block b: c0 (row g, vector 8b + 2t), c1 (g, 8b + 2t+1), c2 (g+8, 8b + 2t), c3 (g+8, 8b + 2t+1)
+#pragma unroll
+    for (int b = 0; b < NVB; ++b) {
+        warp_part[warp][g * NV + 8 * b + 2 * t] = c[b][0];
+        warp_part[warp][g * NV + 8 * b + 2 * t + 1] = c[b][1];
+        warp_part[warp][(g + 8) * NV + 8 * b + 2 * t] = c[b][2];
+        warp_part[warp][(g + 8) * NV + 8 * b + 2 * t + 1] = c[b][3];
+    }
     __syncthreads();
-    if (threadIdx.x < 128) {
+    for (int i = static_cast<int>(threadIdx.x); i < 16 * NV; i += 256) {
         float s = 0.0f;
 #pragma unroll
-        for (int wi = 0; wi < WARPS; ++wi) s += warp_part[wi][threadIdx.x];
-        cta_part[threadIdx.x] = s;
+        for (int wi = 0; wi < WARPS; ++wi) s += warp_part[wi][i];
+        cta_part[i] = s;
     }
     if (ks > 1) cg::this_cluster().sync();
-    if (rank == 0 && threadIdx.x < 128) {
-        float s = cta_part[threadIdx.x];
+    for (int i = static_cast<int>(threadIdx.x); rank == 0 && i < 16 * NV; i += 256) {
+        float s = cta_part[i];
         if (ks > 1) {
             cg::cluster_group cluster = cg::this_cluster();
-            for (int r = 1; r < ks; ++r) s += *cluster.map_shared_rank(&cta_part[threadIdx.x], r);
+            for (int r = 1; r < ks; ++r) s += *cluster.map_shared_rank(&cta_part[i], r);
         }
-        const int64_t row = r0 + static_cast<int>(threadIdx.x) / 8;
-        const int vec = static_cast<int>(threadIdx.x) % 8;
+        const int64_t row = r0 + i / NV;
+        const int vec = i % NV;
         if (row < p.R && vec < p.nvec) {
             float v[1] = {p.alpha * s};
             if (p.beta != 0.0f) v[0] = fmaf(p.beta, gemv_load_out(p.C, row * p.c_row_stride + vec * p.c_vec_stride, p.out_kind), v[0]);

@@ -19,9 +19,13 @@ DEV = "cuda"
 @pytest.fixture(autouse=True)
 def _clean_status():
     sg.set_tuning(-1, -1)
+    sg.set_option("gemv_max_vectors", -1)
+    sg.set_option("no_gemv", -1)
     yield
     torch.cuda.synchronize()
     sg.poll_status()
+    sg.set_option("gemv_max_vectors", -1)
+    sg.set_option("no_gemv", -1)
 
 
 def _took_vector_path():
@@ -148,12 +152,18 @@ def test_results_do_not_depend_on_the_run():
 def test_other_forms_still_go_through_the_tiles():
     g = torch.Generator().manual_seed(4)
     A = torch.randn(256, 64, generator=g).to(torch.bfloat16)
-    B9 = torch.randn(9, 64, generator=g).to(torch.bfloat16)
-    out = torch.empty(256, 16, dtype=torch.bfloat16, device=DEV)
-    sg.gemm(A.to(DEV), B9.to(DEV), out=out[:, :9])
+    B33 = torch.randn(33, 64, generator=g).to(torch.bfloat16)
+    out = torch.empty(256, 40, dtype=torch.bfloat16, device=DEV)
+    sg.gemm(A.to(DEV), B33.to(DEV), out=out[:, :33])
     assert not _took_vector_path()
-    ref, absacc = orc.gemm(A, B9)
-    parity.assert_matches(out[:, :9], ref, absacc, "N = 9")
+    ref, absacc = orc.gemm(A, B33)
+    parity.assert_matches(out[:, :33], ref, absacc, "N = 33")
+    # nine vectors against a matrix too large for the many-vector form of the kernel (more than 48 MB)
+    Wbig = torch.randn(6200, 4096, generator=g).to(torch.bfloat16)
+    X9 = torch.randn(9, 4096, generator=g).to(torch.bfloat16)
+    D9 = sg.gemm(X9.to(DEV), Wbig.to(DEV))
+    assert not _took_vector_path()
+    parity.assert_matches(D9[:, :64], *[t[:, :64] for t in orc.gemm(X9, Wbig[:64])], "nine vectors, large matrix")
     # a K x 2 row-major B is not a pair of contiguous vectors
     Brow = torch.randn(64, 8, generator=g).to(torch.bfloat16)
     sg.gemm(A.to(DEV), Brow.to(DEV)[:, :2], layout_b="row", out=out[:, :2])
@@ -166,6 +176,8 @@ def test_other_forms_still_go_through_the_tiles():
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
 def test_few_rows_against_a_large_matrix_on_the_tiles(M, dtype):
     # 9..64 rows: the tensor-core tiles with only 32 or 64 rows of A loaded per stage; 65: the full A tile
+    # (a matrix this small would go to the matrix-vector kernels with up to 32 rows: keep those to eight vectors here)
+    sg.set_option("gemv_max_vectors", 8)
     g = torch.Generator().manual_seed(100 + M)
     N, K = 1080, 2056
     A = (torch.randn(M, K, generator=g) / 8).to(dtype)
@@ -186,6 +198,7 @@ def test_few_rows_against_a_large_matrix_on_the_tiles(M, dtype):
         sg.gemm(Ai.to(DEV), Wi.to(DEV), out=Di)
         parity.assert_bit_exact(Di, refi, f"{M} integer rows, tile width {tile_n}")
     sg.set_tuning(-1, -1)
+    sg.set_option("gemv_max_vectors", -1)
 
 
 def test_few_rows_batched():
@@ -218,3 +231,54 @@ def test_several_vectors_k_not_a_multiple_of_a_warp_step(R, K, nvec):
     sg.gemm(W.to(DEV), X.to(DEV), out=D)
     assert _took_vector_path()
     parity.assert_bit_exact(D, ref, f"{R}x{K} times {nvec} vectors")
+
+
+@pytest.mark.parametrize("nvec", [9, 12, 16, 17, 24, 31, 32])
+@pytest.mark.parametrize("R,K", [(512, 1024), (130, 4104), (37, 264), (2048, 2048), (5, 72)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_nine_to_32_vectors_in_one_pass(R, K, nvec, dtype):
+    # blocks of eight vectors share one pass over the matrix (two blocks up to 16 vectors, four up to 32)
+    g = torch.Generator().manual_seed(R + K + nvec)
+    W = (torch.randn(R, K, generator=g) / 8).to(dtype)
+    X = (torch.randn(nvec, K, generator=g) / 8).to(dtype)
+    fewer = min(nvec, R)                      # the operand with fewer rows supplies the vectors
+    blocks = 1 if fewer <= 8 else (2 if fewer <= 16 else 4)
+    # vectors on the left (a decode batch): D [nvec, R], bias per matrix row, residual
+    Ct = torch.randn(nvec, R, generator=g).to(dtype)
+    biasR = torch.randn(R, generator=g).to(dtype)
+    ref, absacc = orc.gemm(X, W, C=Ct, bias=biasR, alpha=0.75, beta=0.5, epi="silu")
+    D = sg.gemm(X.to(DEV), W.to(DEV), C=Ct.to(DEV), bias=biasR.to(DEV), alpha=0.75, beta=0.5, epi="silu", out_dtype=dtype)
+    assert _took_vector_path() and sg.last_kernel_name().endswith(f", {blocks}>"), sg.last_kernel_name()
+    parity.assert_matches(D, ref, absacc, f"{nvec} vectors times {R}x{K} {dtype}")
+    # matrix on the left: D [R, nvec], bias per vector, fp32 output inside NaN guard columns
+    bias = torch.randn(nvec, generator=g).to(dtype)
+    ref, absacc = orc.gemm(W, X, bias=bias, epi="gelu")
+    whole = torch.full((R, 40), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(W.to(DEV), X.to(DEV), bias=bias.to(DEV), epi="gelu", out=whole[:, :nvec])
+    assert _took_vector_path()
+    parity.assert_matches(whole[:, :nvec], ref, absacc, f"{R}x{K} times {nvec} vectors {dtype}")
+    assert bool(torch.isnan(whole[:, nvec:]).all())
+    # small integers: exact, both forms
+    Wi = inputs.small_integers([R, K], 95, 1, lo=-2, hi=2).to(dtype)
+    Xi = inputs.small_integers([nvec, K], 95, 2, lo=-2, hi=2).to(dtype)
+    refi, _ = orc.gemm(Xi, Wi)
+    Di = torch.full((nvec, R), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(Xi.to(DEV), Wi.to(DEV), out=Di)
+    parity.assert_bit_exact(Di, refi, f"{nvec} integer vectors times {R}x{K} {dtype}")
+    refi, _ = orc.gemm(Wi, Xi)
+    Di = torch.full((R, nvec), float("nan"), dtype=torch.float32, device=DEV)
+    sg.gemm(Wi.to(DEV), Xi.to(DEV), out=Di)
+    parity.assert_bit_exact(Di, refi, f"{R}x{K} times {nvec} integer vectors {dtype}")
+
+
+def test_many_vectors_match_the_tiles_bit_for_bit_on_integers():
+    # the same product through both paths of the library
+    W = inputs.small_integers([700, 1544], 96, 1, lo=-2, hi=2)
+    X = inputs.small_integers([20, 1544], 96, 2, lo=-2, hi=2)
+    a = sg.gemm(X.to(DEV), W.to(DEV), out_dtype=torch.float32)
+    assert _took_vector_path()
+    sg.set_option("no_gemv", 1)
+    b = sg.gemm(X.to(DEV), W.to(DEV), out_dtype=torch.float32)
+    sg.set_option("no_gemv", -1)
+    assert not _took_vector_path()
+    assert torch.equal(a, b)
