@@ -120,7 +120,9 @@ typedef struct sg_gemm_desc {
  *   also be stored as K x 1 with a leading dimension of 1), and in_dtype is SG_BF16, SG_F16 or SG_F32, the product
  *   runs as one pass over the matrix at HBM speed instead of through tensor-core tiles.  In that form ldc and ldd may
  *   be any value >= N (no 16-byte rule) and C, D and bias need only their element alignment; results are reproducible
- *   from run to run.
+ *   from run to run.  A small product of 16-bit K-contiguous operands (at most 160 M multiply-adds, and few enough
+ *   outputs that one CTA per 16 x 32 of them fits on the GPU at once) runs on the same kernels, in groups of 32 vectors,
+ *   for their shorter start and end; a tile shape forced through sg_set_tuning keeps it on the tiles.
  */
 sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C,
                     const void* bias, void* D, void* cuda_stream);
@@ -361,9 +363,9 @@ const char* sg_last_error(void);
  * sg_poll_status: reads (and clears) the device-side status word of the current device.  Call it
  * after synchronising the stream(s) the work was enqueued on; `cuda_stream` is used for the read.
  * SG_OK, or SG_ERR_TIMEOUT with the role / tile / barrier that gave up in sg_last_error().  While
- * the word is set, later launches of the tensor-core contraction kernel (every entry point above except the
- * matrix-vector form of sg_gemm and sg_transpose, whose kernels contain no waits and do not read the word) return
- * at once without computing and leave their outputs untouched; the poll that reports the word also clears it and
+ * the word is set, later launches of the tensor-core contraction kernel return at once without computing, and the
+ * kernels of the matrix-vector / small-product form of sg_gemm store nothing: their outputs stay untouched
+ * (sg_transpose, whose kernel waits on nothing outside its own CTA, does not read the word); the poll that reports the word also clears it and
  * the K-range counters of a lent scratch, after which calls compute again.
  */
 sg_status_t sg_poll_status(void* cuda_stream);
@@ -438,7 +440,8 @@ typedef enum {
                                    there are SMs to go round) */
     SG_OPT_SPLIT_K_REDUCE_WARPS = 16, /* second pass of a two-pass K split: 1, 2, 4 or 8 warps share the parts of a column slice */
     SG_OPT_GEMV_MAX_VECTORS = 17, /* most vectors (4..32) the matrix-vector kernels take before the tiles do; default 32 */
-    SG_OPT_COUNT_ = 18
+    SG_OPT_GEMV_SMALL_LOG2 = 18,  /* products of at most 2^value multiply-adds (16-bit operands) run on the warp-level MMA kernel; 0 = none */
+    SG_OPT_COUNT_ = 19
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

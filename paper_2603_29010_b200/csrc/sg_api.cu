@@ -334,6 +334,8 @@ struct Shape {
 inline double ksplit_exchange_us(int64_t ks) { return ks > 1 ? 6.0 + 0.5 * static_cast<double>(ks - 1) : 0.0; }
 // The same for the two-pass form (every part parks all its sums and exits; a second kernel adds them up): flat in ks.
 constexpr int kTwoPassMinKb = 4;           // k-blocks per part at least
+constexpr double kGemvSmallMacs = 160.0e6;         // products of at most this many multiply-adds run on the warp-level MMA
+                                                    // kernel when its CTAs all fit on the GPU at once (see try_gemv)
 // Modelled time (us) of a two-pass K split with `ks` parts per tile: the longer of the parts' tensor time and of streaming
 // the operands from HBM (a CTA pulls about 38 GB/s, all of them together about 5.5 TB/s), plus a fixed 3 us for the
 // second kernel, plus writing and re-reading the parked sums.  Fitted to 256 x 256 x {8192 .. 131072}, 512 x 512 x 16384,
@@ -959,13 +961,15 @@ cudaError_t launch_gemv(const GemvParams& gp, int rb, int ctas, cudaStream_t str
     cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
     cfg.blockDim = dim3(256, 1, 1);
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(gp.ksplit);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // (the kernel waits for its predecessor itself)
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = opt(SG_OPT_NO_PDL) > 0 ? 1 : 2;
     const int nv = gp.nvec <= 1 ? 1 : (gp.nvec == 2 ? 2 : 4);
 #define SG_GEMV_CASE(RB_)                                                             \
     case RB_:                                                                         \
@@ -992,8 +996,28 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     const bool no_mma = opt(SG_OPT_GEMV_NO_MMA) > 0;      // FMA kernel only (<= 4 vectors)
     const int64_t mma_vec = opt(SG_OPT_GEMV_MAX_VECTORS) > 0 ? std::min<int64_t>(32, opt(SG_OPT_GEMV_MAX_VECTORS)) : 32;
     const int64_t max_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? std::max<int64_t>(mma_vec, 4) : 4;
-    const bool mat_a = desc->N <= max_vec && desc->M >= desc->N;
-    if (!mat_a && desc->M > max_vec) return SG_OK;
+    // A small product of 16-bit operands runs on the same warp-level MMA kernel with the vectors in groups of 32 along the
+    // grid's second dimension: it is bound by launch and memory latency, which that kernel has less of than the tiles (no
+    // tensor-memory allocation, no barrier set-up, no shared-memory staging, no TMA store).  It pays while all its CTAs
+    // (16 x 32 outputs each) are resident at once and the K loop is short: measured against the tiles, 256^3 2.75 against
+    // 3.6 us, 128^3 2.2 / 3.2, 384^3 3.4 / 4.1, 256 x 256 x 1024 3.9 / 6.5, 256 x 256 x 2048 5.8 / 7.9, 384 x 384 x 1024
+    // 4.6 / 6.5, 64 x 64 x 4096 5.3 / 6.9, 512 x 64 x 512 3.0 / 4.5 -- but 400^3 5.4 / 4.5, 512^3 6.3 / 4.5, 512 x 512 x 128
+    // 5.0 / 3.3, 256 x 1024 x 256 7.0 / 3.7 (more CTAs than fit) and 256 x 256 x 4096 11.6 / 10.4, 160 x 160 x 8192 12.3 / 9.6
+    // (long K).  Taken up to two CTAs per SM and 160 M multiply-adds (SG_OPT_GEMV_SMALL_LOG2 pins the second limit and
+    // lifts the first).
+    const bool small_forced = opt(SG_OPT_GEMV_SMALL_LOG2) >= 0;
+    const double small_macs = small_forced ? std::ldexp(1.0, static_cast<int>(std::min<int64_t>(40, opt(SG_OPT_GEMV_SMALL_LOG2)))) : kGemvSmallMacs;
+    // (16 rows of the operand with more rows x 32 rows of the other per CTA, two CTAs per SM)
+    const int64_t small_ctas = ((std::max(desc->M, desc->N) + 15) / 16) * ((std::min(desc->M, desc->N) + 31) / 32);
+    bool small = es == 2 && !no_mma && desc->K % 8 == 0 && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0 &&
+                 g_tune_tile_n.load() <= 0 && g_tune_pair.load() < 0 &&      // (a forced tile shape means the tiles)
+                 static_cast<double>(desc->M) * static_cast<double>(desc->N) * static_cast<double>(desc->K) <= small_macs;
+    if (small && !small_forced) {
+        DeviceState* ds = nullptr;
+        small = device_state(&ds) == SG_OK && ds && small_ctas <= 2 * static_cast<int64_t>(ds->sm_count);
+    }
+    const bool mat_a = small ? desc->M >= desc->N : (desc->N <= max_vec && desc->M >= desc->N);
+    if (!small && !mat_a && desc->M > max_vec) return SG_OK;
     // the matrix K-contiguous, the vectors contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
     const bool a_kc = desc->layout_a == SG_ROW_MAJOR, b_kc = desc->layout_b == SG_COL_MAJOR;
     const void* W = mat_a ? A : B;
@@ -1005,7 +1029,7 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     if (mat_a ? !(a_kc && (b_kc || (nvec == 1 && desc->ldb == 1))) : !(b_kc && (a_kc || (nvec == 1 && desc->lda == 1)))) return SG_OK;
     if (R > INT32_MAX || ld < desc->K || (ld * es) % 16 || !W || !x || !aligned16(W) || !aligned16(x)) return SG_OK;
     if (nvec > 1 && (x_stride < desc->K || (x_stride * es) % 16)) return SG_OK;
-    if (nvec > 8 && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0) {
+    if (nvec > 8 && !small && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0) {
         // Nine to 32 vectors: every CTA re-reads its K range of all vectors from the L2 and holds fewer matrix loads in
         // flight, so the stream over a large matrix is slower than the tiles' (16 x 8192 x 8192: 33 against 28 us); what
         // this path saves is the tiles' fixed cost, which decides small problems (16 x 1024 x 1024: 2.6 against 6.4 us,
@@ -1041,6 +1065,7 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     gp.C = desc->beta != 0.0f ? C : nullptr;
     gp.bias = bias;
     gp.D = D;
+    gp.status = d->status_dev;
     gp.ld = ld;
     gp.x_stride = x_stride;
     gp.c_row_stride = mat_a ? desc->ldc : 1;
@@ -1068,8 +1093,10 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         // K ranges only until there are two CTAs per SM: more (to even out the 16-row units over the SMs) measured
         // slower (8192 x 8192: 30 -> 33 us)
         const int64_t want_mma = 2 * static_cast<int64_t>(d->sm_count);
+        const int nvb = nvec <= 8 ? 0 : (nvec <= 16 ? 1 : 2);        // blocks of eight vectors per CTA: 1, 2 or 4
+        const int64_t vgroups = (nvec + (8 << nvb) - 1) / (8 << nvb);
         int64_t ks = 1;
-        while (ks < 8 && ks * 2 <= ks_max && blocks * ks < want_mma) ks *= 2;
+        while (ks < 8 && ks * 2 <= ks_max && blocks * vgroups * ks < want_mma) ks *= 2;
         const bool no_wide = opt(SG_OPT_GEMV_NO_WIDE) > 0;
         const bool wide = !no_wide && desc->K % 16 == 0 && (ld * 2) % 32 == 0 && (x_stride * 2) % 32 == 0 &&
                           reinterpret_cast<uintptr_t>(W) % 32 == 0 && reinterpret_cast<uintptr_t>(x) % 32 == 0;
@@ -1083,23 +1110,25 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         if (ctas > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many rows for the matrix-vector path");
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
-        cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
+        if (vgroups > 65535) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many vectors for the matrix-vector path");
+        cfg.gridDim = dim3(static_cast<unsigned>(ctas), static_cast<unsigned>(vgroups), 1);
         cfg.blockDim = dim3(256, 1, 1);
         cfg.stream = cs;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = static_cast<unsigned>(ks);
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // (the kernel waits for its predecessor itself)
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = opt(SG_OPT_NO_PDL) > 0 ? 1 : 2;
         using GemvMmaFn = void (*)(const GemvParams);
         static const GemvMmaFn table[2][2][3] = {
             {{gemv_mma_kernel<__nv_bfloat16, false, 1>, gemv_mma_kernel<__nv_bfloat16, false, 2>, gemv_mma_kernel<__nv_bfloat16, false, 4>},
              {gemv_mma_kernel<__nv_bfloat16, true, 1>, gemv_mma_kernel<__nv_bfloat16, true, 2>, gemv_mma_kernel<__nv_bfloat16, true, 4>}},
             {{gemv_mma_kernel<__half, false, 1>, gemv_mma_kernel<__half, false, 2>, gemv_mma_kernel<__half, false, 4>},
              {gemv_mma_kernel<__half, true, 1>, gemv_mma_kernel<__half, true, 2>, gemv_mma_kernel<__half, true, 4>}}};
-        const int nvb = nvec <= 8 ? 0 : (nvec <= 16 ? 1 : 2);        // blocks of eight vectors: 1, 2 or 4
         cudaError_t e = cudaLaunchKernelEx(&cfg, table[desc->in_dtype == SG_F16 ? 1 : 0][wide ? 1 : 0][nvb], gp);
         if (e != cudaSuccess) return fail(SG_ERR_CUDA, "matrix-vector (MMA) kernel launch: %s", cudaGetErrorString(e));
         g_launches.fetch_add(1);
@@ -1110,7 +1139,7 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         t_last_plan[2] = -static_cast<int32_t>(ks);
         t_last_plan[3] = 16;
         t_last_plan[4] = 0;
-        t_last_plan[5] = static_cast<int32_t>(ctas);
+        t_last_plan[5] = static_cast<int32_t>(ctas * vgroups);
         return SG_OK;
     }
     // Geometry: at least two CTAs per SM where the problem has that much work; K ranges (CTAs of one cluster, at

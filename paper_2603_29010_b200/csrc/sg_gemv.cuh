@@ -25,11 +25,13 @@ struct GemvParams {
     const void* C;        // residual (output type) or null
     const void* bias;     // input type (fp32 for fp32 inputs) or null
     void* D;
+    const uint32_t* status;   // the library's device status word: while it is set (an expired wait of an earlier launch,
+                              // not yet reported by sg_poll_status) nothing is stored
     int64_t ld;           // elements between rows of W
     int64_t x_stride;
     int64_t c_row_stride, c_vec_stride, d_row_stride, d_vec_stride;   // element (row r, vector v) of C and D
     int32_t R, K;
-    int32_t nvec;         // 1..32 (gemv_kernel: 1..4)
+    int32_t nvec;         // gemv_kernel: 1..4; gemv_mma_kernel: any number, in groups of 8, 16 or 32 along gridDim.y
     int32_t kchunk;       // K elements per cluster rank (a multiple of 256 vectors)
     int32_t ksplit;       // CTAs per cluster
     int32_t bias_row_stride, bias_vec_stride;   // (0, 1): one bias per vector (the matrix is A); (1, 0): one per row
@@ -112,6 +114,12 @@ __global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4 && NV == 1) ? 
     constexpr int NACC = RB * NV;
     __shared__ float warp_part[WARPS][NACC];
     __shared__ float cta_part[NACC];
+    // Programmatic dependent launch: the CTAs of this launch may become resident while the previous kernel of the stream
+    // is still finishing; nothing of global memory is touched before that kernel has completed.
+    grid_dependency_wait();
+    grid_launch_dependents();
+    // fetched now, looked at before the stores at the very end: the load's latency hides behind the sweep
+    const uint32_t sticky = p.status != nullptr ? *reinterpret_cast<const volatile uint32_t*>(p.status) : 0u;
 
     const int ks = p.ksplit;
     const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));      // = rank in the (ks, 1, 1) cluster
@@ -209,7 +217,7 @@ __global__ void __launch_bounds__(256, (sizeof(T) == 2 && RB == 4 && NV == 1) ? 
             if (p.bias != nullptr)
                 v[0] += GemvVec<T>::exact(reinterpret_cast<const T*>(p.bias) + row * p.bias_row_stride + vec * p.bias_vec_stride);
             if (p.epi >= EPI_RELU) apply_act_chunk<false, 1>(v, p.epi, p.a0, p.a1);
-            gemv_store_out(p.D, row * p.d_row_stride + vec * p.d_vec_stride, p.out_kind, v[0]);
+            if (!sticky) gemv_store_out(p.D, row * p.d_row_stride + vec * p.d_vec_stride, p.out_kind, v[0]);
         }
     }
     if (ks > 1) cg::this_cluster().sync();      // keep every rank's shared memory alive until rank 0 has read it
@@ -266,7 +274,9 @@ __device__ __forceinline__ U8 ldg_cached32(const void* p) {
 // kWide = true: 32-byte pieces; requires K % 16 == 0, kchunk % 512 == 0 and 32-byte aligned rows and vectors.
 // NVB: blocks of eight vectors (1, 2 or 4: up to 8, 16 or 32 vectors).  Every block is one more MMA per piece of W on
 // the same A fragment and four more accumulator registers; thread group g loads vectors g, g + 8, g + 16, g + 24.
-// Grid: ceil(R / 16) row blocks x ksplit ranks.
+// Grid: x = ceil(R / 16) row blocks x ksplit ranks; y = groups of 8 NVB vectors (more than one group: a small GEMM whose
+// every CTA reads 16 rows of one operand and 8 NVB rows of the other once -- no shared-memory staging, no tensor
+// memory, one memory round trip: what a product of a few hundred rows and columns needs is latency, not tiles).
 template <typename T, bool kWide, int NVB = 1>
 __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     namespace cg = cooperative_groups;
@@ -277,6 +287,12 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     constexpr int NV = 8 * NVB;               // vector slots
     __shared__ float warp_part[WARPS][16 * NV];   // 16 rows x NV vectors per warp
     __shared__ float cta_part[16 * NV];
+    // Programmatic dependent launch: the CTAs of this launch may become resident while the previous kernel of the stream
+    // is still finishing; nothing of global memory is touched before that kernel has completed.
+    grid_dependency_wait();
+    grid_launch_dependents();
+    // fetched now, looked at before the stores at the very end: the load's latency hides behind the sweep
+    const uint32_t sticky = p.status != nullptr ? *reinterpret_cast<const volatile uint32_t*>(p.status) : 0u;
 
     const int ks = p.ksplit;
     const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));
@@ -285,6 +301,7 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     const int kend = min(p.K, kbeg + p.kchunk);
     const int warp = static_cast<int>(threadIdx.x) >> 5, lane = static_cast<int>(threadIdx.x) & 31;
     const int g = lane >> 2, t = lane & 3;
+    const int v0 = static_cast<int>(blockIdx.y) * NV;        // first vector of this CTA's group
 
     const T* wlo = reinterpret_cast<const T*>(p.W) + min(r0 + g, static_cast<int64_t>(p.R) - 1) * p.ld;
     const T* whi = reinterpret_cast<const T*>(p.W) + min(r0 + g + 8, static_cast<int64_t>(p.R) - 1) * p.ld;
@@ -292,7 +309,7 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     float c[NVB][4];
 #pragma unroll
     for (int j = 0; j < NVB; ++j) {
-        xv[j] = reinterpret_cast<const T*>(p.x) + static_cast<int64_t>(min(g + 8 * j, p.nvec - 1)) * p.x_stride;
+        xv[j] = reinterpret_cast<const T*>(p.x) + static_cast<int64_t>(min(v0 + g + 8 * j, p.nvec - 1)) * p.x_stride;
         c[j][0] = c[j][1] = c[j][2] = c[j][3] = 0.0f;
     }
 
@@ -403,14 +420,14 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
             for (int r = 1; r < ks; ++r) s += *cluster.map_shared_rank(&cta_part[i], r);
         }
         const int64_t row = r0 + i / NV;
-        const int vec = i % NV;
+        const int vec = v0 + i % NV;
         if (row < p.R && vec < p.nvec) {
             float v[1] = {p.alpha * s};
             if (p.beta != 0.0f) v[0] = fmaf(p.beta, gemv_load_out(p.C, row * p.c_row_stride + vec * p.c_vec_stride, p.out_kind), v[0]);
             if (p.bias != nullptr)
                 v[0] += GemvVec<T>::exact(reinterpret_cast<const T*>(p.bias) + row * p.bias_row_stride + vec * p.bias_vec_stride);
             if (p.epi >= EPI_RELU) apply_act_chunk<false, 1>(v, p.epi, p.a0, p.a1);
-            gemv_store_out(p.D, row * p.d_row_stride + vec * p.d_vec_stride, p.out_kind, v[0]);
+            if (!sticky) gemv_store_out(p.D, row * p.d_row_stride + vec * p.d_vec_stride, p.out_kind, v[0]);
         }
     }
     if (ks > 1) cg::this_cluster().sync();

@@ -27,6 +27,8 @@ CFG = inputs.CONFIGS
 @pytest.fixture(autouse=True)
 def _clean_status():
     sg.set_tuning(-1, -1)
+    sg.set_option("gemv_small_log2", -1)      # the launch configuration bench.py times: the library's own choice of path
+    sg.set_option("gemv_max_vectors", -1)
     yield
     torch.cuda.synchronize()
     sg.poll_status()
@@ -68,7 +70,14 @@ def test_c1_gemm_256_every_element():
     A, B, _ = inputs.make_gemm(c["M"], c["N"], c["K"], c["dist"], c["scale"])
     ref, absacc = orc.gemm(A, B)
     D = sg.gemm(A.to(DEV), B.to(DEV))
+    assert "gemv_mma_kernel" in sg.last_kernel_name()      # (a product this small runs on the warp-level MMA kernel)
     parity.assert_matches(D, ref, absacc, "c1")
+    assert_tight(D, ref, absacc, "c1")
+    # and through the tensor-core tiles, which a forced tile shape keeps it on
+    sg.set_tuning(64, 0)
+    D = sg.gemm(A.to(DEV), B.to(DEV))
+    assert "contract_kernel" in sg.last_kernel_name()
+    parity.assert_matches(D, ref, absacc, "c1 on the tiles")
 
 
 @pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])

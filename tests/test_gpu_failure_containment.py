@@ -128,3 +128,33 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_exact(tile_n, pai
         torch.cuda.synchronize()
         sg.poll_status()
         parity.assert_bit_exact(D3, ref, "after a timed-out launch")
+
+
+def test_matrix_vector_and_small_product_kernels_store_nothing_while_the_word_is_set():
+    sg.set_option("gemv_small_log2", -1)              # the library's own choice of path
+    sg.set_option("gemv_max_vectors", -1)
+    W = inputs.small_integers([1000, 520], 921, 1)
+    X = inputs.small_integers([3, 520], 921, 2)       # three vectors: the matrix-vector kernels
+    A = inputs.small_integers([256, 264], 922, 1)
+    B = inputs.small_integers([200, 264], 922, 2)     # a small product: the warp-level MMA kernel with groups of vectors
+    dW, dX, dA, dB = W.to(DEV), X.to(DEV), A.to(DEV), B.to(DEV)
+
+    def run_all():
+        Dv = torch.full((3, 1000), NAN, dtype=torch.float32, device=DEV)
+        Ds = torch.full((256, 200), NAN, dtype=torch.float32, device=DEV)
+        sg.gemm(dX, dW, out=Dv)
+        assert sg.last_launch_plan()["tile_n"] == 0
+        sg.gemm(dA, dB, out=Ds)
+        assert sg.last_launch_plan()["tile_n"] == 0 and "gemv_mma_kernel" in sg.last_kernel_name()
+        torch.cuda.synchronize()
+        return Dv, Ds
+
+    torch.cuda.synchronize()
+    sg.test_set_status_word((3 << 24) | 5)
+    Dv, Ds = run_all()
+    assert bool(torch.isnan(Dv).all()) and bool(torch.isnan(Ds).all())
+    _expect_timeout()
+    Dv, Ds = run_all()
+    parity.assert_bit_exact(Dv, orc.gemm(X, W)[0], "vectors after the poll")
+    parity.assert_bit_exact(Ds, orc.gemm(A, B)[0], "small product after the poll")
+    sg.poll_status()

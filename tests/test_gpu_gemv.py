@@ -19,12 +19,14 @@ DEV = "cuda"
 @pytest.fixture(autouse=True)
 def _clean_status():
     sg.set_tuning(-1, -1)
-    sg.set_option("gemv_max_vectors", -1)
+    sg.set_option("gemv_max_vectors", -1)        # this module tests the library's own choice of path
+    sg.set_option("gemv_small_log2", -1)
     sg.set_option("no_gemv", -1)
     yield
     torch.cuda.synchronize()
     sg.poll_status()
     sg.set_option("gemv_max_vectors", -1)
+    sg.set_option("gemv_small_log2", -1)
     sg.set_option("no_gemv", -1)
 
 
@@ -151,6 +153,7 @@ def test_results_do_not_depend_on_the_run():
 
 def test_other_forms_still_go_through_the_tiles():
     g = torch.Generator().manual_seed(4)
+    sg.set_option("gemv_small_log2", 0)           # (a product this small would otherwise go to the MMA kernel whole)
     A = torch.randn(256, 64, generator=g).to(torch.bfloat16)
     B33 = torch.randn(33, 64, generator=g).to(torch.bfloat16)
     out = torch.empty(256, 40, dtype=torch.bfloat16, device=DEV)
@@ -178,6 +181,7 @@ def test_few_rows_against_a_large_matrix_on_the_tiles(M, dtype):
     # 9..64 rows: the tensor-core tiles with only 32 or 64 rows of A loaded per stage; 65: the full A tile
     # (a matrix this small would go to the matrix-vector kernels with up to 32 rows: keep those to eight vectors here)
     sg.set_option("gemv_max_vectors", 8)
+    sg.set_option("gemv_small_log2", 0)
     g = torch.Generator().manual_seed(100 + M)
     N, K = 1080, 2056
     A = (torch.randn(M, K, generator=g) / 8).to(dtype)
@@ -282,3 +286,56 @@ def test_many_vectors_match_the_tiles_bit_for_bit_on_integers():
     sg.set_option("no_gemv", -1)
     assert not _took_vector_path()
     assert torch.equal(a, b)
+
+
+SMALL = [(256, 256, 256), (128, 128, 128), (300, 200, 136), (129, 72, 8), (384, 384, 1024), (64, 64, 4096), (512, 64, 512),
+         (33, 77, 4104), (100, 100, 2048), (40, 1000, 264)]
+
+
+@pytest.mark.parametrize("M,N,K", SMALL)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_small_products_run_on_the_mma_kernel(M, N, K, dtype):
+    # groups of 32 rows of the operand with fewer rows along the grid's second dimension: a small GEMM without tiles
+    g = torch.Generator().manual_seed(M + N + K)
+    A = (torch.randn(M, K, generator=g) / 8).to(dtype)
+    B = (torch.randn(N, K, generator=g) / 8).to(dtype)
+    C = torch.randn(M, N, generator=g).to(dtype)
+    bias = torch.randn(N, generator=g).to(dtype)
+    ref, absacc = orc.gemm(A, B, C=C, bias=bias, alpha=0.75, beta=0.5, epi="gelu")
+    whole = torch.full((M + 4, (N + 15) // 8 * 8), float("nan"), dtype=dtype, device=DEV)
+    out = whole[2:2 + M, :N]
+    sg.gemm(A.to(DEV), B.to(DEV), C=C.to(DEV), bias=bias.to(DEV), alpha=0.75, beta=0.5, epi="gelu", out=out)
+    assert _took_vector_path() and "gemv_mma_kernel" in sg.last_kernel_name(), sg.last_kernel_name()
+    parity.assert_matches(out, ref, absacc, f"small product {M}x{N}x{K} {dtype}")
+    assert bool(torch.isnan(whole[:2]).all()) and bool(torch.isnan(whole[2 + M:]).all()) and bool(torch.isnan(whole[:, N:]).all())
+    # exact on small integers, fp32 out; and the same bits as the tiles give
+    Ai = inputs.small_integers([M, K], 97, 1, lo=-2, hi=2).to(dtype)
+    Bi = inputs.small_integers([N, K], 97, 2, lo=-2, hi=2).to(dtype)
+    refi, _ = orc.gemm(Ai, Bi)
+    Di = sg.gemm(Ai.to(DEV), Bi.to(DEV), out_dtype=torch.float32)
+    assert _took_vector_path()
+    parity.assert_bit_exact(Di, refi, f"small integer product {M}x{N}x{K} {dtype}")
+    sg.set_option("gemv_small_log2", 0)
+    sg.set_option("gemv_max_vectors", 8)
+    Dt = torch.empty(M, (N + 7) // 8 * 8, dtype=torch.float32, device=DEV)[:, :N]      # (the tiles want 16-byte row pitches)
+    sg.gemm(Ai.to(DEV), Bi.to(DEV), out=Dt)
+    assert not _took_vector_path() or min(M, N) <= 8
+    assert torch.equal(Di, Dt)
+
+
+def test_products_too_large_for_the_small_form_use_the_tiles():
+    for M, N, K in [(512, 512, 512), (256, 1024, 256), (400, 400, 400), (256, 256, 4096)]:
+        A = torch.zeros(M, K, dtype=torch.bfloat16, device=DEV)
+        B = torch.zeros(N, K, dtype=torch.bfloat16, device=DEV)
+        sg.gemm(A, B)
+        assert not _took_vector_path(), (M, N, K)
+
+
+def test_forced_tile_shapes_keep_small_products_on_the_tiles():
+    A = torch.zeros(256, 256, dtype=torch.bfloat16, device=DEV)
+    sg.set_tuning(64, 0)
+    sg.gemm(A, A)
+    assert not _took_vector_path()
+    sg.set_tuning(-1, -1)
+    sg.gemm(A, A)
+    assert _took_vector_path()

@@ -28,11 +28,15 @@ EPIS = ["none", "none", "relu", "gelu", "silu", "sigmoid", "tanh", "hardswish"]
 EDGE = [1, 2, 7, 8, 31, 32, 33, 63, 64, 65, 127, 128, 129, 191, 255, 256, 257, 300, 383, 511, 513]
 
 
-@pytest.fixture(autouse=True)
-def _clean_status():
+@pytest.fixture(autouse=True, params=["tiles", "own choice"])
+def _clean_status(request):
+    # every case twice: on the tensor-core tiles (the matrix-vector kernels kept to eight vectors, no small-product form),
+    # and under the library's own choice of path
     sg.set_tuning(-1, -1)
     sg.set_tail_mode(-1)
     sg.enable_scratch(True)
+    sg.set_option("gemv_small_log2", 0 if request.param == "tiles" else -1)
+    sg.set_option("gemv_max_vectors", 8 if request.param == "tiles" else -1)
     yield
     torch.cuda.synchronize()
     sg.poll_status()
