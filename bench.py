@@ -313,6 +313,8 @@ def bench_per_config(sg, inputs, sharding, torch, dist, dev, peaks, rank: int, w
             times, launches, graph = time_graph_repeats(w["fns"], torch, w["launches"], repeats)
             mhz = sg.last_kernel_clock_mhz()
             plan, kernel = sg.last_launch_plan(), sg.last_kernel_name()
+            if "contract_kernel" not in kernel:
+                mhz = 0.0                      # only the contraction kernel counts its own clock
             del graph
             # the warm regime: the same launch on ONE buffer set, back to back (operands the L2 can hold stay there)
             warm_times, _, graph = time_graph_repeats([w["fns"][0]] * min(8, max(2, len(w["fns"]))), torch, w["launches"], 5)
@@ -345,7 +347,7 @@ def bench_per_config(sg, inputs, sharding, torch, dist, dev, peaks, rank: int, w
                "bound": "tensor" if sol_m["compute_bound"] else "hbm",
                "t_sol_measured_us": sol_m["t_sol_s"] * 1e6, "frac_of_sol_measured": sol_m["t_sol_s"] / med / (world if copies == 1 else 1),
                "t_sol_spec_us": sol_s["t_sol_s"] * 1e6, "frac_of_sol_spec": sol_s["t_sol_s"] / med / (world if copies == 1 else 1),
-               "sm_mhz_in_kernel": round(mhz, 1), "tiling": plan, "kernel": kernel, "buffer_sets": len(w["fns"]),
+               "sm_mhz_in_kernel": round(mhz, 1) if mhz else None, "tiling": plan, "kernel": kernel, "buffer_sets": len(w["fns"]),
                "partition": w["partition"] if world > 1 else "whole problem",
                "timing": "CUDA graph of one launch per buffer set (sets exceed L2), replayed for ~3 ms after 30 ms idle; us = median, us_best = best of the repeats; "
                          "us_warm_l2 = the same protocol on one buffer set (median of 5): context, never the reported number"}
