@@ -10,6 +10,8 @@ store -- over one batch: a single ``sg_gemm`` launch of the GEMM 4096^3 + bias +
 * ``value``      TFLOP/s of the whole job (all ranks), operands resident in HBM, CUDA-event timed,
                  max over ranks; every step uses the next of several distinct buffer sets whose total
                  size exceeds the 126 MB L2, so no step finds its operands left in L2 by the step before.
+                 The K timed steps are the K kernel nodes of one CUDA graph (one untimed replay, then the timed
+                 one); ``ms_per_step_plain_launches`` is the same K steps launched one by one.
 * ``e2e``        the same metric through the public API with pinned HOST buffers: H2D of A, B, bias,
                  the kernel, and D2H of D inside the timed region.
 * ``roofline``   the kernel's achieved TFLOP/s against the measured dense-bf16 peak of this machine.
@@ -695,21 +697,32 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     barrier()
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
+    # The K timed steps are one CUDA graph (K kernel nodes, one per step, each on the next buffer set), replayed once
+    # untimed (the upload) and once timed; the same K steps as plain launches are timed first and reported beside it.
+    dt_plain = time_steps(step, args.steps, torch)
+    barrier()
     launches0 = sg.launch_count()
+    timed_graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(timed_graph):
+        for i in range(args.steps):
+            step(i)
+    launches = sg.launch_count() - launches0      # kernel nodes of the graph = launches of the timed region
+    plan = sg.last_launch_plan()                 # of the timed launches (read before anything else is launched)
+    kernel_name = sg.last_kernel_name()
+    timed_graph.replay()
+    barrier()
     torch.cuda.profiler.start()            # lets `ncu --profile-from-start off` see the timed region only
-    dt = time_steps(step, args.steps, torch)
+    dt = time_steps(lambda i: timed_graph.replay(), 1, torch)
     torch.cuda.profiler.stop()
     sampler.sample_once()
     kernel_mhz = sg.last_kernel_clock_mhz()      # cycle counter / ns timer inside the last timed kernel
-    launches = sg.launch_count() - launches0
-    plan = sg.last_launch_plan()                 # of the timed launches (read before anything else is launched)
-    kernel_name = sg.last_kernel_name()
     barrier()
     clocks = sampler.stop()
     clocks["sm_mhz_in_kernel"] = round(kernel_mhz, 1)
     clocks["note"] = "sm_mhz is the management library's figure (on this pool: the requested clock); sm_mhz_in_kernel is counted inside the timed kernel"
     sg.poll_status()
     dt = max_over_ranks(dt)
+    dt_plain = max_over_ranks(dt_plain)
 
     # ---- burst and sustained, side by side (one GPU's figure; every rank runs it so that the GPUs stay in step)
     burst, sustained_rec = None, None
@@ -802,11 +815,14 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         "config": {"workload": WORKLOAD, "M": M, "N": N, "K": K, "layout": "A row-major, B column-major",
                    "epilogue": "bias+relu", "accumulate": "fp32", "out": "bf16",
                    "l2": f"inputs larger than L2: {sets} distinct buffer sets ({sets * footprint / 1e6:.0f} MB) used in turn",
+                   "launch": "the K timed steps are the K kernel nodes of one CUDA graph (replayed once untimed, once timed, CUDA "
+                             "events around the timed replay); ms_per_step_plain_launches is the same K steps as plain launches",
                    "per_gpu": "value: every rank runs the whole problem on its own GPU (no collective); per_config: every "
                               "rank runs its shard of each problem (rows / batch entries / images / whole groups)"},
         "clocks": clocks,
         "e2e": {"value": world * flops / (dt_e2e / e2e_steps) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": dt_e2e / e2e_steps * 1e3},
+        "ms_per_step_plain_launches": dt_plain / args.steps * 1e3,
         "gpu_launches": launches,
         "kernels_in_timed_region": {
             "names": [kernel_name], "launches": launches, "one_launch_per_step": bool(launches == args.steps),
