@@ -115,16 +115,16 @@ typedef struct sg_gemm_desc {
  *   D      device, out_dtype, [M,N] row-major; written in full (all M x N elements).
  * M == 0 or N == 0: SG_OK, nothing is launched.  K == 0: D = act(beta*C + bias).
  * Matrix-vector form (the workload list's single-token decode product): when N <= 8 (or M <= 8; 4 for SG_F32 inputs or
- *   when K is no multiple of 8; also 9..32 for 16-bit inputs against a matrix of at most 48 MB, 12 MB from 17 vectors
- *   on, where the tiles' fixed cost would decide the time), the matrix operand is
+ *   when K is no multiple of 8; also 9..32 for 16-bit inputs against a matrix of at most 48 MB and few enough rows that
+ *   the groups of eight vectors are all resident at once), the matrix operand is
  *   K-contiguous (A row-major, resp. B column-major) and 16-byte aligned with a leading dimension that is a multiple
  *   of 16 bytes, the vectors are K-contiguous, 16-byte aligned and a multiple of 16 bytes apart (a single vector may
  *   also be stored as K x 1 with a leading dimension of 1), and in_dtype is SG_BF16, SG_F16 or SG_F32, the product
  *   runs as one pass over the matrix at HBM speed instead of through tensor-core tiles.  In that form ldc and ldd may
  *   be any value >= N (no 16-byte rule) and C, D and bias need only their element alignment; results are reproducible
  *   from run to run.  A small product of 16-bit K-contiguous operands (at most 160 M multiply-adds, and few enough
- *   outputs that one CTA per 16 x 32 of them fits on the GPU at once) runs on the same kernels, in groups of 32 vectors,
- *   for their shorter start and end; a tile shape forced through sg_set_tuning keeps it on the tiles.
+ *   outputs that one CTA per 16 x 8, 16 x 16 or 16 x 32 of them fits on the GPU at once) runs on the same kernels, in
+ *   groups of vectors, for their shorter start and end; a tile shape forced through sg_set_tuning keeps it on the tiles.
  */
 sg_status_t sg_gemm(const sg_gemm_desc_t* desc, const void* A, const void* B, const void* C,
                     const void* bias, void* D, void* cuda_stream);
@@ -443,7 +443,8 @@ typedef enum {
     SG_OPT_SPLIT_K_REDUCE_WARPS = 16, /* second pass of a two-pass K split: 1, 2, 4 or 8 warps share the parts of a column slice */
     SG_OPT_GEMV_MAX_VECTORS = 17, /* most vectors (4..32) the matrix-vector kernels take before the tiles do; default 32 */
     SG_OPT_GEMV_SMALL_LOG2 = 18,  /* products of at most 2^value multiply-adds (16-bit operands) run on the warp-level MMA kernel; 0 = none */
-    SG_OPT_COUNT_ = 19
+    SG_OPT_GEMV_VECTOR_BLOCKS = 19, /* blocks of eight vectors a CTA of the warp-level MMA kernel takes: 1, 2 or 4 */
+    SG_OPT_COUNT_ = 20
 } sg_option_t;
 sg_status_t sg_set_option(int32_t option, int64_t value);
 

@@ -994,30 +994,51 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     if (desc->in_dtype != SG_BF16 && desc->in_dtype != SG_F16 && desc->in_dtype != SG_F32) return SG_OK;
     const int es = desc->in_dtype == SG_F32 ? 4 : 2;
     const bool no_mma = opt(SG_OPT_GEMV_NO_MMA) > 0;      // FMA kernel only (<= 4 vectors)
-    const int64_t mma_vec = opt(SG_OPT_GEMV_MAX_VECTORS) > 0 ? std::min<int64_t>(32, opt(SG_OPT_GEMV_MAX_VECTORS)) : 32;
-    const int64_t max_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? std::max<int64_t>(mma_vec, 4) : 4;
-    // A small product of 16-bit operands runs on the same warp-level MMA kernel with the vectors in groups of 32 along the
-    // grid's second dimension: it is bound by launch and memory latency, which that kernel has less of than the tiles (no
-    // tensor-memory allocation, no barrier set-up, no shared-memory staging, no TMA store).  It pays while all its CTAs
-    // (16 x 32 outputs each) are resident at once and the K loop is short: measured against the tiles, 256^3 2.75 against
-    // 3.6 us, 128^3 2.2 / 3.2, 384^3 3.4 / 4.1, 256 x 256 x 1024 3.9 / 6.5, 256 x 256 x 2048 5.8 / 7.9, 384 x 384 x 1024
-    // 4.6 / 6.5, 64 x 64 x 4096 5.3 / 6.9, 512 x 64 x 512 3.0 / 4.5 -- but 400^3 5.4 / 4.5, 512^3 6.3 / 4.5, 512 x 512 x 128
-    // 5.0 / 3.3, 256 x 1024 x 256 7.0 / 3.7 (more CTAs than fit) and 256 x 256 x 4096 11.6 / 10.4, 160 x 160 x 8192 12.3 / 9.6
-    // (long K).  Taken up to two CTAs per SM and 160 M multiply-adds (SG_OPT_GEMV_SMALL_LOG2 pins the second limit and
-    // lifts the first).
+    // More than eight vectors (16-bit operands, K % 8 == 0) run on the same warp-level MMA kernel in GROUPS of 8, 16 or 32
+    // vectors along the grid: a CTA takes 16 rows of the operand with more rows ("the matrix") and one group of rows of
+    // the other, straight from the L2 into MMA fragments -- one memory round trip, no tensor-memory allocation, no
+    // barrier set-up, no staging, no TMA store -- and the CTAs that share 16 rows of the matrix are neighbours in launch
+    // order.  That has less start and end than the tiles and, with groups of eight, as many loads of the matrix in
+    // flight as the plain matrix-vector form; it pays as long as all CTAs are resident at once (4, 3 or 2 per SM for
+    // groups of 8, 16 or 32: registers), beyond which the tiles' operand reuse wins.  Measured against the tiles (us):
+    //   nine to 32 rows against a matrix, groups of 8: 9 x 4096 x 4096 10.2 / 19.3, 16 x 4096 x 4096 10.2 / 14.6,
+    //   24 x 3072 x 3072 7.9 / 12.2, 32 x 2048 x 2048 5.7 / 10.0, 24 x 2048 x 4096 8.4 / 11.9, 32 x 1024 x 8192 9.9 / 11.3,
+    //   16 x 1024 x 1024 2.9 / 6.0 -- but (more CTAs than fit) 32 x 4096 x 4096 15.4 / 15.2, 16 x 8192 x 4096 17.9 / 16.5,
+    //   20 x 8192 x 2048 13.4 / 10.2, 16 x 8192 x 8192 31.5 / 28.6;
+    //   small products, the smallest group size that fits: 256^3 2.7-2.9 / 3.6, 128^3 1.8 / 3.2, 384^3 3.4 / 4.1,
+    //   256 x 256 x 1024 3.9-4.1 / 6.5, 256 x 256 x 2048 5.1 / 7.9, 384 x 384 x 1024 4.6 / 6.5, 64 x 64 x 4096 4.0 / 7.0,
+    //   512 x 64 x 512 2.5 / 4.5 -- but 400^3 5.4 / 4.5, 512^3 6.5 / 4.5, 512 x 512 x 128 5.2 / 3.3, 256 x 1024 x 256
+    //   6.5 / 3.7 (more CTAs than fit) and 256 x 256 x 4096 11.6 / 10.4, 160 x 160 x 8192 12.3 / 9.6 (long K: taken up to
+    //   160 M multiply-adds; SG_OPT_GEMV_SMALL_LOG2 pins that limit and lifts the residency rule).
+    // A tile shape forced through sg_set_tuning keeps a product on the tiles; SG_OPT_GEMV_MAX_VECTORS > 0 restores the
+    // plain limit on the number of vectors and nothing else.
     const bool small_forced = opt(SG_OPT_GEMV_SMALL_LOG2) >= 0;
     const double small_macs = small_forced ? std::ldexp(1.0, static_cast<int>(std::min<int64_t>(40, opt(SG_OPT_GEMV_SMALL_LOG2)))) : kGemvSmallMacs;
-    // (16 rows of the operand with more rows x 32 rows of the other per CTA, two CTAs per SM)
-    const int64_t small_ctas = ((std::max(desc->M, desc->N) + 15) / 16) * ((std::min(desc->M, desc->N) + 31) / 32);
-    bool small = es == 2 && !no_mma && desc->K % 8 == 0 && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0 &&
-                 g_tune_tile_n.load() <= 0 && g_tune_pair.load() < 0 &&      // (a forced tile shape means the tiles)
-                 static_cast<double>(desc->M) * static_cast<double>(desc->N) * static_cast<double>(desc->K) <= small_macs;
-    if (small && !small_forced) {
+    const bool groups_ok = es == 2 && !no_mma && desc->K % 8 == 0 && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0 &&
+                           g_tune_tile_n.load() <= 0 && g_tune_pair.load() < 0;
+    const int64_t few = std::min(desc->M, desc->N), many = std::max(desc->M, desc->N);
+    int group_blocks = 0;            // 1, 2 or 4 blocks of eight vectors per CTA when the grouped form is taken
+    if (groups_ok && few > 8) {
+        const bool is_small = static_cast<double>(desc->M) * static_cast<double>(desc->N) * static_cast<double>(desc->K) <= small_macs;
+        const bool few_rows = few <= 32 && static_cast<double>(many) * static_cast<double>(desc->K) * es <= 48.0e6;
         DeviceState* ds = nullptr;
-        small = device_state(&ds) == SG_OK && ds && small_ctas <= 2 * static_cast<int64_t>(ds->sm_count);
+        if ((is_small || few_rows) && device_state(&ds) == SG_OK && ds) {
+            const int64_t row_blocks = (many + 15) / 16;
+            const int per_sm[3] = {4, 3, 2};
+            // (groups of 32 only with the 32-byte row pieces: with 16-byte pieces they measured slower than the tiles)
+            const bool wide_ok = desc->K % 16 == 0 && (desc->lda * 2) % 32 == 0 && (desc->ldb * 2) % 32 == 0;
+            for (int b = 0; b < 3 && !group_blocks; ++b) {
+                if (!is_small && b > 0) break;           // a few rows against a matrix: groups of eight or the tiles
+                if (b == 2 && !wide_ok && !small_forced) break;
+                const int64_t ctas = row_blocks * ((few + (8 << b) - 1) / (8 << b));
+                if (ctas <= per_sm[b] * static_cast<int64_t>(ds->sm_count) || (small_forced && is_small && b == 2)) group_blocks = 1 << b;
+            }
+        }
     }
-    const bool mat_a = small ? desc->M >= desc->N : (desc->N <= max_vec && desc->M >= desc->N);
-    if (!small && !mat_a && desc->M > max_vec) return SG_OK;
+    const bool grouped = group_blocks > 0;
+    const int64_t plain_vec = (es == 2 && !no_mma && desc->K % 8 == 0) ? (opt(SG_OPT_GEMV_MAX_VECTORS) > 0 ? std::max<int64_t>(4, std::min<int64_t>(32, opt(SG_OPT_GEMV_MAX_VECTORS))) : 8) : 4;
+    const bool mat_a = grouped ? desc->M >= desc->N : (desc->N <= plain_vec && desc->M >= desc->N);
+    if (!grouped && !mat_a && desc->M > plain_vec) return SG_OK;
     // the matrix K-contiguous, the vectors contiguous (a K x 1 row-major B with ldb = 1 is as good as a column-major one)
     const bool a_kc = desc->layout_a == SG_ROW_MAJOR, b_kc = desc->layout_b == SG_COL_MAJOR;
     const void* W = mat_a ? A : B;
@@ -1029,14 +1050,6 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
     if (mat_a ? !(a_kc && (b_kc || (nvec == 1 && desc->ldb == 1))) : !(b_kc && (a_kc || (nvec == 1 && desc->lda == 1)))) return SG_OK;
     if (R > INT32_MAX || ld < desc->K || (ld * es) % 16 || !W || !x || !aligned16(W) || !aligned16(x)) return SG_OK;
     if (nvec > 1 && (x_stride < desc->K || (x_stride * es) % 16)) return SG_OK;
-    if (nvec > 8 && !small && opt(SG_OPT_GEMV_MAX_VECTORS) <= 0) {
-        // Nine to 32 vectors: every CTA re-reads its K range of all vectors from the L2 and holds fewer matrix loads in
-        // flight, so the stream over a large matrix is slower than the tiles' (16 x 8192 x 8192: 33 against 28 us); what
-        // this path saves is the tiles' fixed cost, which decides small problems (16 x 1024 x 1024: 2.6 against 6.4 us,
-        // 32 x 2048 x 2048: 6.7 against 10.2, 12 x 4096 x 4096: 13.5 against 20.5).  Measured crossovers:
-        const double w_bytes = static_cast<double>(R) * static_cast<double>(desc->K) * es;
-        if (w_bytes > (nvec <= 16 ? 48.0e6 : 12.0e6)) return SG_OK;
-    }
     *taken = true;
 
     Checked c;
@@ -1093,10 +1106,19 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         // K ranges only until there are two CTAs per SM: more (to even out the 16-row units over the SMs) measured
         // slower (8192 x 8192: 30 -> 33 us)
         const int64_t want_mma = 2 * static_cast<int64_t>(d->sm_count);
-        const int nvb = nvec <= 8 ? 0 : (nvec <= 16 ? 1 : 2);        // blocks of eight vectors per CTA: 1, 2 or 4
+        // blocks of eight vectors per CTA: the grouped form's choice; else (a pinned vector limit) as few as hold them all
+        int nvb = grouped ? (group_blocks == 1 ? 0 : (group_blocks == 2 ? 1 : 2)) : (nvec <= 8 ? 0 : (nvec <= 16 ? 1 : 2));
+        if (opt(SG_OPT_GEMV_VECTOR_BLOCKS) == 1 || opt(SG_OPT_GEMV_VECTOR_BLOCKS) == 2 || opt(SG_OPT_GEMV_VECTOR_BLOCKS) == 4)
+            nvb = opt(SG_OPT_GEMV_VECTOR_BLOCKS) == 1 ? 0 : (opt(SG_OPT_GEMV_VECTOR_BLOCKS) == 2 ? 1 : 2);
         const int64_t vgroups = (nvec + (8 << nvb) - 1) / (8 << nvb);
         int64_t ks = 1;
-        while (ks < 8 && ks * 2 <= ks_max && blocks * vgroups * ks < want_mma) ks *= 2;
+        if (vgroups > 1) {
+            // several groups: K ranges only while all CTAs stay resident at once
+            const int64_t resident = (nvb == 0 ? 4 : (nvb == 1 ? 3 : 2)) * static_cast<int64_t>(d->sm_count);
+            while (ks < 8 && ks * 2 <= ks_max && blocks * vgroups * ks * 2 <= resident) ks *= 2;
+        } else {
+            while (ks < 8 && ks * 2 <= ks_max && blocks * ks < want_mma) ks *= 2;
+        }
         const bool no_wide = opt(SG_OPT_GEMV_NO_WIDE) > 0;
         const bool wide = !no_wide && desc->K % 16 == 0 && (ld * 2) % 32 == 0 && (x_stride * 2) % 32 == 0 &&
                           reinterpret_cast<uintptr_t>(W) % 32 == 0 && reinterpret_cast<uintptr_t>(x) % 32 == 0;
@@ -1110,8 +1132,10 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
         if (ctas > INT32_MAX) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many rows for the matrix-vector path");
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
-        if (vgroups > 65535) return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many vectors for the matrix-vector path");
-        cfg.gridDim = dim3(static_cast<unsigned>(ctas), static_cast<unsigned>(vgroups), 1);
+        if (vgroups > 65535 || (vgroups > 1 && blocks > 65535))
+            return fail(SG_ERR_UNSUPPORTED, "sg_gemm: too many vectors or rows for the matrix-vector path");
+        cfg.gridDim = vgroups > 1 ? dim3(static_cast<unsigned>(ks), static_cast<unsigned>(vgroups), static_cast<unsigned>(blocks))
+                                  : dim3(static_cast<unsigned>(ctas), 1, 1);
         cfg.blockDim = dim3(256, 1, 1);
         cfg.stream = cs;
         cudaLaunchAttribute attr[2];

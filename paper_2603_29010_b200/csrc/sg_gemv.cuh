@@ -295,8 +295,11 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const GemvParams p) {
     const uint32_t sticky = p.status != nullptr ? *reinterpret_cast<const volatile uint32_t*>(p.status) : 0u;
 
     const int ks = p.ksplit;
-    const int rank = static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));
-    const int64_t r0 = static_cast<int64_t>(blockIdx.x / static_cast<unsigned>(ks)) * 16;
+    // x = row blocks x ranks with one group of vectors; with several groups x = ranks, y = groups, z = row blocks, so
+    // that the CTAs that read the same 16 rows of W are neighbours in launch order and find them in the L2
+    const bool grouped = gridDim.y > 1;
+    const int rank = grouped ? static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x % static_cast<unsigned>(ks));
+    const int64_t r0 = static_cast<int64_t>(grouped ? blockIdx.z : blockIdx.x / static_cast<unsigned>(ks)) * 16;
     const int kbeg = rank * p.kchunk;
     const int kend = min(p.K, kbeg + p.kchunk);
     const int warp = static_cast<int>(threadIdx.x) >> 5, lane = static_cast<int>(threadIdx.x) & 31;

@@ -44,7 +44,7 @@ EXPORTED = ["sg_gemm", "sg_batched_gemm", "sg_grouped_gemm_workspace_size", "sg_
 OPTIONS = {"epi_warps": 0, "tail_split": 1, "tail_ksplit": 2, "band_m": 3, "general_kernel": 4, "no_pdl": 5, "no_short_a": 6,
            "no_gemv": 7, "gemv_no_mma": 8, "gemv_no_wide": 9, "gemv_rows": 10, "wait_limit_ns": 11, "l2_warm_kblocks": 12, "transpose_plain": 13, "early_donors": 14,
            "two_pass_split_k": 15, "split_k_reduce_warps": 16,
-           "gemv_max_vectors": 17, "gemv_small_log2": 18}
+           "gemv_max_vectors": 17, "gemv_small_log2": 18, "gemv_vector_blocks": 19}
 
 
 class SolgemmError(RuntimeError):

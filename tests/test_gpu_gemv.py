@@ -162,11 +162,15 @@ def test_other_forms_still_go_through_the_tiles():
     ref, absacc = orc.gemm(A, B33)
     parity.assert_matches(out[:, :33], ref, absacc, "N = 33")
     # nine vectors against a matrix too large for the many-vector form of the kernel (more than 48 MB)
+    sg.set_option("gemv_small_log2", -1)
     Wbig = torch.randn(6200, 4096, generator=g).to(torch.bfloat16)
     X9 = torch.randn(9, 4096, generator=g).to(torch.bfloat16)
     D9 = sg.gemm(X9.to(DEV), Wbig.to(DEV))
     assert not _took_vector_path()
     parity.assert_matches(D9[:, :64], *[t[:, :64] for t in orc.gemm(X9, Wbig[:64])], "nine vectors, large matrix")
+    # ... or with more groups of eight than are resident at once (512 row blocks x 3 groups)
+    sg.gemm(torch.zeros(20, 2048, dtype=torch.bfloat16, device=DEV), torch.zeros(8192, 2048, dtype=torch.bfloat16, device=DEV))
+    assert not _took_vector_path()
     # a K x 2 row-major B is not a pair of contiguous vectors
     Brow = torch.randn(64, 8, generator=g).to(torch.bfloat16)
     sg.gemm(A.to(DEV), Brow.to(DEV)[:, :2], layout_b="row", out=out[:, :2])
@@ -240,13 +244,18 @@ def test_several_vectors_k_not_a_multiple_of_a_warp_step(R, K, nvec):
 @pytest.mark.parametrize("nvec", [9, 12, 16, 17, 24, 31, 32])
 @pytest.mark.parametrize("R,K", [(512, 1024), (130, 4104), (37, 264), (2048, 2048), (5, 72)])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
-def test_nine_to_32_vectors_in_one_pass(R, K, nvec, dtype):
-    # blocks of eight vectors share one pass over the matrix (two blocks up to 16 vectors, four up to 32)
+@pytest.mark.parametrize("form", ["groups of eight", "blocks in one CTA"])
+def test_nine_to_32_vectors(R, K, nvec, dtype, form):
+    # the library's own choice: groups of eight vectors along the grid (CTAs that share rows of the matrix are neighbours);
+    # with the vector limit pinned to 32: blocks of eight vectors inside one CTA (two up to 16 vectors, four up to 32)
     g = torch.Generator().manual_seed(R + K + nvec)
     W = (torch.randn(R, K, generator=g) / 8).to(dtype)
     X = (torch.randn(nvec, K, generator=g) / 8).to(dtype)
     fewer = min(nvec, R)                      # the operand with fewer rows supplies the vectors
-    blocks = 1 if fewer <= 8 else (2 if fewer <= 16 else 4)
+    blocks = 1
+    if form == "blocks in one CTA":
+        sg.set_option("gemv_max_vectors", 32)
+        blocks = 1 if fewer <= 8 else (2 if fewer <= 16 else 4)
     # vectors on the left (a decode batch): D [nvec, R], bias per matrix row, residual
     Ct = torch.randn(nvec, R, generator=g).to(dtype)
     biasR = torch.randn(R, generator=g).to(dtype)
