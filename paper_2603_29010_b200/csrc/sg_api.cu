@@ -1027,9 +1027,14 @@ sg_status_t try_gemv(const sg_gemm_desc_t* desc, const void* A, const void* B, c
             const int per_sm[3] = {4, 3, 2};
             // (groups of 32 only with the 32-byte row pieces: with 16-byte pieces they measured slower than the tiles)
             const bool wide_ok = desc->K % 16 == 0 && (desc->lda * 2) % 32 == 0 && (desc->ldb * 2) % 32 == 0;
-            for (int b = 0; b < 3 && !group_blocks; ++b) {
-                if (!is_small && b > 0) break;           // a few rows against a matrix: groups of eight or the tiles
-                if (b == 2 && !wide_ok && !small_forced) break;
+            // Which group size, where several fit: groups of eight keep the most loads in flight (long K loops, few
+            // CTAs); with more than two CTAs per SM of them and a short K loop larger groups are quicker -- fewer CTAs,
+            // less re-reading (256^3: 2.72 us in groups of 32, 2.90 in groups of 8; 256 x 256 x 2048: 5.8 against 5.1).
+            const bool small_first = row_blocks * ((few + 7) / 8) <= 2 * static_cast<int64_t>(ds->sm_count) || desc->K > 1024;
+            for (int i = 0; i < 3 && !group_blocks; ++i) {
+                const int b = small_first ? i : 2 - i;
+                if (!is_small && b > 0) continue;        // a few rows against a matrix: groups of eight or the tiles
+                if (b == 2 && !wide_ok && !small_forced) continue;
                 const int64_t ctas = row_blocks * ((few + (8 << b) - 1) / (8 << b));
                 if (ctas <= per_sm[b] * static_cast<int64_t>(ds->sm_count) || (small_forced && is_small && b == 2)) group_blocks = 1 << b;
             }
