@@ -441,8 +441,11 @@ typedef enum {
                                    into ranges summed by a second kernel, k >= 2 = at most k ranges (default: as many as
                                    there are SMs to go round) */
     SG_OPT_SPLIT_K_REDUCE_WARPS = 16, /* second pass of a two-pass K split: 1, 2, 4 or 8 warps share the parts of a column slice */
-    SG_OPT_GEMV_MAX_VECTORS = 17, /* most vectors (4..32) the matrix-vector kernels take before the tiles do; default 32 */
-    SG_OPT_GEMV_SMALL_LOG2 = 18,  /* products of at most 2^value multiply-adds (16-bit operands) run on the warp-level MMA kernel; 0 = none */
+    SG_OPT_GEMV_MAX_VECTORS = 17, /* > 0: the matrix-vector kernels take at most this many vectors (4..32), all of them in one
+                                   CTA, and the grouped form below is off (default: 8 in one CTA, more in groups) */
+    SG_OPT_GEMV_SMALL_LOG2 = 18,  /* products of at most 2^value multiply-adds (16-bit operands) run on the warp-level MMA
+                                   kernel in groups of vectors, whether or not their CTAs are all resident; 0 = none
+                                   (default: 160 M multiply-adds, resident CTAs only) */
     SG_OPT_GEMV_VECTOR_BLOCKS = 19, /* blocks of eight vectors a CTA of the warp-level MMA kernel takes: 1, 2 or 4 */
     SG_OPT_COUNT_ = 20
 } sg_option_t;
